@@ -1,0 +1,447 @@
+#!/usr/bin/env python
+"""Benchmark of the quantize -> integer aggregate -> reconstruct hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl reference]
+
+One step = one pass of the whole path (agree scale, [select scale index], encode, fused
+aggregate+decode) over one batch of synthetic gradients of M workers.  The metric is gradient
+GB/s: bytes of gradient input (M * d * sizeof(element)) per second of the whole step.
+The path does not shard: with N GPUs every rank runs an independent replica ("replicas only")
+and the value is the sum over ranks; timing is the max over ranks of device-event time.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead (test
+infrastructure, executed here only as the reported baseline).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+from paper_2109_12497_b200 import workloads as wl  # noqa: E402
+
+METRIC = "gradient GB/s through encode+aggregate+decode; % of B200 HBM roofline"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only without MEASURED_PEAKS.json
+
+# DRAM traffic per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum) from
+# the ncu captures summarised under profiles/, keyed by workload; None = not captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def hbm_peak():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            return float(json.loads(p.read_text())["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# ---------------------------------------------------------------------------------------------
+# algorithmic bytes per launch of each kernel (what the method must move)
+# ---------------------------------------------------------------------------------------------
+
+def algorithmic_bytes(w: wl.Workload) -> dict:
+    e = 4 if w.dtype == wl.F32 else 2
+    lev = 1.0 if w.fmt == "i8" else 0.5
+    ib = w.idx_bits / 8.0
+    M, d = w.M, w.d
+    b = {"agree_scale": e * M * d}
+    if w.quantizer == "multi":
+        b["select_scale"] = e * M * d + ib * d
+        b["encode"] = (e + lev + ib) * M * d          # every worker re-reads the shared index
+    else:
+        b["encode"] = (e + lev) * M * d
+    b["aggregate_decode"] = lev * M * d + ib * d + 4 * d
+    return b
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self) -> dict | None:
+        if self.proc is None:
+            return None
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 6:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return None
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------------------
+# GPU arm
+# ---------------------------------------------------------------------------------------------
+
+STAGES_SINGLE = ["agree_scale", "encode", "aggregate_decode"]
+STAGES_MULTI = ["agree_scale", "select_scale", "encode", "aggregate_decode"]
+
+
+def run_stages(q, g, seed, events=None):
+    """One step; events (if given) is a list of len(stages)+1 CUDA events recorded around the stages."""
+    import torch
+    st = torch.cuda.current_stream()
+    k = 0
+    if events: events[k].record(st)
+    q.agree_scale(g); k += 1
+    if events: events[k].record(st)
+    if q.multi:
+        q.select_scale(g); k += 1
+        if events: events[k].record(st)
+    q.encode(g, seed); k += 1
+    if events: events[k].record(st)
+    q.aggregate_decode(); k += 1
+    if events: events[k].record(st)
+
+
+def time_device_resident(q, g, w, steps, warmup, barrier):
+    """(ms per step, {stage: mean ms}) with inputs resident in HBM, timed with CUDA events."""
+    import torch
+    stages = STAGES_MULTI if q.multi else STAGES_SINGLE
+    for _ in range(warmup):
+        run_stages(q, g, w.seed)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(stages) + 1)] for _ in range(steps)]
+    torch.cuda.synchronize(); barrier()
+    for k in range(steps):
+        run_stages(q, g, w.seed + k, evs[k])
+    torch.cuda.synchronize(); barrier()
+    total_ms = evs[0][0].elapsed_time(evs[-1][-1])
+    per_stage = {s: statistics.fmean(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(steps))
+                 for i, s in enumerate(stages)}
+    return total_ms / steps, per_stage
+
+
+def time_end_to_end(q, g_host, out_host, g_dev, w, steps, warmup, barrier):
+    """ms per step with the gradients starting in pinned host memory and the result read back."""
+    import torch
+    st = torch.cuda.current_stream()
+
+    def one(k):
+        g_dev.copy_(g_host, non_blocking=True)
+        out = q.step(g_dev, w.seed + k)
+        out_host.copy_(out, non_blocking=True)
+
+    for k in range(min(warmup, 3)):
+        one(k)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(); barrier()
+    e0.record(st)
+    for k in range(steps):
+        one(k)
+    e1.record(st)
+    torch.cuda.synchronize(); barrier()
+    return e0.elapsed_time(e1) / steps
+
+
+def l2_flush_buffer():
+    import torch
+    return torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+
+def resolve_workload(name, d=None, rng_bits=None):
+    """The named workload, optionally at a smaller d (same recipe; used for ncu captures, which
+    must stay small) or with the other random-draw width."""
+    w = wl.WORKLOADS[name]
+    if d is not None and d != w.d:
+        w = wl.scaled(name, d)
+        if wl.WORKLOADS[name].segments == "buckets25MiB":
+            import dataclasses
+            w = dataclasses.replace(w, bucket_elems=wl.WORKLOADS[name].bucket_elems)
+    if rng_bits is not None:
+        import dataclasses
+        w = dataclasses.replace(w, rng_bits=rng_bits)
+    return w
+
+
+def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=False):
+    """Times one workload on the current device.  Returns a dict of raw numbers."""
+    import torch
+    from paper_2109_12497_b200.pipeline import from_workload
+    np_dtype = np.float32 if w.dtype == wl.F32 else np.uint16
+    if want_e2e:
+        g_host = torch.empty((w.M, w.stride), dtype=torch.float32 if w.dtype == wl.F32 else torch.int16,
+                             pin_memory=True)
+        wl.generate(w, out=g_host.numpy().view(np_dtype), threads=threads)
+    else:
+        g_host = torch.from_numpy(wl.generate(w, threads=threads).view(np.float32 if w.dtype == wl.F32 else np.int16))
+    if w.dtype == wl.BF16:
+        g_host = g_host.view(torch.bfloat16)
+    q = from_workload(w)
+    g_dev = torch.empty(g_host.shape, dtype=g_host.dtype, device="cuda")
+    for m in range(w.M):                       # row by row keeps the staging small for pageable memory
+        g_dev[m].copy_(g_host[m])
+    torch.cuda.synchronize()
+
+    res = {"workload": w, "q": q}
+    if flush_between:
+        # working set smaller than L2: time each step alone after overwriting L2
+        flush = l2_flush_buffer()
+        for _ in range(warmup):
+            run_stages(q, g_dev, w.seed)
+        stages = STAGES_MULTI if q.multi else STAGES_SINGLE
+        tot, per = [], {s: [] for s in stages}
+        for k in range(steps):
+            flush.fill_(k & 0xFF)
+            evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(stages) + 1)]
+            run_stages(q, g_dev, w.seed + k, evs)
+            torch.cuda.synchronize()
+            tot.append(evs[0].elapsed_time(evs[-1]))
+            for i, s in enumerate(stages):
+                per[s].append(evs[i].elapsed_time(evs[i + 1]))
+        res["ms_cold"] = statistics.fmean(tot)
+        res["stages_cold_ms"] = {s: statistics.fmean(v) for s, v in per.items()}
+        del flush
+    res["ms"], res["stages_ms"] = time_device_resident(q, g_dev, w, steps, warmup, barrier)
+    res["h2d"], res["d2h"], res["e2e_ms"] = 0, 0, None
+    if want_e2e:
+        out_host = torch.empty(w.d, dtype=torch.float32, pin_memory=True)
+        res["e2e_ms"] = time_end_to_end(q, g_host, out_host, g_dev, w, steps, warmup, barrier)
+        res["h2d"] = g_host.numel() * g_host.element_size()
+        res["d2h"] = out_host.numel() * 4
+    res["status"] = q.status_bits()
+    return res
+
+
+def summarize(res, peak_gbs):
+    w = res["workload"]
+    ab = algorithmic_bytes(w)
+    out = {"gradient_GBps": w.in_bytes / res["ms"] / 1e6, "ms_per_step": res["ms"], "kernels": {}}
+    for s, ms in res["stages_ms"].items():
+        gbs = ab[s] / ms / 1e6
+        out["kernels"][s] = {"ms": round(ms, 5), "algorithmic_MB": round(ab[s] / 1e6, 2),
+                             "GBps": round(gbs, 1), "frac_of_hbm_peak": round(gbs / peak_gbs, 4)}
+    if "ms_cold" in res:
+        out["cold_l2"] = {"ms_per_step": res["ms_cold"], "gradient_GBps": w.in_bytes / res["ms_cold"] / 1e6,
+                          "kernels_ms": {s: round(v, 5) for s, v in res["stages_cold_ms"].items()}}
+    return out
+
+
+def cpu_baseline(name, threads, max_coords):
+    """The oracle, as it stands, on the host cores, over the first `max_coords` coordinates of
+    the workload (all M workers, the segments that fall in that window)."""
+    from oracle import uq_oracle as o
+    w = wl.WORKLOADS[name]
+    n = min(w.d, max_coords)
+    seg_full = wl.segment_offsets(w)
+    seg = np.unique(np.concatenate([seg_full[seg_full < n], [n]])).astype(np.int64)
+    sub = wl.scaled(name, n) if n < w.d else w
+    if n < w.d:                                 # same recipe at the window's size
+        import dataclasses
+        sub = dataclasses.replace(w, d=n, segments="one")
+    g = wl.generate(sub, threads=threads)[:, :n]
+    o.set_threads(threads)
+    norm = o.NORM_L2 if w.norm == wl.NORM_L2 else o.NORM_LINF
+    t0 = time.perf_counter()
+    W = o.agree_scale(g, seg, norm)
+    if w.quantizer == "multi":
+        idx = o.select_scale_multi(g, W, w.scales, seg_off=seg)
+        lev = o.encode_multi(g, W, w.scales, idx, w.seed, w.rng_bits, seg_off=seg)
+        S = o.aggregate(lev)
+        o.decode(S, w.M, W, scales=w.scales, idx=idx, seg_off=seg)
+    else:
+        lev = o.encode_single(g, W, w.s, w.seed, w.rng_bits, seg_off=seg)
+        S = o.aggregate(lev)
+        o.decode(S, w.M, W, s=w.s, seg_off=seg)
+    dt = time.perf_counter() - t0
+    in_bytes = w.M * n * (4 if w.dtype == wl.F32 else 2)
+    sample = "full workload" if n == w.d else f"first {n} of {w.d} coordinates of all {w.M} workers"
+    return {"value": in_bytes / dt / 1e9, "unit": UNIT, "cores": o.get_threads(), "kind": "oracle",
+            "sample": sample, "seconds": round(dt, 3)}
+
+
+def gpu_main(args):
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (the quantizer has no CPU path; use --impl reference "
+                         "for the oracle baseline)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    threads = max(1, min(16, (os.cpu_count() or 8) // max(1, world)))
+    peak, peak_kind = hbm_peak()
+    name = args.workload
+    w = resolve_workload(name, args.d, args.rng_bits)
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    res = bench_workload(w, args.steps, args.warmup, barrier, threads, want_e2e=not args.no_e2e)
+    clocks = sampler.stop()
+
+    ms, e2e_ms = res["ms"], res["e2e_ms"] or float("nan")
+    if world > 1:
+        t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = float(t[0]), float(t[1])
+    summ = summarize(res, peak)
+    q = res["q"]
+    dom = max(summ["kernels"], key=lambda s: summ["kernels"][s]["ms"])
+    ab = algorithmic_bytes(w)
+    dom_gbs = ab[dom] / res["stages_ms"][dom] / 1e6
+    line = {
+        "metric": METRIC, "value": round(world * w.in_bytes / ms / 1e6, 2), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms, 5),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32" if w.dtype == wl.F32 else "bf16",
+        "data": "synthetic",
+        "config": {
+            "workload": f"{name}: {w.quantizer}-scale, M={w.M}, d={w.d} {w.dtype}, {len(wl.segment_offsets(w)) - 1} "
+                        f"segments, s={w.s}, scales={list(w.scales)}, levels {w.fmt}, idx_bits={w.idx_bits}, "
+                        f"norm={w.norm}, rng_bits={w.rng_bits}",
+            "parallelism": "replicas only" if world > 1 else "single GPU, M workers emulated as resident buffers",
+            "l2": f"inputs {w.in_bytes / 1e6:.0f} MB per step > 126 MB L2, no flush between steps",
+            "status_word": res["status"],
+        },
+        "e2e": None if args.no_e2e else {
+            "value": round(world * w.in_bytes / e2e_ms / 1e6, 2), "unit": UNIT, "ms_per_step": round(e2e_ms, 4),
+            "h2d_bytes_per_step": res["h2d"], "d2h_bytes_per_step": res["d2h"]},
+        "gpu_launches": q.kernels_per_step() * args.steps,
+        "clocks": clocks,
+        "roofline": {
+            "bound": "hbm", "kernel": dom, "achieved": round(dom_gbs, 1), "peak": peak, "unit": "GB/s",
+            "frac": round(dom_gbs / peak, 4), "peak_kind": f"of {peak_kind}",
+            "algorithmic_bytes_per_launch": int(ab[dom]),
+            "avg_launch_ms": round(res["stages_ms"][dom], 5),
+            "traffic": NCU_TRAFFIC_BYTES.get(name),
+        },
+        "kernels": summ["kernels"],
+    }
+    if rank == 0 and world == 1:
+        # the other four workloads (parity-test cases; reported for context, a few steps each)
+        if not args.no_extra and args.d is None:
+            extra = {}
+            for other in ("c1", "c3", "c4", "c5"):
+                del res, q
+                torch.cuda.empty_cache()
+                small = wl.WORKLOADS[other].in_bytes < (126 << 20)
+                res = bench_workload(wl.WORKLOADS[other], max(3, min(args.steps, 10)), 3, lambda: None, threads,
+                                     want_e2e=False, flush_between=small)
+                q = res["q"]
+                extra[other] = summarize(res, peak)
+                extra[other]["status_word"] = res["status"]
+            line["other_workloads"] = extra
+        if not args.no_cpu:
+            line["cpu_baseline"] = cpu_baseline(name, max(1, os.cpu_count() or 1), args.cpu_coords)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle
+# ---------------------------------------------------------------------------------------------
+
+def reference_main(args):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    w = wl.WORKLOADS[args.workload]
+    threads = max(1, os.cpu_count() or 1)
+    n = min(w.d, args.ref_coords)
+    vals = []
+    for k in range(args.warmup + args.steps):
+        r = cpu_baseline(args.workload, threads, n)
+        if k >= args.warmup:
+            vals.append(r)
+    secs = statistics.fmean(v["seconds"] for v in vals)
+    in_bytes = w.M * n * (4 if w.dtype == wl.F32 else 2)
+    value = in_bytes / secs / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(secs * 1e3, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32" if w.dtype == wl.F32 else "bf16", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: CPU oracle on {vals[-1]['sample']}"},
+        "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "cores": vals[-1]["cores"], "kind": "oracle",
+                         "sample": vals[-1]["sample"]},
+        "e2e": {"value": round(value, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--no-extra", action="store_true", help="skip the four context workloads")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end timing")
+    ap.add_argument("--d", type=int, default=None, help="run the workload's recipe at this smaller d (profiling)")
+    ap.add_argument("--rng-bits", type=int, default=None, choices=[16, 32], help="override the draw width")
+    ap.add_argument("--cpu-coords", type=int, default=25_557_032,
+                    help="coordinates of the workload the CPU baseline covers")
+    ap.add_argument("--ref-coords", type=int, default=1 << 20,
+                    help="coordinates per step of the reference (oracle) arm")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        reference_main(args)
+    else:
+        gpu_main(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,190 @@
+/*
+ * uq — all-reduce-compatible unbiased gradient quantizers on one B200 (sm_100a).
+ *
+ * C ABI of the data-parallel hot path of "Unbiased Single-scale and Multi-scale Quantizers for
+ * Distributed Optimization": shared max-norm scale -> [per-coordinate scale index] ->
+ * stochastic quantization to small integers -> integer sum over workers -> reconstruction of
+ * the average gradient (Algorithm 1, QSGDMaxNorm; Algorithm 2, QSGDMaxNormMultiScale).
+ *
+ * The M workers are M resident device buffers; the paper's three all-reduces (max of the norm,
+ * min of the scale index, sum of the levels) are on-device reductions over those buffers.
+ *
+ * Common rules
+ *   - Every data pointer is a DEVICE pointer owned by the caller unless marked "host".
+ *     The library allocates no device memory and keeps no state between calls.
+ *   - Every call only enqueues kernels on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     default stream) and returns at once; it never synchronizes.
+ *   - Return value: UQ_OK or a UQ_ERR_* code.  Argument errors are found on the host before
+ *     anything is launched.  Data-dependent problems (non-finite input, a malformed segment
+ *     table, s/W overflowing) never trap: the kernels OR a UQ_STATUS_* bit into the caller's
+ *     device word `status` (may be NULL to ignore) and still write in-bounds values.
+ *   - Layout.  Worker m's gradient is g + m*worker_stride elements, coordinates 0..d-1.
+ *     worker_stride is a multiple of 32 and >= d; the padding d..worker_stride-1 of each row
+ *     must be readable (its values are ignored).  Level rows use the same stride in coordinates
+ *     (int8: worker_stride bytes per row; 4-bit: worker_stride/2 bytes); the library may write
+ *     zeros into a level row's padding.  g and lev must be 16-byte aligned.
+ *   - Segments.  The paper's vector v in R^n is a segment: coordinates seg_off[j]..seg_off[j+1]-1
+ *     share the scale W[j].  seg_off is a device array of nseg+1 non-decreasing offsets with
+ *     seg_off[0] = 0 and seg_off[nseg] = d; seg_off = NULL (with nseg = 1) means one segment.
+ *   - Arithmetic.  Integer results (levels, indices, sums) are defined bit-exactly by the
+ *     binary32 operation order stated per call; no fused multiply-add is used where a
+ *     floating-point value decides an integer.
+ *   - Random draws (the paper's "independent random variables xi_i"): Philox4x32-10 with
+ *     key = (seed low, seed high) and counter = (block low, block high, worker m, 0).
+ *       rng_bits = 32: block = i/4, coordinate i takes word i%4, h = word >> 9 (23 bits)
+ *       rng_bits = 16: block = i/8, word (i%8)/2, even i the low half, h = that half (16 bits)
+ *     With b the width of h, a coordinate rounds up iff h < rint(p * 2^b) (ties to even), i.e.
+ *     with the multiple of 2^-b nearest to the paper's probability p.  i is the coordinate's
+ *     index in the worker's whole d-vector.
+ */
+#ifndef UQ_H
+#define UQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    UQ_OK = 0,
+    UQ_ERR_BAD_ARG = 1,     /* null/unaligned pointer, size or parameter out of range */
+    UQ_ERR_CUDA = 2,        /* a launch failed; uq_last_cuda_error() has the CUDA code */
+    UQ_ERR_UNSUPPORTED = 3, /* a combination this build does not implement */
+    UQ_ERR_WORKSPACE = 4    /* workspace too small or missing */
+};
+
+enum { UQ_F32 = 0, UQ_BF16 = 1 };              /* gradient element type */
+enum { UQ_NORM_LINF = 0, UQ_NORM_L2 = 2 };     /* which norm defines the shared scale */
+enum { UQ_FMT_I8 = 0, UQ_FMT_I4X2 = 1 };       /* level wire format */
+enum { UQ_SRC_LEVELS = 0, UQ_SRC_SUMS = 1 };   /* what uq_decode reads */
+
+/* bits OR-ed into the device status word */
+enum {
+    UQ_STATUS_NONFINITE = 1,      /* a NaN/Inf input or a non-finite scale */
+    UQ_STATUS_BAD_SEGMENTS = 2,   /* seg_off not non-decreasing from 0 to d */
+    UQ_STATUS_SCALE_OVERFLOW = 4  /* s / W is not finite (W subnormal-small) */
+};
+
+#define UQ_MAX_WORKERS 64
+#define UQ_MAX_SCALES 16
+
+typedef struct uq_layout {
+    int64_t d;              /* coordinates per worker, >= 0 */
+    int64_t worker_stride;  /* coordinates between consecutive workers' rows; multiple of 32, >= d */
+    const int64_t *seg_off; /* device, nseg+1 entries, or NULL for a single segment */
+    int32_t M;              /* workers, 1..UQ_MAX_WORKERS */
+    int32_t nseg;           /* segments, >= 1 */
+    int32_t dtype;          /* UQ_F32 or UQ_BF16 (bf16 = upper half of a binary32) */
+    int32_t reserved;       /* must be 0 */
+} uq_layout;
+
+/* Library version (major*10000 + minor*100 + patch). */
+int uq_version(void);
+
+/* CUDA error code of the most recent failed launch on the calling thread (0 if none). */
+int uq_last_cuda_error(void);
+
+/* Static description of a UQ_ERR_* code. */
+const char *uq_error_string(int code);
+
+/* Bytes of device scratch uq_agree_scale needs for this layout (0 on a bad layout). */
+size_t uq_workspace_bytes(const uq_layout *layout);
+
+/* Bytes of a packed scale-index stream for this layout: worker_stride * idx_bits / 8. */
+size_t uq_index_bytes(const uq_layout *layout, int idx_bits);
+
+/*
+ * Shared scale — Algorithm 1 / Algorithm 2, line "MaxAllReduce Norm":
+ *   W[j] = max over workers m of || g^m restricted to segment j ||.
+ * norm = UQ_NORM_L2 is the paper's definition: every square is formed exactly in binary64,
+ * summed in binary64 in a fixed order that does not depend on the launch, and
+ * W[j] = (float) sqrt(max_m sum).  norm = UQ_NORM_LINF gives max |g^m_i| exactly.
+ * An empty or all-zero segment has W[j] = 0.
+ *   g          in   [M][worker_stride] of layout->dtype
+ *   W          out  [nseg] float
+ *   status     i/o  device word or NULL; NONFINITE if any W[j] is not finite (NaN/Inf input),
+ *                   BAD_SEGMENTS if seg_off is malformed (results then unspecified, in bounds)
+ *   workspace  scratch of at least uq_workspace_bytes(layout) bytes, 8-byte aligned; contents
+ *              need no initialisation and are garbage afterwards
+ * Errors: UQ_ERR_BAD_ARG, UQ_ERR_WORKSPACE, UQ_ERR_CUDA.
+ */
+int uq_agree_scale(const uq_layout *layout, const void *g, int norm, float *W, uint32_t *status,
+                   void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Single-scale quantizer Q_s — Section "QSGDMaxNorm Quantization" (Eq. Q_s, definition of
+ * xi_i), Algorithm 1 line "Quantize gradient", for all M workers:
+ *   inv = (float)s / W[j]  (0 if W[j] = 0);  x = min(|v| * inv, (float)s);  l = floor(x);
+ *   p = x - l;  level = l + [h < rint(p * 2^b)];  zeta = v < 0 ? -level : level.
+ *   lev  out  fmt I8:   int8 [M][worker_stride]               (1 <= s <= 127)
+ *             fmt I4X2: two's-complement nibbles, even coordinate in the low nibble,
+ *                       [M][worker_stride/2] bytes            (1 <= s <= 7)
+ *   W    in   [nseg], e.g. from uq_agree_scale; any W[j] >= max|v| keeps |zeta| <= s, and
+ *             the clamp keeps it so for any W.
+ * Errors: UQ_ERR_BAD_ARG, UQ_ERR_CUDA.
+ */
+int uq_encode_single(const uq_layout *layout, const void *g, const float *W, int s, uint64_t seed,
+                     int rng_bits, int fmt, void *lev, uint32_t *status, void *stream);
+
+/*
+ * Per-coordinate scale index with scale sharing — Section "QSGDMaxNormMultiScale
+ * Quantization" (the inequality that defines s*_i, and "scale sharing"), Algorithm 2 lines
+ * "Compute coordinate scales" and "Scale sharing":
+ *   worker's own index  k^m_i = largest k with |g^m_i| * ((float)scales[k] / W[j]) <= (float)scales[0]
+ *                       (k = 0 if none; a zero coordinate or W[j] = 0 gives N-1)
+ *   shared index        k_i = min over workers of k^m_i.
+ *   scales    host  N ascending integers >= 1, N <= UQ_MAX_SCALES; scales[0] is the smallest scale
+ *   idx_bits  2 (N <= 4), 4 (N <= 16) or 8
+ *   idx       out   packed little-endian within each byte (coordinate i at bit (i*idx_bits)%8
+ *                   of byte (i*idx_bits)/8), uq_index_bytes(layout, idx_bits) bytes; bits
+ *                   belonging to coordinates >= d are written as 0
+ * Errors: UQ_ERR_BAD_ARG, UQ_ERR_CUDA.
+ */
+int uq_select_scale_multi(const uq_layout *layout, const void *g, const float *W,
+                          const int32_t *scales, int N, int idx_bits, uint8_t *idx,
+                          uint32_t *status, void *stream);
+
+/*
+ * Multi-scale quantizer Q_{s_} — Section "QSGDMaxNormMultiScale Quantization" (Eq. Q_{s_}),
+ * Algorithm 2 line "Quantize with s*": coordinate i of every worker is quantized as in
+ * uq_encode_single with s replaced by scales[k_i] in inv and the level clamped to scales[0]
+ * (the level fits the bits of the smallest scale).
+ *   idx  in  the shared indices written by uq_select_scale_multi (same idx_bits)
+ *   fmt  I8 needs scales[0] <= 127, I4X2 needs scales[0] <= 7
+ * Errors: UQ_ERR_BAD_ARG, UQ_ERR_CUDA.
+ */
+int uq_encode_multi(const uq_layout *layout, const void *g, const float *W, const int32_t *scales,
+                    int N, const uint8_t *idx, int idx_bits, uint64_t seed, int rng_bits, int fmt,
+                    void *lev, uint32_t *status, void *stream);
+
+/*
+ * Integer aggregation — Algorithm 1 / 2 line "AllReduce gradients" without the 1/M:
+ *   S[i] = sum over workers of zeta^m_i, in int32.
+ *   lev  in   level rows as written by the encoders (layout->dtype is ignored)
+ *   S    out  [d] int32, 4-byte aligned
+ * Errors: UQ_ERR_BAD_ARG, UQ_ERR_CUDA.
+ */
+int uq_aggregate(const uq_layout *layout, const void *lev, int fmt, int32_t *S, void *stream);
+
+/*
+ * Reconstruction of the average gradient — Eq. R_s after Algorithm 1 and Eq. R_{s_} after
+ * Algorithm 2, applied to the averaged levels:
+ *   c = W[j] / ((float)s_i * (float)M);  out[i] = (float)S[i] * c,
+ * with s_i = s (scales = NULL) or scales[k_i] (scales, N, idx, idx_bits as in the encoder).
+ *   src_kind = UQ_SRC_LEVELS: src is the level rows; the sum over workers and the
+ *              reconstruction run fused in one kernel (the sums stay in registers);
+ *              S_opt, if not NULL, also receives the int32 sums [d].
+ *   src_kind = UQ_SRC_SUMS:   src is int32 S[d] (fmt and S_opt are ignored).
+ *   out  [d] float, 4-byte aligned (no padding is required or written)
+ * Errors: UQ_ERR_BAD_ARG, UQ_ERR_CUDA.
+ */
+int uq_decode(const uq_layout *layout, const void *src, int src_kind, int fmt, const float *W, int s,
+              const int32_t *scales, int N, const uint8_t *idx, int idx_bits, float *out,
+              int32_t *S_opt, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* UQ_H */

@@ -197,6 +197,8 @@ def pack_levels_i4(lev: np.ndarray) -> np.ndarray:
     """Two 4-bit two's-complement levels per byte (row stride must be even)."""
     assert lev.dtype == np.int8
     M, d, stride = _check_g(lev)
+    if M == 1:
+        stride += stride & 1                 # a single row has no stride to respect
     assert stride % 2 == 0, "the row stride must be even"
     packed = np.zeros((M, stride // 2), dtype=np.uint8)
     lib().uqo_pack_levels_i4(_p(lev), M, C.c_int64(d), C.c_int64(stride), _p(packed))

@@ -1,1 +1,11 @@
-"""placeholder"""
+"""uq — all-reduce-compatible unbiased gradient quantizers, hand-written CUDA for B200 (sm_100a).
+
+``binding`` exposes the C ABI of ``include/uq.h`` one to one; ``workloads`` makes the seeded
+synthetic gradients; ``build`` compiles the library in-tree with nvcc.
+"""
+from .binding import (  # noqa: F401
+    Layout, UqError, lib, uq_version,
+    uq_agree_scale, uq_encode_single, uq_select_scale_multi, uq_encode_multi, uq_aggregate, uq_decode,
+    UQ_F32, UQ_BF16, UQ_NORM_LINF, UQ_NORM_L2, UQ_FMT_I8, UQ_FMT_I4X2, UQ_SRC_LEVELS, UQ_SRC_SUMS,
+    UQ_STATUS_NONFINITE, UQ_STATUS_BAD_SEGMENTS, UQ_STATUS_SCALE_OVERFLOW,
+)

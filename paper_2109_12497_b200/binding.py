@@ -1,0 +1,222 @@
+"""Thin ctypes binding of the C ABI in ``include/uq.h``.
+
+Argument marshalling only: every function takes torch CUDA tensors (device memory and the
+current stream are torch's), checks shapes and dtypes, and calls the C entry point of the same
+name.  All arithmetic runs in the CUDA kernels of ``libuq_b200.so``; there is no CPU path, and
+a missing or unloadable library is an error.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from pathlib import Path
+from typing import Optional, Sequence
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libuq_b200.so"
+
+UQ_OK, UQ_ERR_BAD_ARG, UQ_ERR_CUDA, UQ_ERR_UNSUPPORTED, UQ_ERR_WORKSPACE = range(5)
+UQ_F32, UQ_BF16 = 0, 1
+UQ_NORM_LINF, UQ_NORM_L2 = 0, 2
+UQ_FMT_I8, UQ_FMT_I4X2 = 0, 1
+UQ_SRC_LEVELS, UQ_SRC_SUMS = 0, 1
+UQ_STATUS_NONFINITE, UQ_STATUS_BAD_SEGMENTS, UQ_STATUS_SCALE_OVERFLOW = 1, 2, 4
+
+EXPORTS = (
+    "uq_version", "uq_last_cuda_error", "uq_error_string", "uq_workspace_bytes", "uq_index_bytes",
+    "uq_agree_scale", "uq_encode_single", "uq_select_scale_multi", "uq_encode_multi",
+    "uq_aggregate", "uq_decode",
+)
+
+
+class uq_layout(C.Structure):
+    _fields_ = [
+        ("d", C.c_int64),
+        ("worker_stride", C.c_int64),
+        ("seg_off", C.c_void_p),
+        ("M", C.c_int32),
+        ("nseg", C.c_int32),
+        ("dtype", C.c_int32),
+        ("reserved", C.c_int32),
+    ]
+
+
+class UqError(RuntimeError):
+    def __init__(self, fn: str, code: int):
+        msg = lib().uq_error_string(code).decode()
+        if code == UQ_ERR_CUDA:
+            msg += f" [cuda error {lib().uq_last_cuda_error()}]"
+        super().__init__(f"{fn}: {msg} (code {code})")
+        self.code = code
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def lib() -> C.CDLL:
+    """The loaded CUDA library; raises if it has not been built (there is no fallback)."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2109_12497_b200.build` "
+                "(the quantizer has no CPU fallback)")
+        L = C.CDLL(str(LIB_PATH))
+        P, I, U64, SZ = C.c_void_p, C.c_int, C.c_uint64, C.c_size_t
+        LP = C.POINTER(uq_layout)
+        L.uq_version.restype = I
+        L.uq_last_cuda_error.restype = I
+        L.uq_error_string.restype = C.c_char_p
+        L.uq_error_string.argtypes = [I]
+        L.uq_workspace_bytes.restype = SZ
+        L.uq_workspace_bytes.argtypes = [LP]
+        L.uq_index_bytes.restype = SZ
+        L.uq_index_bytes.argtypes = [LP, I]
+        L.uq_agree_scale.argtypes = [LP, P, I, P, P, P, SZ, P]
+        L.uq_encode_single.argtypes = [LP, P, P, I, U64, I, I, P, P, P]
+        L.uq_select_scale_multi.argtypes = [LP, P, P, P, I, I, P, P, P]
+        L.uq_encode_multi.argtypes = [LP, P, P, P, I, P, I, U64, I, I, P, P, P]
+        L.uq_aggregate.argtypes = [LP, P, I, P, P]
+        L.uq_decode.argtypes = [LP, P, I, I, P, I, P, I, P, I, P, P, P]
+        for name in EXPORTS[5:]:
+            getattr(L, name).restype = I
+        _lib = L
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("uq: tensors must live on a CUDA device")
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(fn: str, code: int) -> None:
+    if code != UQ_OK:
+        raise UqError(fn, code)
+
+
+def _scales(scales: Sequence[int]):
+    arr = (C.c_int32 * len(scales))(*[int(s) for s in scales])
+    return arr, len(scales)
+
+
+class Layout:
+    """Shape of the M workers' gradient buffers: d coordinates per worker in rows of
+    ``worker_stride`` coordinates, cut into segments that each share one scale."""
+
+    def __init__(self, M: int, d: int, worker_stride: int, dtype: torch.dtype,
+                 seg_off: Optional[torch.Tensor] = None):
+        if dtype not in (torch.float32, torch.bfloat16):
+            raise ValueError("uq: gradients are float32 or bfloat16")
+        if seg_off is not None:
+            if seg_off.dtype != torch.int64 or not seg_off.is_cuda or seg_off.dim() != 1:
+                raise ValueError("uq: seg_off is a 1-D int64 CUDA tensor")
+            seg_off = seg_off.contiguous()
+        self.M, self.d, self.worker_stride, self.dtype, self.seg_off = M, d, worker_stride, dtype, seg_off
+        self.nseg = 1 if seg_off is None else seg_off.numel() - 1
+        self.c = uq_layout(d, worker_stride, _ptr(seg_off), M, self.nseg,
+                           UQ_F32 if dtype == torch.float32 else UQ_BF16, 0)
+
+    def ref(self):
+        return C.byref(self.c)
+
+    def workspace_bytes(self) -> int:
+        return int(lib().uq_workspace_bytes(self.ref()))
+
+    def index_bytes(self, idx_bits: int) -> int:
+        return int(lib().uq_index_bytes(self.ref(), idx_bits))
+
+    def level_row_bytes(self, fmt: int) -> int:
+        return self.worker_stride if fmt == UQ_FMT_I8 else self.worker_stride // 2
+
+    def check_g(self, g: torch.Tensor) -> None:
+        if g.dtype != self.dtype or g.dim() != 2 or g.shape[0] != self.M or g.shape[1] != self.worker_stride \
+                or not g.is_contiguous():
+            raise ValueError(f"uq: g must be a contiguous [{self.M}, {self.worker_stride}] {self.dtype} tensor")
+
+    def check_lev(self, lev: torch.Tensor, fmt: int) -> None:
+        if lev.dtype not in (torch.int8, torch.uint8) or lev.dim() != 2 or lev.shape[0] != self.M \
+                or lev.shape[1] != self.level_row_bytes(fmt) or not lev.is_contiguous():
+            raise ValueError(f"uq: lev must be a contiguous [{self.M}, {self.level_row_bytes(fmt)}] byte tensor")
+
+    def check_vec(self, t: torch.Tensor, dtype: torch.dtype, n: int, what: str) -> None:
+        if t.dtype != dtype or t.dim() != 1 or t.numel() < n or not t.is_contiguous():
+            raise ValueError(f"uq: {what} must be a contiguous 1-D {dtype} tensor with >= {n} elements")
+
+
+def uq_version() -> int:
+    return int(lib().uq_version())
+
+
+def uq_agree_scale(layout: Layout, g: torch.Tensor, norm: int, W: torch.Tensor,
+                   status: Optional[torch.Tensor], workspace: torch.Tensor) -> None:
+    layout.check_g(g)
+    layout.check_vec(W, torch.float32, layout.nseg, "W")
+    _check("uq_agree_scale", lib().uq_agree_scale(
+        layout.ref(), _ptr(g), norm, _ptr(W), _ptr(status), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _stream()))
+
+
+def uq_encode_single(layout: Layout, g: torch.Tensor, W: torch.Tensor, s: int, seed: int, rng_bits: int,
+                     fmt: int, lev: torch.Tensor, status: Optional[torch.Tensor]) -> None:
+    layout.check_g(g)
+    layout.check_lev(lev, fmt)
+    layout.check_vec(W, torch.float32, layout.nseg, "W")
+    _check("uq_encode_single", lib().uq_encode_single(
+        layout.ref(), _ptr(g), _ptr(W), s, seed, rng_bits, fmt, _ptr(lev), _ptr(status), _stream()))
+
+
+def uq_select_scale_multi(layout: Layout, g: torch.Tensor, W: torch.Tensor, scales: Sequence[int],
+                          idx_bits: int, idx: torch.Tensor, status: Optional[torch.Tensor]) -> None:
+    layout.check_g(g)
+    layout.check_vec(W, torch.float32, layout.nseg, "W")
+    layout.check_vec(idx, torch.uint8, layout.index_bytes(idx_bits), "idx")
+    arr, N = _scales(scales)
+    _check("uq_select_scale_multi", lib().uq_select_scale_multi(
+        layout.ref(), _ptr(g), _ptr(W), arr, N, idx_bits, _ptr(idx), _ptr(status), _stream()))
+
+
+def uq_encode_multi(layout: Layout, g: torch.Tensor, W: torch.Tensor, scales: Sequence[int],
+                    idx: torch.Tensor, idx_bits: int, seed: int, rng_bits: int, fmt: int,
+                    lev: torch.Tensor, status: Optional[torch.Tensor]) -> None:
+    layout.check_g(g)
+    layout.check_lev(lev, fmt)
+    layout.check_vec(W, torch.float32, layout.nseg, "W")
+    layout.check_vec(idx, torch.uint8, layout.index_bytes(idx_bits), "idx")
+    arr, N = _scales(scales)
+    _check("uq_encode_multi", lib().uq_encode_multi(
+        layout.ref(), _ptr(g), _ptr(W), arr, N, _ptr(idx), idx_bits, seed, rng_bits, fmt, _ptr(lev),
+        _ptr(status), _stream()))
+
+
+def uq_aggregate(layout: Layout, lev: torch.Tensor, fmt: int, S: torch.Tensor) -> None:
+    layout.check_lev(lev, fmt)
+    layout.check_vec(S, torch.int32, layout.d, "S")
+    _check("uq_aggregate", lib().uq_aggregate(layout.ref(), _ptr(lev), fmt, _ptr(S), _stream()))
+
+
+def uq_decode(layout: Layout, src: torch.Tensor, src_kind: int, fmt: int, W: torch.Tensor, s: int,
+              scales: Optional[Sequence[int]], idx: Optional[torch.Tensor], idx_bits: int,
+              out: torch.Tensor, S_opt: Optional[torch.Tensor] = None) -> None:
+    if src_kind == UQ_SRC_LEVELS:
+        layout.check_lev(src, fmt)
+    else:
+        layout.check_vec(src, torch.int32, layout.d, "src")
+    layout.check_vec(W, torch.float32, layout.nseg, "W")
+    layout.check_vec(out, torch.float32, layout.d, "out")
+    if S_opt is not None:
+        layout.check_vec(S_opt, torch.int32, layout.d, "S_opt")
+    arr, N = (None, 0)
+    if scales is not None:
+        arr, N = _scales(scales)
+        layout.check_vec(idx, torch.uint8, layout.index_bytes(idx_bits), "idx")
+    _check("uq_decode", lib().uq_decode(
+        layout.ref(), _ptr(src), src_kind, fmt, _ptr(W), s, arr, N, _ptr(idx) if scales is not None else None,
+        idx_bits, _ptr(out), _ptr(S_opt), _stream()))

@@ -1,0 +1,175 @@
+// Shared scale W[j] = max_m || g^m on segment j ||   (Algorithm 1, line "MaxAllReduce Norm").
+//
+// Two launches.  (1) norm_partials: the coordinate axis is cut into fixed tiles of kNormTile
+// coordinates; the CTA of (tile t, worker m) reduces every segment that crosses its tile and
+// stores one partial per (tile, segment) pair in slot t + j of worker m's scratch row.  Tiles and
+// segments are both ordered, so t + j is unique for every pair and the row needs
+// ntiles + nseg slots.  (2) norm_finalize: one CTA per segment adds that segment's slots in a
+// fixed order, takes the max over workers, and writes W[j].  The summation tree depends only on
+// (d, seg_off), never on the grid or on timing, so W is reproducible bit for bit.
+#include "uq_device.cuh"
+
+namespace uq {
+
+template <int NORM> struct Acc;
+template <> struct Acc<UQ_NORM_L2> {            // sum of exact binary64 squares
+    double a = 0.0;
+    __device__ __forceinline__ void add(float v) { double x = (double)v; a = __dadd_rn(a, __dmul_rn(x, x)); }
+    __device__ __forceinline__ void merge(double o) { a = __dadd_rn(a, o); }
+    __device__ __forceinline__ double value() const { return a; }
+};
+template <> struct Acc<UQ_NORM_LINF> {          // max of |v| as an integer compare of the bits
+    uint32_t a = 0u;                            // (NaN > Inf > finite, so non-finite input survives)
+    __device__ __forceinline__ void add(float v) { a = max(a, __float_as_uint(v) & 0x7FFFFFFFu); }
+    __device__ __forceinline__ void merge(double o) { a = max(a, (uint32_t)o); }
+    __device__ __forceinline__ double value() const { return (double)a; }
+};
+
+template <int NORM> __device__ __forceinline__ double combine(double x, double y)
+{
+    return NORM == UQ_NORM_L2 ? __dadd_rn(x, y) : fmax(x, y);
+}
+
+template <int NORM> __device__ __forceinline__ double warp_reduce(double x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x = combine<NORM>(x, __shfl_xor_sync(0xFFFFFFFFu, x, o));
+    return x;
+}
+
+template <int DT, int NORM>
+__global__ void __launch_bounds__(kThreads)
+norm_partials_kernel(const void *__restrict__ g, int64_t d, int64_t stride, int nseg,
+                     const int64_t *__restrict__ seg_off, int64_t ntiles, double *__restrict__ part)
+{
+    using E = Elem<DT>;
+    const int64_t tile = blockIdx.x;
+    const int m = blockIdx.y;
+    const int64_t t0 = tile * kNormTile;
+    const int64_t t1 = min(t0 + (int64_t)kNormTile, d);
+    const char *row = (const char *)g + (size_t)m * (size_t)stride * E::BYTES;
+    double *prow = part + (size_t)m * (size_t)(ntiles + nseg);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    const int j0 = find_segment(seg_off, nseg, t0);
+    if (segment_end(seg_off, nseg, j0, d) >= t1) {
+        // the whole tile lies in segment j0: vector loads, one block reduction
+        constexpr int UNITS = kNormTile / (kThreads * E::G);
+        uint4 q[UNITS];
+#pragma unroll
+        for (int u = 0; u < UNITS; ++u) {
+            int64_t i = t0 + (int64_t)(u * kThreads + tid) * E::G;
+            q[u] = i < t1 ? ld_stream(row + i * E::BYTES) : make_uint4(0, 0, 0, 0);
+        }
+        Acc<NORM> acc;
+#pragma unroll
+        for (int u = 0; u < UNITS; ++u) {
+            int64_t i = t0 + (int64_t)(u * kThreads + tid) * E::G;
+            float v[E::G];
+            E::unpack(q[u], v);
+#pragma unroll
+            for (int e = 0; e < E::G; ++e)
+                if (i + e < t1) acc.add(v[e]);    // the row's padding beyond d is not data
+        }
+        __shared__ double sh[kWarps];
+        double w = warp_reduce<NORM>(acc.value());
+        if (lane == 0) sh[warp] = w;
+        __syncthreads();
+        if (tid == 0) {
+            double tot = sh[0];
+#pragma unroll
+            for (int k = 1; k < kWarps; ++k) tot = combine<NORM>(tot, sh[k]);
+            prow[tile + j0] = tot;
+        }
+    } else {
+        // several segments cross this tile: the warps take them in turn
+        for (int j = j0 + warp; j < nseg; j += kWarps) {
+            int64_t a = __ldg(seg_off + j), b = __ldg(seg_off + j + 1);
+            if (a >= t1) break;
+            a = max(a, t0); b = min(b, t1);
+            if (a >= b) continue;
+            Acc<NORM> acc;
+            for (int64_t i = a + lane; i < b; i += 32) {
+                float v = DT == UQ_F32 ? __ldg((const float *)row + i)
+                                       : __uint_as_float((uint32_t)__ldg((const uint16_t *)row + i) << 16);
+                acc.add(v);
+            }
+            double w = warp_reduce<NORM>(acc.value());
+            if (lane == 0) prow[tile + j] = w;
+        }
+    }
+}
+
+template <int NORM>
+__global__ void __launch_bounds__(kThreads)
+norm_finalize_kernel(const double *__restrict__ part, int M, int64_t d, int nseg,
+                     const int64_t *__restrict__ seg_off, int64_t ntiles, float *__restrict__ W,
+                     uint32_t *__restrict__ status)
+{
+    const int j = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int64_t a = seg_off ? __ldg(seg_off + j) : 0;
+    int64_t b = seg_off ? __ldg(seg_off + j + 1) : d;
+    const bool bad = a < 0 || b > d || a > b || (j == 0 && a != 0) || (j == nseg - 1 && b != d);
+    a = min(max(a, (int64_t)0), d);
+    b = min(max(b, a), d);
+
+    double best = 0.0;
+    if (a < b) {
+        const int64_t first = a / kNormTile, last = (b - 1) / kNormTile;
+        for (int m = warp; m < M; m += kWarps) {
+            const double *prow = part + (size_t)m * (size_t)(ntiles + nseg) + j;
+            double acc = 0.0;
+            for (int64_t t = first + lane; t <= last; t += 32) acc = combine<NORM>(acc, prow[t]);
+            const double r = warp_reduce<NORM>(acc);
+            best = (r != r || best != best) ? r + best : fmax(best, r);   // keep a NaN alive
+        }
+    }
+    __shared__ double sh[kWarps];
+    if (lane == 0) sh[warp] = best;
+    __syncthreads();
+    if (tid == 0) {
+        // fmax drops NaN, so look for it explicitly
+        bool nan = false;
+        double top = 0.0;
+        for (int k = 0; k < kWarps; ++k) { nan |= sh[k] != sh[k]; top = fmax(top, sh[k]); }
+        float w;
+        if (NORM == UQ_NORM_L2) w = nan ? __uint_as_float(0x7FC00000u) : __double2float_rn(sqrt(top));
+        else w = __uint_as_float((uint32_t)top);
+        W[j] = w;
+        uint32_t flags = 0;
+        if ((__float_as_uint(w) & 0x7F800000u) == 0x7F800000u) flags |= UQ_STATUS_NONFINITE;
+        if (bad) flags |= UQ_STATUS_BAD_SEGMENTS;
+        if (flags && status) atomicOr(status, flags);
+    }
+}
+
+template <int DT, int NORM>
+static cudaError_t launch(const uq_layout &L, const void *g, float *W, uint32_t *status, double *part,
+                          int64_t ntiles, cudaStream_t st)
+{
+    if (L.d > 0) {
+        dim3 grid((unsigned)ntiles, (unsigned)L.M);
+        norm_partials_kernel<DT, NORM><<<grid, kThreads, 0, st>>>(g, L.d, L.worker_stride, L.nseg,
+                                                                 L.seg_off, ntiles, part);
+    }
+    norm_finalize_kernel<NORM><<<L.nseg, kThreads, 0, st>>>(part, L.M, L.d, L.nseg, L.seg_off, ntiles, W,
+                                                          status);
+    return cudaGetLastError();
+}
+
+int64_t norm_tiles(int64_t d) { return (d + kNormTile - 1) / kNormTile; }
+
+cudaError_t launch_agree_scale(const uq_layout &L, const void *g, int norm, float *W, uint32_t *status,
+                               void *workspace, cudaStream_t st)
+{
+    const int64_t ntiles = norm_tiles(L.d);
+    double *part = (double *)workspace;
+    if (L.dtype == UQ_F32)
+        return norm == UQ_NORM_L2 ? launch<UQ_F32, UQ_NORM_L2>(L, g, W, status, part, ntiles, st)
+                                  : launch<UQ_F32, UQ_NORM_LINF>(L, g, W, status, part, ntiles, st);
+    return norm == UQ_NORM_L2 ? launch<UQ_BF16, UQ_NORM_L2>(L, g, W, status, part, ntiles, st)
+                              : launch<UQ_BF16, UQ_NORM_LINF>(L, g, W, status, part, ntiles, st);
+}
+
+}  // namespace uq

@@ -1,0 +1,193 @@
+// The C ABI declared in include/uq.h: argument validation on the host, then kernel launches.
+// No allocation, no synchronization, no state besides a thread-local last CUDA error.
+#include "uq_device.cuh"
+
+namespace uq {
+int64_t norm_tiles(int64_t d);
+cudaError_t launch_agree_scale(const uq_layout &L, const void *g, int norm, float *W, uint32_t *status,
+                               void *workspace, cudaStream_t st);
+cudaError_t launch_encode(const uq_layout &L, const void *g, const float *W, const ScaleSet &scales,
+                          const uint8_t *idx, int idx_bits, uint64_t seed, int rng_bits, int fmt, void *lev,
+                          uint32_t *status, cudaStream_t st);
+cudaError_t launch_select(const uq_layout &L, const void *g, const float *W, const ScaleSet &scales,
+                          int idx_bits, uint8_t *idx, uint32_t *status, cudaStream_t st);
+cudaError_t launch_aggregate_decode(const uq_layout &L, const void *lev, int fmt, const float *W,
+                                    const ScaleSet &scales, const uint8_t *idx, int idx_bits, float *out,
+                                    int32_t *S, cudaStream_t st);
+cudaError_t launch_decode_sums(const uq_layout &L, const int32_t *S, const float *W, const ScaleSet &scales,
+                               const uint8_t *idx, int idx_bits, float *out, cudaStream_t st);
+}  // namespace uq
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+int finish(cudaError_t e)
+{
+    if (e == cudaSuccess) return UQ_OK;
+    g_last_cuda_error = (int)e;
+    return UQ_ERR_CUDA;
+}
+
+bool aligned(const void *p, size_t a) { return ((uintptr_t)p & (a - 1)) == 0; }
+
+bool layout_ok(const uq_layout *L)
+{
+    if (L == nullptr) return false;
+    if (L->d < 0 || L->M < 1 || L->M > UQ_MAX_WORKERS || L->nseg < 1 || L->reserved != 0) return false;
+    if (L->dtype != UQ_F32 && L->dtype != UQ_BF16) return false;
+    if (L->worker_stride < L->d || (L->worker_stride & 31) != 0) return false;
+    if (L->seg_off == nullptr && L->nseg != 1) return false;
+    if (L->seg_off != nullptr && !aligned(L->seg_off, 8)) return false;
+    if (L->d > (int64_t)1 << 40) return false;
+    return true;
+}
+
+bool fmt_ok(int fmt, int s_hat)
+{
+    if (fmt == UQ_FMT_I8) return s_hat >= 1 && s_hat <= 127;
+    if (fmt == UQ_FMT_I4X2) return s_hat >= 1 && s_hat <= 7;
+    return false;
+}
+
+// Copies an ascending scale set into the kernel-parameter form; false if it is not valid.
+bool scales_ok(const int32_t *scales, int N, int idx_bits, uq::ScaleSet *out)
+{
+    if (scales == nullptr || N < 1 || N > UQ_MAX_SCALES) return false;
+    if (idx_bits != 2 && idx_bits != 4 && idx_bits != 8) return false;
+    if (idx_bits < 8 && N > (1 << idx_bits)) return false;
+    for (int k = 0; k < N; ++k) {
+        if (scales[k] < 1) return false;
+        if (k > 0 && scales[k] <= scales[k - 1]) return false;
+        out->s[k] = scales[k];
+    }
+    for (int k = N; k < UQ_MAX_SCALES; ++k) out->s[k] = scales[N - 1];
+    out->N = N;
+    return true;
+}
+
+uq::ScaleSet single_scale(int s)
+{
+    uq::ScaleSet set;
+    for (int k = 0; k < UQ_MAX_SCALES; ++k) set.s[k] = s;
+    set.N = 1;
+    return set;
+}
+
+}  // namespace
+
+extern "C" {
+
+int uq_version(void) { return 100; }
+
+int uq_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char *uq_error_string(int code)
+{
+    switch (code) {
+    case UQ_OK: return "ok";
+    case UQ_ERR_BAD_ARG: return "bad argument";
+    case UQ_ERR_CUDA: return "CUDA launch failed (see uq_last_cuda_error)";
+    case UQ_ERR_UNSUPPORTED: return "unsupported combination";
+    case UQ_ERR_WORKSPACE: return "workspace missing or too small";
+    default: return "unknown error code";
+    }
+}
+
+size_t uq_workspace_bytes(const uq_layout *L)
+{
+    if (!layout_ok(L)) return 0;
+    return (size_t)L->M * (size_t)(uq::norm_tiles(L->d) + L->nseg) * sizeof(double);
+}
+
+size_t uq_index_bytes(const uq_layout *L, int idx_bits)
+{
+    if (!layout_ok(L) || (idx_bits != 2 && idx_bits != 4 && idx_bits != 8)) return 0;
+    return (size_t)L->worker_stride * (size_t)idx_bits / 8;
+}
+
+int uq_agree_scale(const uq_layout *L, const void *g, int norm, float *W, uint32_t *status, void *workspace,
+                   size_t workspace_bytes, void *stream)
+{
+    if (!layout_ok(L) || W == nullptr || !aligned(W, 4) || !aligned(status, 4)) return UQ_ERR_BAD_ARG;
+    if (norm != UQ_NORM_L2 && norm != UQ_NORM_LINF) return UQ_ERR_BAD_ARG;
+    if (L->d > 0 && (g == nullptr || !aligned(g, 16))) return UQ_ERR_BAD_ARG;
+    if (workspace == nullptr || !aligned(workspace, 8) || workspace_bytes < uq_workspace_bytes(L))
+        return UQ_ERR_WORKSPACE;
+    return finish(uq::launch_agree_scale(*L, g, norm, W, status, workspace, (cudaStream_t)stream));
+}
+
+int uq_encode_single(const uq_layout *L, const void *g, const float *W, int s, uint64_t seed, int rng_bits,
+                     int fmt, void *lev, uint32_t *status, void *stream)
+{
+    if (!layout_ok(L) || W == nullptr || !aligned(status, 4)) return UQ_ERR_BAD_ARG;
+    if (!fmt_ok(fmt, s) || (rng_bits != 32 && rng_bits != 16)) return UQ_ERR_BAD_ARG;
+    if (L->d > 0 && (g == nullptr || lev == nullptr || !aligned(g, 16) || !aligned(lev, 16)))
+        return UQ_ERR_BAD_ARG;
+    return finish(uq::launch_encode(*L, g, W, single_scale(s), nullptr, 0, seed, rng_bits, fmt, lev, status,
+                                    (cudaStream_t)stream));
+}
+
+int uq_select_scale_multi(const uq_layout *L, const void *g, const float *W, const int32_t *scales, int N,
+                          int idx_bits, uint8_t *idx, uint32_t *status, void *stream)
+{
+    uq::ScaleSet set;
+    if (!layout_ok(L) || W == nullptr || !aligned(status, 4)) return UQ_ERR_BAD_ARG;
+    if (!scales_ok(scales, N, idx_bits, &set)) return UQ_ERR_BAD_ARG;
+    if (L->d > 0 && (g == nullptr || idx == nullptr || !aligned(g, 16) || !aligned(idx, 16)))
+        return UQ_ERR_BAD_ARG;
+    return finish(uq::launch_select(*L, g, W, set, idx_bits, idx, status, (cudaStream_t)stream));
+}
+
+int uq_encode_multi(const uq_layout *L, const void *g, const float *W, const int32_t *scales, int N,
+                    const uint8_t *idx, int idx_bits, uint64_t seed, int rng_bits, int fmt, void *lev,
+                    uint32_t *status, void *stream)
+{
+    uq::ScaleSet set;
+    if (!layout_ok(L) || W == nullptr || !aligned(status, 4)) return UQ_ERR_BAD_ARG;
+    if (!scales_ok(scales, N, idx_bits, &set)) return UQ_ERR_BAD_ARG;
+    if (!fmt_ok(fmt, set.s[0]) || (rng_bits != 32 && rng_bits != 16)) return UQ_ERR_BAD_ARG;
+    if (L->d > 0 && (g == nullptr || lev == nullptr || idx == nullptr || !aligned(g, 16) || !aligned(lev, 16) ||
+                     !aligned(idx, 16)))
+        return UQ_ERR_BAD_ARG;
+    return finish(uq::launch_encode(*L, g, W, set, idx, idx_bits, seed, rng_bits, fmt, lev, status,
+                                    (cudaStream_t)stream));
+}
+
+int uq_aggregate(const uq_layout *L, const void *lev, int fmt, int32_t *S, void *stream)
+{
+    if (!layout_ok(L) || (fmt != UQ_FMT_I8 && fmt != UQ_FMT_I4X2)) return UQ_ERR_BAD_ARG;
+    if (L->d > 0 && (lev == nullptr || S == nullptr || !aligned(lev, 16) || !aligned(S, 16)))
+        return UQ_ERR_BAD_ARG;
+    return finish(uq::launch_aggregate_decode(*L, lev, fmt, nullptr, single_scale(1), nullptr, 0, nullptr, S,
+                                              (cudaStream_t)stream));
+}
+
+int uq_decode(const uq_layout *L, const void *src, int src_kind, int fmt, const float *W, int s,
+              const int32_t *scales, int N, const uint8_t *idx, int idx_bits, float *out, int32_t *S_opt,
+              void *stream)
+{
+    if (!layout_ok(L) || W == nullptr) return UQ_ERR_BAD_ARG;
+    if (src_kind != UQ_SRC_LEVELS && src_kind != UQ_SRC_SUMS) return UQ_ERR_BAD_ARG;
+    uq::ScaleSet set;
+    if (scales != nullptr) {
+        if (!scales_ok(scales, N, idx_bits, &set)) return UQ_ERR_BAD_ARG;
+        if (L->d > 0 && (idx == nullptr || !aligned(idx, 16))) return UQ_ERR_BAD_ARG;
+    } else {
+        if (s < 1) return UQ_ERR_BAD_ARG;
+        set = single_scale(s);
+        idx_bits = 0;
+        idx = nullptr;
+    }
+    if (L->d > 0 && (src == nullptr || out == nullptr || !aligned(src, 16) || !aligned(out, 16)))
+        return UQ_ERR_BAD_ARG;
+    if (src_kind == UQ_SRC_SUMS)
+        return finish(uq::launch_decode_sums(*L, (const int32_t *)src, W, set, idx, idx_bits, out,
+                                             (cudaStream_t)stream));
+    if (fmt != UQ_FMT_I8 && fmt != UQ_FMT_I4X2) return UQ_ERR_BAD_ARG;
+    if (S_opt != nullptr && !aligned(S_opt, 16)) return UQ_ERR_BAD_ARG;
+    return finish(uq::launch_aggregate_decode(*L, src, fmt, W, set, idx, idx_bits, out, S_opt,
+                                              (cudaStream_t)stream));
+}
+
+}  // extern "C"

@@ -1,0 +1,287 @@
+// Integer aggregation of the workers' levels and reconstruction of the average gradient:
+// S_i = sum_m zeta^m_i (Algorithm 1 / 2, line "AllReduce gradients") and
+// g_hat_i = W_j * S_i / (s_i * M)  (Eq. R_s after Algorithm 1, Eq. R_{s_} after Algorithm 2).
+//
+// The fused kernel reads the M level streams once, keeps the sums in registers and writes only
+// the fp32 average (and, on request, the int32 sums).  A thread owns 16 B of every worker's
+// stream: 16 coordinates of int8 levels or 32 coordinates of packed 4-bit levels.
+#include "uq_device.cuh"
+
+namespace uq {
+
+struct DecodeParams {
+    const void *lev;          // level rows, or int32 sums for the sums-only kernel
+    const float *W;
+    const int64_t *seg_off;
+    const uint8_t *idx;
+    float *out;               // may be NULL (aggregate only)
+    int32_t *S;               // may be NULL
+    int64_t d, stride;
+    int32_t nseg, M;
+    ScaleSet scales;          // single-scale: N = 1
+};
+
+// W / ((float)s * (float)M): product, then one IEEE division.
+__device__ __forceinline__ float decode_factor(float W, int32_t s, int M)
+{
+    return __fdiv_rn(W, __fmul_rn((float)s, (float)M));
+}
+
+template <int IDXB> __device__ __forceinline__ int index_at(const uint8_t *idx, int64_t i)
+{
+    if (IDXB == 8) return idx[i];
+    const int per = 8 / IDXB;
+    return (idx[i / per] >> ((int)(i % per) * IDXB)) & ((1 << IDXB) - 1);
+}
+
+// Sums of C coordinates held by one thread.
+template <int FMT> struct Unit;
+
+template <> struct Unit<UQ_FMT_I8> {
+    static constexpr int C = 16;
+    // Bytes are biased to unsigned (x ^ 0x80) and added in 16-bit lanes: two lanes per word,
+    // M <= 64 workers * 255 < 2^16.  lane layout of word w: even = bytes 0,2; odd = bytes 1,3.
+    uint32_t even[4] = {0, 0, 0, 0}, odd[4] = {0, 0, 0, 0};
+    __device__ __forceinline__ void add(const uint4 &q)
+    {
+        const uint32_t w[4] = { q.x, q.y, q.z, q.w };
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t b = w[k] ^ 0x80808080u;
+            even[k] += b & 0x00FF00FFu;
+            odd[k] += (b >> 8) & 0x00FF00FFu;
+        }
+    }
+    __device__ __forceinline__ void finish(int M, int (&s)[16]) const
+    {
+        const int bias = 128 * M;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            s[4 * k + 0] = (int)(even[k] & 0xFFFFu) - bias;
+            s[4 * k + 1] = (int)(odd[k] & 0xFFFFu) - bias;
+            s[4 * k + 2] = (int)(even[k] >> 16) - bias;
+            s[4 * k + 3] = (int)(odd[k] >> 16) - bias;
+        }
+    }
+};
+
+template <> struct Unit<UQ_FMT_I4X2> {
+    static constexpr int C = 32;
+    // Nibbles are biased to unsigned (x ^ 8) and added in byte lanes for up to 16 workers
+    // (16 * 15 < 256), then widened into 16-bit lanes.
+    uint32_t lo8[4] = {0, 0, 0, 0}, hi8[4] = {0, 0, 0, 0};       // byte lanes: even / odd nibbles
+    uint32_t acc[4][4] = {};                                    // 16-bit lanes, see finish()
+    int pending = 0;
+    __device__ __forceinline__ void flush()
+    {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            acc[k][0] += lo8[k] & 0x00FF00FFu;          // nibbles 0, 4
+            acc[k][1] += (lo8[k] >> 8) & 0x00FF00FFu;   // nibbles 2, 6
+            acc[k][2] += hi8[k] & 0x00FF00FFu;          // nibbles 1, 5
+            acc[k][3] += (hi8[k] >> 8) & 0x00FF00FFu;   // nibbles 3, 7
+            lo8[k] = 0; hi8[k] = 0;
+        }
+        pending = 0;
+    }
+    __device__ __forceinline__ void add(const uint4 &q)
+    {
+        const uint32_t w[4] = { q.x, q.y, q.z, q.w };
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t b = w[k] ^ 0x88888888u;
+            lo8[k] += b & 0x0F0F0F0Fu;
+            hi8[k] += (b >> 4) & 0x0F0F0F0Fu;
+        }
+        if (++pending == 16) flush();
+    }
+    __device__ __forceinline__ void finish(int M, int (&s)[32])
+    {
+        flush();
+        const int bias = 8 * M;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            s[8 * k + 0] = (int)(acc[k][0] & 0xFFFFu) - bias;
+            s[8 * k + 4] = (int)(acc[k][0] >> 16) - bias;
+            s[8 * k + 2] = (int)(acc[k][1] & 0xFFFFu) - bias;
+            s[8 * k + 6] = (int)(acc[k][1] >> 16) - bias;
+            s[8 * k + 1] = (int)(acc[k][2] & 0xFFFFu) - bias;
+            s[8 * k + 5] = (int)(acc[k][2] >> 16) - bias;
+            s[8 * k + 3] = (int)(acc[k][3] & 0xFFFFu) - bias;
+            s[8 * k + 7] = (int)(acc[k][3] >> 16) - bias;
+        }
+    }
+};
+
+template <int FMT, int IDXB>
+__global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const DecodeParams p)
+{
+    using U = Unit<FMT>;
+    constexpr int C = U::C;
+    constexpr bool MULTI = IDXB != 0;
+    constexpr int TILE = kThreads * C;
+    const int64_t t0 = (int64_t)blockIdx.x * TILE;
+    const int64_t t1 = min(t0 + (int64_t)TILE, p.d);
+    const int tid = threadIdx.x;
+    const int64_t i = t0 + (int64_t)tid * C;
+    const size_t row_bytes = FMT == UQ_FMT_I8 ? (size_t)p.stride : (size_t)(p.stride >> 1);
+
+    U unit;
+    if (i < t1) {
+        const char *col = (const char *)p.lev + (size_t)i * 16 / C;
+        int m = 0;
+        for (; m + 8 <= p.M; m += 8) {          // eight workers' loads in flight
+            uint4 q[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) q[k] = ld_stream(col + (size_t)(m + k) * row_bytes);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) unit.add(q[k]);
+        }
+        for (; m < p.M; ++m) unit.add(ld_stream(col + (size_t)m * row_bytes));
+    }
+
+    // reconstruction factors of this tile's segment, one per scale
+    __shared__ float sh_c[UQ_MAX_SCALES];
+    const int j0 = find_segment(p.seg_off, p.nseg, t0);
+    const bool uniform = segment_end(p.seg_off, p.nseg, j0, p.d) >= t1;
+    if (p.out != nullptr && tid < p.scales.N) sh_c[tid] = decode_factor(__ldg(p.W + j0), p.scales.s[tid], p.M);
+    __syncthreads();
+    if (i >= t1) return;
+
+    int s[C];
+    unit.finish(p.M, s);
+
+    const bool full = i + C <= p.d;
+    if (p.S != nullptr) {
+        if (full) {
+#pragma unroll
+            for (int e = 0; e < C; e += 4)
+                st_stream((int4 *)(p.S + i + e), make_int4(s[e], s[e + 1], s[e + 2], s[e + 3]));
+        } else {
+            for (int e = 0; e < C; ++e)
+                if (i + e < p.d) p.S[i + e] = s[e];
+        }
+    }
+    if (p.out == nullptr) return;
+
+    float r[C];
+    if (uniform) {
+        if (MULTI) {
+            // idx bits of coordinates i..i+C-1 start at byte i*IDXB/8 (a multiple of 4 bytes)
+            constexpr int WORDS = C * (MULTI ? IDXB : 8) / 32;
+            uint32_t kw[WORDS];
+            const uint32_t *ip = (const uint32_t *)(p.idx + (size_t)i * IDXB / 8);
+#pragma unroll
+            for (int w = 0; w < WORDS; ++w) kw[w] = __ldg(ip + w);
+#pragma unroll
+            for (int e = 0; e < C; ++e) {
+                const int k = (kw[(e * IDXB) >> 5] >> ((e * IDXB) & 31)) & ((1 << IDXB) - 1);
+                r[e] = __fmul_rn((float)s[e], sh_c[k & (UQ_MAX_SCALES - 1)]);
+            }
+        } else {
+            const float c = sh_c[0];
+#pragma unroll
+            for (int e = 0; e < C; ++e) r[e] = __fmul_rn((float)s[e], c);
+        }
+    } else {
+        int j = find_segment(p.seg_off, p.nseg, i);
+        for (int e = 0; e < C; ++e) {
+            r[e] = 0.0f;
+            if (i + e >= p.d) continue;
+            j = advance_segment(p.seg_off, p.nseg, j, i + e);
+            const int k = MULTI ? index_at<MULTI ? IDXB : 8>(p.idx, i + e) : 0;
+            r[e] = __fmul_rn((float)s[e], decode_factor(__ldg(p.W + j), p.scales.s[k & (UQ_MAX_SCALES - 1)], p.M));
+        }
+    }
+    if (full) {
+#pragma unroll
+        for (int e = 0; e < C; e += 4)
+            st_stream((float4 *)(p.out + i + e), make_float4(r[e], r[e + 1], r[e + 2], r[e + 3]));
+    } else {
+        for (int e = 0; e < C; ++e)
+            if (i + e < p.d) p.out[i + e] = r[e];
+    }
+}
+
+// Reconstruction from already-summed levels (one thread per 4 coordinates).
+template <int IDXB>
+__global__ void __launch_bounds__(kThreads) decode_sums_kernel(const DecodeParams p)
+{
+    constexpr bool MULTI = IDXB != 0;
+    const int64_t i = ((int64_t)blockIdx.x * kThreads + threadIdx.x) * 4;
+    if (i >= p.d) return;
+    const int32_t *S = (const int32_t *)p.lev;
+    int s[4] = {0, 0, 0, 0};
+    const bool full = i + 4 <= p.d;
+    if (full) {
+        const int4 q = *(const int4 *)(S + i);
+        s[0] = q.x; s[1] = q.y; s[2] = q.z; s[3] = q.w;
+    } else {
+        for (int e = 0; e < 4; ++e)
+            if (i + e < p.d) s[e] = S[i + e];
+    }
+    float r[4];
+    int j = find_segment(p.seg_off, p.nseg, i);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        r[e] = 0.0f;
+        if (i + e >= p.d) continue;
+        j = advance_segment(p.seg_off, p.nseg, j, i + e);
+        const int k = MULTI ? index_at<MULTI ? IDXB : 8>(p.idx, i + e) : 0;
+        r[e] = __fmul_rn((float)s[e], decode_factor(__ldg(p.W + j), p.scales.s[k & (UQ_MAX_SCALES - 1)], p.M));
+    }
+    if (full) *(float4 *)(p.out + i) = make_float4(r[0], r[1], r[2], r[3]);
+    else
+        for (int e = 0; e < 4; ++e)
+            if (i + e < p.d) p.out[i + e] = r[e];
+}
+
+template <int FMT>
+static cudaError_t dispatch_levels(const DecodeParams &p, int idx_bits, cudaStream_t st)
+{
+    constexpr int TILE = kThreads * Unit<FMT>::C;
+    const int64_t blocks = (p.d + TILE - 1) / TILE;
+    if (blocks == 0) return cudaSuccess;
+    if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    const unsigned nb = (unsigned)blocks;
+    switch (idx_bits) {
+    case 0: aggregate_decode_kernel<FMT, 0><<<nb, kThreads, 0, st>>>(p); break;
+    case 2: aggregate_decode_kernel<FMT, 2><<<nb, kThreads, 0, st>>>(p); break;
+    case 4: aggregate_decode_kernel<FMT, 4><<<nb, kThreads, 0, st>>>(p); break;
+    default: aggregate_decode_kernel<FMT, 8><<<nb, kThreads, 0, st>>>(p); break;
+    }
+    return cudaGetLastError();
+}
+
+// out == NULL: aggregate only.  idx_bits == 0: single scale (scales = {s}).
+cudaError_t launch_aggregate_decode(const uq_layout &L, const void *lev, int fmt, const float *W,
+                                    const ScaleSet &scales, const uint8_t *idx, int idx_bits, float *out,
+                                    int32_t *S, cudaStream_t st)
+{
+    DecodeParams p;
+    p.lev = lev; p.W = W; p.seg_off = L.seg_off; p.idx = idx; p.out = out; p.S = S;
+    p.d = L.d; p.stride = L.worker_stride; p.nseg = L.nseg; p.M = L.M; p.scales = scales;
+    return fmt == UQ_FMT_I8 ? dispatch_levels<UQ_FMT_I8>(p, idx_bits, st)
+                            : dispatch_levels<UQ_FMT_I4X2>(p, idx_bits, st);
+}
+
+cudaError_t launch_decode_sums(const uq_layout &L, const int32_t *S, const float *W, const ScaleSet &scales,
+                               const uint8_t *idx, int idx_bits, float *out, cudaStream_t st)
+{
+    DecodeParams p;
+    p.lev = S; p.W = W; p.seg_off = L.seg_off; p.idx = idx; p.out = out; p.S = nullptr;
+    p.d = L.d; p.stride = L.worker_stride; p.nseg = L.nseg; p.M = L.M; p.scales = scales;
+    const int64_t blocks = (L.d + kThreads * 4 - 1) / (kThreads * 4);
+    if (blocks == 0) return cudaSuccess;
+    if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    const unsigned nb = (unsigned)blocks;
+    switch (idx_bits) {
+    case 0: decode_sums_kernel<0><<<nb, kThreads, 0, st>>>(p); break;
+    case 2: decode_sums_kernel<2><<<nb, kThreads, 0, st>>>(p); break;
+    case 4: decode_sums_kernel<4><<<nb, kThreads, 0, st>>>(p); break;
+    default: decode_sums_kernel<8><<<nb, kThreads, 0, st>>>(p); break;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace uq

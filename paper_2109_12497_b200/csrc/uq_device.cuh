@@ -1,0 +1,154 @@
+// Device-side helpers shared by the uq kernels (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "uq.h"
+
+namespace uq {
+
+constexpr int kThreads = 256;            // threads per CTA in every streaming kernel
+constexpr int kWarps = kThreads / 32;
+constexpr int kNormTile = 8192;          // coordinates per partial of the norm reduction
+
+struct ScaleSet {                        // the scale set s_ of the multi-scale quantizer
+    int32_t s[UQ_MAX_SCALES];
+    int32_t N;
+};
+
+// ---------------------------------------------------------------------------------------------
+// loads / stores
+// ---------------------------------------------------------------------------------------------
+
+// Streaming 128-bit load: the data is read once, keep it out of L1.
+__device__ __forceinline__ uint4 ld_stream(const void *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+template <typename T> __device__ __forceinline__ void st_stream(T *p, T v) { __stcs(p, v); }
+
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// Coordinates per 16-byte granule, and unpacking of a granule to binary32.
+template <int DT> struct Elem;
+template <> struct Elem<UQ_F32> {
+    static constexpr int G = 4;
+    static constexpr int BYTES = 4;
+    __device__ static __forceinline__ void unpack(const uint4 &q, float (&v)[4])
+    {
+        v[0] = __uint_as_float(q.x); v[1] = __uint_as_float(q.y);
+        v[2] = __uint_as_float(q.z); v[3] = __uint_as_float(q.w);
+    }
+};
+template <> struct Elem<UQ_BF16> {
+    static constexpr int G = 8;
+    static constexpr int BYTES = 2;
+    __device__ static __forceinline__ void unpack(const uint4 &q, float (&v)[8])
+    {
+        v[0] = bf16lo(q.x); v[1] = bf16hi(q.x); v[2] = bf16lo(q.y); v[3] = bf16hi(q.y);
+        v[4] = bf16lo(q.z); v[5] = bf16hi(q.z); v[6] = bf16lo(q.w); v[7] = bf16hi(q.w);
+    }
+};
+
+// ---------------------------------------------------------------------------------------------
+// segments
+// ---------------------------------------------------------------------------------------------
+
+// The segment that holds coordinate i: smallest j with seg_off[j+1] > i, clamped to
+// [0, nseg-1] so that a malformed table can never index outside W.
+__device__ __forceinline__ int find_segment(const int64_t *__restrict__ seg_off, int nseg, int64_t i)
+{
+    if (seg_off == nullptr) return 0;
+    int lo = 0, hi = nseg - 1;
+    while (lo < hi) {
+        int mid = (lo + hi) >> 1;
+        if (__ldg(seg_off + mid + 1) <= i) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+// Advance j (a segment at or before coordinate i's) to the segment holding i.
+__device__ __forceinline__ int advance_segment(const int64_t *__restrict__ seg_off, int nseg, int j, int64_t i)
+{
+    while (j + 1 < nseg && __ldg(seg_off + j + 1) <= i) ++j;
+    return j;
+}
+
+__device__ __forceinline__ int64_t segment_end(const int64_t *__restrict__ seg_off, int nseg, int j, int64_t d)
+{
+    return (seg_off == nullptr || j + 1 >= nseg) ? d : __ldg(seg_off + j + 1);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Philox4x32-10, counter = (block low, block high, worker, 0), key = seed
+// ---------------------------------------------------------------------------------------------
+
+struct PhiloxKey { uint32_t k0[10], k1[10]; };   // the ten round keys (uniform over the grid)
+
+__device__ __forceinline__ PhiloxKey philox_key(uint64_t seed)
+{
+    PhiloxKey k;
+    uint32_t a = (uint32_t)seed, b = (uint32_t)(seed >> 32);
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        k.k0[r] = a; k.k1[r] = b;
+        a += 0x9E3779B9u; b += 0xBB67AE85u;
+    }
+    return k;
+}
+
+__device__ __forceinline__ uint4 philox4x32_10(const PhiloxKey &k, uint64_t block, uint32_t worker)
+{
+    uint32_t c0 = (uint32_t)block, c1 = (uint32_t)(block >> 32), c2 = worker, c3 = 0u;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k.k0[r];
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k.k1[r];
+        c1 = (uint32_t)p1; c3 = (uint32_t)p0; c0 = n0; c2 = n2;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+// ---------------------------------------------------------------------------------------------
+// one coordinate of Q_s
+// ---------------------------------------------------------------------------------------------
+
+// x = min(|v| * inv, cap) with a single rounding; NaN collapses to cap.
+__device__ __forceinline__ float scaled_magnitude(float v, float inv, float cap)
+{
+    return fminf(__fmul_rn(fabsf(v), inv), cap);
+}
+
+// 23-bit draw: level = floor(x) + [h < rint((x - floor(x)) * 2^23)], 0 <= x <= 127.
+// floor comes from a round-down add of 2^23 (its low mantissa bits are floor(x)); the
+// threshold from a round-to-nearest add of 1.0 (its mantissa is rint(p * 2^23), and the carry
+// into the exponent makes it 2^23 when p rounds up to 1).
+__device__ __forceinline__ int level_draw23(float x, uint32_t word)
+{
+    float t = __fadd_rd(x, 8388608.0f);
+    float lf = __fsub_rn(t, 8388608.0f);
+    float p = __fsub_rn(x, lf);
+    uint32_t thr = __float_as_uint(__fadd_rn(p, 1.0f)) - 0x3F800000u;
+    uint32_t h = word >> 9;
+    return (int)(__float_as_uint(t) & 0xFFu) + (h < thr ? 1 : 0);
+}
+
+// 16-bit draw: x + 128 rounds x to 16 fractional bits (ties to even), so the mantissa of the
+// sum is floor(x)*2^16 + rint(p*2^16); adding 0xFFFF - h carries into bit 16 iff h < rint(p*2^16).
+__device__ __forceinline__ int level_draw16(float x, uint32_t h16)
+{
+    uint32_t fixed = __float_as_uint(__fadd_rn(x, 128.0f));
+    return (int)(((fixed + 0xFFFFu - h16) >> 16) & 0xFFu);
+}
+
+__device__ __forceinline__ int apply_sign(float v, int level) { return v < 0.0f ? -level : level; }
+
+}  // namespace uq

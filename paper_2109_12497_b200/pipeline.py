@@ -1,0 +1,92 @@
+"""One quantize -> aggregate -> reconstruct step over M resident worker buffers.
+
+``Quantizer`` owns the device buffers of one configuration (scales, scale indices, levels,
+scratch, output) and enqueues the C-ABI calls of Algorithm 1 (single-scale) or Algorithm 2
+(multi-scale) in order on the current stream.  It holds no arithmetic: each stage is one call
+into the CUDA library.
+"""
+from __future__ import annotations
+
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+class Quantizer:
+    def __init__(self, M: int, d: int, dtype: torch.dtype = torch.float32,
+                 seg_off: Optional[Sequence[int]] = None, s: int = 127,
+                 scales: Optional[Sequence[int]] = None, fmt: int = B.UQ_FMT_I8, idx_bits: int = 0,
+                 norm: int = B.UQ_NORM_L2, rng_bits: int = 32, keep_sums: bool = False,
+                 device: str | torch.device = "cuda"):
+        B.lib()                                     # fail now if the CUDA library is not built
+        dev = torch.device(device)
+        self.M, self.d, self.dtype = M, d, dtype
+        self.stride = -(-d // 32) * 32
+        self.multi = scales is not None and idx_bits != 0
+        self.s = int(scales[0]) if self.multi else int(s)
+        self.scales = [int(x) for x in scales] if self.multi else None
+        self.fmt, self.idx_bits, self.norm, self.rng_bits = fmt, idx_bits if self.multi else 0, norm, rng_bits
+        seg_dev = None
+        if seg_off is not None and len(seg_off) > 2:
+            seg_dev = torch.as_tensor(np.asarray(seg_off, dtype=np.int64), device=dev)
+        self.layout = B.Layout(M, d, self.stride, dtype, seg_dev)
+        nseg = self.layout.nseg
+        self.W = torch.zeros(nseg, dtype=torch.float32, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.workspace = torch.empty(max(8, self.layout.workspace_bytes()), dtype=torch.uint8, device=dev)
+        self.lev = torch.empty((M, self.layout.level_row_bytes(fmt)), dtype=torch.int8, device=dev)
+        self.idx = (torch.empty(max(16, self.layout.index_bytes(self.idx_bits)), dtype=torch.uint8, device=dev)
+                    if self.multi else None)
+        self.out = torch.empty(max(d, 1), dtype=torch.float32, device=dev)
+        self.S = torch.empty(max(d, 1), dtype=torch.int32, device=dev) if keep_sums else None
+
+    # the four stages, each one C-ABI call -------------------------------------------------------
+    def agree_scale(self, g: torch.Tensor) -> None:
+        B.uq_agree_scale(self.layout, g, self.norm, self.W, self.status, self.workspace)
+
+    def select_scale(self, g: torch.Tensor) -> None:
+        B.uq_select_scale_multi(self.layout, g, self.W, self.scales, self.idx_bits, self.idx, self.status)
+
+    def encode(self, g: torch.Tensor, seed: int) -> None:
+        if self.multi:
+            B.uq_encode_multi(self.layout, g, self.W, self.scales, self.idx, self.idx_bits, seed,
+                              self.rng_bits, self.fmt, self.lev, self.status)
+        else:
+            B.uq_encode_single(self.layout, g, self.W, self.s, seed, self.rng_bits, self.fmt, self.lev,
+                               self.status)
+
+    def aggregate_decode(self) -> None:
+        B.uq_decode(self.layout, self.lev, B.UQ_SRC_LEVELS, self.fmt, self.W, self.s, self.scales, self.idx,
+                    self.idx_bits, self.out, self.S)
+
+    def step(self, g: torch.Tensor, seed: int = 0) -> torch.Tensor:
+        """g: [M, stride] gradients of all workers -> the reconstructed average gradient [d]."""
+        self.agree_scale(g)
+        if self.multi:
+            self.select_scale(g)
+        self.encode(g, seed)
+        self.aggregate_decode()
+        return self.out[: self.d]
+
+    def kernels_per_step(self) -> int:
+        """Kernel launches one step enqueues (norm partials + finalize, [select], encode, decode)."""
+        return (2 if self.d > 0 else 1) + (1 if self.multi and self.d > 0 else 0) + (2 if self.d > 0 else 0)
+
+    def status_bits(self) -> int:
+        """Synchronizes and returns the device status word (0 = clean)."""
+        return int(self.status.item())
+
+
+def from_workload(w, keep_sums: bool = False, device="cuda") -> Quantizer:
+    """A Quantizer configured like a ``workloads.Workload``."""
+    from . import workloads as wl
+    seg = wl.segment_offsets(w)
+    return Quantizer(
+        M=w.M, d=w.d, dtype=torch.float32 if w.dtype == wl.F32 else torch.bfloat16, seg_off=seg, s=w.s,
+        scales=list(w.scales) if w.quantizer == "multi" else None,
+        fmt=B.UQ_FMT_I8 if w.fmt == "i8" else B.UQ_FMT_I4X2, idx_bits=w.idx_bits,
+        norm=B.UQ_NORM_L2 if w.norm == wl.NORM_L2 else B.UQ_NORM_LINF, rng_bits=w.rng_bits,
+        keep_sums=keep_sums, device=device)

@@ -1,0 +1,99 @@
+"""The C-ABI library loads without a GPU, exports everything include/uq.h declares, and its
+host-side argument validation rejects bad calls before any launch."""
+import ctypes as C
+import re
+from pathlib import Path
+
+import pytest
+
+from paper_2109_12497_b200 import binding as B
+from paper_2109_12497_b200 import build as uq_build
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module")
+def lib():
+    uq_build.build()
+    return B.lib()
+
+
+def declared_functions():
+    text = (ROOT / "include" / "uq.h").read_text()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(uq_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_functions()
+    assert set(names) == set(B.EXPORTS)
+    for n in names:
+        assert getattr(lib, n) is not None
+
+
+def test_constants_match_the_header():
+    text = (ROOT / "include" / "uq.h").read_text()
+    for name in ("UQ_OK", "UQ_ERR_BAD_ARG", "UQ_ERR_CUDA", "UQ_ERR_UNSUPPORTED", "UQ_ERR_WORKSPACE",
+                 "UQ_F32", "UQ_BF16", "UQ_NORM_LINF", "UQ_NORM_L2", "UQ_FMT_I8", "UQ_FMT_I4X2",
+                 "UQ_SRC_LEVELS", "UQ_SRC_SUMS", "UQ_STATUS_NONFINITE", "UQ_STATUS_BAD_SEGMENTS",
+                 "UQ_STATUS_SCALE_OVERFLOW"):
+        m = re.search(rf"\b{name}\s*=\s*(\d+)", text)
+        assert m and int(m.group(1)) == getattr(B, name), name
+
+
+def _layout(**kw):
+    base = dict(d=1000, worker_stride=1024, seg_off=None, M=2, nseg=1, dtype=B.UQ_F32, reserved=0)
+    base.update(kw)
+    return B.uq_layout(**base)
+
+
+def test_sizes(lib):
+    L = _layout()
+    assert lib.uq_workspace_bytes(C.byref(L)) == 2 * (1 + 1) * 8
+    assert lib.uq_index_bytes(C.byref(L), 2) == 256 and lib.uq_index_bytes(C.byref(L), 4) == 512
+    assert lib.uq_index_bytes(C.byref(L), 3) == 0
+    assert lib.uq_workspace_bytes(C.byref(_layout(worker_stride=1000))) == 0      # not a multiple of 32
+    assert lib.uq_version() >= 100
+    assert lib.uq_error_string(B.UQ_ERR_BAD_ARG) == b"bad argument"
+
+
+def test_bad_arguments_are_rejected_on_the_host(lib):
+    """None of these reaches a launch, so they run without a GPU (pointers are fake but aligned)."""
+    p = 0x10000
+    ok = _layout()
+    bad_layouts = [_layout(M=0), _layout(M=65), _layout(d=-1), _layout(worker_stride=992), _layout(nseg=2),
+                   _layout(dtype=5), _layout(reserved=1), _layout(nseg=0)]
+    for L in bad_layouts:
+        assert lib.uq_agree_scale(C.byref(L), p, B.UQ_NORM_L2, p, None, p, 1 << 20, None) == B.UQ_ERR_BAD_ARG
+        assert lib.uq_encode_single(C.byref(L), p, p, 127, 0, 32, B.UQ_FMT_I8, p, None, None) == B.UQ_ERR_BAD_ARG
+    r = C.byref(ok)
+    assert lib.uq_agree_scale(r, p, 1, p, None, p, 1 << 20, None) == B.UQ_ERR_BAD_ARG            # norm
+    assert lib.uq_agree_scale(r, p, B.UQ_NORM_L2, p, None, p, 8, None) == B.UQ_ERR_WORKSPACE      # too small
+    assert lib.uq_agree_scale(r, p, B.UQ_NORM_L2, p, None, None, 1 << 20, None) == B.UQ_ERR_WORKSPACE
+    assert lib.uq_agree_scale(r, p + 4, B.UQ_NORM_L2, p, None, p, 1 << 20, None) == B.UQ_ERR_BAD_ARG  # alignment
+    for s, fmt in ((0, B.UQ_FMT_I8), (128, B.UQ_FMT_I8), (8, B.UQ_FMT_I4X2), (5, 2)):
+        assert lib.uq_encode_single(r, p, p, s, 0, 32, fmt, p, None, None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_encode_single(r, p, p, 127, 0, 24, B.UQ_FMT_I8, p, None, None) == B.UQ_ERR_BAD_ARG  # rng_bits
+    assert lib.uq_encode_single(r, p, None, 127, 0, 32, B.UQ_FMT_I8, p, None, None) == B.UQ_ERR_BAD_ARG
+
+    def scales(*v):
+        return (C.c_int32 * len(v))(*v)
+    for sc, n, bits in ((scales(127, 127), 2, 2), (scales(127, 64), 2, 2), (scales(0, 5), 2, 2),
+                        (scales(1, 2, 3, 4, 5), 5, 2), (scales(127, 1016), 2, 3), (scales(127), 0, 2)):
+        assert lib.uq_select_scale_multi(r, p, p, sc, n, bits, p, None, None) == B.UQ_ERR_BAD_ARG
+        assert lib.uq_encode_multi(r, p, p, sc, n, p, bits, 0, 32, B.UQ_FMT_I8, p, None, None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_encode_multi(r, p, p, scales(200, 400), 2, p, 2, 0, 32, B.UQ_FMT_I8, p, None, None) \
+        == B.UQ_ERR_BAD_ARG                                                                        # s_hat > 127
+    assert lib.uq_aggregate(r, p, 7, p, None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_decode(r, p, 2, B.UQ_FMT_I8, p, 127, None, 0, None, 0, p, None, None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_decode(r, p, B.UQ_SRC_LEVELS, B.UQ_FMT_I8, p, 0, None, 0, None, 0, p, None, None) \
+        == B.UQ_ERR_BAD_ARG
+    assert lib.uq_decode(r, p, B.UQ_SRC_LEVELS, B.UQ_FMT_I8, p, 127, None, 0, None, 0, p + 4, None, None) \
+        == B.UQ_ERR_BAD_ARG
+
+
+def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "LIB_PATH", tmp_path / "missing.so")
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        B.lib()

@@ -1,0 +1,95 @@
+"""Parity at the full sizes of the five workloads, in the launch configuration the benchmark
+times.  c1-c3 are compared in full; c4 and c5 on the complete scale vector plus windows of
+coordinates (first, last with the ragged tail, bucket boundaries, random offsets) where every
+level, index, sum and reconstructed value is compared with the oracle."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import uq_oracle as o
+from paper_2109_12497_b200 import workloads as wl
+from paper_2109_12497_b200.pipeline import from_workload
+from parity import FP32_RTOL, check_parity, to_device, ulp_distance
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True)
+def _oracle_threads():
+    o.set_threads(max(1, os.cpu_count() or 1))
+    yield
+    o.set_threads(1)
+
+
+@pytest.mark.parametrize("name", ["c1", "c2", "c3"])
+def test_full_workload(name):
+    w = wl.WORKLOADS[name]
+    r = check_parity(w, wl.generate(w))
+    lev = r["ref"]["lev_raw"]
+    assert np.abs(lev.astype(int)).max() <= w.s
+    if name == "c1":                       # max|g| scale: the whole level range is in use
+        assert np.abs(lev.astype(int)).max() == 127 and len(np.unique(lev)) > 200
+
+
+def _windows(w, seg, rng, n_random=6, size=1 << 18):
+    d = w.d
+    wins = [(0, min(d, size)), (max(0, d - size - 13), d)]
+    for e in seg[1:-1][:: max(1, (len(seg) - 2) // 4)]:           # around segment boundaries
+        wins.append((max(0, int(e) - size // 2), min(d, int(e) + size // 2)))
+    for a in rng.integers(0, max(1, d - size), size=n_random):
+        a = int(a) | 1                                            # odd offsets too
+        wins.append((a, min(d, a + size)))
+    return wins
+
+
+@pytest.mark.parametrize("name", ["c4", "c5"])
+def test_sampled_windows_of_large_workload(name):
+    w = wl.WORKLOADS[name]
+    g_np = wl.generate(w, threads=max(1, os.cpu_count() or 1))
+    seg = wl.segment_offsets(w)
+    q = from_workload(w, keep_sums=True)
+    g = torch.empty((w.M, w.stride), dtype=torch.float32 if w.dtype == wl.F32 else torch.bfloat16,
+                    device="cuda")
+    for m in range(w.M):
+        g[m].copy_(to_device(w, g_np[m: m + 1])[0])
+    q.step(g, w.seed)
+    torch.cuda.synchronize()
+    assert q.status_bits() == 0
+    del g
+    W = q.W.cpu().numpy()
+    W_ref = o.agree_scale(g_np[:, : w.d], seg, o.NORM_L2)
+    assert ulp_distance(W, W_ref).max() <= 1
+    rng = np.random.default_rng(17)
+    for a, b in _windows(w, seg, rng):
+        gw = np.ascontiguousarray(g_np[:, a:b])
+        if w.quantizer == "multi":
+            idx = o.select_scale_multi(gw, W, w.scales, seg_off=seg, coord0=a)
+            lev = o.encode_multi(gw, W, w.scales, idx, w.seed, w.rng_bits, seg_off=seg, coord0=a)
+            out = o.decode(o.aggregate(lev), w.M, W, scales=w.scales, idx=idx, seg_off=seg, coord0=a)
+            per = 8 // w.idx_bits
+            a8, b8 = -(-a // per) * per, b // per * per           # whole index bytes inside the window
+            got = q.idx[a8 // per: b8 // per].cpu().numpy()
+            assert np.array_equal(got, o.pack_index(idx[a8 - a: b8 - a], w.idx_bits)), (a, b)
+        else:
+            lev = o.encode_single(gw, W, w.s, w.seed, w.rng_bits, seg_off=seg, coord0=a)
+            out = o.decode(o.aggregate(lev), w.M, W, s=w.s, seg_off=seg, coord0=a)
+        if w.fmt == "i4x2":
+            a2, b2 = a + (a & 1), b - (b & 1)                      # whole bytes inside the window
+            got = q.lev[:, a2 // 2: b2 // 2].cpu().numpy().view(np.uint8)
+            want = o.pack_levels_i4(_even_stride(lev[:, a2 - a: b2 - a]))
+            assert np.array_equal(got, want), (a, b)
+        else:
+            assert np.array_equal(q.lev[:, a:b].cpu().numpy(), lev), (a, b)
+        assert np.array_equal(q.S[a:b].cpu().numpy(), o.aggregate(lev)), (a, b)
+        assert np.allclose(q.out[a:b].cpu().numpy(), out, rtol=FP32_RTOL, atol=0), (a, b)
+        assert np.abs(lev.astype(int)).max() <= w.s
+
+
+def _even_stride(lev):
+    """Copy with an even row stride, as the 4-bit packer needs."""
+    M, n = lev.shape
+    buf = np.zeros((M, n + (n & 1) + 2), dtype=np.int8)
+    buf[:, :n] = lev
+    return buf[:, :n]

@@ -1,0 +1,183 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2109_12497_b200 import binding as B
+from paper_2109_12497_b200 import workloads as wl
+from parity import check_parity, run_gpu, run_oracle, to_device
+
+pytestmark = pytest.mark.gpu
+
+# sizes: below one unit, around unit / tile boundaries, several tiles with a ragged tail
+SIZES = [1, 2, 3, 7, 8, 9, 15, 16, 17, 31, 33, 255, 4095, 4097, 8191, 8193, 20011, 70001]
+
+
+@pytest.mark.parametrize("d", SIZES)
+@pytest.mark.parametrize("name", ["c1", "c4"])
+def test_one_segment_sizes(name, d):
+    w = wl.scaled(name, d, M=3)
+    check_parity(w, wl.generate(w))
+
+
+@pytest.mark.parametrize("d", [161 * 8, 20011, 300007])
+@pytest.mark.parametrize("name", ["c2", "c3", "c5"])
+@pytest.mark.parametrize("rng_bits", [32, 16])
+def test_segmented_workloads_small(name, d, rng_bits):
+    w = wl.scaled(name, d, rng_bits=rng_bits)
+    r = check_parity(w, wl.generate(w))
+    lev = r["ref"]["lev_raw"]
+    assert np.abs(lev.astype(int)).max() <= w.s
+
+
+@pytest.mark.parametrize("norm", [wl.NORM_L2, wl.NORM_LINF])
+@pytest.mark.parametrize("fmt,s", [("i8", 127), ("i8", 1), ("i8", 5), ("i4x2", 7), ("i4x2", 1)])
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+def test_single_scale_variants(norm, fmt, s, dtype):
+    w = wl.scaled("c2", 50021, M=4, norm=norm, fmt=fmt, s=s, scales=(s,), dtype=dtype)
+    check_parity(w, wl.generate(w))
+
+
+@pytest.mark.parametrize("idx_bits,N", [(2, 2), (2, 4), (4, 3), (4, 8), (4, 16), (8, 5), (8, 16)])
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+@pytest.mark.parametrize("fmt,s,ratio", [("i8", 127, 8), ("i4x2", 7, 16), ("i8", 31, 2)])
+def test_multi_scale_variants(idx_bits, N, dtype, fmt, s, ratio):
+    if s * ratio ** (N - 1) >= 2 ** 31:
+        pytest.skip("scale does not fit int32")
+    scales = tuple(s * ratio ** k for k in range(N))
+    w = wl.scaled("c3", 40009, M=5, idx_bits=idx_bits, scales=scales, s=s, fmt=fmt, dtype=dtype)
+    r = check_parity(w, wl.generate(w))
+    assert len(np.unique(r["ref"]["idx_raw"])) >= 2          # more than one scale is in use
+
+
+@pytest.mark.parametrize("M", [1, 2, 7, 8, 9, 16, 17, 33, 64])
+def test_worker_counts(M):
+    for name in ("c1", "c4", "c3"):
+        w = wl.scaled(name, 9001, M=M)
+        check_parity(w, wl.generate(w))
+
+
+def test_seed_changes_the_draws_only():
+    w = wl.scaled("c1", 30000, M=2)
+    g = wl.generate(w)
+    a = check_parity(w, g, seed=0)
+    b = check_parity(w, g, seed=(1 << 40) + 12345)
+    assert (a["lev"] != b["lev"]).mean() > 0.2
+    assert np.abs(a["lev"].view(np.int8).astype(int) - b["lev"].view(np.int8)).max() <= 1
+
+
+def test_full_level_range_and_saturation():
+    """Values at, just below and (with a caller-supplied scale) above W: levels reach +-s and
+    never leave [-s, s]."""
+    w = wl.scaled("c1", 4096, M=2)
+    g = wl.generate(w)
+    g[0, 5] = np.abs(g).max() * 3
+    r = check_parity(w, g)
+    lev = r["lev"].view(np.int8)
+    assert lev[0, 5] == 127 and np.abs(lev.astype(int)).max() == 127
+    # a scale smaller than the data: the clamp saturates instead of overflowing int8
+    q = r["q"]
+    gd = to_device(w, g)
+    q.W.fill_(float(np.abs(g).max()) / 50)
+    q.encode(gd, 0)
+    torch.cuda.synchronize()
+    lev = q.lev.cpu().numpy()
+    ref = run_oracle(w, g, q.W.cpu().numpy())["lev_raw"]
+    assert np.array_equal(lev[:, : w.d], ref) and np.abs(lev.astype(int)).max() == 127
+
+
+def test_zero_and_empty_inputs():
+    w = wl.scaled("c3", 5000, M=3)
+    g = np.zeros((w.M, w.stride), dtype=np.float32)
+    r = check_parity(w, g)
+    assert not r["W"].any() and not r["S"].any() and not r["out"].any()
+    assert (r["ref"]["idx_raw"] == len(w.scales) - 1).all()
+    # segments that are empty or all zero next to ordinary ones
+    w = dataclasses.replace(wl.scaled("c2", 6000, M=3), segments="one")
+    g = wl.generate(w)
+    g[:, 1000:2000] = 0
+    seg = np.array([0, 0, 1000, 2000, 2000, 4097, 6000], dtype=np.int64)
+    from paper_2109_12497_b200.pipeline import Quantizer
+    from oracle import uq_oracle as o
+    q = Quantizer(w.M, w.d, seg_off=seg, s=127, keep_sums=True)
+    out = q.step(torch.from_numpy(g).cuda(), 3).cpu().numpy()
+    W = o.agree_scale(g[:, : w.d], seg)
+    assert np.array_equal(q.W.cpu().numpy(), W) and W[0] == 0 and W[2] == 0 and W[3] == 0
+    lev = o.encode_single(g[:, : w.d], W, 127, 3, seg_off=seg)
+    assert np.array_equal(q.lev.cpu().numpy()[:, : w.d], lev)
+    assert np.allclose(out, o.decode(o.aggregate(lev), w.M, W, s=127, seg_off=seg), rtol=1e-6, atol=0)
+    assert q.status_bits() == 0
+    # d = 0 launches nothing and succeeds
+    q0 = Quantizer(2, 0)
+    q0.step(torch.zeros((2, 0), dtype=torch.float32, device="cuda"))
+    assert q0.status_bits() == 0
+
+
+def test_aggregate_and_decode_entry_points_agree_with_the_fused_kernel():
+    for name in ("c2", "c4", "c5"):
+        w = wl.scaled(name, 33333)
+        r = check_parity(w, wl.generate(w))
+        q = r["q"]
+        S = torch.empty(w.d, dtype=torch.int32, device="cuda")
+        B.uq_aggregate(q.layout, q.lev, q.fmt, S)
+        out = torch.empty(w.d, dtype=torch.float32, device="cuda")
+        B.uq_decode(q.layout, S, B.UQ_SRC_SUMS, q.fmt, q.W, q.s, q.scales, q.idx, q.idx_bits, out)
+        torch.cuda.synchronize()
+        assert np.array_equal(S.cpu().numpy(), r["S"])
+        assert np.array_equal(out.cpu().numpy(), r["out"])
+
+
+def test_outputs_stay_inside_their_buffers():
+    """Canaries around out / S / idx survive; level padding may be written but stays small."""
+    w = wl.scaled("c3", 10007, M=3)
+    g = wl.generate(w)
+    q = run_gpu(w, g)["q"]
+    pad = 64
+    out = torch.full((w.d + 2 * pad,), 7.0, dtype=torch.float32, device="cuda")
+    S = torch.full((w.d + 2 * pad,), 7, dtype=torch.int32, device="cuda")
+    # slices keep 16-byte alignment (pad is a multiple of 4 elements)
+    B.uq_decode(q.layout, q.lev, B.UQ_SRC_LEVELS, q.fmt, q.W, q.s, q.scales, q.idx, q.idx_bits,
+                out[pad: pad + w.d], S[pad: pad + w.d])
+    torch.cuda.synchronize()
+    for t in (out, S):
+        t = t.cpu().numpy()
+        assert (t[:pad] == 7).all() and (t[pad + w.d:] == 7).all()
+    nbytes = q.layout.index_bytes(w.idx_bits)
+    idx = torch.full((nbytes + 32,), 0xAB, dtype=torch.uint8, device="cuda")
+    B.uq_select_scale_multi(q.layout, to_device(w, g), q.W, q.scales, q.idx_bits, idx[16: 16 + nbytes], None)
+    torch.cuda.synchronize()
+    idx = idx.cpu().numpy()
+    assert (idx[:16] == 0xAB).all() and (idx[16 + nbytes:] == 0xAB).all()
+
+
+def test_status_word_reports_bad_data_without_trapping():
+    w = wl.scaled("c2", 20000, M=2)
+    g = wl.generate(w)
+    for bad in (np.nan, np.inf, -np.inf):
+        for norm in (wl.NORM_L2, wl.NORM_LINF):
+            ww = dataclasses.replace(w, norm=norm)
+            gg = g.copy(); gg[1, 12345] = bad
+            r = run_gpu(ww, gg)
+            assert r["status"] & B.UQ_STATUS_NONFINITE
+            assert np.abs(r["lev"].view(np.int8).astype(int)).max() <= 127
+    # a segment table that does not end at d / is not monotone
+    from paper_2109_12497_b200.pipeline import Quantizer
+    for seg in ([0, 100, 50, 20000], [0, 100, 19000], [5, 100, 20000]):
+        q = Quantizer(2, 20000, seg_off=np.array(seg))
+        q.step(torch.from_numpy(g).cuda())
+        assert q.status_bits() & B.UQ_STATUS_BAD_SEGMENTS
+    # a scale so small that s / W overflows
+    q = Quantizer(2, 20000)
+    q.W.fill_(1e-44)
+    q.encode(torch.from_numpy(g).cuda(), 0)
+    assert q.status_bits() & B.UQ_STATUS_SCALE_OVERFLOW
+
+
+def test_reproducible_bit_for_bit():
+    w = wl.scaled("c5", 200003)
+    g = wl.generate(w)
+    a, b = run_gpu(w, g), run_gpu(w, g)
+    for k in ("W", "lev", "idx", "S", "out"):
+        assert np.array_equal(a[k], b[k])
