@@ -91,7 +91,7 @@ __device__ __forceinline__ int64_t segment_end(const int64_t *__restrict__ seg_o
 
 struct PhiloxKey { uint32_t k0[10], k1[10]; };   // the ten round keys (uniform over the grid)
 
-__device__ __forceinline__ PhiloxKey philox_key(uint64_t seed)
+__host__ __device__ __forceinline__ PhiloxKey philox_key(uint64_t seed)
 {
     PhiloxKey k;
     uint32_t a = (uint32_t)seed, b = (uint32_t)(seed >> 32);
@@ -103,9 +103,9 @@ __device__ __forceinline__ PhiloxKey philox_key(uint64_t seed)
     return k;
 }
 
-__device__ __forceinline__ uint4 philox4x32_10(const PhiloxKey &k, uint64_t block, uint32_t worker)
+__device__ __forceinline__ uint4 philox4x32_10(const PhiloxKey &k, uint32_t block_lo, uint32_t block_hi, uint32_t worker)
 {
-    uint32_t c0 = (uint32_t)block, c1 = (uint32_t)(block >> 32), c2 = worker, c3 = 0u;
+    uint32_t c0 = block_lo, c1 = block_hi, c2 = worker, c3 = 0u;
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
         uint64_t p0 = (uint64_t)0xD2511F53u * c0;
@@ -127,28 +127,67 @@ __device__ __forceinline__ float scaled_magnitude(float v, float inv, float cap)
     return fminf(__fmul_rn(fabsf(v), inv), cap);
 }
 
-// 23-bit draw: level = floor(x) + [h < rint((x - floor(x)) * 2^23)], 0 <= x <= 127.
-// floor comes from a round-down add of 2^23 (its low mantissa bits are floor(x)); the
-// threshold from a round-to-nearest add of 1.0 (its mantissa is rint(p * 2^23), and the carry
-// into the exponent makes it 2^23 when p rounds up to 1).
-__device__ __forceinline__ int level_draw23(float x, uint32_t word)
+// 23-bit draw.  Returns a word whose LOW byte is the signed level
+//   zeta = sign(v) * (floor(x) + [h < rint((x - floor(x)) * 2^23)]),  h = word >> 9,  0 <= x <= 127.
+// t = x + 2^23 rounded down holds floor(x) in its low mantissa bits; t - (2^23 + 1) = floor(x) - 1
+// exactly, so x - that is p + 1 with one rounding: its mantissa is rint(p * 2^23), and the carry
+// into the exponent makes it 2^23 when p rounds up to 1.  The draw is placed under the same
+// exponent by one funnel shift, so the test is a single unsigned compare.
+__device__ __forceinline__ uint32_t signed_level_draw23(float v, float x, uint32_t word)
 {
-    float t = __fadd_rd(x, 8388608.0f);
-    float lf = __fsub_rn(t, 8388608.0f);
-    float p = __fsub_rn(x, lf);
-    uint32_t thr = __float_as_uint(__fadd_rn(p, 1.0f)) - 0x3F800000u;
-    uint32_t h = word >> 9;
-    return (int)(__float_as_uint(t) & 0xFFu) + (h < thr ? 1 : 0);
+    const float t = __fadd_rd(x, 8388608.0f);
+    const float p1 = __fsub_rn(x, __fsub_rn(t, 8388609.0f));
+    const uint32_t hb = __funnelshift_r(word, 0x7Fu, 9);          // 0x3F800000 | (word >> 9)
+    uint32_t lv = __float_as_uint(t) + (hb < __float_as_uint(p1) ? 1u : 0u);
+    if (v < 0.0f) lv = 0u - lv;                                   // low byte: two's complement
+    return lv;
+}
+constexpr uint32_t kLevelByte23 = 0;      // which byte of the returned word holds the level
+
+// 16-bit draw.  Returns a word whose byte 2 is the signed level (h16 = the 16-bit draw).
+// x + 128 rounds x to 16 fractional bits (ties to even): the mantissa of the sum is
+// floor(x) * 2^16 + rint(p * 2^16); adding 0xFFFF - h carries into bit 16 iff h < rint(p * 2^16).
+// 0xFFFF - sum = ~sum + 0x10000 negates byte 2 in two's complement.
+__device__ __forceinline__ uint32_t signed_level_draw16(float v, float x, uint32_t h16)
+{
+    uint32_t sum = __float_as_uint(__fadd_rn(x, 128.0f)) + 0xFFFFu - h16;
+    if (v < 0.0f) sum = 0xFFFFu - sum;
+    return sum;
+}
+constexpr uint32_t kLevelByte16 = 2;
+
+// Gathers byte B of four words into one word (coordinate order = byte order).
+template <uint32_t B> __device__ __forceinline__ uint32_t gather_bytes(uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    constexpr uint32_t sel = B | ((B + 4) << 4);
+    return __byte_perm(__byte_perm(a, b, sel), __byte_perm(c, d, sel), 0x5410);
 }
 
-// 16-bit draw: x + 128 rounds x to 16 fractional bits (ties to even), so the mantissa of the
-// sum is floor(x)*2^16 + rint(p*2^16); adding 0xFFFF - h carries into bit 16 iff h < rint(p*2^16).
-__device__ __forceinline__ int level_draw16(float x, uint32_t h16)
-{
-    uint32_t fixed = __float_as_uint(__fadd_rn(x, 128.0f));
-    return (int)(((fixed + 0xFFFFu - h16) >> 16) & 0xFFu);
-}
+// ---------------------------------------------------------------------------------------------
+// the segment of a tile, found by one warp without shared memory
+// ---------------------------------------------------------------------------------------------
 
-__device__ __forceinline__ int apply_sign(float v, int level) { return v < 0.0f ? -level : level; }
+// Smallest j in [0, nseg-1] with seg_off[j+1] > i, searched by all 32 lanes of the calling warp
+// together: every step probes 32 evenly spaced entries and a ballot narrows the range 32-fold,
+// so nseg <= 1024 costs two dependent loads.  The result is clamped to the table whatever the
+// table holds.  Must be called by a full warp with the same arguments in every lane.
+__device__ __forceinline__ int warp_find_segment(const int64_t *__restrict__ seg_off, int nseg, int64_t i)
+{
+    if (seg_off == nullptr) return 0;
+    const int lane = threadIdx.x & 31;
+    int lo = 0, hi = nseg - 1;
+    while (lo < hi) {
+        const int len = hi - lo + 1;
+        const int step = (len + 31) >> 5;
+        const int j = min(lo + (lane + 1) * step - 1, hi);           // last candidate of my slice
+        const bool beyond = j >= hi || __ldg(seg_off + j + 1) > i;     // answer is at or before j
+        const unsigned vote = __ballot_sync(0xFFFFFFFFu, beyond);
+        const int first = __ffs(vote) - 1;                             // vote != 0: the last lane sees j >= hi
+        const int nlo = lo + first * step;
+        hi = min(nlo + step - 1, hi);
+        lo = min(nlo, hi);
+    }
+    return lo;
+}
 
 }  // namespace uq

@@ -18,14 +18,14 @@ struct EncodeParams {
     const uint8_t *idx;
     uint32_t *status;
     int64_t d, stride;
-    uint64_t seed;
     int32_t nseg, M;
     float cap;                // (float) of the smallest scale: the largest level
-    ScaleSet scales;          // single-scale: N = 1, s[0] = s
+    ScaleSet scales;          // single-scale: every entry is s
+    PhiloxKey key;            // the ten round keys of the seed
 };
 
 template <int DT> struct EncodeShape {
-    static constexpr int UNITS = DT == UQ_F32 ? 2 : 4;          // 64 B of input per thread
+    static constexpr int UNITS = DT == UQ_F32 ? 4 : 8;          // 128 B of input per thread
     static constexpr int TILE = kThreads * UNITS * 8;
 };
 
@@ -35,116 +35,159 @@ __device__ __forceinline__ float inv_scale(int32_t s, float W)
     return W > 0.0f ? __fdiv_rn((float)s, W) : 0.0f;
 }
 
-template <int IDXB> __device__ __forceinline__ uint64_t load_idx8(const uint8_t *idx, int64_t i)
+__device__ __forceinline__ bool not_finite(float x) { return (__float_as_uint(x) & 0x7F800000u) == 0x7F800000u; }
+
+// The idx_bits * 8 bits that belong to 8 consecutive coordinates starting at a multiple of 8.
+template <int IDXB> struct IdxBits;
+template <> struct IdxBits<2> { using T = uint32_t; static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg((const uint16_t *)p); } };
+template <> struct IdxBits<4> { using T = uint32_t; static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg((const uint32_t *)p); } };
+template <> struct IdxBits<8> { using T = uint64_t; static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg((const unsigned long long *)p); } };
+
+// Eight coordinates: magnitudes scaled by inv[e], random words from the block(s) starting at
+// (blk_lo, blk_hi), signed levels packed into the wire format and stored at `dst`.
+// coordinate c uses word c%4 of block c/4 (32-bit draws) or half (c%8)%2 of word (c%8)/2 of block
+// c/8 (16-bit draws).
+template <int FMT, int RNG>
+__device__ __forceinline__ void quantize_unit(const float (&v)[8], const float (&inv)[8], float cap,
+                                              const PhiloxKey &key, uint32_t blk_lo, uint32_t blk_hi, uint32_t m,
+                                              void *dst)
 {
-    // the idx_bits * 8 bits that belong to coordinates i..i+7 (i is a multiple of 8)
-    if (IDXB == 2) return *(const uint16_t *)(idx + (i >> 2));
-    if (IDXB == 4) return *(const uint32_t *)(idx + (i >> 1));
-    return *(const uint64_t *)(idx + i);
+    constexpr uint32_t LB = RNG == 32 ? kLevelByte23 : kLevelByte16;
+    uint32_t z[8];
+    if (RNG == 32) {
+        const uint4 r0 = philox4x32_10(key, blk_lo, blk_hi, m);
+        const uint4 r1 = philox4x32_10(key, blk_lo + 1u, blk_hi, m);      // blk_lo is even: no carry
+        const uint32_t w[8] = { r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w };
+#pragma unroll
+        for (int e = 0; e < 8; ++e) z[e] = signed_level_draw23(v[e], scaled_magnitude(v[e], inv[e], cap), w[e]);
+    } else {
+        const uint4 r = philox4x32_10(key, blk_lo, blk_hi, m);
+        const uint32_t w[4] = { r.x, r.y, r.z, r.w };
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const uint32_t h16 = (e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu);
+            z[e] = signed_level_draw16(v[e], scaled_magnitude(v[e], inv[e], cap), h16);
+        }
+    }
+    if (FMT == UQ_FMT_I8) {
+        uint2 out;
+        out.x = gather_bytes<LB>(z[0], z[1], z[2], z[3]);
+        out.y = gather_bytes<LB>(z[4], z[5], z[6], z[7]);
+        st_stream((uint2 *)dst, out);
+    } else {
+        uint32_t out = 0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) out |= ((z[e] >> (8 * LB)) & 0xFu) << (4 * e);
+        st_stream((uint32_t *)dst, out);
+    }
+}
+
+// Coordinates [a, b) of worker m with per-coordinate scale lookup and bounds: the ragged last
+// tile and the 256-coordinate rows that a segment boundary crosses.  `who` of `many` cooperating
+// threads takes every many-th unit.  Rare (a few rows per segment), so kept out of line.
+template <int DT, int FMT, int RNG, int IDXB>
+__device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, int64_t a, int64_t b, int who, int many)
+{
+    using E = Elem<DT>;
+    constexpr bool MULTI = IDXB != 0;
+    constexpr int IB = MULTI ? IDXB : 8;
+    const char *row = (const char *)p.g + (size_t)m * (size_t)p.stride * E::BYTES;
+    for (int64_t i = a + (int64_t)who * 8; i < b; i += (int64_t)many * 8) {
+        float v[8];
+#pragma unroll
+        for (int h = 0; h < 8 / E::G; ++h)
+            E::unpack(ld_stream(row + (i + h * E::G) * E::BYTES), *(float(*)[E::G])(v + h * E::G));
+        typename IdxBits<IB>::T kbits = 0;
+        if (MULTI) kbits = IdxBits<IB>::load(p.idx + i * IB / 8);
+        float inv[8];
+        int j = find_segment(p.seg_off, p.nseg, i);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            if (i + e >= p.d) v[e] = 0.0f;                        // padding quantizes to level 0
+            j = advance_segment(p.seg_off, p.nseg, j, i + e);
+            const int k = MULTI ? (int)((kbits >> (e * IB)) & ((1u << IB) - 1u)) : 0;
+            inv[e] = inv_scale(p.scales.s[k & (UQ_MAX_SCALES - 1)], __ldg(p.W + j));
+            if (not_finite(inv[e]) && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
+        }
+        const uint64_t blk = RNG == 32 ? (uint64_t)(i >> 2) : (uint64_t)(i >> 3);
+        char *dst = FMT == UQ_FMT_I8 ? (char *)p.lev + (size_t)m * (size_t)p.stride + i
+                                     : (char *)p.lev + (size_t)m * (size_t)(p.stride >> 1) + (i >> 1);
+        quantize_unit<FMT, RNG>(v, inv, p.cap, p.key, (uint32_t)blk, (uint32_t)(blk >> 32), (uint32_t)m, dst);
+    }
 }
 
 template <int DT, int FMT, int RNG, int IDXB>
-__global__ void __launch_bounds__(kThreads) encode_kernel(const EncodeParams p)
+__global__ void __launch_bounds__(kThreads) encode_kernel(const __grid_constant__ EncodeParams p)
 {
     using E = Elem<DT>;
     using S = EncodeShape<DT>;
     constexpr bool MULTI = IDXB != 0;
+    constexpr int IB = MULTI ? IDXB : 8;
+    constexpr int H = 8 / E::G;                                  // 16-byte loads per unit
+    constexpr uint32_t BPU = RNG == 32 ? 2u : 1u;                // Philox blocks per unit
     const int m = blockIdx.x % p.M;
     const int64_t tile = blockIdx.x / p.M;
     const int64_t t0 = tile * S::TILE;
     const int64_t t1 = min(t0 + (int64_t)S::TILE, p.d);
-    const int tid = threadIdx.x;
-    const char *row = (const char *)p.g + (size_t)m * (size_t)p.stride * E::BYTES;
+    const int tid = threadIdx.x, lane = tid & 31;
 
-    // issue the gradient loads first; everything below overlaps with them
-    uint4 q[S::UNITS][8 / E::G];
-    uint64_t kbits[S::UNITS];
+    if (t1 - t0 != S::TILE) {                                    // the ragged last tile
+        encode_span_general<DT, FMT, RNG, IDXB>(p, m, t0, t1, tid, kThreads);
+        return;
+    }
+    // issue the loads of the full tile first; the segment lookup overlaps with them
+    const char *gp = (const char *)p.g + ((size_t)m * (size_t)p.stride + (size_t)t0 + (size_t)tid * 8) * E::BYTES;
+    const uint8_t *ip = MULTI ? p.idx + ((size_t)t0 + (size_t)tid * 8) * IB / 8 : nullptr;
+    uint4 q[S::UNITS][H];
+    typename IdxBits<IB>::T kbits[S::UNITS];
 #pragma unroll
     for (int u = 0; u < S::UNITS; ++u) {
-        const int64_t i = t0 + (int64_t)(u * kThreads + tid) * 8;
-        if (i < t1) {
 #pragma unroll
-            for (int h = 0; h < 8 / E::G; ++h) q[u][h] = ld_stream(row + (i + h * E::G) * E::BYTES);
-            kbits[u] = MULTI ? load_idx8<IDXB == 0 ? 8 : IDXB>(p.idx, i) : 0;
-        }
+        for (int h = 0; h < H; ++h) q[u][h] = ld_stream(gp + (u * kThreads * 8 + h * E::G) * E::BYTES);
+        if (MULTI) kbits[u] = IdxBits<IB>::load(ip + u * kThreads * IB);
     }
+    // every warp looks the segment up for itself (no shared memory, no barrier): once for the
+    // tile if one segment covers it, else once per 256-coordinate row of the warp.
+    // lane k holds s_k / W_j (single-scale: every lane holds s / W_j)
+    int j = warp_find_segment(p.seg_off, p.nseg, t0);
+    const bool tile_uniform = segment_end(p.seg_off, p.nseg, j, p.d) >= t1;
+    float inv_lane = inv_scale(p.scales.s[lane & (UQ_MAX_SCALES - 1)], __ldg(p.W + j));
+    bool overflow = not_finite(inv_lane);
 
-    // scale of this tile: uniform if one segment covers it (the common case)
-    __shared__ float sh_inv[UQ_MAX_SCALES];
-    const int j0 = find_segment(p.seg_off, p.nseg, t0);
-    const bool uniform = segment_end(p.seg_off, p.nseg, j0, p.d) >= t1;
-    if (tid < p.scales.N) {
-        const float inv = inv_scale(p.scales.s[tid], __ldg(p.W + j0));
-        sh_inv[tid] = inv;
-        if (uniform && (__float_as_uint(inv) & 0x7F800000u) == 0x7F800000u && p.status)
-            atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
-    }
-    __syncthreads();
-    const float inv_single = sh_inv[0];
-    const PhiloxKey key = philox_key(p.seed);
-
+    const uint64_t blk0 = RNG == 32 ? (uint64_t)(t0 >> 2) : (uint64_t)(t0 >> 3);           // low bits are 0
+    const uint32_t blk_hi = (uint32_t)(blk0 >> 32);
+    const uint32_t blk_lo = (uint32_t)blk0 + (uint32_t)tid * BPU;
+    char *lp = FMT == UQ_FMT_I8 ? (char *)p.lev + (size_t)m * (size_t)p.stride + (size_t)t0 + tid * 8
+                                : (char *)p.lev + (size_t)m * (size_t)(p.stride >> 1) + (size_t)(t0 >> 1) + tid * 4;
+    uint32_t crossed = 0;                                        // rows left to the general path
 #pragma unroll
     for (int u = 0; u < S::UNITS; ++u) {
-        const int64_t i = t0 + (int64_t)(u * kThreads + tid) * 8;
-        if (i >= t1) continue;
-        float v[8];
-#pragma unroll
-        for (int h = 0; h < 8 / E::G; ++h) E::unpack(q[u][h], *(float(*)[E::G])(v + h * E::G));
-        if (i + 8 > p.d) {
-#pragma unroll
-            for (int e = 0; e < 8; ++e)
-                if (i + e >= p.d) v[e] = 0.0f;      // padding quantizes to level 0
-        }
-
-        // per-coordinate s_i / W_j
-        float inv[8];
-        if (uniform) {
-#pragma unroll
-            for (int e = 0; e < 8; ++e)
-                inv[e] = MULTI ? sh_inv[(kbits[u] >> (e * IDXB)) & ((1u << IDXB) - 1u) & (UQ_MAX_SCALES - 1)]
-                               : inv_single;
-        } else {
-            int j = find_segment(p.seg_off, p.nseg, i);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                j = advance_segment(p.seg_off, p.nseg, j, i + e);
-                const int k = MULTI ? (int)((kbits[u] >> (e * IDXB)) & ((1u << IDXB) - 1u)) : 0;
-                inv[e] = inv_scale(p.scales.s[k & (UQ_MAX_SCALES - 1)], __ldg(p.W + j));
-                if ((__float_as_uint(inv[e]) & 0x7F800000u) == 0x7F800000u && p.status)
-                    atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
+        if (!tile_uniform) {                                     // warp-uniform branch
+            const int64_t r0 = t0 + (int64_t)(u * kThreads + (tid & ~31)) * 8;
+            j = warp_find_segment(p.seg_off, p.nseg, r0);
+            if (segment_end(p.seg_off, p.nseg, j, p.d) < r0 + 256) {
+                crossed |= 1u << u;
+                continue;
             }
+            inv_lane = inv_scale(p.scales.s[lane & (UQ_MAX_SCALES - 1)], __ldg(p.W + j));
+            overflow |= not_finite(inv_lane);
         }
-
-        // random words: coordinate c uses word c%4 of block c/4 (32-bit draws) or half
-        // (c%8)%2 of word (c%8)/2 of block c/8 (16-bit draws)
-        int z[8];
-        if (RNG == 32) {
-            const uint4 r0 = philox4x32_10(key, (uint64_t)(i >> 2), (uint32_t)m);
-            const uint4 r1 = philox4x32_10(key, (uint64_t)(i >> 2) + 1, (uint32_t)m);
-            const uint32_t w[8] = { r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w };
+        float v[8], inv[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e)
-                z[e] = apply_sign(v[e], level_draw23(scaled_magnitude(v[e], inv[e], p.cap), w[e]));
-        } else {
-            const uint4 r = philox4x32_10(key, (uint64_t)(i >> 3), (uint32_t)m);
-            const uint32_t w[4] = { r.x, r.y, r.z, r.w };
+        for (int h = 0; h < H; ++h) E::unpack(q[u][h], *(float(*)[E::G])(v + h * E::G));
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const uint32_t h16 = (e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu);
-                z[e] = apply_sign(v[e], level_draw16(scaled_magnitude(v[e], inv[e], p.cap), h16));
-            }
-        }
-
-        if (FMT == UQ_FMT_I8) {
-            uint2 out;
-            out.x = (z[0] & 0xFF) | ((z[1] & 0xFF) << 8) | ((z[2] & 0xFF) << 16) | ((uint32_t)z[3] << 24);
-            out.y = (z[4] & 0xFF) | ((z[5] & 0xFF) << 8) | ((z[6] & 0xFF) << 16) | ((uint32_t)z[7] << 24);
-            st_stream((uint2 *)((char *)p.lev + (size_t)m * (size_t)p.stride + i), out);
-        } else {
-            uint32_t out = 0;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) out |= (uint32_t)(z[e] & 0xF) << (4 * e);
-            st_stream((uint32_t *)((char *)p.lev + (size_t)m * (size_t)(p.stride >> 1) + (i >> 1)), out);
+        for (int e = 0; e < 8; ++e)
+            inv[e] = MULTI ? __shfl_sync(0xFFFFFFFFu, inv_lane, (int)((kbits[u] >> (e * IB)) & ((1u << IB) - 1u)))
+                           : inv_lane;
+        quantize_unit<FMT, RNG>(v, inv, p.cap, p.key, blk_lo + u * kThreads * BPU, blk_hi, (uint32_t)m,
+                                lp + u * kThreads * (FMT == UQ_FMT_I8 ? 8 : 4));
+    }
+    if (overflow && lane < p.scales.N && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
+    // rows crossed by a segment boundary, once the tile's registers are free
+    for (int u = 0; crossed != 0; ++u, crossed >>= 1) {
+        if (crossed & 1u) {
+            const int64_t r0 = t0 + (int64_t)(u * kThreads + (tid & ~31)) * 8;
+            encode_span_general<DT, FMT, RNG, IDXB>(p, m, r0, r0 + 256, lane, 32);
         }
     }
 }
@@ -189,7 +232,8 @@ cudaError_t launch_encode(const uq_layout &L, const void *g, const float *W, con
 {
     EncodeParams p;
     p.g = g; p.lev = lev; p.W = W; p.seg_off = L.seg_off; p.idx = idx; p.status = status;
-    p.d = L.d; p.stride = L.worker_stride; p.seed = seed; p.nseg = L.nseg; p.M = L.M;
+    p.d = L.d; p.stride = L.worker_stride; p.nseg = L.nseg; p.M = L.M;
+    p.key = philox_key(seed);
     p.cap = (float)scales.s[0];
     p.scales = scales;
     return L.dtype == UQ_F32 ? dispatch_fmt<UQ_F32>(p, fmt, rng_bits, idx_bits, st)

@@ -64,8 +64,8 @@ def test_seed_changes_the_draws_only():
     g = wl.generate(w)
     a = check_parity(w, g, seed=0)
     b = check_parity(w, g, seed=(1 << 40) + 12345)
-    assert (a["lev"] != b["lev"]).mean() > 0.2
-    assert np.abs(a["lev"].view(np.int8).astype(int) - b["lev"].view(np.int8)).max() <= 1
+    la, lb = a["lev"].view(np.int8)[:, : w.d].astype(int), b["lev"].view(np.int8)[:, : w.d].astype(int)
+    assert (la != lb).mean() > 0.2 and np.abs(la - lb).max() <= 1
 
 
 def test_full_level_range_and_saturation():
@@ -179,5 +179,8 @@ def test_reproducible_bit_for_bit():
     w = wl.scaled("c5", 200003)
     g = wl.generate(w)
     a, b = run_gpu(w, g), run_gpu(w, g)
-    for k in ("W", "lev", "idx", "S", "out"):
+    for k in ("W", "S", "out"):
         assert np.array_equal(a[k], b[k])
+    assert np.array_equal(a["lev"][:, : w.d], b["lev"][:, : w.d])          # padding is not data
+    nb = w.d * w.idx_bits // 8
+    assert np.array_equal(a["idx"][:nb], b["idx"][:nb])
