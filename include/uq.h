@@ -138,8 +138,9 @@ int uq_encode_single(const uq_layout *layout, const void *g, const float *W, int
  *   scales    host  N ascending integers >= 1, N <= UQ_MAX_SCALES; scales[0] is the smallest scale
  *   idx_bits  2 (N <= 4), 4 (N <= 16) or 8
  *   idx       out   packed little-endian within each byte (coordinate i at bit (i*idx_bits)%8
- *                   of byte (i*idx_bits)/8), uq_index_bytes(layout, idx_bits) bytes; bits
- *                   belonging to coordinates >= d are written as 0
+ *                   of byte (i*idx_bits)/8); the buffer holds uq_index_bytes(layout, idx_bits)
+ *                   bytes and is 16-byte aligned; the bits of coordinates d .. 8*ceil(d/8)-1
+ *                   are written as 0, later bytes are left untouched
  * Errors: UQ_ERR_BAD_ARG, UQ_ERR_CUDA.
  */
 int uq_select_scale_multi(const uq_layout *layout, const void *g, const float *W,
@@ -163,7 +164,7 @@ int uq_encode_multi(const uq_layout *layout, const void *g, const float *W, cons
  * Integer aggregation — Algorithm 1 / 2 line "AllReduce gradients" without the 1/M:
  *   S[i] = sum over workers of zeta^m_i, in int32.
  *   lev  in   level rows as written by the encoders (layout->dtype is ignored)
- *   S    out  [d] int32, 4-byte aligned
+ *   S    out  [d] int32, 32-byte aligned (no padding is required or written)
  * Errors: UQ_ERR_BAD_ARG, UQ_ERR_CUDA.
  */
 int uq_aggregate(const uq_layout *layout, const void *lev, int fmt, int32_t *S, void *stream);
@@ -177,7 +178,7 @@ int uq_aggregate(const uq_layout *layout, const void *lev, int fmt, int32_t *S, 
  *              reconstruction run fused in one kernel (the sums stay in registers);
  *              S_opt, if not NULL, also receives the int32 sums [d].
  *   src_kind = UQ_SRC_SUMS:   src is int32 S[d] (fmt and S_opt are ignored).
- *   out  [d] float, 4-byte aligned (no padding is required or written)
+ *   out  [d] float, 32-byte aligned (no padding is required or written); S_opt likewise
  * Errors: UQ_ERR_BAD_ARG, UQ_ERR_CUDA.
  */
 int uq_decode(const uq_layout *layout, const void *src, int src_kind, int fmt, const float *W, int s,

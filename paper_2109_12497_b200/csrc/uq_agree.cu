@@ -14,7 +14,8 @@ namespace uq {
 template <int NORM> struct Acc;
 template <> struct Acc<UQ_NORM_L2> {            // sum of exact binary64 squares
     double a = 0.0;
-    __device__ __forceinline__ void add(float v) { double x = (double)v; a = __dadd_rn(a, __dmul_rn(x, x)); }
+    // x*x is exact in binary64, so the fused multiply-add rounds once, exactly like add(a, x*x)
+    __device__ __forceinline__ void add(float v) { double x = (double)v; a = __fma_rn(x, x, a); }
     __device__ __forceinline__ void merge(double o) { a = __dadd_rn(a, o); }
     __device__ __forceinline__ double value() const { return a; }
 };
@@ -43,6 +44,7 @@ norm_partials_kernel(const void *__restrict__ g, int64_t d, int64_t stride, int 
                      const int64_t *__restrict__ seg_off, int64_t ntiles, double *__restrict__ part)
 {
     using E = Elem<DT>;
+    constexpr int UNITS = kNormTile / (kThreads * E::G);
     const int64_t tile = blockIdx.x;
     const int m = blockIdx.y;
     const int64_t t0 = tile * kNormTile;
@@ -51,25 +53,38 @@ norm_partials_kernel(const void *__restrict__ g, int64_t d, int64_t stride, int 
     double *prow = part + (size_t)m * (size_t)(ntiles + nseg);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    const int j0 = find_segment(seg_off, nseg, t0);
-    if (segment_end(seg_off, nseg, j0, d) >= t1) {
-        // the whole tile lies in segment j0: vector loads, one block reduction
-        constexpr int UNITS = kNormTile / (kThreads * E::G);
-        uint4 q[UNITS];
+    // The tile's vector loads (the row is padded, so a 16-byte load that starts before d is
+    // legal) are issued before the segment lookup when they fit few registers (bf16: 4 loads),
+    // after it otherwise (fp32: 8 loads; the lookup is two dependent loads for up to 1024
+    // segments, hidden by the other resident CTAs).
+    constexpr bool LOADS_FIRST = UNITS <= 4;
+    uint4 q[UNITS];
+    if (LOADS_FIRST) {
 #pragma unroll
         for (int u = 0; u < UNITS; ++u) {
-            int64_t i = t0 + (int64_t)(u * kThreads + tid) * E::G;
+            const int64_t i = t0 + (int64_t)(u * kThreads + tid) * E::G;
             q[u] = i < t1 ? ld_stream(row + i * E::BYTES) : make_uint4(0, 0, 0, 0);
+        }
+    }
+    const int j0 = warp_find_segment(seg_off, nseg, t0);
+    if (segment_end(seg_off, nseg, j0, d) >= t1) {
+        // the whole tile lies in segment j0: one block reduction in a fixed order
+        if (!LOADS_FIRST) {
+#pragma unroll
+            for (int u = 0; u < UNITS; ++u) {
+                const int64_t i = t0 + (int64_t)(u * kThreads + tid) * E::G;
+                q[u] = i < t1 ? ld_stream(row + i * E::BYTES) : make_uint4(0, 0, 0, 0);
+            }
         }
         Acc<NORM> acc;
 #pragma unroll
         for (int u = 0; u < UNITS; ++u) {
-            int64_t i = t0 + (int64_t)(u * kThreads + tid) * E::G;
+            const int64_t i = t0 + (int64_t)(u * kThreads + tid) * E::G;
             float v[E::G];
             E::unpack(q[u], v);
 #pragma unroll
             for (int e = 0; e < E::G; ++e)
-                if (i + e < t1) acc.add(v[e]);    // the row's padding beyond d is not data
+                if (i + e < t1) acc.add(v[e]);        // the row's padding beyond d is not data
         }
         __shared__ double sh[kWarps];
         double w = warp_reduce<NORM>(acc.value());

@@ -157,7 +157,7 @@ int uq_encode_multi(const uq_layout *L, const void *g, const float *W, const int
 int uq_aggregate(const uq_layout *L, const void *lev, int fmt, int32_t *S, void *stream)
 {
     if (!layout_ok(L) || (fmt != UQ_FMT_I8 && fmt != UQ_FMT_I4X2)) return UQ_ERR_BAD_ARG;
-    if (L->d > 0 && (lev == nullptr || S == nullptr || !aligned(lev, 16) || !aligned(S, 16)))
+    if (L->d > 0 && (lev == nullptr || S == nullptr || !aligned(lev, 16) || !aligned(S, 32)))
         return UQ_ERR_BAD_ARG;
     return finish(uq::launch_aggregate_decode(*L, lev, fmt, nullptr, single_scale(1), nullptr, 0, nullptr, S,
                                               (cudaStream_t)stream));
@@ -179,13 +179,13 @@ int uq_decode(const uq_layout *L, const void *src, int src_kind, int fmt, const 
         idx_bits = 0;
         idx = nullptr;
     }
-    if (L->d > 0 && (src == nullptr || out == nullptr || !aligned(src, 16) || !aligned(out, 16)))
+    if (L->d > 0 && (src == nullptr || out == nullptr || !aligned(src, 16) || !aligned(out, 32)))
         return UQ_ERR_BAD_ARG;
     if (src_kind == UQ_SRC_SUMS)
         return finish(uq::launch_decode_sums(*L, (const int32_t *)src, W, set, idx, idx_bits, out,
                                              (cudaStream_t)stream));
     if (fmt != UQ_FMT_I8 && fmt != UQ_FMT_I4X2) return UQ_ERR_BAD_ARG;
-    if (S_opt != nullptr && !aligned(S_opt, 16)) return UQ_ERR_BAD_ARG;
+    if (S_opt != nullptr && !aligned(S_opt, 32)) return UQ_ERR_BAD_ARG;
     return finish(uq::launch_aggregate_decode(*L, src, fmt, W, set, idx, idx_bits, out, S_opt,
                                               (cudaStream_t)stream));
 }

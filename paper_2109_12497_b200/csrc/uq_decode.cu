@@ -114,20 +114,23 @@ template <> struct Unit<UQ_FMT_I4X2> {
 };
 
 template <int FMT, int IDXB>
-__global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const DecodeParams p)
+__global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const __grid_constant__ DecodeParams p)
 {
     using U = Unit<FMT>;
     constexpr int C = U::C;
     constexpr bool MULTI = IDXB != 0;
-    constexpr int TILE = kThreads * C;
-    const int64_t t0 = (int64_t)blockIdx.x * TILE;
-    const int64_t t1 = min(t0 + (int64_t)TILE, p.d);
-    const int tid = threadIdx.x;
-    const int64_t i = t0 + (int64_t)tid * C;
+    constexpr int IB = MULTI ? IDXB : 8;
+    constexpr int WORDS = C * IB / 32;                              // idx words per thread
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int64_t i = ((int64_t)blockIdx.x * kThreads + tid) * C;  // my first coordinate
+    const int64_t row0 = i - (int64_t)lane * C;                    // my warp's first coordinate
+    if (row0 >= p.d) return;                                       // warp-uniform
+    const bool active = i < p.d;
     const size_t row_bytes = FMT == UQ_FMT_I8 ? (size_t)p.stride : (size_t)(p.stride >> 1);
 
     U unit;
-    if (i < t1) {
+    uint32_t kw[WORDS];
+    if (active) {
         const char *col = (const char *)p.lev + (size_t)i * 16 / C;
         int m = 0;
         for (; m + 8 <= p.M; m += 8) {          // eight workers' loads in flight
@@ -138,25 +141,21 @@ __global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const Decode
             for (int k = 0; k < 8; ++k) unit.add(q[k]);
         }
         for (; m < p.M; ++m) unit.add(ld_stream(col + (size_t)m * row_bytes));
+        if (MULTI && p.out != nullptr) {
+            // idx bits of coordinates i..i+C-1 start at byte i*IB/8 (a multiple of 4 bytes)
+            const uint32_t *ip = (const uint32_t *)(p.idx + (size_t)i * IB / 8);
+#pragma unroll
+            for (int w = 0; w < WORDS; ++w) kw[w] = __ldg(ip + w);
+        }
     }
-
-    // reconstruction factors of this tile's segment, one per scale
-    __shared__ float sh_c[UQ_MAX_SCALES];
-    const int j0 = find_segment(p.seg_off, p.nseg, t0);
-    const bool uniform = segment_end(p.seg_off, p.nseg, j0, p.d) >= t1;
-    if (p.out != nullptr && tid < p.scales.N) sh_c[tid] = decode_factor(__ldg(p.W + j0), p.scales.s[tid], p.M);
-    __syncthreads();
-    if (i >= t1) return;
 
     int s[C];
     unit.finish(p.M, s);
-
     const bool full = i + C <= p.d;
-    if (p.S != nullptr) {
+    if (p.S != nullptr && active) {
         if (full) {
 #pragma unroll
-            for (int e = 0; e < C; e += 4)
-                st_stream((int4 *)(p.S + i + e), make_int4(s[e], s[e + 1], s[e + 2], s[e + 3]));
+            for (int e = 0; e < C; e += 8) st_stream256(p.S + i + e, *(const uint32_t(*)[8])(s + e));
         } else {
             for (int e = 0; e < C; ++e)
                 if (i + e < p.d) p.S[i + e] = s[e];
@@ -164,39 +163,33 @@ __global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const Decode
     }
     if (p.out == nullptr) return;
 
+    // every warp looks up the segment of its own row of 32*C coordinates; lane k holds the
+    // reconstruction factor of scale k (single-scale: every lane holds the same factor)
+    const int64_t row1 = min(row0 + 32 * C, p.d);
+    const int j0 = warp_find_segment(p.seg_off, p.nseg, row0);
     float r[C];
-    if (uniform) {
-        if (MULTI) {
-            // idx bits of coordinates i..i+C-1 start at byte i*IDXB/8 (a multiple of 4 bytes)
-            constexpr int WORDS = C * (MULTI ? IDXB : 8) / 32;
-            uint32_t kw[WORDS];
-            const uint32_t *ip = (const uint32_t *)(p.idx + (size_t)i * IDXB / 8);
+    if (segment_end(p.seg_off, p.nseg, j0, p.d) >= row1) {
+        const float c_lane = decode_factor(__ldg(p.W + j0), p.scales.s[lane & (UQ_MAX_SCALES - 1)], p.M);
 #pragma unroll
-            for (int w = 0; w < WORDS; ++w) kw[w] = __ldg(ip + w);
-#pragma unroll
-            for (int e = 0; e < C; ++e) {
-                const int k = (kw[(e * IDXB) >> 5] >> ((e * IDXB) & 31)) & ((1 << IDXB) - 1);
-                r[e] = __fmul_rn((float)s[e], sh_c[k & (UQ_MAX_SCALES - 1)]);
-            }
-        } else {
-            const float c = sh_c[0];
-#pragma unroll
-            for (int e = 0; e < C; ++e) r[e] = __fmul_rn((float)s[e], c);
+        for (int e = 0; e < C; ++e) {
+            const int k = MULTI ? (kw[(e * IB) >> 5] >> ((e * IB) & 31)) & ((1 << IB) - 1) : 0;
+            const float c = MULTI ? __shfl_sync(0xFFFFFFFFu, c_lane, active ? k : 0) : c_lane;
+            r[e] = __fmul_rn((float)s[e], c);
         }
-    } else {
+    } else if (active) {
         int j = find_segment(p.seg_off, p.nseg, i);
         for (int e = 0; e < C; ++e) {
             r[e] = 0.0f;
             if (i + e >= p.d) continue;
             j = advance_segment(p.seg_off, p.nseg, j, i + e);
-            const int k = MULTI ? index_at<MULTI ? IDXB : 8>(p.idx, i + e) : 0;
+            const int k = MULTI ? index_at<IB>(p.idx, i + e) : 0;
             r[e] = __fmul_rn((float)s[e], decode_factor(__ldg(p.W + j), p.scales.s[k & (UQ_MAX_SCALES - 1)], p.M));
         }
     }
+    if (!active) return;
     if (full) {
 #pragma unroll
-        for (int e = 0; e < C; e += 4)
-            st_stream((float4 *)(p.out + i + e), make_float4(r[e], r[e + 1], r[e + 2], r[e + 3]));
+        for (int e = 0; e < C; e += 8) st_stream256(p.out + i + e, *(const uint32_t(*)[8])(r + e));
     } else {
         for (int e = 0; e < C; ++e)
             if (i + e < p.d) p.out[i + e] = r[e];

@@ -32,6 +32,27 @@ __device__ __forceinline__ uint4 ld_stream(const void *p)
 
 template <typename T> __device__ __forceinline__ void st_stream(T *p, T v) { __stcs(p, v); }
 
+// 256-bit streaming load / store (sm_100 and later): 32 bytes per lane in one instruction.
+// The address must be 32-byte aligned.
+struct alignas(32) uint8x { uint32_t w[8]; };
+
+__device__ __forceinline__ uint8x ld_stream256(const void *p)
+{
+    uint8x v;
+    asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]), "=r"(v.w[4]), "=r"(v.w[5]), "=r"(v.w[6]),
+                   "=r"(v.w[7])
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ void st_stream256(void *p, const uint32_t (&w)[8])
+{
+    asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 :: "l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                 : "memory");
+}
+
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
@@ -144,13 +165,13 @@ __device__ __forceinline__ uint32_t signed_level_draw23(float v, float x, uint32
 }
 constexpr uint32_t kLevelByte23 = 0;      // which byte of the returned word holds the level
 
-// 16-bit draw.  Returns a word whose byte 2 is the signed level (h16 = the 16-bit draw).
+// 16-bit draw.  Returns a word whose byte 2 is the signed level.
 // x + 128 rounds x to 16 fractional bits (ties to even): the mantissa of the sum is
-// floor(x) * 2^16 + rint(p * 2^16); adding 0xFFFF - h carries into bit 16 iff h < rint(p * 2^16).
-// 0xFFFF - sum = ~sum + 0x10000 negates byte 2 in two's complement.
-__device__ __forceinline__ uint32_t signed_level_draw16(float v, float x, uint32_t h16)
+// floor(x) * 2^16 + rint(p * 2^16); adding nh = 0xFFFF - h carries into bit 16 iff
+// h < rint(p * 2^16).  0xFFFF - sum = ~sum + 0x10000 negates byte 2 in two's complement.
+__device__ __forceinline__ uint32_t signed_level_draw16(float v, float x, uint32_t nh)
 {
-    uint32_t sum = __float_as_uint(__fadd_rn(x, 128.0f)) + 0xFFFFu - h16;
+    uint32_t sum = nh + __float_as_uint(__fadd_rn(x, 128.0f));
     if (v < 0.0f) sum = 0xFFFFu - sum;
     return sum;
 }

@@ -62,11 +62,11 @@ __device__ __forceinline__ void quantize_unit(const float (&v)[8], const float (
         for (int e = 0; e < 8; ++e) z[e] = signed_level_draw23(v[e], scaled_magnitude(v[e], inv[e], cap), w[e]);
     } else {
         const uint4 r = philox4x32_10(key, blk_lo, blk_hi, m);
-        const uint32_t w[4] = { r.x, r.y, r.z, r.w };
+        const uint32_t nw[4] = { ~r.x, ~r.y, ~r.z, ~r.w };       // 0xFFFF - h for both halves at once
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-            const uint32_t h16 = (e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu);
-            z[e] = signed_level_draw16(v[e], scaled_magnitude(v[e], inv[e], cap), h16);
+            const uint32_t nh = (e & 1) ? (nw[e >> 1] >> 16) : (nw[e >> 1] & 0xFFFFu);
+            z[e] = signed_level_draw16(v[e], scaled_magnitude(v[e], inv[e], cap), nh);
         }
     }
     if (FMT == UQ_FMT_I8) {
@@ -151,7 +151,8 @@ __global__ void __launch_bounds__(kThreads) encode_kernel(const __grid_constant_
     // lane k holds s_k / W_j (single-scale: every lane holds s / W_j)
     int j = warp_find_segment(p.seg_off, p.nseg, t0);
     const bool tile_uniform = segment_end(p.seg_off, p.nseg, j, p.d) >= t1;
-    float inv_lane = inv_scale(p.scales.s[lane & (UQ_MAX_SCALES - 1)], __ldg(p.W + j));
+    constexpr int KMASK = IB < 4 ? (1 << IB) - 1 : UQ_MAX_SCALES - 1;    // lane L holds scale L & KMASK
+    float inv_lane = inv_scale(p.scales.s[lane & KMASK], __ldg(p.W + j));
     bool overflow = not_finite(inv_lane);
 
     const uint64_t blk0 = RNG == 32 ? (uint64_t)(t0 >> 2) : (uint64_t)(t0 >> 3);           // low bits are 0
@@ -169,16 +170,17 @@ __global__ void __launch_bounds__(kThreads) encode_kernel(const __grid_constant_
                 crossed |= 1u << u;
                 continue;
             }
-            inv_lane = inv_scale(p.scales.s[lane & (UQ_MAX_SCALES - 1)], __ldg(p.W + j));
+            inv_lane = inv_scale(p.scales.s[lane & KMASK], __ldg(p.W + j));
             overflow |= not_finite(inv_lane);
         }
         float v[8], inv[8];
 #pragma unroll
         for (int h = 0; h < H; ++h) E::unpack(q[u][h], *(float(*)[E::G])(v + h * E::G));
+        // the shuffle reads its source lane modulo 32 and the table repeats every 2^IB lanes (an
+        // 8-bit index is below 16), so the index bits need a shift but no mask
 #pragma unroll
         for (int e = 0; e < 8; ++e)
-            inv[e] = MULTI ? __shfl_sync(0xFFFFFFFFu, inv_lane, (int)((kbits[u] >> (e * IB)) & ((1u << IB) - 1u)))
-                           : inv_lane;
+            inv[e] = MULTI ? __shfl_sync(0xFFFFFFFFu, inv_lane, (int)(uint32_t)(kbits[u] >> (e * IB))) : inv_lane;
         quantize_unit<FMT, RNG>(v, inv, p.cap, p.key, blk_lo + u * kThreads * BPU, blk_hi, (uint32_t)m,
                                 lp + u * kThreads * (FMT == UQ_FMT_I8 ? 8 : 4));
     }
