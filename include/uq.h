@@ -69,6 +69,7 @@ enum {
 
 #define UQ_MAX_WORKERS 64
 #define UQ_MAX_SCALES 16
+#define UQ_STATIC_SCRATCH_BYTES (4u << 20) /* scratch built into the library, see uq_agree_scale_static */
 
 typedef struct uq_layout {
     int64_t d;              /* coordinates per worker, >= 0 */
@@ -112,6 +113,37 @@ size_t uq_index_bytes(const uq_layout *layout, int idx_bits);
  */
 int uq_agree_scale(const uq_layout *layout, const void *g, int norm, float *W, uint32_t *status,
                    void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * uq_agree_scale for callers that may not allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of the call above, not a step of the method.)
+ *
+ * Who needs it: code that runs where allocation is off limits - a gradient hook invoked while
+ * the framework's device allocator must not be entered, a service whose device memory was
+ * budgeted and handed out at start-up, a plug-in that only receives the tensors it works on.
+ * Such a caller has nowhere to get the scratch buffer that uq_agree_scale asks for, so here
+ * the scratch is a fixed array of UQ_STATIC_SCRATCH_BYTES (4 MiB) inside the library image
+ * itself.  The cost: every GPU that loads the library carries those 4 MiB until the process
+ * exits, whether or not this call is used.
+ *
+ * Arguments, results and status bits are those of uq_agree_scale without workspace and
+ * workspace_bytes; W is bit-identical to what uq_agree_scale writes for the same input.
+ *   - Limit: uq_workspace_bytes(layout) must not exceed UQ_STATIC_SCRATCH_BYTES, i.e.
+ *     M * (ceil(d / 8192) + nseg) <= 524288 (M = 8 reaches d of about 5e8).  Larger layouts
+ *     return UQ_ERR_WORKSPACE and launch nothing; use uq_agree_scale with your own buffer.
+ *   - The call itself allocates nothing: no cudaMalloc, cudaFree or other allocating routine.
+ *   - The first call on each device looks up the array's device address (one
+ *     cudaGetSymbolAddress with that device current) and remembers it; later calls on that
+ *     device only launch.  Make that first call during set-up, before any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left
+ *     in it.  That is harmless here - every slot is written before it is read, nothing has to
+ *     start at zero - but two calls whose kernels overlap on the GPU (different streams, or
+ *     different host threads) race on it and produce garbage.  Keep them on one stream, or
+ *     order them with events.
+ * Errors: UQ_ERR_BAD_ARG, UQ_ERR_WORKSPACE (layout too large), UQ_ERR_CUDA.
+ */
+int uq_agree_scale_static(const uq_layout *layout, const void *g, int norm, float *W, uint32_t *status,
+                          void *stream);
 
 /*
  * Single-scale quantizer Q_s — Section "QSGDMaxNorm Quantization" (Eq. Q_s, definition of

@@ -25,7 +25,7 @@ UQ_STATUS_NONFINITE, UQ_STATUS_BAD_SEGMENTS, UQ_STATUS_SCALE_OVERFLOW = 1, 2, 4
 
 EXPORTS = (
     "uq_version", "uq_last_cuda_error", "uq_error_string", "uq_workspace_bytes", "uq_index_bytes",
-    "uq_agree_scale", "uq_encode_single", "uq_select_scale_multi", "uq_encode_multi",
+    "uq_agree_scale", "uq_agree_scale_static", "uq_encode_single", "uq_select_scale_multi", "uq_encode_multi",
     "uq_aggregate", "uq_decode",
 )
 
@@ -74,6 +74,7 @@ def lib() -> C.CDLL:
         L.uq_index_bytes.restype = SZ
         L.uq_index_bytes.argtypes = [LP, I]
         L.uq_agree_scale.argtypes = [LP, P, I, P, P, P, SZ, P]
+        L.uq_agree_scale_static.argtypes = [LP, P, I, P, P, P]
         L.uq_encode_single.argtypes = [LP, P, P, I, U64, I, I, P, P, P]
         L.uq_select_scale_multi.argtypes = [LP, P, P, P, I, I, P, P, P]
         L.uq_encode_multi.argtypes = [LP, P, P, P, I, P, I, U64, I, I, P, P, P]
@@ -162,6 +163,21 @@ def uq_agree_scale(layout: Layout, g: torch.Tensor, norm: int, W: torch.Tensor,
     _check("uq_agree_scale", lib().uq_agree_scale(
         layout.ref(), _ptr(g), norm, _ptr(W), _ptr(status), _ptr(workspace),
         workspace.numel() * workspace.element_size(), _stream()))
+
+
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def uq_agree_scale_static(layout: Layout, g: torch.Tensor, norm: int, W: torch.Tensor,
+                          status: Optional[torch.Tensor]) -> None:
+    """uq_agree_scale without a workspace argument, for callers that cannot allocate one: the
+    scratch is a 4 MiB array inside the library (layouts that need more raise UqError with
+    UQ_ERR_WORKSPACE).  Calls on one device share that array, so keep them on one stream; the
+    first call on a device does a one-time address lookup and belongs in set-up code."""
+    layout.check_g(g)
+    layout.check_vec(W, torch.float32, layout.nseg, "W")
+    _check("uq_agree_scale_static", lib().uq_agree_scale_static(
+        layout.ref(), _ptr(g), norm, _ptr(W), _ptr(status), _stream()))
 
 
 def uq_encode_single(layout: Layout, g: torch.Tensor, W: torch.Tensor, s: int, seed: int, rng_bits: int,

@@ -188,3 +188,53 @@ cudaError_t launch_agree_scale(const uq_layout &L, const void *g, int norm, floa
 }
 
 }  // namespace uq
+
+// ---------------------------------------------------------------------------------------------
+// uq_agree_scale_static: the same computation with the scratch held inside the library
+// ---------------------------------------------------------------------------------------------
+#include <mutex>
+
+namespace {
+
+// Scratch for the norm partials, part of the library image: every GPU that loads the library
+// holds these bytes until the process exits.  In host code this name is only a handle; the
+// device address comes from cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_static_scratch[UQ_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void *g_scratch_addr[kMaxDevices] = {};      // device address of g_static_scratch, per device ordinal
+
+// Device address of the scratch array on the current device, resolved once per device.
+cudaError_t static_scratch(void **out)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (g_scratch_addr[dev] == nullptr) {
+        void *addr = nullptr;
+        e = cudaGetSymbolAddress(&addr, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        if (addr == nullptr) return cudaErrorInvalidSymbol;
+        g_scratch_addr[dev] = addr;
+    }
+    *out = g_scratch_addr[dev];
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int uq_agree_scale_static(const uq_layout *layout, const void *g, int norm, float *W,
+                                     uint32_t *status, void *stream)
+{
+    // size first: a layout that cannot fit is refused before CUDA is touched
+    const size_t need = uq_workspace_bytes(layout);
+    if (need == 0) return UQ_ERR_BAD_ARG;                       // the layout itself is invalid
+    if (need > (size_t)UQ_STATIC_SCRATCH_BYTES) return UQ_ERR_WORKSPACE;
+    void *scratch = nullptr;
+    if (static_scratch(&scratch) != cudaSuccess) return UQ_ERR_CUDA;
+    // the partials are all written before they are read, so nothing in the array needs clearing
+    return uq_agree_scale(layout, g, norm, W, status, scratch, (size_t)UQ_STATIC_SCRATCH_BYTES, stream);
+}
