@@ -45,6 +45,8 @@ norm_partials_kernel(const void *__restrict__ g, int64_t d, int64_t stride, int 
 {
     using E = Elem<DT>;
     constexpr int UNITS = kNormTile / (kThreads * E::G);
+    // worker-major order (one worker's row is streamed front to back before the next worker's):
+    // consecutive CTAs read consecutive memory, and the kernel ends on the last worker's row
     const int64_t tile = blockIdx.x;
     const int m = blockIdx.y;
     const int64_t t0 = tile * kNormTile;
@@ -77,14 +79,25 @@ norm_partials_kernel(const void *__restrict__ g, int64_t d, int64_t stride, int 
             }
         }
         Acc<NORM> acc;
+        if (LOADS_FIRST && t1 - t0 == kNormTile) {    // full bf16 tile: no per-element bounds (for
+                                                      // fp32 the unguarded form costs 2.5x the registers)
 #pragma unroll
-        for (int u = 0; u < UNITS; ++u) {
-            const int64_t i = t0 + (int64_t)(u * kThreads + tid) * E::G;
-            float v[E::G];
-            E::unpack(q[u], v);
+            for (int u = 0; u < UNITS; ++u) {
+                float v[E::G];
+                E::unpack(q[u], v);
 #pragma unroll
-            for (int e = 0; e < E::G; ++e)
-                if (i + e < t1) acc.add(v[e]);        // the row's padding beyond d is not data
+                for (int e = 0; e < E::G; ++e) acc.add(v[e]);
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < UNITS; ++u) {
+                const int64_t i = t0 + (int64_t)(u * kThreads + tid) * E::G;
+                float v[E::G];
+                E::unpack(q[u], v);
+#pragma unroll
+                for (int e = 0; e < E::G; ++e)
+                    if (i + e < t1) acc.add(v[e]);    // the row's padding beyond d is not data
+            }
         }
         __shared__ double sh[kWarps];
         double w = warp_reduce<NORM>(acc.value());
@@ -164,6 +177,7 @@ static cudaError_t launch(const uq_layout &L, const void *g, float *W, uint32_t 
                           int64_t ntiles, cudaStream_t st)
 {
     if (L.d > 0) {
+        if (ntiles > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
         dim3 grid((unsigned)ntiles, (unsigned)L.M);
         norm_partials_kernel<DT, NORM><<<grid, kThreads, 0, st>>>(g, L.d, L.worker_stride, L.nseg,
                                                                  L.seg_off, ntiles, part);

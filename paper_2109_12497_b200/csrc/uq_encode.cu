@@ -19,6 +19,7 @@ struct EncodeParams {
     uint32_t *status;
     int64_t d, stride;
     int32_t nseg, M;
+    int64_t ntiles;
     float cap;                // (float) of the smallest scale: the largest level
     ScaleSet scales;          // single-scale: every entry is s
     PhiloxKey key;            // the ten round keys of the seed
@@ -125,8 +126,10 @@ __global__ void __launch_bounds__(kThreads) encode_kernel(const __grid_constant_
     constexpr int IB = MULTI ? IDXB : 8;
     constexpr int H = 8 / E::G;                                  // 16-byte loads per unit
     constexpr uint32_t BPU = RNG == 32 ? 2u : 1u;                // Philox blocks per unit
-    const int m = blockIdx.x % p.M;
-    const int64_t tile = blockIdx.x / p.M;
+    // CTAs walk the tiles back to front with the worker varying fastest (see launch_encode)
+    const uint32_t rev = gridDim.x - 1u - blockIdx.x;
+    const int m = (int)(rev % (uint32_t)p.M);
+    const int64_t tile = rev / (uint32_t)p.M;
     const int64_t t0 = tile * S::TILE;
     const int64_t t1 = min(t0 + (int64_t)S::TILE, p.d);
     const int tid = threadIdx.x, lane = tid & 31;
@@ -195,11 +198,11 @@ __global__ void __launch_bounds__(kThreads) encode_kernel(const __grid_constant_
 }
 
 template <int DT, int FMT, int RNG, int IDXB>
-static cudaError_t launch(const EncodeParams &p, cudaStream_t st)
+static cudaError_t launch(EncodeParams p, cudaStream_t st)
 {
     using S = EncodeShape<DT>;
-    const int64_t tiles = (p.d + S::TILE - 1) / S::TILE;
-    const int64_t blocks = tiles * p.M;
+    p.ntiles = (p.d + S::TILE - 1) / S::TILE;
+    const int64_t blocks = p.ntiles * p.M;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     encode_kernel<DT, FMT, RNG, IDXB><<<(unsigned)blocks, kThreads, 0, st>>>(p);
@@ -236,6 +239,12 @@ cudaError_t launch_encode(const uq_layout &L, const void *g, const float *W, con
     p.g = g; p.lev = lev; p.W = W; p.seg_off = L.seg_off; p.idx = idx; p.status = status;
     p.d = L.d; p.stride = L.worker_stride; p.nseg = L.nseg; p.M = L.M;
     p.key = philox_key(seed);
+    // CTA order (set in the kernel): the tiles are walked back to front with the worker varying fastest.  The
+    // kernel before this one in a step (agree-scale or the selector) ends on the high tiles, so
+    // part of what is read first is still in L2; all M workers of a tile run together, which
+    // keeps one copy of the shared index tile in L2 and spreads the streams over the memory
+    // channels (measured faster than walking worker by worker); and the kernel ends on the lowest
+    // tiles, where the aggregation starts.
     p.cap = (float)scales.s[0];
     p.scales = scales;
     return L.dtype == UQ_F32 ? dispatch_fmt<UQ_F32>(p, fmt, rng_bits, idx_bits, st)
