@@ -186,6 +186,28 @@ def time_end_to_end(q, g_host, out_host, g_dev, w, steps, warmup, barrier):
     return e0.elapsed_time(e1) / steps
 
 
+def time_encode_other_mode(q, g, w, reps):
+    """Mean ms of the encode kernel alone with the other random-draw width (context: the step
+    itself runs in the workload's own mode).  W and idx are those of the last step."""
+    import torch
+    st = torch.cuda.current_stream()
+    keep = q.rng_bits
+    q.rng_bits = 32 if keep == 16 else 16
+    try:
+        for _ in range(2):
+            q.encode(g, w.seed)
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+        torch.cuda.synchronize()
+        for k in range(reps):
+            evs[k].record(st)
+            q.encode(g, w.seed + k)
+        evs[reps].record(st)
+        torch.cuda.synchronize()
+        return evs[0].elapsed_time(evs[reps]) / reps
+    finally:
+        q.rng_bits = keep
+
+
 def l2_flush_buffer():
     import torch
     return torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
@@ -245,6 +267,7 @@ def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=F
         res["stages_cold_ms"] = {s: statistics.fmean(v) for s, v in per.items()}
         del flush
     res["ms"], res["stages_ms"] = time_device_resident(q, g_dev, w, steps, warmup, barrier)
+    res["encode_other_ms"] = time_encode_other_mode(q, g_dev, w, min(steps, 10))
     res["h2d"], res["d2h"], res["e2e_ms"] = 0, 0, None
     if want_e2e:
         out_host = torch.empty(w.d, dtype=torch.float32, pin_memory=True)
@@ -263,6 +286,11 @@ def summarize(res, peak_gbs):
         gbs = ab[s] / ms / 1e6
         out["kernels"][s] = {"ms": round(ms, 5), "algorithmic_MB": round(ab[s] / 1e6, 2),
                              "GBps": round(gbs, 1), "frac_of_hbm_peak": round(gbs / peak_gbs, 4)}
+    other = 32 if w.rng_bits == 16 else 16
+    ms = res["encode_other_ms"]
+    out["kernels"][f"encode_rng{other}"] = {
+        "ms": round(ms, 5), "algorithmic_MB": round(ab["encode"] / 1e6, 2), "GBps": round(ab["encode"] / ms / 1e6, 1),
+        "frac_of_hbm_peak": round(ab["encode"] / ms / 1e6 / peak_gbs, 4), "note": "timed alone, not part of the step"}
     if "ms_cold" in res:
         out["cold_l2"] = {"ms_per_step": res["ms_cold"], "gradient_GBps": w.in_bytes / res["ms_cold"] / 1e6,
                           "kernels_ms": {s: round(v, 5) for s, v in res["stages_cold_ms"].items()}}
@@ -302,6 +330,23 @@ def cpu_baseline(name, threads, max_coords):
             "sample": sample, "seconds": round(dt, 3)}
 
 
+def max_over_ranks(values, device):
+    """Element-wise max of a list of floats over all ranks (every rank gets the result).
+    Replicas do not exchange data; this is the only collective of a multi-GPU run."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return list(values)
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def whole_job_value(world, in_bytes, ms):
+    """Gradient GB/s of the whole job: every one of `world` replicas processed in_bytes in ms."""
+    return world * in_bytes / ms / 1e6
+
+
 def gpu_main(args):
     import torch
     import torch.distributed as dist
@@ -329,18 +374,14 @@ def gpu_main(args):
     res = bench_workload(w, args.steps, args.warmup, barrier, threads, want_e2e=not args.no_e2e)
     clocks = sampler.stop()
 
-    ms, e2e_ms = res["ms"], res["e2e_ms"] or float("nan")
-    if world > 1:
-        t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = float(t[0]), float(t[1])
+    ms, e2e_ms = max_over_ranks([res["ms"], res["e2e_ms"] or float("nan")], "cuda")
     summ = summarize(res, peak)
     q = res["q"]
-    dom = max(summ["kernels"], key=lambda s: summ["kernels"][s]["ms"])
+    dom = max(res["stages_ms"], key=lambda s: res["stages_ms"][s])
     ab = algorithmic_bytes(w)
     dom_gbs = ab[dom] / res["stages_ms"][dom] / 1e6
     line = {
-        "metric": METRIC, "value": round(world * w.in_bytes / ms / 1e6, 2), "unit": UNIT,
+        "metric": METRIC, "value": round(whole_job_value(world, w.in_bytes, ms), 2), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms, 5),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32" if w.dtype == wl.F32 else "bf16",
         "data": "synthetic",
@@ -353,7 +394,7 @@ def gpu_main(args):
             "status_word": res["status"],
         },
         "e2e": None if args.no_e2e else {
-            "value": round(world * w.in_bytes / e2e_ms / 1e6, 2), "unit": UNIT, "ms_per_step": round(e2e_ms, 4),
+            "value": round(whole_job_value(world, w.in_bytes, e2e_ms), 2), "unit": UNIT, "ms_per_step": round(e2e_ms, 4),
             "h2d_bytes_per_step": res["h2d"], "d2h_bytes_per_step": res["d2h"]},
         "gpu_launches": q.kernels_per_step() * args.steps,
         "clocks": clocks,
@@ -374,7 +415,8 @@ def gpu_main(args):
                 del res, q
                 torch.cuda.empty_cache()
                 small = wl.WORKLOADS[other].in_bytes < (126 << 20)
-                res = bench_workload(wl.WORKLOADS[other], max(3, min(args.steps, 10)), 3, lambda: None, threads,
+                res = bench_workload(resolve_workload(other, None, args.rng_bits), max(3, min(args.steps, 10)), 3,
+                                     lambda: None, threads,
                                      want_e2e=False, flush_between=small)
                 q = res["q"]
                 extra[other] = summarize(res, peak)

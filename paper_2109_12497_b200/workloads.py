@@ -17,6 +17,9 @@ and layer structure are stated recipes:
   c5  multi-scale, M=8, d=335,141,888 bf16, N(0, 0.02^2) with 1% of the coordinates x100
       (same coordinates on every worker), 25 MiB buckets, scale set {127 * 8^k, k<8}, 4-bit index
 
+All five use 16-bit random draws per coordinate (``rng_bits``), the mode in which the encoder
+is bandwidth-bound; 32-bit draws are the other supported mode and are tested and timed as well.
+
 ``scaled(name, d)`` gives the same recipe at a smaller d for tests.
 """
 from __future__ import annotations
@@ -48,7 +51,7 @@ class Workload:
     norm: str
     seed: int                 # seed of the quantizer's random draws
     data_seed: int
-    rng_bits: int = 32
+    rng_bits: int = 16        # width of the random draw per coordinate (16 or 32 Philox bits)
     nseg_hint: int = 1
     bucket_elems: int = 0
 

@@ -2,6 +2,7 @@
 times.  c1-c3 are compared in full; c4 and c5 on the complete scale vector plus windows of
 coordinates (first, last with the ragged tail, bucket boundaries, random offsets) where every
 level, index, sum and reconstructed value is compared with the oracle."""
+import dataclasses
 import os
 
 import numpy as np
@@ -23,9 +24,9 @@ def _oracle_threads():
     o.set_threads(1)
 
 
-@pytest.mark.parametrize("name", ["c1", "c2", "c3"])
-def test_full_workload(name):
-    w = wl.WORKLOADS[name]
+@pytest.mark.parametrize("name,rng_bits", [("c1", 16), ("c1", 32), ("c2", 16), ("c2", 32), ("c3", 16)])
+def test_full_workload(name, rng_bits):
+    w = dataclasses.replace(wl.WORKLOADS[name], rng_bits=rng_bits)
     r = check_parity(w, wl.generate(w))
     lev = r["ref"]["lev_raw"]
     assert np.abs(lev.astype(int)).max() <= w.s
