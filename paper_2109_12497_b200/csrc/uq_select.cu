@@ -32,79 +32,159 @@ __device__ __forceinline__ float inv_scale_sel(int32_t s, float W)
     return W > 0.0f ? __fdiv_rn((float)s, W) : 0.0f;
 }
 
-template <int DT, int IDXB>
-__global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p)
+// Largest non-negative binary32 bit pattern t with fl(t * inv) <= s_hat, or -1 if not even 0
+// passes.  fl(t * inv) is non-decreasing in t, so "passes" is a prefix of the magnitudes and the
+// test |v| * inv <= s_hat is the integer compare bits(|v|) <= t.  The quotient s_hat / inv lands
+// within a few units of the answer; the two bounded loops settle it exactly.
+__device__ __forceinline__ int32_t pass_threshold(float inv, float s_hat)
+{
+    if (!(inv > 0.0f)) return inv == 0.0f ? 0x7F7FFFFF : -1;       // W = 0: every finite value passes
+    if (!(__fmul_rn(0.0f, inv) <= s_hat)) return -1;                // inv = Inf: 0 * Inf is NaN
+    int32_t b = __float_as_int(fminf(__fdiv_rn(s_hat, inv), 3.402823466e38f));
+    for (int it = 0; it < 64 && b < 0x7F7FFFFF && __fmul_rn(__int_as_float(b + 1), inv) <= s_hat; ++it) ++b;
+    for (int it = 0; it < 64 && b >= 0 && !(__fmul_rn(__int_as_float(b), inv) <= s_hat); ++it) --b;
+    return b;
+}
+
+// The general path for one thread's 8 coordinates (row crossed by a segment boundary): the test
+// is evaluated as written, with one division per scale and coordinate.  Rare, kept out of line.
+__device__ __noinline__ uint64_t select_general(const SelectParams &p, int64_t i, const uint32_t (&amag)[8], int idxb)
+{
+    uint64_t packed = 0;
+    int j = find_segment(p.seg_off, p.nseg, i);
+    for (int e = 0; e < 8; ++e) {
+        int k = 0;
+        if (i + e < p.d) {                                          // padding keeps index 0
+            j = advance_segment(p.seg_off, p.nseg, j, i + e);
+            const float Wj = __ldg(p.W + j), a = __uint_as_float(amag[e]);
+            for (int kk = 1; kk < p.scales.N; ++kk)
+                if (__fmul_rn(a, inv_scale_sel(p.scales.s[kk], Wj)) <= p.s_hat) k = kk;
+        }
+        packed |= (uint64_t)k << (e * idxb);
+    }
+    return packed;
+}
+
+// LEVELS = ceil(log2 N): the per-coordinate search is a bisection over the N thresholds.
+template <int DT, int IDXB, int LEVELS>
+__global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant__ SelectParams p)
 {
     using E = Elem<DT>;
-    const int64_t t0 = (int64_t)blockIdx.x * kSelectTile;
-    const int64_t t1 = min(t0 + (int64_t)kSelectTile, p.d);
-    const int tid = threadIdx.x;
-    const int64_t i = t0 + (int64_t)tid * 8;
-    const int N = p.scales.N;
+    constexpr int H = 8 / E::G;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t i = ((int64_t)blockIdx.x * kThreads + tid) * 8;   // my first coordinate
+    const int64_t row0 = i - (int64_t)lane * 8;                     // my warp's first coordinate
+    if (row0 >= p.d) return;                                        // warp-uniform
+    const bool active = i < p.d;
 
-    float amax[8];
+    // max over the workers of the magnitude bits (bf16: two coordinates per word)
+    uint32_t amag[8];
+    if (DT == UQ_F32) {
+        float amax[8];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) amax[e] = 0.0f;
-    if (i < t1) {
-        const char *col = (const char *)p.g + (size_t)i * E::BYTES;
-        int m = 0;
-        // four workers' loads in flight at a time
-        for (; m + 4 <= p.M; m += 4) {
-            uint4 q[4][8 / E::G];
+        for (int e = 0; e < 8; ++e) amax[e] = 0.0f;
+        if (active) {
+            const char *col = (const char *)p.g + (size_t)i * E::BYTES;
+            int m = 0;
+            for (; m + 4 <= p.M; m += 4) {                          // four workers' loads in flight
+                uint4 q[4][H];
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
+                for (int k = 0; k < 4; ++k)
 #pragma unroll
-                for (int h = 0; h < 8 / E::G; ++h)
-                    q[k][h] = ld_stream(col + ((size_t)(m + k) * (size_t)p.stride + h * E::G) * E::BYTES);
+                    for (int h = 0; h < H; ++h)
+                        q[k][h] = ld_stream(col + ((size_t)(m + k) * (size_t)p.stride + h * E::G) * E::BYTES);
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
+                for (int k = 0; k < 4; ++k) {
+                    float v[8];
+#pragma unroll
+                    for (int h = 0; h < H; ++h) E::unpack(q[k][h], *(float(*)[E::G])(v + h * E::G));
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) amax[e] = fmaxf(amax[e], fabsf(v[e]));
+                }
+            }
+            for (; m < p.M; ++m) {
                 float v[8];
 #pragma unroll
-                for (int h = 0; h < 8 / E::G; ++h) E::unpack(q[k][h], *(float(*)[E::G])(v + h * E::G));
+                for (int h = 0; h < H; ++h)
+                    E::unpack(ld_stream(col + ((size_t)m * (size_t)p.stride + h * E::G) * E::BYTES),
+                              *(float(*)[E::G])(v + h * E::G));
 #pragma unroll
                 for (int e = 0; e < 8; ++e) amax[e] = fmaxf(amax[e], fabsf(v[e]));
             }
         }
-        for (; m < p.M; ++m) {
-            float v[8];
 #pragma unroll
-            for (int h = 0; h < 8 / E::G; ++h) {
-                uint4 q = ld_stream(col + ((size_t)m * (size_t)p.stride + h * E::G) * E::BYTES);
-                E::unpack(q, *(float(*)[E::G])(v + h * E::G));
+        for (int e = 0; e < 8; ++e) amag[e] = __float_as_uint(amax[e]);
+    } else {
+        // bf16 magnitudes order like unsigned 15-bit integers: packed 16-bit max, no unpacking
+        uint32_t am[4] = {0u, 0u, 0u, 0u};
+        if (active) {
+            const char *col = (const char *)p.g + (size_t)i * E::BYTES;
+            int m = 0;
+            for (; m + 8 <= p.M; m += 8) {                          // eight workers' loads in flight
+                uint4 q[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) q[k] = ld_stream(col + (size_t)(m + k) * (size_t)p.stride * E::BYTES);
+#pragma unroll
+                for (int k = 0; k < 8; k += 2) {
+                    am[0] = __vimax3_u16x2(am[0], q[k].x & 0x7FFF7FFFu, q[k + 1].x & 0x7FFF7FFFu);
+                    am[1] = __vimax3_u16x2(am[1], q[k].y & 0x7FFF7FFFu, q[k + 1].y & 0x7FFF7FFFu);
+                    am[2] = __vimax3_u16x2(am[2], q[k].z & 0x7FFF7FFFu, q[k + 1].z & 0x7FFF7FFFu);
+                    am[3] = __vimax3_u16x2(am[3], q[k].w & 0x7FFF7FFFu, q[k + 1].w & 0x7FFF7FFFu);
+                }
             }
-#pragma unroll
-            for (int e = 0; e < 8; ++e) amax[e] = fmaxf(amax[e], fabsf(v[e]));
+            for (; m < p.M; ++m) {
+                const uint4 q = ld_stream(col + (size_t)m * (size_t)p.stride * E::BYTES);
+                am[0] = __vmaxu2(am[0], q.x & 0x7FFF7FFFu);
+                am[1] = __vmaxu2(am[1], q.y & 0x7FFF7FFFu);
+                am[2] = __vmaxu2(am[2], q.z & 0x7FFF7FFFu);
+                am[3] = __vmaxu2(am[3], q.w & 0x7FFF7FFFu);
+            }
         }
+#pragma unroll
+        for (int w = 0; w < 4; ++w) { amag[2 * w] = am[w] << 16; amag[2 * w + 1] = am[w] & 0xFFFF0000u; }
     }
 
-    __shared__ float sh_inv[UQ_MAX_SCALES];
-    const int j0 = find_segment(p.seg_off, p.nseg, t0);
-    const bool uniform = segment_end(p.seg_off, p.nseg, j0, p.d) >= t1;
-    if (tid < N) sh_inv[tid] = inv_scale_sel(p.scales.s[tid], __ldg(p.W + j0));
-    __syncthreads();
-    if (i >= t1) return;
-
+    // every warp looks up the segment of its own row of 256 coordinates and builds the threshold
+    // table of that segment in its own slice of shared memory: entry k is the largest magnitude
+    // that passes scale k, -1 beyond the last scale
+    __shared__ int32_t sh_thr[kWarps][2 * UQ_MAX_SCALES];
+    const int64_t row1 = min(row0 + 256, p.d);
+    const int j0 = warp_find_segment(p.seg_off, p.nseg, row0);
     uint64_t packed = 0;
-    int j = uniform ? j0 : find_segment(p.seg_off, p.nseg, i);
+    if (segment_end(p.seg_off, p.nseg, j0, p.d) >= row1) {
+        int32_t thr = -1;
+        if (lane < p.scales.N) thr = pass_threshold(inv_scale_sel(p.scales.s[lane], __ldg(p.W + j0)), p.s_hat);
+        sh_thr[warp][lane] = thr;
+        __syncwarp();
+        const int32_t *T = sh_thr[warp];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        int k = 0;
-        if (i + e < p.d) {                          // padding keeps index 0
-            if (uniform) {
-                for (int kk = 1; kk < N; ++kk)
-                    if (__fmul_rn(amax[e], sh_inv[kk]) <= p.s_hat) k = kk;
-            } else {
-                j = advance_segment(p.seg_off, p.nseg, j, i + e);
-                const float Wj = __ldg(p.W + j);
-                for (int kk = 1; kk < N; ++kk)
-                    if (__fmul_rn(amax[e], inv_scale_sel(p.scales.s[kk], Wj)) <= p.s_hat) k = kk;
-            }
+        for (int e = 0; e < 8; ++e) {
+            const int32_t a = (int32_t)amag[e];
+            int k = 0;
+#pragma unroll
+            for (int step = 1 << (LEVELS - 1); step >= 1; step >>= 1)
+                if (a <= T[k + step]) k += step;                    // k + step < 2^LEVELS <= 16
+            if (i + e >= p.d) k = 0;                                // padding keeps index 0
+            packed |= (uint64_t)k << (e * IDXB);
         }
-        packed |= (uint64_t)k << (e * IDXB);
+    } else if (active) {
+        packed = select_general(p, i, amag, IDXB);
     }
+    if (!active) return;
     if (IDXB == 2) *(uint16_t *)(p.idx + (i >> 2)) = (uint16_t)packed;
     else if (IDXB == 4) *(uint32_t *)(p.idx + (i >> 1)) = (uint32_t)packed;
     else *(uint64_t *)(p.idx + i) = packed;
+}
+
+template <int DT, int IDXB>
+static cudaError_t dispatch_levels(const SelectParams &p, unsigned blocks, cudaStream_t st)
+{
+    const int N = p.scales.N;
+    if (N <= 2) select_kernel<DT, IDXB, 1><<<blocks, kThreads, 0, st>>>(p);
+    else if (N <= 4) select_kernel<DT, IDXB, 2><<<blocks, kThreads, 0, st>>>(p);
+    else if (N <= 8) select_kernel<DT, IDXB, 3><<<blocks, kThreads, 0, st>>>(p);
+    else select_kernel<DT, IDXB, 4><<<blocks, kThreads, 0, st>>>(p);
+    return cudaGetLastError();
 }
 
 template <int DT>
@@ -113,10 +193,9 @@ static cudaError_t dispatch(const SelectParams &p, int idx_bits, cudaStream_t st
     const int64_t blocks = (p.d + kSelectTile - 1) / kSelectTile;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
-    if (idx_bits == 2) select_kernel<DT, 2><<<(unsigned)blocks, kThreads, 0, st>>>(p);
-    else if (idx_bits == 4) select_kernel<DT, 4><<<(unsigned)blocks, kThreads, 0, st>>>(p);
-    else select_kernel<DT, 8><<<(unsigned)blocks, kThreads, 0, st>>>(p);
-    return cudaGetLastError();
+    if (idx_bits == 2) return dispatch_levels<DT, 2>(p, (unsigned)blocks, st);
+    if (idx_bits == 4) return dispatch_levels<DT, 4>(p, (unsigned)blocks, st);
+    return dispatch_levels<DT, 8>(p, (unsigned)blocks, st);
 }
 
 cudaError_t launch_select(const uq_layout &L, const void *g, const float *W, const ScaleSet &scales,
