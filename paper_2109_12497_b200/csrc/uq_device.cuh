@@ -148,32 +148,28 @@ __device__ __forceinline__ float scaled_magnitude(float v, float inv, float cap)
     return fminf(__fmul_rn(fabsf(v), inv), cap);
 }
 
-// 23-bit draw.  Returns a word whose LOW byte is the signed level
-//   zeta = sign(v) * (floor(x) + [h < rint((x - floor(x)) * 2^23)]),  h = word >> 9,  0 <= x <= 127.
+// 23-bit draw.  Returns a word whose LOW byte is the unsigned level
+//   floor(x) + [h < rint((x - floor(x)) * 2^23)],  h = word >> 9,  0 <= x <= 127.
 // t = x + 2^23 rounded down holds floor(x) in its low mantissa bits; t - (2^23 + 1) = floor(x) - 1
 // exactly, so x - that is p + 1 with one rounding: its mantissa is rint(p * 2^23), and the carry
 // into the exponent makes it 2^23 when p rounds up to 1.  The draw is placed under the same
 // exponent by one funnel shift, so the test is a single unsigned compare.
-__device__ __forceinline__ uint32_t signed_level_draw23(float v, float x, uint32_t word)
+__device__ __forceinline__ uint32_t level_draw23(float x, uint32_t word)
 {
     const float t = __fadd_rd(x, 8388608.0f);
     const float p1 = __fsub_rn(x, __fsub_rn(t, 8388609.0f));
     const uint32_t hb = __funnelshift_r(word, 0x7Fu, 9);          // 0x3F800000 | (word >> 9)
-    uint32_t lv = __float_as_uint(t) + (hb < __float_as_uint(p1) ? 1u : 0u);
-    if (v < 0.0f) lv = 0u - lv;                                   // low byte: two's complement
-    return lv;
+    return __float_as_uint(t) + (hb < __float_as_uint(p1) ? 1u : 0u);
 }
 constexpr uint32_t kLevelByte23 = 0;      // which byte of the returned word holds the level
 
-// 16-bit draw.  Returns a word whose byte 2 is the signed level.
+// 16-bit draw.  Returns a word whose byte 2 is the unsigned level.
 // x + 128 rounds x to 16 fractional bits (ties to even): the mantissa of the sum is
 // floor(x) * 2^16 + rint(p * 2^16); adding nh = 0xFFFF - h carries into bit 16 iff
-// h < rint(p * 2^16).  0xFFFF - sum = ~sum + 0x10000 negates byte 2 in two's complement.
-__device__ __forceinline__ uint32_t signed_level_draw16(float v, float x, uint32_t nh)
+// h < rint(p * 2^16).
+__device__ __forceinline__ uint32_t level_draw16(float x, uint32_t nh)
 {
-    uint32_t sum = nh + __float_as_uint(__fadd_rn(x, 128.0f));
-    if (v < 0.0f) sum = 0xFFFFu - sum;
-    return sum;
+    return nh + __float_as_uint(__fadd_rn(x, 128.0f));
 }
 constexpr uint32_t kLevelByte16 = 2;
 
@@ -182,6 +178,45 @@ template <uint32_t B> __device__ __forceinline__ uint32_t gather_bytes(uint32_t 
 {
     constexpr uint32_t sel = B | ((B + 4) << 4);
     return __byte_perm(__byte_perm(a, b, sel), __byte_perm(c, d, sel), 0x5410);
+}
+
+// Byte permute with the full selector: a selector nibble with bit 3 set replicates the top bit of
+// the selected byte over the whole result byte (the __byte_perm intrinsic keeps only 3 bits).
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+// Byte masks (0xFF where negative) of four binary32 values / of the four bf16 values in two words.
+__device__ __forceinline__ uint32_t sign_bytes_f32(float a, float b, float c, float d)
+{
+    const uint32_t lo = prmt(__float_as_uint(a), __float_as_uint(b), 0x00FBu);   // sign of bytes 3 and 7
+    const uint32_t hi = prmt(__float_as_uint(c), __float_as_uint(d), 0x00FBu);
+    return __byte_perm(lo, hi, 0x5410);
+}
+__device__ __forceinline__ uint32_t sign_bytes_bf16(uint32_t w01, uint32_t w23)
+{
+    return prmt(w01, w23, 0xFDB9u);                                              // sign of bytes 1, 3, 5, 7
+}
+
+// Four levels 0..127 in the bytes of `mag`; bytes selected by `neg` (0xFF / 0x00) are negated
+// in two's complement.  0x80 - L never borrows from the next byte (L <= 127), and flipping the
+// top bit turns it into 0x100 - L for L > 0 and into 0 for L = 0.
+__device__ __forceinline__ uint32_t negate_bytes(uint32_t mag, uint32_t neg)
+{
+    const uint32_t minus = (0x80808080u - mag) ^ 0x80808080u;
+    return (mag & ~neg) | (minus & neg);
+}
+
+// The low nibbles of the eight bytes of (lo, hi), packed into 32 bits (byte k -> nibble k).
+__device__ __forceinline__ uint32_t bytes_to_nibbles(uint32_t lo, uint32_t hi)
+{
+    lo &= 0x0F0F0F0Fu; hi &= 0x0F0F0F0Fu;
+    lo = (lo | (lo >> 4)) & 0x00FF00FFu; hi = (hi | (hi >> 4)) & 0x00FF00FFu;
+    lo = (lo | (lo >> 8)) & 0x0000FFFFu; hi = (hi | (hi >> 8)) & 0x0000FFFFu;
+    return lo | (hi << 16);
 }
 
 // ---------------------------------------------------------------------------------------------

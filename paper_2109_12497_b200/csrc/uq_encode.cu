@@ -45,13 +45,14 @@ template <> struct IdxBits<4> { using T = uint32_t; static __device__ __forceinl
 template <> struct IdxBits<8> { using T = uint64_t; static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg((const unsigned long long *)p); } };
 
 // Eight coordinates: magnitudes scaled by inv[e], random words from the block(s) starting at
-// (blk_lo, blk_hi), signed levels packed into the wire format and stored at `dst`.
+// (blk_lo, blk_hi), levels gathered four to a word, signs applied bytewise (`neg` holds 0xFF in
+// the bytes of negative coordinates), packed into the wire format and stored at `dst`.
 // coordinate c uses word c%4 of block c/4 (32-bit draws) or half (c%8)%2 of word (c%8)/2 of block
 // c/8 (16-bit draws).
 template <int FMT, int RNG>
 __device__ __forceinline__ void quantize_unit(const float (&v)[8], const float (&inv)[8], float cap,
-                                              const PhiloxKey &key, uint32_t blk_lo, uint32_t blk_hi, uint32_t m,
-                                              void *dst)
+                                              uint32_t neg_lo, uint32_t neg_hi, const PhiloxKey &key,
+                                              uint32_t blk_lo, uint32_t blk_hi, uint32_t m, void *dst)
 {
     constexpr uint32_t LB = RNG == 32 ? kLevelByte23 : kLevelByte16;
     uint32_t z[8];
@@ -60,26 +61,33 @@ __device__ __forceinline__ void quantize_unit(const float (&v)[8], const float (
         const uint4 r1 = philox4x32_10(key, blk_lo + 1u, blk_hi, m);      // blk_lo is even: no carry
         const uint32_t w[8] = { r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w };
 #pragma unroll
-        for (int e = 0; e < 8; ++e) z[e] = signed_level_draw23(v[e], scaled_magnitude(v[e], inv[e], cap), w[e]);
+        for (int e = 0; e < 8; ++e) z[e] = level_draw23(scaled_magnitude(v[e], inv[e], cap), w[e]);
     } else {
         const uint4 r = philox4x32_10(key, blk_lo, blk_hi, m);
         const uint32_t nw[4] = { ~r.x, ~r.y, ~r.z, ~r.w };       // 0xFFFF - h for both halves at once
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
             const uint32_t nh = (e & 1) ? (nw[e >> 1] >> 16) : (nw[e >> 1] & 0xFFFFu);
-            z[e] = signed_level_draw16(v[e], scaled_magnitude(v[e], inv[e], cap), nh);
+            z[e] = level_draw16(scaled_magnitude(v[e], inv[e], cap), nh);
         }
     }
-    if (FMT == UQ_FMT_I8) {
-        uint2 out;
-        out.x = gather_bytes<LB>(z[0], z[1], z[2], z[3]);
-        out.y = gather_bytes<LB>(z[4], z[5], z[6], z[7]);
-        st_stream((uint2 *)dst, out);
+    const uint32_t lo = negate_bytes(gather_bytes<LB>(z[0], z[1], z[2], z[3]), neg_lo);
+    const uint32_t hi = negate_bytes(gather_bytes<LB>(z[4], z[5], z[6], z[7]), neg_hi);
+    if (FMT == UQ_FMT_I8) st_stream((uint2 *)dst, make_uint2(lo, hi));
+    else st_stream((uint32_t *)dst, bytes_to_nibbles(lo, hi));
+}
+
+// The sign masks of a unit, from the raw loaded words (before any padding is zeroed).
+template <int DT> __device__ __forceinline__ void unit_signs(const uint4 *q, uint32_t &neg_lo, uint32_t &neg_hi)
+{
+    if (DT == UQ_F32) {
+        neg_lo = sign_bytes_f32(__uint_as_float(q[0].x), __uint_as_float(q[0].y), __uint_as_float(q[0].z),
+                                __uint_as_float(q[0].w));
+        neg_hi = sign_bytes_f32(__uint_as_float(q[1].x), __uint_as_float(q[1].y), __uint_as_float(q[1].z),
+                                __uint_as_float(q[1].w));
     } else {
-        uint32_t out = 0;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) out |= ((z[e] >> (8 * LB)) & 0xFu) << (4 * e);
-        st_stream((uint32_t *)dst, out);
+        neg_lo = sign_bytes_bf16(q[0].x, q[0].y);
+        neg_hi = sign_bytes_bf16(q[0].z, q[0].w);
     }
 }
 
@@ -95,9 +103,14 @@ __device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, i
     const char *row = (const char *)p.g + (size_t)m * (size_t)p.stride * E::BYTES;
     for (int64_t i = a + (int64_t)who * 8; i < b; i += (int64_t)many * 8) {
         float v[8];
+        uint4 q[8 / E::G];
 #pragma unroll
-        for (int h = 0; h < 8 / E::G; ++h)
-            E::unpack(ld_stream(row + (i + h * E::G) * E::BYTES), *(float(*)[E::G])(v + h * E::G));
+        for (int h = 0; h < 8 / E::G; ++h) {
+            q[h] = ld_stream(row + (i + h * E::G) * E::BYTES);
+            E::unpack(q[h], *(float(*)[E::G])(v + h * E::G));
+        }
+        uint32_t neg_lo, neg_hi;
+        unit_signs<DT>(q, neg_lo, neg_hi);          // the sign of a padding coordinate is harmless: its level is 0
         typename IdxBits<IB>::T kbits = 0;
         if (MULTI) kbits = IdxBits<IB>::load(p.idx + i * IB / 8);
         float inv[8];
@@ -113,7 +126,8 @@ __device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, i
         const uint64_t blk = RNG == 32 ? (uint64_t)(i >> 2) : (uint64_t)(i >> 3);
         char *dst = FMT == UQ_FMT_I8 ? (char *)p.lev + (size_t)m * (size_t)p.stride + i
                                      : (char *)p.lev + (size_t)m * (size_t)(p.stride >> 1) + (i >> 1);
-        quantize_unit<FMT, RNG>(v, inv, p.cap, p.key, (uint32_t)blk, (uint32_t)(blk >> 32), (uint32_t)m, dst);
+        quantize_unit<FMT, RNG>(v, inv, p.cap, neg_lo, neg_hi, p.key, (uint32_t)blk, (uint32_t)(blk >> 32), (uint32_t)m,
+                                dst);
     }
 }
 
@@ -184,7 +198,9 @@ __global__ void __launch_bounds__(kThreads) encode_kernel(const __grid_constant_
 #pragma unroll
         for (int e = 0; e < 8; ++e)
             inv[e] = MULTI ? __shfl_sync(0xFFFFFFFFu, inv_lane, (int)(uint32_t)(kbits[u] >> (e * IB))) : inv_lane;
-        quantize_unit<FMT, RNG>(v, inv, p.cap, p.key, blk_lo + u * kThreads * BPU, blk_hi, (uint32_t)m,
+        uint32_t neg_lo, neg_hi;
+        unit_signs<DT>(q[u], neg_lo, neg_hi);
+        quantize_unit<FMT, RNG>(v, inv, p.cap, neg_lo, neg_hi, p.key, blk_lo + u * kThreads * BPU, blk_hi, (uint32_t)m,
                                 lp + u * kThreads * (FMT == UQ_FMT_I8 ? 8 : 4));
     }
     if (overflow && lane < p.scales.N && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
