@@ -25,8 +25,18 @@ struct EncodeParams {
     PhiloxKey key;            // the ten round keys of the seed
 };
 
+// Tuning knobs (overridable with -D for sweeps): a thread owns UNITS units of 8 coordinates
+// (256 B of fp32 or 128 B of bf16 in flight per thread) and at least three CTAs share an SM
+// (up to 85 registers per thread).  Measured best on B200 among {64,128,256} B x {1..6} CTAs.
+#ifndef UQ_ENCODE_MIN_CTAS
+#define UQ_ENCODE_MIN_CTAS 3
+#endif
+#ifndef UQ_ENCODE_UNITS
+#define UQ_ENCODE_UNITS 8
+#endif
+
 template <int DT> struct EncodeShape {
-    static constexpr int UNITS = DT == UQ_F32 ? 4 : 8;          // 128 B of input per thread
+    static constexpr int UNITS = UQ_ENCODE_UNITS;
     static constexpr int TILE = kThreads * UNITS * 8;
 };
 
@@ -132,7 +142,7 @@ __device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, i
 }
 
 template <int DT, int FMT, int RNG, int IDXB>
-__global__ void __launch_bounds__(kThreads) encode_kernel(const __grid_constant__ EncodeParams p)
+__global__ void __launch_bounds__(kThreads, UQ_ENCODE_MIN_CTAS) encode_kernel(const __grid_constant__ EncodeParams p)
 {
     using E = Elem<DT>;
     using S = EncodeShape<DT>;
