@@ -32,6 +32,18 @@ def test_segmented_workloads_small(name, d, rng_bits):
     assert np.abs(lev.astype(int)).max() <= w.s
 
 
+@pytest.mark.parametrize("name,d,M,kw", [
+    ("c2", 2_100_003, 8, {}), ("c2", 2_100_003, 8, dict(rng_bits=32)), ("c3", 2_100_003, 8, {}),
+    ("c4", 1_060_013, 16, {}), ("c5", 1_060_013, 16, {}), ("c5", 2_100_003, 8, dict(rng_bits=32, idx_bits=8)),
+    ("c3", 2_100_003, 8, dict(dtype=wl.BF16, fmt="i4x2", s=7, scales=(7, 112, 1792))),
+])
+def test_mid_size_workloads(name, d, M, kw):
+    """A few million coordinates per worker: hundreds of tiles per kernel, a ragged last tile and
+    rows crossed by segment boundaries, in every wire format."""
+    w = wl.scaled(name, d, M=M, **kw)
+    check_parity(w, wl.generate(w))
+
+
 @pytest.mark.parametrize("norm", [wl.NORM_L2, wl.NORM_LINF])
 @pytest.mark.parametrize("fmt,s", [("i8", 127), ("i8", 1), ("i8", 5), ("i4x2", 7), ("i4x2", 1)])
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
