@@ -160,12 +160,13 @@ norm_partials_kernel(const void *__restrict__ g, int64_t d, int64_t stride, int 
         } else {
 #pragma unroll
             for (int u = 0; u < UNITS; ++u) {
-                const int64_t i = t0 + (int64_t)(u * kThreads + tid) * E::G;
+                // elements of this unit that are data (the row's padding beyond d is not)
+                const int valid = (int)min((int64_t)E::G, t1 - (t0 + (int64_t)(u * kThreads + tid) * E::G));
                 float v[E::G];
                 E::unpack(q[u], v);
 #pragma unroll
                 for (int e = 0; e < E::G; ++e)
-                    if (i + e < t1) acc.add(v[e]);    // the row's padding beyond d is not data
+                    if (e < valid) acc.add(v[e]);
             }
         }
         __shared__ double sh[kWarps];
