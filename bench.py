@@ -37,7 +37,10 @@ FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only
 
 # DRAM traffic per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum) from
 # the ncu captures summarised under profiles/, keyed by workload; None = not captured.
-NCU_TRAFFIC_BYTES = {}
+# c2: (268.8 MB read + 39.0 MB written) captured at d = 8,388,608, scaled by 25,557,032 / 8,388,608
+# (every coordinate is read and written once, so traffic is proportional to d); see
+# profiles/kernels_c2_small_ncu_full.md.
+NCU_TRAFFIC_BYTES = {"c2": 937.7e6}
 
 
 def hbm_peak():
@@ -431,7 +434,7 @@ def gpu_main(args):
             "frac": round(dom_gbs / peak, 4), "peak_kind": f"of {peak_kind}",
             "algorithmic_bytes_per_launch": int(ab[dom]),
             "avg_launch_ms": round(res["stages_ms"][dom], 5),
-            "traffic": NCU_TRAFFIC_BYTES.get(name),
+            "traffic": NCU_TRAFFIC_BYTES.get(name) if args.d is None and dom == "encode" else None,
         },
         "kernels": summ["kernels"],
     }
