@@ -177,7 +177,7 @@ __global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const __grid
             r[e] = __fmul_rn((float)s[e], c);
         }
     } else if (active) {
-        int j = find_segment(p.seg_off, p.nseg, i);
+        int j = j0;                              // the row's first segment; walk on from there
         for (int e = 0; e < C; ++e) {
             r[e] = 0.0f;
             if (i + e >= p.d) continue;

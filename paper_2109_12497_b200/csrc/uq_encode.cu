@@ -20,6 +20,7 @@ struct EncodeParams {
     int64_t d, stride;
     int32_t nseg, M;
     int64_t ntiles;
+    uint32_t main_blocks;     // CTAs that own tiles; the CTAs after them own rows crossed by boundaries
     float cap;                // (float) of the smallest scale: the largest level
     ScaleSet scales;          // single-scale: every entry is s
     PhiloxKey key;            // the ten round keys of the seed
@@ -62,7 +63,8 @@ template <> struct IdxBits<8> { using T = uint64_t; static __device__ __forceinl
 template <int FMT, int RNG>
 __device__ __forceinline__ void quantize_unit(const float (&v)[8], const float (&inv)[8], float cap,
                                               uint32_t neg_lo, uint32_t neg_hi, const PhiloxKey &key,
-                                              uint32_t blk_lo, uint32_t blk_hi, uint32_t m, void *dst)
+                                              uint32_t blk_lo, uint32_t blk_hi, uint32_t m, void *dst,
+                                              bool store = true)
 {
     constexpr uint32_t LB = RNG == 32 ? kLevelByte23 : kLevelByte16;
     uint32_t z[8];
@@ -83,6 +85,7 @@ __device__ __forceinline__ void quantize_unit(const float (&v)[8], const float (
     }
     const uint32_t lo = negate_bytes(gather_bytes<LB>(z[0], z[1], z[2], z[3]), neg_lo);
     const uint32_t hi = negate_bytes(gather_bytes<LB>(z[4], z[5], z[6], z[7]), neg_hi);
+    if (!store) return;
     if (FMT == UQ_FMT_I8) st_stream((uint2 *)dst, make_uint2(lo, hi));
     else st_stream((uint32_t *)dst, bytes_to_nibbles(lo, hi));
 }
@@ -102,8 +105,12 @@ template <int DT> __device__ __forceinline__ void unit_signs(const uint4 *q, uin
 }
 
 // Coordinates [a, b) of worker m with per-coordinate scale lookup and bounds: the ragged last
-// tile and the 256-coordinate rows that a segment boundary crosses.  `who` of `many` cooperating
-// threads takes every many-th unit.  Rare (a few rows per segment), so kept out of line.
+// tile and the 256-coordinate rows that a segment boundary crosses.  Thread `who` of `many`
+// cooperating threads (whole warps) takes every many-th unit, so a warp owns a row of 256
+// consecutive coordinates per round.  The warp looks the row's first segment up together; lane L
+// then holds the end and the scale of segment (first + L), and a coordinate's segment is the
+// number of ends at or before it, counted with shuffles: no dependent loads per coordinate.
+// Rare (a few rows per segment), so kept out of line.
 template <int DT, int FMT, int RNG, int IDXB>
 __device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, int64_t a, int64_t b, int who, int many)
 {
@@ -111,7 +118,34 @@ __device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, i
     constexpr bool MULTI = IDXB != 0;
     constexpr int IB = MULTI ? IDXB : 8;
     const char *row = (const char *)p.g + (size_t)m * (size_t)p.stride * E::BYTES;
-    for (int64_t i = a + (int64_t)who * 8; i < b; i += (int64_t)many * 8) {
+    const int lane = who & 31;
+    for (int64_t row0 = a + (int64_t)(who - lane) * 8; row0 < b; row0 += (int64_t)many * 8) {
+        const int64_t row1 = min(row0 + 256, b);
+        const int j_row = warp_find_segment(p.seg_off, p.nseg, row0);
+        const int jl = j_row + lane;
+        const int64_t my_end = jl < p.nseg ? segment_end(p.seg_off, p.nseg, jl, p.d) : INT64_MAX;
+        const float my_W = __ldg(p.W + min(jl, p.nseg - 1));
+        const int64_t i = min(row0 + lane * 8, b - 1);            // lanes beyond b idle but take part in the shuffles
+        int seg[8] = {0, 0, 0, 0, 0, 0, 0, 0};                    // segment of each coordinate, relative to j_row
+        int nb = 0;
+        for (; nb < 32; ++nb) {                                   // warp-uniform loop over the ends inside the row
+            const int64_t end = __shfl_sync(0xFFFFFFFFu, my_end, nb);
+            if (end >= row1) break;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) seg[e] += end <= i + e ? 1 : 0;
+        }
+        float Wc[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) Wc[e] = __shfl_sync(0xFFFFFFFFu, my_W, seg[e]);
+        if (nb == 32) {                                           // more than 32 segments in one row: walk the table
+            int j = j_row;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                j = advance_segment(p.seg_off, p.nseg, j, i + e);
+                Wc[e] = __ldg(p.W + j);
+            }
+        }
+        if (row0 + lane * 8 >= b) continue;
         float v[8];
         uint4 q[8 / E::G];
 #pragma unroll
@@ -124,15 +158,15 @@ __device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, i
         typename IdxBits<IB>::T kbits = 0;
         if (MULTI) kbits = IdxBits<IB>::load(p.idx + i * IB / 8);
         float inv[8];
-        int j = find_segment(p.seg_off, p.nseg, i);
+        bool overflow = false;
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
             if (i + e >= p.d) v[e] = 0.0f;                        // padding quantizes to level 0
-            j = advance_segment(p.seg_off, p.nseg, j, i + e);
             const int k = MULTI ? (int)((kbits >> (e * IB)) & ((1u << IB) - 1u)) : 0;
-            inv[e] = inv_scale(p.scales.s[k & (UQ_MAX_SCALES - 1)], __ldg(p.W + j));
-            if (not_finite(inv[e]) && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
+            inv[e] = inv_scale(p.scales.s[k & (UQ_MAX_SCALES - 1)], Wc[e]);
+            overflow |= not_finite(inv[e]);
         }
+        if (overflow && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
         const uint64_t blk = RNG == 32 ? (uint64_t)(i >> 2) : (uint64_t)(i >> 3);
         char *dst = FMT == UQ_FMT_I8 ? (char *)p.lev + (size_t)m * (size_t)p.stride + i
                                      : (char *)p.lev + (size_t)m * (size_t)(p.stride >> 1) + (i >> 1);
@@ -150,13 +184,30 @@ __global__ void __launch_bounds__(kThreads, UQ_ENCODE_MIN_CTAS) encode_kernel(co
     constexpr int IB = MULTI ? IDXB : 8;
     constexpr int H = 8 / E::G;                                  // 16-byte loads per unit
     constexpr uint32_t BPU = RNG == 32 ? 2u : 1u;                // Philox blocks per unit
+    const int tid = threadIdx.x, lane = tid & 31;
+    if (blockIdx.x >= p.main_blocks) {
+        // A CTA of the second kind: each warp takes one segment boundary and, if the boundary lies
+        // strictly inside a 256-coordinate row of a full tile, quantizes that row with per-coordinate
+        // scales (the tile's own CTA skips it).  Keeping these rows out of the tile CTAs keeps
+        // their lifetime short: the slow path no longer holds a whole CTA slot.
+        const uint32_t x = blockIdx.x - p.main_blocks;
+        const int m = (int)(x % (uint32_t)p.M);
+        const int64_t k = 1 + (int64_t)(x / (uint32_t)p.M) * kWarps + (tid >> 5);
+        if (k >= p.nseg) return;
+        const int64_t b = __ldg(p.seg_off + k), prev = __ldg(p.seg_off + k - 1);
+        const int64_t r0 = b & ~(int64_t)255;
+        const int64_t full_end = p.d / S::TILE * S::TILE;          // rows beyond belong to the ragged tile's CTA
+        if (b <= 0 || b == r0 || r0 >= full_end) return;           // not strictly inside a row of a full tile
+        if (prev > r0 && prev <= b) return;                        // an earlier boundary in the same row takes it
+        encode_span_general<DT, FMT, RNG, IDXB>(p, m, r0, r0 + 256, lane, 32);
+        return;
+    }
     // CTAs walk the tiles back to front with the worker varying fastest (see launch_encode)
-    const uint32_t rev = gridDim.x - 1u - blockIdx.x;
+    const uint32_t rev = p.main_blocks - 1u - blockIdx.x;
     const int m = (int)(rev % (uint32_t)p.M);
     const int64_t tile = rev / (uint32_t)p.M;
     const int64_t t0 = tile * S::TILE;
     const int64_t t1 = min(t0 + (int64_t)S::TILE, p.d);
-    const int tid = threadIdx.x, lane = tid & 31;
 
     if (t1 - t0 != S::TILE) {                                    // the ragged last tile
         encode_span_general<DT, FMT, RNG, IDXB>(p, m, t0, t1, tid, kThreads);
@@ -176,30 +227,51 @@ __global__ void __launch_bounds__(kThreads, UQ_ENCODE_MIN_CTAS) encode_kernel(co
     // every warp looks the segment up for itself (no shared memory, no barrier): once for the
     // tile if one segment covers it, else once per 256-coordinate row of the warp.
     // lane k holds s_k / W_j (single-scale: every lane holds s / W_j)
-    int j = warp_find_segment(p.seg_off, p.nseg, t0);
+    const int j = warp_find_segment(p.seg_off, p.nseg, t0);
     const bool tile_uniform = segment_end(p.seg_off, p.nseg, j, p.d) >= t1;
     constexpr int KMASK = IB < 4 ? (1 << IB) - 1 : UQ_MAX_SCALES - 1;    // lane L holds scale L & KMASK
-    float inv_lane = inv_scale(p.scales.s[lane & KMASK], __ldg(p.W + j));
-    bool overflow = not_finite(inv_lane);
+    const int32_t my_scale = p.scales.s[lane & KMASK];
+    float inv_row[S::UNITS];                                     // my lane's s_k / W for each of my warp's rows
+    uint32_t crossed = 0;                                        // rows that a segment boundary crosses
+    if (tile_uniform) {
+        const float inv_lane = inv_scale(my_scale, __ldg(p.W + j));
+#pragma unroll
+        for (int u = 0; u < S::UNITS; ++u) inv_row[u] = inv_lane;
+    } else {
+        // A segment boundary crosses the tile.  Lane L takes the end of segment j + L, so the
+        // segment of any row is j + (number of ends at or before the row's start): one ballot per
+        // row instead of a search, and the scales of all rows are fetched together.
+        const int64_t my_end = j + lane < p.nseg ? segment_end(p.seg_off, p.nseg, j + lane, p.d) : INT64_MAX;
+#pragma unroll
+        for (int u = 0; u < S::UNITS; ++u) {
+            const int64_t r0 = t0 + (int64_t)(u * kThreads + (tid & ~31)) * 8;
+            const int cnt = __popc(__ballot_sync(0xFFFFFFFFu, my_end <= r0));
+            int jr;
+            int64_t end;
+            if (cnt < 32) {
+                jr = j + cnt;
+                end = __shfl_sync(0xFFFFFFFFu, my_end, cnt);
+            } else {                                             // more than 32 segments inside one tile
+                jr = warp_find_segment(p.seg_off, p.nseg, r0);
+                end = segment_end(p.seg_off, p.nseg, jr, p.d);
+            }
+            if (end < r0 + 256) crossed |= 1u << u;
+            inv_row[u] = inv_scale(my_scale, __ldg(p.W + jr));
+        }
+    }
+    bool overflow = false;
 
     const uint64_t blk0 = RNG == 32 ? (uint64_t)(t0 >> 2) : (uint64_t)(t0 >> 3);           // low bits are 0
     const uint32_t blk_hi = (uint32_t)(blk0 >> 32);
     const uint32_t blk_lo = (uint32_t)blk0 + (uint32_t)tid * BPU;
     char *lp = FMT == UQ_FMT_I8 ? (char *)p.lev + (size_t)m * (size_t)p.stride + (size_t)t0 + tid * 8
                                 : (char *)p.lev + (size_t)m * (size_t)(p.stride >> 1) + (size_t)(t0 >> 1) + tid * 4;
-    uint32_t crossed = 0;                                        // rows left to the general path
+    // One straight-line pass over all units, so the compiler can interleave them.  A crossed row
+    // runs through the arithmetic too but is not stored: a CTA of the second kind owns it.
 #pragma unroll
     for (int u = 0; u < S::UNITS; ++u) {
-        if (!tile_uniform) {                                     // warp-uniform branch
-            const int64_t r0 = t0 + (int64_t)(u * kThreads + (tid & ~31)) * 8;
-            j = warp_find_segment(p.seg_off, p.nseg, r0);
-            if (segment_end(p.seg_off, p.nseg, j, p.d) < r0 + 256) {
-                crossed |= 1u << u;
-                continue;
-            }
-            inv_lane = inv_scale(p.scales.s[lane & KMASK], __ldg(p.W + j));
-            overflow |= not_finite(inv_lane);
-        }
+        const float inv_lane = inv_row[u];
+        overflow |= not_finite(inv_lane);
         float v[8], inv[8];
 #pragma unroll
         for (int h = 0; h < H; ++h) E::unpack(q[u][h], *(float(*)[E::G])(v + h * E::G));
@@ -211,16 +283,9 @@ __global__ void __launch_bounds__(kThreads, UQ_ENCODE_MIN_CTAS) encode_kernel(co
         uint32_t neg_lo, neg_hi;
         unit_signs<DT>(q[u], neg_lo, neg_hi);
         quantize_unit<FMT, RNG>(v, inv, p.cap, neg_lo, neg_hi, p.key, blk_lo + u * kThreads * BPU, blk_hi, (uint32_t)m,
-                                lp + u * kThreads * (FMT == UQ_FMT_I8 ? 8 : 4));
+                                lp + u * kThreads * (FMT == UQ_FMT_I8 ? 8 : 4), !((crossed >> u) & 1u));
     }
     if (overflow && lane < p.scales.N && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
-    // rows crossed by a segment boundary, once the tile's registers are free
-    for (int u = 0; crossed != 0; ++u, crossed >>= 1) {
-        if (crossed & 1u) {
-            const int64_t r0 = t0 + (int64_t)(u * kThreads + (tid & ~31)) * 8;
-            encode_span_general<DT, FMT, RNG, IDXB>(p, m, r0, r0 + 256, lane, 32);
-        }
-    }
 }
 
 template <int DT, int FMT, int RNG, int IDXB>
@@ -228,8 +293,11 @@ static cudaError_t launch(EncodeParams p, cudaStream_t st)
 {
     using S = EncodeShape<DT>;
     p.ntiles = (p.d + S::TILE - 1) / S::TILE;
-    const int64_t blocks = p.ntiles * p.M;
+    int64_t blocks = p.ntiles * p.M;
     if (blocks == 0) return cudaSuccess;
+    if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    p.main_blocks = (uint32_t)blocks;
+    if (p.seg_off != nullptr && p.nseg > 1) blocks += (int64_t)((p.nseg - 1 + kWarps - 1) / kWarps) * p.M;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     encode_kernel<DT, FMT, RNG, IDXB><<<(unsigned)blocks, kThreads, 0, st>>>(p);
     return cudaGetLastError();

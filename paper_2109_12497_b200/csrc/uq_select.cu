@@ -48,10 +48,10 @@ __device__ __forceinline__ int32_t pass_threshold(float inv, float s_hat)
 
 // The general path for one thread's 8 coordinates (row crossed by a segment boundary): the test
 // is evaluated as written, with one division per scale and coordinate.  Rare, kept out of line.
-__device__ __noinline__ uint64_t select_general(const SelectParams &p, int64_t i, const uint32_t (&amag)[8], int idxb)
+__device__ __noinline__ uint64_t select_general(const SelectParams &p, int64_t i, const uint32_t (&amag)[8], int idxb,
+                                                 int j)      // j: a segment at or before coordinate i's
 {
     uint64_t packed = 0;
-    int j = find_segment(p.seg_off, p.nseg, i);
     for (int e = 0; e < 8; ++e) {
         int k = 0;
         if (i + e < p.d) {                                          // padding keeps index 0
@@ -168,7 +168,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
             packed |= (uint64_t)k << (e * IDXB);
         }
     } else if (active) {
-        packed = select_general(p, i, amag, IDXB);
+        packed = select_general(p, i, amag, IDXB, j0);
     }
     if (!active) return;
     if (IDXB == 2) *(uint16_t *)(p.idx + (i >> 2)) = (uint16_t)packed;
