@@ -26,18 +26,18 @@ struct EncodeParams {
     PhiloxKey key;            // the ten round keys of the seed
 };
 
-// Tuning knobs (overridable with -D for sweeps): a thread owns UNITS units of 8 coordinates
-// (256 B of fp32 or 128 B of bf16 in flight per thread) and at least three CTAs share an SM
-// (up to 85 registers per thread).  Measured best on B200 among {64,128,256} B x {1..6} CTAs.
-#ifndef UQ_ENCODE_MIN_CTAS
-#define UQ_ENCODE_MIN_CTAS 3
+// Launch shape per variant, from sweeps on B200 over {4, 8} units x {2..5} CTAs per SM: a thread
+// owns UNITS units of 8 coordinates and at least MIN_CTAS CTAs share an SM (which caps the
+// registers per thread).  -DUQ_ENCODE_UNITS / -DUQ_ENCODE_MIN_CTAS override all variants (sweeps).
+template <int DT, bool MULTI> struct EncodeShape {
+#if defined(UQ_ENCODE_UNITS) && defined(UQ_ENCODE_MIN_CTAS)
+    static constexpr int UNITS = UQ_ENCODE_UNITS, MIN_CTAS = UQ_ENCODE_MIN_CTAS;
+#else
+    // fp32 multi-scale: the index shuffles want registers and short unit chains -> 4 units, 4 CTAs
+    // bf16 multi-scale: 8 units (128 B in flight per thread), 4 CTAs; single-scale: 8 units, 3 CTAs
+    static constexpr int UNITS = (DT == UQ_F32 && MULTI) ? 4 : 8;
+    static constexpr int MIN_CTAS = MULTI ? 4 : 3;
 #endif
-#ifndef UQ_ENCODE_UNITS
-#define UQ_ENCODE_UNITS 8
-#endif
-
-template <int DT> struct EncodeShape {
-    static constexpr int UNITS = UQ_ENCODE_UNITS;
     static constexpr int TILE = kThreads * UNITS * 8;
 };
 
@@ -176,10 +176,10 @@ __device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, i
 }
 
 template <int DT, int FMT, int RNG, int IDXB>
-__global__ void __launch_bounds__(kThreads, UQ_ENCODE_MIN_CTAS) encode_kernel(const __grid_constant__ EncodeParams p)
+__global__ void __launch_bounds__(kThreads, (EncodeShape<DT, IDXB != 0>::MIN_CTAS)) encode_kernel(const __grid_constant__ EncodeParams p)
 {
     using E = Elem<DT>;
-    using S = EncodeShape<DT>;
+    using S = EncodeShape<DT, IDXB != 0>;
     constexpr bool MULTI = IDXB != 0;
     constexpr int IB = MULTI ? IDXB : 8;
     constexpr int H = 8 / E::G;                                  // 16-byte loads per unit
@@ -291,7 +291,7 @@ __global__ void __launch_bounds__(kThreads, UQ_ENCODE_MIN_CTAS) encode_kernel(co
 template <int DT, int FMT, int RNG, int IDXB>
 static cudaError_t launch(EncodeParams p, cudaStream_t st)
 {
-    using S = EncodeShape<DT>;
+    using S = EncodeShape<DT, IDXB != 0>;
     p.ntiles = (p.d + S::TILE - 1) / S::TILE;
     int64_t blocks = p.ntiles * p.M;
     if (blocks == 0) return cudaSuccess;
