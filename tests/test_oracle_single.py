@@ -99,6 +99,12 @@ def test_level_range_on_adversarial_inputs(s):
         assert np.abs(lev.astype(int)).max() <= s
         assert lev[0, 0] == s and lev[0, 1] == -s and lev[0, 2] == s and lev[0, 3] == -s
         assert lev[0, 4] == 0 and lev[0, 5] == 0                  # sign(0) = 0, Q(0) = 0
+    # a caller-supplied scale smaller than the data: a = |v| / W > 1 has no level below s, the
+    # level saturates at s (and never wraps around in int8)
+    big = np.array([[2 * W, -3 * W, 1.5 * W, W / 2]], dtype=np.float32)
+    for seed in range(5):
+        lev = o.encode_single(big, np.array([W]), s, seed)
+        assert lev[0, :3].tolist() == [s, -s, s] and abs(int(lev[0, 3])) <= s
     # an all-zero vector has W = 0 and quantizes to zero
     z = np.zeros((2, 16), dtype=np.float32)
     Wz = o.agree_scale(z)
