@@ -236,6 +236,25 @@ def time_graph_replay(q, g, w, reps):
     return e0.elapsed_time(e1) / reps
 
 
+def time_fused_update(q, w, reps):
+    """Mean ms of the fused aggregate + reconstruct + SGD-with-momentum kernel alone (the levels
+    are those of the last step; it replaces aggregate_decode when the caller wants the update)."""
+    import torch
+    st = torch.cuda.current_stream()
+    theta = torch.zeros(max(w.d, 1), dtype=torch.float32, device="cuda")
+    mom = torch.zeros_like(theta)
+    for _ in range(2):
+        q.aggregate_decode_update(theta, mom, 0.1, 0.9, 5e-4)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(st)
+    for _ in range(reps):
+        q.aggregate_decode_update(theta, mom, 0.1, 0.9, 5e-4)
+    e1.record(st)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
 def l2_flush_buffer():
     import torch
     return torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
@@ -297,6 +316,7 @@ def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=F
         res["ms_graph"] = time_graph_replay(q, g_dev, w, max(steps, 20))
     res["ms"], res["stages_ms"] = time_device_resident(q, g_dev, w, steps, warmup, barrier)
     res["encode_other_ms"] = time_encode_other_mode(q, g_dev, w, min(steps, 10))
+    res["update_ms"] = time_fused_update(q, w, min(steps, 10))
     res["h2d"], res["d2h"], res["e2e_ms"] = 0, 0, None
     if want_e2e:
         out_host = torch.empty(w.d, dtype=torch.float32, pin_memory=True)
@@ -320,6 +340,13 @@ def summarize(res, peak_gbs):
     out["kernels"][f"encode_rng{other}"] = {
         "ms": round(ms, 5), "algorithmic_MB": round(ab["encode"] / 1e6, 2), "GBps": round(ab["encode"] / ms / 1e6, 1),
         "frac_of_hbm_peak": round(ab["encode"] / ms / 1e6 / peak_gbs, 4), "note": "timed alone, not part of the step"}
+    lev = 1.0 if w.fmt == "i8" else 0.5
+    upd_bytes = lev * w.M * w.d + w.idx_bits / 8.0 * w.d + 16 * w.d      # levels, index, theta and momentum r/w
+    ms = res["update_ms"]
+    out["kernels"]["aggregate_decode_update"] = {
+        "ms": round(ms, 5), "algorithmic_MB": round(upd_bytes / 1e6, 2), "GBps": round(upd_bytes / ms / 1e6, 1),
+        "frac_of_hbm_peak": round(upd_bytes / ms / 1e6 / peak_gbs, 4),
+        "note": "fused SGD-momentum update, timed alone, not part of the step"}
     if "ms_cold" in res:
         out["cold_l2"] = {"ms_per_step": res["ms_cold"], "gradient_GBps": w.in_bytes / res["ms_cold"] / 1e6,
                           "kernels_ms": {s: round(v, 5) for s, v in res["stages_cold_ms"].items()}}

@@ -217,6 +217,27 @@ int uq_decode(const uq_layout *layout, const void *src, int src_kind, int fmt, c
               const int32_t *scales, int N, const uint8_t *idx, int idx_bits, float *out,
               int32_t *S_opt, void *stream);
 
+/*
+ * Reconstruction fused with the parameter update — Algorithm 1 / 2, lines "AllReduce gradients",
+ * "Reconstruct gradient" and "Update parameters" (theta_{t+1} = theta_t - eta_t * g_hat_t) in one
+ * kernel: the level rows are summed and reconstructed as in uq_decode(src = LEVELS) and the
+ * result goes from registers into the parameters.  Reading of the optimizer the paper's
+ * experiments name (SGD with momentum 0.9 and weight decay 5e-4): per coordinate, in binary32,
+ * one IEEE operation per step,
+ *   u = g_hat + wd * theta            (skipped when wd == 0)
+ *   buf = mu * buf + u;  u = buf      (only when momentum != NULL)
+ *   theta = theta - lr * u.
+ * momentum = NULL, wd = 0 is the update of Algorithm 1 as printed.
+ *   theta     i/o  [d] float, 32-byte aligned, updated in place
+ *   momentum  i/o  [d] float, 32-byte aligned, or NULL
+ *   out_opt   out  [d] float, 32-byte aligned, or NULL: also receives g_hat
+ * scales = NULL selects the single scale s; otherwise scales, N, idx, idx_bits as in the encoder.
+ * Errors: UQ_ERR_BAD_ARG (also for NaN lr / mu / wd), UQ_ERR_CUDA.
+ */
+int uq_decode_update(const uq_layout *layout, const void *lev, int fmt, const float *W, int s,
+                     const int32_t *scales, int N, const uint8_t *idx, int idx_bits, float *theta,
+                     float *momentum, float lr, float mu, float wd, float *out_opt, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -315,6 +315,25 @@ void uqo_decode_f64(const int32_t *S, int M, int64_t coord0, int64_t d, int nseg
 }
 
 /* ------------------------------------------------------------------------------------------
+ * Algorithm 1 / 2, line "Update parameters": theta_{t+1} = theta_t - eta_t * g_hat_t.
+ * Reading of the optimizer named in Section "Experiments" (SGD, momentum mu, weight decay wd):
+ *   u = g_hat + wd * theta;  buf = mu * buf + u, u = buf (if a momentum buffer is given);
+ *   theta = theta - lr * u.       mom == NULL, wd = 0 is the printed update.
+ * Binary32, one IEEE operation per written operator (the weight-decay term is skipped when
+ * wd == 0, so that the printed update is exactly theta - lr * g_hat).
+ * ------------------------------------------------------------------------------------------ */
+void uqo_sgd_update(const float *g_hat, int64_t d, float *theta, float *mom, float lr, float mu, float wd)
+{
+    for (int64_t i = 0; i < d; ++i) {
+        float u = g_hat[i];
+        if (wd != 0.0f) { float t = wd * theta[i]; u = u + t; }
+        if (mom) { float t = mu * mom[i]; mom[i] = t + u; u = mom[i]; }
+        float step = lr * u;
+        theta[i] = theta[i] - step;
+    }
+}
+
+/* ------------------------------------------------------------------------------------------
  * Wire formats (the bit counts r = ceil(log s) + 1 and + ceil(log N) of the two sections).
  * ------------------------------------------------------------------------------------------ */
 

@@ -211,3 +211,14 @@ def pack_index(idx: np.ndarray, idx_bits: int) -> np.ndarray:
     packed = np.zeros((idx.size + per - 1) // per, dtype=np.uint8)
     lib().uqo_pack_index(_p(idx), C.c_int64(idx.size), idx_bits, _p(packed))
     return packed
+
+
+def sgd_update(g_hat, theta, mom=None, lr=0.1, mu=0.0, wd=0.0):
+    """theta (and the momentum buffer) after one step; inputs are not modified."""
+    g_hat = np.ascontiguousarray(g_hat, dtype=np.float32)
+    theta = np.array(theta, dtype=np.float32, copy=True)
+    mom = None if mom is None else np.array(mom, dtype=np.float32, copy=True)
+    assert theta.shape == g_hat.shape and (mom is None or mom.shape == g_hat.shape)
+    lib().uqo_sgd_update(_p(g_hat), C.c_int64(g_hat.size), _p(theta), _p(mom), C.c_float(lr), C.c_float(mu),
+                         C.c_float(wd))
+    return theta, mom

@@ -26,7 +26,7 @@ UQ_STATUS_NONFINITE, UQ_STATUS_BAD_SEGMENTS, UQ_STATUS_SCALE_OVERFLOW = 1, 2, 4
 EXPORTS = (
     "uq_version", "uq_last_cuda_error", "uq_error_string", "uq_workspace_bytes", "uq_index_bytes",
     "uq_agree_scale", "uq_agree_scale_static", "uq_encode_single", "uq_select_scale_multi", "uq_encode_multi",
-    "uq_aggregate", "uq_decode",
+    "uq_aggregate", "uq_decode", "uq_decode_update",
 )
 
 
@@ -80,6 +80,8 @@ def lib() -> C.CDLL:
         L.uq_encode_multi.argtypes = [LP, P, P, P, I, P, I, U64, I, I, P, P, P]
         L.uq_aggregate.argtypes = [LP, P, I, P, P]
         L.uq_decode.argtypes = [LP, P, I, I, P, I, P, I, P, I, P, P, P]
+        F = C.c_float
+        L.uq_decode_update.argtypes = [LP, P, I, P, I, P, I, P, I, P, P, F, F, F, P, P]
         for name in EXPORTS[5:]:
             getattr(L, name).restype = I
         _lib = L
@@ -236,3 +238,25 @@ def uq_decode(layout: Layout, src: torch.Tensor, src_kind: int, fmt: int, W: tor
     _check("uq_decode", lib().uq_decode(
         layout.ref(), _ptr(src), src_kind, fmt, _ptr(W), s, arr, N, _ptr(idx) if scales is not None else None,
         idx_bits, _ptr(out), _ptr(S_opt), _stream()))
+
+
+def uq_decode_update(layout: Layout, lev: torch.Tensor, fmt: int, W: torch.Tensor, s: int,
+                     scales: Optional[Sequence[int]], idx: Optional[torch.Tensor], idx_bits: int,
+                     theta: torch.Tensor, momentum: Optional[torch.Tensor], lr: float, mu: float = 0.0,
+                     wd: float = 0.0, out: Optional[torch.Tensor] = None) -> None:
+    """Sum of the level rows, reconstruction and the SGD step on theta (and the momentum buffer)
+    in one kernel; ``out`` optionally also receives the reconstructed gradient."""
+    layout.check_lev(lev, fmt)
+    layout.check_vec(W, torch.float32, layout.nseg, "W")
+    layout.check_vec(theta, torch.float32, layout.d, "theta")
+    if momentum is not None:
+        layout.check_vec(momentum, torch.float32, layout.d, "momentum")
+    if out is not None:
+        layout.check_vec(out, torch.float32, layout.d, "out")
+    arr, N = (None, 0)
+    if scales is not None:
+        arr, N = _scales(scales)
+        layout.check_vec(idx, torch.uint8, layout.index_bytes(idx_bits), "idx")
+    _check("uq_decode_update", lib().uq_decode_update(
+        layout.ref(), _ptr(lev), fmt, _ptr(W), s, arr, N, _ptr(idx) if scales is not None else None, idx_bits,
+        _ptr(theta), _ptr(momentum), lr, mu, wd, _ptr(out), _stream()))

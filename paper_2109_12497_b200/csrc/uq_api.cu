@@ -13,7 +13,8 @@ cudaError_t launch_select(const uq_layout &L, const void *g, const float *W, con
                           int idx_bits, uint8_t *idx, uint32_t *status, cudaStream_t st);
 cudaError_t launch_aggregate_decode(const uq_layout &L, const void *lev, int fmt, const float *W,
                                     const ScaleSet &scales, const uint8_t *idx, int idx_bits, float *out,
-                                    int32_t *S, cudaStream_t st);
+                                    int32_t *S, cudaStream_t st, float *theta = nullptr, float *mom = nullptr,
+                                    float lr = 0.0f, float mu = 0.0f, float wd = 0.0f);
 cudaError_t launch_decode_sums(const uq_layout &L, const int32_t *S, const float *W, const ScaleSet &scales,
                                const uint8_t *idx, int idx_bits, float *out, cudaStream_t st);
 }  // namespace uq
@@ -188,6 +189,29 @@ int uq_decode(const uq_layout *L, const void *src, int src_kind, int fmt, const 
     if (S_opt != nullptr && !aligned(S_opt, 32)) return UQ_ERR_BAD_ARG;
     return finish(uq::launch_aggregate_decode(*L, src, fmt, W, set, idx, idx_bits, out, S_opt,
                                               (cudaStream_t)stream));
+}
+
+int uq_decode_update(const uq_layout *L, const void *lev, int fmt, const float *W, int s, const int32_t *scales,
+                     int N, const uint8_t *idx, int idx_bits, float *theta, float *momentum, float lr, float mu,
+                     float wd, float *out_opt, void *stream)
+{
+    if (!layout_ok(L) || W == nullptr || (fmt != UQ_FMT_I8 && fmt != UQ_FMT_I4X2)) return UQ_ERR_BAD_ARG;
+    if (!(lr == lr) || !(mu == mu) || !(wd == wd)) return UQ_ERR_BAD_ARG;                  // NaN hyper-parameters
+    uq::ScaleSet set;
+    if (scales != nullptr) {
+        if (!scales_ok(scales, N, idx_bits, &set)) return UQ_ERR_BAD_ARG;
+        if (L->d > 0 && (idx == nullptr || !aligned(idx, 16))) return UQ_ERR_BAD_ARG;
+    } else {
+        if (s < 1) return UQ_ERR_BAD_ARG;
+        set = single_scale(s);
+        idx_bits = 0;
+        idx = nullptr;
+    }
+    if (L->d > 0 && (lev == nullptr || theta == nullptr || !aligned(lev, 16) || !aligned(theta, 32))) return UQ_ERR_BAD_ARG;
+    if (!aligned(momentum, 32) || !aligned(out_opt, 32)) return UQ_ERR_BAD_ARG;
+    if (L->d == 0) return UQ_OK;
+    return finish(uq::launch_aggregate_decode(*L, lev, fmt, W, set, idx, idx_bits, out_opt, nullptr, (cudaStream_t)stream,
+                                              theta, momentum, lr, mu, wd));
 }
 
 }  // extern "C"

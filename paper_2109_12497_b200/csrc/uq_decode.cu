@@ -19,7 +19,23 @@ struct DecodeParams {
     int64_t d, stride;
     int32_t nseg, M;
     ScaleSet scales;          // single-scale: N = 1
+    // fused parameter update (theta == NULL: none)
+    float *theta;             // parameters, updated in place
+    float *mom;               // momentum buffer, updated in place; NULL for plain SGD
+    float lr, mu, wd;         // step size, momentum factor, weight decay
 };
+
+// One coordinate of the update theta <- theta - lr * u with
+//   u = g_hat + wd * theta (weight decay, skipped when wd == 0) and, with a momentum buffer,
+//   buf <- mu * buf + u,  u = buf.   One IEEE operation per step, nothing fused.
+__device__ __forceinline__ void sgd_coordinate(float g_hat, float &theta, float &buf, bool has_mom, float lr, float mu,
+                                               float wd)
+{
+    float u = g_hat;
+    if (wd != 0.0f) u = __fadd_rn(u, __fmul_rn(wd, theta));
+    if (has_mom) { buf = __fadd_rn(__fmul_rn(mu, buf), u); u = buf; }
+    theta = __fsub_rn(theta, __fmul_rn(lr, u));
+}
 
 // W / ((float)s * (float)M): product, then one IEEE division.
 __device__ __forceinline__ float decode_factor(float W, int32_t s, int M)
@@ -113,7 +129,9 @@ template <> struct Unit<UQ_FMT_I4X2> {
     }
 };
 
-template <int FMT, int IDXB>
+// UPDATE selects the variant that also applies the parameter update (kept apart so that the plain
+// reconstruction keeps its register count).
+template <int FMT, int IDXB, bool UPDATE>
 __global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const __grid_constant__ DecodeParams p)
 {
     using U = Unit<FMT>;
@@ -161,7 +179,7 @@ __global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const __grid
                 if (i + e < p.d) p.S[i + e] = s[e];
         }
     }
-    if (p.out == nullptr) return;
+    if (p.out == nullptr && !UPDATE) return;
 
     // every warp looks up the segment of its own row of 32*C coordinates; lane k holds the
     // reconstruction factor of scale k (single-scale: every lane holds the same factor)
@@ -187,6 +205,42 @@ __global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const __grid
         }
     }
     if (!active) return;
+    if (UPDATE) {
+        // Algorithm 1 / 2, line "Update parameters", fused: the reconstructed gradient goes straight
+        // from registers into the parameters (and the momentum buffer)
+        const bool has_mom = p.mom != nullptr;
+        if (full) {
+            // 16 coordinates at a time: their eight 16-byte loads are issued together
+#pragma unroll
+            for (int e0 = 0; e0 < C; e0 += 16) {
+                float4 th[4], bf[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    th[k] = *(const float4 *)(p.theta + i + e0 + 4 * k);
+                    bf[k] = has_mom ? *(const float4 *)(p.mom + i + e0 + 4 * k) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int e = e0 + 4 * k;
+                    sgd_coordinate(r[e + 0], th[k].x, bf[k].x, has_mom, p.lr, p.mu, p.wd);
+                    sgd_coordinate(r[e + 1], th[k].y, bf[k].y, has_mom, p.lr, p.mu, p.wd);
+                    sgd_coordinate(r[e + 2], th[k].z, bf[k].z, has_mom, p.lr, p.mu, p.wd);
+                    sgd_coordinate(r[e + 3], th[k].w, bf[k].w, has_mom, p.lr, p.mu, p.wd);
+                    *(float4 *)(p.theta + i + e) = th[k];
+                    if (has_mom) *(float4 *)(p.mom + i + e) = bf[k];
+                }
+            }
+        } else {
+            for (int e = 0; e < C; ++e) {
+                if (i + e >= p.d) break;
+                float th = p.theta[i + e], bf = has_mom ? p.mom[i + e] : 0.0f;
+                sgd_coordinate(r[e], th, bf, has_mom, p.lr, p.mu, p.wd);
+                p.theta[i + e] = th;
+                if (has_mom) p.mom[i + e] = bf;
+            }
+        }
+    }
+    if (p.out == nullptr) return;
     if (full) {
 #pragma unroll
         for (int e = 0; e < C; e += 8) st_stream256(p.out + i + e, *(const uint32_t(*)[8])(r + e));
@@ -237,11 +291,20 @@ static cudaError_t dispatch_levels(const DecodeParams &p, int idx_bits, cudaStre
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     const unsigned nb = (unsigned)blocks;
+    if (p.theta != nullptr) {
+        switch (idx_bits) {
+        case 0: aggregate_decode_kernel<FMT, 0, true><<<nb, kThreads, 0, st>>>(p); break;
+        case 2: aggregate_decode_kernel<FMT, 2, true><<<nb, kThreads, 0, st>>>(p); break;
+        case 4: aggregate_decode_kernel<FMT, 4, true><<<nb, kThreads, 0, st>>>(p); break;
+        default: aggregate_decode_kernel<FMT, 8, true><<<nb, kThreads, 0, st>>>(p); break;
+        }
+        return cudaGetLastError();
+    }
     switch (idx_bits) {
-    case 0: aggregate_decode_kernel<FMT, 0><<<nb, kThreads, 0, st>>>(p); break;
-    case 2: aggregate_decode_kernel<FMT, 2><<<nb, kThreads, 0, st>>>(p); break;
-    case 4: aggregate_decode_kernel<FMT, 4><<<nb, kThreads, 0, st>>>(p); break;
-    default: aggregate_decode_kernel<FMT, 8><<<nb, kThreads, 0, st>>>(p); break;
+    case 0: aggregate_decode_kernel<FMT, 0, false><<<nb, kThreads, 0, st>>>(p); break;
+    case 2: aggregate_decode_kernel<FMT, 2, false><<<nb, kThreads, 0, st>>>(p); break;
+    case 4: aggregate_decode_kernel<FMT, 4, false><<<nb, kThreads, 0, st>>>(p); break;
+    default: aggregate_decode_kernel<FMT, 8, false><<<nb, kThreads, 0, st>>>(p); break;
     }
     return cudaGetLastError();
 }
@@ -249,11 +312,13 @@ static cudaError_t dispatch_levels(const DecodeParams &p, int idx_bits, cudaStre
 // out == NULL: aggregate only.  idx_bits == 0: single scale (scales = {s}).
 cudaError_t launch_aggregate_decode(const uq_layout &L, const void *lev, int fmt, const float *W,
                                     const ScaleSet &scales, const uint8_t *idx, int idx_bits, float *out,
-                                    int32_t *S, cudaStream_t st)
+                                    int32_t *S, cudaStream_t st, float *theta, float *mom, float lr, float mu,
+                                    float wd)
 {
     DecodeParams p;
     p.lev = lev; p.W = W; p.seg_off = L.seg_off; p.idx = idx; p.out = out; p.S = S;
     p.d = L.d; p.stride = L.worker_stride; p.nseg = L.nseg; p.M = L.M; p.scales = scales;
+    p.theta = theta; p.mom = mom; p.lr = lr; p.mu = mu; p.wd = wd;
     return fmt == UQ_FMT_I8 ? dispatch_levels<UQ_FMT_I8>(p, idx_bits, st)
                             : dispatch_levels<UQ_FMT_I4X2>(p, idx_bits, st);
 }
@@ -263,6 +328,7 @@ cudaError_t launch_decode_sums(const uq_layout &L, const int32_t *S, const float
 {
     DecodeParams p;
     p.lev = S; p.W = W; p.seg_off = L.seg_off; p.idx = idx; p.out = out; p.S = nullptr;
+    p.theta = nullptr; p.mom = nullptr; p.lr = p.mu = p.wd = 0.0f;
     p.d = L.d; p.stride = L.worker_stride; p.nseg = L.nseg; p.M = L.M; p.scales = scales;
     const int64_t blocks = (L.d + kThreads * 4 - 1) / (kThreads * 4);
     if (blocks == 0) return cudaSuccess;

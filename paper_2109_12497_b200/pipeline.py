@@ -62,6 +62,12 @@ class Quantizer:
         B.uq_decode(self.layout, self.lev, B.UQ_SRC_LEVELS, self.fmt, self.W, self.s, self.scales, self.idx,
                     self.idx_bits, self.out, self.S)
 
+    def aggregate_decode_update(self, theta: torch.Tensor, momentum: Optional[torch.Tensor], lr: float,
+                                mu: float = 0.0, wd: float = 0.0) -> None:
+        """Fused aggregation, reconstruction and SGD step on theta (Algorithm 1/2, last three lines)."""
+        B.uq_decode_update(self.layout, self.lev, self.fmt, self.W, self.s, self.scales, self.idx, self.idx_bits,
+                           theta, momentum, lr, mu, wd)
+
     def step(self, g: torch.Tensor, seed: int = 0) -> torch.Tensor:
         """g: [M, stride] gradients of all workers -> the reconstructed average gradient [d]."""
         self.agree_scale(g)
