@@ -59,7 +59,7 @@ def hbm_peak():
 
 def algorithmic_bytes(w: wl.Workload) -> dict:
     e = 4 if w.dtype == wl.F32 else 2
-    lev = 1.0 if w.fmt == "i8" else 0.5
+    lev = {"i8": 1.0, "i4x2": 0.5, "i2x4": 0.25}[w.fmt]
     ib = w.idx_bits / 8.0
     M, d = w.M, w.d
     b = {"agree_scale": e * M * d}
@@ -340,7 +340,7 @@ def summarize(res, peak_gbs):
     out["kernels"][f"encode_rng{other}"] = {
         "ms": round(ms, 5), "algorithmic_MB": round(ab["encode"] / 1e6, 2), "GBps": round(ab["encode"] / ms / 1e6, 1),
         "frac_of_hbm_peak": round(ab["encode"] / ms / 1e6 / peak_gbs, 4), "note": "timed alone, not part of the step"}
-    lev = 1.0 if w.fmt == "i8" else 0.5
+    lev = {"i8": 1.0, "i4x2": 0.5, "i2x4": 0.25}[w.fmt]
     upd_bytes = lev * w.M * w.d + w.idx_bits / 8.0 * w.d + 16 * w.d      # levels, index, theta and momentum r/w
     ms = res["update_ms"]
     out["kernels"]["aggregate_decode_update"] = {
@@ -469,12 +469,16 @@ def gpu_main(args):
         # the other four workloads (parity-test cases; reported for context, a few steps each)
         if not args.no_extra and args.d is None:
             extra = {}
-            for other in ("c1", "c3", "c4", "c5"):
+            import dataclasses
+            others = [(o_, resolve_workload(o_, None, args.rng_bits)) for o_ in ("c1", "c3", "c4", "c5")]
+            # c2 on the 2-bit wire (s = 1: levels -1, 0, 1, four per byte)
+            others.append(("c2_levels_2bit", dataclasses.replace(resolve_workload("c2", None, args.rng_bits),
+                                                                 fmt="i2x4", s=1, scales=(1,))))
+            for other, wo in others:
                 del res, q
                 torch.cuda.empty_cache()
-                small = wl.WORKLOADS[other].in_bytes < (126 << 20)
-                res = bench_workload(resolve_workload(other, None, args.rng_bits), max(3, min(args.steps, 10)), 3,
-                                     lambda: None, threads,
+                small = wo.in_bytes < (126 << 20)
+                res = bench_workload(wo, max(3, min(args.steps, 10)), 3, lambda: None, threads,
                                      want_e2e=False, flush_between=small)
                 q = res["q"]
                 extra[other] = summarize(res, peak)

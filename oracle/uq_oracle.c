@@ -350,6 +350,21 @@ void uqo_pack_levels_i4(const int8_t *lev, int M, int64_t d, int64_t stride, uin
         }
 }
 
+/* 2-bit levels (s = 1, zeta in {-1, 0, 1}): two's-complement 2-bit fields, four coordinates per
+ * byte, coordinate 4q+t in bits 2t..2t+1; packed[m*stride/4 + q]; fields beyond d are zero. */
+void uqo_pack_levels_i2(const int8_t *lev, int M, int64_t d, int64_t stride, uint8_t *packed)
+{
+    for (int m = 0; m < M; ++m)
+        for (int64_t q = 0; 4 * q < d; ++q) {
+            unsigned byte = 0;
+            for (int t = 0; t < 4; ++t) {
+                int64_t i = 4 * q + t;
+                if (i < d) byte |= ((unsigned)lev[(int64_t)m * stride + i] & 3u) << (2 * t);
+            }
+            packed[(int64_t)m * (stride / 4) + q] = (uint8_t)byte;
+        }
+}
+
 /* Scale indices packed idx_bits (2, 4 or 8) per coordinate, little-endian inside the byte:
  * coordinate i sits at bit (i * idx_bits) % 8 of byte (i * idx_bits) / 8; unused tail bits 0. */
 void uqo_pack_index(const uint8_t *idx, int64_t d, int idx_bits, uint8_t *packed)

@@ -205,6 +205,18 @@ def pack_levels_i4(lev: np.ndarray) -> np.ndarray:
     return packed[:, : (d + 1) // 2]
 
 
+def pack_levels_i2(lev: np.ndarray) -> np.ndarray:
+    """Four 2-bit two's-complement levels per byte (row stride must be a multiple of 4)."""
+    assert lev.dtype == np.int8
+    M, d, stride = _check_g(lev)
+    if M == 1:
+        stride = -(-stride // 4) * 4
+    assert stride % 4 == 0, "the row stride must be a multiple of 4"
+    packed = np.zeros((M, stride // 4), dtype=np.uint8)
+    lib().uqo_pack_levels_i2(_p(lev), M, C.c_int64(d), C.c_int64(stride), _p(packed))
+    return packed[:, : (d + 3) // 4]
+
+
 def pack_index(idx: np.ndarray, idx_bits: int) -> np.ndarray:
     idx = np.ascontiguousarray(idx, dtype=np.uint8)
     per = 8 // idx_bits

@@ -44,10 +44,13 @@ bool layout_ok(const uq_layout *L)
     return true;
 }
 
+bool fmt_known(int fmt) { return fmt == UQ_FMT_I8 || fmt == UQ_FMT_I4X2 || fmt == UQ_FMT_I2X4; }
+
 bool fmt_ok(int fmt, int s_hat)
 {
     if (fmt == UQ_FMT_I8) return s_hat >= 1 && s_hat <= 127;
     if (fmt == UQ_FMT_I4X2) return s_hat >= 1 && s_hat <= 7;
+    if (fmt == UQ_FMT_I2X4) return s_hat == 1;
     return false;
 }
 
@@ -157,7 +160,7 @@ int uq_encode_multi(const uq_layout *L, const void *g, const float *W, const int
 
 int uq_aggregate(const uq_layout *L, const void *lev, int fmt, int32_t *S, void *stream)
 {
-    if (!layout_ok(L) || (fmt != UQ_FMT_I8 && fmt != UQ_FMT_I4X2)) return UQ_ERR_BAD_ARG;
+    if (!layout_ok(L) || !fmt_known(fmt)) return UQ_ERR_BAD_ARG;
     if (L->d > 0 && (lev == nullptr || S == nullptr || !aligned(lev, 16) || !aligned(S, 32)))
         return UQ_ERR_BAD_ARG;
     return finish(uq::launch_aggregate_decode(*L, lev, fmt, nullptr, single_scale(1), nullptr, 0, nullptr, S,
@@ -185,7 +188,7 @@ int uq_decode(const uq_layout *L, const void *src, int src_kind, int fmt, const 
     if (src_kind == UQ_SRC_SUMS)
         return finish(uq::launch_decode_sums(*L, (const int32_t *)src, W, set, idx, idx_bits, out,
                                              (cudaStream_t)stream));
-    if (fmt != UQ_FMT_I8 && fmt != UQ_FMT_I4X2) return UQ_ERR_BAD_ARG;
+    if (!fmt_known(fmt)) return UQ_ERR_BAD_ARG;
     if (S_opt != nullptr && !aligned(S_opt, 32)) return UQ_ERR_BAD_ARG;
     return finish(uq::launch_aggregate_decode(*L, src, fmt, W, set, idx, idx_bits, out, S_opt,
                                               (cudaStream_t)stream));
@@ -195,7 +198,7 @@ int uq_decode_update(const uq_layout *L, const void *lev, int fmt, const float *
                      int N, const uint8_t *idx, int idx_bits, float *theta, float *momentum, float lr, float mu,
                      float wd, float *out_opt, void *stream)
 {
-    if (!layout_ok(L) || W == nullptr || (fmt != UQ_FMT_I8 && fmt != UQ_FMT_I4X2)) return UQ_ERR_BAD_ARG;
+    if (!layout_ok(L) || W == nullptr || !fmt_known(fmt)) return UQ_ERR_BAD_ARG;
     if (!(lr == lr) || !(mu == mu) || !(wd == wd)) return UQ_ERR_BAD_ARG;                  // NaN hyper-parameters
     uq::ScaleSet set;
     if (scales != nullptr) {

@@ -55,6 +55,8 @@ template <int FMT> struct Unit;
 
 template <> struct Unit<UQ_FMT_I8> {
     static constexpr int C = 16;
+    using Q = uint4;                                             // one worker's levels of the unit
+    static __device__ __forceinline__ Q load(const void *p) { return ld_stream(p); }
     // Bytes are biased to unsigned (x ^ 0x80) and added in 16-bit lanes: two lanes per word,
     // M <= 64 workers * 255 < 2^16.  lane layout of word w: even = bytes 0,2; odd = bytes 1,3.
     uint32_t even[4] = {0, 0, 0, 0}, odd[4] = {0, 0, 0, 0};
@@ -83,6 +85,8 @@ template <> struct Unit<UQ_FMT_I8> {
 
 template <> struct Unit<UQ_FMT_I4X2> {
     static constexpr int C = 32;
+    using Q = uint4;
+    static __device__ __forceinline__ Q load(const void *p) { return ld_stream(p); }
     // Nibbles are biased to unsigned (x ^ 8) and added in byte lanes for up to 16 workers
     // (16 * 15 < 256), then widened into 16-bit lanes.
     uint32_t lo8[4] = {0, 0, 0, 0}, hi8[4] = {0, 0, 0, 0};       // byte lanes: even / odd nibbles
@@ -129,6 +133,35 @@ template <> struct Unit<UQ_FMT_I4X2> {
     }
 };
 
+template <> struct Unit<UQ_FMT_I2X4> {
+    static constexpr int C = 32;
+    using Q = uint2;
+    static __device__ __forceinline__ Q load(const void *p) { return ld_stream64(p); }
+    // 2-bit fields are biased to unsigned (x ^ 2, so 1..3) and added in byte lanes: field t of
+    // every byte of word w goes to acc[w][t]; 64 workers * 3 < 256, so a byte lane never carries.
+    uint32_t acc[2][4] = {};
+    __device__ __forceinline__ void add(const uint2 &q)
+    {
+        const uint32_t w[2] = { q.x, q.y };
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const uint32_t b = w[k] ^ 0xAAAAAAAAu;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) acc[k][t] += (b >> (2 * t)) & 0x03030303u;
+        }
+    }
+    __device__ __forceinline__ void finish(int M, int (&s)[32]) const
+    {
+        const int bias = 2 * M;
+#pragma unroll
+        for (int k = 0; k < 2; ++k)
+#pragma unroll
+            for (int y = 0; y < 4; ++y)
+#pragma unroll
+                for (int t = 0; t < 4; ++t) s[16 * k + 4 * y + t] = (int)((acc[k][t] >> (8 * y)) & 0xFFu) - bias;
+    }
+};
+
 // UPDATE selects the variant that also applies the parameter update (kept apart so that the plain
 // reconstruction keeps its register count).
 template <int FMT, int IDXB, bool UPDATE>
@@ -144,21 +177,22 @@ __global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const __grid
     const int64_t row0 = i - (int64_t)lane * C;                    // my warp's first coordinate
     if (row0 >= p.d) return;                                       // warp-uniform
     const bool active = i < p.d;
-    const size_t row_bytes = FMT == UQ_FMT_I8 ? (size_t)p.stride : (size_t)(p.stride >> 1);
+    using Q = typename U::Q;
+    const size_t row_bytes = (size_t)(p.stride >> FMT);            // 8 >> FMT bits per level
 
     U unit;
     uint32_t kw[WORDS];
     if (active) {
-        const char *col = (const char *)p.lev + (size_t)i * 16 / C;
+        const char *col = (const char *)p.lev + (size_t)(i >> FMT);
         int m = 0;
         for (; m + 8 <= p.M; m += 8) {          // eight workers' loads in flight
-            uint4 q[8];
+            Q q[8];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) q[k] = ld_stream(col + (size_t)(m + k) * row_bytes);
+            for (int k = 0; k < 8; ++k) q[k] = U::load(col + (size_t)(m + k) * row_bytes);
 #pragma unroll
             for (int k = 0; k < 8; ++k) unit.add(q[k]);
         }
-        for (; m < p.M; ++m) unit.add(ld_stream(col + (size_t)m * row_bytes));
+        for (; m < p.M; ++m) unit.add(U::load(col + (size_t)m * row_bytes));
         if (MULTI && p.out != nullptr) {
             // idx bits of coordinates i..i+C-1 start at byte i*IB/8 (a multiple of 4 bytes)
             const uint32_t *ip = (const uint32_t *)(p.idx + (size_t)i * IB / 8);
@@ -319,8 +353,9 @@ cudaError_t launch_aggregate_decode(const uq_layout &L, const void *lev, int fmt
     p.lev = lev; p.W = W; p.seg_off = L.seg_off; p.idx = idx; p.out = out; p.S = S;
     p.d = L.d; p.stride = L.worker_stride; p.nseg = L.nseg; p.M = L.M; p.scales = scales;
     p.theta = theta; p.mom = mom; p.lr = lr; p.mu = mu; p.wd = wd;
-    return fmt == UQ_FMT_I8 ? dispatch_levels<UQ_FMT_I8>(p, idx_bits, st)
-                            : dispatch_levels<UQ_FMT_I4X2>(p, idx_bits, st);
+    if (fmt == UQ_FMT_I8) return dispatch_levels<UQ_FMT_I8>(p, idx_bits, st);
+    if (fmt == UQ_FMT_I4X2) return dispatch_levels<UQ_FMT_I4X2>(p, idx_bits, st);
+    return dispatch_levels<UQ_FMT_I2X4>(p, idx_bits, st);
 }
 
 cudaError_t launch_decode_sums(const uq_layout &L, const int32_t *S, const float *W, const ScaleSet &scales,

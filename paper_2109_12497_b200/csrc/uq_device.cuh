@@ -17,6 +17,16 @@ struct ScaleSet {                        // the scale set s_ of the multi-scale 
     int32_t N;
 };
 
+// The low two bits of the eight bytes of (lo, hi), coordinate order kept: byte t of lo lands in
+// bits 2t..2t+1, byte t of hi in bits 8+2t..9+2t (levels -1, 0, 1 as two's-complement 2-bit fields).
+__device__ __forceinline__ uint32_t bytes_to_crumbs(uint32_t lo, uint32_t hi)
+{
+    lo &= 0x03030303u; hi &= 0x03030303u;
+    lo = (lo | (lo >> 6)) & 0x000F000Fu; hi = (hi | (hi >> 6)) & 0x000F000Fu;
+    lo = (lo | (lo >> 12)) & 0x000000FFu; hi = (hi | (hi >> 12)) & 0x000000FFu;
+    return lo | (hi << 8);
+}
+
 // ---------------------------------------------------------------------------------------------
 // loads / stores
 // ---------------------------------------------------------------------------------------------
@@ -27,6 +37,14 @@ __device__ __forceinline__ uint4 ld_stream(const void *p)
     uint4 v;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+// Streaming 64-bit load (8-byte aligned).
+__device__ __forceinline__ uint2 ld_stream64(const void *p)
+{
+    uint2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
     return v;
 }
 

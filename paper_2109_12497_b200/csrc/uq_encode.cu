@@ -4,7 +4,7 @@
 // Algorithm 2 line "Quantize with s*").
 //
 // One streaming pass: a thread owns units of 8 consecutive coordinates (32 B of fp32 or 16 B of
-// bf16 in, 8 B of int8 or 4 B of packed 4-bit levels out); a CTA owns one tile of one worker.
+// bf16 in, 8 B of int8, 4 B of packed 4-bit or 2 B of packed 2-bit levels out); a CTA owns one tile of one worker.
 // A worker's CTA reads only that worker's gradient plus the agreed values W and idx.
 #include "uq_device.cuh"
 
@@ -87,7 +87,8 @@ __device__ __forceinline__ void quantize_unit(const float (&v)[8], const float (
     const uint32_t hi = negate_bytes(gather_bytes<LB>(z[4], z[5], z[6], z[7]), neg_hi);
     if (!store) return;
     if (FMT == UQ_FMT_I8) st_stream((uint2 *)dst, make_uint2(lo, hi));
-    else st_stream((uint32_t *)dst, bytes_to_nibbles(lo, hi));
+    else if (FMT == UQ_FMT_I4X2) st_stream((uint32_t *)dst, bytes_to_nibbles(lo, hi));
+    else st_stream((unsigned short *)dst, (unsigned short)bytes_to_crumbs(lo, hi));
 }
 
 // The sign masks of a unit, from the raw loaded words (before any padding is zeroed).
@@ -168,8 +169,7 @@ __device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, i
         }
         if (overflow && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
         const uint64_t blk = RNG == 32 ? (uint64_t)(i >> 2) : (uint64_t)(i >> 3);
-        char *dst = FMT == UQ_FMT_I8 ? (char *)p.lev + (size_t)m * (size_t)p.stride + i
-                                     : (char *)p.lev + (size_t)m * (size_t)(p.stride >> 1) + (i >> 1);
+        char *dst = (char *)p.lev + (size_t)m * (size_t)(p.stride >> FMT) + (i >> FMT);     // 8 >> FMT bits per level
         quantize_unit<FMT, RNG>(v, inv, p.cap, neg_lo, neg_hi, p.key, (uint32_t)blk, (uint32_t)(blk >> 32), (uint32_t)m,
                                 dst);
     }
@@ -264,8 +264,8 @@ __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, IDXB != 0>::MIN_CTA
     const uint64_t blk0 = RNG == 32 ? (uint64_t)(t0 >> 2) : (uint64_t)(t0 >> 3);           // low bits are 0
     const uint32_t blk_hi = (uint32_t)(blk0 >> 32);
     const uint32_t blk_lo = (uint32_t)blk0 + (uint32_t)tid * BPU;
-    char *lp = FMT == UQ_FMT_I8 ? (char *)p.lev + (size_t)m * (size_t)p.stride + (size_t)t0 + tid * 8
-                                : (char *)p.lev + (size_t)m * (size_t)(p.stride >> 1) + (size_t)(t0 >> 1) + tid * 4;
+    constexpr int UB = 8 >> FMT;                                 // bytes of levels per unit: 8, 4 or 2
+    char *lp = (char *)p.lev + (size_t)m * (size_t)(p.stride >> FMT) + (size_t)(t0 >> FMT) + tid * UB;
     // One straight-line pass over all units, so the compiler can interleave them.  A crossed row
     // runs through the arithmetic too but is not stored: a CTA of the second kind owns it.
 #pragma unroll
@@ -283,7 +283,7 @@ __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, IDXB != 0>::MIN_CTA
         uint32_t neg_lo, neg_hi;
         unit_signs<DT>(q[u], neg_lo, neg_hi);
         quantize_unit<FMT, RNG>(v, inv, p.cap, neg_lo, neg_hi, p.key, blk_lo + u * kThreads * BPU, blk_hi, (uint32_t)m,
-                                lp + u * kThreads * (FMT == UQ_FMT_I8 ? 8 : 4), !((crossed >> u) & 1u));
+                                lp + u * kThreads * UB, !((crossed >> u) & 1u));
     }
     if (overflow && lane < p.scales.N && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
 }
@@ -320,8 +320,11 @@ static cudaError_t dispatch_fmt(const EncodeParams &p, int fmt, int rng_bits, in
     if (fmt == UQ_FMT_I8)
         return rng_bits == 32 ? dispatch_idx<DT, UQ_FMT_I8, 32>(p, idx_bits, st)
                               : dispatch_idx<DT, UQ_FMT_I8, 16>(p, idx_bits, st);
-    return rng_bits == 32 ? dispatch_idx<DT, UQ_FMT_I4X2, 32>(p, idx_bits, st)
-                          : dispatch_idx<DT, UQ_FMT_I4X2, 16>(p, idx_bits, st);
+    if (fmt == UQ_FMT_I4X2)
+        return rng_bits == 32 ? dispatch_idx<DT, UQ_FMT_I4X2, 32>(p, idx_bits, st)
+                              : dispatch_idx<DT, UQ_FMT_I4X2, 16>(p, idx_bits, st);
+    return rng_bits == 32 ? dispatch_idx<DT, UQ_FMT_I2X4, 32>(p, idx_bits, st)
+                          : dispatch_idx<DT, UQ_FMT_I2X4, 16>(p, idx_bits, st);
 }
 
 // idx_bits == 0 selects the single-scale quantizer (scales = {s}).

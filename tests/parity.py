@@ -59,6 +59,8 @@ def run_oracle(w, g_np, W=None, seed=None):
     res["lev_raw"] = lev
     if w.fmt == "i4x2":
         res["lev"] = o.pack_levels_i4(lev)
+    elif w.fmt == "i2x4":
+        res["lev"] = o.pack_levels_i2(lev)
     else:
         res["lev"] = np.ascontiguousarray(lev).view(np.uint8)
     res.update(S=S, out=out)

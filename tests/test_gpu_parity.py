@@ -36,6 +36,8 @@ def test_segmented_workloads_small(name, d, rng_bits):
     ("c2", 2_100_003, 8, {}), ("c2", 2_100_003, 8, dict(rng_bits=32)), ("c3", 2_100_003, 8, {}),
     ("c4", 1_060_013, 16, {}), ("c5", 1_060_013, 16, {}), ("c5", 2_100_003, 8, dict(rng_bits=32, idx_bits=8)),
     ("c3", 2_100_003, 8, dict(dtype=wl.BF16, fmt="i4x2", s=7, scales=(7, 112, 1792))),
+    ("c2", 2_100_003, 8, dict(fmt="i2x4", s=1, scales=(1,))),
+    ("c3", 2_100_003, 8, dict(dtype=wl.BF16, fmt="i2x4", s=1, scales=(1, 16, 256))),
 ])
 def test_mid_size_workloads(name, d, M, kw):
     """A few million coordinates per worker: hundreds of tiles per kernel, a ragged last tile and
@@ -45,7 +47,7 @@ def test_mid_size_workloads(name, d, M, kw):
 
 
 @pytest.mark.parametrize("norm", [wl.NORM_L2, wl.NORM_LINF])
-@pytest.mark.parametrize("fmt,s", [("i8", 127), ("i8", 1), ("i8", 5), ("i4x2", 7), ("i4x2", 1)])
+@pytest.mark.parametrize("fmt,s", [("i8", 127), ("i8", 1), ("i8", 5), ("i4x2", 7), ("i4x2", 1), ("i2x4", 1)])
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
 def test_single_scale_variants(norm, fmt, s, dtype):
     w = wl.scaled("c2", 50021, M=4, norm=norm, fmt=fmt, s=s, scales=(s,), dtype=dtype)
@@ -54,7 +56,7 @@ def test_single_scale_variants(norm, fmt, s, dtype):
 
 @pytest.mark.parametrize("idx_bits,N", [(2, 2), (2, 4), (4, 3), (4, 8), (4, 16), (8, 5), (8, 16)])
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
-@pytest.mark.parametrize("fmt,s,ratio", [("i8", 127, 8), ("i4x2", 7, 16), ("i8", 31, 2)])
+@pytest.mark.parametrize("fmt,s,ratio", [("i8", 127, 8), ("i4x2", 7, 16), ("i8", 31, 2), ("i2x4", 1, 4)])
 def test_multi_scale_variants(idx_bits, N, dtype, fmt, s, ratio):
     if s * ratio ** (N - 1) >= 2 ** 31:
         pytest.skip("scale does not fit int32")
@@ -69,6 +71,20 @@ def test_worker_counts(M):
     for name in ("c1", "c4", "c3"):
         w = wl.scaled(name, 9001, M=M)
         check_parity(w, wl.generate(w))
+
+
+@pytest.mark.parametrize("M", [1, 3, 8, 15, 63, 64])
+@pytest.mark.parametrize("d", [5, 31, 33, 8191, 70001])
+def test_two_bit_levels(M, d):
+    """Levels -1, 0, 1 at four per byte: every worker count up to the byte-lane limit of the
+    aggregation, sizes around the 32-coordinate unit, and the format limit s = 1."""
+    w = wl.scaled("c1", d, M=M, fmt="i2x4", s=1, scales=(1,))
+    r = check_parity(w, wl.generate(w))
+    assert set(np.unique(r["ref"]["lev_raw"]).tolist()) <= {-1, 0, 1}
+    from paper_2109_12497_b200.pipeline import from_workload
+    bad = from_workload(dataclasses.replace(w, s=2, scales=(2,)))             # the format takes s = 1 only
+    with pytest.raises(B.UqError):
+        bad.encode(to_device(w, wl.generate(w)), 0)
 
 
 def test_seed_changes_the_draws_only():

@@ -16,7 +16,16 @@ pytestmark = pytest.mark.gpu
 @pytest.mark.parametrize("lr,mu,wd,use_mom", [(0.1, 0.0, 0.0, False), (0.1, 0.9, 5e-4, True), (0.05, 0.9, 0.0, True),
                                               (0.1, 0.0, 5e-4, False)])
 def test_fused_update_matches_oracle(name, d, lr, mu, wd, use_mom):
-    w = wl.scaled(name, d)
+    _fused_update_case(wl.scaled(name, d), lr, mu, wd, use_mom)
+
+
+def test_fused_update_two_bit_levels():
+    _fused_update_case(wl.scaled("c2", 100_003, fmt="i2x4", s=1, scales=(1,)), 0.1, 0.9, 5e-4, True)
+    _fused_update_case(wl.scaled("c3", 70_001, fmt="i2x4", s=1, scales=(1, 16, 256)), 0.1, 0.0, 0.0, False)
+
+
+def _fused_update_case(w, lr, mu, wd, use_mom):
+    d = w.d
     r = run_gpu(w, wl.generate(w))
     q = r["q"]
     rng = np.random.default_rng(d)

@@ -209,3 +209,17 @@ def test_int4_packing_layout():
     packed = o.pack_levels_i4(padded[:, :5])
     assert packed.shape == (2, 3)
     assert packed[0].tolist() == [0x79, 0xF0, 0x03] and packed[1].tolist() == [0x21, 0x43, 0x05]
+
+
+def test_int2_packing_layout():
+    """Four two's-complement 2-bit fields per byte, the lowest coordinate in the lowest bits."""
+    lev = np.array([[-1, 1, 0, -1, 1], [0, 0, 1, 1, -1]], dtype=np.int8)
+    padded = np.zeros((2, 32), dtype=np.int8); padded[:, :5] = lev
+    packed = o.pack_levels_i2(padded[:, :5])
+    assert packed.shape == (2, 2)
+    # row 0: fields 11 01 00 11 -> 0b11000111, then 01;   row 1: 00 00 01 01 -> 0b01010000, then 11
+    assert packed[0].tolist() == [0b11000111, 0b01] and packed[1].tolist() == [0b01010000, 0b11]
+    # unpacking with sign extension gives the levels back
+    for m in range(2):
+        bits = np.repeat(packed[m], 4) >> np.tile(np.arange(4) * 2, 2) & 3
+        assert (((bits ^ 2) - 2)[:5] == lev[m]).all()
