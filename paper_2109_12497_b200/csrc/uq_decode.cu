@@ -244,24 +244,23 @@ __global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const __grid
         // from registers into the parameters (and the momentum buffer)
         const bool has_mom = p.mom != nullptr;
         if (full) {
-            // 16 coordinates at a time: their eight 16-byte loads are issued together
+            // 16 coordinates at a time as 256-bit accesses: a lane's 32 bytes are one whole sector,
+            // so nothing depends on L1 keeping the other half of a sector until the next access
 #pragma unroll
             for (int e0 = 0; e0 < C; e0 += 16) {
-                float4 th[4], bf[4];
+                float th[2][8], bf[2][8] = {};
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    th[k] = *(const float4 *)(p.theta + i + e0 + 4 * k);
-                    bf[k] = has_mom ? *(const float4 *)(p.mom + i + e0 + 4 * k) : make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int k = 0; k < 2; ++k) {
+                    ld256(p.theta + i + e0 + 8 * k, th[k]);
+                    if (has_mom) ld256(p.mom + i + e0 + 8 * k, bf[k]);
                 }
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const int e = e0 + 4 * k;
-                    sgd_coordinate(r[e + 0], th[k].x, bf[k].x, has_mom, p.lr, p.mu, p.wd);
-                    sgd_coordinate(r[e + 1], th[k].y, bf[k].y, has_mom, p.lr, p.mu, p.wd);
-                    sgd_coordinate(r[e + 2], th[k].z, bf[k].z, has_mom, p.lr, p.mu, p.wd);
-                    sgd_coordinate(r[e + 3], th[k].w, bf[k].w, has_mom, p.lr, p.mu, p.wd);
-                    *(float4 *)(p.theta + i + e) = th[k];
-                    if (has_mom) *(float4 *)(p.mom + i + e) = bf[k];
+                for (int k = 0; k < 2; ++k) {
+#pragma unroll
+                    for (int t = 0; t < 8; ++t)
+                        sgd_coordinate(r[e0 + 8 * k + t], th[k][t], bf[k][t], has_mom, p.lr, p.mu, p.wd);
+                    st256(p.theta + i + e0 + 8 * k, th[k]);
+                    if (has_mom) st256(p.mom + i + e0 + 8 * k, bf[k]);
                 }
             }
         } else {

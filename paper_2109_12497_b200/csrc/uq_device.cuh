@@ -64,6 +64,21 @@ __device__ __forceinline__ uint8x ld_stream256(const void *p)
     return v;
 }
 
+// 256-bit load / store of data that the same kernel both reads and writes (coherent path).
+__device__ __forceinline__ void ld256(const void *p, float (&f)[8])
+{
+    asm volatile("ld.global.L1::no_allocate.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(f[0]), "=f"(f[1]), "=f"(f[2]), "=f"(f[3]), "=f"(f[4]), "=f"(f[5]), "=f"(f[6]), "=f"(f[7])
+                 : "l"(p) : "memory");
+}
+
+__device__ __forceinline__ void st256(void *p, const float (&f)[8])
+{
+    asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 :: "l"(p), "f"(f[0]), "f"(f[1]), "f"(f[2]), "f"(f[3]), "f"(f[4]), "f"(f[5]), "f"(f[6]), "f"(f[7])
+                 : "memory");
+}
+
 __device__ __forceinline__ void st_stream256(void *p, const uint32_t (&w)[8])
 {
     asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
