@@ -380,3 +380,75 @@ void uqo_pack_index(const uint8_t *idx, int64_t d, int idx_bits, uint8_t *packed
         packed[q] = (uint8_t)byte;
     }
 }
+
+/* ------------------------------------------------------------------------------------------
+ * GlobalRandKMaxNorm / GlobalRandKMaxNormMultiScale (Sections "GlobalRandKMaxNorm Compression"
+ * and "GlobalRandKMaxNormMultiScale Compression"): every worker keeps the same K coordinates,
+ * chosen uniformly, and the quantizer of Algorithm 1 / 2 runs on the K-vector.
+ *
+ * Reading (the paper says only "choosing K coordinates uniformly"): the K coordinates are
+ * distinct; they are sel[t] = pi(t), t = 0..K-1, for a pseudo-random permutation pi of
+ * [0, d) keyed by the shared seed, so all workers agree without communicating.  pi is an
+ * alternating Feistel network on b = max(2, ceil(log2 d)) bits whose round function is a
+ * Philox4x32-10 word, restricted to [0, d) by cycle walking (apply the network until the
+ * value is below d; 2^b < 2d, so a step leaves the range with probability < 1/2).  The
+ * network has 8 rounds, 24 when b < 8: round functions of one to three bits carry so little
+ * randomness that a short network visibly favours some orderings of a tiny domain.
+ * No rescaling by d/K: the paper states none.
+ * ------------------------------------------------------------------------------------------ */
+static uint64_t randk_network(uint64_t x, int b, uint64_t seed)
+{
+    int a = b / 2, c = b - a;                         /* widths of the left and right part */
+    uint64_t L = x >> c, R = x & (((uint64_t)1 << c) - 1);
+    const uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    const uint32_t rounds = b < 8 ? 24u : 8u;
+    for (uint32_t r = 0; r < rounds; ++r) {
+        /* counter word 3 is a tag that the rounding draws (which use 0 there) never use */
+        const uint32_t ctr[4] = { (uint32_t)R, r, 0u, 0x4B646E52u };
+        uint32_t out[4];
+        uqo_philox4x32_10(ctr, key, out);
+        const uint64_t newR = L ^ ((uint64_t)out[0] & (((uint64_t)1 << a) - 1));
+        L = R; R = newR;                              /* the parts swap, and so do their widths */
+        const int t = a; a = c; c = t;
+    }
+    return (L << c) | R;                              /* an even number of rounds: the widths are back in place */
+}
+
+void uqo_randk_indices(int64_t d, int64_t K, uint64_t seed, int64_t *sel)
+{
+    int b = 2;
+    while (((int64_t)1 << b) < d) ++b;
+    for (int64_t t = 0; t < K; ++t) {
+        uint64_t x = (uint64_t)t;
+        do x = randk_network(x, b, seed); while (x >= (uint64_t)d);
+        sel[t] = (int64_t)x;
+    }
+}
+
+/* gk[m][t] = g[m][sel[t]]; elements t = K .. strideK-1 of every row are zero. */
+void uqo_randk_gather(const void *g, int dtype, int M, int64_t stride, int64_t K, const int64_t *sel,
+                      void *gk, int64_t strideK)
+{
+    const size_t eb = dtype == 0 ? 4 : 2;
+    memset(gk, 0, (size_t)M * (size_t)strideK * eb);
+    for (int m = 0; m < M; ++m)
+        for (int64_t t = 0; t < K; ++t)
+            memcpy((char *)gk + ((size_t)m * (size_t)strideK + (size_t)t) * eb,
+                   (const char *)g + ((size_t)m * (size_t)stride + (size_t)sel[t]) * eb, eb);
+}
+
+/* out[sel[t]] = vals[t] (vals == NULL: 0), the other coordinates of out are left alone. */
+void uqo_randk_scatter(int64_t K, const int64_t *sel, const float *vals, float *out)
+{
+    for (int64_t t = 0; t < K; ++t) out[sel[t]] = vals ? vals[t] : 0.0f;
+}
+
+/* Algorithm 1 / 2, line "Update parameters", with a gradient that is zero off the chosen set:
+ * theta[sel[t]] -= lr * vals[t] (binary32, product then difference). */
+void uqo_randk_update(int64_t K, const int64_t *sel, const float *vals, float *theta, float lr)
+{
+    for (int64_t t = 0; t < K; ++t) {
+        const float step = lr * vals[t];
+        theta[sel[t]] = theta[sel[t]] - step;
+    }
+}

@@ -234,3 +234,45 @@ def sgd_update(g_hat, theta, mom=None, lr=0.1, mu=0.0, wd=0.0):
     lib().uqo_sgd_update(_p(g_hat), C.c_int64(g_hat.size), _p(theta), _p(mom), C.c_float(lr), C.c_float(mu),
                          C.c_float(wd))
     return theta, mom
+
+
+# ---------------------------------------------------------------------------------------------
+# GlobalRandK (Sections "GlobalRandKMaxNorm Compression", "GlobalRandKMaxNormMultiScale Compression")
+# ---------------------------------------------------------------------------------------------
+
+def randk_indices(d: int, K: int, seed: int) -> np.ndarray:
+    """The K distinct coordinates every worker keeps at this seed, in selection order."""
+    assert 0 <= K <= d
+    sel = np.zeros(K, dtype=np.int64)
+    lib().uqo_randk_indices(C.c_int64(d), C.c_int64(K), C.c_uint64(seed), _p(sel))
+    return sel
+
+
+def randk_gather(g: np.ndarray, sel: np.ndarray) -> np.ndarray:
+    """[M, K] view (row stride = K rounded up to 32) of the chosen coordinates of every worker."""
+    M, d, stride = _check_g(g)
+    sel = np.ascontiguousarray(sel, dtype=np.int64)
+    K = sel.size
+    strideK = max(32, -(-K // 32) * 32)
+    gk = np.zeros((M, strideK), dtype=g.dtype)
+    lib().uqo_randk_gather(_p(g), _dtype_of(g), M, C.c_int64(stride), C.c_int64(K), _p(sel), _p(gk),
+                           C.c_int64(strideK))
+    return gk[:, :K]
+
+
+def randk_scatter(sel: np.ndarray, vals, out: np.ndarray) -> np.ndarray:
+    """out with out[sel[t]] = vals[t] (vals None: 0); modifies and returns out (float32)."""
+    sel = np.ascontiguousarray(sel, dtype=np.int64)
+    assert out.dtype == np.float32 and out.flags.c_contiguous
+    vals = None if vals is None else np.ascontiguousarray(vals, dtype=np.float32)
+    lib().uqo_randk_scatter(C.c_int64(sel.size), _p(sel), _p(vals), _p(out))
+    return out
+
+
+def randk_update(sel: np.ndarray, vals: np.ndarray, theta: np.ndarray, lr: float) -> np.ndarray:
+    """A copy of theta after theta[sel] -= lr * vals."""
+    sel = np.ascontiguousarray(sel, dtype=np.int64)
+    vals = np.ascontiguousarray(vals, dtype=np.float32)
+    theta = np.array(theta, dtype=np.float32, copy=True)
+    lib().uqo_randk_update(C.c_int64(sel.size), _p(sel), _p(vals), _p(theta), C.c_float(lr))
+    return theta
