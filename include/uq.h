@@ -65,7 +65,8 @@ enum { UQ_SRC_LEVELS = 0, UQ_SRC_SUMS = 1 };   /* what uq_decode reads */
 enum {
     UQ_STATUS_NONFINITE = 1,      /* a NaN/Inf input or a non-finite scale */
     UQ_STATUS_BAD_SEGMENTS = 2,   /* seg_off not non-decreasing from 0 to d */
-    UQ_STATUS_SCALE_OVERFLOW = 4  /* s / W is not finite (W subnormal-small) */
+    UQ_STATUS_SCALE_OVERFLOW = 4, /* s / W is not finite (W subnormal-small) */
+    UQ_STATUS_BAD_INDEX = 8       /* a chosen-coordinate index outside [0, d) (uq_randk_*) */
 };
 
 #define UQ_MAX_WORKERS 64
@@ -240,6 +241,47 @@ int uq_decode(const uq_layout *layout, const void *src, int src_kind, int fmt, c
 int uq_decode_update(const uq_layout *layout, const void *lev, int fmt, const float *W, int s,
                      const int32_t *scales, int N, const uint8_t *idx, int idx_bits, float *theta,
                      float *momentum, float lr, float mu, float wd, float *out_opt, void *stream);
+
+/*
+ * GlobalRandKMaxNorm / GlobalRandKMaxNormMultiScale — Sections "GlobalRandKMaxNorm Compression"
+ * and "GlobalRandKMaxNormMultiScale Compression": every worker keeps the same K coordinates,
+ * chosen uniformly at every iteration, and the quantizer of Algorithm 1 / 2 runs on them.
+ * The calls below add the choice + gather before, and the scatter after, the dense calls above,
+ * which then run on the compact [M][gk_stride] buffer with d = K and one segment.
+ *
+ * Reading of "choosing K coordinates uniformly": K distinct coordinates sel[t] = pi(t),
+ * t = 0..K-1, where pi is a pseudo-random permutation of [0, d) keyed by `seed` (all workers
+ * hold the same seed, so they agree without communicating): an alternating Feistel network on
+ * b = max(2, ceil(log2 d)) bits (left part b/2 bits; right part the rest; the parts swap each
+ * round; new right = old left XOR the low bits of word 0 of Philox4x32-10 with key = seed and
+ * counter = (old right, round, 0, 0x4B646E52)), 8 rounds (24 when b < 8), repeated until the
+ * value is below d.  No d/K rescaling is applied: the paper states none.
+ *
+ * uq_randk_gather: sel[t] as above and gk[m][t] = g[m][sel[t]] for every worker.
+ *   layout   in   the dense layout of g (d, worker_stride, M, dtype; seg_off / nseg are ignored:
+ *                 the K-vector is one vector with one scale)
+ *   K             0 <= K <= d
+ *   sel      out  [K] int64 device, 8-byte aligned, selection order (not sorted)
+ *   gk       out  [M][gk_stride] elements of layout->dtype, 16-byte aligned; gk_stride is a
+ *                 multiple of 32 and >= K; elements K .. gk_stride-1 of every row are zeroed
+ *   status        UQ_STATUS_BAD_INDEX if a cycle walk did not end within 256 steps
+ *                 (probability below 2^-256; the coordinate t is used instead)
+ * uq_randk_scatter: out[sel[t]] = vals[t] for t < K; vals = NULL writes zeros (clearing the
+ *   entries of an earlier step).  out is [d] float; the other coordinates are not touched.
+ * uq_randk_update: theta[sel[t]] = theta[sel[t]] - lr * vals[t] (binary32, product then
+ *   difference): Algorithm 1 / 2 line "Update parameters" for a gradient that is zero off the
+ *   chosen set.
+ *   sel entries outside [0, d) are skipped and set UQ_STATUS_BAD_INDEX; sel must hold distinct
+ *   values (as uq_randk_gather writes them), otherwise the result of a repeated entry is
+ *   whichever write lands last.
+ * Errors: UQ_ERR_BAD_ARG (K outside 0..d, bad stride or alignment, NaN lr), UQ_ERR_CUDA.
+ */
+int uq_randk_gather(const uq_layout *layout, const void *g, int64_t K, uint64_t seed, int64_t *sel,
+                    void *gk, int64_t gk_stride, uint32_t *status, void *stream);
+int uq_randk_scatter(int64_t d, int64_t K, const int64_t *sel, const float *vals, float *out,
+                     uint32_t *status, void *stream);
+int uq_randk_update(int64_t d, int64_t K, const int64_t *sel, const float *vals, float *theta,
+                    float lr, uint32_t *status, void *stream);
 
 #ifdef __cplusplus
 }

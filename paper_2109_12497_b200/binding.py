@@ -21,12 +21,12 @@ UQ_F32, UQ_BF16 = 0, 1
 UQ_NORM_LINF, UQ_NORM_L2 = 0, 2
 UQ_FMT_I8, UQ_FMT_I4X2, UQ_FMT_I2X4 = 0, 1, 2
 UQ_SRC_LEVELS, UQ_SRC_SUMS = 0, 1
-UQ_STATUS_NONFINITE, UQ_STATUS_BAD_SEGMENTS, UQ_STATUS_SCALE_OVERFLOW = 1, 2, 4
+UQ_STATUS_NONFINITE, UQ_STATUS_BAD_SEGMENTS, UQ_STATUS_SCALE_OVERFLOW, UQ_STATUS_BAD_INDEX = 1, 2, 4, 8
 
 EXPORTS = (
     "uq_version", "uq_last_cuda_error", "uq_error_string", "uq_workspace_bytes", "uq_index_bytes",
     "uq_agree_scale", "uq_agree_scale_static", "uq_encode_single", "uq_select_scale_multi", "uq_encode_multi",
-    "uq_aggregate", "uq_decode", "uq_decode_update",
+    "uq_aggregate", "uq_decode", "uq_decode_update", "uq_randk_gather", "uq_randk_scatter", "uq_randk_update",
 )
 
 
@@ -82,6 +82,10 @@ def lib() -> C.CDLL:
         L.uq_decode.argtypes = [LP, P, I, I, P, I, P, I, P, I, P, P, P]
         F = C.c_float
         L.uq_decode_update.argtypes = [LP, P, I, P, I, P, I, P, I, P, P, F, F, F, P, P]
+        I64 = C.c_int64
+        L.uq_randk_gather.argtypes = [LP, P, I64, U64, P, P, I64, P, P]
+        L.uq_randk_scatter.argtypes = [I64, I64, P, P, P, P, P]
+        L.uq_randk_update.argtypes = [I64, I64, P, P, P, F, P, P]
         for name in EXPORTS[5:]:
             getattr(L, name).restype = I
         _lib = L
@@ -260,3 +264,37 @@ def uq_decode_update(layout: Layout, lev: torch.Tensor, fmt: int, W: torch.Tenso
     _check("uq_decode_update", lib().uq_decode_update(
         layout.ref(), _ptr(lev), fmt, _ptr(W), s, arr, N, _ptr(idx) if scales is not None else None, idx_bits,
         _ptr(theta), _ptr(momentum), lr, mu, wd, _ptr(out), _stream()))
+
+
+def uq_randk_gather(layout: Layout, g: torch.Tensor, K: int, seed: int, sel: torch.Tensor, gk: torch.Tensor,
+                    status: Optional[torch.Tensor] = None) -> None:
+    """The K coordinates all workers keep at this seed (sel, int64 [K]) and their values
+    gk[m, t] = g[m, sel[t]] in a compact [M, gk_stride] buffer whose row padding is zeroed."""
+    layout.check_g(g)
+    if gk.dtype != layout.dtype or gk.dim() != 2 or gk.shape[0] != layout.M or not gk.is_contiguous():
+        raise ValueError(f"uq: gk must be a contiguous [{layout.M}, gk_stride] {layout.dtype} tensor")
+    layout.check_vec(sel, torch.int64, K, "sel")
+    _check("uq_randk_gather", lib().uq_randk_gather(
+        layout.ref(), _ptr(g), K, seed, _ptr(sel), _ptr(gk), gk.shape[1], _ptr(status), _stream()))
+
+
+def _check_randk(d: int, K: int, sel: torch.Tensor, vals: Optional[torch.Tensor], dst: torch.Tensor, what: str):
+    for t, dt, n, name in ((sel, torch.int64, K, "sel"), (vals, torch.float32, K, "vals"), (dst, torch.float32, d, what)):
+        if t is not None and (t.dtype != dt or t.dim() != 1 or t.numel() < n or not t.is_contiguous()):
+            raise ValueError(f"uq: {name} must be a contiguous 1-D {dt} tensor with >= {n} elements")
+
+
+def uq_randk_scatter(d: int, K: int, sel: torch.Tensor, vals: Optional[torch.Tensor], out: torch.Tensor,
+                     status: Optional[torch.Tensor] = None) -> None:
+    """out[sel[t]] = vals[t] (vals None: 0); the other coordinates of out are left alone."""
+    _check_randk(d, K, sel, vals, out, "out")
+    _check("uq_randk_scatter", lib().uq_randk_scatter(d, K, _ptr(sel), _ptr(vals), _ptr(out), _ptr(status),
+                                                      _stream()))
+
+
+def uq_randk_update(d: int, K: int, sel: torch.Tensor, vals: torch.Tensor, theta: torch.Tensor, lr: float,
+                    status: Optional[torch.Tensor] = None) -> None:
+    """theta[sel[t]] -= lr * vals[t]."""
+    _check_randk(d, K, sel, vals, theta, "theta")
+    _check("uq_randk_update", lib().uq_randk_update(d, K, _ptr(sel), _ptr(vals), _ptr(theta), lr, _ptr(status),
+                                                    _stream()))

@@ -17,6 +17,10 @@ cudaError_t launch_aggregate_decode(const uq_layout &L, const void *lev, int fmt
                                     float lr = 0.0f, float mu = 0.0f, float wd = 0.0f);
 cudaError_t launch_decode_sums(const uq_layout &L, const int32_t *S, const float *W, const ScaleSet &scales,
                                const uint8_t *idx, int idx_bits, float *out, cudaStream_t st);
+cudaError_t launch_randk_gather(const uq_layout &L, const void *g, int64_t K, uint64_t seed, int64_t *sel,
+                                void *gk, int64_t gk_stride, uint32_t *status, cudaStream_t st);
+cudaError_t launch_randk_scatter(int64_t d, int64_t K, const int64_t *sel, const float *vals, float *dst, bool update,
+                                 float lr, uint32_t *status, cudaStream_t st);
 }  // namespace uq
 
 namespace {
@@ -215,6 +219,41 @@ int uq_decode_update(const uq_layout *L, const void *lev, int fmt, const float *
     if (L->d == 0) return UQ_OK;
     return finish(uq::launch_aggregate_decode(*L, lev, fmt, W, set, idx, idx_bits, out_opt, nullptr, (cudaStream_t)stream,
                                               theta, momentum, lr, mu, wd));
+}
+
+int uq_randk_gather(const uq_layout *L, const void *g, int64_t K, uint64_t seed, int64_t *sel, void *gk,
+                    int64_t gk_stride, uint32_t *status, void *stream)
+{
+    if (L == nullptr) return UQ_ERR_BAD_ARG;
+    uq_layout dense = *L;                         // segments do not apply to the K-vector
+    dense.seg_off = nullptr;
+    dense.nseg = 1;
+    if (!layout_ok(&dense) || !aligned(status, 4)) return UQ_ERR_BAD_ARG;
+    if (K < 0 || K > dense.d || gk_stride < K || (gk_stride & 31) != 0) return UQ_ERR_BAD_ARG;
+    if (gk_stride > 0 && (gk == nullptr || !aligned(gk, 16))) return UQ_ERR_BAD_ARG;
+    if (K > 0 && (g == nullptr || sel == nullptr || !aligned(g, 16) || !aligned(sel, 8))) return UQ_ERR_BAD_ARG;
+    return finish(uq::launch_randk_gather(dense, g, K, seed, sel, gk, gk_stride, status, (cudaStream_t)stream));
+}
+
+static int randk_scatter_common(int64_t d, int64_t K, const int64_t *sel, const float *vals, float *dst, bool update,
+                                float lr, uint32_t *status, void *stream)
+{
+    if (d < 0 || d > (int64_t)1 << 40 || K < 0 || K > d || !aligned(status, 4)) return UQ_ERR_BAD_ARG;
+    if (K > 0 && (sel == nullptr || dst == nullptr || !aligned(sel, 8) || !aligned(dst, 4))) return UQ_ERR_BAD_ARG;
+    if (!aligned(vals, 4) || (update && (vals == nullptr && K > 0)) || !(lr == lr)) return UQ_ERR_BAD_ARG;
+    return finish(uq::launch_randk_scatter(d, K, sel, vals, dst, update, lr, status, (cudaStream_t)stream));
+}
+
+int uq_randk_scatter(int64_t d, int64_t K, const int64_t *sel, const float *vals, float *out, uint32_t *status,
+                     void *stream)
+{
+    return randk_scatter_common(d, K, sel, vals, out, false, 0.0f, status, stream);
+}
+
+int uq_randk_update(int64_t d, int64_t K, const int64_t *sel, const float *vals, float *theta, float lr,
+                    uint32_t *status, void *stream)
+{
+    return randk_scatter_common(d, K, sel, vals, theta, true, lr, status, stream);
 }
 
 }  // extern "C"

@@ -140,7 +140,7 @@ __device__ __forceinline__ int64_t segment_end(const int64_t *__restrict__ seg_o
 }
 
 // ---------------------------------------------------------------------------------------------
-// Philox4x32-10, counter = (block low, block high, worker, 0), key = seed
+// Philox4x32-10, counter = (block low, block high, worker, tag), key = seed; the rounding draws use tag 0
 // ---------------------------------------------------------------------------------------------
 
 struct PhiloxKey { uint32_t k0[10], k1[10]; };   // the ten round keys (uniform over the grid)
@@ -157,9 +157,10 @@ __host__ __device__ __forceinline__ PhiloxKey philox_key(uint64_t seed)
     return k;
 }
 
-__device__ __forceinline__ uint4 philox4x32_10(const PhiloxKey &k, uint32_t block_lo, uint32_t block_hi, uint32_t worker)
+__device__ __forceinline__ uint4 philox4x32_10(const PhiloxKey &k, uint32_t block_lo, uint32_t block_hi, uint32_t worker,
+                                               uint32_t tag = 0u)
 {
-    uint32_t c0 = block_lo, c1 = block_hi, c2 = worker, c3 = 0u;
+    uint32_t c0 = block_lo, c1 = block_hi, c2 = worker, c3 = tag;
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
         uint64_t p0 = (uint64_t)0xD2511F53u * c0;

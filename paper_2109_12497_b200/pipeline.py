@@ -86,6 +86,54 @@ class Quantizer:
         return int(self.status.item())
 
 
+class RandKQuantizer:
+    """GlobalRandKMaxNorm / GlobalRandKMaxNormMultiScale: the K coordinates of this step's shared
+    choice are gathered into a compact buffer, the dense quantizer (single- or multi-scale) runs
+    on it as one vector, and the K reconstructed values are scattered back."""
+
+    def __init__(self, M: int, d: int, K: int, dtype: torch.dtype = torch.float32, **quantizer_args):
+        if not 0 <= K <= d:
+            raise ValueError("uq: K must lie in 0..d")
+        quantizer_args.pop("seg_off", None)                  # the K-vector is one vector with one scale
+        dev = torch.device(quantizer_args.get("device", "cuda"))
+        self.M, self.d, self.K = M, d, K
+        self.dense_layout = B.Layout(M, d, -(-d // 32) * 32, dtype, None)
+        self.inner = Quantizer(M, K, dtype, **quantizer_args)
+        self.sel = torch.empty(max(K, 1), dtype=torch.int64, device=dev)
+        self.gk = torch.empty((M, self.inner.stride), dtype=dtype, device=dev)
+        self.status = self.inner.status
+
+    def gather(self, g: torch.Tensor, seed: int) -> None:
+        B.uq_randk_gather(self.dense_layout, g, self.K, seed, self.sel, self.gk, self.status)
+
+    def quantize(self, seed: int) -> torch.Tensor:
+        """Agree-scale, [select], encode, aggregate + reconstruct on the compact buffer -> [K] values."""
+        return self.inner.step(self.gk, seed)
+
+    def scatter(self, out: torch.Tensor) -> None:
+        B.uq_randk_scatter(self.d, self.K, self.sel, self.inner.out, out, self.status)
+
+    def clear(self, out: torch.Tensor) -> None:
+        """Zero the entries of ``out`` that the last scatter wrote."""
+        B.uq_randk_scatter(self.d, self.K, self.sel, None, out, self.status)
+
+    def update(self, theta: torch.Tensor, lr: float) -> None:
+        B.uq_randk_update(self.d, self.K, self.sel, self.inner.out, theta, lr, self.status)
+
+    def step(self, g: torch.Tensor, out: torch.Tensor, seed: int = 0) -> torch.Tensor:
+        """g: [M, stride] gradients -> out (dense [d], zero off the chosen set if it was zero before)."""
+        self.gather(g, seed)
+        self.quantize(seed)
+        self.scatter(out)
+        return out
+
+    def kernels_per_step(self) -> int:
+        return 2 + self.inner.kernels_per_step() if self.K > 0 else 1
+
+    def status_bits(self) -> int:
+        return int(self.status.item())
+
+
 def from_workload(w, keep_sums: bool = False, device="cuda") -> Quantizer:
     """A Quantizer configured like a ``workloads.Workload``."""
     from . import workloads as wl

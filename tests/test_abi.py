@@ -36,7 +36,7 @@ def test_constants_match_the_header():
     for name in ("UQ_OK", "UQ_ERR_BAD_ARG", "UQ_ERR_CUDA", "UQ_ERR_UNSUPPORTED", "UQ_ERR_WORKSPACE",
                  "UQ_F32", "UQ_BF16", "UQ_NORM_LINF", "UQ_NORM_L2", "UQ_FMT_I8", "UQ_FMT_I4X2", "UQ_FMT_I2X4",
                  "UQ_SRC_LEVELS", "UQ_SRC_SUMS", "UQ_STATUS_NONFINITE", "UQ_STATUS_BAD_SEGMENTS",
-                 "UQ_STATUS_SCALE_OVERFLOW"):
+                 "UQ_STATUS_SCALE_OVERFLOW", "UQ_STATUS_BAD_INDEX"):
         m = re.search(rf"\b{name}\s*=\s*(\d+)", text)
         assert m and int(m.group(1)) == getattr(B, name), name
 
