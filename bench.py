@@ -236,6 +236,55 @@ def time_graph_replay(q, g, w, reps):
     return e0.elapsed_time(e1) / reps
 
 
+def time_randk(w, g, K, reps):
+    """GlobalRandK step on the workload's gradients: choose + gather K coordinates, the dense
+    stages on the K-vector, sparse parameter update.  ms per step as stream launches and as a
+    CUDA-graph replay (K is tiny, so launch latency sets the time; the replay repeats one seed
+    and is a latency figure only)."""
+    import torch
+    from paper_2109_12497_b200.pipeline import randk_from_workload
+    rq = randk_from_workload(w, K)
+    theta = torch.zeros(max(w.d, 1), dtype=torch.float32, device="cuda")
+
+    def step(seed):
+        rq.gather(g, seed)
+        rq.quantize(seed)
+        rq.update(theta, 0.1)
+
+    st = torch.cuda.current_stream()
+    for k in range(3):
+        step(k)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(st)
+    for k in range(reps):
+        step(100 + k)
+    e1.record(st)
+    torch.cuda.synchronize()
+    ms_stream = e0.elapsed_time(e1) / reps
+    side = torch.cuda.Stream()
+    side.wait_stream(st)
+    with torch.cuda.stream(side):
+        step(7)
+    st.wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step(7)
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(reps):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return {"K": K, "ms_per_step": round(ms_stream, 5), "cuda_graph_ms_per_step": round(e0.elapsed_time(e1) / reps, 5),
+            "kernels_per_step": rq.kernels_per_step(), "status_word": rq.status_bits(),
+            "note": "choice + gather, agree-scale, [select], encode, aggregate + reconstruct, sparse update; "
+                    "latency-bound (K values per worker)"}
+
+
 def time_fused_update(q, w, reps):
     """Mean ms of the fused aggregate + reconstruct + SGD-with-momentum kernel alone (the levels
     are those of the last step; it replaces aggregate_decode when the caller wants the update)."""
@@ -275,7 +324,7 @@ def resolve_workload(name, d=None, rng_bits=None):
     return w
 
 
-def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=False):
+def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=False, randk_K=0):
     """Times one workload on the current device.  Returns a dict of raw numbers."""
     import torch
     from paper_2109_12497_b200.pipeline import from_workload
@@ -317,6 +366,8 @@ def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=F
     res["ms"], res["stages_ms"] = time_device_resident(q, g_dev, w, steps, warmup, barrier)
     res["encode_other_ms"] = time_encode_other_mode(q, g_dev, w, min(steps, 10))
     res["update_ms"] = time_fused_update(q, w, min(steps, 10))
+    if randk_K:
+        res["randk"] = time_randk(w, g_dev, min(randk_K, w.d), 50)
     res["h2d"], res["d2h"], res["e2e_ms"] = 0, 0, None
     if want_e2e:
         out_host = torch.empty(w.d, dtype=torch.float32, pin_memory=True)
@@ -429,7 +480,8 @@ def gpu_main(args):
 
     sampler = ClockSampler(local)
     sampler.start()
-    res = bench_workload(w, args.steps, args.warmup, barrier, threads, want_e2e=not args.no_e2e)
+    res = bench_workload(w, args.steps, args.warmup, barrier, threads, want_e2e=not args.no_e2e,
+                         randk_K=0 if args.no_extra else 10_000)
     clocks = sampler.stop()
 
     ms, e2e_ms = max_over_ranks([res["ms"], res["e2e_ms"] or float("nan")], "cuda")
@@ -465,6 +517,8 @@ def gpu_main(args):
         },
         "kernels": summ["kernels"],
     }
+    if "randk" in res:
+        line["global_randk"] = res["randk"]
     if rank == 0 and world == 1:
         # the other four workloads (parity-test cases; reported for context, a few steps each)
         if not args.no_extra and args.d is None:

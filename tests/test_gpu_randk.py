@@ -10,19 +10,14 @@ import torch
 from oracle import uq_oracle as o
 from paper_2109_12497_b200 import binding as B
 from paper_2109_12497_b200 import workloads as wl
-from paper_2109_12497_b200.pipeline import RandKQuantizer
+from paper_2109_12497_b200.pipeline import randk_from_workload
 from parity import FP32_RTOL, check_parity, to_device
 
 pytestmark = pytest.mark.gpu
 
 
 def _randk(w, K):
-    multi = w.quantizer == "multi"
-    return RandKQuantizer(
-        w.M, w.d, K, torch.float32 if w.dtype == wl.F32 else torch.bfloat16, s=w.s,
-        scales=list(w.scales) if multi else None,
-        fmt={"i8": B.UQ_FMT_I8, "i4x2": B.UQ_FMT_I4X2, "i2x4": B.UQ_FMT_I2X4}[w.fmt], idx_bits=w.idx_bits,
-        norm=B.UQ_NORM_L2 if w.norm == wl.NORM_L2 else B.UQ_NORM_LINF, rng_bits=w.rng_bits)
+    return randk_from_workload(w, K)
 
 
 @pytest.mark.parametrize("name,d,K,M", [
