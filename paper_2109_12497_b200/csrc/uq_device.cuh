@@ -172,6 +172,32 @@ __device__ __forceinline__ uint4 philox4x32_10(const PhiloxKey &k, uint32_t bloc
     return make_uint4(c0, c1, c2, c3);
 }
 
+// N blocks at once, block n at counter (block_lo[n], block_hi, worker): the N chains advance
+// round by round together, so one fetch of a round key serves all of them and the chains' wide
+// multiplies overlap.
+template <int N>
+__device__ __forceinline__ void philox4x32_10_xN(const PhiloxKey &k, const uint32_t (&block_lo)[N], uint32_t block_hi,
+                                                 uint32_t worker, uint4 (&out)[N])
+{
+    uint32_t c0[N], c1[N], c2[N], c3[N];
+#pragma unroll
+    for (int n = 0; n < N; ++n) { c0[n] = block_lo[n]; c1[n] = block_hi; c2[n] = worker; c3[n] = 0u; }
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t k0 = k.k0[r], k1 = k.k1[r];
+#pragma unroll
+        for (int n = 0; n < N; ++n) {
+            const uint64_t p0 = (uint64_t)0xD2511F53u * c0[n];
+            const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2[n];
+            const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1[n] ^ k0;
+            const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3[n] ^ k1;
+            c1[n] = (uint32_t)p1; c3[n] = (uint32_t)p0; c0[n] = n0; c2[n] = n2;
+        }
+    }
+#pragma unroll
+    for (int n = 0; n < N; ++n) out[n] = make_uint4(c0[n], c1[n], c2[n], c3[n]);
+}
+
 // ---------------------------------------------------------------------------------------------
 // one coordinate of Q_s
 // ---------------------------------------------------------------------------------------------
@@ -199,11 +225,11 @@ constexpr uint32_t kLevelByte23 = 0;      // which byte of the returned word hol
 
 // 16-bit draw.  Returns a word whose byte 2 is the unsigned level.
 // x + 128 rounds x to 16 fractional bits (ties to even): the mantissa of the sum is
-// floor(x) * 2^16 + rint(p * 2^16); adding nh = 0xFFFF - h carries into bit 16 iff
-// h < rint(p * 2^16).
-__device__ __forceinline__ uint32_t level_draw16(float x, uint32_t nh)
+// floor(x) * 2^16 + rint(p * 2^16); adding 0xFFFF - h carries into bit 16 iff
+// h < rint(p * 2^16) (one three-input add: the subtraction is an operand modifier).
+__device__ __forceinline__ uint32_t level_draw16(float x, uint32_t h)
 {
-    return nh + __float_as_uint(__fadd_rn(x, 128.0f));
+    return __float_as_uint(__fadd_rn(x, 128.0f)) + 0xFFFFu - h;
 }
 constexpr uint32_t kLevelByte16 = 2;
 

@@ -39,6 +39,13 @@ template <int DT, bool MULTI> struct EncodeShape {
     static constexpr int MIN_CTAS = MULTI ? 4 : 3;
 #endif
     static constexpr int TILE = kThreads * UNITS * 8;
+    // 16-bit draws: units whose Philox blocks advance round by round together (one fetch of a round
+    // key serves them all).  Measured: helps the bf16 multi-scale variant, costs the others.
+#ifdef UQ_PHILOX_GROUP
+    static constexpr int PHILOX_GROUP = UQ_PHILOX_GROUP;
+#else
+    static constexpr int PHILOX_GROUP = (DT == UQ_BF16 && MULTI) ? 2 : 1;
+#endif
 };
 
 // (float)s_k / W with one IEEE division; 0 for an all-zero segment.
@@ -60,35 +67,63 @@ template <> struct IdxBits<8> { using T = uint64_t; static __device__ __forceinl
 // the bytes of negative coordinates), packed into the wire format and stored at `dst`.
 // coordinate c uses word c%4 of block c/4 (32-bit draws) or half (c%8)%2 of word (c%8)/2 of block
 // c/8 (16-bit draws).
+// The random words of a unit: RNG == 32 takes blocks blk_lo and blk_lo + 1 (blk_lo is even: no
+// carry), RNG == 16 the single block blk_lo.
+template <int RNG> struct UnitWords { uint4 r[RNG == 32 ? 2 : 1]; };
+
+template <int RNG>
+__device__ __forceinline__ UnitWords<RNG> unit_words(const PhiloxKey &key, uint32_t blk_lo, uint32_t blk_hi, uint32_t m)
+{
+    UnitWords<RNG> w;
+    if (RNG == 32) {
+        const uint32_t b[2] = { blk_lo, blk_lo + 1u };
+        uint4 r[2];
+        philox4x32_10_xN<2>(key, b, blk_hi, m, r);
+        w.r[0] = r[0]; w.r[RNG == 32 ? 1 : 0] = r[1];
+    } else {
+        w.r[0] = philox4x32_10(key, blk_lo, blk_hi, m);
+    }
+    return w;
+}
+
+template <int FMT, int RNG>
+__device__ __forceinline__ void quantize_unit_words(const float (&v)[8], const float (&inv)[8], float cap,
+                                                    uint32_t neg_lo, uint32_t neg_hi, const UnitWords<RNG> &rw,
+                                                    void *dst, bool store = true)
+{
+    constexpr uint32_t LB = RNG == 32 ? kLevelByte23 : kLevelByte16;
+    uint32_t z[8];
+    if (RNG == 32) {
+        const uint4 r0 = rw.r[0], r1 = rw.r[RNG == 32 ? 1 : 0];
+        const uint32_t w[8] = { r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w };
+#pragma unroll
+        for (int e = 0; e < 8; ++e) z[e] = level_draw23(scaled_magnitude(v[e], inv[e], cap), w[e]);
+    } else {
+        const uint4 r = rw.r[0];
+        const uint32_t w[4] = { r.x, r.y, r.z, r.w };
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const uint32_t h = (e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu);
+            z[e] = level_draw16(scaled_magnitude(v[e], inv[e], cap), h);
+        }
+    }
+    const uint32_t lo = negate_bytes(gather_bytes<LB>(z[0], z[1], z[2], z[3]), neg_lo);
+    const uint32_t hi = negate_bytes(gather_bytes<LB>(z[4], z[5], z[6], z[7]), neg_hi);
+    if (!store) return;
+    // plain stores (not evict-first ones): the aggregation kernel that follows reads the levels
+    // back, and what is still in L2 then costs no DRAM read (measured: 7-9 % off that kernel)
+    if (FMT == UQ_FMT_I8) *(uint2 *)dst = make_uint2(lo, hi);
+    else if (FMT == UQ_FMT_I4X2) *(uint32_t *)dst = bytes_to_nibbles(lo, hi);
+    else *(unsigned short *)dst = (unsigned short)bytes_to_crumbs(lo, hi);
+}
+
 template <int FMT, int RNG>
 __device__ __forceinline__ void quantize_unit(const float (&v)[8], const float (&inv)[8], float cap,
                                               uint32_t neg_lo, uint32_t neg_hi, const PhiloxKey &key,
                                               uint32_t blk_lo, uint32_t blk_hi, uint32_t m, void *dst,
                                               bool store = true)
 {
-    constexpr uint32_t LB = RNG == 32 ? kLevelByte23 : kLevelByte16;
-    uint32_t z[8];
-    if (RNG == 32) {
-        const uint4 r0 = philox4x32_10(key, blk_lo, blk_hi, m);
-        const uint4 r1 = philox4x32_10(key, blk_lo + 1u, blk_hi, m);      // blk_lo is even: no carry
-        const uint32_t w[8] = { r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w };
-#pragma unroll
-        for (int e = 0; e < 8; ++e) z[e] = level_draw23(scaled_magnitude(v[e], inv[e], cap), w[e]);
-    } else {
-        const uint4 r = philox4x32_10(key, blk_lo, blk_hi, m);
-        const uint32_t nw[4] = { ~r.x, ~r.y, ~r.z, ~r.w };       // 0xFFFF - h for both halves at once
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const uint32_t nh = (e & 1) ? (nw[e >> 1] >> 16) : (nw[e >> 1] & 0xFFFFu);
-            z[e] = level_draw16(scaled_magnitude(v[e], inv[e], cap), nh);
-        }
-    }
-    const uint32_t lo = negate_bytes(gather_bytes<LB>(z[0], z[1], z[2], z[3]), neg_lo);
-    const uint32_t hi = negate_bytes(gather_bytes<LB>(z[4], z[5], z[6], z[7]), neg_hi);
-    if (!store) return;
-    if (FMT == UQ_FMT_I8) st_stream((uint2 *)dst, make_uint2(lo, hi));
-    else if (FMT == UQ_FMT_I4X2) st_stream((uint32_t *)dst, bytes_to_nibbles(lo, hi));
-    else st_stream((unsigned short *)dst, (unsigned short)bytes_to_crumbs(lo, hi));
+    quantize_unit_words<FMT, RNG>(v, inv, cap, neg_lo, neg_hi, unit_words<RNG>(key, blk_lo, blk_hi, m), dst, store);
 }
 
 // The sign masks of a unit, from the raw loaded words (before any padding is zeroed).
@@ -184,6 +219,7 @@ __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, IDXB != 0>::MIN_CTA
     constexpr int IB = MULTI ? IDXB : 8;
     constexpr int H = 8 / E::G;                                  // 16-byte loads per unit
     constexpr uint32_t BPU = RNG == 32 ? 2u : 1u;                // Philox blocks per unit
+    constexpr int PG = RNG == 16 ? S::PHILOX_GROUP : 1;            // units whose Philox blocks advance together
     const int tid = threadIdx.x, lane = tid & 31;
     if (blockIdx.x >= p.main_blocks) {
         // A CTA of the second kind: each warp takes one segment boundary and, if the boundary lies
@@ -269,21 +305,38 @@ __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, IDXB != 0>::MIN_CTA
     // One straight-line pass over all units, so the compiler can interleave them.  A crossed row
     // runs through the arithmetic too but is not stored: a CTA of the second kind owns it.
 #pragma unroll
-    for (int u = 0; u < S::UNITS; ++u) {
-        const float inv_lane = inv_row[u];
-        overflow |= not_finite(inv_lane);
-        float v[8], inv[8];
+    for (int u0 = 0; u0 < S::UNITS; u0 += PG) {
+        // the random words of PG units together (16-bit draws: one Philox block per unit)
+        UnitWords<RNG> rw[PG];
+        if (RNG == 16) {
+            uint32_t b[PG];
+            uint4 r[PG];
 #pragma unroll
-        for (int h = 0; h < H; ++h) E::unpack(q[u][h], *(float(*)[E::G])(v + h * E::G));
-        // the shuffle reads its source lane modulo 32 and the table repeats every 2^IB lanes (an
-        // 8-bit index is below 16), so the index bits need a shift but no mask
+            for (int n = 0; n < PG; ++n) b[n] = blk_lo + (u0 + n) * kThreads * BPU;
+            philox4x32_10_xN<PG>(p.key, b, blk_hi, (uint32_t)m, r);
 #pragma unroll
-        for (int e = 0; e < 8; ++e)
-            inv[e] = MULTI ? __shfl_sync(0xFFFFFFFFu, inv_lane, (int)(uint32_t)(kbits[u] >> (e * IB))) : inv_lane;
-        uint32_t neg_lo, neg_hi;
-        unit_signs<DT>(q[u], neg_lo, neg_hi);
-        quantize_unit<FMT, RNG>(v, inv, p.cap, neg_lo, neg_hi, p.key, blk_lo + u * kThreads * BPU, blk_hi, (uint32_t)m,
-                                lp + u * kThreads * UB, !((crossed >> u) & 1u));
+            for (int n = 0; n < PG; ++n) rw[n].r[0] = r[n];
+        } else {
+            rw[0] = unit_words<RNG>(p.key, blk_lo + u0 * kThreads * BPU, blk_hi, (uint32_t)m);
+        }
+#pragma unroll
+        for (int n = 0; n < PG; ++n) {
+            const int u = u0 + n;
+            const float inv_lane = inv_row[u];
+            overflow |= not_finite(inv_lane);
+            float v[8], inv[8];
+#pragma unroll
+            for (int h = 0; h < H; ++h) E::unpack(q[u][h], *(float(*)[E::G])(v + h * E::G));
+            // the shuffle reads its source lane modulo 32 and the table repeats every 2^IB lanes (an
+            // 8-bit index is below 16), so the index bits need a shift but no mask
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+                inv[e] = MULTI ? __shfl_sync(0xFFFFFFFFu, inv_lane, (int)(uint32_t)(kbits[u] >> (e * IB))) : inv_lane;
+            uint32_t neg_lo, neg_hi;
+            unit_signs<DT>(q[u], neg_lo, neg_hi);
+            quantize_unit_words<FMT, RNG>(v, inv, p.cap, neg_lo, neg_hi, rw[n], lp + u * kThreads * UB,
+                                          !((crossed >> u) & 1u));
+        }
     }
     if (overflow && lane < p.scales.N && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
 }
