@@ -37,10 +37,9 @@ FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only
 
 # DRAM traffic per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum) from
 # the ncu captures summarised under profiles/, keyed by workload; None = not captured.
-# c2: (268.8 MB read + 39.0 MB written) captured at d = 8,388,608, scaled by 25,557,032 / 8,388,608
-# (every coordinate is read and written once, so traffic is proportional to d); see
-# profiles/kernels_c2_small_ncu_full.md.
-NCU_TRAFFIC_BYTES = {"c2": 937.7e6}
+# c2: 819.2 MB read + 159.6 MB written by the encode kernel in a capture at full size
+# (profiles/traffic_c2_full_size.md).
+NCU_TRAFFIC_BYTES = {"c2": 978.8e6}
 
 
 def hbm_peak():
