@@ -66,6 +66,19 @@ def test_multi_scale_variants(idx_bits, N, dtype, fmt, s, ratio):
     assert len(np.unique(r["ref"]["idx_raw"])) >= 2          # more than one scale is in use
 
 
+@pytest.mark.parametrize("bits,fmt", [((8, 12), "i8"), ((6, 10), "i8"), ((4, 8), "i4x2"), ((2, 6), "i2x4")])
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+def test_two_scale_pairs_of_the_experiments(bits, fmt, dtype):
+    """The two-scale compressors of the paper's experiments, named by the bit widths of their two
+    scales: a scale of r bits has s = 2^(r-1) - 1 levels.  The levels travel in the narrowest
+    supported format that holds the smaller scale, the one-bit choice in the 2-bit index field."""
+    scales = tuple(2 ** (r - 1) - 1 for r in bits)
+    w = wl.scaled("c3", 120_011, M=8, idx_bits=2, scales=scales, s=scales[0], fmt=fmt, dtype=dtype)
+    r = check_parity(w, wl.generate(w))
+    assert set(np.unique(r["ref"]["idx_raw"]).tolist()) == {0, 1}
+    assert np.abs(r["ref"]["lev_raw"].astype(int)).max() <= scales[0]
+
+
 @pytest.mark.parametrize("M", [1, 2, 7, 8, 9, 16, 17, 33, 64])
 def test_worker_counts(M):
     for name in ("c1", "c4", "c3"):
