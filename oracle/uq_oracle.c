@@ -194,10 +194,13 @@ static int quantize_coord(float v, float inv, float s_cap, uint32_t h, int b)
 /* Algorithm 1 line "Quantize gradient" for every worker: zeta^m = Q_s(g^m, ||w||_2).
  * lev[m*stride + i] receives zeta^m_i as int8 (s <= 127).
  * h_inject != NULL replaces the Philox draw of coordinate (m, i) by h_inject[m*stride + i]
- * (used by the worked examples). */
+ * (used by the worked examples).
+ * worker0: the rows of g are workers worker0 .. worker0+M-1 of the whole job (a process that
+ * holds only some of the M workers passes its first worker's number; the draws are keyed by
+ * the worker's number in the job, so the levels do not depend on who computes them). */
 void uqo_encode_single(const void *g, int dtype, int M, int64_t coord0, int64_t d, int64_t stride,
                        int nseg, const int64_t *seg_off, const float *W, int32_t s,
-                       uint64_t seed, int rng_bits, const uint32_t *h_inject, int8_t *lev)
+                       uint64_t seed, int rng_bits, const uint32_t *h_inject, int8_t *lev, int worker0)
 {
     int b = draw_width(rng_bits);
     for (int m = 0; m < M; ++m) {
@@ -207,7 +210,7 @@ void uqo_encode_single(const void *g, int dtype, int M, int64_t coord0, int64_t 
             float inv = inv_scale(s, W[j]);
             float v = load_elem(g, dtype, (int64_t)m * stride + i);
             uint32_t h = h_inject ? h_inject[(int64_t)m * stride + i]
-                                  : uqo_draw(seed, (uint32_t)m, (uint64_t)(coord0 + i), rng_bits);
+                                  : uqo_draw(seed, (uint32_t)(worker0 + m), (uint64_t)(coord0 + i), rng_bits);
             lev[(int64_t)m * stride + i] = (int8_t)quantize_coord(v, inv, (float)s, h, b);
         }
     }
@@ -252,7 +255,7 @@ void uqo_select_scale_multi(const void *g, int dtype, int M, int64_t coord0, int
 void uqo_encode_multi(const void *g, int dtype, int M, int64_t coord0, int64_t d, int64_t stride,
                       int nseg, const int64_t *seg_off, const float *W, const int32_t *scales,
                       int N, const uint8_t *idx, uint64_t seed, int rng_bits,
-                      const uint32_t *h_inject, int8_t *lev)
+                      const uint32_t *h_inject, int8_t *lev, int worker0)
 {
     int b = draw_width(rng_bits);
     float s_hat = (float)scales[0];
@@ -264,7 +267,7 @@ void uqo_encode_multi(const void *g, int dtype, int M, int64_t coord0, int64_t d
             float inv = inv_scale(scales[idx[i]], W[j]);
             float v = load_elem(g, dtype, (int64_t)m * stride + i);
             uint32_t h = h_inject ? h_inject[(int64_t)m * stride + i]
-                                  : uqo_draw(seed, (uint32_t)m, (uint64_t)(coord0 + i), rng_bits);
+                                  : uqo_draw(seed, (uint32_t)(worker0 + m), (uint64_t)(coord0 + i), rng_bits);
             lev[(int64_t)m * stride + i] = (int8_t)quantize_coord(v, inv, s_hat, h, b);
         }
     }
@@ -363,6 +366,19 @@ void uqo_pack_levels_i2(const int8_t *lev, int M, int64_t d, int64_t stride, uin
             }
             packed[(int64_t)m * (stride / 4) + q] = (uint8_t)byte;
         }
+}
+
+/* Scale sharing across processes (Algorithm 2 line "Scale sharing" when each process holds
+ * some of the workers): rows[r*d + i] is the minimum over process r's workers, the shared
+ * index is the minimum over the R rows. */
+void uqo_index_min(const uint8_t *rows, int R, int64_t d, uint8_t *idx)
+{
+    for (int64_t i = 0; i < d; ++i) {
+        uint8_t k = rows[i];
+        for (int r = 1; r < R; ++r)
+            if (rows[(int64_t)r * d + i] < k) k = rows[(int64_t)r * d + i];
+        idx[i] = k;
+    }
 }
 
 /* Scale indices packed idx_bits (2, 4 or 8) per coordinate, little-endian inside the byte:

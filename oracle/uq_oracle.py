@@ -120,7 +120,7 @@ def agree_scale(g: np.ndarray, seg_off=None, norm: int = NORM_L2) -> np.ndarray:
     return W
 
 
-def encode_single(g, W, s, seed, rng_bits=32, seg_off=None, coord0=0, h_inject=None):
+def encode_single(g, W, s, seed, rng_bits=32, seg_off=None, coord0=0, h_inject=None, worker0=0):
     """Levels zeta[m, i] (int8) of every worker; g holds coordinates coord0.. of each worker."""
     M, d, stride = _check_g(g)
     nseg, so = _seg(seg_off)
@@ -130,7 +130,7 @@ def encode_single(g, W, s, seed, rng_bits=32, seg_off=None, coord0=0, h_inject=N
     lev = _rows(M, d, stride, np.int8)
     lib().uqo_encode_single(_p(g), _dtype_of(g), M, C.c_int64(coord0), C.c_int64(d),
                             C.c_int64(stride), nseg, _p(so), _p(W), C.c_int32(s), C.c_uint64(seed),
-                            rng_bits, _p(h_inject), _p(lev))
+                            rng_bits, _p(h_inject), _p(lev), worker0)
     return lev
 
 
@@ -149,7 +149,7 @@ def select_scale_multi(g, W, scales, seg_off=None, coord0=0, return_own=False):
     return (idx, own) if return_own else idx
 
 
-def encode_multi(g, W, scales, idx, seed, rng_bits=32, seg_off=None, coord0=0, h_inject=None):
+def encode_multi(g, W, scales, idx, seed, rng_bits=32, seg_off=None, coord0=0, h_inject=None, worker0=0):
     M, d, stride = _check_g(g)
     nseg, so = _seg(seg_off)
     W = np.ascontiguousarray(W, dtype=np.float32)
@@ -162,7 +162,7 @@ def encode_multi(g, W, scales, idx, seed, rng_bits=32, seg_off=None, coord0=0, h
     lib().uqo_encode_multi(_p(g), _dtype_of(g), M, C.c_int64(coord0), C.c_int64(d),
                            C.c_int64(stride),
                            nseg, _p(so), _p(W), _p(scales), len(scales), _p(idx),
-                           C.c_uint64(seed), rng_bits, _p(h_inject), _p(lev))
+                           C.c_uint64(seed), rng_bits, _p(h_inject), _p(lev), worker0)
     return lev
 
 
@@ -215,6 +215,15 @@ def pack_levels_i2(lev: np.ndarray) -> np.ndarray:
     packed = np.zeros((M, stride // 4), dtype=np.uint8)
     lib().uqo_pack_levels_i2(_p(lev), M, C.c_int64(d), C.c_int64(stride), _p(packed))
     return packed[:, : (d + 3) // 4]
+
+
+def index_min(rows: np.ndarray) -> np.ndarray:
+    """Minimum over the rows of an [R, d] array of (unpacked) scale indices."""
+    rows = np.ascontiguousarray(rows, dtype=np.uint8)
+    R, d = rows.shape
+    idx = np.zeros(d, dtype=np.uint8)
+    lib().uqo_index_min(_p(rows), R, C.c_int64(d), _p(idx))
+    return idx
 
 
 def pack_index(idx: np.ndarray, idx_bits: int) -> np.ndarray:

@@ -157,3 +157,28 @@ def test_index_packing_layout():
     assert o.pack_index(idx, 2).tolist() == [0b11100100, 0b00011011]
     assert o.pack_index(idx, 4).tolist() == [0x10, 0x32, 0x23, 0x01]
     assert o.pack_index(idx, 8).tolist() == idx.tolist()
+
+
+def test_workers_split_over_processes_give_the_same_result():
+    """A job whose M workers are spread over R processes: every process quantizes its own rows
+    with its first worker's number, the shared index is the minimum of the per-process minima.
+    Both must equal the one-process result (the draws are keyed by the worker's number in the
+    job, and a minimum of minima is the minimum)."""
+    w = wl.scaled("c3", 3001, M=6)
+    g = wl.generate(w)[:, : w.d]
+    seg = wl.segment_offsets(w)
+    W = o.agree_scale(g, seg, o.NORM_L2)
+    idx = o.select_scale_multi(g, W, w.scales, seg_off=seg)
+    lev = o.encode_multi(g, W, w.scales, idx, 11, 16, seg_off=seg)
+    lev1 = o.encode_single(g, W, 127, 11, 32, seg_off=seg)
+    parts = [(0, 2), (2, 3), (3, 6)]
+    # the scale: a maximum of per-process maxima
+    W_parts = np.stack([o.agree_scale(g[a:b], seg, o.NORM_L2) for a, b in parts])
+    assert np.array_equal(W_parts.max(axis=0), W)
+    rows = np.stack([o.select_scale_multi(g[a:b], W, w.scales, seg_off=seg) for a, b in parts])
+    assert np.array_equal(o.index_min(rows), idx) and np.array_equal(rows.min(axis=0), idx)
+    for a, b in parts:
+        assert np.array_equal(o.encode_multi(g[a:b], W, w.scales, idx, 11, 16, seg_off=seg, worker0=a), lev[a:b])
+        assert np.array_equal(o.encode_single(g[a:b], W, 127, 11, 32, seg_off=seg, worker0=a), lev1[a:b])
+    # and the worker number matters: the wrong one gives other draws
+    assert not np.array_equal(o.encode_single(g[2:3], W, 127, 11, 32, seg_off=seg, worker0=0), lev1[2:3])
