@@ -80,7 +80,10 @@ typedef struct uq_layout {
     int32_t M;              /* workers, 1..UQ_MAX_WORKERS */
     int32_t nseg;           /* segments, >= 1 */
     int32_t dtype;          /* UQ_F32 or UQ_BF16 (bf16 = upper half of a binary32) */
-    int32_t reserved;       /* must be 0 */
+    int32_t worker0;        /* number, in the whole job, of the worker in row 0 (>= 0); 0 when the
+                               buffer holds all workers.  Only the encoders use it: the random
+                               draws of row m are those of worker worker0 + m, so a process that
+                               holds some of the job's workers produces the same levels */
 } uq_layout;
 
 /* Library version (major*10000 + minor*100 + patch). */
@@ -241,6 +244,21 @@ int uq_decode(const uq_layout *layout, const void *src, int src_kind, int fmt, c
 int uq_decode_update(const uq_layout *layout, const void *lev, int fmt, const float *W, int s,
                      const int32_t *scales, int N, const uint8_t *idx, int idx_bits, float *theta,
                      float *momentum, float lr, float mu, float wd, float *out_opt, void *stream);
+
+/*
+ * Scale sharing across processes — Algorithm 2 line "Scale sharing" (s*_i = min over workers)
+ * when the M workers are spread over R processes: each process runs uq_select_scale_multi on
+ * its own workers (with the job-wide W), the R packed index rows are brought together (an
+ * all-gather), and the shared index is their field-wise minimum.
+ *   rows      in   [R][row_bytes] packed indices, device, 8-byte aligned, row r = process r
+ *   R              1..UQ_MAX_WORKERS
+ *   row_bytes      distance between rows, a multiple of 8, >= nbytes
+ *   nbytes         bytes of one row to reduce, a multiple of 8 (uq_index_bytes() is one)
+ *   idx       out  [nbytes] packed shared indices, 8-byte aligned; may be row 0 of rows
+ * Errors: UQ_ERR_BAD_ARG, UQ_ERR_CUDA.
+ */
+int uq_index_min(const uint8_t *rows, int R, int64_t row_bytes, int64_t nbytes, int idx_bits,
+                 uint8_t *idx, void *stream);
 
 /*
  * GlobalRandKMaxNorm / GlobalRandKMaxNormMultiScale — Sections "GlobalRandKMaxNorm Compression"

@@ -26,7 +26,7 @@ UQ_STATUS_NONFINITE, UQ_STATUS_BAD_SEGMENTS, UQ_STATUS_SCALE_OVERFLOW, UQ_STATUS
 EXPORTS = (
     "uq_version", "uq_last_cuda_error", "uq_error_string", "uq_workspace_bytes", "uq_index_bytes",
     "uq_agree_scale", "uq_agree_scale_static", "uq_encode_single", "uq_select_scale_multi", "uq_encode_multi",
-    "uq_aggregate", "uq_decode", "uq_decode_update", "uq_randk_gather", "uq_randk_scatter", "uq_randk_update",
+    "uq_aggregate", "uq_decode", "uq_decode_update", "uq_randk_gather", "uq_randk_scatter", "uq_randk_update", "uq_index_min",
 )
 
 
@@ -38,7 +38,7 @@ class uq_layout(C.Structure):
         ("M", C.c_int32),
         ("nseg", C.c_int32),
         ("dtype", C.c_int32),
-        ("reserved", C.c_int32),
+        ("worker0", C.c_int32),
     ]
 
 
@@ -83,6 +83,7 @@ def lib() -> C.CDLL:
         F = C.c_float
         L.uq_decode_update.argtypes = [LP, P, I, P, I, P, I, P, I, P, P, F, F, F, P, P]
         I64 = C.c_int64
+        L.uq_index_min.argtypes = [P, I, I64, I64, I, P, P]
         L.uq_randk_gather.argtypes = [LP, P, I64, U64, P, P, I64, P, P]
         L.uq_randk_scatter.argtypes = [I64, I64, P, P, P, P, P]
         L.uq_randk_update.argtypes = [I64, I64, P, P, P, F, P, P]
@@ -119,7 +120,7 @@ class Layout:
     ``worker_stride`` coordinates, cut into segments that each share one scale."""
 
     def __init__(self, M: int, d: int, worker_stride: int, dtype: torch.dtype,
-                 seg_off: Optional[torch.Tensor] = None):
+                 seg_off: Optional[torch.Tensor] = None, worker0: int = 0):
         if dtype not in (torch.float32, torch.bfloat16):
             raise ValueError("uq: gradients are float32 or bfloat16")
         if seg_off is not None:
@@ -128,8 +129,9 @@ class Layout:
             seg_off = seg_off.contiguous()
         self.M, self.d, self.worker_stride, self.dtype, self.seg_off = M, d, worker_stride, dtype, seg_off
         self.nseg = 1 if seg_off is None else seg_off.numel() - 1
+        self.worker0 = worker0
         self.c = uq_layout(d, worker_stride, _ptr(seg_off), M, self.nseg,
-                           UQ_F32 if dtype == torch.float32 else UQ_BF16, 0)
+                           UQ_F32 if dtype == torch.float32 else UQ_BF16, worker0)
 
     def ref(self):
         return C.byref(self.c)
@@ -298,3 +300,15 @@ def uq_randk_update(d: int, K: int, sel: torch.Tensor, vals: torch.Tensor, theta
     _check_randk(d, K, sel, vals, theta, "theta")
     _check("uq_randk_update", lib().uq_randk_update(d, K, _ptr(sel), _ptr(vals), _ptr(theta), lr, _ptr(status),
                                                     _stream()))
+
+
+def uq_index_min(rows: torch.Tensor, idx_bits: int, idx: torch.Tensor, nbytes: Optional[int] = None) -> None:
+    """Field-wise minimum over the rows of a [R, row_bytes] uint8 tensor of packed scale indices
+    (one row per process) into idx; nbytes defaults to the whole row."""
+    if rows.dtype != torch.uint8 or rows.dim() != 2 or not rows.is_contiguous():
+        raise ValueError("uq: rows must be a contiguous [R, row_bytes] uint8 tensor")
+    nbytes = rows.shape[1] if nbytes is None else nbytes
+    if idx.dtype != torch.uint8 or idx.dim() != 1 or idx.numel() < nbytes or not idx.is_contiguous():
+        raise ValueError(f"uq: idx must be a contiguous uint8 tensor with >= {nbytes} elements")
+    _check("uq_index_min", lib().uq_index_min(_ptr(rows), rows.shape[0], rows.shape[1], nbytes, idx_bits, _ptr(idx),
+                                              _stream()))

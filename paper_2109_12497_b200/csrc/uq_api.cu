@@ -17,6 +17,8 @@ cudaError_t launch_aggregate_decode(const uq_layout &L, const void *lev, int fmt
                                     float lr = 0.0f, float mu = 0.0f, float wd = 0.0f);
 cudaError_t launch_decode_sums(const uq_layout &L, const int32_t *S, const float *W, const ScaleSet &scales,
                                const uint8_t *idx, int idx_bits, float *out, cudaStream_t st);
+cudaError_t launch_index_min(const uint8_t *rows, int R, int64_t row_bytes, int64_t nbytes, int idx_bits, uint8_t *idx,
+                             cudaStream_t st);
 cudaError_t launch_randk_gather(const uq_layout &L, const void *g, int64_t K, uint64_t seed, int64_t *sel,
                                 void *gk, int64_t gk_stride, uint32_t *status, cudaStream_t st);
 cudaError_t launch_randk_scatter(int64_t d, int64_t K, const int64_t *sel, const float *vals, float *dst, bool update,
@@ -39,7 +41,7 @@ bool aligned(const void *p, size_t a) { return ((uintptr_t)p & (a - 1)) == 0; }
 bool layout_ok(const uq_layout *L)
 {
     if (L == nullptr) return false;
-    if (L->d < 0 || L->M < 1 || L->M > UQ_MAX_WORKERS || L->nseg < 1 || L->reserved != 0) return false;
+    if (L->d < 0 || L->M < 1 || L->M > UQ_MAX_WORKERS || L->nseg < 1 || L->worker0 < 0 || L->worker0 > 0x7FFFFFFF - L->M) return false;
     if (L->dtype != UQ_F32 && L->dtype != UQ_BF16) return false;
     if (L->worker_stride < L->d || (L->worker_stride & 31) != 0) return false;
     if (L->seg_off == nullptr && L->nseg != 1) return false;
@@ -221,6 +223,15 @@ int uq_decode_update(const uq_layout *L, const void *lev, int fmt, const float *
                                               theta, momentum, lr, mu, wd));
 }
 
+int uq_index_min(const uint8_t *rows, int R, int64_t row_bytes, int64_t nbytes, int idx_bits, uint8_t *idx, void *stream)
+{
+    if (R < 1 || R > UQ_MAX_WORKERS || nbytes < 0 || (nbytes & 7) != 0 || row_bytes < nbytes || (row_bytes & 7) != 0)
+        return UQ_ERR_BAD_ARG;
+    if (idx_bits != 2 && idx_bits != 4 && idx_bits != 8) return UQ_ERR_BAD_ARG;
+    if (nbytes > 0 && (rows == nullptr || idx == nullptr || !aligned(rows, 8) || !aligned(idx, 8))) return UQ_ERR_BAD_ARG;
+    return finish(uq::launch_index_min(rows, R, row_bytes, nbytes, idx_bits, idx, (cudaStream_t)stream));
+}
+
 int uq_randk_gather(const uq_layout *L, const void *g, int64_t K, uint64_t seed, int64_t *sel, void *gk,
                     int64_t gk_stride, uint32_t *status, void *stream)
 {
@@ -228,6 +239,7 @@ int uq_randk_gather(const uq_layout *L, const void *g, int64_t K, uint64_t seed,
     uq_layout dense = *L;                         // segments do not apply to the K-vector
     dense.seg_off = nullptr;
     dense.nseg = 1;
+    dense.worker0 = 0;
     if (!layout_ok(&dense) || !aligned(status, 4)) return UQ_ERR_BAD_ARG;
     if (K < 0 || K > dense.d || gk_stride < K || (gk_stride & 31) != 0) return UQ_ERR_BAD_ARG;
     if (gk_stride > 0 && (gk == nullptr || !aligned(gk, 16))) return UQ_ERR_BAD_ARG;

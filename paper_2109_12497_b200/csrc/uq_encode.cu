@@ -19,6 +19,7 @@ struct EncodeParams {
     uint32_t *status;
     int64_t d, stride;
     int32_t nseg, M;
+    int32_t worker0;          // number, in the whole job, of the worker in row 0 (keys the draws)
     int64_t ntiles;
     uint32_t main_blocks;     // CTAs that own tiles; the CTAs after them own rows crossed by boundaries
     float cap;                // (float) of the smallest scale: the largest level
@@ -205,7 +206,7 @@ __device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, i
         if (overflow && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
         const uint64_t blk = RNG == 32 ? (uint64_t)(i >> 2) : (uint64_t)(i >> 3);
         char *dst = (char *)p.lev + (size_t)m * (size_t)(p.stride >> FMT) + (i >> FMT);     // 8 >> FMT bits per level
-        quantize_unit<FMT, RNG>(v, inv, p.cap, neg_lo, neg_hi, p.key, (uint32_t)blk, (uint32_t)(blk >> 32), (uint32_t)m,
+        quantize_unit<FMT, RNG>(v, inv, p.cap, neg_lo, neg_hi, p.key, (uint32_t)blk, (uint32_t)(blk >> 32), (uint32_t)(m + p.worker0),
                                 dst);
     }
 }
@@ -315,11 +316,11 @@ __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, IDXB != 0>::MIN_CTA
             uint4 r[PG];
 #pragma unroll
             for (int n = 0; n < PG; ++n) b[n] = blk_lo + (u0 + n) * kThreads * BPU;
-            philox4x32_10_xN<PG>(p.key, b, blk_hi, (uint32_t)m, r);
+            philox4x32_10_xN<PG>(p.key, b, blk_hi, (uint32_t)(m + p.worker0), r);
 #pragma unroll
             for (int n = 0; n < PG; ++n) rw[n].r[0] = r[n];
         } else {
-            rw[0] = unit_words<RNG>(p.key, blk_lo + u0 * kThreads * BPU, blk_hi, (uint32_t)m);
+            rw[0] = unit_words<RNG>(p.key, blk_lo + u0 * kThreads * BPU, blk_hi, (uint32_t)(m + p.worker0));
         }
 #pragma unroll
         for (int n = 0; n < PG; ++n) {
@@ -392,7 +393,7 @@ cudaError_t launch_encode(const uq_layout &L, const void *g, const float *W, con
 {
     EncodeParams p;
     p.g = g; p.lev = lev; p.W = W; p.seg_off = L.seg_off; p.idx = idx; p.status = status;
-    p.d = L.d; p.stride = L.worker_stride; p.nseg = L.nseg; p.M = L.M;
+    p.d = L.d; p.stride = L.worker_stride; p.nseg = L.nseg; p.M = L.M; p.worker0 = L.worker0;
     p.key = philox_key(seed);
     // CTA order (set in the kernel): the tiles are walked back to front with the worker varying fastest.  The
     // kernel before this one in a step (agree-scale or the selector) ends on the high tiles, so

@@ -209,4 +209,50 @@ cudaError_t launch_select(const uq_layout &L, const void *g, const float *W, con
     return L.dtype == UQ_F32 ? dispatch<UQ_F32>(p, idx_bits, st) : dispatch<UQ_BF16>(p, idx_bits, st);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Scale sharing across processes (Algorithm 2 line "Scale sharing" when the workers are spread
+// over several processes): every process has the minimum over its own workers, packed as the
+// selector writes it; the shared index is the field-wise minimum over the R packed rows.
+// ---------------------------------------------------------------------------------------------
+
+// Field-wise unsigned minimum of two words holding 4, 8 or 16 fields of 8, 4 or 2 bits.
+template <int IDXB> __device__ __forceinline__ uint32_t min_fields(uint32_t a, uint32_t b)
+{
+    if (IDXB == 8) return __vminu4(a, b);
+    constexpr uint32_t mask = IDXB == 4 ? 0x0F0F0F0Fu : 0x03030303u;
+    uint32_t r = 0;
+#pragma unroll
+    for (int t = 0; t < 8; t += IDXB) r |= __vminu4((a >> t) & mask, (b >> t) & mask) << t;
+    return r;
+}
+
+template <int IDXB>
+__global__ void __launch_bounds__(kThreads) index_min_kernel(const uint8_t *__restrict__ rows, int R, int64_t row_bytes,
+                                                             int64_t nwords, uint8_t *__restrict__ idx)
+{
+    const int64_t w = (int64_t)blockIdx.x * kThreads + threadIdx.x;      // my 8-byte word
+    if (w >= nwords) return;
+    uint2 acc = ld_stream64(rows + w * 8);
+    for (int r = 1; r < R; ++r) {
+        const uint2 q = ld_stream64(rows + (size_t)r * (size_t)row_bytes + w * 8);
+        acc.x = min_fields<IDXB>(acc.x, q.x);
+        acc.y = min_fields<IDXB>(acc.y, q.y);
+    }
+    *(uint2 *)(idx + w * 8) = acc;
+}
+
+cudaError_t launch_index_min(const uint8_t *rows, int R, int64_t row_bytes, int64_t nbytes, int idx_bits, uint8_t *idx,
+                             cudaStream_t st)
+{
+    const int64_t nwords = nbytes / 8;
+    const int64_t blocks = (nwords + kThreads - 1) / kThreads;
+    if (blocks == 0) return cudaSuccess;
+    if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    const unsigned nb = (unsigned)blocks;
+    if (idx_bits == 2) index_min_kernel<2><<<nb, kThreads, 0, st>>>(rows, R, row_bytes, nwords, idx);
+    else if (idx_bits == 4) index_min_kernel<4><<<nb, kThreads, 0, st>>>(rows, R, row_bytes, nwords, idx);
+    else index_min_kernel<8><<<nb, kThreads, 0, st>>>(rows, R, row_bytes, nwords, idx);
+    return cudaGetLastError();
+}
+
 }  // namespace uq

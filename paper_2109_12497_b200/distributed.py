@@ -1,0 +1,115 @@
+"""Algorithm 1 / 2 with the M workers spread over processes (one process per GPU).
+
+Every process holds ``M_local`` of the job's ``M = world_size * M_local`` gradients.  The paper's
+three all-reduces become three exchanges between processes:
+
+  max of the norm        local ``uq_agree_scale``            -> all-reduce(MAX) of W[nseg]
+  min of the scale index local ``uq_select_scale_multi``     -> all-gather of the packed rows,
+                                                                ``uq_index_min`` (field-wise minimum)
+  sum of the levels      local ``uq_encode_*`` (draws keyed  -> all-gather of the level rows,
+                         by the worker's number in the job)     fused sum + reconstruction over all
+                                                                M rows (``uq_decode``)
+
+so every process ends the step with the same reconstructed average, bit for bit the one a single
+process holding all M rows computes.  The level rows travel as they are on the wire (int8, or
+packed 4-/2-bit): (world_size - 1) * d * bits / 8 bytes received per process and step.
+
+The exchanges are ``torch.distributed`` collectives (NCCL on GPUs); every arithmetic step is one
+call of the C ABI.  ``kernels`` is the module that provides those calls; it defaults to the CUDA
+binding and exists so that the exchange logic can be exercised without GPUs by handing in a
+stand-in with the same functions (there is no automatic substitution: without the CUDA library
+the default raises).
+"""
+from __future__ import annotations
+
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+import torch.distributed as dist
+
+
+class DistributedQuantizer:
+    def __init__(self, M_local: int, d: int, dtype: torch.dtype = torch.float32,
+                 seg_off: Optional[Sequence[int]] = None, s: int = 127,
+                 scales: Optional[Sequence[int]] = None, fmt: int = 0, idx_bits: int = 0, norm: int = 2,
+                 rng_bits: int = 32, group=None, device: str | torch.device = "cuda", kernels=None):
+        if kernels is None:
+            from . import binding as kernels
+            kernels.lib()                               # fail now if the CUDA library is not built
+        self.k = kernels
+        self.group = group
+        self.rank, self.world = dist.get_rank(group), dist.get_world_size(group)
+        self.M_local, self.M, self.d, self.dtype = M_local, M_local * self.world, d, dtype
+        if self.M > 64:
+            raise ValueError("uq: at most 64 workers in a job")
+        dev = torch.device(device)
+        self.stride = -(-d // 32) * 32
+        self.multi = scales is not None and idx_bits != 0
+        self.s = int(scales[0]) if self.multi else int(s)
+        self.scales = [int(x) for x in scales] if self.multi else None
+        self.fmt, self.idx_bits, self.norm, self.rng_bits = fmt, idx_bits if self.multi else 0, norm, rng_bits
+        seg_dev = None
+        if seg_off is not None and len(seg_off) > 2:
+            seg_dev = torch.as_tensor(np.asarray(seg_off, dtype=np.int64), device=dev)
+        # my rows are workers rank*M_local .. of the job; the gathered rows are all of them
+        self.local = self.k.Layout(M_local, d, self.stride, dtype, seg_dev, worker0=self.rank * M_local)
+        self.total = self.k.Layout(self.M, d, self.stride, dtype, seg_dev)
+        nseg = self.local.nseg
+        row_bytes = self.local.level_row_bytes(fmt)
+        self.W = torch.zeros(nseg, dtype=torch.float32, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.workspace = torch.empty(max(8, self.local.workspace_bytes()), dtype=torch.uint8, device=dev)
+        self.lev_local = torch.empty((M_local, row_bytes), dtype=torch.int8, device=dev)
+        self.lev_all = torch.empty((self.M, row_bytes), dtype=torch.int8, device=dev)
+        self.idx = self.idx_local = self.idx_rows = None
+        if self.multi:
+            nb = max(16, self.local.index_bytes(self.idx_bits))
+            self.idx_local = torch.empty(nb, dtype=torch.uint8, device=dev)
+            self.idx_rows = torch.empty((self.world, nb), dtype=torch.uint8, device=dev)
+            self.idx = torch.empty(nb, dtype=torch.uint8, device=dev)
+        self.out = torch.empty(max(d, 1), dtype=torch.float32, device=dev)
+
+    # the three exchanges ------------------------------------------------------------------------
+    def agree_scale(self, g: torch.Tensor) -> None:
+        """Algorithm 1 / 2 line "MaxAllReduce Norm"."""
+        self.k.uq_agree_scale(self.local, g, self.norm, self.W, self.status, self.workspace)
+        dist.all_reduce(self.W, op=dist.ReduceOp.MAX, group=self.group)
+
+    def share_scale_index(self, g: torch.Tensor) -> None:
+        """Algorithm 2 lines "Compute coordinate scales" and "Scale sharing"."""
+        self.k.uq_select_scale_multi(self.local, g, self.W, self.scales, self.idx_bits, self.idx_local, self.status)
+        dist.all_gather_into_tensor(self.idx_rows.view(-1), self.idx_local, group=self.group)
+        self.k.uq_index_min(self.idx_rows, self.idx_bits, self.idx)
+
+    def encode(self, g: torch.Tensor, seed: int) -> None:
+        if self.multi:
+            self.k.uq_encode_multi(self.local, g, self.W, self.scales, self.idx, self.idx_bits, seed, self.rng_bits,
+                                   self.fmt, self.lev_local, self.status)
+        else:
+            self.k.uq_encode_single(self.local, g, self.W, self.s, seed, self.rng_bits, self.fmt, self.lev_local,
+                                    self.status)
+
+    def exchange_and_reconstruct(self) -> None:
+        """Algorithm 1 / 2 lines "AllReduce gradients" and "Reconstruct gradient": the level rows of
+        all processes are gathered as they are on the wire, summed and reconstructed in one kernel."""
+        dist.all_gather_into_tensor(self.lev_all.view(-1), self.lev_local.view(-1), group=self.group)
+        self.k.uq_decode(self.total, self.lev_all, self.k.UQ_SRC_LEVELS, self.fmt, self.W, self.s, self.scales,
+                         self.idx, self.idx_bits, self.out, None)
+
+    def step(self, g: torch.Tensor, seed: int = 0) -> torch.Tensor:
+        """g: [M_local, stride] gradients of my workers -> the average gradient of the job [d]."""
+        self.agree_scale(g)
+        if self.multi:
+            self.share_scale_index(g)
+        self.encode(g, seed)
+        self.exchange_and_reconstruct()
+        return self.out[: self.d]
+
+    def wire_bytes_per_step(self) -> int:
+        """Bytes this process receives from the others in one step."""
+        others = self.world - 1
+        n = others * self.lev_local.numel() + (self.W.numel() * 4 if others else 0)
+        if self.multi:
+            n += others * self.idx_local.numel()
+        return n

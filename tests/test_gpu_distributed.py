@@ -1,0 +1,137 @@
+"""The pieces the distributed step adds, on one GPU with the real kernels: rows encoded with
+their worker's number in the job, the field-wise minimum of packed index rows, and the whole
+exchange replayed rank by rank (copies stand in for the collectives) against the oracle's
+single-process result."""
+import os
+import socket
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import uq_oracle as o
+from paper_2109_12497_b200 import binding as B
+from paper_2109_12497_b200 import workloads as wl
+from paper_2109_12497_b200.pipeline import from_workload
+from parity import run_gpu, run_oracle, to_device, ulp_distance
+
+pytestmark = pytest.mark.gpu
+
+FMT = {"i8": B.UQ_FMT_I8, "i4x2": B.UQ_FMT_I4X2, "i2x4": B.UQ_FMT_I2X4}
+
+
+@pytest.mark.parametrize("idx_bits", [2, 4, 8])
+@pytest.mark.parametrize("R", [1, 2, 3, 8, 64])
+def test_index_min_matches_oracle(idx_bits, R):
+    d = 70_016                                      # a multiple of 32 coordinates: whole 8-byte words
+    rng = np.random.default_rng(R * 10 + idx_bits)
+    raw = rng.integers(0, min(16, 1 << idx_bits), size=(R, d), dtype=np.uint8)
+    packed = np.stack([o.pack_index(raw[r], idx_bits) for r in range(R)])
+    rows = torch.from_numpy(packed).cuda()
+    idx = torch.full((packed.shape[1] + 8,), 0xEE, dtype=torch.uint8, device="cuda")
+    B.uq_index_min(rows, idx_bits, idx[: packed.shape[1]])
+    want = o.pack_index(o.index_min(raw), idx_bits)
+    got = idx.cpu().numpy()
+    assert np.array_equal(got[: want.size], want) and (got[packed.shape[1]:] == 0xEE).all()
+    B.uq_index_min(rows, idx_bits, rows[0])         # in place into row 0
+    assert np.array_equal(rows[0].cpu().numpy(), want)
+
+
+def test_index_min_argument_checks():
+    rows = torch.zeros((2, 64), dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.UqError):
+        B.uq_index_min(rows, 3, rows[0])
+    with pytest.raises(B.UqError):
+        B.uq_index_min(rows, 4, rows[0], nbytes=12)                       # not whole 8-byte words
+
+
+@pytest.mark.parametrize("name,d,M,parts,kw", [
+    ("c2", 300_007, 8, [(0, 1), (1, 4), (4, 8)], {}),
+    ("c3", 300_007, 8, [(0, 4), (4, 8)], {}),
+    ("c5", 200_003, 6, [(0, 1), (1, 2), (2, 3), (3, 4), (4, 5), (5, 6)], {}),
+    ("c4", 100_003, 16, [(0, 8), (8, 16)], {}),
+    ("c3", 150_001, 4, [(0, 2), (2, 4)], dict(fmt="i2x4", s=1, scales=(1, 16, 256), rng_bits=32)),
+])
+def test_exchange_replayed_rank_by_rank(name, d, M, parts, kw):
+    """Every 'rank' runs the local calls on its own rows; tensor copies play the collectives."""
+    w = wl.scaled(name, d, M=M, **kw)
+    g_np = wl.generate(w)
+    g = to_device(w, g_np)
+    seg = wl.segment_offsets(w)
+    seg_dev = torch.as_tensor(np.asarray(seg, dtype=np.int64), device="cuda") if len(seg) > 2 else None
+    stride, fmt, multi = g.shape[1], FMT[w.fmt], w.quantizer == "multi"
+    norm = B.UQ_NORM_L2 if w.norm == wl.NORM_L2 else B.UQ_NORM_LINF
+    lays = [B.Layout(b - a, d, stride, g.dtype, seg_dev, worker0=a) for a, b in parts]
+    total = B.Layout(M, d, stride, g.dtype, seg_dev)
+    nseg = total.nseg
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    # max of the norm
+    Ws = []
+    for (a, b), lay in zip(parts, lays):
+        W_r = torch.zeros(nseg, device="cuda")
+        ws = torch.empty(max(8, lay.workspace_bytes()), dtype=torch.uint8, device="cuda")
+        B.uq_agree_scale(lay, g[a:b], norm, W_r, status, ws)
+        Ws.append(W_r)
+    W = torch.stack(Ws).max(dim=0).values.contiguous()
+    # min of the scale index
+    idx = None
+    if multi:
+        nb = total.index_bytes(w.idx_bits)
+        rows = torch.empty((len(parts), nb), dtype=torch.uint8, device="cuda")
+        for r, ((a, b), lay) in enumerate(zip(parts, lays)):
+            B.uq_select_scale_multi(lay, g[a:b], W, list(w.scales), w.idx_bits, rows[r], status)
+        idx = torch.empty(nb, dtype=torch.uint8, device="cuda")
+        B.uq_index_min(rows, w.idx_bits, idx)
+    # levels of every rank's rows, gathered in worker order, then the fused sum + reconstruction
+    lev_all = torch.empty((M, total.level_row_bytes(fmt)), dtype=torch.int8, device="cuda")
+    for (a, b), lay in zip(parts, lays):
+        if multi:
+            B.uq_encode_multi(lay, g[a:b], W, list(w.scales), idx, w.idx_bits, w.seed, w.rng_bits, fmt, lev_all[a:b], status)
+        else:
+            B.uq_encode_single(lay, g[a:b], W, w.s, w.seed, w.rng_bits, fmt, lev_all[a:b], status)
+    out = torch.empty(d, device="cuda")
+    B.uq_decode(total, lev_all, B.UQ_SRC_LEVELS, fmt, W, w.s, list(w.scales) if multi else None, idx, w.idx_bits, out)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+
+    one = run_gpu(w, g_np)                                   # one process holding all M rows
+    assert np.array_equal(W.cpu().numpy(), one["W"])
+    assert np.array_equal(lev_all.cpu().numpy().view(np.uint8)[:, : (d >> fmt)], one["lev"][:, : (d >> fmt)])
+    if multi:
+        assert np.array_equal(idx.cpu().numpy()[: d * w.idx_bits // 8], one["idx"][: d * w.idx_bits // 8])
+    assert np.array_equal(out.cpu().numpy(), one["out"])
+    ref = run_oracle(w, g_np, one["W"])                      # and the oracle, given the same scale bits
+    assert ulp_distance(one["W"], run_oracle(w, g_np)["W"]).max() <= 1
+    assert np.array_equal(lev_all.cpu().numpy().view(np.uint8)[:, : ref["lev"].shape[1]], ref["lev"])
+    assert np.allclose(out.cpu().numpy(), ref["out"], rtol=1e-6, atol=0)
+
+
+def test_worker_number_is_validated():
+    with pytest.raises(B.UqError):
+        lay = B.Layout(2, 100, 128, torch.float32, None, worker0=-1)
+        g = torch.zeros((2, 128), device="cuda")
+        B.uq_encode_single(lay, g, torch.ones(1, device="cuda"), 127, 0, 32, B.UQ_FMT_I8,
+                           torch.empty((2, 128), dtype=torch.int8, device="cuda"), None)
+
+
+def test_distributed_quantizer_on_one_rank_equals_the_pipeline():
+    """DistributedQuantizer with the CUDA binding and a one-rank NCCL group."""
+    import torch.distributed as dist
+    from paper_2109_12497_b200.distributed import DistributedQuantizer
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda:0"))
+    try:
+        for name in ("c2", "c3"):
+            w = wl.scaled(name, 200_003, M=4)
+            g_np = wl.generate(w)
+            q = DistributedQuantizer(
+                w.M, w.d, torch.float32, seg_off=wl.segment_offsets(w), s=w.s,
+                scales=list(w.scales) if w.quantizer == "multi" else None, fmt=FMT[w.fmt], idx_bits=w.idx_bits,
+                norm=B.UQ_NORM_L2, rng_bits=w.rng_bits)
+            got = q.step(to_device(w, g_np), w.seed).cpu().numpy()
+            assert np.array_equal(got, run_gpu(w, g_np)["out"]) and int(q.status.item()) == 0
+    finally:
+        dist.destroy_process_group()
