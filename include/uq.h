@@ -225,6 +225,21 @@ int uq_decode(const uq_layout *layout, const void *src, int src_kind, int fmt, c
               int32_t *S_opt, void *stream);
 
 /*
+ * uq_decode(src_kind = UQ_SRC_LEVELS) with the level rows given one by one: lev_rows is a HOST
+ * array of layout->M device pointers, lev_rows[m] = start of worker m's level row (16-byte
+ * aligned, layout as the encoders write it).  The rows need not lie in one buffer, nor on this
+ * GPU: a row in a peer GPU's memory that is mapped into this process (peer access, an IPC or
+ * symmetric-memory mapping) is read with ordinary loads over NVLink while it is being summed, so
+ * "AllReduce gradients" + "Reconstruct gradient" of Algorithm 1 / 2 run as one kernel that pulls
+ * the other workers' levels itself.  The caller orders the call after the peers' encoders (a
+ * barrier between the processes); nothing in the kernel waits on another GPU.
+ * The array is copied at the call; the other arguments and errors are those of uq_decode.
+ */
+int uq_decode_rows(const uq_layout *layout, const void *const *lev_rows, int fmt, const float *W, int s,
+                   const int32_t *scales, int N, const uint8_t *idx, int idx_bits, float *out,
+                   int32_t *S_opt, void *stream);
+
+/*
  * Reconstruction fused with the parameter update — Algorithm 1 / 2, lines "AllReduce gradients",
  * "Reconstruct gradient" and "Update parameters" (theta_{t+1} = theta_t - eta_t * g_hat_t) in one
  * kernel: the level rows are summed and reconstructed as in uq_decode(src = LEVELS) and the

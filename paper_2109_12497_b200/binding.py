@@ -26,7 +26,7 @@ UQ_STATUS_NONFINITE, UQ_STATUS_BAD_SEGMENTS, UQ_STATUS_SCALE_OVERFLOW, UQ_STATUS
 EXPORTS = (
     "uq_version", "uq_last_cuda_error", "uq_error_string", "uq_workspace_bytes", "uq_index_bytes",
     "uq_agree_scale", "uq_agree_scale_static", "uq_encode_single", "uq_select_scale_multi", "uq_encode_multi",
-    "uq_aggregate", "uq_decode", "uq_decode_update", "uq_randk_gather", "uq_randk_scatter", "uq_randk_update", "uq_index_min",
+    "uq_aggregate", "uq_decode", "uq_decode_update", "uq_randk_gather", "uq_randk_scatter", "uq_randk_update", "uq_index_min", "uq_decode_rows",
 )
 
 
@@ -83,6 +83,7 @@ def lib() -> C.CDLL:
         F = C.c_float
         L.uq_decode_update.argtypes = [LP, P, I, P, I, P, I, P, I, P, P, F, F, F, P, P]
         I64 = C.c_int64
+        L.uq_decode_rows.argtypes = [LP, P, I, P, I, P, I, P, I, P, P, P]
         L.uq_index_min.argtypes = [P, I, I64, I64, I, P, P]
         L.uq_randk_gather.argtypes = [LP, P, I64, U64, P, P, I64, P, P]
         L.uq_randk_scatter.argtypes = [I64, I64, P, P, P, P, P]
@@ -312,3 +313,24 @@ def uq_index_min(rows: torch.Tensor, idx_bits: int, idx: torch.Tensor, nbytes: O
         raise ValueError(f"uq: idx must be a contiguous uint8 tensor with >= {nbytes} elements")
     _check("uq_index_min", lib().uq_index_min(_ptr(rows), rows.shape[0], rows.shape[1], nbytes, idx_bits, _ptr(idx),
                                               _stream()))
+
+
+def uq_decode_rows(layout: Layout, lev_rows: Sequence[int], fmt: int, W: torch.Tensor, s: int,
+                   scales: Optional[Sequence[int]], idx: Optional[torch.Tensor], idx_bits: int,
+                   out: torch.Tensor, S_opt: Optional[torch.Tensor] = None) -> None:
+    """uq_decode over level rows given as M device addresses (one per worker, in worker order);
+    a row may live in a peer GPU's memory that is mapped into this process."""
+    if len(lev_rows) != layout.M:
+        raise ValueError(f"uq: lev_rows must hold {layout.M} addresses")
+    layout.check_vec(W, torch.float32, layout.nseg, "W")
+    layout.check_vec(out, torch.float32, layout.d, "out")
+    if S_opt is not None:
+        layout.check_vec(S_opt, torch.int32, layout.d, "S_opt")
+    arr, N = (None, 0)
+    if scales is not None:
+        arr, N = _scales(scales)
+        layout.check_vec(idx, torch.uint8, layout.index_bytes(idx_bits), "idx")
+    rows = (C.c_void_p * layout.M)(*[int(a) for a in lev_rows])
+    _check("uq_decode_rows", lib().uq_decode_rows(
+        layout.ref(), rows, fmt, _ptr(W), s, arr, N, _ptr(idx) if scales is not None else None, idx_bits,
+        _ptr(out), _ptr(S_opt), _stream()))

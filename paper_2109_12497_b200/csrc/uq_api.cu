@@ -15,6 +15,9 @@ cudaError_t launch_aggregate_decode(const uq_layout &L, const void *lev, int fmt
                                     const ScaleSet &scales, const uint8_t *idx, int idx_bits, float *out,
                                     int32_t *S, cudaStream_t st, float *theta = nullptr, float *mom = nullptr,
                                     float lr = 0.0f, float mu = 0.0f, float wd = 0.0f);
+cudaError_t launch_aggregate_decode_rows(const uq_layout &L, const void *const *lev_rows, int fmt, const float *W,
+                                         const ScaleSet &scales, const uint8_t *idx, int idx_bits, float *out,
+                                         int32_t *S, cudaStream_t st);
 cudaError_t launch_decode_sums(const uq_layout &L, const int32_t *S, const float *W, const ScaleSet &scales,
                                const uint8_t *idx, int idx_bits, float *out, cudaStream_t st);
 cudaError_t launch_index_min(const uint8_t *rows, int R, int64_t row_bytes, int64_t nbytes, int idx_bits, uint8_t *idx,
@@ -198,6 +201,30 @@ int uq_decode(const uq_layout *L, const void *src, int src_kind, int fmt, const 
     if (S_opt != nullptr && !aligned(S_opt, 32)) return UQ_ERR_BAD_ARG;
     return finish(uq::launch_aggregate_decode(*L, src, fmt, W, set, idx, idx_bits, out, S_opt,
                                               (cudaStream_t)stream));
+}
+
+int uq_decode_rows(const uq_layout *L, const void *const *lev_rows, int fmt, const float *W, int s,
+                   const int32_t *scales, int N, const uint8_t *idx, int idx_bits, float *out, int32_t *S_opt,
+                   void *stream)
+{
+    if (!layout_ok(L) || W == nullptr || lev_rows == nullptr || !fmt_known(fmt)) return UQ_ERR_BAD_ARG;
+    uq::ScaleSet set;
+    if (scales != nullptr) {
+        if (!scales_ok(scales, N, idx_bits, &set)) return UQ_ERR_BAD_ARG;
+        if (L->d > 0 && (idx == nullptr || !aligned(idx, 16))) return UQ_ERR_BAD_ARG;
+    } else {
+        if (s < 1) return UQ_ERR_BAD_ARG;
+        set = single_scale(s);
+        idx_bits = 0;
+        idx = nullptr;
+    }
+    if (L->d > 0) {
+        if (out == nullptr || !aligned(out, 32) || !aligned(S_opt, 32)) return UQ_ERR_BAD_ARG;
+        for (int m = 0; m < L->M; ++m)
+            if (lev_rows[m] == nullptr || !aligned(lev_rows[m], 16)) return UQ_ERR_BAD_ARG;
+    }
+    return finish(uq::launch_aggregate_decode_rows(*L, lev_rows, fmt, W, set, idx, idx_bits, out, S_opt,
+                                                   (cudaStream_t)stream));
 }
 
 int uq_decode_update(const uq_layout *L, const void *lev, int fmt, const float *W, int s, const int32_t *scales,

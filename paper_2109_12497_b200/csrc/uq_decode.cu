@@ -23,6 +23,9 @@ struct DecodeParams {
     float *theta;             // parameters, updated in place
     float *mom;               // momentum buffer, updated in place; NULL for plain SGD
     float lr, mu, wd;         // step size, momentum factor, weight decay
+    // ROWS variant: where each worker's level row starts (rows need not be one buffer, nor all on
+    // this GPU: a peer's row is read with ordinary loads over NVLink); lev is unused then
+    const void *rows[UQ_MAX_WORKERS];
 };
 
 // One coordinate of the update theta <- theta - lr * u with
@@ -164,7 +167,7 @@ template <> struct Unit<UQ_FMT_I2X4> {
 
 // UPDATE selects the variant that also applies the parameter update (kept apart so that the plain
 // reconstruction keeps its register count).
-template <int FMT, int IDXB, bool UPDATE>
+template <int FMT, int IDXB, bool UPDATE, bool ROWS = false>
 __global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const __grid_constant__ DecodeParams p)
 {
     using U = Unit<FMT>;
@@ -183,16 +186,18 @@ __global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const __grid
     U unit;
     uint32_t kw[WORDS];
     if (active) {
-        const char *col = (const char *)p.lev + (size_t)(i >> FMT);
+        const size_t off = (size_t)(i >> FMT);                     // my bytes inside a level row
+        const char *col = (const char *)p.lev + off;
         int m = 0;
         for (; m + 8 <= p.M; m += 8) {          // eight workers' loads in flight
             Q q[8];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) q[k] = U::load(col + (size_t)(m + k) * row_bytes);
+            for (int k = 0; k < 8; ++k)
+                q[k] = U::load(ROWS ? (const char *)p.rows[m + k] + off : col + (size_t)(m + k) * row_bytes);
 #pragma unroll
             for (int k = 0; k < 8; ++k) unit.add(q[k]);
         }
-        for (; m < p.M; ++m) unit.add(U::load(col + (size_t)m * row_bytes));
+        for (; m < p.M; ++m) unit.add(U::load(ROWS ? (const char *)p.rows[m] + off : col + (size_t)m * row_bytes));
         if (MULTI && p.out != nullptr) {
             // idx bits of coordinates i..i+C-1 start at byte i*IB/8 (a multiple of 4 bytes)
             const uint32_t *ip = (const uint32_t *)(p.idx + (size_t)i * IB / 8);
@@ -317,13 +322,22 @@ __global__ void __launch_bounds__(kThreads) decode_sums_kernel(const DecodeParam
 }
 
 template <int FMT>
-static cudaError_t dispatch_levels(const DecodeParams &p, int idx_bits, cudaStream_t st)
+static cudaError_t dispatch_levels(const DecodeParams &p, int idx_bits, cudaStream_t st, bool rows = false)
 {
     constexpr int TILE = kThreads * Unit<FMT>::C;
     const int64_t blocks = (p.d + TILE - 1) / TILE;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     const unsigned nb = (unsigned)blocks;
+    if (rows) {
+        switch (idx_bits) {
+        case 0: aggregate_decode_kernel<FMT, 0, false, true><<<nb, kThreads, 0, st>>>(p); break;
+        case 2: aggregate_decode_kernel<FMT, 2, false, true><<<nb, kThreads, 0, st>>>(p); break;
+        case 4: aggregate_decode_kernel<FMT, 4, false, true><<<nb, kThreads, 0, st>>>(p); break;
+        default: aggregate_decode_kernel<FMT, 8, false, true><<<nb, kThreads, 0, st>>>(p); break;
+        }
+        return cudaGetLastError();
+    }
     if (p.theta != nullptr) {
         switch (idx_bits) {
         case 0: aggregate_decode_kernel<FMT, 0, true><<<nb, kThreads, 0, st>>>(p); break;
@@ -348,7 +362,7 @@ cudaError_t launch_aggregate_decode(const uq_layout &L, const void *lev, int fmt
                                     int32_t *S, cudaStream_t st, float *theta, float *mom, float lr, float mu,
                                     float wd)
 {
-    DecodeParams p;
+    DecodeParams p = DecodeParams();
     p.lev = lev; p.W = W; p.seg_off = L.seg_off; p.idx = idx; p.out = out; p.S = S;
     p.d = L.d; p.stride = L.worker_stride; p.nseg = L.nseg; p.M = L.M; p.scales = scales;
     p.theta = theta; p.mom = mom; p.lr = lr; p.mu = mu; p.wd = wd;
@@ -357,10 +371,25 @@ cudaError_t launch_aggregate_decode(const uq_layout &L, const void *lev, int fmt
     return dispatch_levels<UQ_FMT_I2X4>(p, idx_bits, st);
 }
 
+// The same with the level rows given one by one (lev_rows[m] = start of worker m's row).
+cudaError_t launch_aggregate_decode_rows(const uq_layout &L, const void *const *lev_rows, int fmt, const float *W,
+                                         const ScaleSet &scales, const uint8_t *idx, int idx_bits, float *out,
+                                         int32_t *S, cudaStream_t st)
+{
+    DecodeParams p = DecodeParams();
+    p.lev = nullptr; p.W = W; p.seg_off = L.seg_off; p.idx = idx; p.out = out; p.S = S;
+    p.d = L.d; p.stride = L.worker_stride; p.nseg = L.nseg; p.M = L.M; p.scales = scales;
+    p.theta = nullptr; p.mom = nullptr; p.lr = p.mu = p.wd = 0.0f;
+    for (int m = 0; m < UQ_MAX_WORKERS; ++m) p.rows[m] = m < L.M ? lev_rows[m] : nullptr;
+    if (fmt == UQ_FMT_I8) return dispatch_levels<UQ_FMT_I8>(p, idx_bits, st, true);
+    if (fmt == UQ_FMT_I4X2) return dispatch_levels<UQ_FMT_I4X2>(p, idx_bits, st, true);
+    return dispatch_levels<UQ_FMT_I2X4>(p, idx_bits, st, true);
+}
+
 cudaError_t launch_decode_sums(const uq_layout &L, const int32_t *S, const float *W, const ScaleSet &scales,
                                const uint8_t *idx, int idx_bits, float *out, cudaStream_t st)
 {
-    DecodeParams p;
+    DecodeParams p = DecodeParams();
     p.lev = S; p.W = W; p.seg_off = L.seg_off; p.idx = idx; p.out = out; p.S = nullptr;
     p.theta = nullptr; p.mom = nullptr; p.lr = p.mu = p.wd = 0.0f;
     p.d = L.d; p.stride = L.worker_stride; p.nseg = L.nseg; p.M = L.M; p.scales = scales;

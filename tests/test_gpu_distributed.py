@@ -106,6 +106,29 @@ def test_exchange_replayed_rank_by_rank(name, d, M, parts, kw):
     assert np.allclose(out.cpu().numpy(), ref["out"], rtol=1e-6, atol=0)
 
 
+@pytest.mark.parametrize("name,d,M", [("c2", 300_007, 8), ("c3", 200_003, 5), ("c4", 100_003, 16), ("c5", 150_001, 9),
+                                      ("c1", 33, 2)])
+def test_decode_over_separate_rows(name, d, M):
+    """uq_decode_rows: every worker's level row in an allocation of its own (as a peer's row would
+    be), handed over as addresses; same sums and values as the one-buffer call."""
+    w = wl.scaled(name, d, M=M)
+    r = run_gpu(w, wl.generate(w))
+    q = r["q"]
+    rows = [q.lev[m].clone() for m in reversed(range(M))][::-1]          # allocated in reverse order
+    out = torch.full((d + 16,), 7.0, device="cuda")
+    S = torch.empty(d, dtype=torch.int32, device="cuda")
+    B.uq_decode_rows(q.layout, [t.data_ptr() for t in rows], q.fmt, q.W, q.s, q.scales, q.idx, q.idx_bits,
+                     out[8: 8 + d], S)
+    got = out.cpu().numpy()
+    assert np.array_equal(got[8: 8 + d], r["out"]) and (got[:8] == 7).all() and (got[8 + d:] == 7).all()
+    assert np.array_equal(S.cpu().numpy(), r["S"])
+    with pytest.raises(B.UqError):
+        B.uq_decode_rows(q.layout, [t.data_ptr() + 1 for t in rows], q.fmt, q.W, q.s, q.scales, q.idx, q.idx_bits,
+                         out[8: 8 + d])
+    with pytest.raises(ValueError):
+        B.uq_decode_rows(q.layout, [rows[0].data_ptr()], q.fmt, q.W, q.s, q.scales, q.idx, q.idx_bits, out[8: 8 + d])
+
+
 def test_worker_number_is_validated():
     with pytest.raises(B.UqError):
         lay = B.Layout(2, 100, 128, torch.float32, None, worker0=-1)
