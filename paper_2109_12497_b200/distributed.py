@@ -14,6 +14,15 @@ so every process ends the step with the same reconstructed average, bit for bit 
 process holding all M rows computes.  The level rows travel as they are on the wire (int8, or
 packed 4-/2-bit): (world_size - 1) * d * bits / 8 bytes received per process and step.
 
+``pull_levels=True`` replaces the last all-gather by peer loads: the level rows live in symmetric
+memory (every process maps the others' rows), and after a stream-ordered barrier between the
+processes ``uq_decode_rows`` reads all M rows where they are, its own from HBM and the peers' over
+NVLink with ordinary loads, while it sums them: exchange and arithmetic in one kernel, no staging
+copy of the gathered rows (2 * (world_size - 1) * d * bits / 8 bytes of HBM traffic less per step).
+The barriers are one-element NCCL all-reduces, so a peer that never arrives ends in NCCL's own
+timeout handling rather than in a kernel of this library waiting on a flag.  This mode needs
+GPUs that can map each other's memory; it has run here on a one-rank group only.
+
 The exchanges are ``torch.distributed`` collectives (NCCL on GPUs); every arithmetic step is one
 call of the C ABI.  ``kernels`` is the module that provides those calls; it defaults to the CUDA
 binding and exists so that the exchange logic can be exercised without GPUs by handing in a
@@ -33,7 +42,8 @@ class DistributedQuantizer:
     def __init__(self, M_local: int, d: int, dtype: torch.dtype = torch.float32,
                  seg_off: Optional[Sequence[int]] = None, s: int = 127,
                  scales: Optional[Sequence[int]] = None, fmt: int = 0, idx_bits: int = 0, norm: int = 2,
-                 rng_bits: int = 32, group=None, device: str | torch.device = "cuda", kernels=None):
+                 rng_bits: int = 32, group=None, device: str | torch.device = "cuda", kernels=None,
+                 pull_levels: bool = False):
         if kernels is None:
             from . import binding as kernels
             kernels.lib()                               # fail now if the CUDA library is not built
@@ -60,8 +70,18 @@ class DistributedQuantizer:
         self.W = torch.zeros(nseg, dtype=torch.float32, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.workspace = torch.empty(max(8, self.local.workspace_bytes()), dtype=torch.uint8, device=dev)
-        self.lev_local = torch.empty((M_local, row_bytes), dtype=torch.int8, device=dev)
-        self.lev_all = torch.empty((self.M, row_bytes), dtype=torch.int8, device=dev)
+        self.pull_levels = pull_levels
+        if pull_levels:
+            import torch.distributed._symmetric_memory as symm_mem
+            self.lev_local = symm_mem.empty((M_local, row_bytes), dtype=torch.int8, device=dev)
+            self._mapping = symm_mem.rendezvous(self.lev_local, dist.group.WORLD if group is None else group)
+            base = self._mapping.buffer_ptrs                       # where rank r's rows are mapped here
+            self.peer_rows = [base[r] + m * row_bytes for r in range(self.world) for m in range(M_local)]
+            self._flag = torch.zeros(1, dtype=torch.int32, device=dev)
+            self.lev_all = None
+        else:
+            self.lev_local = torch.empty((M_local, row_bytes), dtype=torch.int8, device=dev)
+            self.lev_all = torch.empty((self.M, row_bytes), dtype=torch.int8, device=dev)
         self.idx = self.idx_local = self.idx_rows = None
         if self.multi:
             nb = max(16, self.local.index_bytes(self.idx_bits))
@@ -93,6 +113,12 @@ class DistributedQuantizer:
     def exchange_and_reconstruct(self) -> None:
         """Algorithm 1 / 2 lines "AllReduce gradients" and "Reconstruct gradient": the level rows of
         all processes are gathered as they are on the wire, summed and reconstructed in one kernel."""
+        if self.pull_levels:
+            dist.all_reduce(self._flag, group=self.group)          # every process has finished its encoder
+            self.k.uq_decode_rows(self.total, self.peer_rows, self.fmt, self.W, self.s, self.scales, self.idx,
+                                  self.idx_bits, self.out, None)
+            dist.all_reduce(self._flag, group=self.group)          # every process has read my rows
+            return
         dist.all_gather_into_tensor(self.lev_all.view(-1), self.lev_local.view(-1), group=self.group)
         self.k.uq_decode(self.total, self.lev_all, self.k.UQ_SRC_LEVELS, self.fmt, self.W, self.s, self.scales,
                          self.idx, self.idx_bits, self.out, None)

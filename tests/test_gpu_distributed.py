@@ -156,5 +156,13 @@ def test_distributed_quantizer_on_one_rank_equals_the_pipeline():
                 norm=B.UQ_NORM_L2, rng_bits=w.rng_bits)
             got = q.step(to_device(w, g_np), w.seed).cpu().numpy()
             assert np.array_equal(got, run_gpu(w, g_np)["out"]) and int(q.status.item()) == 0
+            # the same with the level rows in symmetric memory, read where they are
+            qp = DistributedQuantizer(
+                w.M, w.d, torch.float32, seg_off=wl.segment_offsets(w), s=w.s,
+                scales=list(w.scales) if w.quantizer == "multi" else None, fmt=FMT[w.fmt], idx_bits=w.idx_bits,
+                norm=B.UQ_NORM_L2, rng_bits=w.rng_bits, pull_levels=True)
+            for _ in range(2):
+                got = qp.step(to_device(w, g_np), w.seed).cpu().numpy()
+                assert np.array_equal(got, run_gpu(w, g_np)["out"]) and int(qp.status.item()) == 0
     finally:
         dist.destroy_process_group()
