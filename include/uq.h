@@ -84,6 +84,12 @@ typedef struct uq_layout {
                                buffer holds all workers.  Only the encoders use it: the random
                                draws of row m are those of worker worker0 + m, so a process that
                                holds some of the job's workers produces the same levels */
+    int64_t coord0;         /* index, in the worker's whole gradient, of coordinate 0 of this buffer
+                               (>= 0, a multiple of 8); 0 when the buffer holds the whole gradient.
+                               Only the encoders use it: coordinate i draws the random number of
+                               coordinate coord0 + i, so a gradient handed over piece by piece (a
+                               bucket at a time, with seg_off counted from the piece's start) gets
+                               the levels of the one-piece call */
 } uq_layout;
 
 /* Library version (major*10000 + minor*100 + patch). */

@@ -39,6 +39,7 @@ class uq_layout(C.Structure):
         ("nseg", C.c_int32),
         ("dtype", C.c_int32),
         ("worker0", C.c_int32),
+        ("coord0", C.c_int64),
     ]
 
 
@@ -121,7 +122,7 @@ class Layout:
     ``worker_stride`` coordinates, cut into segments that each share one scale."""
 
     def __init__(self, M: int, d: int, worker_stride: int, dtype: torch.dtype,
-                 seg_off: Optional[torch.Tensor] = None, worker0: int = 0):
+                 seg_off: Optional[torch.Tensor] = None, worker0: int = 0, coord0: int = 0):
         if dtype not in (torch.float32, torch.bfloat16):
             raise ValueError("uq: gradients are float32 or bfloat16")
         if seg_off is not None:
@@ -130,9 +131,9 @@ class Layout:
             seg_off = seg_off.contiguous()
         self.M, self.d, self.worker_stride, self.dtype, self.seg_off = M, d, worker_stride, dtype, seg_off
         self.nseg = 1 if seg_off is None else seg_off.numel() - 1
-        self.worker0 = worker0
+        self.worker0, self.coord0 = worker0, coord0
         self.c = uq_layout(d, worker_stride, _ptr(seg_off), M, self.nseg,
-                           UQ_F32 if dtype == torch.float32 else UQ_BF16, worker0)
+                           UQ_F32 if dtype == torch.float32 else UQ_BF16, worker0, coord0)
 
     def ref(self):
         return C.byref(self.c)

@@ -50,6 +50,7 @@ bool layout_ok(const uq_layout *L)
     if (L->seg_off == nullptr && L->nseg != 1) return false;
     if (L->seg_off != nullptr && !aligned(L->seg_off, 8)) return false;
     if (L->d > (int64_t)1 << 40) return false;
+    if (L->coord0 < 0 || (L->coord0 & 7) != 0 || L->coord0 > (int64_t)1 << 40) return false;
     return true;
 }
 
@@ -267,6 +268,7 @@ int uq_randk_gather(const uq_layout *L, const void *g, int64_t K, uint64_t seed,
     dense.seg_off = nullptr;
     dense.nseg = 1;
     dense.worker0 = 0;
+    dense.coord0 = 0;
     if (!layout_ok(&dense) || !aligned(status, 4)) return UQ_ERR_BAD_ARG;
     if (K < 0 || K > dense.d || gk_stride < K || (gk_stride & 31) != 0) return UQ_ERR_BAD_ARG;
     if (gk_stride > 0 && (gk == nullptr || !aligned(gk, 16))) return UQ_ERR_BAD_ARG;

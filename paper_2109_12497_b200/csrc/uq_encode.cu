@@ -20,6 +20,7 @@ struct EncodeParams {
     int64_t d, stride;
     int32_t nseg, M;
     int32_t worker0;          // number, in the whole job, of the worker in row 0 (keys the draws)
+    int64_t coord0;           // index, in the whole gradient, of coordinate 0 (keys the draws)
     int64_t ntiles;
     uint32_t main_blocks;     // CTAs that own tiles; the CTAs after them own rows crossed by boundaries
     float cap;                // (float) of the smallest scale: the largest level
@@ -204,7 +205,7 @@ __device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, i
             overflow |= not_finite(inv[e]);
         }
         if (overflow && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
-        const uint64_t blk = RNG == 32 ? (uint64_t)(i >> 2) : (uint64_t)(i >> 3);
+        const uint64_t blk = RNG == 32 ? (uint64_t)((p.coord0 + i) >> 2) : (uint64_t)((p.coord0 + i) >> 3);
         char *dst = (char *)p.lev + (size_t)m * (size_t)(p.stride >> FMT) + (i >> FMT);     // 8 >> FMT bits per level
         quantize_unit<FMT, RNG>(v, inv, p.cap, neg_lo, neg_hi, p.key, (uint32_t)blk, (uint32_t)(blk >> 32), (uint32_t)(m + p.worker0),
                                 dst);
@@ -246,7 +247,13 @@ __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, IDXB != 0>::MIN_CTA
     const int64_t t0 = tile * S::TILE;
     const int64_t t1 = min(t0 + (int64_t)S::TILE, p.d);
 
-    if (t1 - t0 != S::TILE) {                                    // the ragged last tile
+    // Philox block of the tile's first unit.  The units of a tile add less than 2^13 to it; the
+    // straight-line path keeps the high word fixed, so the one tile in 2^35 coordinates in which
+    // the low word wraps takes the general path (64-bit block numbers) like the ragged last tile.
+    constexpr int BSH = RNG == 32 ? 2 : 3;                       // coordinates per Philox block, log2
+    const uint64_t blk0 = (uint64_t)(p.coord0 >> BSH) + (uint64_t)tile * (uint32_t)(S::TILE >> BSH);
+    const bool wraps = (uint32_t)blk0 > 0xFFFFFFFFu - (uint32_t)(S::TILE >> BSH);
+    if (t1 - t0 != S::TILE || wraps) {
         encode_span_general<DT, FMT, RNG, IDXB>(p, m, t0, t1, tid, kThreads);
         return;
     }
@@ -300,7 +307,6 @@ __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, IDXB != 0>::MIN_CTA
         }
     }
 
-    const uint64_t blk0 = RNG == 32 ? (uint64_t)(t0 >> 2) : (uint64_t)(t0 >> 3);           // low bits are 0
     const uint32_t blk_hi = (uint32_t)(blk0 >> 32);
     const uint32_t blk_lo = (uint32_t)blk0 + (uint32_t)tid * BPU;
     constexpr int UB = 8 >> FMT;                                 // bytes of levels per unit: 8, 4 or 2
@@ -393,7 +399,7 @@ cudaError_t launch_encode(const uq_layout &L, const void *g, const float *W, con
 {
     EncodeParams p;
     p.g = g; p.lev = lev; p.W = W; p.seg_off = L.seg_off; p.idx = idx; p.status = status;
-    p.d = L.d; p.stride = L.worker_stride; p.nseg = L.nseg; p.M = L.M; p.worker0 = L.worker0;
+    p.d = L.d; p.stride = L.worker_stride; p.nseg = L.nseg; p.M = L.M; p.worker0 = L.worker0; p.coord0 = L.coord0;
     p.key = philox_key(seed);
     // CTA order (set in the kernel): the tiles are walked back to front with the worker varying fastest.  The
     // kernel before this one in a step (agree-scale or the selector) ends on the high tiles, so

@@ -21,7 +21,8 @@ def lib():
 
 
 class Layout:
-    def __init__(self, M, d, worker_stride, dtype, seg_off=None, worker0=0):
+    def __init__(self, M, d, worker_stride, dtype, seg_off=None, worker0=0, coord0=0):
+        assert coord0 == 0
         self.M, self.d, self.worker_stride, self.dtype, self.seg_off, self.worker0 = M, d, worker_stride, dtype, seg_off, worker0
         self.nseg = 1 if seg_off is None else seg_off.numel() - 1
 

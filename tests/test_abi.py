@@ -42,7 +42,7 @@ def test_constants_match_the_header():
 
 
 def _layout(**kw):
-    base = dict(d=1000, worker_stride=1024, seg_off=None, M=2, nseg=1, dtype=B.UQ_F32, worker0=0)
+    base = dict(d=1000, worker_stride=1024, seg_off=None, M=2, nseg=1, dtype=B.UQ_F32, worker0=0, coord0=0)
     base.update(kw)
     return B.uq_layout(**base)
 
@@ -62,7 +62,7 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     p = 0x10000
     ok = _layout()
     bad_layouts = [_layout(M=0), _layout(M=65), _layout(d=-1), _layout(worker_stride=992), _layout(nseg=2),
-                   _layout(dtype=5), _layout(worker0=-1), _layout(nseg=0)]
+                   _layout(dtype=5), _layout(worker0=-1), _layout(nseg=0), _layout(coord0=4), _layout(coord0=-8)]
     for L in bad_layouts:
         assert lib.uq_agree_scale(C.byref(L), p, B.UQ_NORM_L2, p, None, p, 1 << 20, None) == B.UQ_ERR_BAD_ARG
         assert lib.uq_encode_single(C.byref(L), p, p, 127, 0, 32, B.UQ_FMT_I8, p, None, None) == B.UQ_ERR_BAD_ARG

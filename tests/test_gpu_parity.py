@@ -7,6 +7,7 @@ import torch
 
 from paper_2109_12497_b200 import binding as B
 from paper_2109_12497_b200 import workloads as wl
+from oracle import uq_oracle as o
 from parity import check_parity, run_gpu, run_oracle, to_device
 
 pytestmark = pytest.mark.gpu
@@ -225,3 +226,65 @@ def test_reproducible_bit_for_bit():
     assert np.array_equal(a["lev"][:, : w.d], b["lev"][:, : w.d])          # padding is not data
     nb = w.d * w.idx_bits // 8
     assert np.array_equal(a["idx"][:nb], b["idx"][:nb])
+
+
+@pytest.mark.parametrize("name,kw", [("c2", {}), ("c2", dict(rng_bits=32)), ("c3", {}), ("c5", {}),
+                                      ("c4", {}), ("c3", dict(fmt="i2x4", s=1, scales=(1, 16, 256)))])
+def test_gradient_handed_over_in_pieces(name, kw):
+    """The encoders on pieces of the gradient (layout.coord0 = start of the piece, seg_off counted
+    from the piece's start, pointers moved to the piece) write the levels of the one-piece call."""
+    import ctypes as C
+    d = 250_000
+    w = wl.scaled(name, d, M=4, **kw)
+    g_np = wl.generate(w)
+    one = run_gpu(w, g_np)
+    q = one["q"]
+    g = to_device(w, g_np)
+    seg = np.asarray(wl.segment_offsets(w), dtype=np.int64)
+    eb = 4 if w.dtype == wl.F32 else 2
+    fmt_shift = {"i8": 0, "i4x2": 1, "i2x4": 2}[w.fmt]
+    lev = torch.zeros_like(q.lev)
+    cuts = [0, 256, 16384 + 512, 100_096, d]
+    lib = B.lib()
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        j0 = int(np.searchsorted(seg, a, side="right") - 1)
+        j1 = int(np.searchsorted(seg, b, side="left"))                     # segments j0 .. j1-1 overlap [a, b)
+        sub = np.clip(seg[j0: j1 + 1] - a, 0, b - a)
+        sub_dev = torch.from_numpy(sub).cuda() if len(sub) > 2 else None
+        lay = B.uq_layout(b - a, q.stride, None if sub_dev is None else sub_dev.data_ptr(), w.M, len(sub) - 1,
+                          B.UQ_F32 if w.dtype == wl.F32 else B.UQ_BF16, 0, a)
+        gp, lp, Wp = g.data_ptr() + a * eb, lev.data_ptr() + (a >> fmt_shift), q.W.data_ptr() + 4 * j0
+        if q.multi:
+            sc = (C.c_int32 * len(q.scales))(*q.scales)
+            rc = lib.uq_encode_multi(C.byref(lay), gp, Wp, sc, len(q.scales), q.idx.data_ptr() + a * q.idx_bits // 8,
+                                     q.idx_bits, w.seed, w.rng_bits, q.fmt, lp, q.status.data_ptr(), None)
+        else:
+            rc = lib.uq_encode_single(C.byref(lay), gp, Wp, q.s, w.seed, w.rng_bits, q.fmt, lp, q.status.data_ptr(), None)
+        assert rc == 0
+    torch.cuda.synchronize()
+    nb = d >> fmt_shift
+    assert np.array_equal(lev.cpu().numpy().view(np.uint8)[:, :nb], one["lev"][:, :nb])
+    assert q.status_bits() == 0
+
+
+@pytest.mark.parametrize("rng_bits", [16, 32])
+def test_block_counter_wraps_inside_a_tile(rng_bits):
+    """A piece that starts just below the coordinate where the low word of the Philox block
+    number wraps (2^35 for 16-bit draws, 2^34 for 32-bit draws): levels match the oracle's."""
+    import ctypes as C
+    wrap = 2 ** 35 if rng_bits == 16 else 2 ** 34
+    coord0, d, M = wrap - 40_000, 100_003, 3
+    w = wl.scaled("c1", d, M=M, rng_bits=rng_bits, norm=wl.NORM_L2)
+    g_np = wl.generate(w)
+    g = to_device(w, g_np)
+    stride = g.shape[1]
+    W = torch.from_numpy(o.agree_scale(g_np[:, :d], None, o.NORM_L2)).cuda()
+    lev = torch.zeros((M, stride), dtype=torch.int8, device="cuda")
+    lay = B.uq_layout(d, stride, None, M, 1, B.UQ_F32, 0, coord0)
+    rc = B.lib().uq_encode_single(C.byref(lay), g.data_ptr(), W.data_ptr(), 127, 5, rng_bits, B.UQ_FMT_I8, lev.data_ptr(),
+                                  None, None)
+    assert rc == 0
+    want = o.encode_single(g_np[:, :d], W.cpu().numpy(), 127, 5, rng_bits, coord0=coord0)
+    assert np.array_equal(lev.cpu().numpy()[:, :d], want)
+    # the draws really moved: the same data at coord0 = 0 gives other levels
+    assert not np.array_equal(o.encode_single(g_np[:, :d], W.cpu().numpy(), 127, 5, rng_bits), want)

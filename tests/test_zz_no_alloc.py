@@ -59,9 +59,9 @@ def test_layouts_beyond_the_built_in_scratch_are_refused_before_any_launch():
     runs without a GPU (the pointers are never used)."""
     lib = B.lib()
     p = 0x10000
-    big = B.uq_layout(d=1 << 33, worker_stride=1 << 33, seg_off=None, M=8, nseg=1, dtype=B.UQ_F32, worker0=0)
+    big = B.uq_layout(d=1 << 33, worker_stride=1 << 33, seg_off=None, M=8, nseg=1, dtype=B.UQ_F32, worker0=0, coord0=0)
     assert lib.uq_workspace_bytes(C.byref(big)) > B.STATIC_SCRATCH_BYTES
     assert lib.uq_agree_scale_static(C.byref(big), p, B.UQ_NORM_L2, p, None, None) == B.UQ_ERR_WORKSPACE
-    bad = B.uq_layout(d=100, worker_stride=100, seg_off=None, M=8, nseg=1, dtype=B.UQ_F32, worker0=0)
+    bad = B.uq_layout(d=100, worker_stride=100, seg_off=None, M=8, nseg=1, dtype=B.UQ_F32, worker0=0, coord0=0)
     assert lib.uq_agree_scale_static(C.byref(bad), p, B.UQ_NORM_L2, p, None, None) == B.UQ_ERR_BAD_ARG
     assert b"workspace" in lib.uq_error_string(B.UQ_ERR_WORKSPACE)
