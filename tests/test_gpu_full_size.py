@@ -94,3 +94,49 @@ def _even_stride(lev):
     buf = np.zeros((M, n + (n & 1) + 2), dtype=np.int8)
     buf[:, :n] = lev
     return buf[:, :n]
+
+
+@pytest.mark.parametrize("quantizer", ["single", "multi"])
+def test_more_than_2_31_coordinates(quantizer):
+    """d = 2^31 + 4099 (bf16, two workers): every index, offset and block number beyond 32 bits.
+    The data are drawn on the GPU (seeded) with |v| <= 4 and one planted value of 8, so the L-inf
+    scale is 8 by construction; windows around 2^31, 2^32 bytes and the ragged end are compared
+    with the oracle coordinate by coordinate."""
+    from paper_2109_12497_b200 import binding as B
+    from paper_2109_12497_b200.pipeline import Quantizer
+    d, M = 2 ** 31 + 4099, 2
+    scales = (127, 1016, 8128) if quantizer == "multi" else None
+    q = Quantizer(M, d, torch.bfloat16, s=127, scales=scales, fmt=B.UQ_FMT_I8, idx_bits=2 if scales else 0,
+                  norm=B.UQ_NORM_LINF, rng_bits=16, keep_sums=True)
+    g = torch.empty((M, q.stride), dtype=torch.bfloat16, device="cuda")
+    gen = torch.Generator(device="cuda").manual_seed(2031)
+    chunk = 1 << 28
+    for m in range(M):
+        for a in range(0, q.stride, chunk):
+            n = min(chunk, q.stride - a)
+            g[m, a: a + n] = (torch.randn(n, device="cuda", generator=gen) * 0.7).clamp_(-4, 4).to(torch.bfloat16)
+    g[:, d:] = 0
+    g[1, 2 ** 31 + 5] = -8.0
+    q.step(g, 3)
+    torch.cuda.synchronize()
+    assert q.status_bits() == 0
+    W = q.W.cpu().numpy()
+    assert W.tolist() == [8.0]
+    size = 20_000
+    for a in (0, 2 ** 30 - 77, 2 ** 31 - size // 2, 2 ** 31 + 4099 - size, 1_500_000_001):
+        b = min(d, a + size)
+        gw = g[:, a:b].contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+        if scales:
+            idx = o.select_scale_multi(gw, W, scales, coord0=a)
+            lev = o.encode_multi(gw, W, scales, idx, 3, 16, coord0=a)
+            out = o.decode(o.aggregate(lev), M, W, scales=scales, idx=idx, coord0=a)
+            a4, b4 = -(-a // 4) * 4, b // 4 * 4
+            assert np.array_equal(q.idx[a4 // 4: b4 // 4].cpu().numpy(), o.pack_index(idx[a4 - a: b4 - a], 2)), a
+        else:
+            lev = o.encode_single(gw, W, 127, 3, 16, coord0=a)
+            out = o.decode(o.aggregate(lev), M, W, s=127, coord0=a)
+        assert np.array_equal(q.lev[:, a:b].cpu().numpy(), lev), a
+        assert np.array_equal(q.S[a:b].cpu().numpy(), o.aggregate(lev)), a
+        assert np.allclose(q.out[a:b].cpu().numpy(), out, rtol=FP32_RTOL, atol=0), a
+    del g, q
+    torch.cuda.empty_cache()
