@@ -181,7 +181,8 @@ int uq_encode_single(const uq_layout *layout, const void *g, const float *W, int
  *                       (k = 0 if none; a zero coordinate or W[j] = 0 gives N-1)
  *   shared index        k_i = min over workers of k^m_i.
  *   scales    host  N ascending integers >= 1, N <= UQ_MAX_SCALES; scales[0] is the smallest scale
- *   idx_bits  2 (N <= 4), 4 (N <= 16) or 8
+ *   idx_bits  1 (N <= 2: the two-scale compressors of the paper's experiments), 2 (N <= 4),
+ *             4 (N <= 16) or 8
  *   idx       out   packed little-endian within each byte (coordinate i at bit (i*idx_bits)%8
  *                   of byte (i*idx_bits)/8); the buffer holds uq_index_bytes(layout, idx_bits)
  *                   bytes and is 16-byte aligned; the bits of coordinates d .. 8*ceil(d/8)-1
@@ -271,11 +272,11 @@ int uq_decode_update(const uq_layout *layout, const void *lev, int fmt, const fl
  * when the M workers are spread over R processes: each process runs uq_select_scale_multi on
  * its own workers (with the job-wide W), the R packed index rows are brought together (an
  * all-gather), and the shared index is their field-wise minimum.
- *   rows      in   [R][row_bytes] packed indices, device, 8-byte aligned, row r = process r
+ *   rows      in   [R][row_bytes] packed indices, device, 4-byte aligned, row r = process r
  *   R              1..UQ_MAX_WORKERS
- *   row_bytes      distance between rows, a multiple of 8, >= nbytes
- *   nbytes         bytes of one row to reduce, a multiple of 8 (uq_index_bytes() is one)
- *   idx       out  [nbytes] packed shared indices, 8-byte aligned; may be row 0 of rows
+ *   row_bytes      distance between rows, a multiple of 4, >= nbytes
+ *   nbytes         bytes of one row to reduce, a multiple of 4 (uq_index_bytes() is one)
+ *   idx       out  [nbytes] packed shared indices, 4-byte aligned; may be row 0 of rows
  * Errors: UQ_ERR_BAD_ARG, UQ_ERR_CUDA.
  */
 int uq_index_min(const uint8_t *rows, int R, int64_t row_bytes, int64_t nbytes, int idx_bits,

@@ -54,6 +54,8 @@ bool layout_ok(const uq_layout *L)
     return true;
 }
 
+bool idx_bits_ok(int b) { return b == 1 || b == 2 || b == 4 || b == 8; }
+
 bool fmt_known(int fmt) { return fmt == UQ_FMT_I8 || fmt == UQ_FMT_I4X2 || fmt == UQ_FMT_I2X4; }
 
 bool fmt_ok(int fmt, int s_hat)
@@ -68,7 +70,7 @@ bool fmt_ok(int fmt, int s_hat)
 bool scales_ok(const int32_t *scales, int N, int idx_bits, uq::ScaleSet *out)
 {
     if (scales == nullptr || N < 1 || N > UQ_MAX_SCALES) return false;
-    if (idx_bits != 2 && idx_bits != 4 && idx_bits != 8) return false;
+    if (!idx_bits_ok(idx_bits)) return false;
     if (idx_bits < 8 && N > (1 << idx_bits)) return false;
     for (int k = 0; k < N; ++k) {
         if (scales[k] < 1) return false;
@@ -116,7 +118,7 @@ size_t uq_workspace_bytes(const uq_layout *L)
 
 size_t uq_index_bytes(const uq_layout *L, int idx_bits)
 {
-    if (!layout_ok(L) || (idx_bits != 2 && idx_bits != 4 && idx_bits != 8)) return 0;
+    if (!layout_ok(L) || !idx_bits_ok(idx_bits)) return 0;
     return (size_t)L->worker_stride * (size_t)idx_bits / 8;
 }
 
@@ -253,10 +255,10 @@ int uq_decode_update(const uq_layout *L, const void *lev, int fmt, const float *
 
 int uq_index_min(const uint8_t *rows, int R, int64_t row_bytes, int64_t nbytes, int idx_bits, uint8_t *idx, void *stream)
 {
-    if (R < 1 || R > UQ_MAX_WORKERS || nbytes < 0 || (nbytes & 7) != 0 || row_bytes < nbytes || (row_bytes & 7) != 0)
+    if (R < 1 || R > UQ_MAX_WORKERS || nbytes < 0 || (nbytes & 3) != 0 || row_bytes < nbytes || (row_bytes & 3) != 0)
         return UQ_ERR_BAD_ARG;
-    if (idx_bits != 2 && idx_bits != 4 && idx_bits != 8) return UQ_ERR_BAD_ARG;
-    if (nbytes > 0 && (rows == nullptr || idx == nullptr || !aligned(rows, 8) || !aligned(idx, 8))) return UQ_ERR_BAD_ARG;
+    if (!idx_bits_ok(idx_bits)) return UQ_ERR_BAD_ARG;
+    if (nbytes > 0 && (rows == nullptr || idx == nullptr || !aligned(rows, 4) || !aligned(idx, 4))) return UQ_ERR_BAD_ARG;
     return finish(uq::launch_index_min(rows, R, row_bytes, nbytes, idx_bits, idx, (cudaStream_t)stream));
 }
 

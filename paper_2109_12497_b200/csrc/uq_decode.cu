@@ -174,7 +174,7 @@ __global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const __grid
     constexpr int C = U::C;
     constexpr bool MULTI = IDXB != 0;
     constexpr int IB = MULTI ? IDXB : 8;
-    constexpr int WORDS = C * IB / 32;                              // idx words per thread
+    constexpr int WORDS = C * IB >= 32 ? C * IB / 32 : 1;           // idx words per thread (a half word for 16 bits)
     const int tid = threadIdx.x, lane = tid & 31;
     const int64_t i = ((int64_t)blockIdx.x * kThreads + tid) * C;  // my first coordinate
     const int64_t row0 = i - (int64_t)lane * C;                    // my warp's first coordinate
@@ -199,10 +199,14 @@ __global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const __grid
         }
         for (; m < p.M; ++m) unit.add(U::load(ROWS ? (const char *)p.rows[m] + off : col + (size_t)m * row_bytes));
         if (MULTI && p.out != nullptr) {
-            // idx bits of coordinates i..i+C-1 start at byte i*IB/8 (a multiple of 4 bytes)
-            const uint32_t *ip = (const uint32_t *)(p.idx + (size_t)i * IB / 8);
+            // idx bits of coordinates i..i+C-1 start at byte i*IB/8 (a multiple of 4 bytes, of 2 for 16 bits)
+            if (C * IB == 16) {
+                kw[0] = __ldg((const uint16_t *)(p.idx + (size_t)i * IB / 8));
+            } else {
+                const uint32_t *ip = (const uint32_t *)(p.idx + (size_t)i * IB / 8);
 #pragma unroll
-            for (int w = 0; w < WORDS; ++w) kw[w] = __ldg(ip + w);
+                for (int w = 0; w < WORDS; ++w) kw[w] = __ldg(ip + w);
+            }
         }
     }
 
@@ -332,6 +336,7 @@ static cudaError_t dispatch_levels(const DecodeParams &p, int idx_bits, cudaStre
     if (rows) {
         switch (idx_bits) {
         case 0: aggregate_decode_kernel<FMT, 0, false, true><<<nb, kThreads, 0, st>>>(p); break;
+        case 1: aggregate_decode_kernel<FMT, 1, false, true><<<nb, kThreads, 0, st>>>(p); break;
         case 2: aggregate_decode_kernel<FMT, 2, false, true><<<nb, kThreads, 0, st>>>(p); break;
         case 4: aggregate_decode_kernel<FMT, 4, false, true><<<nb, kThreads, 0, st>>>(p); break;
         default: aggregate_decode_kernel<FMT, 8, false, true><<<nb, kThreads, 0, st>>>(p); break;
@@ -341,6 +346,7 @@ static cudaError_t dispatch_levels(const DecodeParams &p, int idx_bits, cudaStre
     if (p.theta != nullptr) {
         switch (idx_bits) {
         case 0: aggregate_decode_kernel<FMT, 0, true><<<nb, kThreads, 0, st>>>(p); break;
+        case 1: aggregate_decode_kernel<FMT, 1, true><<<nb, kThreads, 0, st>>>(p); break;
         case 2: aggregate_decode_kernel<FMT, 2, true><<<nb, kThreads, 0, st>>>(p); break;
         case 4: aggregate_decode_kernel<FMT, 4, true><<<nb, kThreads, 0, st>>>(p); break;
         default: aggregate_decode_kernel<FMT, 8, true><<<nb, kThreads, 0, st>>>(p); break;
@@ -349,6 +355,7 @@ static cudaError_t dispatch_levels(const DecodeParams &p, int idx_bits, cudaStre
     }
     switch (idx_bits) {
     case 0: aggregate_decode_kernel<FMT, 0, false><<<nb, kThreads, 0, st>>>(p); break;
+    case 1: aggregate_decode_kernel<FMT, 1, false><<<nb, kThreads, 0, st>>>(p); break;
     case 2: aggregate_decode_kernel<FMT, 2, false><<<nb, kThreads, 0, st>>>(p); break;
     case 4: aggregate_decode_kernel<FMT, 4, false><<<nb, kThreads, 0, st>>>(p); break;
     default: aggregate_decode_kernel<FMT, 8, false><<<nb, kThreads, 0, st>>>(p); break;
@@ -399,6 +406,7 @@ cudaError_t launch_decode_sums(const uq_layout &L, const int32_t *S, const float
     const unsigned nb = (unsigned)blocks;
     switch (idx_bits) {
     case 0: decode_sums_kernel<0><<<nb, kThreads, 0, st>>>(p); break;
+    case 1: decode_sums_kernel<1><<<nb, kThreads, 0, st>>>(p); break;
     case 2: decode_sums_kernel<2><<<nb, kThreads, 0, st>>>(p); break;
     case 4: decode_sums_kernel<4><<<nb, kThreads, 0, st>>>(p); break;
     default: decode_sums_kernel<8><<<nb, kThreads, 0, st>>>(p); break;

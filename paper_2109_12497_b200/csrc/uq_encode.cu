@@ -60,6 +60,7 @@ __device__ __forceinline__ bool not_finite(float x) { return (__float_as_uint(x)
 
 // The idx_bits * 8 bits that belong to 8 consecutive coordinates starting at a multiple of 8.
 template <int IDXB> struct IdxBits;
+template <> struct IdxBits<1> { using T = uint32_t; static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg(p); } };
 template <> struct IdxBits<2> { using T = uint32_t; static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg((const uint16_t *)p); } };
 template <> struct IdxBits<4> { using T = uint32_t; static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg((const uint32_t *)p); } };
 template <> struct IdxBits<8> { using T = uint64_t; static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg((const unsigned long long *)p); } };
@@ -373,6 +374,7 @@ static cudaError_t dispatch_idx(const EncodeParams &p, int idx_bits, cudaStream_
 {
     switch (idx_bits) {
     case 0: return launch<DT, FMT, RNG, 0>(p, st);
+    case 1: return launch<DT, FMT, RNG, 1>(p, st);
     case 2: return launch<DT, FMT, RNG, 2>(p, st);
     case 4: return launch<DT, FMT, RNG, 4>(p, st);
     default: return launch<DT, FMT, RNG, 8>(p, st);

@@ -171,7 +171,8 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
         packed = select_general(p, i, amag, IDXB, j0);
     }
     if (!active) return;
-    if (IDXB == 2) *(uint16_t *)(p.idx + (i >> 2)) = (uint16_t)packed;
+    if (IDXB == 1) p.idx[i >> 3] = (uint8_t)packed;
+    else if (IDXB == 2) *(uint16_t *)(p.idx + (i >> 2)) = (uint16_t)packed;
     else if (IDXB == 4) *(uint32_t *)(p.idx + (i >> 1)) = (uint32_t)packed;
     else *(uint64_t *)(p.idx + i) = packed;
 }
@@ -193,6 +194,7 @@ static cudaError_t dispatch(const SelectParams &p, int idx_bits, cudaStream_t st
     const int64_t blocks = (p.d + kSelectTile - 1) / kSelectTile;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    if (idx_bits == 1) { select_kernel<DT, 1, 1><<<(unsigned)blocks, kThreads, 0, st>>>(p); return cudaGetLastError(); }
     if (idx_bits == 2) return dispatch_levels<DT, 2>(p, (unsigned)blocks, st);
     if (idx_bits == 4) return dispatch_levels<DT, 4>(p, (unsigned)blocks, st);
     return dispatch_levels<DT, 8>(p, (unsigned)blocks, st);
@@ -215,9 +217,10 @@ cudaError_t launch_select(const uq_layout &L, const void *g, const float *W, con
 // selector writes it; the shared index is the field-wise minimum over the R packed rows.
 // ---------------------------------------------------------------------------------------------
 
-// Field-wise unsigned minimum of two words holding 4, 8 or 16 fields of 8, 4 or 2 bits.
+// Field-wise unsigned minimum of two words holding 4, 8, 16 or 32 fields of 8, 4, 2 or 1 bits.
 template <int IDXB> __device__ __forceinline__ uint32_t min_fields(uint32_t a, uint32_t b)
 {
+    if (IDXB == 1) return a & b;
     if (IDXB == 8) return __vminu4(a, b);
     constexpr uint32_t mask = IDXB == 4 ? 0x0F0F0F0Fu : 0x03030303u;
     uint32_t r = 0;
@@ -230,26 +233,24 @@ template <int IDXB>
 __global__ void __launch_bounds__(kThreads) index_min_kernel(const uint8_t *__restrict__ rows, int R, int64_t row_bytes,
                                                              int64_t nwords, uint8_t *__restrict__ idx)
 {
-    const int64_t w = (int64_t)blockIdx.x * kThreads + threadIdx.x;      // my 8-byte word
+    const int64_t w = (int64_t)blockIdx.x * kThreads + threadIdx.x;      // my 4-byte word
     if (w >= nwords) return;
-    uint2 acc = ld_stream64(rows + w * 8);
-    for (int r = 1; r < R; ++r) {
-        const uint2 q = ld_stream64(rows + (size_t)r * (size_t)row_bytes + w * 8);
-        acc.x = min_fields<IDXB>(acc.x, q.x);
-        acc.y = min_fields<IDXB>(acc.y, q.y);
-    }
-    *(uint2 *)(idx + w * 8) = acc;
+    uint32_t acc = __ldg((const uint32_t *)rows + w);
+    for (int r = 1; r < R; ++r)
+        acc = min_fields<IDXB>(acc, __ldg((const uint32_t *)(rows + (size_t)r * (size_t)row_bytes) + w));
+    ((uint32_t *)idx)[w] = acc;
 }
 
 cudaError_t launch_index_min(const uint8_t *rows, int R, int64_t row_bytes, int64_t nbytes, int idx_bits, uint8_t *idx,
                              cudaStream_t st)
 {
-    const int64_t nwords = nbytes / 8;
+    const int64_t nwords = nbytes / 4;
     const int64_t blocks = (nwords + kThreads - 1) / kThreads;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     const unsigned nb = (unsigned)blocks;
-    if (idx_bits == 2) index_min_kernel<2><<<nb, kThreads, 0, st>>>(rows, R, row_bytes, nwords, idx);
+    if (idx_bits == 1) index_min_kernel<1><<<nb, kThreads, 0, st>>>(rows, R, row_bytes, nwords, idx);
+    else if (idx_bits == 2) index_min_kernel<2><<<nb, kThreads, 0, st>>>(rows, R, row_bytes, nwords, idx);
     else if (idx_bits == 4) index_min_kernel<4><<<nb, kThreads, 0, st>>>(rows, R, row_bytes, nwords, idx);
     else index_min_kernel<8><<<nb, kThreads, 0, st>>>(rows, R, row_bytes, nwords, idx);
     return cudaGetLastError();

@@ -20,7 +20,7 @@ pytestmark = pytest.mark.gpu
 FMT = {"i8": B.UQ_FMT_I8, "i4x2": B.UQ_FMT_I4X2, "i2x4": B.UQ_FMT_I2X4}
 
 
-@pytest.mark.parametrize("idx_bits", [2, 4, 8])
+@pytest.mark.parametrize("idx_bits", [1, 2, 4, 8])
 @pytest.mark.parametrize("R", [1, 2, 3, 8, 64])
 def test_index_min_matches_oracle(idx_bits, R):
     d = 70_016                                      # a multiple of 32 coordinates: whole 8-byte words
@@ -42,7 +42,7 @@ def test_index_min_argument_checks():
     with pytest.raises(B.UqError):
         B.uq_index_min(rows, 3, rows[0])
     with pytest.raises(B.UqError):
-        B.uq_index_min(rows, 4, rows[0], nbytes=12)                       # not whole 8-byte words
+        B.uq_index_min(rows, 4, rows[0], nbytes=10)                       # not whole 4-byte words
 
 
 @pytest.mark.parametrize("name,d,M,parts,kw", [

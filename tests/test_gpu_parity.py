@@ -55,7 +55,7 @@ def test_single_scale_variants(norm, fmt, s, dtype):
     check_parity(w, wl.generate(w))
 
 
-@pytest.mark.parametrize("idx_bits,N", [(2, 2), (2, 4), (4, 3), (4, 8), (4, 16), (8, 5), (8, 16)])
+@pytest.mark.parametrize("idx_bits,N", [(1, 2), (2, 2), (2, 4), (4, 3), (4, 8), (4, 16), (8, 5), (8, 16)])
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
 @pytest.mark.parametrize("fmt,s,ratio", [("i8", 127, 8), ("i4x2", 7, 16), ("i8", 31, 2), ("i2x4", 1, 4)])
 def test_multi_scale_variants(idx_bits, N, dtype, fmt, s, ratio):
@@ -69,12 +69,13 @@ def test_multi_scale_variants(idx_bits, N, dtype, fmt, s, ratio):
 
 @pytest.mark.parametrize("bits,fmt", [((8, 12), "i8"), ((6, 10), "i8"), ((4, 8), "i4x2"), ((2, 6), "i2x4")])
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
-def test_two_scale_pairs_of_the_experiments(bits, fmt, dtype):
+@pytest.mark.parametrize("idx_bits", [1, 2])
+def test_two_scale_pairs_of_the_experiments(bits, fmt, dtype, idx_bits):
     """The two-scale compressors of the paper's experiments, named by the bit widths of their two
     scales: a scale of r bits has s = 2^(r-1) - 1 levels.  The levels travel in the narrowest
-    supported format that holds the smaller scale, the one-bit choice in the 2-bit index field."""
+    supported format that holds the smaller scale, the choice of scale in a 1-bit (or 2-bit) field."""
     scales = tuple(2 ** (r - 1) - 1 for r in bits)
-    w = wl.scaled("c3", 120_011, M=8, idx_bits=2, scales=scales, s=scales[0], fmt=fmt, dtype=dtype)
+    w = wl.scaled("c3", 120_011, M=8, idx_bits=idx_bits, scales=scales, s=scales[0], fmt=fmt, dtype=dtype)
     r = check_parity(w, wl.generate(w))
     assert set(np.unique(r["ref"]["idx_raw"]).tolist()) == {0, 1}
     assert np.abs(r["ref"]["lev_raw"].astype(int)).max() <= scales[0]
