@@ -58,7 +58,7 @@ def hbm_peak():
 
 def algorithmic_bytes(w: wl.Workload) -> dict:
     e = 4 if w.dtype == wl.F32 else 2
-    lev = {"i8": 1.0, "i4x2": 0.5, "i2x4": 0.25}[w.fmt]
+    lev = {"i8": 1.0, "i4x2": 0.5, "i2x4": 0.25, "i6p": 0.75}[w.fmt]
     ib = w.idx_bits / 8.0
     M, d = w.M, w.d
     b = {"agree_scale": e * M * d}
@@ -390,7 +390,7 @@ def summarize(res, peak_gbs):
     out["kernels"][f"encode_rng{other}"] = {
         "ms": round(ms, 5), "algorithmic_MB": round(ab["encode"] / 1e6, 2), "GBps": round(ab["encode"] / ms / 1e6, 1),
         "frac_of_hbm_peak": round(ab["encode"] / ms / 1e6 / peak_gbs, 4), "note": "timed alone, not part of the step"}
-    lev = {"i8": 1.0, "i4x2": 0.5, "i2x4": 0.25}[w.fmt]
+    lev = {"i8": 1.0, "i4x2": 0.5, "i2x4": 0.25, "i6p": 0.75}[w.fmt]
     upd_bytes = lev * w.M * w.d + w.idx_bits / 8.0 * w.d + 16 * w.d      # levels, index, theta and momentum r/w
     ms = res["update_ms"]
     out["kernels"]["aggregate_decode_update"] = {

@@ -21,7 +21,8 @@
  *   - Layout.  Worker m's gradient is g + m*worker_stride elements, coordinates 0..d-1.
  *     worker_stride is a multiple of 32 and >= d; the padding d..worker_stride-1 of each row
  *     must be readable (its values are ignored).  Level rows use the same stride in coordinates
- *     (int8: worker_stride bytes per row; 4-bit: worker_stride/2 bytes; 2-bit: worker_stride/4 bytes); the library may write
+ *     (int8: worker_stride bytes per row; 4-bit: worker_stride/2 bytes; 2-bit: worker_stride/4 bytes;
+ *     6-bit: 3*worker_stride/4 bytes rounded up to 16); the library may write
  *     zeros into a level row's padding.  g and lev must be 16-byte aligned (8-byte rows result for the
  *     2-bit format when worker_stride is not a multiple of 64; that is allowed).
  *   - Segments.  The paper's vector v in R^n is a segment: coordinates seg_off[j]..seg_off[j+1]-1
@@ -58,7 +59,7 @@ enum {
 
 enum { UQ_F32 = 0, UQ_BF16 = 1 };              /* gradient element type */
 enum { UQ_NORM_LINF = 0, UQ_NORM_L2 = 2 };     /* which norm defines the shared scale */
-enum { UQ_FMT_I8 = 0, UQ_FMT_I4X2 = 1, UQ_FMT_I2X4 = 2 }; /* level wire format: 8, 4 or 2 bits per coordinate */
+enum { UQ_FMT_I8 = 0, UQ_FMT_I4X2 = 1, UQ_FMT_I2X4 = 2, UQ_FMT_I6P = 3 }; /* level wire format: 8, 4, 2 or 6 bits per coordinate */
 enum { UQ_SRC_LEVELS = 0, UQ_SRC_SUMS = 1 };   /* what uq_decode reads */
 
 /* bits OR-ed into the device status word */
@@ -166,6 +167,11 @@ int uq_agree_scale_static(const uq_layout *layout, const void *g, int norm, floa
  *                       [M][worker_stride/2] bytes            (1 <= s <= 7)
  *             fmt I2X4: two's-complement 2-bit fields, coordinate 4q+t in bits 2t..2t+1 of
  *                       byte q, [M][worker_stride/4] bytes    (s = 1: levels -1, 0, 1)
+ *             fmt I6P:  two's-complement 6-bit levels in two planes per row: bits 0..3 of every
+ *                       level as nibbles (laid out as I4X2) in the first worker_stride/2 bytes,
+ *                       bits 4..5 as 2-bit fields (laid out as I2X4) in the worker_stride/4
+ *                       bytes after them; rows are 3*worker_stride/4 bytes rounded up to 16
+ *                                                              (1 <= s <= 31)
  *   W    in   [nseg], e.g. from uq_agree_scale; any W[j] >= max|v| keeps |zeta| <= s, and
  *             the clamp keeps it so for any W.
  * Errors: UQ_ERR_BAD_ARG, UQ_ERR_CUDA.
@@ -199,7 +205,7 @@ int uq_select_scale_multi(const uq_layout *layout, const void *g, const float *W
  * uq_encode_single with s replaced by scales[k_i] in inv and the level clamped to scales[0]
  * (the level fits the bits of the smallest scale).
  *   idx  in  the shared indices written by uq_select_scale_multi (same idx_bits)
- *   fmt  I8 needs scales[0] <= 127, I4X2 needs scales[0] <= 7, I2X4 needs scales[0] = 1
+ *   fmt  I8 needs scales[0] <= 127, I6P <= 31, I4X2 <= 7, I2X4 needs scales[0] = 1
  * Errors: UQ_ERR_BAD_ARG, UQ_ERR_CUDA.
  */
 int uq_encode_multi(const uq_layout *layout, const void *g, const float *W, const int32_t *scales,

@@ -368,6 +368,24 @@ void uqo_pack_levels_i2(const int8_t *lev, int M, int64_t d, int64_t stride, uin
         }
 }
 
+/* 6-bit levels (s <= 31) in two planes per row: bits 0..3 of the two's-complement level as
+ * nibbles (even coordinate in the low nibble) in the first stride/2 bytes of the row, bits 4..5
+ * as 2-bit fields (coordinate 4q+t in bits 2t..2t+1 of byte q) in the stride/4 bytes after
+ * them (stride = the layout's row stride in coordinates); rows are row_bytes apart; everything
+ * else in a row is zero. */
+void uqo_pack_levels_i6p(const int8_t *lev, int M, int64_t d, int64_t lev_stride, int64_t stride, int64_t row_bytes,
+                         uint8_t *packed)
+{
+    memset(packed, 0, (size_t)M * (size_t)row_bytes);
+    for (int m = 0; m < M; ++m)
+        for (int64_t i = 0; i < d; ++i) {
+            const unsigned u = (unsigned)lev[(int64_t)m * lev_stride + i] & 63u;     /* lev rows are lev_stride apart */
+            uint8_t *row = packed + (int64_t)m * row_bytes;
+            row[i / 2] |= (uint8_t)((u & 15u) << (4 * (i % 2)));
+            row[stride / 2 + i / 4] |= (uint8_t)((u >> 4) << (2 * (i % 4)));
+        }
+}
+
 /* Scale sharing across processes (Algorithm 2 line "Scale sharing" when each process holds
  * some of the workers): rows[r*d + i] is the minimum over process r's workers, the shared
  * index is the minimum over the R rows. */

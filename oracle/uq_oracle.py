@@ -217,6 +217,19 @@ def pack_levels_i2(lev: np.ndarray) -> np.ndarray:
     return packed[:, : (d + 3) // 4]
 
 
+def pack_levels_i6p(lev: np.ndarray, stride: int) -> np.ndarray:
+    """6-bit levels in two planes per row ([M, row_bytes]: nibbles of bits 0..3 in the first
+    stride/2 bytes, 2-bit fields of bits 4..5 after them); stride = the layout's row stride in
+    coordinates (a multiple of 32), rows are 3*stride/4 bytes rounded up to 16."""
+    assert lev.dtype == np.int8 and stride % 32 == 0
+    M, d, lev_stride = _check_g(lev)
+    row_bytes = (stride // 2 + stride // 4 + 15) // 16 * 16
+    packed = np.zeros((M, row_bytes), dtype=np.uint8)
+    lib().uqo_pack_levels_i6p(_p(lev), M, C.c_int64(d), C.c_int64(lev_stride), C.c_int64(stride), C.c_int64(row_bytes),
+                              _p(packed))
+    return packed
+
+
 def index_min(rows: np.ndarray) -> np.ndarray:
     """Minimum over the rows of an [R, d] array of (unpacked) scale indices."""
     rows = np.ascontiguousarray(rows, dtype=np.uint8)

@@ -19,7 +19,7 @@ LIB_PATH = _PKG / "libuq_b200.so"
 UQ_OK, UQ_ERR_BAD_ARG, UQ_ERR_CUDA, UQ_ERR_UNSUPPORTED, UQ_ERR_WORKSPACE = range(5)
 UQ_F32, UQ_BF16 = 0, 1
 UQ_NORM_LINF, UQ_NORM_L2 = 0, 2
-UQ_FMT_I8, UQ_FMT_I4X2, UQ_FMT_I2X4 = 0, 1, 2
+UQ_FMT_I8, UQ_FMT_I4X2, UQ_FMT_I2X4, UQ_FMT_I6P = 0, 1, 2, 3
 UQ_SRC_LEVELS, UQ_SRC_SUMS = 0, 1
 UQ_STATUS_NONFINITE, UQ_STATUS_BAD_SEGMENTS, UQ_STATUS_SCALE_OVERFLOW, UQ_STATUS_BAD_INDEX = 1, 2, 4, 8
 
@@ -145,6 +145,8 @@ class Layout:
         return int(lib().uq_index_bytes(self.ref(), idx_bits))
 
     def level_row_bytes(self, fmt: int) -> int:
+        if fmt == UQ_FMT_I6P:                       # a nibble plane and a 2-bit plane, rows rounded up to 16 bytes
+            return (self.worker_stride // 2 + self.worker_stride // 4 + 15) // 16 * 16
         return self.worker_stride >> fmt            # 1, 2 or 4 coordinates per byte
 
     def check_g(self, g: torch.Tensor) -> None:

@@ -56,13 +56,14 @@ bool layout_ok(const uq_layout *L)
 
 bool idx_bits_ok(int b) { return b == 1 || b == 2 || b == 4 || b == 8; }
 
-bool fmt_known(int fmt) { return fmt == UQ_FMT_I8 || fmt == UQ_FMT_I4X2 || fmt == UQ_FMT_I2X4; }
+bool fmt_known(int fmt) { return fmt == UQ_FMT_I8 || fmt == UQ_FMT_I4X2 || fmt == UQ_FMT_I2X4 || fmt == UQ_FMT_I6P; }
 
 bool fmt_ok(int fmt, int s_hat)
 {
     if (fmt == UQ_FMT_I8) return s_hat >= 1 && s_hat <= 127;
     if (fmt == UQ_FMT_I4X2) return s_hat >= 1 && s_hat <= 7;
     if (fmt == UQ_FMT_I2X4) return s_hat == 1;
+    if (fmt == UQ_FMT_I6P) return s_hat >= 1 && s_hat <= 31;
     return false;
 }
 

@@ -59,7 +59,8 @@ template <int FMT> struct Unit;
 template <> struct Unit<UQ_FMT_I8> {
     static constexpr int C = 16;
     using Q = uint4;                                             // one worker's levels of the unit
-    static __device__ __forceinline__ Q load(const void *p) { return ld_stream(p); }
+    // row = start of the worker's level row, i = first coordinate of the unit
+    static __device__ __forceinline__ Q load(const char *row, int64_t i, int64_t) { return ld_stream(row + i); }
     // Bytes are biased to unsigned (x ^ 0x80) and added in 16-bit lanes: two lanes per word,
     // M <= 64 workers * 255 < 2^16.  lane layout of word w: even = bytes 0,2; odd = bytes 1,3.
     uint32_t even[4] = {0, 0, 0, 0}, odd[4] = {0, 0, 0, 0};
@@ -89,7 +90,7 @@ template <> struct Unit<UQ_FMT_I8> {
 template <> struct Unit<UQ_FMT_I4X2> {
     static constexpr int C = 32;
     using Q = uint4;
-    static __device__ __forceinline__ Q load(const void *p) { return ld_stream(p); }
+    static __device__ __forceinline__ Q load(const char *row, int64_t i, int64_t) { return ld_stream(row + (i >> 1)); }
     // Nibbles are biased to unsigned (x ^ 8) and added in byte lanes for up to 16 workers
     // (16 * 15 < 256), then widened into 16-bit lanes.
     uint32_t lo8[4] = {0, 0, 0, 0}, hi8[4] = {0, 0, 0, 0};       // byte lanes: even / odd nibbles
@@ -139,7 +140,7 @@ template <> struct Unit<UQ_FMT_I4X2> {
 template <> struct Unit<UQ_FMT_I2X4> {
     static constexpr int C = 32;
     using Q = uint2;
-    static __device__ __forceinline__ Q load(const void *p) { return ld_stream64(p); }
+    static __device__ __forceinline__ Q load(const char *row, int64_t i, int64_t) { return ld_stream64(row + (i >> 2)); }
     // 2-bit fields are biased to unsigned (x ^ 2, so 1..3) and added in byte lanes: field t of
     // every byte of word w goes to acc[w][t]; 64 workers * 3 < 256, so a byte lane never carries.
     uint32_t acc[2][4] = {};
@@ -165,6 +166,75 @@ template <> struct Unit<UQ_FMT_I2X4> {
     }
 };
 
+// 6-bit levels in two planes: zeta = 16 * sx2(bits 4..5) + (bits 0..3), so the sum over workers is
+// 16 * (sum of the 2-bit plane read as signed) + (sum of the nibble plane read as unsigned).
+template <> struct Unit<UQ_FMT_I6P> {
+    static constexpr int C = 32;
+    struct Q { uint4 n; uint2 c; };
+    static __device__ __forceinline__ Q load(const char *row, int64_t i, int64_t stride)
+    {
+        Q q;
+        q.n = ld_stream(row + (i >> 1));
+        q.c = ld_stream64(row + (stride >> 1) + (i >> 2));
+        return q;
+    }
+    uint32_t lo8[4] = {0, 0, 0, 0}, hi8[4] = {0, 0, 0, 0};       // nibble plane, byte lanes: even / odd nibbles
+    uint32_t acc[4][4] = {};                                    // nibble plane, 16-bit lanes
+    uint32_t cr[2][4] = {};                                     // 2-bit plane, byte lanes (biased by 2)
+    int pending = 0;
+    __device__ __forceinline__ void flush()
+    {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            acc[k][0] += lo8[k] & 0x00FF00FFu;
+            acc[k][1] += (lo8[k] >> 8) & 0x00FF00FFu;
+            acc[k][2] += hi8[k] & 0x00FF00FFu;
+            acc[k][3] += (hi8[k] >> 8) & 0x00FF00FFu;
+            lo8[k] = 0; hi8[k] = 0;
+        }
+        pending = 0;
+    }
+    __device__ __forceinline__ void add(const Q &q)
+    {
+        const uint32_t w[4] = { q.n.x, q.n.y, q.n.z, q.n.w };
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            lo8[k] += w[k] & 0x0F0F0F0Fu;                        // unsigned nibbles: 16 * 15 < 256
+            hi8[k] += (w[k] >> 4) & 0x0F0F0F0Fu;
+        }
+        if (++pending == 16) flush();
+        const uint32_t c[2] = { q.c.x, q.c.y };
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const uint32_t b = c[k] ^ 0xAAAAAAAAu;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) cr[k][t] += (b >> (2 * t)) & 0x03030303u;
+        }
+    }
+    __device__ __forceinline__ void finish(int M, int (&s)[32])
+    {
+        flush();
+        int lo[32];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            lo[8 * k + 0] = (int)(acc[k][0] & 0xFFFFu); lo[8 * k + 4] = (int)(acc[k][0] >> 16);
+            lo[8 * k + 2] = (int)(acc[k][1] & 0xFFFFu); lo[8 * k + 6] = (int)(acc[k][1] >> 16);
+            lo[8 * k + 1] = (int)(acc[k][2] & 0xFFFFu); lo[8 * k + 5] = (int)(acc[k][2] >> 16);
+            lo[8 * k + 3] = (int)(acc[k][3] & 0xFFFFu); lo[8 * k + 7] = (int)(acc[k][3] >> 16);
+        }
+        const int bias = 2 * M;
+#pragma unroll
+        for (int k = 0; k < 2; ++k)
+#pragma unroll
+            for (int y = 0; y < 4; ++y)
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const int e = 16 * k + 4 * y + t;
+                    s[e] = 16 * ((int)((cr[k][t] >> (8 * y)) & 0xFFu) - bias) + lo[e];
+                }
+    }
+};
+
 // UPDATE selects the variant that also applies the parameter update (kept apart so that the plain
 // reconstruction keeps its register count).
 template <int FMT, int IDXB, bool UPDATE, bool ROWS = false>
@@ -181,23 +251,23 @@ __global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const __grid
     if (row0 >= p.d) return;                                       // warp-uniform
     const bool active = i < p.d;
     using Q = typename U::Q;
-    const size_t row_bytes = (size_t)(p.stride >> FMT);            // 8 >> FMT bits per level
+    const size_t row_bytes = LevelFmt<FMT>::row_bytes(p.stride);
 
     U unit;
     uint32_t kw[WORDS];
     if (active) {
-        const size_t off = (size_t)(i >> FMT);                     // my bytes inside a level row
-        const char *col = (const char *)p.lev + off;
         int m = 0;
         for (; m + 8 <= p.M; m += 8) {          // eight workers' loads in flight
             Q q[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k)
-                q[k] = U::load(ROWS ? (const char *)p.rows[m + k] + off : col + (size_t)(m + k) * row_bytes);
+                q[k] = U::load(ROWS ? (const char *)p.rows[m + k] : (const char *)p.lev + (size_t)(m + k) * row_bytes, i,
+                               p.stride);
 #pragma unroll
             for (int k = 0; k < 8; ++k) unit.add(q[k]);
         }
-        for (; m < p.M; ++m) unit.add(U::load(ROWS ? (const char *)p.rows[m] + off : col + (size_t)m * row_bytes));
+        for (; m < p.M; ++m)
+            unit.add(U::load(ROWS ? (const char *)p.rows[m] : (const char *)p.lev + (size_t)m * row_bytes, i, p.stride));
         if (MULTI && p.out != nullptr) {
             // idx bits of coordinates i..i+C-1 start at byte i*IB/8 (a multiple of 4 bytes, of 2 for 16 bits)
             if (C * IB == 16) {
@@ -375,7 +445,8 @@ cudaError_t launch_aggregate_decode(const uq_layout &L, const void *lev, int fmt
     p.theta = theta; p.mom = mom; p.lr = lr; p.mu = mu; p.wd = wd;
     if (fmt == UQ_FMT_I8) return dispatch_levels<UQ_FMT_I8>(p, idx_bits, st);
     if (fmt == UQ_FMT_I4X2) return dispatch_levels<UQ_FMT_I4X2>(p, idx_bits, st);
-    return dispatch_levels<UQ_FMT_I2X4>(p, idx_bits, st);
+    if (fmt == UQ_FMT_I2X4) return dispatch_levels<UQ_FMT_I2X4>(p, idx_bits, st);
+    return dispatch_levels<UQ_FMT_I6P>(p, idx_bits, st);
 }
 
 // The same with the level rows given one by one (lev_rows[m] = start of worker m's row).
@@ -390,7 +461,8 @@ cudaError_t launch_aggregate_decode_rows(const uq_layout &L, const void *const *
     for (int m = 0; m < UQ_MAX_WORKERS; ++m) p.rows[m] = m < L.M ? lev_rows[m] : nullptr;
     if (fmt == UQ_FMT_I8) return dispatch_levels<UQ_FMT_I8>(p, idx_bits, st, true);
     if (fmt == UQ_FMT_I4X2) return dispatch_levels<UQ_FMT_I4X2>(p, idx_bits, st, true);
-    return dispatch_levels<UQ_FMT_I2X4>(p, idx_bits, st, true);
+    if (fmt == UQ_FMT_I2X4) return dispatch_levels<UQ_FMT_I2X4>(p, idx_bits, st, true);
+    return dispatch_levels<UQ_FMT_I6P>(p, idx_bits, st, true);
 }
 
 cudaError_t launch_decode_sums(const uq_layout &L, const int32_t *S, const float *W, const ScaleSet &scales,

@@ -280,6 +280,25 @@ __device__ __forceinline__ uint32_t bytes_to_nibbles(uint32_t lo, uint32_t hi)
 }
 
 // ---------------------------------------------------------------------------------------------
+// Level wire formats: bytes of one worker's level row, and where the levels of the unit of 8
+// coordinates that starts at coordinate i (a multiple of 8) sit in it.  UQ_FMT_I6P keeps two
+// planes per row: the low four bits of every level as nibbles (as UQ_FMT_I4X2) in the first
+// stride/2 bytes, bits 4 and 5 as 2-bit fields (as UQ_FMT_I2X4) in the stride/4 bytes that follow.
+// ---------------------------------------------------------------------------------------------
+template <int FMT> struct LevelFmt {
+    static constexpr int UB = 8 >> FMT;                                        // bytes per unit
+    static __host__ __device__ __forceinline__ size_t row_bytes(int64_t stride) { return (size_t)(stride >> FMT); }
+    static __host__ __device__ __forceinline__ size_t off(int64_t i) { return (size_t)(i >> FMT); }
+    static __host__ __device__ __forceinline__ size_t off2(int64_t, int64_t) { return 0; }
+};
+template <> struct LevelFmt<UQ_FMT_I6P> {
+    static constexpr int UB = 4, UB2 = 2;                                      // nibble plane, 2-bit plane
+    static __host__ __device__ __forceinline__ size_t row_bytes(int64_t stride) { return ((size_t)(stride >> 1) + (size_t)(stride >> 2) + 15) & ~(size_t)15; }
+    static __host__ __device__ __forceinline__ size_t off(int64_t i) { return (size_t)(i >> 1); }
+    static __host__ __device__ __forceinline__ size_t off2(int64_t i, int64_t stride) { return (size_t)(stride >> 1) + (size_t)(i >> 2); }
+};
+
+// ---------------------------------------------------------------------------------------------
 // the segment of a tile, found by one warp without shared memory
 // ---------------------------------------------------------------------------------------------
 

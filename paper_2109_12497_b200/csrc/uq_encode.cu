@@ -92,7 +92,7 @@ __device__ __forceinline__ UnitWords<RNG> unit_words(const PhiloxKey &key, uint3
 template <int FMT, int RNG>
 __device__ __forceinline__ void quantize_unit_words(const float (&v)[8], const float (&inv)[8], float cap,
                                                     uint32_t neg_lo, uint32_t neg_hi, const UnitWords<RNG> &rw,
-                                                    void *dst, bool store = true)
+                                                    void *dst, void *dst2, bool store = true)
 {
     constexpr uint32_t LB = RNG == 32 ? kLevelByte23 : kLevelByte16;
     uint32_t z[8];
@@ -117,16 +117,20 @@ __device__ __forceinline__ void quantize_unit_words(const float (&v)[8], const f
     // back, and what is still in L2 then costs no DRAM read (measured: 7-9 % off that kernel)
     if (FMT == UQ_FMT_I8) *(uint2 *)dst = make_uint2(lo, hi);
     else if (FMT == UQ_FMT_I4X2) *(uint32_t *)dst = bytes_to_nibbles(lo, hi);
-    else *(unsigned short *)dst = (unsigned short)bytes_to_crumbs(lo, hi);
+    else if (FMT == UQ_FMT_I2X4) *(unsigned short *)dst = (unsigned short)bytes_to_crumbs(lo, hi);
+    else {                                          // 6-bit: bits 0..3 as nibbles, bits 4..5 as 2-bit fields
+        *(uint32_t *)dst = bytes_to_nibbles(lo, hi);
+        *(unsigned short *)dst2 = (unsigned short)bytes_to_crumbs(lo >> 4, hi >> 4);
+    }
 }
 
 template <int FMT, int RNG>
 __device__ __forceinline__ void quantize_unit(const float (&v)[8], const float (&inv)[8], float cap,
                                               uint32_t neg_lo, uint32_t neg_hi, const PhiloxKey &key,
                                               uint32_t blk_lo, uint32_t blk_hi, uint32_t m, void *dst,
-                                              bool store = true)
+                                              void *dst2, bool store = true)
 {
-    quantize_unit_words<FMT, RNG>(v, inv, cap, neg_lo, neg_hi, unit_words<RNG>(key, blk_lo, blk_hi, m), dst, store);
+    quantize_unit_words<FMT, RNG>(v, inv, cap, neg_lo, neg_hi, unit_words<RNG>(key, blk_lo, blk_hi, m), dst, dst2, store);
 }
 
 // The sign masks of a unit, from the raw loaded words (before any padding is zeroed).
@@ -207,9 +211,9 @@ __device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, i
         }
         if (overflow && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
         const uint64_t blk = RNG == 32 ? (uint64_t)((p.coord0 + i) >> 2) : (uint64_t)((p.coord0 + i) >> 3);
-        char *dst = (char *)p.lev + (size_t)m * (size_t)(p.stride >> FMT) + (i >> FMT);     // 8 >> FMT bits per level
+        char *lrow = (char *)p.lev + (size_t)m * LevelFmt<FMT>::row_bytes(p.stride);
         quantize_unit<FMT, RNG>(v, inv, p.cap, neg_lo, neg_hi, p.key, (uint32_t)blk, (uint32_t)(blk >> 32), (uint32_t)(m + p.worker0),
-                                dst);
+                                lrow + LevelFmt<FMT>::off(i), lrow + LevelFmt<FMT>::off2(i, p.stride));
     }
 }
 
@@ -310,8 +314,12 @@ __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, IDXB != 0>::MIN_CTA
 
     const uint32_t blk_hi = (uint32_t)(blk0 >> 32);
     const uint32_t blk_lo = (uint32_t)blk0 + (uint32_t)tid * BPU;
-    constexpr int UB = 8 >> FMT;                                 // bytes of levels per unit: 8, 4 or 2
-    char *lp = (char *)p.lev + (size_t)m * (size_t)(p.stride >> FMT) + (size_t)(t0 >> FMT) + tid * UB;
+    using LF = LevelFmt<FMT>;
+    constexpr int UB = LF::UB;                                   // bytes of levels per unit: 8, 4 or 2
+    constexpr int UB2 = FMT == UQ_FMT_I6P ? 2 : 0;               // and in the second plane of the 6-bit format
+    char *lrow = (char *)p.lev + (size_t)m * LF::row_bytes(p.stride);
+    char *lp = lrow + LF::off(t0) + tid * UB;
+    char *lp2 = lrow + LF::off2(t0, p.stride) + tid * UB2;
     // One straight-line pass over all units, so the compiler can interleave them.  A crossed row
     // runs through the arithmetic too but is not stored: a CTA of the second kind owns it.
 #pragma unroll
@@ -348,7 +356,7 @@ __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, IDXB != 0>::MIN_CTA
             uint32_t neg_lo, neg_hi;
             unit_signs<DT>(q[u], neg_lo, neg_hi);
             quantize_unit_words<FMT, RNG>(v, inv, p.cap, neg_lo, neg_hi, rw[n], lp + u * kThreads * UB,
-                                          !((crossed >> u) & 1u));
+                                          lp2 + u * kThreads * UB2, !((crossed >> u) & 1u));
         }
     }
     if (overflow && lane < p.scales.N && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
@@ -390,8 +398,11 @@ static cudaError_t dispatch_fmt(const EncodeParams &p, int fmt, int rng_bits, in
     if (fmt == UQ_FMT_I4X2)
         return rng_bits == 32 ? dispatch_idx<DT, UQ_FMT_I4X2, 32>(p, idx_bits, st)
                               : dispatch_idx<DT, UQ_FMT_I4X2, 16>(p, idx_bits, st);
-    return rng_bits == 32 ? dispatch_idx<DT, UQ_FMT_I2X4, 32>(p, idx_bits, st)
-                          : dispatch_idx<DT, UQ_FMT_I2X4, 16>(p, idx_bits, st);
+    if (fmt == UQ_FMT_I2X4)
+        return rng_bits == 32 ? dispatch_idx<DT, UQ_FMT_I2X4, 32>(p, idx_bits, st)
+                              : dispatch_idx<DT, UQ_FMT_I2X4, 16>(p, idx_bits, st);
+    return rng_bits == 32 ? dispatch_idx<DT, UQ_FMT_I6P, 32>(p, idx_bits, st)
+                          : dispatch_idx<DT, UQ_FMT_I6P, 16>(p, idx_bits, st);
 }
 
 // idx_bits == 0 selects the single-scale quantizer (scales = {s}).

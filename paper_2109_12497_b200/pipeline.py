@@ -141,7 +141,7 @@ def from_workload(w, keep_sums: bool = False, device="cuda") -> Quantizer:
     return Quantizer(
         M=w.M, d=w.d, dtype=torch.float32 if w.dtype == wl.F32 else torch.bfloat16, seg_off=seg, s=w.s,
         scales=list(w.scales) if w.quantizer == "multi" else None,
-        fmt={"i8": B.UQ_FMT_I8, "i4x2": B.UQ_FMT_I4X2, "i2x4": B.UQ_FMT_I2X4}[w.fmt], idx_bits=w.idx_bits,
+        fmt={"i8": B.UQ_FMT_I8, "i4x2": B.UQ_FMT_I4X2, "i2x4": B.UQ_FMT_I2X4, "i6p": B.UQ_FMT_I6P}[w.fmt], idx_bits=w.idx_bits,
         norm=B.UQ_NORM_L2 if w.norm == wl.NORM_L2 else B.UQ_NORM_LINF, rng_bits=w.rng_bits,
         keep_sums=keep_sums, device=device)
 
@@ -153,5 +153,5 @@ def randk_from_workload(w, K: int, device="cuda") -> RandKQuantizer:
     return RandKQuantizer(
         w.M, w.d, K, torch.float32 if w.dtype == wl.F32 else torch.bfloat16, s=w.s,
         scales=list(w.scales) if w.quantizer == "multi" else None,
-        fmt={"i8": B.UQ_FMT_I8, "i4x2": B.UQ_FMT_I4X2, "i2x4": B.UQ_FMT_I2X4}[w.fmt], idx_bits=w.idx_bits,
+        fmt={"i8": B.UQ_FMT_I8, "i4x2": B.UQ_FMT_I4X2, "i2x4": B.UQ_FMT_I2X4, "i6p": B.UQ_FMT_I6P}[w.fmt], idx_bits=w.idx_bits,
         norm=B.UQ_NORM_L2 if w.norm == wl.NORM_L2 else B.UQ_NORM_LINF, rng_bits=w.rng_bits, device=device)

@@ -46,7 +46,7 @@ class Workload:
     segments: str             # "one" | "layers161" | "buckets25MiB"
     s: int                    # levels of the (smallest) scale
     scales: Tuple[int, ...]   # ascending scale set; (s,) for single-scale
-    fmt: str                  # "i8" | "i4x2" | "i2x4"
+    fmt: str                  # "i8" | "i4x2" | "i2x4" | "i6p"
     idx_bits: int             # 0 for single-scale
     norm: str
     seed: int                 # seed of the quantizer's random draws

@@ -61,6 +61,8 @@ def run_oracle(w, g_np, W=None, seed=None):
         res["lev"] = o.pack_levels_i4(lev)
     elif w.fmt == "i2x4":
         res["lev"] = o.pack_levels_i2(lev)
+    elif w.fmt == "i6p":
+        res["lev"] = o.pack_levels_i6p(lev, -(-w.d // 32) * 32)
     else:
         res["lev"] = np.ascontiguousarray(lev).view(np.uint8)
     res.update(S=S, out=out)
@@ -87,8 +89,13 @@ def check_parity(w, g_np, seed=None):
         assert dist.max(initial=0) <= 1, f"W differs by {dist.max()} ulp"
     # downstream stages are compared with the oracle fed the GPU's scale bits
     ref = ref_own if dist.max(initial=0) == 0 else run_oracle(w, g_np, gpu["W"], seed)
-    nb_lev = ref["lev"].shape[1]
-    assert np.array_equal(gpu["lev"][:, :nb_lev], ref["lev"]), "levels differ"
+    if w.fmt == "i6p":                       # two planes per row; the rest of a row is padding
+        half = (-(-w.d // 32) * 32) // 2
+        for a, n in ((0, -(-w.d // 2)), (half, -(-w.d // 4))):
+            assert np.array_equal(gpu["lev"][:, a: a + n], ref["lev"][:, a: a + n]), "levels differ"
+    else:
+        nb_lev = ref["lev"].shape[1]
+        assert np.array_equal(gpu["lev"][:, :nb_lev], ref["lev"]), "levels differ"
     if w.quantizer == "multi":
         nb = ref["idx"].size
         assert np.array_equal(gpu["idx"][:nb], ref["idx"]), "scale indices differ"

@@ -34,7 +34,7 @@ def test_every_declared_symbol_is_exported(lib):
 def test_constants_match_the_header():
     text = (ROOT / "include" / "uq.h").read_text()
     for name in ("UQ_OK", "UQ_ERR_BAD_ARG", "UQ_ERR_CUDA", "UQ_ERR_UNSUPPORTED", "UQ_ERR_WORKSPACE",
-                 "UQ_F32", "UQ_BF16", "UQ_NORM_LINF", "UQ_NORM_L2", "UQ_FMT_I8", "UQ_FMT_I4X2", "UQ_FMT_I2X4",
+                 "UQ_F32", "UQ_BF16", "UQ_NORM_LINF", "UQ_NORM_L2", "UQ_FMT_I8", "UQ_FMT_I4X2", "UQ_FMT_I2X4", "UQ_FMT_I6P",
                  "UQ_SRC_LEVELS", "UQ_SRC_SUMS", "UQ_STATUS_NONFINITE", "UQ_STATUS_BAD_SEGMENTS",
                  "UQ_STATUS_SCALE_OVERFLOW", "UQ_STATUS_BAD_INDEX"):
         m = re.search(rf"\b{name}\s*=\s*(\d+)", text)
@@ -71,7 +71,7 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     assert lib.uq_agree_scale(r, p, B.UQ_NORM_L2, p, None, p, 8, None) == B.UQ_ERR_WORKSPACE      # too small
     assert lib.uq_agree_scale(r, p, B.UQ_NORM_L2, p, None, None, 1 << 20, None) == B.UQ_ERR_WORKSPACE
     assert lib.uq_agree_scale(r, p + 4, B.UQ_NORM_L2, p, None, p, 1 << 20, None) == B.UQ_ERR_BAD_ARG  # alignment
-    for s, fmt in ((0, B.UQ_FMT_I8), (128, B.UQ_FMT_I8), (8, B.UQ_FMT_I4X2), (2, B.UQ_FMT_I2X4), (5, 3)):
+    for s, fmt in ((0, B.UQ_FMT_I8), (128, B.UQ_FMT_I8), (8, B.UQ_FMT_I4X2), (2, B.UQ_FMT_I2X4), (32, B.UQ_FMT_I6P), (5, 4)):
         assert lib.uq_encode_single(r, p, p, s, 0, 32, fmt, p, None, None) == B.UQ_ERR_BAD_ARG
     assert lib.uq_encode_single(r, p, p, 127, 0, 24, B.UQ_FMT_I8, p, None, None) == B.UQ_ERR_BAD_ARG  # rng_bits
     assert lib.uq_encode_single(r, p, None, 127, 0, 32, B.UQ_FMT_I8, p, None, None) == B.UQ_ERR_BAD_ARG

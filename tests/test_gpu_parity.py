@@ -38,6 +38,8 @@ def test_segmented_workloads_small(name, d, rng_bits):
     ("c4", 1_060_013, 16, {}), ("c5", 1_060_013, 16, {}), ("c5", 2_100_003, 8, dict(rng_bits=32, idx_bits=8)),
     ("c3", 2_100_003, 8, dict(dtype=wl.BF16, fmt="i4x2", s=7, scales=(7, 112, 1792))),
     ("c2", 2_100_003, 8, dict(fmt="i2x4", s=1, scales=(1,))),
+    ("c2", 2_100_003, 8, dict(fmt="i6p", s=31, scales=(31,))),
+    ("c5", 1_060_013, 16, dict(fmt="i6p", s=31, scales=tuple(31 * 8 ** k for k in range(8)))),
     ("c3", 2_100_003, 8, dict(dtype=wl.BF16, fmt="i2x4", s=1, scales=(1, 16, 256))),
 ])
 def test_mid_size_workloads(name, d, M, kw):
@@ -48,7 +50,7 @@ def test_mid_size_workloads(name, d, M, kw):
 
 
 @pytest.mark.parametrize("norm", [wl.NORM_L2, wl.NORM_LINF])
-@pytest.mark.parametrize("fmt,s", [("i8", 127), ("i8", 1), ("i8", 5), ("i4x2", 7), ("i4x2", 1), ("i2x4", 1)])
+@pytest.mark.parametrize("fmt,s", [("i8", 127), ("i8", 1), ("i8", 5), ("i4x2", 7), ("i4x2", 1), ("i2x4", 1), ("i6p", 31), ("i6p", 9)])
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
 def test_single_scale_variants(norm, fmt, s, dtype):
     w = wl.scaled("c2", 50021, M=4, norm=norm, fmt=fmt, s=s, scales=(s,), dtype=dtype)
@@ -57,7 +59,7 @@ def test_single_scale_variants(norm, fmt, s, dtype):
 
 @pytest.mark.parametrize("idx_bits,N", [(1, 2), (2, 2), (2, 4), (4, 3), (4, 8), (4, 16), (8, 5), (8, 16)])
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
-@pytest.mark.parametrize("fmt,s,ratio", [("i8", 127, 8), ("i4x2", 7, 16), ("i8", 31, 2), ("i2x4", 1, 4)])
+@pytest.mark.parametrize("fmt,s,ratio", [("i8", 127, 8), ("i4x2", 7, 16), ("i8", 31, 2), ("i2x4", 1, 4), ("i6p", 31, 16)])
 def test_multi_scale_variants(idx_bits, N, dtype, fmt, s, ratio):
     if s * ratio ** (N - 1) >= 2 ** 31:
         pytest.skip("scale does not fit int32")
@@ -67,7 +69,7 @@ def test_multi_scale_variants(idx_bits, N, dtype, fmt, s, ratio):
     assert len(np.unique(r["ref"]["idx_raw"])) >= 2          # more than one scale is in use
 
 
-@pytest.mark.parametrize("bits,fmt", [((8, 12), "i8"), ((6, 10), "i8"), ((4, 8), "i4x2"), ((2, 6), "i2x4")])
+@pytest.mark.parametrize("bits,fmt", [((8, 12), "i8"), ((6, 10), "i8"), ((6, 10), "i6p"), ((4, 8), "i4x2"), ((2, 6), "i2x4")])
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
 @pytest.mark.parametrize("idx_bits", [1, 2])
 def test_two_scale_pairs_of_the_experiments(bits, fmt, dtype, idx_bits):
@@ -98,6 +100,20 @@ def test_two_bit_levels(M, d):
     assert set(np.unique(r["ref"]["lev_raw"]).tolist()) <= {-1, 0, 1}
     from paper_2109_12497_b200.pipeline import from_workload
     bad = from_workload(dataclasses.replace(w, s=2, scales=(2,)))             # the format takes s = 1 only
+    with pytest.raises(B.UqError):
+        bad.encode(to_device(w, wl.generate(w)), 0)
+
+
+@pytest.mark.parametrize("M", [1, 3, 16, 17, 33, 64])
+@pytest.mark.parametrize("d", [5, 31, 33, 8191, 70001])
+def test_six_bit_levels(M, d):
+    """Levels -31..31 in two planes: worker counts across the flush of the nibble lanes (16) up
+    to the limit, sizes around the 32-coordinate unit, and the format limit s <= 31."""
+    w = wl.scaled("c1", d, M=M, fmt="i6p", s=31, scales=(31,))
+    r = check_parity(w, wl.generate(w))
+    assert np.abs(r["ref"]["lev_raw"].astype(int)).max() == 31        # max|g| scale: the top level is in use
+    from paper_2109_12497_b200.pipeline import from_workload
+    bad = from_workload(dataclasses.replace(w, s=32, scales=(32,)))
     with pytest.raises(B.UqError):
         bad.encode(to_device(w, wl.generate(w)), 0)
 

@@ -223,3 +223,19 @@ def test_int2_packing_layout():
     for m in range(2):
         bits = np.repeat(packed[m], 4) >> np.tile(np.arange(4) * 2, 2) & 3
         assert (((bits ^ 2) - 2)[:5] == lev[m]).all()
+
+
+def test_int6_planar_packing_layout():
+    """Two planes per row: nibbles of bits 0..3, then 2-bit fields of bits 4..5 at byte stride/2."""
+    lev = np.array([[-31, 31, 0, -1, 17, -16]], dtype=np.int8)
+    buf = np.zeros((1, 32), dtype=np.int8); buf[:, :6] = lev
+    packed = o.pack_levels_i6p(buf[:, :6], 32)
+    assert packed.shape == (1, 32)                   # 16 + 8 = 24 bytes, rounded up to 16
+    # 6-bit codes: -31 = 100001, 31 = 011111, 0, -1 = 111111, 17 = 010001, -16 = 110000
+    assert packed[0, :3].tolist() == [0xF1, 0xF0, 0x01]                       # nibbles 1 F | 0 F | 1 0
+    assert packed[0, 16:18].tolist() == [0b11_00_01_10, 0b11_01]             # fields 10 01 00 11 | 01 11
+    assert not packed[0, 3:16].any() and not packed[0, 18:].any()
+    # reading the planes back: 16 * signed(2-bit field) + nibble
+    nib = np.repeat(packed[0, :16], 2) >> np.tile([0, 4], 16) & 15
+    cr = np.repeat(packed[0, 16:24], 4) >> np.tile([0, 2, 4, 6], 8) & 3
+    assert ((16 * ((cr ^ 2) - 2) + nib)[:6] == lev[0]).all()
