@@ -217,6 +217,64 @@ __device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, i
     }
 }
 
+// A full tile that a segment boundary crosses, all 256 threads: the warps walk their 256-coordinate
+// rows one by one.  Lane L takes the end of segment j + L (j = the tile's first segment), so the
+// segment of a row is j + (number of ends at or before the row's start): one ballot per row instead
+// of a search.  A row that itself contains a boundary is skipped: a CTA of the second kind owns it.
+template <int DT, int FMT, int RNG, int IDXB>
+__device__ __noinline__ void encode_tile_mixed(const EncodeParams &p, int m, int64_t t0, int j)
+{
+    using E = Elem<DT>;
+    using S = EncodeShape<DT, IDXB != 0>;
+    using LF = LevelFmt<FMT>;
+    constexpr bool MULTI = IDXB != 0;
+    constexpr int IB = MULTI ? IDXB : 8;
+    constexpr int H = 8 / E::G;
+    constexpr int KMASK = IB < 4 ? (1 << IB) - 1 : UQ_MAX_SCALES - 1;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int32_t my_scale = p.scales.s[lane & KMASK];
+    const int64_t my_end = j + lane < p.nseg ? segment_end(p.seg_off, p.nseg, j + lane, p.d) : INT64_MAX;
+    const char *grow = (const char *)p.g + (size_t)m * (size_t)p.stride * E::BYTES;
+    char *lrow = (char *)p.lev + (size_t)m * LF::row_bytes(p.stride);
+    bool overflow = false;
+#pragma unroll 1
+    for (int u = 0; u < S::UNITS; ++u) {
+        const int64_t r0 = t0 + (int64_t)(u * kThreads + (tid & ~31)) * 8;
+        const int cnt = __popc(__ballot_sync(0xFFFFFFFFu, my_end <= r0));
+        int jr;
+        int64_t end;
+        if (cnt < 32) {
+            jr = j + cnt;
+            end = __shfl_sync(0xFFFFFFFFu, my_end, cnt);
+        } else {                                                 // more than 32 segments inside one tile
+            jr = warp_find_segment(p.seg_off, p.nseg, r0);
+            end = segment_end(p.seg_off, p.nseg, jr, p.d);
+        }
+        if (end < r0 + 256) continue;                            // warp-uniform
+        const float inv_lane = inv_scale(my_scale, __ldg(p.W + jr));
+        overflow |= not_finite(inv_lane);
+        const int64_t i = r0 + lane * 8;
+        uint4 q[H];
+        float v[8], inv[8];
+#pragma unroll
+        for (int h = 0; h < H; ++h) {
+            q[h] = ld_stream(grow + (i + h * E::G) * E::BYTES);
+            E::unpack(q[h], *(float(*)[E::G])(v + h * E::G));
+        }
+        typename IdxBits<IB>::T kbits = 0;
+        if (MULTI) kbits = IdxBits<IB>::load(p.idx + i * IB / 8);
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+            inv[e] = MULTI ? __shfl_sync(0xFFFFFFFFu, inv_lane, (int)(uint32_t)(kbits >> (e * IB))) : inv_lane;
+        uint32_t neg_lo, neg_hi;
+        unit_signs<DT>(q, neg_lo, neg_hi);
+        const uint64_t blk = RNG == 32 ? (uint64_t)((p.coord0 + i) >> 2) : (uint64_t)((p.coord0 + i) >> 3);
+        quantize_unit<FMT, RNG>(v, inv, p.cap, neg_lo, neg_hi, p.key, (uint32_t)blk, (uint32_t)(blk >> 32),
+                                (uint32_t)(m + p.worker0), lrow + LF::off(i), lrow + LF::off2(i, p.stride));
+    }
+    if (overflow && lane < p.scales.N && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
+}
+
 template <int DT, int FMT, int RNG, int IDXB>
 __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, IDXB != 0>::MIN_CTAS)) encode_kernel(const __grid_constant__ EncodeParams p)
 {
@@ -278,39 +336,17 @@ __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, IDXB != 0>::MIN_CTA
     // lane k holds s_k / W_j (single-scale: every lane holds s / W_j)
     const int j = warp_find_segment(p.seg_off, p.nseg, t0);
     const bool tile_uniform = segment_end(p.seg_off, p.nseg, j, p.d) >= t1;
-    constexpr int KMASK = IB < 4 ? (1 << IB) - 1 : UQ_MAX_SCALES - 1;    // lane L holds scale L & KMASK
-    const int32_t my_scale = p.scales.s[lane & KMASK];
-    float inv_row[S::UNITS];                                     // my lane's s_k / W for each of my warp's rows
-    uint32_t crossed = 0;                                        // rows that a segment boundary crosses
-    bool overflow = false;                                       // some s_k / W is not finite
-    if (tile_uniform) {
-        const float inv_lane = inv_scale(my_scale, __ldg(p.W + j));
-        if (MULTI) overflow = not_finite(inv_lane);
-#pragma unroll
-        for (int u = 0; u < S::UNITS; ++u) inv_row[u] = inv_lane;
-    } else {
-        // A segment boundary crosses the tile.  Lane L takes the end of segment j + L, so the
-        // segment of any row is j + (number of ends at or before the row's start): one ballot per
-        // row instead of a search, and the scales of all rows are fetched together.
-        const int64_t my_end = j + lane < p.nseg ? segment_end(p.seg_off, p.nseg, j + lane, p.d) : INT64_MAX;
-#pragma unroll
-        for (int u = 0; u < S::UNITS; ++u) {
-            const int64_t r0 = t0 + (int64_t)(u * kThreads + (tid & ~31)) * 8;
-            const int cnt = __popc(__ballot_sync(0xFFFFFFFFu, my_end <= r0));
-            int jr;
-            int64_t end;
-            if (cnt < 32) {
-                jr = j + cnt;
-                end = __shfl_sync(0xFFFFFFFFu, my_end, cnt);
-            } else {                                             // more than 32 segments inside one tile
-                jr = warp_find_segment(p.seg_off, p.nseg, r0);
-                end = segment_end(p.seg_off, p.nseg, jr, p.d);
-            }
-            if (end < r0 + 256) crossed |= 1u << u;
-            inv_row[u] = inv_scale(my_scale, __ldg(p.W + jr));
-            if (MULTI) overflow |= not_finite(inv_row[u]);
-        }
+    if (!tile_uniform) {
+        // A segment boundary crosses the tile (at most nseg - 1 tiles per worker): a compact loop
+        // over the rows, kept out of line so that its registers do not weigh on the path below.
+        // (The loads issued above are dropped; that loop fetches its rows again, from L2.)
+        encode_tile_mixed<DT, FMT, RNG, IDXB>(p, m, t0, j);
+        return;
     }
+    constexpr int KMASK = IB < 4 ? (1 << IB) - 1 : UQ_MAX_SCALES - 1;    // lane L holds scale L & KMASK
+    const float inv_lane = inv_scale(p.scales.s[lane & KMASK], __ldg(p.W + j));
+    bool overflow = false;                                       // some s_k / W is not finite
+    if (MULTI) overflow = not_finite(inv_lane);
 
     const uint32_t blk_hi = (uint32_t)(blk0 >> 32);
     const uint32_t blk_lo = (uint32_t)blk0 + (uint32_t)tid * BPU;
@@ -320,8 +356,7 @@ __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, IDXB != 0>::MIN_CTA
     char *lrow = (char *)p.lev + (size_t)m * LF::row_bytes(p.stride);
     char *lp = lrow + LF::off(t0) + tid * UB;
     char *lp2 = lrow + LF::off2(t0, p.stride) + tid * UB2;
-    // One straight-line pass over all units, so the compiler can interleave them.  A crossed row
-    // runs through the arithmetic too but is not stored: a CTA of the second kind owns it.
+    // One straight-line pass over all units, so the compiler can interleave them.
 #pragma unroll
     for (int u0 = 0; u0 < S::UNITS; u0 += PG) {
         // the random words of PG units together (16-bit draws: one Philox block per unit)
@@ -340,7 +375,6 @@ __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, IDXB != 0>::MIN_CTA
 #pragma unroll
         for (int n = 0; n < PG; ++n) {
             const int u = u0 + n;
-            const float inv_lane = inv_row[u];
             // where the finiteness check sits is a measured choice: ahead of the loop for the
             // multi-scale variants (1.5 % faster on bf16), inside it for the single-scale ones (the
             // hoisted form compiles to a 3-7 % slower kernel there)
@@ -356,7 +390,7 @@ __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, IDXB != 0>::MIN_CTA
             uint32_t neg_lo, neg_hi;
             unit_signs<DT>(q[u], neg_lo, neg_hi);
             quantize_unit_words<FMT, RNG>(v, inv, p.cap, neg_lo, neg_hi, rw[n], lp + u * kThreads * UB,
-                                          lp2 + u * kThreads * UB2, !((crossed >> u) & 1u));
+                                          lp2 + u * kThreads * UB2);
         }
     }
     if (overflow && lane < p.scales.N && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
