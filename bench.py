@@ -37,9 +37,9 @@ FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only
 
 # DRAM traffic per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum) from
 # the ncu captures summarised under profiles/, keyed by workload; None = not captured.
-# c2: 819.2 MB read + 159.6 MB written by the encode kernel in a capture at full size
+# c2: 838.3 MB read + 155.8 MB written by the encode kernel in a capture at full size
 # (profiles/traffic_c2_full_size.md).
-NCU_TRAFFIC_BYTES = {"c2": 978.8e6}
+NCU_TRAFFIC_BYTES = {"c2": 994.1e6}
 
 
 def hbm_peak():
