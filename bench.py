@@ -150,18 +150,30 @@ def run_stages(q, g, seed, events=None):
 
 
 def time_device_resident(q, g, w, steps, warmup, barrier):
-    """(ms per step, {stage: mean ms}) with inputs resident in HBM, timed with CUDA events."""
+    """(ms per step, {stage: mean ms}) with inputs resident in HBM, timed with CUDA events.
+    The step time comes from a region that holds nothing but the K steps (an event recorded
+    between two kernels would keep the second from being scheduled while the first drains, which
+    the library's launches otherwise allow); the per-stage times come from a second pass with an
+    event after every stage."""
     import torch
+    st = torch.cuda.current_stream()
     stages = STAGES_MULTI if q.multi else STAGES_SINGLE
     for _ in range(warmup):
         run_stages(q, g, w.seed)
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(stages) + 1)] for _ in range(steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize(); barrier()
+    e0.record(st)
     for k in range(steps):
-        run_stages(q, g, w.seed + k, evs[k])
+        run_stages(q, g, w.seed + k)
+    e1.record(st)
     torch.cuda.synchronize(); barrier()
-    total_ms = evs[0][0].elapsed_time(evs[-1][-1])
-    per_stage = {s: statistics.fmean(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(steps))
+    total_ms = e0.elapsed_time(e1)
+    n = min(steps, 10)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(stages) + 1)] for _ in range(n)]
+    for k in range(n):
+        run_stages(q, g, w.seed + k, evs[k])
+    torch.cuda.synchronize()
+    per_stage = {s: statistics.fmean(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(n))
                  for i, s in enumerate(stages)}
     return total_ms / steps, per_stage
 

@@ -114,6 +114,7 @@ __global__ void __launch_bounds__(kThreads, 8)     // 32 registers: eight CTAs p
 norm_partials_kernel(const void *__restrict__ g, int64_t d, int64_t stride, int nseg,
                      const int64_t *__restrict__ seg_off, int64_t ntiles, double *__restrict__ part)
 {
+    grid_dependency_prologue();
     using E = Elem<DT>;
     constexpr int UNITS = kNormTile / (kThreads * E::G);
     constexpr bool TILE_MAJOR = DT == UQ_F32;
@@ -203,6 +204,7 @@ norm_finalize_kernel(const double *__restrict__ part, int M, int64_t d, int nseg
                      const int64_t *__restrict__ seg_off, int64_t ntiles, float *__restrict__ W,
                      uint32_t *__restrict__ status)
 {
+    grid_dependency_prologue();
     const int j = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int64_t a = seg_off ? __ldg(seg_off + j) : 0;
@@ -252,10 +254,10 @@ static cudaError_t launch(const uq_layout &L, const void *g, float *W, uint32_t 
         dim3 grid((unsigned)ntiles, (unsigned)L.M);
         if (DT == UQ_F32)
             grid = dim3((unsigned)L.M * (unsigned)min(ntiles, (int64_t)kSlab), (unsigned)((ntiles + kSlab - 1) / kSlab));
-        norm_partials_kernel<DT, NORM><<<grid, kThreads, 0, st>>>(g, L.d, L.worker_stride, L.nseg,
+        launch_k(norm_partials_kernel<DT, NORM>, grid, kThreads, st, g, L.d, L.worker_stride, L.nseg,
                                                                  L.seg_off, ntiles, part);
     }
-    norm_finalize_kernel<NORM><<<L.nseg, kThreads, 0, st>>>(part, L.M, L.d, L.nseg, L.seg_off, ntiles, W,
+    launch_k(norm_finalize_kernel<NORM>, L.nseg, kThreads, st, part, L.M, L.d, L.nseg, L.seg_off, ntiles, W,
                                                           status);
     return cudaGetLastError();
 }

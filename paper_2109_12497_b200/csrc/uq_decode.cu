@@ -240,6 +240,7 @@ template <> struct Unit<UQ_FMT_I6P> {
 template <int FMT, int IDXB, bool UPDATE, bool ROWS = false>
 __global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const __grid_constant__ DecodeParams p)
 {
+    grid_dependency_prologue();
     using U = Unit<FMT>;
     constexpr int C = U::C;
     constexpr bool MULTI = IDXB != 0;
@@ -366,6 +367,7 @@ __global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const __grid
 template <int IDXB>
 __global__ void __launch_bounds__(kThreads) decode_sums_kernel(const DecodeParams p)
 {
+    grid_dependency_prologue();
     constexpr bool MULTI = IDXB != 0;
     const int64_t i = ((int64_t)blockIdx.x * kThreads + threadIdx.x) * 4;
     if (i >= p.d) return;
@@ -405,30 +407,30 @@ static cudaError_t dispatch_levels(const DecodeParams &p, int idx_bits, cudaStre
     const unsigned nb = (unsigned)blocks;
     if (rows) {
         switch (idx_bits) {
-        case 0: aggregate_decode_kernel<FMT, 0, false, true><<<nb, kThreads, 0, st>>>(p); break;
-        case 1: aggregate_decode_kernel<FMT, 1, false, true><<<nb, kThreads, 0, st>>>(p); break;
-        case 2: aggregate_decode_kernel<FMT, 2, false, true><<<nb, kThreads, 0, st>>>(p); break;
-        case 4: aggregate_decode_kernel<FMT, 4, false, true><<<nb, kThreads, 0, st>>>(p); break;
-        default: aggregate_decode_kernel<FMT, 8, false, true><<<nb, kThreads, 0, st>>>(p); break;
+        case 0: launch_k(aggregate_decode_kernel<FMT, 0, false, true>, nb, kThreads, st, p); break;
+        case 1: launch_k(aggregate_decode_kernel<FMT, 1, false, true>, nb, kThreads, st, p); break;
+        case 2: launch_k(aggregate_decode_kernel<FMT, 2, false, true>, nb, kThreads, st, p); break;
+        case 4: launch_k(aggregate_decode_kernel<FMT, 4, false, true>, nb, kThreads, st, p); break;
+        default: launch_k(aggregate_decode_kernel<FMT, 8, false, true>, nb, kThreads, st, p); break;
         }
         return cudaGetLastError();
     }
     if (p.theta != nullptr) {
         switch (idx_bits) {
-        case 0: aggregate_decode_kernel<FMT, 0, true><<<nb, kThreads, 0, st>>>(p); break;
-        case 1: aggregate_decode_kernel<FMT, 1, true><<<nb, kThreads, 0, st>>>(p); break;
-        case 2: aggregate_decode_kernel<FMT, 2, true><<<nb, kThreads, 0, st>>>(p); break;
-        case 4: aggregate_decode_kernel<FMT, 4, true><<<nb, kThreads, 0, st>>>(p); break;
-        default: aggregate_decode_kernel<FMT, 8, true><<<nb, kThreads, 0, st>>>(p); break;
+        case 0: launch_k(aggregate_decode_kernel<FMT, 0, true>, nb, kThreads, st, p); break;
+        case 1: launch_k(aggregate_decode_kernel<FMT, 1, true>, nb, kThreads, st, p); break;
+        case 2: launch_k(aggregate_decode_kernel<FMT, 2, true>, nb, kThreads, st, p); break;
+        case 4: launch_k(aggregate_decode_kernel<FMT, 4, true>, nb, kThreads, st, p); break;
+        default: launch_k(aggregate_decode_kernel<FMT, 8, true>, nb, kThreads, st, p); break;
         }
         return cudaGetLastError();
     }
     switch (idx_bits) {
-    case 0: aggregate_decode_kernel<FMT, 0, false><<<nb, kThreads, 0, st>>>(p); break;
-    case 1: aggregate_decode_kernel<FMT, 1, false><<<nb, kThreads, 0, st>>>(p); break;
-    case 2: aggregate_decode_kernel<FMT, 2, false><<<nb, kThreads, 0, st>>>(p); break;
-    case 4: aggregate_decode_kernel<FMT, 4, false><<<nb, kThreads, 0, st>>>(p); break;
-    default: aggregate_decode_kernel<FMT, 8, false><<<nb, kThreads, 0, st>>>(p); break;
+    case 0: launch_k(aggregate_decode_kernel<FMT, 0, false>, nb, kThreads, st, p); break;
+    case 1: launch_k(aggregate_decode_kernel<FMT, 1, false>, nb, kThreads, st, p); break;
+    case 2: launch_k(aggregate_decode_kernel<FMT, 2, false>, nb, kThreads, st, p); break;
+    case 4: launch_k(aggregate_decode_kernel<FMT, 4, false>, nb, kThreads, st, p); break;
+    default: launch_k(aggregate_decode_kernel<FMT, 8, false>, nb, kThreads, st, p); break;
     }
     return cudaGetLastError();
 }
@@ -477,11 +479,11 @@ cudaError_t launch_decode_sums(const uq_layout &L, const int32_t *S, const float
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     const unsigned nb = (unsigned)blocks;
     switch (idx_bits) {
-    case 0: decode_sums_kernel<0><<<nb, kThreads, 0, st>>>(p); break;
-    case 1: decode_sums_kernel<1><<<nb, kThreads, 0, st>>>(p); break;
-    case 2: decode_sums_kernel<2><<<nb, kThreads, 0, st>>>(p); break;
-    case 4: decode_sums_kernel<4><<<nb, kThreads, 0, st>>>(p); break;
-    default: decode_sums_kernel<8><<<nb, kThreads, 0, st>>>(p); break;
+    case 0: launch_k(decode_sums_kernel<0>, nb, kThreads, st, p); break;
+    case 1: launch_k(decode_sums_kernel<1>, nb, kThreads, st, p); break;
+    case 2: launch_k(decode_sums_kernel<2>, nb, kThreads, st, p); break;
+    case 4: launch_k(decode_sums_kernel<4>, nb, kThreads, st, p); break;
+    default: launch_k(decode_sums_kernel<8>, nb, kThreads, st, p); break;
     }
     return cudaGetLastError();
 }

@@ -8,6 +8,42 @@
 
 namespace uq {
 
+// ---------------------------------------------------------------------------------------------
+// Programmatic dependent launch: every kernel of the library is launched with the attribute that
+// lets the GPU schedule its CTAs while the kernel before it in the stream is still draining, and
+// starts with grid_dependency_prologue(): it first lets the kernel AFTER it be scheduled the same
+// way, then waits until the kernel before it has completed and its writes are visible.  No read of
+// global memory may come before the prologue.  What overlaps is launch latency and the ramp of the
+// CTAs, not the work; a predecessor that knows nothing of this (a framework kernel, a copy) simply
+// counts as complete when it ends.  -DUQ_NO_PDL launches the plain way.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void grid_dependency_prologue()
+{
+#ifndef UQ_NO_PDL
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+#endif
+}
+
+template <typename... P, typename... A>
+inline void launch_k(void (*kernel)(P...), dim3 grid, dim3 block, cudaStream_t st, A &&...args)
+{
+#ifdef UQ_NO_PDL
+    kernel<<<grid, block, 0, st>>>(static_cast<A &&>(args)...);
+#else
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, static_cast<A &&>(args)...);    // an error stays for cudaGetLastError()
+#endif
+}
+
 constexpr int kThreads = 256;            // threads per CTA in every streaming kernel
 constexpr int kWarps = kThreads / 32;
 constexpr int kNormTile = 8192;          // coordinates per partial of the norm reduction

@@ -278,6 +278,7 @@ __device__ __noinline__ void encode_tile_mixed(const EncodeParams &p, int m, int
 template <int DT, int FMT, int RNG, int IDXB>
 __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, IDXB != 0>::MIN_CTAS)) encode_kernel(const __grid_constant__ EncodeParams p)
 {
+    grid_dependency_prologue();
     using E = Elem<DT>;
     using S = EncodeShape<DT, IDXB != 0>;
     constexpr bool MULTI = IDXB != 0;
@@ -407,7 +408,7 @@ static cudaError_t launch(EncodeParams p, cudaStream_t st)
     p.main_blocks = (uint32_t)blocks;
     if (p.seg_off != nullptr && p.nseg > 1) blocks += (int64_t)((p.nseg - 1 + kWarps - 1) / kWarps) * p.M;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
-    encode_kernel<DT, FMT, RNG, IDXB><<<(unsigned)blocks, kThreads, 0, st>>>(p);
+    launch_k(encode_kernel<DT, FMT, RNG, IDXB>, (unsigned)blocks, kThreads, st, p);
     return cudaGetLastError();
 }
 

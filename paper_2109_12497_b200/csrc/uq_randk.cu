@@ -44,6 +44,7 @@ struct RandkParams {
 template <int DT>
 __global__ void __launch_bounds__(kThreads) randk_gather_kernel(const __grid_constant__ RandkParams p)
 {
+    grid_dependency_prologue();
     using T = typename std::conditional<DT == UQ_F32, uint32_t, uint16_t>::type;
     const int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     if (t >= p.gk_stride) return;
@@ -78,6 +79,7 @@ __global__ void __launch_bounds__(kThreads) randk_scatter_kernel(int64_t d, int6
                                                                  const float *vals, float *dst, float lr,
                                                                  uint32_t *status)
 {
+    grid_dependency_prologue();
     const int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     if (t >= K) return;
     const int64_t i = __ldg(sel + t);
@@ -102,8 +104,8 @@ cudaError_t launch_randk_gather(const uq_layout &L, const void *g, int64_t K, ui
     p.key = philox_key(seed);
     const int64_t blocks = (gk_stride + kThreads - 1) / kThreads;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
-    if (L.dtype == UQ_F32) randk_gather_kernel<UQ_F32><<<(unsigned)blocks, kThreads, 0, st>>>(p);
-    else randk_gather_kernel<UQ_BF16><<<(unsigned)blocks, kThreads, 0, st>>>(p);
+    if (L.dtype == UQ_F32) launch_k(randk_gather_kernel<UQ_F32>, (unsigned)blocks, kThreads, st, p);
+    else launch_k(randk_gather_kernel<UQ_BF16>, (unsigned)blocks, kThreads, st, p);
     return cudaGetLastError();
 }
 
@@ -113,8 +115,8 @@ cudaError_t launch_randk_scatter(int64_t d, int64_t K, const int64_t *sel, const
     if (K == 0) return cudaSuccess;
     const int64_t blocks = (K + kThreads - 1) / kThreads;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
-    if (update) randk_scatter_kernel<true><<<(unsigned)blocks, kThreads, 0, st>>>(d, K, sel, vals, dst, lr, status);
-    else randk_scatter_kernel<false><<<(unsigned)blocks, kThreads, 0, st>>>(d, K, sel, vals, dst, lr, status);
+    if (update) launch_k(randk_scatter_kernel<true>, (unsigned)blocks, kThreads, st, d, K, sel, vals, dst, lr, status);
+    else launch_k(randk_scatter_kernel<false>, (unsigned)blocks, kThreads, st, d, K, sel, vals, dst, lr, status);
     return cudaGetLastError();
 }
 

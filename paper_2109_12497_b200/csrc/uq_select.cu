@@ -69,6 +69,7 @@ __device__ __noinline__ uint64_t select_general(const SelectParams &p, int64_t i
 template <int DT, int IDXB, int LEVELS>
 __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant__ SelectParams p)
 {
+    grid_dependency_prologue();
     using E = Elem<DT>;
     constexpr int H = 8 / E::G;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -181,10 +182,10 @@ template <int DT, int IDXB>
 static cudaError_t dispatch_levels(const SelectParams &p, unsigned blocks, cudaStream_t st)
 {
     const int N = p.scales.N;
-    if (N <= 2) select_kernel<DT, IDXB, 1><<<blocks, kThreads, 0, st>>>(p);
-    else if (N <= 4) select_kernel<DT, IDXB, 2><<<blocks, kThreads, 0, st>>>(p);
-    else if (N <= 8) select_kernel<DT, IDXB, 3><<<blocks, kThreads, 0, st>>>(p);
-    else select_kernel<DT, IDXB, 4><<<blocks, kThreads, 0, st>>>(p);
+    if (N <= 2) launch_k(select_kernel<DT, IDXB, 1>, blocks, kThreads, st, p);
+    else if (N <= 4) launch_k(select_kernel<DT, IDXB, 2>, blocks, kThreads, st, p);
+    else if (N <= 8) launch_k(select_kernel<DT, IDXB, 3>, blocks, kThreads, st, p);
+    else launch_k(select_kernel<DT, IDXB, 4>, blocks, kThreads, st, p);
     return cudaGetLastError();
 }
 
@@ -194,7 +195,7 @@ static cudaError_t dispatch(const SelectParams &p, int idx_bits, cudaStream_t st
     const int64_t blocks = (p.d + kSelectTile - 1) / kSelectTile;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
-    if (idx_bits == 1) { select_kernel<DT, 1, 1><<<(unsigned)blocks, kThreads, 0, st>>>(p); return cudaGetLastError(); }
+    if (idx_bits == 1) { launch_k(select_kernel<DT, 1, 1>, (unsigned)blocks, kThreads, st, p); return cudaGetLastError(); }
     if (idx_bits == 2) return dispatch_levels<DT, 2>(p, (unsigned)blocks, st);
     if (idx_bits == 4) return dispatch_levels<DT, 4>(p, (unsigned)blocks, st);
     return dispatch_levels<DT, 8>(p, (unsigned)blocks, st);
@@ -233,6 +234,7 @@ template <int IDXB>
 __global__ void __launch_bounds__(kThreads) index_min_kernel(const uint8_t *__restrict__ rows, int R, int64_t row_bytes,
                                                              int64_t nwords, uint8_t *__restrict__ idx)
 {
+    grid_dependency_prologue();
     const int64_t w = (int64_t)blockIdx.x * kThreads + threadIdx.x;      // my 4-byte word
     if (w >= nwords) return;
     uint32_t acc = __ldg((const uint32_t *)rows + w);
@@ -249,10 +251,10 @@ cudaError_t launch_index_min(const uint8_t *rows, int R, int64_t row_bytes, int6
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     const unsigned nb = (unsigned)blocks;
-    if (idx_bits == 1) index_min_kernel<1><<<nb, kThreads, 0, st>>>(rows, R, row_bytes, nwords, idx);
-    else if (idx_bits == 2) index_min_kernel<2><<<nb, kThreads, 0, st>>>(rows, R, row_bytes, nwords, idx);
-    else if (idx_bits == 4) index_min_kernel<4><<<nb, kThreads, 0, st>>>(rows, R, row_bytes, nwords, idx);
-    else index_min_kernel<8><<<nb, kThreads, 0, st>>>(rows, R, row_bytes, nwords, idx);
+    if (idx_bits == 1) launch_k(index_min_kernel<1>, nb, kThreads, st, rows, R, row_bytes, nwords, idx);
+    else if (idx_bits == 2) launch_k(index_min_kernel<2>, nb, kThreads, st, rows, R, row_bytes, nwords, idx);
+    else if (idx_bits == 4) launch_k(index_min_kernel<4>, nb, kThreads, st, rows, R, row_bytes, nwords, idx);
+    else launch_k(index_min_kernel<8>, nb, kThreads, st, rows, R, row_bytes, nwords, idx);
     return cudaGetLastError();
 }
 
