@@ -179,23 +179,36 @@ def time_device_resident(q, g, w, steps, warmup, barrier):
 
 
 def time_end_to_end(q, g_host, out_host, g_dev, w, steps, warmup, barrier):
-    """ms per step with the gradients starting in pinned host memory and the result read back."""
+    """ms per step with the gradients starting in pinned host memory and the result read back.
+    Every step copies its own inputs in and its own result out; the read-back of step k runs on
+    a second stream while the inputs of step k+1 arrive (the two directions of the link are
+    independent), ordered by events: kernels(k) after copy-in(k); copy-in(k+1) and read-back(k)
+    after kernels(k); kernels(k+1) after read-back(k)."""
     import torch
-    st = torch.cuda.current_stream()
+    main = torch.cuda.current_stream()
+    back = torch.cuda.Stream()
+    done = [torch.cuda.Event() for _ in range(2)]             # kernels of a step finished / result read back
 
     def one(k):
-        g_dev.copy_(g_host, non_blocking=True)
+        g_dev.copy_(g_host, non_blocking=True)                # main: inputs of this step
+        main.wait_event(done[1])                              # the previous result has left the output buffer
         out = q.step(g_dev, w.seed + k)
-        out_host.copy_(out, non_blocking=True)
+        done[0].record(main)
+        back.wait_event(done[0])
+        with torch.cuda.stream(back):
+            out_host.copy_(out, non_blocking=True)
+            done[1].record(back)
 
+    done[1].record(main)
     for k in range(min(warmup, 3)):
         one(k)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize(); barrier()
-    e0.record(st)
+    e0.record(main)
     for k in range(steps):
         one(k)
-    e1.record(st)
+    main.wait_event(done[1])                                  # the last read-back is inside the timed region
+    e1.record(main)
     torch.cuda.synchronize(); barrier()
     return e0.elapsed_time(e1) / steps
 
