@@ -3,8 +3,9 @@
 // g_hat_i = W_j * S_i / (s_i * M)  (Eq. R_s after Algorithm 1, Eq. R_{s_} after Algorithm 2).
 //
 // The fused kernel reads the M level streams once, keeps the sums in registers and writes only
-// the fp32 average (and, on request, the int32 sums).  A thread owns 16 B of every worker's
-// stream: 16 coordinates of int8 levels or 32 coordinates of packed 4-bit levels.
+// the fp32 average (and, on request, the int32 sums).  A thread owns 16 coordinates of int8 levels
+// (16 B of every worker's stream) or 32 coordinates of the packed formats (16 B of 4-bit, 8 B of
+// 2-bit, 16 + 8 B of the two planes of 6-bit levels).
 #include "uq_device.cuh"
 
 namespace uq {

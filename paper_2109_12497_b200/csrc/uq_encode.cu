@@ -4,7 +4,8 @@
 // Algorithm 2 line "Quantize with s*").
 //
 // One streaming pass: a thread owns units of 8 consecutive coordinates (32 B of fp32 or 16 B of
-// bf16 in, 8 B of int8, 4 B of packed 4-bit or 2 B of packed 2-bit levels out); a CTA owns one tile of one worker.
+// bf16 in; 8 B of int8, 6 B of two-plane 6-bit, 4 B of packed 4-bit or 2 B of packed 2-bit levels
+// out); a CTA owns one tile of one worker.
 // A worker's CTA reads only that worker's gradient plus the agreed values W and idx.
 #include "uq_device.cuh"
 
