@@ -305,3 +305,37 @@ def test_block_counter_wraps_inside_a_tile(rng_bits):
     assert np.array_equal(lev.cpu().numpy()[:, :d], want)
     # the draws really moved: the same data at coord0 = 0 gives other levels
     assert not np.array_equal(o.encode_single(g_np[:, :d], W.cpu().numpy(), 127, 5, rng_bits), want)
+
+
+def test_step_right_after_an_asynchronous_copy():
+    """Inputs arriving by an asynchronous copy from pinned host memory on the same stream, the
+    step enqueued right behind it and the result read back asynchronously: the kernels (which may
+    be scheduled while their predecessor drains) still see the complete copy, step after step."""
+    w = wl.scaled("c3", 1_000_003, M=4)
+    g_np = wl.generate(w)
+    ref = run_oracle(w, g_np)
+    from paper_2109_12497_b200.pipeline import from_workload
+    q = from_workload(w, keep_sums=True)
+    host = torch.from_numpy(g_np).pin_memory()
+    g = torch.zeros_like(host, device="cuda")
+    out_host = torch.empty(w.d, dtype=torch.float32).pin_memory()
+    junk = torch.from_numpy(np.full_like(g_np, 3.0)).pin_memory()
+    for k in range(3):
+        g.copy_(junk, non_blocking=True)                       # what a stale read would see
+        g.copy_(host, non_blocking=True)
+        out = q.step(g, w.seed)
+        out_host.copy_(out, non_blocking=True)
+        torch.cuda.synchronize()
+        assert np.array_equal(q.S.cpu().numpy()[: w.d], ref["S"]), k
+        assert np.allclose(out_host.numpy(), ref["out"], rtol=1e-6, atol=0), k
+    # the same behind kernels that know nothing of the library's launch attribute
+    src = host.cuda()
+    for k in range(3):
+        g.fill_(3.0)
+        g.copy_(src)
+        g.mul_(1.0)
+        out = q.step(g, w.seed)
+        got = out.clone()                                      # a framework kernel right behind the step
+        torch.cuda.synchronize()
+        assert np.array_equal(q.S.cpu().numpy()[: w.d], ref["S"]), k
+        assert np.allclose(got.cpu().numpy(), ref["out"], rtol=1e-6, atol=0), k
