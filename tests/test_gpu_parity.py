@@ -339,3 +339,32 @@ def test_step_right_after_an_asynchronous_copy():
         torch.cuda.synchronize()
         assert np.array_equal(q.S.cpu().numpy()[: w.d], ref["S"]), k
         assert np.allclose(got.cpu().numpy(), ref["out"], rtol=1e-6, atol=0), k
+
+
+def _random_workload(rng):
+    name = ["c1", "c2", "c3", "c4", "c5"][rng.integers(5)]
+    d = int([rng.integers(1, 300), rng.integers(300, 40_000), rng.integers(40_000, 400_000)][rng.integers(3)])
+    M = int([1, 2, 3, 5, 8, 13, 16, 17, 31, 64][rng.integers(10)])
+    if d * M > 6_000_000:
+        M = max(1, 6_000_000 // d)
+    fmt, smax = [("i8", 127), ("i6p", 31), ("i4x2", 7), ("i2x4", 1)][rng.integers(4)]
+    s = int(rng.integers(1, smax + 1))
+    kw = dict(fmt=fmt, s=s, scales=(s,), dtype=[wl.F32, wl.BF16][rng.integers(2)], rng_bits=[16, 32][rng.integers(2)],
+              norm=[wl.NORM_L2, wl.NORM_LINF][rng.integers(2)], seed=int(rng.integers(0, 2**62)))
+    if wl.WORKLOADS[name].quantizer == "multi":
+        idx_bits = int([1, 2, 4, 8][rng.integers(4)])
+        N = int(rng.integers(1, min(16, 1 << idx_bits) + 1))
+        ratio = int([2, 3, 8, 16][rng.integers(4)])
+        scales = [s]
+        while len(scales) < N and scales[-1] * ratio < 2**31:
+            scales.append(scales[-1] * ratio)
+        kw.update(idx_bits=idx_bits, scales=tuple(scales))
+    return wl.scaled(name, d, M=M, **kw)
+
+
+@pytest.mark.parametrize("case", range(48))
+def test_randomized_configurations(case):
+    """Seeded random draws over every argument of the path (workload recipe, d, M, element type,
+    wire format, level count, scale set, index width, norm, draw width, seed)."""
+    w = _random_workload(np.random.default_rng(9000 + case))
+    check_parity(w, wl.generate(w))
