@@ -235,9 +235,11 @@ def time_encode_other_mode(q, g, w, reps):
         q.rng_bits = keep
 
 
-def time_graph_replay(q, g, w, reps):
+def time_graph_replay(q, g, w, reps, stats=False):
     """ms per step when the step's launches are captured once in a CUDA graph and replayed: the
-    figure for a working set so small that launch latency, not memory, sets the time."""
+    figure for a working set so small that launch latency, not memory, sets the time.  stats:
+    time every replay by itself and return (mean, median, min) instead of the mean of a burst.
+    (A replay repeats the captured seed: a latency figure, not a training loop.)"""
     import torch
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
@@ -248,10 +250,19 @@ def time_graph_replay(q, g, w, reps):
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
         q.step(g, w.seed)
-    for _ in range(3):
+    for _ in range(5):
         graph.replay()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
+    if stats:
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for a, b in evs:
+            a.record()
+            graph.replay()
+            b.record()
+        torch.cuda.synchronize()
+        t = sorted(a.elapsed_time(b) for a, b in evs)
+        return statistics.fmean(t), statistics.median(t), t[0]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(reps):
         graph.replay()
@@ -392,6 +403,7 @@ def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=F
     res["update_ms"] = time_fused_update(q, w, min(steps, 10))
     if randk_K:
         res["randk"] = time_randk(w, g_dev, min(randk_K, w.d), 50)
+        res["graph_stats"] = time_graph_replay(q, g_dev, w, max(steps, 20), stats=True)
     res["h2d"], res["d2h"], res["e2e_ms"] = 0, 0, None
     if want_e2e:
         out_host = torch.empty(w.d, dtype=torch.float32, pin_memory=True)
@@ -543,6 +555,12 @@ def gpu_main(args):
     }
     if "randk" in res:
         line["global_randk"] = res["randk"]
+    if "graph_stats" in res:
+        mean, med, lo = res["graph_stats"]
+        line["cuda_graph_replay"] = {"ms_per_step_mean": round(mean, 5), "ms_per_step_median": round(med, 5),
+                                     "ms_per_step_min": round(lo, 5), "replays": max(args.steps, 20),
+                                     "gradient_GBps_median": round(w.in_bytes / med / 1e6, 1),
+                                     "note": "the whole step captured once and replayed, each replay timed by itself"}
     if rank == 0 and world == 1:
         # the other four workloads (parity-test cases; reported for context, a few steps each)
         if not args.no_extra and args.d is None:
