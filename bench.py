@@ -65,6 +65,7 @@ def algorithmic_bytes(w: wl.Workload) -> dict:
     if w.quantizer == "multi":
         b["select_scale"] = e * M * d + ib * d
         b["encode"] = (e + lev + ib) * M * d          # every worker re-reads the shared index
+        b["select_encode"] = (e + lev) * M * d + ib * d   # fused: gradients read once, index written once
     else:
         b["encode"] = (e + lev) * M * d
     b["aggregate_decode"] = lev * M * d + ib * d + 4 * d
@@ -140,11 +141,15 @@ def run_stages(q, g, seed, events=None):
     if events: events[k].record(st)
     q.agree_scale(g); k += 1
     if events: events[k].record(st)
-    if q.multi:
-        q.select_scale(g); k += 1
+    if q.multi and q.fused_select:
+        q.select_encode(g, seed); k += 1
         if events: events[k].record(st)
-    q.encode(g, seed); k += 1
-    if events: events[k].record(st)
+    else:
+        if q.multi:
+            q.select_scale(g); k += 1
+            if events: events[k].record(st)
+        q.encode(g, seed); k += 1
+        if events: events[k].record(st)
     q.aggregate_decode(); k += 1
     if events: events[k].record(st)
 
@@ -233,6 +238,23 @@ def time_encode_other_mode(q, g, w, reps):
         return evs[0].elapsed_time(evs[reps]) / reps
     finally:
         q.rng_bits = keep
+
+
+def time_fused_select_encode(q, g, w, reps):
+    """Multi-scale: mean ms of the one-kernel form of selection + encoding (the step itself runs
+    the two kernels, which measure no slower), timed alone."""
+    import torch
+    st = torch.cuda.current_stream()
+    for k in range(2):
+        q.select_encode(g, w.seed + k)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(st)
+    for k in range(reps):
+        q.select_encode(g, w.seed + k)
+    e1.record(st)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
 
 
 def time_graph_replay(q, g, w, reps, stats=False):
@@ -401,6 +423,8 @@ def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=F
     res["ms"], res["stages_ms"] = time_device_resident(q, g_dev, w, steps, warmup, barrier)
     res["encode_other_ms"] = time_encode_other_mode(q, g_dev, w, min(steps, 10))
     res["update_ms"] = time_fused_update(q, w, min(steps, 10))
+    if q.multi:
+        res["fused_select_ms"] = time_fused_select_encode(q, g_dev, w, min(steps, 10))
     if randk_K:
         res["randk"] = time_randk(w, g_dev, min(randk_K, w.d), 50)
         res["graph_stats"] = time_graph_replay(q, g_dev, w, max(steps, 20), stats=True)
@@ -427,6 +451,13 @@ def summarize(res, peak_gbs):
     out["kernels"][f"encode_rng{other}"] = {
         "ms": round(ms, 5), "algorithmic_MB": round(ab["encode"] / 1e6, 2), "GBps": round(ab["encode"] / ms / 1e6, 1),
         "frac_of_hbm_peak": round(ab["encode"] / ms / 1e6 / peak_gbs, 4), "note": "timed alone, not part of the step"}
+    if "fused_select_ms" in res:
+        ms = res["fused_select_ms"]
+        out["kernels"]["select_encode"] = {
+            "ms": round(ms, 5), "algorithmic_MB": round(ab["select_encode"] / 1e6, 2),
+            "GBps": round(ab["select_encode"] / ms / 1e6, 1),
+            "frac_of_hbm_peak": round(ab["select_encode"] / ms / 1e6 / peak_gbs, 4),
+            "note": "selection + encoding as one kernel, timed alone, not part of the step"}
     lev = {"i8": 1.0, "i4x2": 0.5, "i2x4": 0.25, "i6p": 0.75}[w.fmt]
     upd_bytes = lev * w.M * w.d + w.idx_bits / 8.0 * w.d + 16 * w.d      # levels, index, theta and momentum r/w
     ms = res["update_ms"]

@@ -213,6 +213,18 @@ int uq_encode_multi(const uq_layout *layout, const void *g, const float *W, cons
                     void *lev, uint32_t *status, void *stream);
 
 /*
+ * uq_select_scale_multi followed by uq_encode_multi in one kernel — Algorithm 2 lines "Compute
+ * coordinate scales", "Scale sharing" and "Quantize with s*".  For callers whose M workers are all
+ * in this buffer: a thread reads the 8 coordinates of every worker once to form max_m |g^m_i|,
+ * finds the shared indices, and quantizes every worker's coordinates with them, so the gradients
+ * cross the memory interface once instead of twice.  idx and lev receive, bit for bit, what the two
+ * separate calls write; arguments and errors are theirs.
+ */
+int uq_select_encode_multi(const uq_layout *layout, const void *g, const float *W, const int32_t *scales,
+                           int N, int idx_bits, uint64_t seed, int rng_bits, int fmt, uint8_t *idx,
+                           void *lev, uint32_t *status, void *stream);
+
+/*
  * Integer aggregation — Algorithm 1 / 2 line "AllReduce gradients" without the 1/M:
  *   S[i] = sum over workers of zeta^m_i, in int32.
  *   lev  in   level rows as written by the encoders (layout->dtype is ignored)

@@ -26,7 +26,7 @@ UQ_STATUS_NONFINITE, UQ_STATUS_BAD_SEGMENTS, UQ_STATUS_SCALE_OVERFLOW, UQ_STATUS
 EXPORTS = (
     "uq_version", "uq_last_cuda_error", "uq_error_string", "uq_workspace_bytes", "uq_index_bytes",
     "uq_agree_scale", "uq_agree_scale_static", "uq_encode_single", "uq_select_scale_multi", "uq_encode_multi",
-    "uq_aggregate", "uq_decode", "uq_decode_update", "uq_randk_gather", "uq_randk_scatter", "uq_randk_update", "uq_index_min", "uq_decode_rows",
+    "uq_aggregate", "uq_decode", "uq_decode_update", "uq_randk_gather", "uq_randk_scatter", "uq_randk_update", "uq_index_min", "uq_decode_rows", "uq_select_encode_multi",
 )
 
 
@@ -84,6 +84,7 @@ def lib() -> C.CDLL:
         F = C.c_float
         L.uq_decode_update.argtypes = [LP, P, I, P, I, P, I, P, I, P, P, F, F, F, P, P]
         I64 = C.c_int64
+        L.uq_select_encode_multi.argtypes = [LP, P, P, P, I, I, U64, I, I, P, P, P, P]
         L.uq_decode_rows.argtypes = [LP, P, I, P, I, P, I, P, I, P, P, P]
         L.uq_index_min.argtypes = [P, I, I64, I64, I, P, P]
         L.uq_randk_gather.argtypes = [LP, P, I64, U64, P, P, I64, P, P]
@@ -337,3 +338,17 @@ def uq_decode_rows(layout: Layout, lev_rows: Sequence[int], fmt: int, W: torch.T
     _check("uq_decode_rows", lib().uq_decode_rows(
         layout.ref(), rows, fmt, _ptr(W), s, arr, N, _ptr(idx) if scales is not None else None, idx_bits,
         _ptr(out), _ptr(S_opt), _stream()))
+
+
+def uq_select_encode_multi(layout: Layout, g: torch.Tensor, W: torch.Tensor, scales: Sequence[int], idx_bits: int,
+                           seed: int, rng_bits: int, fmt: int, idx: torch.Tensor, lev: torch.Tensor,
+                           status: Optional[torch.Tensor]) -> None:
+    """uq_select_scale_multi + uq_encode_multi in one kernel (all workers in this buffer)."""
+    layout.check_g(g)
+    layout.check_lev(lev, fmt)
+    layout.check_vec(W, torch.float32, layout.nseg, "W")
+    layout.check_vec(idx, torch.uint8, layout.index_bytes(idx_bits), "idx")
+    arr, N = _scales(scales)
+    _check("uq_select_encode_multi", lib().uq_select_encode_multi(
+        layout.ref(), _ptr(g), _ptr(W), arr, N, idx_bits, seed, rng_bits, fmt, _ptr(idx), _ptr(lev), _ptr(status),
+        _stream()))

@@ -20,6 +20,9 @@ cudaError_t launch_aggregate_decode_rows(const uq_layout &L, const void *const *
                                          int32_t *S, cudaStream_t st);
 cudaError_t launch_decode_sums(const uq_layout &L, const int32_t *S, const float *W, const ScaleSet &scales,
                                const uint8_t *idx, int idx_bits, float *out, cudaStream_t st);
+cudaError_t launch_select_encode(const uq_layout &L, const void *g, const float *W, const ScaleSet &scales, int idx_bits,
+                                 uint64_t seed, int rng_bits, int fmt, uint8_t *idx, void *lev, uint32_t *status,
+                                 cudaStream_t st);
 cudaError_t launch_index_min(const uint8_t *rows, int R, int64_t row_bytes, int64_t nbytes, int idx_bits, uint8_t *idx,
                              cudaStream_t st);
 cudaError_t launch_randk_gather(const uq_layout &L, const void *g, int64_t K, uint64_t seed, int64_t *sel,
@@ -169,6 +172,21 @@ int uq_encode_multi(const uq_layout *L, const void *g, const float *W, const int
         return UQ_ERR_BAD_ARG;
     return finish(uq::launch_encode(*L, g, W, set, idx, idx_bits, seed, rng_bits, fmt, lev, status,
                                     (cudaStream_t)stream));
+}
+
+int uq_select_encode_multi(const uq_layout *L, const void *g, const float *W, const int32_t *scales, int N,
+                           int idx_bits, uint64_t seed, int rng_bits, int fmt, uint8_t *idx, void *lev,
+                           uint32_t *status, void *stream)
+{
+    uq::ScaleSet set;
+    if (!layout_ok(L) || W == nullptr || !aligned(status, 4)) return UQ_ERR_BAD_ARG;
+    if (!scales_ok(scales, N, idx_bits, &set)) return UQ_ERR_BAD_ARG;
+    if (!fmt_ok(fmt, set.s[0]) || (rng_bits != 32 && rng_bits != 16)) return UQ_ERR_BAD_ARG;
+    if (L->d > 0 && (g == nullptr || lev == nullptr || idx == nullptr || !aligned(g, 16) || !aligned(lev, 16) ||
+                     !aligned(idx, 16)))
+        return UQ_ERR_BAD_ARG;
+    return finish(uq::launch_select_encode(*L, g, W, set, idx_bits, seed, rng_bits, fmt, idx, lev, status,
+                                           (cudaStream_t)stream));
 }
 
 int uq_aggregate(const uq_layout *L, const void *lev, int fmt, int32_t *S, void *stream)

@@ -234,6 +234,30 @@ __device__ __forceinline__ void philox4x32_10_xN(const PhiloxKey &k, const uint3
     for (int n = 0; n < N; ++n) out[n] = make_uint4(c0[n], c1[n], c2[n], c3[n]);
 }
 
+// The same block number for N workers at once (worker[n] in counter word 2).
+template <int N>
+__device__ __forceinline__ void philox4x32_10_workers(const PhiloxKey &k, uint32_t block_lo, uint32_t block_hi,
+                                                      const uint32_t (&worker)[N], uint4 (&out)[N])
+{
+    uint32_t c0[N], c1[N], c2[N], c3[N];
+#pragma unroll
+    for (int n = 0; n < N; ++n) { c0[n] = block_lo; c1[n] = block_hi; c2[n] = worker[n]; c3[n] = 0u; }
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t k0 = k.k0[r], k1 = k.k1[r];
+#pragma unroll
+        for (int n = 0; n < N; ++n) {
+            const uint64_t p0 = (uint64_t)0xD2511F53u * c0[n];
+            const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2[n];
+            const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1[n] ^ k0;
+            const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3[n] ^ k1;
+            c1[n] = (uint32_t)p1; c3[n] = (uint32_t)p0; c0[n] = n0; c2[n] = n2;
+        }
+    }
+#pragma unroll
+    for (int n = 0; n < N; ++n) out[n] = make_uint4(c0[n], c1[n], c2[n], c3[n]);
+}
+
 // ---------------------------------------------------------------------------------------------
 // one coordinate of Q_s
 // ---------------------------------------------------------------------------------------------
@@ -359,6 +383,24 @@ __device__ __forceinline__ int warp_find_segment(const int64_t *__restrict__ seg
         lo = min(nlo, hi);
     }
     return lo;
+}
+
+// ---------------------------------------------------------------------------------------------
+// scale selection: the test |v| * inv <= s_hat as an integer compare
+// ---------------------------------------------------------------------------------------------
+
+// Largest non-negative binary32 bit pattern t with fl(t * inv) <= s_hat, or -1 if not even 0
+// passes.  fl(t * inv) is non-decreasing in t, so "passes" is a prefix of the magnitudes and the
+// test |v| * inv <= s_hat is the integer compare bits(|v|) <= t.  The quotient s_hat / inv lands
+// within a few units of the answer; the two bounded loops settle it exactly.
+__device__ __forceinline__ int32_t pass_threshold(float inv, float s_hat)
+{
+    if (!(inv > 0.0f)) return inv == 0.0f ? 0x7F7FFFFF : -1;       // W = 0: every finite value passes
+    if (!(__fmul_rn(0.0f, inv) <= s_hat)) return -1;                // inv = Inf: 0 * Inf is NaN
+    int32_t b = __float_as_int(fminf(__fdiv_rn(s_hat, inv), 3.402823466e38f));
+    for (int it = 0; it < 64 && b < 0x7F7FFFFF && __fmul_rn(__int_as_float(b + 1), inv) <= s_hat; ++it) ++b;
+    for (int it = 0; it < 64 && b >= 0 && !(__fmul_rn(__int_as_float(b), inv) <= s_hat); ++it) --b;
+    return b;
 }
 
 }  // namespace uq

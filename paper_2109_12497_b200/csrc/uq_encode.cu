@@ -8,6 +8,7 @@
 // out); a CTA owns one tile of one worker.
 // A worker's CTA reads only that worker's gradient plus the agreed values W and idx.
 #include "uq_device.cuh"
+#include "uq_unit.cuh"
 
 namespace uq {
 
@@ -50,103 +51,6 @@ template <int DT, bool MULTI> struct EncodeShape {
     static constexpr int PHILOX_GROUP = (DT == UQ_BF16 && MULTI) ? 2 : 1;
 #endif
 };
-
-// (float)s_k / W with one IEEE division; 0 for an all-zero segment.
-__device__ __forceinline__ float inv_scale(int32_t s, float W)
-{
-    return W > 0.0f ? __fdiv_rn((float)s, W) : 0.0f;
-}
-
-__device__ __forceinline__ bool not_finite(float x) { return (__float_as_uint(x) & 0x7F800000u) == 0x7F800000u; }
-
-// The idx_bits * 8 bits that belong to 8 consecutive coordinates starting at a multiple of 8.
-template <int IDXB> struct IdxBits;
-template <> struct IdxBits<1> { using T = uint32_t; static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg(p); } };
-template <> struct IdxBits<2> { using T = uint32_t; static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg((const uint16_t *)p); } };
-template <> struct IdxBits<4> { using T = uint32_t; static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg((const uint32_t *)p); } };
-template <> struct IdxBits<8> { using T = uint64_t; static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg((const unsigned long long *)p); } };
-
-// Eight coordinates: magnitudes scaled by inv[e], random words from the block(s) starting at
-// (blk_lo, blk_hi), levels gathered four to a word, signs applied bytewise (`neg` holds 0xFF in
-// the bytes of negative coordinates), packed into the wire format and stored at `dst`.
-// coordinate c uses word c%4 of block c/4 (32-bit draws) or half (c%8)%2 of word (c%8)/2 of block
-// c/8 (16-bit draws).
-// The random words of a unit: RNG == 32 takes blocks blk_lo and blk_lo + 1 (blk_lo is even: no
-// carry), RNG == 16 the single block blk_lo.
-template <int RNG> struct UnitWords { uint4 r[RNG == 32 ? 2 : 1]; };
-
-template <int RNG>
-__device__ __forceinline__ UnitWords<RNG> unit_words(const PhiloxKey &key, uint32_t blk_lo, uint32_t blk_hi, uint32_t m)
-{
-    UnitWords<RNG> w;
-    if (RNG == 32) {
-        const uint32_t b[2] = { blk_lo, blk_lo + 1u };
-        uint4 r[2];
-        philox4x32_10_xN<2>(key, b, blk_hi, m, r);
-        w.r[0] = r[0]; w.r[RNG == 32 ? 1 : 0] = r[1];
-    } else {
-        w.r[0] = philox4x32_10(key, blk_lo, blk_hi, m);
-    }
-    return w;
-}
-
-template <int FMT, int RNG>
-__device__ __forceinline__ void quantize_unit_words(const float (&v)[8], const float (&inv)[8], float cap,
-                                                    uint32_t neg_lo, uint32_t neg_hi, const UnitWords<RNG> &rw,
-                                                    void *dst, void *dst2, bool store = true)
-{
-    constexpr uint32_t LB = RNG == 32 ? kLevelByte23 : kLevelByte16;
-    uint32_t z[8];
-    if (RNG == 32) {
-        const uint4 r0 = rw.r[0], r1 = rw.r[RNG == 32 ? 1 : 0];
-        const uint32_t w[8] = { r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w };
-#pragma unroll
-        for (int e = 0; e < 8; ++e) z[e] = level_draw23(scaled_magnitude(v[e], inv[e], cap), w[e]);
-    } else {
-        const uint4 r = rw.r[0];
-        const uint32_t w[4] = { r.x, r.y, r.z, r.w };
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const uint32_t h = (e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu);
-            z[e] = level_draw16(scaled_magnitude(v[e], inv[e], cap), h);
-        }
-    }
-    const uint32_t lo = negate_bytes(gather_bytes<LB>(z[0], z[1], z[2], z[3]), neg_lo);
-    const uint32_t hi = negate_bytes(gather_bytes<LB>(z[4], z[5], z[6], z[7]), neg_hi);
-    if (!store) return;
-    // plain stores (not evict-first ones): the aggregation kernel that follows reads the levels
-    // back, and what is still in L2 then costs no DRAM read (measured: 7-9 % off that kernel)
-    if (FMT == UQ_FMT_I8) *(uint2 *)dst = make_uint2(lo, hi);
-    else if (FMT == UQ_FMT_I4X2) *(uint32_t *)dst = bytes_to_nibbles(lo, hi);
-    else if (FMT == UQ_FMT_I2X4) *(unsigned short *)dst = (unsigned short)bytes_to_crumbs(lo, hi);
-    else {                                          // 6-bit: bits 0..3 as nibbles, bits 4..5 as 2-bit fields
-        *(uint32_t *)dst = bytes_to_nibbles(lo, hi);
-        *(unsigned short *)dst2 = (unsigned short)bytes_to_crumbs(lo >> 4, hi >> 4);
-    }
-}
-
-template <int FMT, int RNG>
-__device__ __forceinline__ void quantize_unit(const float (&v)[8], const float (&inv)[8], float cap,
-                                              uint32_t neg_lo, uint32_t neg_hi, const PhiloxKey &key,
-                                              uint32_t blk_lo, uint32_t blk_hi, uint32_t m, void *dst,
-                                              void *dst2, bool store = true)
-{
-    quantize_unit_words<FMT, RNG>(v, inv, cap, neg_lo, neg_hi, unit_words<RNG>(key, blk_lo, blk_hi, m), dst, dst2, store);
-}
-
-// The sign masks of a unit, from the raw loaded words (before any padding is zeroed).
-template <int DT> __device__ __forceinline__ void unit_signs(const uint4 *q, uint32_t &neg_lo, uint32_t &neg_hi)
-{
-    if (DT == UQ_F32) {
-        neg_lo = sign_bytes_f32(__uint_as_float(q[0].x), __uint_as_float(q[0].y), __uint_as_float(q[0].z),
-                                __uint_as_float(q[0].w));
-        neg_hi = sign_bytes_f32(__uint_as_float(q[1].x), __uint_as_float(q[1].y), __uint_as_float(q[1].z),
-                                __uint_as_float(q[1].w));
-    } else {
-        neg_lo = sign_bytes_bf16(q[0].x, q[0].y);
-        neg_hi = sign_bytes_bf16(q[0].z, q[0].w);
-    }
-}
 
 // Coordinates [a, b) of worker m with per-coordinate scale lookup and bounds: the ragged last
 // tile and the 256-coordinate rows that a segment boundary crosses.  Thread `who` of `many`

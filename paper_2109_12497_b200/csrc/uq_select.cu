@@ -32,20 +32,6 @@ __device__ __forceinline__ float inv_scale_sel(int32_t s, float W)
     return W > 0.0f ? __fdiv_rn((float)s, W) : 0.0f;
 }
 
-// Largest non-negative binary32 bit pattern t with fl(t * inv) <= s_hat, or -1 if not even 0
-// passes.  fl(t * inv) is non-decreasing in t, so "passes" is a prefix of the magnitudes and the
-// test |v| * inv <= s_hat is the integer compare bits(|v|) <= t.  The quotient s_hat / inv lands
-// within a few units of the answer; the two bounded loops settle it exactly.
-__device__ __forceinline__ int32_t pass_threshold(float inv, float s_hat)
-{
-    if (!(inv > 0.0f)) return inv == 0.0f ? 0x7F7FFFFF : -1;       // W = 0: every finite value passes
-    if (!(__fmul_rn(0.0f, inv) <= s_hat)) return -1;                // inv = Inf: 0 * Inf is NaN
-    int32_t b = __float_as_int(fminf(__fdiv_rn(s_hat, inv), 3.402823466e38f));
-    for (int it = 0; it < 64 && b < 0x7F7FFFFF && __fmul_rn(__int_as_float(b + 1), inv) <= s_hat; ++it) ++b;
-    for (int it = 0; it < 64 && b >= 0 && !(__fmul_rn(__int_as_float(b), inv) <= s_hat); ++it) --b;
-    return b;
-}
-
 // The general path for one thread's 8 coordinates (row crossed by a segment boundary): the test
 // is evaluated as written, with one division per scale and coordinate.  Rare, kept out of line.
 __device__ __noinline__ uint64_t select_general(const SelectParams &p, int64_t i, const uint32_t (&amag)[8], int idxb,
