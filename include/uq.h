@@ -158,6 +158,22 @@ int uq_agree_scale_static(const uq_layout *layout, const void *g, int norm, floa
                           void *stream);
 
 /*
+ * uq_agree_scale with a by-product for the multi-scale quantizer: amax[i] = max over the workers of
+ * |g^m_i|, written while the gradients are read for the norms (Algorithm 2, line "MaxAllReduce
+ * Norm").  The shared scale index of a coordinate depends on the gradients only through amax[i]
+ * (binary32 multiplication by a positive constant is monotone, so the smallest own index over the
+ * workers is the index of the largest magnitude), hence
+ *     uq_select_scale_multi(layout with M = 1, g = amax, ...)
+ * writes the indices that the call on all M rows writes, reading 1/M of the bytes.
+ *   amax  out  [worker_stride] elements of layout->dtype, device, 16-byte aligned: the magnitude
+ *              (sign bit clear) of the largest entry of coordinate i; elements d.. are padding
+ * W may differ from uq_agree_scale's in the last bit (another fixed order of additions); every
+ * other argument and error is uq_agree_scale's.
+ */
+int uq_agree_scale_amax(const uq_layout *layout, const void *g, int norm, float *W, void *amax,
+                        uint32_t *status, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Single-scale quantizer Q_s — Section "QSGDMaxNorm Quantization" (Eq. Q_s, definition of
  * xi_i), Algorithm 1 line "Quantize gradient", for all M workers:
  *   inv = (float)s / W[j]  (0 if W[j] = 0);  x = min(|v| * inv, (float)s);  l = floor(x);

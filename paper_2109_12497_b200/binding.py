@@ -26,7 +26,7 @@ UQ_STATUS_NONFINITE, UQ_STATUS_BAD_SEGMENTS, UQ_STATUS_SCALE_OVERFLOW, UQ_STATUS
 EXPORTS = (
     "uq_version", "uq_last_cuda_error", "uq_error_string", "uq_workspace_bytes", "uq_index_bytes",
     "uq_agree_scale", "uq_agree_scale_static", "uq_encode_single", "uq_select_scale_multi", "uq_encode_multi",
-    "uq_aggregate", "uq_decode", "uq_decode_update", "uq_randk_gather", "uq_randk_scatter", "uq_randk_update", "uq_index_min", "uq_decode_rows", "uq_select_encode_multi",
+    "uq_aggregate", "uq_decode", "uq_decode_update", "uq_randk_gather", "uq_randk_scatter", "uq_randk_update", "uq_index_min", "uq_decode_rows", "uq_select_encode_multi", "uq_agree_scale_amax",
 )
 
 
@@ -75,6 +75,7 @@ def lib() -> C.CDLL:
         L.uq_index_bytes.restype = SZ
         L.uq_index_bytes.argtypes = [LP, I]
         L.uq_agree_scale.argtypes = [LP, P, I, P, P, P, SZ, P]
+        L.uq_agree_scale_amax.argtypes = [LP, P, I, P, P, P, P, SZ, P]
         L.uq_agree_scale_static.argtypes = [LP, P, I, P, P, P]
         L.uq_encode_single.argtypes = [LP, P, P, I, U64, I, I, P, P, P]
         L.uq_select_scale_multi.argtypes = [LP, P, P, P, I, I, P, P, P]
@@ -352,3 +353,15 @@ def uq_select_encode_multi(layout: Layout, g: torch.Tensor, W: torch.Tensor, sca
     _check("uq_select_encode_multi", lib().uq_select_encode_multi(
         layout.ref(), _ptr(g), _ptr(W), arr, N, idx_bits, seed, rng_bits, fmt, _ptr(idx), _ptr(lev), _ptr(status),
         _stream()))
+
+
+def uq_agree_scale_amax(layout: Layout, g: torch.Tensor, norm: int, W: torch.Tensor, amax: torch.Tensor,
+                        status: Optional[torch.Tensor], workspace: torch.Tensor) -> None:
+    """uq_agree_scale that also writes amax[i] = max over the workers of |g[m, i]| (one row of
+    layout.worker_stride elements of g's dtype) for the selector to run on."""
+    layout.check_g(g)
+    layout.check_vec(W, torch.float32, layout.nseg, "W")
+    layout.check_vec(amax, layout.dtype, layout.worker_stride, "amax")
+    _check("uq_agree_scale_amax", lib().uq_agree_scale_amax(
+        layout.ref(), _ptr(g), norm, _ptr(W), _ptr(amax), _ptr(status), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _stream()))

@@ -6,6 +6,8 @@ namespace uq {
 int64_t norm_tiles(int64_t d);
 cudaError_t launch_agree_scale(const uq_layout &L, const void *g, int norm, float *W, uint32_t *status,
                                void *workspace, cudaStream_t st);
+cudaError_t launch_agree_scale_amax(const uq_layout &L, const void *g, int norm, float *W, void *amax, uint32_t *status,
+                                    void *workspace, cudaStream_t st);
 cudaError_t launch_encode(const uq_layout &L, const void *g, const float *W, const ScaleSet &scales,
                           const uint8_t *idx, int idx_bits, uint64_t seed, int rng_bits, int fmt, void *lev,
                           uint32_t *status, cudaStream_t st);
@@ -135,6 +137,17 @@ int uq_agree_scale(const uq_layout *L, const void *g, int norm, float *W, uint32
     if (workspace == nullptr || !aligned(workspace, 8) || workspace_bytes < uq_workspace_bytes(L))
         return UQ_ERR_WORKSPACE;
     return finish(uq::launch_agree_scale(*L, g, norm, W, status, workspace, (cudaStream_t)stream));
+}
+
+int uq_agree_scale_amax(const uq_layout *L, const void *g, int norm, float *W, void *amax, uint32_t *status,
+                        void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!layout_ok(L) || W == nullptr || !aligned(W, 4) || !aligned(status, 4)) return UQ_ERR_BAD_ARG;
+    if (norm != UQ_NORM_L2 && norm != UQ_NORM_LINF) return UQ_ERR_BAD_ARG;
+    if (L->d > 0 && (g == nullptr || amax == nullptr || !aligned(g, 16) || !aligned(amax, 16))) return UQ_ERR_BAD_ARG;
+    if (workspace == nullptr || !aligned(workspace, 8) || workspace_bytes < uq_workspace_bytes(L))
+        return UQ_ERR_WORKSPACE;
+    return finish(uq::launch_agree_scale_amax(*L, g, norm, W, amax, status, workspace, (cudaStream_t)stream));
 }
 
 int uq_encode_single(const uq_layout *L, const void *g, const float *W, int s, uint64_t seed, int rng_bits,

@@ -20,10 +20,11 @@ def to_device(w, g_np):
     return t.cuda()
 
 
-def run_gpu(w, g_np, seed=None, fused_select=False):
-    """All stage outputs of the CUDA path as numpy arrays.  fused_select: the multi-scale
-    quantizer selects and encodes in two kernels (the default) or in one."""
-    q = from_workload(w, keep_sums=True, fused_select=fused_select)
+def run_gpu(w, g_np, seed=None, mode="default"):
+    """All stage outputs of the CUDA path as numpy arrays.  mode picks the form of the multi-scale
+    path: "default" = "rows" (the selector reads all M rows), "amax" (agree-scale writes max_m |g|
+    and the selector runs on that row), "fused" (selection and encoding in one kernel)."""
+    q = from_workload(w, keep_sums=True, fused_select=mode == "fused", amax_select=mode == "amax")
     g = to_device(w, g_np)
     q.step(g, w.seed if seed is None else seed)
     torch.cuda.synchronize()
@@ -77,15 +78,16 @@ def ulp_distance(a, b):
 
 
 def check_parity(w, g_np, seed=None):
-    """Full comparison; returns the GPU result for further checks.  A multi-scale workload runs
-    twice, with selection and encoding as two kernels and fused into one: both must match the oracle."""
+    """Full comparison; returns the GPU result for further checks.  A multi-scale workload runs in
+    all three forms of its path (see run_gpu): each must match the oracle."""
     if w.quantizer == "multi":
-        _check_parity(w, g_np, seed, fused_select=True)
-    return _check_parity(w, g_np, seed, fused_select=False)
+        _check_parity(w, g_np, seed, "fused")
+        _check_parity(w, g_np, seed, "amax")
+    return _check_parity(w, g_np, seed, "default")
 
 
-def _check_parity(w, g_np, seed, fused_select):
-    gpu = run_gpu(w, g_np, seed, fused_select)
+def _check_parity(w, g_np, seed, mode):
+    gpu = run_gpu(w, g_np, seed, mode)
     assert gpu["status"] == 0
     ref_own = run_oracle(w, g_np, None, seed)
     # scale: exact for L-infinity; for L2 the binary64 sums may differ in the last bits, which

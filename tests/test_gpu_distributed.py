@@ -94,7 +94,7 @@ def test_exchange_replayed_rank_by_rank(name, d, M, parts, kw):
     torch.cuda.synchronize()
     assert int(status.item()) == 0
 
-    one = run_gpu(w, g_np)                                   # one process holding all M rows
+    one = run_gpu(w, g_np)                      # one process holding all M rows, same kernels
     assert np.array_equal(W.cpu().numpy(), one["W"])
     assert np.array_equal(lev_all.cpu().numpy().view(np.uint8)[:, : (d >> fmt)], one["lev"][:, : (d >> fmt)])
     if multi:

@@ -368,3 +368,12 @@ def test_randomized_configurations(case):
     wire format, level count, scale set, index width, norm, draw width, seed)."""
     w = _random_workload(np.random.default_rng(9000 + case))
     check_parity(w, wl.generate(w))
+
+
+@pytest.mark.parametrize("d", [1, 9, 2047, 2049, 8191, 8193, 70001])
+@pytest.mark.parametrize("name", ["c3", "c5"])
+def test_multi_scale_without_a_segment_table(name, d):
+    """The multi-scale path on one segment (no table at all) with a ragged last tile."""
+    w = wl.scaled(name, d, M=3, segments="one")
+    assert len(wl.segment_offsets(w)) == 2
+    check_parity(w, wl.generate(w))
