@@ -32,12 +32,17 @@
  *     binary32 operation order stated per call; no fused multiply-add is used where a
  *     floating-point value decides an integer.
  *   - Random draws (the paper's "independent random variables xi_i"): Philox4x32-10 with
- *     key = (seed low, seed high) and counter = (block low, block high, worker m, 0).
+ *     key = (seed low, seed high) and counter = (block low, block high, worker, 0), where
+ *     worker = layout.worker0 + m is the row's worker number in the whole job.
  *       rng_bits = 32: block = i/4, coordinate i takes word i%4, h = word >> 9 (23 bits)
  *       rng_bits = 16: block = i/8, word (i%8)/2, even i the low half, h = that half (16 bits)
  *     With b the width of h, a coordinate rounds up iff h < rint(p * 2^b) (ties to even), i.e.
  *     with the multiple of 2^-b nearest to the paper's probability p.  i is the coordinate's
- *     index in the worker's whole d-vector.
+ *     index in the worker's whole gradient (layout.coord0 + its index in the buffer).
+ *   - Stream order.  The kernels are launched so that the GPU may schedule the blocks of one while
+ *     the kernel before it in the stream is still draining (programmatic dependent launch); each
+ *     kernel waits for that predecessor to complete before it reads or writes anything, so the
+ *     results are those of plain stream order.
  */
 #ifndef UQ_H
 #define UQ_H
