@@ -158,8 +158,8 @@ def time_device_resident(q, g, w, steps, warmup, barrier):
     """(ms per step, {stage: mean ms}) with inputs resident in HBM, timed with CUDA events.
     The step time comes from a region that holds nothing but the K steps (an event recorded
     between two kernels would keep the second from being scheduled while the first drains, which
-    the library's launches otherwise allow); the per-stage times come from a second pass with an
-    event after every stage."""
+    the library's launches otherwise allow); the per-stage times (medians) come from a second pass with
+    an event after every stage."""
     import torch
     st = torch.cuda.current_stream()
     stages = STAGES_MULTI if q.multi else STAGES_SINGLE
@@ -178,7 +178,7 @@ def time_device_resident(q, g, w, steps, warmup, barrier):
     for k in range(n):
         run_stages(q, g, w.seed + k, evs[k])
     torch.cuda.synchronize()
-    per_stage = {s: statistics.fmean(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(n))
+    per_stage = {s: statistics.median(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(n))
                  for i, s in enumerate(stages)}
     return total_ms / steps, per_stage
 
