@@ -573,7 +573,7 @@ def gpu_main(args):
         "e2e": None if args.no_e2e else {
             "value": round(whole_job_value(world, w.in_bytes, e2e_ms), 2), "unit": UNIT, "ms_per_step": round(e2e_ms, 4),
             "h2d_bytes_per_step": res["h2d"], "d2h_bytes_per_step": res["d2h"]},
-        "gpu_launches": q.kernels_per_step() * args.steps,
+        "gpu_launches": q.kernels_per_step() * args.steps * world,          # all replicas together
         "clocks": clocks,
         "roofline": {
             "bound": "hbm", "kernel": dom, "achieved": round(dom_gbs, 1), "peak": peak, "unit": "GB/s",
