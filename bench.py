@@ -134,8 +134,12 @@ STAGES_MULTI = ["agree_scale", "select_scale", "encode", "aggregate_decode"]
 
 
 def run_stages(q, g, seed, events=None):
-    """One step; events (if given) is a list of len(stages)+1 CUDA events recorded around the stages."""
+    """One step; events (if given) is a list of len(stages)+1 CUDA events recorded around the stages.
+    Without events the step is the one call a user makes (Quantizer.step)."""
     import torch
+    if not events:
+        q.step(g, seed)
+        return
     st = torch.cuda.current_stream()
     k = 0
     if events: events[k].record(st)

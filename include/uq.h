@@ -322,6 +322,19 @@ int uq_index_min(const uint8_t *rows, int R, int64_t row_bytes, int64_t nbytes, 
                  uint8_t *idx, void *stream);
 
 /*
+ * One whole step in one call — Algorithm 1 lines "MaxAllReduce Norm" to "Reconstruct gradient"
+ * (scales = NULL: uq_agree_scale, uq_encode_single, uq_decode) or Algorithm 2 (scales given:
+ * uq_agree_scale, uq_select_scale_multi, uq_encode_multi, uq_decode), enqueued in that order on
+ * `stream`.  Nothing is computed differently: this saves the caller three trips through the
+ * binding when a step is so small that launch overhead counts.  Arguments are those of the calls
+ * it makes (idx is not used when scales = NULL); the first error stops the sequence and is returned.
+ */
+int uq_step(const uq_layout *layout, const void *g, int norm, int s, const int32_t *scales, int N,
+            int idx_bits, uint64_t seed, int rng_bits, int fmt, float *W, uint8_t *idx, void *lev,
+            float *out, int32_t *S_opt, uint32_t *status, void *workspace, size_t workspace_bytes,
+            void *stream);
+
+/*
  * GlobalRandKMaxNorm / GlobalRandKMaxNormMultiScale — Sections "GlobalRandKMaxNorm Compression"
  * and "GlobalRandKMaxNormMultiScale Compression": every worker keeps the same K coordinates,
  * chosen uniformly at every iteration, and the quantizer of Algorithm 1 / 2 runs on them.

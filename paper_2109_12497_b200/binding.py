@@ -26,7 +26,7 @@ UQ_STATUS_NONFINITE, UQ_STATUS_BAD_SEGMENTS, UQ_STATUS_SCALE_OVERFLOW, UQ_STATUS
 EXPORTS = (
     "uq_version", "uq_last_cuda_error", "uq_error_string", "uq_workspace_bytes", "uq_index_bytes",
     "uq_agree_scale", "uq_agree_scale_static", "uq_encode_single", "uq_select_scale_multi", "uq_encode_multi",
-    "uq_aggregate", "uq_decode", "uq_decode_update", "uq_randk_gather", "uq_randk_scatter", "uq_randk_update", "uq_index_min", "uq_decode_rows", "uq_select_encode_multi", "uq_agree_scale_amax",
+    "uq_aggregate", "uq_decode", "uq_decode_update", "uq_randk_gather", "uq_randk_scatter", "uq_randk_update", "uq_index_min", "uq_decode_rows", "uq_select_encode_multi", "uq_agree_scale_amax", "uq_step",
 )
 
 
@@ -75,6 +75,7 @@ def lib() -> C.CDLL:
         L.uq_index_bytes.restype = SZ
         L.uq_index_bytes.argtypes = [LP, I]
         L.uq_agree_scale.argtypes = [LP, P, I, P, P, P, SZ, P]
+        L.uq_step.argtypes = [LP, P, I, I, P, I, I, U64, I, I, P, P, P, P, P, P, P, SZ, P]
         L.uq_agree_scale_amax.argtypes = [LP, P, I, P, P, P, P, SZ, P]
         L.uq_agree_scale_static.argtypes = [LP, P, I, P, P, P]
         L.uq_encode_single.argtypes = [LP, P, P, I, U64, I, I, P, P, P]
@@ -365,4 +366,25 @@ def uq_agree_scale_amax(layout: Layout, g: torch.Tensor, norm: int, W: torch.Ten
     layout.check_vec(amax, layout.dtype, layout.worker_stride, "amax")
     _check("uq_agree_scale_amax", lib().uq_agree_scale_amax(
         layout.ref(), _ptr(g), norm, _ptr(W), _ptr(amax), _ptr(status), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _stream()))
+
+
+def uq_step(layout: Layout, g: torch.Tensor, norm: int, s: int, scales: Optional[Sequence[int]], idx_bits: int,
+            seed: int, rng_bits: int, fmt: int, W: torch.Tensor, idx: Optional[torch.Tensor], lev: torch.Tensor,
+            out: torch.Tensor, S_opt: Optional[torch.Tensor], status: Optional[torch.Tensor],
+            workspace: torch.Tensor) -> None:
+    """One whole step (agree-scale, [select], encode, aggregate + reconstruct) in one call."""
+    layout.check_g(g)
+    layout.check_lev(lev, fmt)
+    layout.check_vec(W, torch.float32, layout.nseg, "W")
+    layout.check_vec(out, torch.float32, layout.d, "out")
+    if S_opt is not None:
+        layout.check_vec(S_opt, torch.int32, layout.d, "S_opt")
+    arr, N = (None, 0)
+    if scales is not None:
+        arr, N = _scales(scales)
+        layout.check_vec(idx, torch.uint8, layout.index_bytes(idx_bits), "idx")
+    _check("uq_step", lib().uq_step(
+        layout.ref(), _ptr(g), norm, s, arr, N, idx_bits, seed, rng_bits, fmt, _ptr(W),
+        _ptr(idx) if scales is not None else None, _ptr(lev), _ptr(out), _ptr(S_opt), _ptr(status), _ptr(workspace),
         workspace.numel() * workspace.element_size(), _stream()))

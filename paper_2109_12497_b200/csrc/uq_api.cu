@@ -285,6 +285,23 @@ int uq_decode_update(const uq_layout *L, const void *lev, int fmt, const float *
                                               theta, momentum, lr, mu, wd));
 }
 
+int uq_step(const uq_layout *L, const void *g, int norm, int s, const int32_t *scales, int N, int idx_bits,
+            uint64_t seed, int rng_bits, int fmt, float *W, uint8_t *idx, void *lev, float *out, int32_t *S_opt,
+            uint32_t *status, void *workspace, size_t workspace_bytes, void *stream)
+{
+    int rc = uq_agree_scale(L, g, norm, W, status, workspace, workspace_bytes, stream);
+    if (rc != UQ_OK) return rc;
+    if (scales != nullptr) {
+        rc = uq_select_scale_multi(L, g, W, scales, N, idx_bits, idx, status, stream);
+        if (rc != UQ_OK) return rc;
+        rc = uq_encode_multi(L, g, W, scales, N, idx, idx_bits, seed, rng_bits, fmt, lev, status, stream);
+    } else {
+        rc = uq_encode_single(L, g, W, s, seed, rng_bits, fmt, lev, status, stream);
+    }
+    if (rc != UQ_OK) return rc;
+    return uq_decode(L, lev, UQ_SRC_LEVELS, fmt, W, s, scales, N, idx, idx_bits, out, S_opt, stream);
+}
+
 int uq_index_min(const uint8_t *rows, int R, int64_t row_bytes, int64_t nbytes, int idx_bits, uint8_t *idx, void *stream)
 {
     if (R < 1 || R > UQ_MAX_WORKERS || nbytes < 0 || (nbytes & 3) != 0 || row_bytes < nbytes || (row_bytes & 3) != 0)

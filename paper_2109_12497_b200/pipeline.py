@@ -92,6 +92,10 @@ class Quantizer:
 
     def step(self, g: torch.Tensor, seed: int = 0) -> torch.Tensor:
         """g: [M, stride] gradients of all workers -> the reconstructed average gradient [d]."""
+        if not (self.fused_select or self.amax_select):      # the plain sequence: one trip through the binding
+            B.uq_step(self.layout, g, self.norm, self.s, self.scales, self.idx_bits, seed, self.rng_bits, self.fmt,
+                      self.W, self.idx, self.lev, self.out, self.S, self.status, self.workspace)
+            return self.out[: self.d]
         self.agree_scale(g)
         if self.multi and self.fused_select:
             self.select_encode(g, seed)
