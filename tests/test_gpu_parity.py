@@ -377,3 +377,24 @@ def test_multi_scale_without_a_segment_table(name, d):
     w = wl.scaled(name, d, M=3, segments="one")
     assert len(wl.segment_offsets(w)) == 2
     check_parity(w, wl.generate(w))
+
+
+@pytest.mark.parametrize("name", ["c2", "c3"])
+def test_back_to_back_steps_do_not_interfere(name):
+    """A hundred steps enqueued without a host synchronization in between (the launches let a
+    kernel's blocks be scheduled while the kernel before it drains): every step must leave exactly
+    the sums and values of the first one."""
+    w = wl.scaled(name, 1_500_007, M=8)
+    g = to_device(w, wl.generate(w))
+    from paper_2109_12497_b200.pipeline import from_workload
+    q = from_workload(w, keep_sums=True)
+    q.step(g, w.seed)
+    torch.cuda.synchronize()
+    S0, out0, lev0 = q.S.clone(), q.out.clone(), q.lev.clone()
+    bad = torch.zeros((), dtype=torch.int64, device="cuda")
+    for k in range(100):
+        q.lev.fill_(0x55)                                    # stale levels would change the sums
+        q.step(g, w.seed)
+        bad += (q.S != S0).sum() + (q.out != out0).sum() + (q.lev[:, : w.d] != lev0[:, : w.d]).sum()
+    torch.cuda.synchronize()
+    assert int(bad.item()) == 0
