@@ -164,6 +164,99 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
     else *(uint64_t *)(p.idx + i) = packed;
 }
 
+// One row only (M = 1: a single worker, or the row of maxima that uq_agree_scale_amax leaves).
+// With nothing to combine across workers the general kernel's per-row setup (segment lookup: two
+// dependent loads; threshold table: a division and a short search per scale) is all that is left
+// per 256 coordinates, and its latency sets the time.  Here a CTA owns kRowUnits * 2048 coordinates;
+// it looks the segment up once and, when that segment covers the whole tile (the common case),
+// builds the threshold table once per warp for all its rows; a thread's kRowUnits units are all
+// in flight together.  A tile that a boundary crosses falls back to the per-row setup.
+constexpr int kRowUnits = 8;
+
+template <int DT, int IDXB, int LEVELS>
+__global__ void __launch_bounds__(kThreads, 4) select_row_kernel(const __grid_constant__ SelectParams p)
+{
+    grid_dependency_prologue();
+    using E = Elem<DT>;
+    constexpr int H = 8 / E::G;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t t0 = (int64_t)blockIdx.x * (kSelectTile * kRowUnits);
+    const int64_t t1 = min(t0 + (int64_t)kSelectTile * kRowUnits, p.d);
+    uint4 q[kRowUnits][H];
+#pragma unroll
+    for (int u = 0; u < kRowUnits; ++u) {
+        const int64_t i = t0 + (int64_t)u * kSelectTile + tid * 8;
+#pragma unroll
+        for (int h = 0; h < H; ++h)
+            q[u][h] = i < p.d ? ld_stream((const char *)p.g + (size_t)(i + h * E::G) * E::BYTES) : make_uint4(0, 0, 0, 0);
+    }
+    __shared__ int32_t sh_thr[kWarps][2 * UQ_MAX_SCALES];
+    const int jt = warp_find_segment(p.seg_off, p.nseg, t0);
+    const bool tile_uniform = segment_end(p.seg_off, p.nseg, jt, p.d) >= t1;
+    int j_table = -1;                                               // segment whose thresholds the table holds
+    if (tile_uniform) {
+        int32_t thr = -1;
+        if (lane < p.scales.N) thr = pass_threshold(inv_scale_sel(p.scales.s[lane], __ldg(p.W + jt)), p.s_hat);
+        sh_thr[warp][lane] = thr;
+        __syncwarp();
+        j_table = jt;
+    }
+#pragma unroll
+    for (int u = 0; u < kRowUnits; ++u) {
+        const int64_t i = t0 + (int64_t)u * kSelectTile + tid * 8;
+        const int64_t row0 = i - (int64_t)lane * 8;
+        if (row0 >= p.d) break;                                     // warp-uniform
+        uint32_t amag[8];
+        if (DT == UQ_F32) {
+            amag[0] = q[u][0].x & 0x7FFFFFFFu; amag[1] = q[u][0].y & 0x7FFFFFFFu;
+            amag[2] = q[u][0].z & 0x7FFFFFFFu; amag[3] = q[u][0].w & 0x7FFFFFFFu;
+            amag[4] = q[u][H - 1].x & 0x7FFFFFFFu; amag[5] = q[u][H - 1].y & 0x7FFFFFFFu;
+            amag[6] = q[u][H - 1].z & 0x7FFFFFFFu; amag[7] = q[u][H - 1].w & 0x7FFFFFFFu;
+        } else {
+            const uint32_t w[4] = { q[u][0].x & 0x7FFF7FFFu, q[u][0].y & 0x7FFF7FFFu, q[u][0].z & 0x7FFF7FFFu,
+                                    q[u][0].w & 0x7FFF7FFFu };
+#pragma unroll
+            for (int k = 0; k < 4; ++k) { amag[2 * k] = w[k] << 16; amag[2 * k + 1] = w[k] & 0xFFFF0000u; }
+        }
+        int j0 = jt;
+        bool row_uniform = true;
+        if (!tile_uniform) {                                        // per-row setup, as in the general kernel
+            const int64_t row1 = min(row0 + 256, p.d);
+            j0 = warp_find_segment(p.seg_off, p.nseg, row0);
+            row_uniform = segment_end(p.seg_off, p.nseg, j0, p.d) >= row1;
+            if (row_uniform && j0 != j_table) {
+                __syncwarp();
+                int32_t thr = -1;
+                if (lane < p.scales.N) thr = pass_threshold(inv_scale_sel(p.scales.s[lane], __ldg(p.W + j0)), p.s_hat);
+                sh_thr[warp][lane] = thr;
+                __syncwarp();
+                j_table = j0;
+            }
+        }
+        typename std::conditional<IDXB == 8, uint64_t, uint32_t>::type packed = 0;
+        if (row_uniform) {
+            const int32_t *T = sh_thr[warp];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int32_t a = (int32_t)amag[e];
+                int k = 0;
+#pragma unroll
+                for (int step = 1 << (LEVELS - 1); step >= 1; step >>= 1)
+                    if (a <= T[k + step]) k += step;                // k + step < 2^LEVELS <= 16
+                if (i + e >= p.d) k = 0;                            // padding keeps index 0
+                packed |= (decltype(packed))k << (e * IDXB);
+            }
+        } else if (i < p.d) {
+            packed = (decltype(packed))select_general(p, i, amag, IDXB, j0);
+        }
+        if (i >= p.d) continue;
+        if (IDXB == 1) p.idx[i >> 3] = (uint8_t)packed;
+        else if (IDXB == 2) *(uint16_t *)(p.idx + (i >> 2)) = (uint16_t)packed;
+        else if (IDXB == 4) *(uint32_t *)(p.idx + (i >> 1)) = (uint32_t)packed;
+        else *(uint64_t *)(p.idx + i) = packed;
+    }
+}
+
 template <int DT, int IDXB>
 static cudaError_t dispatch_levels(const SelectParams &p, unsigned blocks, cudaStream_t st)
 {
@@ -178,6 +271,28 @@ static cudaError_t dispatch_levels(const SelectParams &p, unsigned blocks, cudaS
 template <int DT>
 static cudaError_t dispatch(const SelectParams &p, int idx_bits, cudaStream_t st)
 {
+    if (p.M == 1 && p.d > 0) {                                      // one row: the kernel without per-row setup
+        const int64_t nb = (p.d + kSelectTile * kRowUnits - 1) / (kSelectTile * kRowUnits);
+        if (nb > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+        const int N = p.scales.N;
+        const int lv = N <= 2 ? 1 : N <= 4 ? 2 : N <= 8 ? 3 : 4;
+#define UQ_ROW(IB, LV) launch_k(select_row_kernel<DT, IB, LV>, (unsigned)nb, kThreads, st, p)
+        switch (idx_bits * 8 + lv) {
+        case 1 * 8 + 1: UQ_ROW(1, 1); break;
+        case 2 * 8 + 1: UQ_ROW(2, 1); break;
+        case 2 * 8 + 2: UQ_ROW(2, 2); break;
+        case 4 * 8 + 1: UQ_ROW(4, 1); break;
+        case 4 * 8 + 2: UQ_ROW(4, 2); break;
+        case 4 * 8 + 3: UQ_ROW(4, 3); break;
+        case 4 * 8 + 4: UQ_ROW(4, 4); break;
+        case 8 * 8 + 1: UQ_ROW(8, 1); break;
+        case 8 * 8 + 2: UQ_ROW(8, 2); break;
+        case 8 * 8 + 3: UQ_ROW(8, 3); break;
+        default: UQ_ROW(8, 4); break;
+        }
+#undef UQ_ROW
+        return cudaGetLastError();
+    }
     const int64_t blocks = (p.d + kSelectTile - 1) / kSelectTile;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
