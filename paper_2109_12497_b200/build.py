@@ -61,7 +61,8 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     with ThreadPoolExecutor(max_workers=len(SOURCES)) as pool:
         objs = list(pool.map(compile_one, SOURCES))
     tmp = LIB.with_suffix(f".{os.getpid()}.tmp")
-    subprocess.run([nvcc, "-shared", "-o", str(tmp), *map(str, objs), "-cudart", "static"], check=True)
+    subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", str(tmp), *map(str, objs),
+                    "-cudart", "static"], check=True)
     os.replace(tmp, LIB)
     return LIB
 
