@@ -92,6 +92,43 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
         == B.UQ_ERR_BAD_ARG
 
 
+def test_later_entry_points_reject_bad_arguments_on_the_host(lib):
+    """The entry points added after the six of the hot path: same rule, nothing is launched."""
+    p = 0x10000
+    F = C.c_float
+    ok, bad = C.byref(_layout()), C.byref(_layout(M=0))
+    sc = (C.c_int32 * 2)(127, 1016)
+    rows = (C.c_void_p * 2)(p, p)
+    assert lib.uq_step(bad, p, B.UQ_NORM_L2, 127, None, 0, 0, 0, 16, B.UQ_FMT_I8, p, None, p, p, None, None, p, 1 << 20,
+                       None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_step(ok, p, B.UQ_NORM_L2, 127, None, 0, 0, 0, 16, B.UQ_FMT_I8, p, None, p, p, None, None, p, 8,
+                       None) == B.UQ_ERR_WORKSPACE
+    assert lib.uq_agree_scale_amax(bad, p, B.UQ_NORM_L2, p, p, None, p, 1 << 20, None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_agree_scale_amax(ok, p, B.UQ_NORM_L2, p, p + 8, None, p, 1 << 20, None) == B.UQ_ERR_BAD_ARG   # alignment
+    assert lib.uq_agree_scale_amax(ok, p, B.UQ_NORM_L2, p, None, None, p, 1 << 20, None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_select_encode_multi(ok, p, p, sc, 2, 3, 0, 16, B.UQ_FMT_I8, p, p, None, None) == B.UQ_ERR_BAD_ARG   # idx_bits
+    assert lib.uq_select_encode_multi(ok, p, p, sc, 2, 2, 0, 16, B.UQ_FMT_I4X2, p, p, None, None) == B.UQ_ERR_BAD_ARG  # s_hat > 7
+    assert lib.uq_select_encode_multi(ok, p, p, sc, 2, 2, 0, 16, B.UQ_FMT_I8, None, p, None, None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_index_min(p, 0, 64, 64, 2, p, None) == B.UQ_ERR_BAD_ARG                    # R
+    assert lib.uq_index_min(p, 2, 64, 62, 2, p, None) == B.UQ_ERR_BAD_ARG                    # whole words
+    assert lib.uq_index_min(p, 2, 32, 64, 2, p, None) == B.UQ_ERR_BAD_ARG                    # rows overlap
+    assert lib.uq_index_min(p, 2, 64, 64, 3, p, None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_decode_rows(ok, None, B.UQ_FMT_I8, p, 127, None, 0, None, 0, p, None, None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_decode_rows(ok, rows, 9, p, 127, None, 0, None, 0, p, None, None) == B.UQ_ERR_BAD_ARG
+    rows[1] = p + 1
+    assert lib.uq_decode_rows(ok, rows, B.UQ_FMT_I8, p, 127, None, 0, None, 0, p, None, None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_decode_update(ok, p, B.UQ_FMT_I8, p, 127, None, 0, None, 0, p, None, F(float("nan")), F(0), F(0), None,
+                                None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_decode_update(ok, p, B.UQ_FMT_I8, p, 127, None, 0, None, 0, p + 4, None, F(0.1), F(0), F(0), None,
+                                None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_randk_gather(ok, p, 1001, 0, p, p, 1024, None, None) == B.UQ_ERR_BAD_ARG     # K > d
+    assert lib.uq_randk_gather(ok, p, 10, 0, p, p, 40, None, None) == B.UQ_ERR_BAD_ARG         # stride % 32
+    assert lib.uq_randk_gather(ok, p, 10, 0, p, p, 0, None, None) == B.UQ_ERR_BAD_ARG          # stride < K
+    assert lib.uq_randk_scatter(100, 101, p, p, p, None, None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_randk_update(100, 10, p, None, p, F(0.1), None, None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_randk_update(100, 10, p, p, p, F(float("nan")), None, None) == B.UQ_ERR_BAD_ARG
+
+
 def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(B, "LIB_PATH", tmp_path / "missing.so")
