@@ -110,6 +110,9 @@ const char *uq_error_string(int code);
 /* Bytes of device scratch uq_agree_scale needs for this layout (0 on a bad layout). */
 size_t uq_workspace_bytes(const uq_layout *layout);
 
+/* Bytes of device scratch uq_agree_scale_amax needs (its partials are finer; 0 on a bad layout). */
+size_t uq_workspace_bytes_amax(const uq_layout *layout);
+
 /* Bytes of a packed scale-index stream for this layout: worker_stride * idx_bits / 8. */
 size_t uq_index_bytes(const uq_layout *layout, int idx_bits);
 
@@ -172,8 +175,9 @@ int uq_agree_scale_static(const uq_layout *layout, const void *g, int norm, floa
  * writes the indices that the call on all M rows writes, reading 1/M of the bytes.
  *   amax  out  [worker_stride] elements of layout->dtype, device, 16-byte aligned: the magnitude
  *              (sign bit clear) of the largest entry of coordinate i; elements d.. are padding
- * W may differ from uq_agree_scale's in the last bit (another fixed order of additions); every
- * other argument and error is uq_agree_scale's.
+ * W may differ from uq_agree_scale's in the last bit (another fixed order of additions); the
+ * workspace holds uq_workspace_bytes_amax(layout) bytes; every other argument and error is
+ * uq_agree_scale's.
  */
 int uq_agree_scale_amax(const uq_layout *layout, const void *g, int norm, float *W, void *amax,
                         uint32_t *status, void *workspace, size_t workspace_bytes, void *stream);

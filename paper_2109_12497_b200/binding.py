@@ -24,7 +24,7 @@ UQ_SRC_LEVELS, UQ_SRC_SUMS = 0, 1
 UQ_STATUS_NONFINITE, UQ_STATUS_BAD_SEGMENTS, UQ_STATUS_SCALE_OVERFLOW, UQ_STATUS_BAD_INDEX = 1, 2, 4, 8
 
 EXPORTS = (
-    "uq_version", "uq_last_cuda_error", "uq_error_string", "uq_workspace_bytes", "uq_index_bytes",
+    "uq_version", "uq_last_cuda_error", "uq_error_string", "uq_workspace_bytes", "uq_index_bytes", "uq_workspace_bytes_amax",
     "uq_agree_scale", "uq_agree_scale_static", "uq_encode_single", "uq_select_scale_multi", "uq_encode_multi",
     "uq_aggregate", "uq_decode", "uq_decode_update", "uq_randk_gather", "uq_randk_scatter", "uq_randk_update", "uq_index_min", "uq_decode_rows", "uq_select_encode_multi", "uq_agree_scale_amax", "uq_step",
 )
@@ -72,6 +72,8 @@ def lib() -> C.CDLL:
         L.uq_error_string.argtypes = [I]
         L.uq_workspace_bytes.restype = SZ
         L.uq_workspace_bytes.argtypes = [LP]
+        L.uq_workspace_bytes_amax.restype = SZ
+        L.uq_workspace_bytes_amax.argtypes = [LP]
         L.uq_index_bytes.restype = SZ
         L.uq_index_bytes.argtypes = [LP, I]
         L.uq_agree_scale.argtypes = [LP, P, I, P, P, P, SZ, P]
@@ -92,7 +94,7 @@ def lib() -> C.CDLL:
         L.uq_randk_gather.argtypes = [LP, P, I64, U64, P, P, I64, P, P]
         L.uq_randk_scatter.argtypes = [I64, I64, P, P, P, P, P]
         L.uq_randk_update.argtypes = [I64, I64, P, P, P, F, P, P]
-        for name in EXPORTS[5:]:
+        for name in EXPORTS[6:]:
             getattr(L, name).restype = I
         _lib = L
     return _lib
@@ -144,6 +146,9 @@ class Layout:
 
     def workspace_bytes(self) -> int:
         return int(lib().uq_workspace_bytes(self.ref()))
+
+    def workspace_bytes_amax(self) -> int:
+        return int(lib().uq_workspace_bytes_amax(self.ref()))
 
     def index_bytes(self, idx_bits: int) -> int:
         return int(lib().uq_index_bytes(self.ref(), idx_bits))

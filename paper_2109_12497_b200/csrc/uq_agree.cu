@@ -107,7 +107,7 @@ template <int NORM>
 __global__ void __launch_bounds__(kThreads)
 norm_finalize_kernel(const double *__restrict__ part, int M, int64_t d, int nseg,
                      const int64_t *__restrict__ seg_off, int64_t ntiles, float *__restrict__ W,
-                     uint32_t *__restrict__ status)
+                     uint32_t *__restrict__ status, int tile_coords)       // tile_coords: coordinates per partial
 {
     grid_dependency_prologue();
     const int j = blockIdx.x;
@@ -120,7 +120,7 @@ norm_finalize_kernel(const double *__restrict__ part, int M, int64_t d, int nseg
 
     double best = 0.0;
     if (a < b) {
-        const int64_t first = a / kNormTile, last = (b - 1) / kNormTile;
+        const int64_t first = a / tile_coords, last = (b - 1) / tile_coords;
         for (int m = warp; m < M; m += kWarps) {
             const double *prow = part + (size_t)m * (size_t)(ntiles + nseg) + j;
             double acc = 0.0;
@@ -163,20 +163,22 @@ static cudaError_t launch(const uq_layout &L, const void *g, float *W, uint32_t 
                                                                  L.seg_off, ntiles, part);
     }
     launch_k(norm_finalize_kernel<NORM>, L.nseg, kThreads, st, part, L.M, L.d, L.nseg, L.seg_off, ntiles, W,
-                                                          status);
+                                                          status, kNormTile);
     return cudaGetLastError();
 }
 
 int64_t norm_tiles(int64_t d) { return (d + kNormTile - 1) / kNormTile; }
 
 // The second launch alone, for the kernel that fills the same scratch slots together with amax.
-cudaError_t launch_norm_finalize(const uq_layout &L, int norm, const double *part, int64_t ntiles, float *W,
-                                 uint32_t *status, cudaStream_t st)
+cudaError_t launch_norm_finalize(const uq_layout &L, int norm, const double *part, int64_t ntiles, int tile_coords,
+                                 float *W, uint32_t *status, cudaStream_t st)
 {
     if (norm == UQ_NORM_L2)
-        launch_k(norm_finalize_kernel<UQ_NORM_L2>, L.nseg, kThreads, st, part, L.M, L.d, L.nseg, L.seg_off, ntiles, W, status);
+        launch_k(norm_finalize_kernel<UQ_NORM_L2>, L.nseg, kThreads, st, part, L.M, L.d, L.nseg, L.seg_off, ntiles, W, status,
+                 tile_coords);
     else
-        launch_k(norm_finalize_kernel<UQ_NORM_LINF>, L.nseg, kThreads, st, part, L.M, L.d, L.nseg, L.seg_off, ntiles, W, status);
+        launch_k(norm_finalize_kernel<UQ_NORM_LINF>, L.nseg, kThreads, st, part, L.M, L.d, L.nseg, L.seg_off, ntiles, W, status,
+                 tile_coords);
     return cudaGetLastError();
 }
 

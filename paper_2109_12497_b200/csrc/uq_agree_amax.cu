@@ -5,12 +5,12 @@
 // the single row amax instead of on all M rows: one of the three passes that the multi-scale path
 // makes over the gradients shrinks to a pass over 1/M of the bytes.
 //
-// A CTA owns one tile of kNormTile coordinates of ALL workers (the plain kernel: of one worker).  A
-// thread takes 8 consecutive coordinates per sub-tile of 2048; it walks the workers, eight at a
+// A CTA owns one tile of kAmaxTile coordinates of ALL workers (the plain kernel: 8192 of one worker).
+// A thread takes 8 consecutive coordinates per sub-tile of 2048; it walks the workers, eight at a
 // time, adding each worker's squares (or magnitudes) to that worker's accumulator and folding the
 // magnitudes into the 8 running maxima, which it stores after the last worker.  The per-worker
-// accumulators are then reduced over the CTA in a fixed order and stored in the same scratch slots
-// (tile + segment) as the plain kernel's, so the finalize kernel is shared.  The order of additions
+// accumulators are then reduced over the CTA in a fixed order and stored in scratch slots
+// (tile + segment) laid out like the plain kernel's, for its own tile size, so the finalize kernel is shared.  The order of additions
 // differs from the plain kernel's (another assignment of coordinates to threads), so the last bit
 // of W may differ between the two; each is reproducible.
 #include "uq_device.cuh"
@@ -18,8 +18,12 @@
 
 namespace uq {
 
+#ifndef UQ_AMAX_TILE
+#define UQ_AMAX_TILE 8192
+#endif
+constexpr int kAmaxTile = UQ_AMAX_TILE;            // coordinates per CTA and per partial (swept: 2048 and 4096 are slower)
 constexpr int kSub = kThreads * 8;                 // coordinates per sub-tile
-constexpr int kSubs = kNormTile / kSub;            // sub-tiles per tile
+constexpr int kSubs = kAmaxTile / kSub;            // sub-tiles per tile
 constexpr int kChunk = 8;                          // workers whose accumulators a thread holds at once
 
 // amax of 8 coordinates, kept in the element type's own magnitude bits:
@@ -62,6 +66,46 @@ template <> struct Amax8<UQ_BF16> {
     __device__ __forceinline__ void store(void *p) const { *(uint4 *)p = make_uint4(a[0], a[1], a[2], a[3]); }
 };
 
+// Eight values per lane reduced over the warp together: three exchange rounds that halve the number
+// of values a lane holds (a lane keeps the half selected by one of its lane bits and adds the
+// partner's copy of that half), then two ordinary rounds on the single value left.  Nine 64-bit
+// exchanges instead of forty; the order of additions is fixed.  Afterwards the lanes with
+// (lane & 3) == 0 hold the warp totals: lane 4 * k' holds value number bitrev3(k')... the mapping is
+// returned in `which` (the index 0..7 of the value this lane ends up with).
+template <int NORM>
+__device__ __forceinline__ double warp_reduce8(const double (&v)[8], int lane, int &which)
+{
+    double a[4], b[2], c;
+    {
+        const bool up = lane & 16;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const double send = up ? v[k] : v[4 + k];
+            const double recv = __shfl_xor_sync(0xFFFFFFFFu, send, 16);
+            a[k] = combine<NORM>(up ? v[4 + k] : v[k], recv);
+        }
+    }
+    {
+        const bool up = lane & 8;
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const double send = up ? a[k] : a[2 + k];
+            const double recv = __shfl_xor_sync(0xFFFFFFFFu, send, 8);
+            b[k] = combine<NORM>(up ? a[2 + k] : a[k], recv);
+        }
+    }
+    {
+        const bool up = lane & 4;
+        const double send = up ? b[0] : b[1];
+        const double recv = __shfl_xor_sync(0xFFFFFFFFu, send, 4);
+        c = combine<NORM>(up ? b[1] : b[0], recv);
+    }
+    c = combine<NORM>(c, __shfl_xor_sync(0xFFFFFFFFu, c, 2));
+    c = combine<NORM>(c, __shfl_xor_sync(0xFFFFFFFFu, c, 1));
+    which = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
+    return c;
+}
+
 template <int DT, int NORM>
 __global__ void __launch_bounds__(kThreads, 3)
 norm_amax_kernel(const void *__restrict__ g, int64_t d, int64_t stride, int M, int nseg,
@@ -71,13 +115,13 @@ norm_amax_kernel(const void *__restrict__ g, int64_t d, int64_t stride, int M, i
     using E = Elem<DT>;
     constexpr int H = 8 / E::G;
     const int64_t tile = blockIdx.x;
-    const int64_t t0 = tile * kNormTile;
-    const int64_t t1 = min(t0 + (int64_t)kNormTile, d);
+    const int64_t t0 = tile * kAmaxTile;
+    const int64_t t1 = min(t0 + (int64_t)kAmaxTile, d);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const size_t slots = (size_t)(ntiles + nseg);
     const int j0 = warp_find_segment(seg_off, nseg, t0);
 
-    const bool full = t1 - t0 == kNormTile;                         // else the ragged last tile
+    const bool full = t1 - t0 == kAmaxTile;                         // else the ragged last tile
     if (segment_end(seg_off, nseg, j0, d) < t1) {
         // a tile that a segment boundary crosses (so there is a segment table): the norms worker by
         // worker through the shared out-of-line path, the maxima in a plain pass of their own
@@ -146,10 +190,14 @@ norm_amax_kernel(const void *__restrict__ g, int64_t d, int64_t stride, int M, i
             am.store((char *)amax + (size_t)i * E::BYTES);
         }
         // one partial per worker of the chunk, reduced over the CTA in a fixed order
+        {
+            static_assert(kChunk == 8, "warp_reduce8 takes eight values");
+            double v[kChunk];
 #pragma unroll
-        for (int k = 0; k < kChunk; ++k) {
-            const double w = warp_reduce<NORM>(acc[k].value());
-            if (lane == 0) sh[k][warp] = w;
+            for (int k = 0; k < kChunk; ++k) v[k] = acc[k].value();
+            int which;
+            const double w = warp_reduce8<NORM>(v, lane, which);
+            if ((lane & 3) == 0) sh[which][warp] = w;
         }
         __syncthreads();
         if (tid < kChunk && c0 + tid < M) {
@@ -163,14 +211,15 @@ norm_amax_kernel(const void *__restrict__ g, int64_t d, int64_t stride, int M, i
 }
 
 // The finalize kernel of uq_agree.cu (same scratch layout).
-cudaError_t launch_norm_finalize(const uq_layout &L, int norm, const double *part, int64_t ntiles, float *W,
-                                 uint32_t *status, cudaStream_t st);
-int64_t norm_tiles(int64_t d);
+cudaError_t launch_norm_finalize(const uq_layout &L, int norm, const double *part, int64_t ntiles, int tile_coords,
+                                 float *W, uint32_t *status, cudaStream_t st);
+
+int64_t norm_tiles_amax(int64_t d) { return (d + kAmaxTile - 1) / kAmaxTile; }
 
 cudaError_t launch_agree_scale_amax(const uq_layout &L, const void *g, int norm, float *W, void *amax, uint32_t *status,
                                     void *workspace, cudaStream_t st)
 {
-    const int64_t ntiles = norm_tiles(L.d);
+    const int64_t ntiles = norm_tiles_amax(L.d);
     double *part = (double *)workspace;
     if (L.d > 0) {
         if (ntiles > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
@@ -183,7 +232,7 @@ cudaError_t launch_agree_scale_amax(const uq_layout &L, const void *g, int norm,
             else launch_k(norm_amax_kernel<UQ_BF16, UQ_NORM_LINF>, nb, kThreads, st, g, L.d, L.worker_stride, L.M, L.nseg, L.seg_off, ntiles, part, amax);
         }
     }
-    return launch_norm_finalize(L, norm, part, ntiles, W, status, st);
+    return launch_norm_finalize(L, norm, part, ntiles, kAmaxTile, W, status, st);
 }
 
 }  // namespace uq

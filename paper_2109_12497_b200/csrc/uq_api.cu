@@ -4,6 +4,7 @@
 
 namespace uq {
 int64_t norm_tiles(int64_t d);
+int64_t norm_tiles_amax(int64_t d);
 cudaError_t launch_agree_scale(const uq_layout &L, const void *g, int norm, float *W, uint32_t *status,
                                void *workspace, cudaStream_t st);
 cudaError_t launch_agree_scale_amax(const uq_layout &L, const void *g, int norm, float *W, void *amax, uint32_t *status,
@@ -122,6 +123,12 @@ size_t uq_workspace_bytes(const uq_layout *L)
     return (size_t)L->M * (size_t)(uq::norm_tiles(L->d) + L->nseg) * sizeof(double);
 }
 
+size_t uq_workspace_bytes_amax(const uq_layout *L)
+{
+    if (!layout_ok(L)) return 0;
+    return (size_t)L->M * (size_t)(uq::norm_tiles_amax(L->d) + L->nseg) * sizeof(double);
+}
+
 size_t uq_index_bytes(const uq_layout *L, int idx_bits)
 {
     if (!layout_ok(L) || !idx_bits_ok(idx_bits)) return 0;
@@ -145,7 +152,7 @@ int uq_agree_scale_amax(const uq_layout *L, const void *g, int norm, float *W, v
     if (!layout_ok(L) || W == nullptr || !aligned(W, 4) || !aligned(status, 4)) return UQ_ERR_BAD_ARG;
     if (norm != UQ_NORM_L2 && norm != UQ_NORM_LINF) return UQ_ERR_BAD_ARG;
     if (L->d > 0 && (g == nullptr || amax == nullptr || !aligned(g, 16) || !aligned(amax, 16))) return UQ_ERR_BAD_ARG;
-    if (workspace == nullptr || !aligned(workspace, 8) || workspace_bytes < uq_workspace_bytes(L))
+    if (workspace == nullptr || !aligned(workspace, 8) || workspace_bytes < uq_workspace_bytes_amax(L))
         return UQ_ERR_WORKSPACE;
     return finish(uq::launch_agree_scale_amax(*L, g, norm, W, amax, status, workspace, (cudaStream_t)stream));
 }

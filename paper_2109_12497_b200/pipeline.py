@@ -43,7 +43,8 @@ class Quantizer:
         nseg = self.layout.nseg
         self.W = torch.zeros(nseg, dtype=torch.float32, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
-        self.workspace = torch.empty(max(8, self.layout.workspace_bytes()), dtype=torch.uint8, device=dev)
+        self.workspace = torch.empty(max(8, self.layout.workspace_bytes(), self.layout.workspace_bytes_amax()),
+                                     dtype=torch.uint8, device=dev)
         self.lev = torch.empty((M, self.layout.level_row_bytes(fmt)), dtype=torch.int8, device=dev)
         self.idx = (torch.empty(max(16, self.layout.index_bytes(self.idx_bits)), dtype=torch.uint8, device=dev)
                     if self.multi else None)
