@@ -23,6 +23,19 @@ The barriers are one-element NCCL all-reduces, so a peer that never arrives ends
 timeout handling rather than in a kernel of this library waiting on a flag.  This mode needs
 GPUs that can map each other's memory; it has run here on a one-rank group only.
 
+``exchange="slices"`` is the reduce-scatter / all-gather form of the last exchange, the one that keeps
+the bytes per process constant as the job grows: the coordinates are cut into ``world_size`` slices of
+equal length, an all-to-all hands process r every worker's levels of slice r (still in their wire
+format), process r sums and reconstructs its slice (``uq_decode`` on the slice's layout: its own
+segment table counted from the slice's start, the matching part of W and of the index), and an
+all-gather of the reconstructed slices gives every process the whole average.  Received per process
+and step: (world_size - 1) / world_size * (M_local * d * bits / 8 + 4 * d) bytes, against
+(world_size - 1) * M_local * d * bits / 8 for the gather of whole rows; fewer from world_size 6 on
+for 8-bit levels and one worker per process.  Integer sums do not depend on the order of the rows,
+so the result is again bit for bit the single-process one.  Rows are padded to a multiple of
+``world_size * 128`` coordinates in this mode (``self.stride``), so that every slice of a level row,
+of the packed index and of the output starts on a 16-byte boundary.
+
 The exchanges are ``torch.distributed`` collectives (NCCL on GPUs); every arithmetic step is one
 call of the C ABI.  ``kernels`` is the module that provides those calls; it defaults to the CUDA
 binding and exists so that the exchange logic can be exercised without GPUs by handing in a
@@ -38,12 +51,19 @@ import torch
 import torch.distributed as dist
 
 
+SLICE_ALIGN = 128      # coordinates: 16 bytes of a 1-bit index, 32 of a 2-bit level row, 512 of the output
+
+
 class DistributedQuantizer:
     def __init__(self, M_local: int, d: int, dtype: torch.dtype = torch.float32,
                  seg_off: Optional[Sequence[int]] = None, s: int = 127,
                  scales: Optional[Sequence[int]] = None, fmt: int = 0, idx_bits: int = 0, norm: int = 2,
                  rng_bits: int = 32, group=None, device: str | torch.device = "cuda", kernels=None,
-                 pull_levels: bool = False):
+                 pull_levels: bool = False, exchange: Optional[str] = None):
+        exchange = exchange or ("pull" if pull_levels else "gather")
+        if exchange not in ("gather", "pull", "slices"):
+            raise ValueError("uq: exchange is 'gather', 'pull' or 'slices'")
+        pull_levels = exchange == "pull"
         if kernels is None:
             from . import binding as kernels
             kernels.lib()                               # fail now if the CUDA library is not built
@@ -54,7 +74,13 @@ class DistributedQuantizer:
         if self.M > 64:
             raise ValueError("uq: at most 64 workers in a job")
         dev = torch.device(device)
+        self.exchange = exchange
         self.stride = -(-d // 32) * 32
+        if exchange == "slices":
+            if fmt not in (0, 1, 2):
+                raise ValueError("uq: the slice exchange needs a level format whose rows are one plane")
+            self.slice_coords = max(1, -(-d // (self.world * SLICE_ALIGN))) * SLICE_ALIGN
+            self.stride = self.world * self.slice_coords
         self.multi = scales is not None and idx_bits != 0
         self.s = int(scales[0]) if self.multi else int(s)
         self.scales = [int(x) for x in scales] if self.multi else None
@@ -89,6 +115,26 @@ class DistributedQuantizer:
             self.idx_rows = torch.empty((self.world, nb), dtype=torch.uint8, device=dev)
             self.idx = torch.empty(nb, dtype=torch.uint8, device=dev)
         self.out = torch.empty(max(d, 1), dtype=torch.float32, device=dev)
+        if exchange == "slices":
+            self._init_slices(seg_off, dev)
+
+    def _init_slices(self, seg_off, dev) -> None:
+        """Layout and buffers of my slice: coordinates [c, c + d_r) of every worker's row."""
+        P, c = self.slice_coords, self.rank * self.slice_coords
+        self.slice_d = d_r = min(max(self.d - c, 0), P)
+        seg = np.asarray([0, self.d] if seg_off is None or len(seg_off) <= 2 else seg_off, dtype=np.int64)
+        j0 = int(np.searchsorted(seg, c, side="right") - 1) if d_r else 0
+        j1 = int(np.searchsorted(seg, c + d_r, side="left")) if d_r else 1      # segments j0 .. j1-1 meet my slice
+        sub = np.clip(seg[j0: j1 + 1] - c, 0, d_r)
+        sub_dev = torch.as_tensor(sub, device=dev) if len(sub) > 2 else None
+        self.slice_layout = self.k.Layout(self.M, d_r, P, self.dtype, sub_dev)
+        self.slice_seg = (j0, j1)
+        self.slice_bytes = self.slice_layout.level_row_bytes(self.fmt)
+        assert self.slice_bytes * self.world == self.local.level_row_bytes(self.fmt)
+        self.lev_recv = torch.empty((self.M_local, self.world, self.slice_bytes), dtype=torch.int8, device=dev)
+        self.out_slice = torch.zeros(P, dtype=torch.float32, device=dev)
+        self.out = self.out_all = torch.empty(self.world * P, dtype=torch.float32, device=dev)
+        self.lev_all = None
 
     # the three exchanges ------------------------------------------------------------------------
     def agree_scale(self, g: torch.Tensor) -> None:
@@ -113,6 +159,8 @@ class DistributedQuantizer:
     def exchange_and_reconstruct(self) -> None:
         """Algorithm 1 / 2 lines "AllReduce gradients" and "Reconstruct gradient": the level rows of
         all processes are gathered as they are on the wire, summed and reconstructed in one kernel."""
+        if self.exchange == "slices":
+            return self._exchange_slices()
         if self.pull_levels:
             dist.all_reduce(self._flag, group=self.group)          # every process has finished its encoder
             self.k.uq_decode_rows(self.total, self.peer_rows, self.fmt, self.W, self.s, self.scales, self.idx,
@@ -122,6 +170,21 @@ class DistributedQuantizer:
         dist.all_gather_into_tensor(self.lev_all.view(-1), self.lev_local.view(-1), group=self.group)
         self.k.uq_decode(self.total, self.lev_all, self.k.UQ_SRC_LEVELS, self.fmt, self.W, self.s, self.scales,
                          self.idx, self.idx_bits, self.out, None)
+
+    def _exchange_slices(self) -> None:
+        """Slice r of every level row goes to process r (one all-to-all per local worker: a row is
+        already laid out slice after slice), process r reconstructs slice r from all M rows, and the
+        slices are gathered.  The received rows are in (local worker, sender) order, which the
+        integer sum does not see."""
+        for m in range(self.M_local):
+            dist.all_to_all_single(self.lev_recv[m].view(-1), self.lev_local[m], group=self.group)
+        if self.slice_d > 0:
+            j0, j1 = self.slice_seg
+            c = self.rank * self.slice_coords
+            idx = None if self.idx is None else self.idx[c * self.idx_bits // 8:]
+            self.k.uq_decode(self.slice_layout, self.lev_recv.view(self.M, self.slice_bytes), self.k.UQ_SRC_LEVELS,
+                             self.fmt, self.W[j0:j1], self.s, self.scales, idx, self.idx_bits, self.out_slice, None)
+        dist.all_gather_into_tensor(self.out_all, self.out_slice, group=self.group)
 
     def step(self, g: torch.Tensor, seed: int = 0) -> torch.Tensor:
         """g: [M_local, stride] gradients of my workers -> the average gradient of the job [d]."""
@@ -135,7 +198,10 @@ class DistributedQuantizer:
     def wire_bytes_per_step(self) -> int:
         """Bytes this process receives from the others in one step."""
         others = self.world - 1
-        n = others * self.lev_local.numel() + (self.W.numel() * 4 if others else 0)
+        if self.exchange == "slices":
+            n = others * (self.M_local * self.slice_bytes + 4 * self.slice_coords) + (self.W.numel() * 4 if others else 0)
+        else:
+            n = others * self.lev_local.numel() + (self.W.numel() * 4 if others else 0)
         if self.multi:
             n += others * self.idx_local.numel()
         return n

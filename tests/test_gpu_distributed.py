@@ -129,6 +129,52 @@ def test_decode_over_separate_rows(name, d, M):
         B.uq_decode_rows(q.layout, [rows[0].data_ptr()], q.fmt, q.W, q.s, q.scales, q.idx, q.idx_bits, out[8: 8 + d])
 
 
+@pytest.mark.parametrize("name,d,M,R,kw", [
+    ("c2", 300_007, 8, 4, {}), ("c3", 300_007, 6, 3, {}), ("c5", 200_003, 8, 8, {}), ("c4", 100_003, 16, 2, {}),
+    ("c3", 1000, 4, 4, dict(fmt="i2x4", s=1, scales=(1, 16, 256), idx_bits=2)), ("c3", 150_001, 4, 2, dict(idx_bits=8)),
+    ("c2", 200, 2, 2, dict(scales=None)),
+])
+def test_slice_exchange_replayed_rank_by_rank(name, d, M, R, kw):
+    """The reduce-scatter form of the last exchange with the real kernels: the rows are cut into R
+    slices, 'rank' r reconstructs slice r from all M rows with the slice's own layout (segment table
+    counted from the slice's start, the matching part of W and of the index; rows handed over in
+    (local worker, sender) order as the all-to-all delivers them), and the slices side by side are
+    the single-process result."""
+    from paper_2109_12497_b200.distributed import SLICE_ALIGN
+    kw = {k: v for k, v in kw.items() if v is not None}
+    w = wl.scaled(name, d, M=M, **kw)
+    g_np = wl.generate(w)
+    one = run_gpu(w, g_np)
+    q = one["q"]
+    P = max(1, -(-d // (R * SLICE_ALIGN))) * SLICE_ALIGN
+    stride, shift, M_local = R * P, FMT[w.fmt], M // R
+    seg = np.asarray(wl.segment_offsets(w), dtype=np.int64)
+    sb = P >> shift
+    lev = torch.zeros((M, stride >> shift), dtype=torch.int8, device="cuda")        # the rows at the padded stride
+    lev[:, : q.lev.shape[1]] = q.lev
+    idx = None
+    if q.multi:
+        idx = torch.zeros(stride * w.idx_bits // 8, dtype=torch.uint8, device="cuda")
+        idx[: q.idx.numel()] = q.idx
+    out = torch.zeros(R * P, device="cuda")
+    for r in range(R):
+        c = r * P
+        d_r = min(max(d - c, 0), P)
+        if d_r == 0:
+            continue
+        j0 = int(np.searchsorted(seg, c, side="right") - 1)
+        j1 = int(np.searchsorted(seg, c + d_r, side="left"))
+        sub = np.clip(seg[j0: j1 + 1] - c, 0, d_r)
+        lay = B.Layout(M, d_r, P, q.layout.dtype, torch.from_numpy(sub).cuda() if len(sub) > 2 else None)
+        # what the all-to-alls deliver to rank r: [local worker][sender][slice bytes]
+        recv = lev.view(R, M_local, R, sb)[:, :, r, :].permute(1, 0, 2).contiguous().view(M, sb)
+        B.uq_decode(lay, recv, B.UQ_SRC_LEVELS, q.fmt, q.W[j0:j1], q.s, q.scales,
+                    None if idx is None else idx[c * w.idx_bits // 8:], q.idx_bits, out[c: c + P])
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy()[:d], one["out"])
+    assert (out.cpu().numpy()[d:] == 0).all()
+
+
 def test_worker_number_is_validated():
     with pytest.raises(B.UqError):
         lay = B.Layout(2, 100, 128, torch.float32, None, worker0=-1)
@@ -164,5 +210,14 @@ def test_distributed_quantizer_on_one_rank_equals_the_pipeline():
             for _ in range(2):
                 got = qp.step(to_device(w, g_np), w.seed).cpu().numpy()
                 assert np.array_equal(got, run_gpu(w, g_np)["out"]) and int(qp.status.item()) == 0
+            # and the reduce-scatter / all-gather form (rows padded to its stride)
+            qs = DistributedQuantizer(
+                w.M, w.d, torch.float32, seg_off=wl.segment_offsets(w), s=w.s,
+                scales=list(w.scales) if w.quantizer == "multi" else None, fmt=FMT[w.fmt], idx_bits=w.idx_bits,
+                norm=B.UQ_NORM_L2, rng_bits=w.rng_bits, exchange="slices")
+            g_pad = torch.zeros((w.M, qs.stride), device="cuda")
+            g_pad[:, : g_np.shape[1]] = to_device(w, g_np)
+            got = qs.step(g_pad, w.seed).cpu().numpy()
+            assert np.array_equal(got, run_gpu(w, g_np)["out"]) and int(qs.status.item()) == 0
     finally:
         dist.destroy_process_group()
