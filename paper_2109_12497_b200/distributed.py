@@ -28,8 +28,9 @@ the bytes per process constant as the job grows: the coordinates are cut into ``
 equal length, an all-to-all hands process r every worker's levels of slice r (still in their wire
 format), process r sums and reconstructs its slice (``uq_decode`` on the slice's layout: its own
 segment table counted from the slice's start, the matching part of W and of the index), and an
-all-gather of the reconstructed slices gives every process the whole average.  Received per process
-and step: (world_size - 1) / world_size * (M_local * d * bits / 8 + 4 * d) bytes, against
+all-gather of the reconstructed slices gives every process the whole average (the packed scale
+indices are shared the same way: slices exchanged, ``uq_index_min`` on my slice, slices gathered).
+Received per process and step: (world_size - 1) / world_size * (M_local * d * bits / 8 + 4 * d) bytes, against
 (world_size - 1) * M_local * d * bits / 8 for the gather of whole rows; fewer from world_size 6 on
 for 8-bit levels and one worker per process.  Integer sums do not depend on the order of the rows,
 so the result is again bit for bit the single-process one.  Rows are padded to a multiple of
@@ -134,6 +135,8 @@ class DistributedQuantizer:
         self.lev_recv = torch.empty((self.M_local, self.world, self.slice_bytes), dtype=torch.int8, device=dev)
         self.out_slice = torch.zeros(P, dtype=torch.float32, device=dev)
         self.out = self.out_all = torch.empty(self.world * P, dtype=torch.float32, device=dev)
+        if self.multi:
+            self.idx_slice = torch.empty(P * self.idx_bits // 8, dtype=torch.uint8, device=dev)
         self.lev_all = None
 
     # the three exchanges ------------------------------------------------------------------------
@@ -145,6 +148,14 @@ class DistributedQuantizer:
     def share_scale_index(self, g: torch.Tensor) -> None:
         """Algorithm 2 lines "Compute coordinate scales" and "Scale sharing"."""
         self.k.uq_select_scale_multi(self.local, g, self.W, self.scales, self.idx_bits, self.idx_local, self.status)
+        if self.exchange == "slices":          # the same in reduce-scatter / all-gather form: my slice from everyone,
+            nb = self.slice_coords * self.idx_bits // 8                                  # its minimum to everyone
+            dist.all_to_all_single(self.idx_rows.view(-1)[: self.world * nb], self.idx_local[: self.world * nb],
+                                   group=self.group)
+            rows = self.idx_rows.view(-1)[: self.world * nb].view(self.world, nb)
+            self.k.uq_index_min(rows, self.idx_bits, self.idx_slice)
+            dist.all_gather_into_tensor(self.idx[: self.world * nb], self.idx_slice, group=self.group)
+            return
         dist.all_gather_into_tensor(self.idx_rows.view(-1), self.idx_local, group=self.group)
         self.k.uq_index_min(self.idx_rows, self.idx_bits, self.idx)
 
@@ -202,6 +213,8 @@ class DistributedQuantizer:
             n = others * (self.M_local * self.slice_bytes + 4 * self.slice_coords) + (self.W.numel() * 4 if others else 0)
         else:
             n = others * self.lev_local.numel() + (self.W.numel() * 4 if others else 0)
-        if self.multi:
+        if self.multi and self.exchange == "slices":
+            n += 2 * others * self.idx_slice.numel()
+        elif self.multi:
             n += others * self.idx_local.numel()
         return n
