@@ -177,14 +177,41 @@ def time_device_resident(q, g, w, steps, warmup, barrier):
     e1.record(st)
     torch.cuda.synchronize(); barrier()
     total_ms = e0.elapsed_time(e1)
-    n = min(steps, 10)
+    # Under continuous load the board reaches its power cap after some 40 ms and every kernel slows by
+    # 8-14 % (see time_sustained).  The copy that defines the HBM peak was timed as a burst, so the
+    # per-stage pass is kept a burst too: the device idles first, and the pass stays below 40 ms.
+    n = max(3, min(steps, 10, int(40.0 / max(total_ms / steps, 1e-3))))
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(stages) + 1)] for _ in range(n)]
+    time.sleep(BURST_IDLE_S)
+    run_stages(q, g, w.seed)
     for k in range(n):
         run_stages(q, g, w.seed + k, evs[k])
     torch.cuda.synchronize()
     per_stage = {s: statistics.median(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(n))
                  for i, s in enumerate(stages)}
     return total_ms / steps, per_stage
+
+
+BURST_IDLE_S = 0.5          # idle time after which the power budget of a burst is available again (measured)
+
+
+def time_sustained(q, g, w, ms_burst, lead_s=0.6, span_s=0.4):
+    """ms per step under continuous load: steps back to back for lead_s seconds untimed, then span_s
+    seconds timed.  On a B200 at its 1000 W cap this is 8-14 % above the burst figure."""
+    import torch
+    st = torch.cuda.current_stream()
+    n_lead = max(1, int(lead_s * 1e3 / ms_burst))
+    n_span = max(1, int(span_s * 1e3 / ms_burst))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    for k in range(n_lead):
+        q.step(g, w.seed + k)
+    e0.record(st)
+    for k in range(n_span):
+        q.step(g, w.seed + k)
+    e1.record(st)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / n_span, n_lead, n_span
 
 
 def time_end_to_end(q, g_host, out_host, g_dev, w, steps, warmup, barrier):
@@ -385,7 +412,7 @@ def resolve_workload(name, d=None, rng_bits=None):
     return w
 
 
-def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=False, randk_K=0):
+def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=False, randk_K=0, sustained=False):
     """Times one workload on the current device.  Returns a dict of raw numbers."""
     import torch
     from paper_2109_12497_b200.pipeline import from_workload
@@ -404,7 +431,7 @@ def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=F
         g_dev[m].copy_(g_host[m])
     torch.cuda.synchronize()
 
-    res = {"workload": w, "q": q}
+    res = {"workload": w, "q": q, "g_dev": g_dev}
     if flush_between:
         # working set smaller than L2: time each step alone after overwriting L2
         flush = l2_flush_buffer()
@@ -425,6 +452,7 @@ def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=F
         del flush
         res["ms_graph"] = time_graph_replay(q, g_dev, w, max(steps, 20))
     res["ms"], res["stages_ms"] = time_device_resident(q, g_dev, w, steps, warmup, barrier)
+    time.sleep(BURST_IDLE_S)
     res["encode_other_ms"] = time_encode_other_mode(q, g_dev, w, min(steps, 10))
     res["update_ms"] = time_fused_update(q, w, min(steps, 10))
     if q.multi:
@@ -438,8 +466,18 @@ def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=F
         res["e2e_ms"] = time_end_to_end(q, g_host, out_host, g_dev, w, steps, warmup, barrier)
         res["h2d"] = g_host.numel() * g_host.element_size()
         res["d2h"] = out_host.numel() * 4
+    if sustained:
+        res["sustained"] = time_sustained(q, g_dev, w, res["ms"])
+        time.sleep(BURST_IDLE_S)
     res["status"] = q.status_bits()
     return res
+
+
+def sustained_summary(w, timing):
+    ms, n_lead, n_span = timing
+    return {"ms_per_step": round(ms, 5), "gradient_GBps": round(w.in_bytes / ms / 1e6, 1),
+            "steps_before": n_lead, "steps_timed": n_span,
+            "note": "steps back to back for 0.6 s untimed, then 0.4 s timed: the rate at the board's power cap"}
 
 
 def summarize(res, peak_gbs):
@@ -469,6 +507,8 @@ def summarize(res, peak_gbs):
         "ms": round(ms, 5), "algorithmic_MB": round(upd_bytes / 1e6, 2), "GBps": round(upd_bytes / ms / 1e6, 1),
         "frac_of_hbm_peak": round(upd_bytes / ms / 1e6 / peak_gbs, 4),
         "note": "fused SGD-momentum update, timed alone, not part of the step"}
+    if "sustained" in res:
+        out["sustained"] = sustained_summary(w, res["sustained"])
     if "ms_cold" in res:
         out["cold_l2"] = {"ms_per_step": res["ms_cold"], "gradient_GBps": w.in_bytes / res["ms_cold"] / 1e6,
                           "kernels_ms": {s: round(v, 5) for s, v in res["stages_cold_ms"].items()}}
@@ -554,6 +594,7 @@ def gpu_main(args):
     res = bench_workload(w, args.steps, args.warmup, barrier, threads, want_e2e=not args.no_e2e,
                          randk_K=0 if args.no_extra else 10_000)
     clocks = sampler.stop()
+    sustained = time_sustained(res["q"], res["g_dev"], w, res["ms"])     # after the clock record of the timed runs
 
     ms, e2e_ms = max_over_ranks([res["ms"], res["e2e_ms"] or float("nan")], "cuda")
     summ = summarize(res, peak)
@@ -587,6 +628,7 @@ def gpu_main(args):
             "traffic": NCU_TRAFFIC_BYTES.get(name) if args.d is None and dom == "encode" else None,
         },
         "kernels": summ["kernels"],
+        "sustained": sustained_summary(w, sustained),
     }
     if "randk" in res:
         line["global_randk"] = res["randk"]
@@ -610,7 +652,7 @@ def gpu_main(args):
                 torch.cuda.empty_cache()
                 small = wo.in_bytes < (126 << 20)
                 res = bench_workload(wo, max(3, min(args.steps, 10)), 3, lambda: None, threads,
-                                     want_e2e=False, flush_between=small)
+                                     want_e2e=False, flush_between=small, sustained=True)
                 q = res["q"]
                 extra[other] = summarize(res, peak)
                 extra[other]["status_word"] = res["status"]
