@@ -61,20 +61,10 @@ __device__ __forceinline__ void quantize_unit_words(const float (&v)[8], const f
         const uint4 r = rw.r[0];
         const uint32_t w[4] = { r.x, r.y, r.z, r.w };
 #pragma unroll
-#ifdef UQ_DRAW16_NOT
-        // 0xFFFF - h is the 16-bit complement of h: one complement per word, then the odd
-        // coordinate's term is a shift that can ride on the add
-        for (int e = 0; e < 8; ++e) {
-            const uint32_t nw = ~w[e >> 1];
-            const uint32_t x = __float_as_uint(__fadd_rn(scaled_magnitude(v[e], inv[e], cap), 128.0f));
-            z[e] = (e & 1) ? x + (nw >> 16) : x + (nw & 0xFFFFu);
-        }
-#else
         for (int e = 0; e < 8; ++e) {
             const uint32_t h = (e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu);
             z[e] = level_draw16(scaled_magnitude(v[e], inv[e], cap), h);
         }
-#endif
     }
     const uint32_t lo = negate_bytes(gather_bytes<LB>(z[0], z[1], z[2], z[3]), neg_lo);
     const uint32_t hi = negate_bytes(gather_bytes<LB>(z[4], z[5], z[6], z[7]), neg_hi);
