@@ -192,6 +192,7 @@ def time_device_resident(q, g, w, steps, warmup, barrier):
     return total_ms / steps, per_stage
 
 
+NOMINAL_HBM_GBS = 8000.0    # the data-sheet figure, reported beside the measured copy rate for context
 BURST_IDLE_S = 0.5          # idle time after which the power budget of a burst is available again (measured)
 
 
@@ -487,7 +488,8 @@ def summarize(res, peak_gbs):
     for s, ms in res["stages_ms"].items():
         gbs = ab[s] / ms / 1e6
         out["kernels"][s] = {"ms": round(ms, 5), "algorithmic_MB": round(ab[s] / 1e6, 2),
-                             "GBps": round(gbs, 1), "frac_of_hbm_peak": round(gbs / peak_gbs, 4)}
+                             "GBps": round(gbs, 1), "frac_of_hbm_peak": round(gbs / peak_gbs, 4),
+                             "frac_of_nominal_8TBps": round(gbs / NOMINAL_HBM_GBS, 4)}
     other = 32 if w.rng_bits == 16 else 16
     ms = res["encode_other_ms"]
     out["kernels"][f"encode_rng{other}"] = {
@@ -623,6 +625,7 @@ def gpu_main(args):
         "roofline": {
             "bound": "hbm", "kernel": dom, "achieved": round(dom_gbs, 1), "peak": peak, "unit": "GB/s",
             "frac": round(dom_gbs / peak, 4), "peak_kind": f"of {peak_kind}",
+            "frac_of_nominal_8TBps": round(dom_gbs / NOMINAL_HBM_GBS, 4),
             "algorithmic_bytes_per_launch": int(ab[dom]),
             "avg_launch_ms": round(res["stages_ms"][dom], 5),
             "traffic": NCU_TRAFFIC_BYTES.get(name) if args.d is None and dom == "encode" else None,
@@ -659,6 +662,9 @@ def gpu_main(args):
             line["other_workloads"] = extra
         if not args.no_cpu:
             line["cpu_baseline"] = cpu_baseline(name, max(1, os.cpu_count() or 1), args.cpu_coords)
+            one = cpu_baseline(name, 1, max(1, min(w.d, args.cpu_coords) // 8))      # one thread, an eighth of the sample
+            line["cpu_baseline"]["single_thread"] = {"value": one["value"], "unit": UNIT, "sample": one["sample"],
+                                                     "seconds": one["seconds"]}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
