@@ -183,7 +183,7 @@ def time_device_resident(q, g, w, steps, warmup, barrier):
     n = max(3, min(steps, 10, int(40.0 / max(total_ms / steps, 1e-3))))
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(stages) + 1)] for _ in range(n)]
     time.sleep(BURST_IDLE_S)
-    run_stages(q, g, w.seed)
+    run_stages(q, g, w.seed, [torch.cuda.Event() for _ in range(len(stages) + 1)])      # the separate calls, untimed
     for k in range(n):
         run_stages(q, g, w.seed + k, evs[k])
     torch.cuda.synchronize()
@@ -443,13 +443,19 @@ def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=F
         for k in range(steps):
             flush.fill_(k & 0xFF)
             evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(stages) + 1)]
-            run_stages(q, g_dev, w.seed + k, evs)
+            if q.one_kernel:                      # the step is one kernel: nothing to time inside it
+                evs[0].record()
+                q.step(g_dev, w.seed + k)
+                evs[-1].record()
+            else:
+                run_stages(q, g_dev, w.seed + k, evs)
             torch.cuda.synchronize()
             tot.append(evs[0].elapsed_time(evs[-1]))
             for i, s in enumerate(stages):
-                per[s].append(evs[i].elapsed_time(evs[i + 1]))
+                if not q.one_kernel:
+                    per[s].append(evs[i].elapsed_time(evs[i + 1]))
         res["ms_cold"] = statistics.fmean(tot)
-        res["stages_cold_ms"] = {s: statistics.fmean(v) for s, v in per.items()}
+        res["stages_cold_ms"] = {s: statistics.fmean(v) for s, v in per.items() if v}
         del flush
         res["ms_graph"] = time_graph_replay(q, g_dev, w, max(steps, 20))
     res["ms"], res["stages_ms"] = time_device_resident(q, g_dev, w, steps, warmup, barrier)
@@ -485,6 +491,9 @@ def summarize(res, peak_gbs):
     w = res["workload"]
     ab = algorithmic_bytes(w)
     out = {"gradient_GBps": w.in_bytes / res["ms"] / 1e6, "ms_per_step": res["ms"], "kernels": {}}
+    if res["q"].one_kernel:
+        out["step_form"] = ("one cooperative kernel (uq_step_small): ms_per_step is that kernel; the entries under "
+                            "kernels are the separate calls, timed one by one for comparison")
     for s, ms in res["stages_ms"].items():
         gbs = ab[s] / ms / 1e6
         out["kernels"][s] = {"ms": round(ms, 5), "algorithmic_MB": round(ab[s] / 1e6, 2),

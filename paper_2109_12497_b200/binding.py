@@ -22,11 +22,14 @@ UQ_NORM_LINF, UQ_NORM_L2 = 0, 2
 UQ_FMT_I8, UQ_FMT_I4X2, UQ_FMT_I2X4, UQ_FMT_I6P = 0, 1, 2, 3
 UQ_SRC_LEVELS, UQ_SRC_SUMS = 0, 1
 UQ_STATUS_NONFINITE, UQ_STATUS_BAD_SEGMENTS, UQ_STATUS_SCALE_OVERFLOW, UQ_STATUS_BAD_INDEX = 1, 2, 4, 8
+UQ_STATUS_TIMEOUT = 16
 
 EXPORTS = (
     "uq_version", "uq_last_cuda_error", "uq_error_string", "uq_workspace_bytes", "uq_index_bytes", "uq_workspace_bytes_amax",
+    "uq_workspace_bytes_small",
     "uq_agree_scale", "uq_agree_scale_static", "uq_encode_single", "uq_select_scale_multi", "uq_encode_multi",
     "uq_aggregate", "uq_decode", "uq_decode_update", "uq_randk_gather", "uq_randk_scatter", "uq_randk_update", "uq_index_min", "uq_decode_rows", "uq_select_encode_multi", "uq_agree_scale_amax", "uq_step",
+    "uq_step_small",
 )
 
 
@@ -79,6 +82,9 @@ def lib() -> C.CDLL:
         L.uq_agree_scale.argtypes = [LP, P, I, P, P, P, SZ, P]
         L.uq_step.argtypes = [LP, P, I, I, P, I, I, U64, I, I, P, P, P, P, P, P, P, SZ, P]
         L.uq_agree_scale_amax.argtypes = [LP, P, I, P, P, P, P, SZ, P]
+        L.uq_step_small.argtypes = [LP, P, I, I, U64, I, I, P, P, P, P, P, P, SZ, P]
+        L.uq_workspace_bytes_small.restype = SZ
+        L.uq_workspace_bytes_small.argtypes = []
         L.uq_agree_scale_static.argtypes = [LP, P, I, P, P, P]
         L.uq_encode_single.argtypes = [LP, P, P, I, U64, I, I, P, P, P]
         L.uq_select_scale_multi.argtypes = [LP, P, P, P, I, I, P, P, P]
@@ -94,7 +100,7 @@ def lib() -> C.CDLL:
         L.uq_randk_gather.argtypes = [LP, P, I64, U64, P, P, I64, P, P]
         L.uq_randk_scatter.argtypes = [I64, I64, P, P, P, P, P]
         L.uq_randk_update.argtypes = [I64, I64, P, P, P, F, P, P]
-        for name in EXPORTS[6:]:
+        for name in EXPORTS[7:]:
             getattr(L, name).restype = I
         _lib = L
     return _lib
@@ -393,3 +399,32 @@ def uq_step(layout: Layout, g: torch.Tensor, norm: int, s: int, scales: Optional
         layout.ref(), _ptr(g), norm, s, arr, N, idx_bits, seed, rng_bits, fmt, _ptr(W),
         _ptr(idx) if scales is not None else None, _ptr(lev), _ptr(out), _ptr(S_opt), _ptr(status), _ptr(workspace),
         workspace.numel() * workspace.element_size(), _stream()))
+
+
+SMALL_STEP_MAX_WORKERS = 8
+
+
+def uq_workspace_bytes_small() -> int:
+    return int(lib().uq_workspace_bytes_small())
+
+
+def small_step_supported(layout: Layout, fmt: int, multi: bool) -> bool:
+    """Whether uq_step_small takes this configuration (single-scale, one segment, M <= 8, one-plane levels)."""
+    return (not multi and layout.nseg == 1 and layout.M <= SMALL_STEP_MAX_WORKERS
+            and fmt in (UQ_FMT_I8, UQ_FMT_I4X2, UQ_FMT_I2X4))
+
+
+def uq_step_small(layout: Layout, g: torch.Tensor, norm: int, s: int, seed: int, rng_bits: int, fmt: int,
+                  W: torch.Tensor, lev: torch.Tensor, out: torch.Tensor, S_opt: Optional[torch.Tensor],
+                  status: Optional[torch.Tensor], workspace: torch.Tensor) -> None:
+    """The whole single-scale step as one cooperative kernel (small gradients).  ``workspace``:
+    zero-filled before its first use (the kernel leaves its counters zero), one call at a time."""
+    layout.check_g(g)
+    layout.check_lev(lev, fmt)
+    layout.check_vec(W, torch.float32, 1, "W")
+    layout.check_vec(out, torch.float32, layout.d, "out")
+    if S_opt is not None:
+        layout.check_vec(S_opt, torch.int32, layout.d, "S_opt")
+    _check("uq_step_small", lib().uq_step_small(
+        layout.ref(), _ptr(g), norm, s, seed, rng_bits, fmt, _ptr(W), _ptr(lev), _ptr(out), _ptr(S_opt), _ptr(status),
+        _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()))

@@ -32,6 +32,11 @@ cudaError_t launch_randk_gather(const uq_layout &L, const void *g, int64_t K, ui
                                 void *gk, int64_t gk_stride, uint32_t *status, cudaStream_t st);
 cudaError_t launch_randk_scatter(int64_t d, int64_t K, const int64_t *sel, const float *vals, float *dst, bool update,
                                  float lr, uint32_t *status, cudaStream_t st);
+bool small_step_supported(const uq_layout &L, int fmt);
+size_t small_workspace_bytes();
+cudaError_t launch_small_step(const uq_layout &L, const void *g, int norm, int s, uint64_t seed, int rng_bits, int fmt,
+                              float *W, void *lev, float *out, int32_t *S, uint32_t *status, void *workspace,
+                              cudaStream_t st);
 }  // namespace uq
 
 namespace {
@@ -307,6 +312,27 @@ int uq_step(const uq_layout *L, const void *g, int norm, int s, const int32_t *s
     }
     if (rc != UQ_OK) return rc;
     return uq_decode(L, lev, UQ_SRC_LEVELS, fmt, W, s, scales, N, idx, idx_bits, out, S_opt, stream);
+}
+
+size_t uq_workspace_bytes_small(void) { return uq::small_workspace_bytes(); }
+
+int uq_step_small(const uq_layout *L, const void *g, int norm, int s, uint64_t seed, int rng_bits, int fmt, float *W,
+                  void *lev, float *out, int32_t *S_opt, uint32_t *status, void *workspace, size_t workspace_bytes,
+                  void *stream)
+{
+    if (!layout_ok(L) || W == nullptr || !aligned(W, 4) || !aligned(status, 4)) return UQ_ERR_BAD_ARG;
+    if (norm != UQ_NORM_L2 && norm != UQ_NORM_LINF) return UQ_ERR_BAD_ARG;
+    if (!fmt_ok(fmt, s) || (rng_bits != 32 && rng_bits != 16)) return UQ_ERR_BAD_ARG;
+    if (L->d > 0 && (g == nullptr || lev == nullptr || out == nullptr || !aligned(g, 16) || !aligned(lev, 16) ||
+                     !aligned(out, 32) || !aligned(S_opt, 32)))
+        return UQ_ERR_BAD_ARG;
+    if (!uq::small_step_supported(*L, fmt)) return UQ_ERR_UNSUPPORTED;
+    if (workspace == nullptr || !aligned(workspace, 8) || workspace_bytes < uq_workspace_bytes_small())
+        return UQ_ERR_WORKSPACE;
+    const cudaError_t e = uq::launch_small_step(*L, g, norm, s, seed, rng_bits, fmt, W, lev, out, S_opt, status, workspace,
+                                                (cudaStream_t)stream);
+    if (e == cudaErrorNotSupported) return UQ_ERR_UNSUPPORTED;
+    return finish(e);
 }
 
 int uq_index_min(const uint8_t *rows, int R, int64_t row_bytes, int64_t nbytes, int idx_bits, uint8_t *idx, void *stream)

@@ -45,10 +45,11 @@ __device__ __forceinline__ UnitWords<RNG> unit_words(const PhiloxKey &key, uint3
     return w;
 }
 
-template <int FMT, int RNG>
-__device__ __forceinline__ void quantize_unit_words(const float (&v)[8], const float (&inv)[8], float cap,
+// The signed levels of a unit as bytes: coordinates 0..3 in `lo`, 4..7 in `hi`.
+template <int RNG>
+__device__ __forceinline__ void quantize_unit_bytes(const float (&v)[8], const float (&inv)[8], float cap,
                                                     uint32_t neg_lo, uint32_t neg_hi, const UnitWords<RNG> &rw,
-                                                    void *dst, void *dst2, bool store = true)
+                                                    uint32_t &lo, uint32_t &hi)
 {
     constexpr uint32_t LB = RNG == 32 ? kLevelByte23 : kLevelByte16;
     uint32_t z[8];
@@ -66,9 +67,13 @@ __device__ __forceinline__ void quantize_unit_words(const float (&v)[8], const f
             z[e] = level_draw16(scaled_magnitude(v[e], inv[e], cap), h);
         }
     }
-    const uint32_t lo = negate_bytes(gather_bytes<LB>(z[0], z[1], z[2], z[3]), neg_lo);
-    const uint32_t hi = negate_bytes(gather_bytes<LB>(z[4], z[5], z[6], z[7]), neg_hi);
-    if (!store) return;
+    lo = negate_bytes(gather_bytes<LB>(z[0], z[1], z[2], z[3]), neg_lo);
+    hi = negate_bytes(gather_bytes<LB>(z[4], z[5], z[6], z[7]), neg_hi);
+}
+
+// The level bytes of a unit packed into the wire format and stored.
+template <int FMT> __device__ __forceinline__ void store_unit(uint32_t lo, uint32_t hi, void *dst, void *dst2)
+{
     // plain stores (not evict-first ones): the aggregation kernel that follows reads the levels
     // back, and what is still in L2 then costs no DRAM read (measured: 7-9 % off that kernel)
     if (FMT == UQ_FMT_I8) *(uint2 *)dst = make_uint2(lo, hi);
@@ -78,6 +83,16 @@ __device__ __forceinline__ void quantize_unit_words(const float (&v)[8], const f
         *(uint32_t *)dst = bytes_to_nibbles(lo, hi);
         *(unsigned short *)dst2 = (unsigned short)bytes_to_crumbs(lo >> 4, hi >> 4);
     }
+}
+
+template <int FMT, int RNG>
+__device__ __forceinline__ void quantize_unit_words(const float (&v)[8], const float (&inv)[8], float cap,
+                                                    uint32_t neg_lo, uint32_t neg_hi, const UnitWords<RNG> &rw,
+                                                    void *dst, void *dst2, bool store = true)
+{
+    uint32_t lo, hi;
+    quantize_unit_bytes<RNG>(v, inv, cap, neg_lo, neg_hi, rw, lo, hi);
+    if (store) store_unit<FMT>(lo, hi, dst, dst2);
 }
 
 template <int FMT, int RNG>

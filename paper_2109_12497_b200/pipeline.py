@@ -15,12 +15,16 @@ import torch
 from . import binding as B
 
 
+ONE_KERNEL_MAX_BYTES = 8 << 20      # gradients of all workers up to this size take the one-kernel step
+
+
 class Quantizer:
     def __init__(self, M: int, d: int, dtype: torch.dtype = torch.float32,
                  seg_off: Optional[Sequence[int]] = None, s: int = 127,
                  scales: Optional[Sequence[int]] = None, fmt: int = B.UQ_FMT_I8, idx_bits: int = 0,
                  norm: int = B.UQ_NORM_L2, rng_bits: int = 32, keep_sums: bool = False,
-                 device: str | torch.device = "cuda", fused_select: bool = False, amax_select: bool = False):
+                 device: str | torch.device = "cuda", fused_select: bool = False, amax_select: bool = False,
+                 one_kernel: Optional[bool] = None):
         B.lib()                                     # fail now if the CUDA library is not built
         dev = torch.device(device)
         self.M, self.d, self.dtype = M, d, dtype
@@ -43,7 +47,16 @@ class Quantizer:
         nseg = self.layout.nseg
         self.W = torch.zeros(nseg, dtype=torch.float32, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
-        self.workspace = torch.empty(max(8, self.layout.workspace_bytes(), self.layout.workspace_bytes_amax()),
+        # single-scale, one segment, few workers, and so small that the step is bound by its five
+        # launches: the whole step as one cooperative kernel (uq_step_small).  None = decide by size.
+        fits = B.small_step_supported(self.layout, fmt, self.multi)
+        if one_kernel and not fits:
+            raise ValueError("uq: the one-kernel step takes the single-scale quantizer, one segment, M <= 8")
+        self.one_kernel = fits and (one_kernel if one_kernel is not None
+                                    else M * d * (4 if dtype == torch.float32 else 2) <= ONE_KERNEL_MAX_BYTES)
+        # zeroed: the one-kernel step wants its counters zero before the first call and leaves them so
+        self.workspace = torch.zeros(max(8, self.layout.workspace_bytes(), self.layout.workspace_bytes_amax(),
+                                         B.uq_workspace_bytes_small() if self.one_kernel else 0),
                                      dtype=torch.uint8, device=dev)
         self.lev = torch.empty((M, self.layout.level_row_bytes(fmt)), dtype=torch.int8, device=dev)
         self.idx = (torch.empty(max(16, self.layout.index_bytes(self.idx_bits)), dtype=torch.uint8, device=dev)
@@ -93,6 +106,10 @@ class Quantizer:
 
     def step(self, g: torch.Tensor, seed: int = 0) -> torch.Tensor:
         """g: [M, stride] gradients of all workers -> the reconstructed average gradient [d]."""
+        if self.one_kernel:
+            B.uq_step_small(self.layout, g, self.norm, self.s, seed, self.rng_bits, self.fmt, self.W, self.lev, self.out,
+                            self.S, self.status, self.workspace)
+            return self.out[: self.d]
         if not (self.fused_select or self.amax_select):      # the plain sequence: one trip through the binding
             B.uq_step(self.layout, g, self.norm, self.s, self.scales, self.idx_bits, seed, self.rng_bits, self.fmt,
                       self.W, self.idx, self.lev, self.out, self.S, self.status, self.workspace)
@@ -109,6 +126,8 @@ class Quantizer:
 
     def kernels_per_step(self) -> int:
         """Kernel launches one step enqueues (norm partials + finalize, [select], encode, decode)."""
+        if self.one_kernel:
+            return 1
         separate_select = self.multi and not self.fused_select and self.d > 0
         return (2 if self.d > 0 else 1) + (1 if separate_select else 0) + (2 if self.d > 0 else 0)
 
@@ -166,7 +185,7 @@ class RandKQuantizer:
 
 
 def from_workload(w, keep_sums: bool = False, device="cuda", fused_select: bool = False,
-                  amax_select: bool = False) -> Quantizer:
+                  amax_select: bool = False, one_kernel: Optional[bool] = None) -> Quantizer:
     """A Quantizer configured like a ``workloads.Workload``."""
     from . import workloads as wl
     seg = wl.segment_offsets(w)
@@ -175,7 +194,7 @@ def from_workload(w, keep_sums: bool = False, device="cuda", fused_select: bool 
         scales=list(w.scales) if w.quantizer == "multi" else None,
         fmt={"i8": B.UQ_FMT_I8, "i4x2": B.UQ_FMT_I4X2, "i2x4": B.UQ_FMT_I2X4, "i6p": B.UQ_FMT_I6P}[w.fmt], idx_bits=w.idx_bits,
         norm=B.UQ_NORM_L2 if w.norm == wl.NORM_L2 else B.UQ_NORM_LINF, rng_bits=w.rng_bits,
-        keep_sums=keep_sums, device=device, fused_select=fused_select, amax_select=amax_select)
+        keep_sums=keep_sums, device=device, fused_select=fused_select, amax_select=amax_select, one_kernel=one_kernel)
 
 
 def randk_from_workload(w, K: int, device="cuda") -> RandKQuantizer:

@@ -23,8 +23,11 @@ def to_device(w, g_np):
 def run_gpu(w, g_np, seed=None, mode="default"):
     """All stage outputs of the CUDA path as numpy arrays.  mode picks the form of the multi-scale
     path: "default" = "rows" (the selector reads all M rows), "amax" (agree-scale writes max_m |g|
-    and the selector runs on that row), "fused" (selection and encoding in one kernel)."""
-    q = from_workload(w, keep_sums=True, fused_select=mode == "fused", amax_select=mode == "amax")
+    and the selector runs on that row), "fused" (selection and encoding in one kernel); of the
+    single-scale path: "one" (the whole step as one cooperative kernel), "separate" (the calls one by
+    one), "default" (the library picks by size)."""
+    one_kernel = {"one": True, "separate": False}.get(mode)       # else: the library decides by size
+    q = from_workload(w, keep_sums=True, fused_select=mode == "fused", amax_select=mode == "amax", one_kernel=one_kernel)
     g = to_device(w, g_np)
     q.step(g, w.seed if seed is None else seed)
     torch.cuda.synchronize()
@@ -79,11 +82,20 @@ def ulp_distance(a, b):
 
 def check_parity(w, g_np, seed=None):
     """Full comparison; returns the GPU result for further checks.  A multi-scale workload runs in
-    all three forms of its path (see run_gpu): each must match the oracle."""
+    all three forms of its path (see run_gpu), a single-scale one that the one-kernel step takes in
+    both of its forms: each must match the oracle."""
     if w.quantizer == "multi":
         _check_parity(w, g_np, seed, "fused")
         _check_parity(w, g_np, seed, "amax")
+    elif one_kernel_takes(w):
+        _check_parity(w, g_np, seed, "one")
+        _check_parity(w, g_np, seed, "separate")
     return _check_parity(w, g_np, seed, "default")
+
+
+def one_kernel_takes(w) -> bool:
+    return (w.quantizer == "single" and len(wl.segment_offsets(w)) == 2 and w.M <= B.SMALL_STEP_MAX_WORKERS
+            and w.fmt in ("i8", "i4x2", "i2x4"))
 
 
 def _check_parity(w, g_np, seed, mode):

@@ -36,7 +36,7 @@ def test_constants_match_the_header():
     for name in ("UQ_OK", "UQ_ERR_BAD_ARG", "UQ_ERR_CUDA", "UQ_ERR_UNSUPPORTED", "UQ_ERR_WORKSPACE",
                  "UQ_F32", "UQ_BF16", "UQ_NORM_LINF", "UQ_NORM_L2", "UQ_FMT_I8", "UQ_FMT_I4X2", "UQ_FMT_I2X4", "UQ_FMT_I6P",
                  "UQ_SRC_LEVELS", "UQ_SRC_SUMS", "UQ_STATUS_NONFINITE", "UQ_STATUS_BAD_SEGMENTS",
-                 "UQ_STATUS_SCALE_OVERFLOW", "UQ_STATUS_BAD_INDEX"):
+                 "UQ_STATUS_SCALE_OVERFLOW", "UQ_STATUS_BAD_INDEX", "UQ_STATUS_TIMEOUT"):
         m = re.search(rf"\b{name}\s*=\s*(\d+)", text)
         assert m and int(m.group(1)) == getattr(B, name), name
 
@@ -103,6 +103,17 @@ def test_later_entry_points_reject_bad_arguments_on_the_host(lib):
                        None) == B.UQ_ERR_BAD_ARG
     assert lib.uq_step(ok, p, B.UQ_NORM_L2, 127, None, 0, 0, 0, 16, B.UQ_FMT_I8, p, None, p, p, None, None, p, 8,
                        None) == B.UQ_ERR_WORKSPACE
+    small = lib.uq_workspace_bytes_small()
+    assert small >= 64 + 148 * 8 * 8 * 8
+    assert lib.uq_step_small(bad, p, B.UQ_NORM_L2, 127, 0, 16, B.UQ_FMT_I8, p, p, p, None, None, p, small, None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_step_small(ok, p, B.UQ_NORM_L2, 128, 0, 16, B.UQ_FMT_I8, p, p, p, None, None, p, small, None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_step_small(ok, p, B.UQ_NORM_L2, 127, 0, 16, B.UQ_FMT_I8, p, p, p + 16, None, None, p, small, None) \
+        == B.UQ_ERR_BAD_ARG                                                                         # out: 32-byte aligned
+    assert lib.uq_step_small(C.byref(_layout(M=9)), p, B.UQ_NORM_L2, 127, 0, 16, B.UQ_FMT_I8, p, p, p, None, None, p, small,
+                             None) == B.UQ_ERR_UNSUPPORTED
+    assert lib.uq_step_small(ok, p, B.UQ_NORM_L2, 31, 0, 16, B.UQ_FMT_I6P, p, p, p, None, None, p, small, None) \
+        == B.UQ_ERR_UNSUPPORTED
+    assert lib.uq_step_small(ok, p, B.UQ_NORM_L2, 127, 0, 16, B.UQ_FMT_I8, p, p, p, None, None, p, 64, None) == B.UQ_ERR_WORKSPACE
     assert lib.uq_agree_scale_amax(bad, p, B.UQ_NORM_L2, p, p, None, p, 1 << 20, None) == B.UQ_ERR_BAD_ARG
     assert lib.uq_agree_scale_amax(ok, p, B.UQ_NORM_L2, p, p + 8, None, p, 1 << 20, None) == B.UQ_ERR_BAD_ARG   # alignment
     assert lib.uq_agree_scale_amax(ok, p, B.UQ_NORM_L2, p, None, None, p, 1 << 20, None) == B.UQ_ERR_BAD_ARG
