@@ -133,7 +133,10 @@ class Quantizer:
 
     def status_bits(self) -> int:
         """Synchronizes and returns the device status word (0 = clean)."""
-        return int(self.status.item())
+        bits = int(self.status.item())
+        if bits & B.UQ_STATUS_TIMEOUT:            # a barrier wait ran out: its counters are not back at zero
+            self.workspace.zero_()
+        return bits
 
 
 class RandKQuantizer:

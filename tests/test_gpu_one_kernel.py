@@ -118,3 +118,25 @@ def test_steps_back_to_back():
     lev = o.encode_single(g_np[:, : w.d], W, w.s, 199, w.rng_bits)
     assert np.array_equal(q.lev.cpu().numpy()[:, : w.d], lev)
     assert np.array_equal(q.S.cpu().numpy()[: w.d], o.aggregate(lev))
+
+
+def test_the_wait_at_the_barrier_is_bounded():
+    """A wait that cannot be satisfied ends by itself: with the arrival counter started just below
+    the wrap of its 32 bits, the CTAs that arrive after the wrap read a count that never reaches the
+    grid size.  They give up after their poll limit (about a second), set UQ_STATUS_TIMEOUT and
+    return; the context stays usable and, with the scratch zeroed again, the next step is right."""
+    w = wl.scaled("c1", 1 << 20, M=2)
+    g_np = wl.generate(w)
+    q = from_workload(w, keep_sums=True, one_kernel=True)
+    g = to_device(w, g_np)
+    q.workspace[:4] = torch.tensor([0xC0, 0xFF, 0xFF, 0xFF], dtype=torch.uint8)     # 2^32 - 64, little endian
+    q.step(g, 0)
+    bits = q.status_bits()                       # synchronizes; zeroes the scratch after a timeout
+    assert bits & B.UQ_STATUS_TIMEOUT
+    assert int(q.workspace[:64].sum().item()) == 0
+    q.status.zero_()
+    _ = q.step(g, w.seed)
+    torch.cuda.synchronize()
+    assert q.status_bits() == 0
+    lev = o.encode_single(g_np[:, : w.d], q.W.cpu().numpy(), w.s, w.seed, w.rng_bits)
+    assert np.array_equal(q.lev.cpu().numpy()[:, : w.d], lev)
