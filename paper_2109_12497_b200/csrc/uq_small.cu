@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(kThreads, 2) small_step_kernel(const __grid_co
     }
 #pragma unroll
     for (int m = 0; m < MW; ++m) {
-        const double w = warp_reduce<NORM>(acc[m].value());
+        const double w = m < p.M ? warp_reduce<NORM>(acc[m].value()) : 0.0;     // uniform: idle workers cost nothing
         if (lane == 0) sh[warp][m] = w;
     }
     __syncthreads();
@@ -120,16 +120,30 @@ __global__ void __launch_bounds__(kThreads, 2) small_step_kernel(const __grid_co
     {
         const int m = tid & (MW - 1), part = tid >> 3;             // 32 strided partial sums per worker
         double a = 0.0;
-        for (unsigned c = part; c < gridDim.x; c += 32) a = combine<NORM>(a, __ldcg(p.part + (size_t)c * MW + m));
+        for (unsigned c0 = part; c0 < gridDim.x; c0 += 32 * 10) {    // ten loads in flight, added in index order
+            double v[10];
+#pragma unroll
+            for (int k = 0; k < 10; ++k) {
+                const unsigned c = c0 + 32u * k;
+                v[k] = c < gridDim.x ? __ldcg(p.part + (size_t)c * MW + m) : 0.0;     // 0 is neutral for both norms
+            }
+#pragma unroll
+            for (int k = 0; k < 10; ++k) a = combine<NORM>(a, v[k]);
+        }
         sh[part][m] = a;
+    }
+    __syncthreads();
+    if (tid < MW) {                                  // thread m: worker m's 32 sums in index order
+        double tot = sh[0][tid];
+        for (int k = 1; k < 32; ++k) tot = combine<NORM>(tot, sh[k][tid]);
+        sh[0][tid] = tot;                            // only thread m touches column m
     }
     __syncthreads();
     if (tid == 0) {
         bool nan = false;
         double top = 0.0;
         for (int m = 0; m < p.M; ++m) {
-            double tot = sh[0][m];
-            for (int k = 1; k < 32; ++k) tot = combine<NORM>(tot, sh[k][m]);
+            const double tot = sh[0][m];
             nan |= tot != tot;
             top = fmax(top, tot);
         }
