@@ -66,6 +66,9 @@ class Quantizer:
             self.layout_amax = B.Layout(1, d, self.stride, dtype, seg_dev)
         self.out = torch.empty(max(d, 1), dtype=torch.float32, device=dev)
         self.S = torch.empty(max(d, 1), dtype=torch.int32, device=dev) if keep_sums else None
+        self._small_call = None
+        self._step_call = None
+        self._out_view = self.out[: self.d]
 
     # the four stages, each one C-ABI call -------------------------------------------------------
     def agree_scale(self, g: torch.Tensor) -> None:
@@ -107,13 +110,37 @@ class Quantizer:
     def step(self, g: torch.Tensor, seed: int = 0) -> torch.Tensor:
         """g: [M, stride] gradients of all workers -> the reconstructed average gradient [d]."""
         if self.one_kernel:
-            B.uq_step_small(self.layout, g, self.norm, self.s, seed, self.rng_bits, self.fmt, self.W, self.lev, self.out,
-                            self.S, self.status, self.workspace)
-            return self.out[: self.d]
+            # every buffer but g is this object's own: their addresses are marshalled once, not per
+            # step (the checked wrapper B.uq_step_small costs about as much host time as the kernel runs)
+            self.layout.check_g(g)
+            if not g.is_cuda:
+                raise ValueError("uq: tensors must live on a CUDA device")
+            if self._small_call is None:
+                ptr = lambda t: None if t is None else t.data_ptr()
+                self._small_call = (B.lib().uq_step_small, self.layout.ref(),
+                                    (ptr(self.W), ptr(self.lev), ptr(self.out), ptr(self.S), ptr(self.status),
+                                     ptr(self.workspace), self.workspace.numel()))
+            fn, ref, tail = self._small_call
+            rc = fn(ref, g.data_ptr(), self.norm, self.s, seed, self.rng_bits, self.fmt, *tail, B._stream())
+            if rc != B.UQ_OK:
+                raise B.UqError("uq_step_small", rc)
+            return self._out_view
         if not (self.fused_select or self.amax_select):      # the plain sequence: one trip through the binding
-            B.uq_step(self.layout, g, self.norm, self.s, self.scales, self.idx_bits, seed, self.rng_bits, self.fmt,
-                      self.W, self.idx, self.lev, self.out, self.S, self.status, self.workspace)
-            return self.out[: self.d]
+            self.layout.check_g(g)
+            if not g.is_cuda:
+                raise ValueError("uq: tensors must live on a CUDA device")
+            if self._step_call is None:                      # addresses of my own buffers, marshalled once
+                ptr = lambda t: None if t is None else t.data_ptr()
+                arr, N = B._scales(self.scales) if self.multi else (None, 0)
+                self._step_call = (B.lib().uq_step, self.layout.ref(), arr, N,
+                                   (ptr(self.W), ptr(self.idx), ptr(self.lev), ptr(self.out), ptr(self.S),
+                                    ptr(self.status), ptr(self.workspace), self.workspace.numel()))
+            fn, ref, arr, N, tail = self._step_call
+            rc = fn(ref, g.data_ptr(), self.norm, self.s, arr, N, self.idx_bits, seed, self.rng_bits, self.fmt, *tail,
+                    B._stream())
+            if rc != B.UQ_OK:
+                raise B.UqError("uq_step", rc)
+            return self._out_view
         self.agree_scale(g)
         if self.multi and self.fused_select:
             self.select_encode(g, seed)
