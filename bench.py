@@ -72,6 +72,15 @@ def algorithmic_bytes(w: wl.Workload) -> dict:
     return b
 
 
+def step_roofline(w: wl.Workload, ms: float, peak_gbs: float) -> dict:
+    """The whole step against the sum of its stages' algorithmic bytes moved at the HBM peak."""
+    ab = algorithmic_bytes(w)
+    total = sum(v for k, v in ab.items() if k != "select_encode")
+    min_ms = total / peak_gbs / 1e6
+    return {"algorithmic_MB": round(total / 1e6, 1), "min_ms_at_peak": round(min_ms, 5), "frac": round(min_ms / ms, 4),
+            "ceiling_gradient_GBps": round(w.in_bytes / min_ms / 1e6, 1)}
+
+
 # ---------------------------------------------------------------------------------------------
 # clocks
 # ---------------------------------------------------------------------------------------------
@@ -490,7 +499,8 @@ def sustained_summary(w, timing):
 def summarize(res, peak_gbs):
     w = res["workload"]
     ab = algorithmic_bytes(w)
-    out = {"gradient_GBps": w.in_bytes / res["ms"] / 1e6, "ms_per_step": res["ms"], "kernels": {}}
+    out = {"gradient_GBps": w.in_bytes / res["ms"] / 1e6, "ms_per_step": res["ms"],
+           "step_roofline": step_roofline(w, res["ms"], peak_gbs), "kernels": {}}
     if res["q"].one_kernel:
         out["step_form"] = ("one cooperative kernel (uq_step_small): ms_per_step is that kernel; the entries under "
                             "kernels are the separate calls, timed one by one for comparison")
@@ -640,6 +650,7 @@ def gpu_main(args):
             "avg_launch_ms": round(res["stages_ms"][dom], 5),
             "traffic": NCU_TRAFFIC_BYTES.get(name) if args.d is None and dom == "encode" else None,
         },
+        "step_roofline": step_roofline(w, ms, peak),
         "kernels": summ["kernels"],
         "sustained": sustained_summary(w, sustained),
     }
