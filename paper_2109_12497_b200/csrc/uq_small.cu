@@ -16,35 +16,9 @@
 // The gradients cross the HBM interface once, the result leaves once.  Levels, sums and the
 // reconstruction are bit for bit those of the separate calls given the same W; W itself is summed
 // in another fixed order (L2: within one unit in the last place of the regular kernel's).
-#include "uq_device.cuh"
-#include "uq_unit.cuh"
-#include "uq_norm.cuh"
+#include "uq_small.cuh"
 
 namespace uq {
-
-constexpr int kSmallMaxWorkers = 8;
-constexpr int kSmallHeader = 64;                  // bytes in front of the partials: arrival and departure counters
-constexpr uint32_t kSmallSpinLimit = 1u << 20;    // polls of the counter before a CTA gives up (about a second)
-
-struct SmallParams {
-    const void *g;
-    void *lev;
-    float *W, *out;
-    int32_t *S;
-    uint32_t *status;
-    uint32_t *counter;        // scratch: [0] arrivals, [1] departures
-    double *part;             // scratch: [gridDim.x][kSmallMaxWorkers]
-    int64_t d, stride, coord0;
-    int32_t M, worker0, s;
-    PhiloxKey key;
-};
-
-__device__ __forceinline__ uint32_t ld_acquire(const uint32_t *p)
-{
-    uint32_t v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
 
 template <int DT, int NORM, int FMT, int RNG>
 __global__ void __launch_bounds__(kThreads, 2) small_step_kernel(const __grid_constant__ SmallParams p)
@@ -52,115 +26,11 @@ __global__ void __launch_bounds__(kThreads, 2) small_step_kernel(const __grid_co
     using E = Elem<DT>;
     using LF = LevelFmt<FMT>;
     constexpr int H = 8 / E::G;
-    constexpr int MW = kSmallMaxWorkers;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x;
     const int64_t nunits = (p.d + 7) >> 3;
     const int64_t u0 = (int64_t)blockIdx.x * kThreads + tid, ustep = (int64_t)gridDim.x * kThreads;
-    __shared__ double sh[32][MW];
-    __shared__ float sh_w;
-    __shared__ int sh_fail;
-
-    // ---- phase 1: per-worker norm partials of my units
-    Acc<NORM> acc[MW];
-    for (int64_t u = u0; u < nunits; u += ustep) {
-        const int64_t i = u << 3;
-        const char *col = (const char *)p.g + (size_t)i * E::BYTES;
-        const int valid = (int)min((int64_t)8, p.d - i);
-#pragma unroll
-        for (int m = 0; m < MW; ++m) {
-            if (m < p.M) {
-                float v[8];
-#pragma unroll
-                for (int h = 0; h < H; ++h)
-                    E::unpack(ld_stream(col + ((size_t)m * (size_t)p.stride + h * E::G) * E::BYTES),
-                              *(float(*)[E::G])(v + h * E::G));
-#pragma unroll
-                for (int e = 0; e < 8; ++e)
-                    if (e < valid) acc[m].add(v[e]);
-            }
-        }
-    }
-#pragma unroll
-    for (int m = 0; m < MW; ++m) {
-        const double w = m < p.M ? warp_reduce<NORM>(acc[m].value()) : 0.0;     // uniform: idle workers cost nothing
-        if (lane == 0) sh[warp][m] = w;
-    }
-    __syncthreads();
-    if (tid < MW) {
-        double tot = sh[0][tid];
-        for (int k = 1; k < kWarps; ++k) tot = combine<NORM>(tot, sh[k][tid]);
-        p.part[(size_t)blockIdx.x * MW + tid] = tot;
-    }
-
-    // ---- the grid-wide barrier (bounded)
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        atomicAdd(p.counter, 1u);
-        uint32_t polls = 0;
-        int fail = 0;
-        while (ld_acquire(p.counter) < gridDim.x) {
-            if (++polls > kSmallSpinLimit) { fail = 1; break; }
-            __nanosleep(32);
-        }
-        if (fail && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_TIMEOUT);
-        sh_fail = fail;
-        // the last CTA to leave the barrier puts both counters back to zero for the next call
-        // (every CTA has read its last value of the arrival counter by then)
-        if (!fail && atomicAdd(p.counter + 1, 1u) == gridDim.x - 1) {
-            p.counter[1] = 0u;
-            __threadfence();
-            p.counter[0] = 0u;
-        }
-    }
-    __syncthreads();
-    if (sh_fail) return;
-
-    // ---- phase 2a: W from all partials, in an order that depends on the grid size only
-    {
-        const int m = tid & (MW - 1), part = tid >> 3;             // 32 strided partial sums per worker
-        double a = 0.0;
-        for (unsigned c0 = part; c0 < gridDim.x; c0 += 32 * 10) {    // ten loads in flight, added in index order
-            double v[10];
-#pragma unroll
-            for (int k = 0; k < 10; ++k) {
-                const unsigned c = c0 + 32u * k;
-                v[k] = c < gridDim.x ? __ldcg(p.part + (size_t)c * MW + m) : 0.0;     // 0 is neutral for both norms
-            }
-#pragma unroll
-            for (int k = 0; k < 10; ++k) a = combine<NORM>(a, v[k]);
-        }
-        sh[part][m] = a;
-    }
-    __syncthreads();
-    if (tid < MW) {                                  // thread m: worker m's 32 sums in index order
-        double tot = sh[0][tid];
-        for (int k = 1; k < 32; ++k) tot = combine<NORM>(tot, sh[k][tid]);
-        sh[0][tid] = tot;                            // only thread m touches column m
-    }
-    __syncthreads();
-    if (tid == 0) {
-        bool nan = false;
-        double top = 0.0;
-        for (int m = 0; m < p.M; ++m) {
-            const double tot = sh[0][m];
-            nan |= tot != tot;
-            top = fmax(top, tot);
-        }
-        float w;
-        if (NORM == UQ_NORM_L2) w = nan ? __uint_as_float(0x7FC00000u) : __double2float_rn(sqrt(top));
-        else w = __uint_as_float((uint32_t)top);
-        sh_w = w;
-        if (blockIdx.x == 0) {
-            p.W[0] = w;
-            uint32_t flags = 0;
-            if (not_finite(w)) flags |= UQ_STATUS_NONFINITE;
-            if (not_finite(inv_scale(p.s, w))) flags |= UQ_STATUS_SCALE_OVERFLOW;
-            if (flags && p.status) atomicOr(p.status, flags);
-        }
-    }
-    __syncthreads();
-    const float W = sh_w;
+    float W;
+    if (!small_agree<DT, NORM>(p, W)) return;
 
     // ---- phase 2b: quantize every worker's unit, add the levels, reconstruct
     float inv[8];
@@ -304,7 +174,8 @@ cudaError_t launch_small_step(const uq_layout &L, const void *g, int norm, int s
                               cudaStream_t st)
 {
     SmallParams p;
-    p.g = g; p.lev = lev; p.W = W; p.out = out; p.S = S; p.status = status;
+    p.g = g; p.lev = lev; p.idx = nullptr; p.W = W; p.out = out; p.S = S; p.status = status;
+    p.fmt = fmt; p.scales = ScaleSet{};
     p.counter = (uint32_t *)workspace;
     p.part = (double *)((char *)workspace + kSmallHeader);
     p.d = L.d; p.stride = L.worker_stride; p.coord0 = L.coord0; p.M = L.M; p.worker0 = L.worker0; p.s = s;
