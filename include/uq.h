@@ -340,29 +340,31 @@ int uq_step(const uq_layout *layout, const void *g, int norm, int s, const int32
             void *stream);
 
 /*
- * Algorithm 1, lines "MaxAllReduce Norm" to "Reconstruct gradient", as ONE kernel, for gradients
- * so small that the launches of uq_step cost more than its arithmetic.  A cooperative grid reads
- * the gradients for the norms, meets at one grid-wide barrier, and reads them again (from L2) to
- * quantize, store the level rows, add the levels and write the reconstructed average.
- * Supported: the single-scale quantizer, one segment (layout->nseg = 1), M <= 8, formats
- * UQ_FMT_I8 / I4X2 / I2X4, both dtypes, norms and draw widths; worker0 and coord0 key the draws as
- * in uq_encode_single.  Anything else returns UQ_ERR_UNSUPPORTED, as does a device without
- * cooperative launches.  Any size is computed correctly; it pays while M * d elements fit in L2.
- *   g, W, lev, out, S_opt (nullable), status (nullable): as in uq_agree_scale, uq_encode_single, uq_decode
+ * One whole step as ONE kernel — Algorithm 1 (scales = NULL) or Algorithm 2 (scales given), lines
+ * "MaxAllReduce Norm" to "Reconstruct gradient" — for gradients so small that the launches of
+ * uq_step cost more than its arithmetic.  A cooperative grid reads the gradients for the norms,
+ * meets at one grid-wide barrier, and reads them again (from L2) to [select and share the scale
+ * indices,] quantize, store the level rows, add the levels and write the reconstructed average.
+ * Arguments as in uq_step.  Supported: one segment (layout->nseg = 1), M <= 8, formats
+ * UQ_FMT_I8 / I4X2 / I2X4, both dtypes, norms, draw widths, every index width; worker0 and coord0
+ * key the draws as in the encoders.  Anything else returns UQ_ERR_UNSUPPORTED, as does a device
+ * without cooperative launches.  Any size is computed correctly; it pays while M * d elements are
+ * a few megabytes.
  *   workspace     scratch, device, 8-byte aligned, >= uq_workspace_bytes_small() bytes, used by one
  *                 call at a time.  Its first 64 bytes must be ZERO before the first call (zero
  *                 the scratch once after allocating it); every call leaves them zero again, except
  *                 one that reports UQ_STATUS_TIMEOUT: zero them again after that.
- * Results: lev, S_opt and out are bit for bit those of uq_step given the same W; W is added up
- * in another fixed order (L-inf: identical; L2: within one unit in the last place).
+ * Results: idx, lev, S_opt and out are bit for bit those of uq_step given the same W; W is added
+ * up in another fixed order (L-inf: identical; L2: within one unit in the last place).
  * The wait at the barrier is bounded: a CTA that gives up sets UQ_STATUS_TIMEOUT and returns
  * (outputs then incomplete).
  * Errors: UQ_ERR_BAD_ARG, UQ_ERR_UNSUPPORTED, UQ_ERR_WORKSPACE, UQ_ERR_CUDA.
  */
 size_t uq_workspace_bytes_small(void);
-int uq_step_small(const uq_layout *layout, const void *g, int norm, int s, uint64_t seed, int rng_bits,
-                  int fmt, float *W, void *lev, float *out, int32_t *S_opt, uint32_t *status,
-                  void *workspace, size_t workspace_bytes, void *stream);
+int uq_step_small(const uq_layout *layout, const void *g, int norm, int s, const int32_t *scales, int N,
+                  int idx_bits, uint64_t seed, int rng_bits, int fmt, float *W, uint8_t *idx, void *lev,
+                  float *out, int32_t *S_opt, uint32_t *status, void *workspace, size_t workspace_bytes,
+                  void *stream);
 
 /*
  * GlobalRandKMaxNorm / GlobalRandKMaxNormMultiScale — Sections "GlobalRandKMaxNorm Compression"

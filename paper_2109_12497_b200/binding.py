@@ -82,7 +82,7 @@ def lib() -> C.CDLL:
         L.uq_agree_scale.argtypes = [LP, P, I, P, P, P, SZ, P]
         L.uq_step.argtypes = [LP, P, I, I, P, I, I, U64, I, I, P, P, P, P, P, P, P, SZ, P]
         L.uq_agree_scale_amax.argtypes = [LP, P, I, P, P, P, P, SZ, P]
-        L.uq_step_small.argtypes = [LP, P, I, I, U64, I, I, P, P, P, P, P, P, SZ, P]
+        L.uq_step_small.argtypes = [LP, P, I, I, P, I, I, U64, I, I, P, P, P, P, P, P, P, SZ, P]
         L.uq_workspace_bytes_small.restype = SZ
         L.uq_workspace_bytes_small.argtypes = []
         L.uq_agree_scale_static.argtypes = [LP, P, I, P, P, P]
@@ -408,23 +408,29 @@ def uq_workspace_bytes_small() -> int:
     return int(lib().uq_workspace_bytes_small())
 
 
-def small_step_supported(layout: Layout, fmt: int, multi: bool) -> bool:
-    """Whether uq_step_small takes this configuration (single-scale, one segment, M <= 8, one-plane levels)."""
-    return (not multi and layout.nseg == 1 and layout.M <= SMALL_STEP_MAX_WORKERS
-            and fmt in (UQ_FMT_I8, UQ_FMT_I4X2, UQ_FMT_I2X4))
+def small_step_supported(layout: Layout, fmt: int) -> bool:
+    """Whether uq_step_small takes this configuration (one segment, M <= 8, one-plane levels)."""
+    return layout.nseg == 1 and layout.M <= SMALL_STEP_MAX_WORKERS and fmt in (UQ_FMT_I8, UQ_FMT_I4X2, UQ_FMT_I2X4)
 
 
-def uq_step_small(layout: Layout, g: torch.Tensor, norm: int, s: int, seed: int, rng_bits: int, fmt: int,
-                  W: torch.Tensor, lev: torch.Tensor, out: torch.Tensor, S_opt: Optional[torch.Tensor],
-                  status: Optional[torch.Tensor], workspace: torch.Tensor) -> None:
-    """The whole single-scale step as one cooperative kernel (small gradients).  ``workspace``:
-    zero-filled before its first use (the kernel leaves its counters zero), one call at a time."""
+def uq_step_small(layout: Layout, g: torch.Tensor, norm: int, s: int, scales: Optional[Sequence[int]], idx_bits: int,
+                  seed: int, rng_bits: int, fmt: int, W: torch.Tensor, idx: Optional[torch.Tensor], lev: torch.Tensor,
+                  out: torch.Tensor, S_opt: Optional[torch.Tensor], status: Optional[torch.Tensor],
+                  workspace: torch.Tensor) -> None:
+    """The whole step of either quantizer as one cooperative kernel (small gradients); arguments as
+    uq_step.  ``workspace``: zero-filled before its first use (the kernel leaves its counters
+    zero), one call at a time."""
     layout.check_g(g)
     layout.check_lev(lev, fmt)
     layout.check_vec(W, torch.float32, 1, "W")
     layout.check_vec(out, torch.float32, layout.d, "out")
     if S_opt is not None:
         layout.check_vec(S_opt, torch.int32, layout.d, "S_opt")
+    arr, N = (None, 0)
+    if scales is not None:
+        arr, N = _scales(scales)
+        layout.check_vec(idx, torch.uint8, layout.index_bytes(idx_bits), "idx")
     _check("uq_step_small", lib().uq_step_small(
-        layout.ref(), _ptr(g), norm, s, seed, rng_bits, fmt, _ptr(W), _ptr(lev), _ptr(out), _ptr(S_opt), _ptr(status),
-        _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()))
+        layout.ref(), _ptr(g), norm, s, arr, N, idx_bits, seed, rng_bits, fmt, _ptr(W),
+        _ptr(idx) if scales is not None else None, _ptr(lev), _ptr(out), _ptr(S_opt), _ptr(status), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _stream()))

@@ -37,6 +37,9 @@ size_t small_workspace_bytes();
 cudaError_t launch_small_step(const uq_layout &L, const void *g, int norm, int s, uint64_t seed, int rng_bits, int fmt,
                               float *W, void *lev, float *out, int32_t *S, uint32_t *status, void *workspace,
                               cudaStream_t st);
+cudaError_t launch_small_step_multi(const uq_layout &L, const void *g, int norm, const ScaleSet &scales, int idx_bits,
+                                    uint64_t seed, int rng_bits, int fmt, float *W, uint8_t *idx, void *lev, float *out,
+                                    int32_t *S, uint32_t *status, void *workspace, cudaStream_t st);
 }  // namespace uq
 
 namespace {
@@ -316,21 +319,27 @@ int uq_step(const uq_layout *L, const void *g, int norm, int s, const int32_t *s
 
 size_t uq_workspace_bytes_small(void) { return uq::small_workspace_bytes(); }
 
-int uq_step_small(const uq_layout *L, const void *g, int norm, int s, uint64_t seed, int rng_bits, int fmt, float *W,
-                  void *lev, float *out, int32_t *S_opt, uint32_t *status, void *workspace, size_t workspace_bytes,
-                  void *stream)
+int uq_step_small(const uq_layout *L, const void *g, int norm, int s, const int32_t *scales, int N, int idx_bits,
+                  uint64_t seed, int rng_bits, int fmt, float *W, uint8_t *idx, void *lev, float *out, int32_t *S_opt,
+                  uint32_t *status, void *workspace, size_t workspace_bytes, void *stream)
 {
+    uq::ScaleSet set;
     if (!layout_ok(L) || W == nullptr || !aligned(W, 4) || !aligned(status, 4)) return UQ_ERR_BAD_ARG;
     if (norm != UQ_NORM_L2 && norm != UQ_NORM_LINF) return UQ_ERR_BAD_ARG;
-    if (!fmt_ok(fmt, s) || (rng_bits != 32 && rng_bits != 16)) return UQ_ERR_BAD_ARG;
+    if (scales != nullptr && !scales_ok(scales, N, idx_bits, &set)) return UQ_ERR_BAD_ARG;
+    if (!fmt_ok(fmt, scales != nullptr ? set.s[0] : s) || (rng_bits != 32 && rng_bits != 16)) return UQ_ERR_BAD_ARG;
     if (L->d > 0 && (g == nullptr || lev == nullptr || out == nullptr || !aligned(g, 16) || !aligned(lev, 16) ||
                      !aligned(out, 32) || !aligned(S_opt, 32)))
         return UQ_ERR_BAD_ARG;
+    if (L->d > 0 && scales != nullptr && (idx == nullptr || !aligned(idx, 16))) return UQ_ERR_BAD_ARG;
     if (!uq::small_step_supported(*L, fmt)) return UQ_ERR_UNSUPPORTED;
     if (workspace == nullptr || !aligned(workspace, 8) || workspace_bytes < uq_workspace_bytes_small())
         return UQ_ERR_WORKSPACE;
-    const cudaError_t e = uq::launch_small_step(*L, g, norm, s, seed, rng_bits, fmt, W, lev, out, S_opt, status, workspace,
-                                                (cudaStream_t)stream);
+    const cudaError_t e = scales != nullptr
+        ? uq::launch_small_step_multi(*L, g, norm, set, idx_bits, seed, rng_bits, fmt, W, idx, lev, out, S_opt, status,
+                                      workspace, (cudaStream_t)stream)
+        : uq::launch_small_step(*L, g, norm, s, seed, rng_bits, fmt, W, lev, out, S_opt, status, workspace,
+                                (cudaStream_t)stream);
     if (e == cudaErrorNotSupported) return UQ_ERR_UNSUPPORTED;
     return finish(e);
 }

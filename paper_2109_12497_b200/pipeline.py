@@ -47,11 +47,10 @@ class Quantizer:
         nseg = self.layout.nseg
         self.W = torch.zeros(nseg, dtype=torch.float32, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
-        # single-scale, one segment, few workers, and so small that the step is bound by its five
-        # launches: the whole step as one cooperative kernel (uq_step_small).  None = decide by size.
-        fits = B.small_step_supported(self.layout, fmt, self.multi)
+        # one segment, few workers, and so small that the step is bound by its launches: the whole step as one cooperative kernel (uq_step_small).  None = decide by size.
+        fits = B.small_step_supported(self.layout, fmt) and not (fused_select or amax_select)
         if one_kernel and not fits:
-            raise ValueError("uq: the one-kernel step takes the single-scale quantizer, one segment, M <= 8")
+            raise ValueError("uq: the one-kernel step takes one segment, M <= 8 and one-plane level formats")
         self.one_kernel = fits and (one_kernel if one_kernel is not None
                                     else M * d * (4 if dtype == torch.float32 else 2) <= ONE_KERNEL_MAX_BYTES)
         # zeroed: the one-kernel step wants its counters zero before the first call and leaves them so
@@ -117,11 +116,13 @@ class Quantizer:
                 raise ValueError("uq: tensors must live on a CUDA device")
             if self._small_call is None:
                 ptr = lambda t: None if t is None else t.data_ptr()
-                self._small_call = (B.lib().uq_step_small, self.layout.ref(),
-                                    (ptr(self.W), ptr(self.lev), ptr(self.out), ptr(self.S), ptr(self.status),
-                                     ptr(self.workspace), self.workspace.numel()))
-            fn, ref, tail = self._small_call
-            rc = fn(ref, g.data_ptr(), self.norm, self.s, seed, self.rng_bits, self.fmt, *tail, B._stream())
+                arr, N = B._scales(self.scales) if self.multi else (None, 0)
+                self._small_call = (B.lib().uq_step_small, self.layout.ref(), arr, N,
+                                    (ptr(self.W), ptr(self.idx), ptr(self.lev), ptr(self.out), ptr(self.S),
+                                     ptr(self.status), ptr(self.workspace), self.workspace.numel()))
+            fn, ref, arr, N, tail = self._small_call
+            rc = fn(ref, g.data_ptr(), self.norm, self.s, arr, N, self.idx_bits, seed, self.rng_bits, self.fmt, *tail,
+                    B._stream())
             if rc != B.UQ_OK:
                 raise B.UqError("uq_step_small", rc)
             return self._out_view

@@ -87,15 +87,14 @@ def check_parity(w, g_np, seed=None):
     if w.quantizer == "multi":
         _check_parity(w, g_np, seed, "fused")
         _check_parity(w, g_np, seed, "amax")
-    elif one_kernel_takes(w):
+    if one_kernel_takes(w):
         _check_parity(w, g_np, seed, "one")
         _check_parity(w, g_np, seed, "separate")
     return _check_parity(w, g_np, seed, "default")
 
 
 def one_kernel_takes(w) -> bool:
-    return (w.quantizer == "single" and len(wl.segment_offsets(w)) == 2 and w.M <= B.SMALL_STEP_MAX_WORKERS
-            and w.fmt in ("i8", "i4x2", "i2x4"))
+    return len(wl.segment_offsets(w)) == 2 and w.M <= B.SMALL_STEP_MAX_WORKERS and w.fmt in ("i8", "i4x2", "i2x4")
 
 
 def _check_parity(w, g_np, seed, mode):

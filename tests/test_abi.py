@@ -103,17 +103,19 @@ def test_later_entry_points_reject_bad_arguments_on_the_host(lib):
                        None) == B.UQ_ERR_BAD_ARG
     assert lib.uq_step(ok, p, B.UQ_NORM_L2, 127, None, 0, 0, 0, 16, B.UQ_FMT_I8, p, None, p, p, None, None, p, 8,
                        None) == B.UQ_ERR_WORKSPACE
-    small = lib.uq_workspace_bytes_small()
-    assert small >= 64 + 148 * 8 * 8 * 8
-    assert lib.uq_step_small(bad, p, B.UQ_NORM_L2, 127, 0, 16, B.UQ_FMT_I8, p, p, p, None, None, p, small, None) == B.UQ_ERR_BAD_ARG
-    assert lib.uq_step_small(ok, p, B.UQ_NORM_L2, 128, 0, 16, B.UQ_FMT_I8, p, p, p, None, None, p, small, None) == B.UQ_ERR_BAD_ARG
-    assert lib.uq_step_small(ok, p, B.UQ_NORM_L2, 127, 0, 16, B.UQ_FMT_I8, p, p, p + 16, None, None, p, small, None) \
-        == B.UQ_ERR_BAD_ARG                                                                         # out: 32-byte aligned
-    assert lib.uq_step_small(C.byref(_layout(M=9)), p, B.UQ_NORM_L2, 127, 0, 16, B.UQ_FMT_I8, p, p, p, None, None, p, small,
-                             None) == B.UQ_ERR_UNSUPPORTED
-    assert lib.uq_step_small(ok, p, B.UQ_NORM_L2, 31, 0, 16, B.UQ_FMT_I6P, p, p, p, None, None, p, small, None) \
-        == B.UQ_ERR_UNSUPPORTED
-    assert lib.uq_step_small(ok, p, B.UQ_NORM_L2, 127, 0, 16, B.UQ_FMT_I8, p, p, p, None, None, p, 64, None) == B.UQ_ERR_WORKSPACE
+    small_bytes = lib.uq_workspace_bytes_small()
+    assert small_bytes >= 64 + 148 * 8 * 8 * 8
+    def small(L, s=127, scales=None, N=0, bits=0, fmt=B.UQ_FMT_I8, out=p, idx=None, ws=small_bytes):
+        return lib.uq_step_small(L, p, B.UQ_NORM_L2, s, scales, N, bits, 0, 16, fmt, p, idx, p, out, None, None, p, ws, None)
+    assert small(bad) == B.UQ_ERR_BAD_ARG
+    assert small(ok, s=128) == B.UQ_ERR_BAD_ARG
+    assert small(ok, out=p + 16) == B.UQ_ERR_BAD_ARG                                      # out: 32-byte aligned
+    assert small(ok, scales=sc, N=2, bits=3, idx=p) == B.UQ_ERR_BAD_ARG                     # idx_bits
+    assert small(ok, scales=sc, N=2, bits=2, idx=None) == B.UQ_ERR_BAD_ARG                  # multi-scale needs idx
+    assert small(C.byref(_layout(M=9))) == B.UQ_ERR_UNSUPPORTED
+    assert small(ok, s=31, fmt=B.UQ_FMT_I6P) == B.UQ_ERR_UNSUPPORTED
+    assert small(ok, ws=64) == B.UQ_ERR_WORKSPACE
+    assert small(ok, scales=sc, N=2, bits=2, idx=p, ws=64) == B.UQ_ERR_WORKSPACE
     assert lib.uq_agree_scale_amax(bad, p, B.UQ_NORM_L2, p, p, None, p, 1 << 20, None) == B.UQ_ERR_BAD_ARG
     assert lib.uq_agree_scale_amax(ok, p, B.UQ_NORM_L2, p, p + 8, None, p, 1 << 20, None) == B.UQ_ERR_BAD_ARG   # alignment
     assert lib.uq_agree_scale_amax(ok, p, B.UQ_NORM_L2, p, None, None, p, 1 << 20, None) == B.UQ_ERR_BAD_ARG

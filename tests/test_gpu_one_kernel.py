@@ -1,5 +1,5 @@
-"""uq_step_small: the whole single-scale step as one cooperative kernel, against the oracle and
-against the separate calls."""
+"""uq_step_small: the whole step of either quantizer as one cooperative kernel, against the oracle
+and against the separate calls."""
 import ctypes as C
 
 import numpy as np
@@ -51,7 +51,8 @@ def test_the_library_picks_the_one_kernel_step_by_size():
     small = from_workload(wl.scaled("c1", 100_000, M=2))
     big = from_workload(wl.scaled("c1", 2_000_000, M=2))              # 16 MB of gradients
     segmented = from_workload(wl.scaled("c2", 100_000, M=2))
-    assert small.one_kernel and not big.one_kernel and not segmented.one_kernel
+    multi = from_workload(wl.scaled("c3", 100_000, M=4, segments="one"))
+    assert small.one_kernel and multi.one_kernel and not big.one_kernel and not segmented.one_kernel
     with pytest.raises(ValueError):
         from_workload(wl.scaled("c2", 100_000, M=2), one_kernel=True)
 
@@ -62,16 +63,17 @@ def test_unsupported_configurations_are_refused():
     W, out = torch.zeros(1, device="cuda"), torch.zeros(128, device="cuda")
     lev = torch.empty((9, 128), dtype=torch.int8, device="cuda")
     with pytest.raises(B.UqError) as e:
-        B.uq_step_small(B.Layout(9, 100, 128, torch.float32), g, B.UQ_NORM_L2, 127, 0, 16, B.UQ_FMT_I8, W, lev, out, None, None, ws)
+        B.uq_step_small(B.Layout(9, 100, 128, torch.float32), g, B.UQ_NORM_L2, 127, None, 0, 0, 16, B.UQ_FMT_I8, W, None, lev, out,
+                        None, None, ws)
     assert e.value.code == B.UQ_ERR_UNSUPPORTED
     lay = B.Layout(2, 100, 128, torch.float32)
     lev6 = torch.empty((2, lay.level_row_bytes(B.UQ_FMT_I6P)), dtype=torch.int8, device="cuda")
     with pytest.raises(B.UqError) as e:
-        B.uq_step_small(lay, g[:2].contiguous(), B.UQ_NORM_L2, 31, 0, 16, B.UQ_FMT_I6P, W, lev6, out, None, None, ws)
+        B.uq_step_small(lay, g[:2].contiguous(), B.UQ_NORM_L2, 31, None, 0, 0, 16, B.UQ_FMT_I6P, W, None, lev6, out, None, None, ws)
     assert e.value.code == B.UQ_ERR_UNSUPPORTED
     with pytest.raises(B.UqError) as e:
-        B.uq_step_small(lay, g[:2].contiguous(), B.UQ_NORM_L2, 127, 0, 16, B.UQ_FMT_I8, W, lev[:2].contiguous(), out, None, None,
-                        ws[:64])
+        B.uq_step_small(lay, g[:2].contiguous(), B.UQ_NORM_L2, 127, None, 0, 0, 16, B.UQ_FMT_I8, W, None, lev[:2].contiguous(), out,
+                        None, None, ws[:64])
     assert e.value.code == B.UQ_ERR_WORKSPACE
 
 
@@ -86,7 +88,7 @@ def test_draws_are_keyed_by_worker_and_coordinate_of_the_job():
     lev = torch.zeros((M, g.shape[1]), dtype=torch.int8, device="cuda")
     ws = torch.zeros(B.uq_workspace_bytes_small(), dtype=torch.uint8, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    B.uq_step_small(lay, g, B.UQ_NORM_L2, 127, 77, 16, B.UQ_FMT_I8, W, lev, out, None, status, ws)
+    B.uq_step_small(lay, g, B.UQ_NORM_L2, 127, None, 0, 77, 16, B.UQ_FMT_I8, W, None, lev, out, None, status, ws)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     want = o.encode_single(g_np[:, :d], W.cpu().numpy(), 127, 77, 16, worker0=worker0, coord0=coord0)
@@ -140,3 +142,45 @@ def test_the_wait_at_the_barrier_is_bounded():
     assert q.status_bits() == 0
     lev = o.encode_single(g_np[:, : w.d], q.W.cpu().numpy(), w.s, w.seed, w.rng_bits)
     assert np.array_equal(q.lev.cpu().numpy()[:, : w.d], lev)
+
+
+@pytest.mark.parametrize("d", [1, 9, 255, 2049, 100_003, 1 << 20])
+@pytest.mark.parametrize("M,dtype,norm,fmt,scales,idx_bits,rng_bits", [
+    (2, wl.F32, wl.NORM_L2, "i8", (127, 1016, 8128, 65024), 2, 16), (3, wl.BF16, wl.NORM_L2, "i8", tuple(127 * 8 ** k for k in range(8)), 4, 16),
+    (8, wl.F32, wl.NORM_LINF, "i4x2", (7, 112), 1, 32), (5, wl.BF16, wl.NORM_LINF, "i2x4", (1, 16, 256), 8, 32),
+    (1, wl.F32, wl.NORM_L2, "i4x2", tuple(5 * 3 ** k for k in range(16)), 4, 32), (4, wl.BF16, wl.NORM_L2, "i8", (100,), 2, 16),
+])
+def test_one_kernel_multi_scale_matches_the_oracle(d, M, dtype, norm, fmt, scales, idx_bits, rng_bits):
+    w = wl.scaled("c3", d, M=M, segments="one", dtype=dtype, norm=norm, fmt=fmt, s=scales[0], scales=scales, idx_bits=idx_bits,
+                  rng_bits=rng_bits, seed=3 * d + M)
+    r = _check_parity(w, wl.generate(w), None, "one")
+    assert r["q"].one_kernel and r["q"].multi and r["q"].kernels_per_step() == 1
+
+
+@pytest.mark.parametrize("name,d,M", [("c3", 1 << 20, 2), ("c5", 700_001, 8), ("c3", 5_000_011, 2)])
+def test_one_kernel_multi_scale_equals_the_separate_calls(name, d, M):
+    w = wl.scaled(name, d, M=M, segments="one", norm=wl.NORM_LINF)             # same W bits on both sides
+    g_np = wl.generate(w)
+    one, sep = run_gpu(w, g_np, mode="one"), run_gpu(w, g_np, mode="separate")
+    assert one["q"].one_kernel and not sep["q"].one_kernel and one["status"] == 0 and sep["status"] == 0
+    assert np.array_equal(one["W"], sep["W"])
+    assert np.array_equal(one["idx"][: w.d * w.idx_bits // 8], sep["idx"][: w.d * w.idx_bits // 8])
+    assert np.array_equal(one["lev"][:, : w.d], sep["lev"][:, : w.d])
+    assert np.array_equal(one["S"], sep["S"]) and np.array_equal(one["out"], sep["out"])
+
+
+def test_multi_scale_steps_back_to_back():
+    w = wl.scaled("c5", 300_001, M=4, segments="one")
+    g_np = wl.generate(w)
+    q = from_workload(w, keep_sums=True, one_kernel=True)
+    g = to_device(w, g_np)
+    for k in range(100):
+        q.step(g, k)
+    torch.cuda.synchronize()
+    assert q.status_bits() == 0
+    W = q.W.cpu().numpy()
+    idx = o.select_scale_multi(g_np[:, : w.d], W, w.scales)
+    lev = o.encode_multi(g_np[:, : w.d], W, w.scales, idx, 99, w.rng_bits)
+    assert np.array_equal(q.lev.cpu().numpy()[:, : w.d], lev)
+    assert np.array_equal(q.S.cpu().numpy()[: w.d], o.aggregate(lev))
+    assert np.array_equal(q.out.cpu().numpy()[: w.d], o.decode(o.aggregate(lev), w.M, W, scales=w.scales, idx=idx))
