@@ -475,6 +475,10 @@ def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=F
         res["fused_select_ms"] = time_fused_select_encode(q, g_dev, w, min(steps, 10))
     if randk_K:
         res["randk"] = time_randk(w, g_dev, min(randk_K, w.d), 50)
+        if w.quantizer == "single":               # the same choice quantized with a two-scale set (GlobalRandK-MN-TS)
+            import dataclasses
+            two = dataclasses.replace(w, quantizer="multi", scales=(w.s, w.s * 16), idx_bits=1)
+            res["randk_two_scale"] = time_randk(two, g_dev, min(randk_K, w.d), 50)
         res["graph_stats"] = time_graph_replay(q, g_dev, w, max(steps, 20), stats=True)
     res["h2d"], res["d2h"], res["e2e_ms"] = 0, 0, None
     if want_e2e:
@@ -656,6 +660,8 @@ def gpu_main(args):
     }
     if "randk" in res:
         line["global_randk"] = res["randk"]
+    if "randk_two_scale" in res:
+        line["global_randk_two_scale"] = res["randk_two_scale"]
     if "graph_stats" in res:
         mean, med, lo = res["graph_stats"]
         line["cuda_graph_replay"] = {"ms_per_step_mean": round(mean, 5), "ms_per_step_median": round(med, 5),
