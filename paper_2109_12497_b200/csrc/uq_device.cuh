@@ -258,6 +258,70 @@ __device__ __forceinline__ void philox4x32_10_workers(const PhiloxKey &k, uint32
     for (int n = 0; n < N; ++n) out[n] = make_uint4(c0[n], c1[n], c2[n], c3[n]);
 }
 
+// The first two rounds of a block split by what they depend on.  Of the counter
+// (block low, block high, worker, 0) only word 0 differs between the threads of a tile and only
+// word 2 between the workers, and the two do not meet before the second round:
+//   round 0: c0 = hi(M1*worker) ^ block_high ^ k0[0]   c1 = lo(M1*worker)       (per worker)
+//            c2 = hi(M0*block_low) ^ k1[0]             c3 = lo(M0*block_low)    (per block)
+//   round 1: c0 = hi(M1*c2) ^ c1 ^ k0[1]   c1 = lo(M1*c2)   c2 = hi(M0*c0) ^ c3 ^ k1[1]   c3 = lo(M0*c0)
+// so a thread that draws the same block for several workers keeps {hi, lo}(M1*c2) and c3 of round 0
+// (PhiloxBlockPart), takes the per-worker words from a table made once per launch
+// (PhiloxWorkerPart, uniform over the grid), joins them with two three-input XORs and runs the
+// remaining eight rounds: 34 instead of 40 multiply / XOR instructions per block.
+struct PhiloxBlockPart { uint32_t a, b, c3; };       // hi(M1*c2), lo(M1*c2), c3 after round 0
+struct PhiloxWorkerPart { uint32_t u1, hq, lq; };    // c1 after round 0; hi, lo of M0 * (c0 after round 0)
+
+constexpr uint32_t kPhiloxM0 = 0xD2511F53u, kPhiloxM1 = 0xCD9E8D57u;
+
+__device__ __forceinline__ PhiloxBlockPart philox_block_part(const PhiloxKey &k, uint32_t block_lo)
+{
+    PhiloxBlockPart r;
+    const uint64_t p0 = (uint64_t)kPhiloxM0 * block_lo;
+    r.c3 = (uint32_t)p0;
+    const uint64_t p1 = (uint64_t)kPhiloxM1 * ((uint32_t)(p0 >> 32) ^ k.k1[0]);
+    r.a = (uint32_t)(p1 >> 32); r.b = (uint32_t)p1;
+    return r;
+}
+
+__host__ __device__ __forceinline__ PhiloxWorkerPart philox_worker_part(const PhiloxKey &k, uint32_t block_hi, uint32_t worker)
+{
+    PhiloxWorkerPart w;
+    const uint64_t pw = (uint64_t)kPhiloxM1 * worker;
+    w.u1 = (uint32_t)pw;
+    const uint64_t q0 = (uint64_t)kPhiloxM0 * ((uint32_t)(pw >> 32) ^ block_hi ^ k.k0[0]);
+    w.hq = (uint32_t)(q0 >> 32); w.lq = (uint32_t)q0;
+    return w;
+}
+
+// Rounds 1 (the joining XORs) to 9 of N blocks of one worker, advanced together.
+template <int N>
+__device__ __forceinline__ void philox_join(const PhiloxKey &k, const PhiloxBlockPart (&blk)[N], const PhiloxWorkerPart &w,
+                                            uint4 (&out)[N])
+{
+    uint32_t c0[N], c1[N], c2[N], c3[N];
+#pragma unroll
+    for (int n = 0; n < N; ++n) {
+        c0[n] = blk[n].a ^ w.u1 ^ k.k0[1];
+        c1[n] = blk[n].b;
+        c2[n] = w.hq ^ blk[n].c3 ^ k.k1[1];
+        c3[n] = w.lq;
+    }
+#pragma unroll
+    for (int r = 2; r < 10; ++r) {
+        const uint32_t k0 = k.k0[r], k1 = k.k1[r];
+#pragma unroll
+        for (int n = 0; n < N; ++n) {
+            const uint64_t p0 = (uint64_t)kPhiloxM0 * c0[n];
+            const uint64_t p1 = (uint64_t)kPhiloxM1 * c2[n];
+            const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1[n] ^ k0;
+            const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3[n] ^ k1;
+            c1[n] = (uint32_t)p1; c3[n] = (uint32_t)p0; c0[n] = n0; c2[n] = n2;
+        }
+    }
+#pragma unroll
+    for (int n = 0; n < N; ++n) out[n] = make_uint4(c0[n], c1[n], c2[n], c3[n]);
+}
+
 // ---------------------------------------------------------------------------------------------
 // one coordinate of Q_s
 // ---------------------------------------------------------------------------------------------
@@ -292,6 +356,33 @@ __device__ __forceinline__ uint32_t level_draw16(float x, uint32_t h)
     return __float_as_uint(__fadd_rn(x, 128.0f)) + 0xFFFFu - h;
 }
 constexpr uint32_t kLevelByte16 = 2;
+
+// The same level with the clamp folded into saturating arithmetic (both on the FMA pipe, where the
+// min of the form above is an ALU instruction).  inv256 = inv / 256 exactly (the caller checks that
+// inv is 0 or at least 2^-100, so nothing is lost to a subnormal), hence |v| * inv256 = x / 256
+// with the rounding of x.  c0 = 1 - cap / 256: the saturating sum reaches 1.0 exactly where x
+// reaches cap, and below 1.0 its unit in the last place is 2^-24, i.e. 2^-16 in x (ties to even as
+// before, since c0 is an even multiple of it).  As an integer the sum is
+//   0x3F000000 + (128 - cap) * 2^16 + floor(x) * 2^16 + rint(p * 2^16),
+// and subtracting h + 1 borrows from the level field iff h >= rint(p * 2^16).  With
+// adj = -1 - (127 - cap) * 2^16 byte 2 of the result is the level.  The saturating product turns a
+// NaN (0 * Inf, a NaN input) into 0 and so into level 0; Inf saturates to level cap.
+__device__ __forceinline__ float mul_sat(float a, float b)
+{
+    float d;
+    asm("mul.rn.sat.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+__device__ __forceinline__ float add_sat(float a, float b)
+{
+    float d;
+    asm("add.rn.sat.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t level_draw16_sat(float v, float inv256, float c0, uint32_t adj, uint32_t h)
+{
+    return __float_as_uint(add_sat(mul_sat(fabsf(v), inv256), c0)) - h + adj;
+}
 
 // Gathers byte B of four words into one word (coordinate order = byte order).
 template <uint32_t B> __device__ __forceinline__ uint32_t gather_bytes(uint32_t a, uint32_t b, uint32_t c, uint32_t d)

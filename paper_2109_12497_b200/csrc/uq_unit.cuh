@@ -71,6 +71,35 @@ __device__ __forceinline__ void quantize_unit_bytes(const float (&v)[8], const f
     hi = negate_bytes(gather_bytes<LB>(z[4], z[5], z[6], z[7]), neg_hi);
 }
 
+// The same for 16-bit draws with the clamp in saturating arithmetic (level_draw16_sat): inv256[e]
+// is the coordinate's factor divided by 256, (c0, adj) come from sat_constants(cap).
+struct SatConstants { float c0; uint32_t adj; };
+__device__ __forceinline__ SatConstants sat_constants(float cap)
+{
+    SatConstants c;
+    c.c0 = __fsub_rn(1.0f, __fmul_rn(cap, 0.00390625f));
+    c.adj = 0xFFFFFFFFu - ((127u - (uint32_t)cap) << 16);
+    return c;
+}
+// Whether the saturating form may be used with smallest factor inv0 (= scales[0] / W): dividing a
+// factor below 2^-100 by 256 could round.  (0, Inf and NaN divide exactly.)
+__device__ __forceinline__ bool sat_form_exact(float inv0) { return !(inv0 > 0.0f && inv0 < 7.888609052e-31f); }
+
+__device__ __forceinline__ void quantize_unit_bytes_sat16(const float (&v)[8], const float (&inv256)[8], const SatConstants &sc,
+                                                          uint32_t neg_lo, uint32_t neg_hi, const uint4 &r, uint32_t &lo,
+                                                          uint32_t &hi)
+{
+    const uint32_t w[4] = { r.x, r.y, r.z, r.w };
+    uint32_t z[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        const uint32_t h = (e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu);
+        z[e] = level_draw16_sat(v[e], inv256[e], sc.c0, sc.adj, h);
+    }
+    lo = negate_bytes(gather_bytes<2>(z[0], z[1], z[2], z[3]), neg_lo);
+    hi = negate_bytes(gather_bytes<2>(z[4], z[5], z[6], z[7]), neg_hi);
+}
+
 // The level bytes of a unit packed into the wire format and stored.
 template <int FMT> __device__ __forceinline__ void store_unit(uint32_t lo, uint32_t hi, void *dst, void *dst2)
 {
