@@ -1,10 +1,11 @@
 #!/usr/bin/env python
 """Benchmark of the quantize -> integer aggregate -> reconstruct hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5] [--impl reference]
 
-One step = one pass of the whole path (agree scale, [select scale index], encode, fused
-aggregate+decode) over one batch of synthetic gradients of M workers.  The metric is gradient
+One step = one pass of the whole path (agree scale, [select + share scale index,] encode, fused
+aggregate+decode) over one batch of synthetic gradients of M workers.  The default workload is
+the largest single-GPU configuration, c5.  The metric is gradient
 GB/s: bytes of gradient input (M * d * sizeof(element)) per second of the whole step.
 The path does not shard: with N GPUs every rank runs an independent replica ("replicas only")
 and the value is the sum over ranks; timing is the max over ranks of device-event time.
@@ -35,11 +36,12 @@ METRIC = "gradient GB/s through encode+aggregate+decode; % of B200 HBM roofline"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only without MEASURED_PEAKS.json
 
-# DRAM traffic per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum) from
-# the ncu captures summarised under profiles/, keyed by workload; None = not captured.
-# c2: 838.3 MB read + 155.8 MB written by the encode kernel in a capture at full size
-# (profiles/traffic_c2_full_size.md).
-NCU_TRAFFIC_BYTES = {"c2": 994.1e6}
+# DRAM traffic of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum under ncu) in
+# bytes per coordinate, from captures of a small case of the same recipe summarised under
+# profiles/ (the full workloads are too large to capture); a launch at full size is taken as
+# bytes per coordinate * d, since every byte of these kernels belongs to a coordinate.
+# Keyed by (workload, kernel); absent = not captured.
+NCU_TRAFFIC_BYTES_PER_COORD = {}
 
 
 def hbm_peak():
@@ -64,8 +66,8 @@ def algorithmic_bytes(w: wl.Workload) -> dict:
     b = {"agree_scale": e * M * d}
     if w.quantizer == "multi":
         b["select_scale"] = e * M * d + ib * d
-        b["encode"] = (e + lev + ib) * M * d          # every worker re-reads the shared index
-        b["select_encode"] = (e + lev) * M * d + ib * d   # fused: gradients read once, index written once
+        b["encode"] = (e + lev + ib) * M * d          # the shared index counted once per worker
+        b["select_encode"] = (e + lev) * M * d + ib * d   # one call: gradients read once, index written once
     else:
         b["encode"] = (e + lev) * M * d
     b["aggregate_decode"] = lev * M * d + ib * d + 4 * d
@@ -75,7 +77,7 @@ def algorithmic_bytes(w: wl.Workload) -> dict:
 def step_roofline(w: wl.Workload, ms: float, peak_gbs: float) -> dict:
     """The whole step against the sum of its stages' algorithmic bytes moved at the HBM peak."""
     ab = algorithmic_bytes(w)
-    total = sum(v for k, v in ab.items() if k != "select_encode")
+    total = sum(ab[k] for k in stages_of(w))
     min_ms = total / peak_gbs / 1e6
     return {"algorithmic_MB": round(total / 1e6, 1), "min_ms_at_peak": round(min_ms, 5), "frac": round(min_ms / ms, 4),
             "ceiling_gradient_GBps": round(w.in_bytes / min_ms / 1e6, 1)}
@@ -139,7 +141,20 @@ class ClockSampler:
 # ---------------------------------------------------------------------------------------------
 
 STAGES_SINGLE = ["agree_scale", "encode", "aggregate_decode"]
-STAGES_MULTI = ["agree_scale", "select_scale", "encode", "aggregate_decode"]
+STAGES_MULTI = ["agree_scale", "select_scale", "encode", "aggregate_decode"]      # the calls uq_step makes
+
+
+def stages_of(w):
+    return STAGES_MULTI if w.quantizer == "multi" else STAGES_SINGLE
+
+
+def stage_calls(q, g):
+    """{stage: function of the seed} for the separate calls of the step."""
+    calls = {"agree_scale": lambda seed: q.agree_scale(g), "aggregate_decode": lambda seed: q.aggregate_decode()}
+    calls["encode"] = lambda seed: q.encode(g, seed)
+    if q.multi:
+        calls["select_scale"] = lambda seed: q.select_scale(g)
+    return calls
 
 
 def run_stages(q, g, seed, events=None):
@@ -150,21 +165,11 @@ def run_stages(q, g, seed, events=None):
         q.step(g, seed)
         return
     st = torch.cuda.current_stream()
-    k = 0
-    if events: events[k].record(st)
-    q.agree_scale(g); k += 1
-    if events: events[k].record(st)
-    if q.multi and q.fused_select:
-        q.select_encode(g, seed); k += 1
-        if events: events[k].record(st)
-    else:
-        if q.multi:
-            q.select_scale(g); k += 1
-            if events: events[k].record(st)
-        q.encode(g, seed); k += 1
-        if events: events[k].record(st)
-    q.aggregate_decode(); k += 1
-    if events: events[k].record(st)
+    calls = stage_calls(q, g)
+    events[0].record(st)
+    for k, name in enumerate(STAGES_MULTI if q.multi else STAGES_SINGLE):
+        calls[name](seed)
+        events[k + 1].record(st)
 
 
 def time_device_resident(q, g, w, steps, warmup, barrier):
@@ -175,7 +180,7 @@ def time_device_resident(q, g, w, steps, warmup, barrier):
     an event after every stage."""
     import torch
     st = torch.cuda.current_stream()
-    stages = STAGES_MULTI if q.multi else STAGES_SINGLE
+    stages = stages_of(w)
     for _ in range(warmup):
         run_stages(q, g, w.seed)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -224,6 +229,28 @@ def time_sustained(q, g, w, ms_burst, lead_s=0.6, span_s=0.4):
     return e0.elapsed_time(e1) / n_span, n_lead, n_span
 
 
+def time_alone(fn, reps, sustained=False, ms_hint=1.0, lead_s=0.6, span_s=0.4):
+    """Mean ms of one call of fn(seed) looped alone.  sustained: after lead_s seconds of the same
+    calls untimed, over span_s seconds (the rate at the board's power cap); else a burst of reps."""
+    import torch
+    st = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if sustained:
+        n_lead = max(1, int(lead_s * 1e3 / ms_hint))
+        reps = max(1, int(span_s * 1e3 / ms_hint))
+    else:
+        n_lead = 2
+    torch.cuda.synchronize()
+    for k in range(n_lead):
+        fn(k)
+    e0.record(st)
+    for k in range(reps):
+        fn(1000 + k)
+    e1.record(st)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
 def time_end_to_end(q, g_host, out_host, g_dev, w, steps, warmup, barrier):
     """ms per step with the gradients starting in pinned host memory and the result read back.
     Every step copies its own inputs in and its own result out; the read-back of step k runs on
@@ -262,40 +289,18 @@ def time_end_to_end(q, g_host, out_host, g_dev, w, steps, warmup, barrier):
 def time_encode_other_mode(q, g, w, reps):
     """Mean ms of the encode kernel alone with the other random-draw width (context: the step
     itself runs in the workload's own mode).  W and idx are those of the last step."""
-    import torch
-    st = torch.cuda.current_stream()
     keep = q.rng_bits
     q.rng_bits = 32 if keep == 16 else 16
     try:
-        for _ in range(2):
-            q.encode(g, w.seed)
-        evs = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
-        torch.cuda.synchronize()
-        for k in range(reps):
-            evs[k].record(st)
-            q.encode(g, w.seed + k)
-        evs[reps].record(st)
-        torch.cuda.synchronize()
-        return evs[0].elapsed_time(evs[reps]) / reps
+        return time_alone(lambda k: q.encode(g, w.seed + k), reps)
     finally:
         q.rng_bits = keep
 
 
 def time_fused_select_encode(q, g, w, reps):
-    """Multi-scale: mean ms of the one-kernel form of selection + encoding (the step itself runs
-    the two kernels, which measure no slower), timed alone."""
-    import torch
-    st = torch.cuda.current_stream()
-    for k in range(2):
-        q.select_encode(g, w.seed + k)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    e0.record(st)
-    for k in range(reps):
-        q.select_encode(g, w.seed + k)
-    e1.record(st)
-    torch.cuda.synchronize()
-    return e0.elapsed_time(e1) / reps
+    """Multi-scale: mean ms of selection + encoding as one call (uq_select_encode_multi: one kernel
+    for M <= 8; the step runs the two streaming kernels), timed alone."""
+    return time_alone(lambda k: q.select_encode(g, w.seed + k), reps)
 
 
 def time_graph_replay(q, g, w, reps, stats=False):
@@ -407,25 +412,35 @@ def l2_flush_buffer():
     return torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
 
 
-def resolve_workload(name, d=None, rng_bits=None):
+LEVEL_WIRES = {"i8": 127, "i6p": 31, "i4x2": 7, "i2x4": 1}       # wire format -> levels of the smallest scale
+
+
+def resolve_workload(name, d=None, rng_bits=None, levels=None):
     """The named workload, optionally at a smaller d (same recipe; used for ncu captures, which
-    must stay small) or with the other random-draw width."""
+    must stay small), with the other random-draw width, or on another level wire format (the
+    scale set keeps its ratios and starts at the format's largest level)."""
     w = wl.WORKLOADS[name]
+    if levels is not None and levels != w.fmt:
+        import dataclasses
+        s_new = LEVEL_WIRES[levels]
+        w = dataclasses.replace(w, fmt=levels, s=s_new, scales=tuple(s_new * (x // w.scales[0]) for x in w.scales))
     if d is not None and d != w.d:
-        w = wl.scaled(name, d)
-        if wl.WORKLOADS[name].segments == "buckets25MiB":
-            import dataclasses
-            w = dataclasses.replace(w, bucket_elems=wl.WORKLOADS[name].bucket_elems)
+        import dataclasses
+        w = dataclasses.replace(w, d=d, name=f"{name}@{d}")
     if rng_bits is not None:
         import dataclasses
         w = dataclasses.replace(w, rng_bits=rng_bits)
     return w
 
 
-def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=False, randk_K=0, sustained=False):
-    """Times one workload on the current device.  Returns a dict of raw numbers."""
+def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=False, randk_K=0, sustained=False,
+                   device_index=0):
+    """Times one workload on the current device.  Returns a dict of raw numbers.  The clocks of
+    the device are sampled over everything timed here (res["clocks"])."""
     import torch
     from paper_2109_12497_b200.pipeline import from_workload
+    sampler = ClockSampler(device_index)
+    sampler.start()
     np_dtype = np.float32 if w.dtype == wl.F32 else np.uint16
     if want_e2e:
         g_host = torch.empty((w.M, w.stride), dtype=torch.float32 if w.dtype == wl.F32 else torch.int16,
@@ -447,7 +462,7 @@ def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=F
         flush = l2_flush_buffer()
         for _ in range(warmup):
             run_stages(q, g_dev, w.seed)
-        stages = STAGES_MULTI if q.multi else STAGES_SINGLE
+        stages = stages_of(w)
         tot, per = [], {s: [] for s in stages}
         for k in range(steps):
             flush.fill_(k & 0xFF)
@@ -486,8 +501,17 @@ def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=F
         res["e2e_ms"] = time_end_to_end(q, g_host, out_host, g_dev, w, steps, warmup, barrier)
         res["h2d"] = g_host.numel() * g_host.element_size()
         res["d2h"] = out_host.numel() * 4
+    res["clocks"] = sampler.stop()           # the record of the burst figures above
     if sustained:
+        # under continuous load: the whole step, then every stage looped alone
         res["sustained"] = time_sustained(q, g_dev, w, res["ms"])
+        if not q.one_kernel:
+            calls = stage_calls(q, g_dev)
+            res["stages_sustained_ms"] = {}
+            for name in stages_of(w):
+                time.sleep(BURST_IDLE_S)
+                res["stages_sustained_ms"][name] = time_alone(calls[name], 0, sustained=True,
+                                                              ms_hint=max(res["stages_ms"][name], 1e-3))
         time.sleep(BURST_IDLE_S)
     res["status"] = q.status_bits()
     return res
@@ -513,6 +537,12 @@ def summarize(res, peak_gbs):
         out["kernels"][s] = {"ms": round(ms, 5), "algorithmic_MB": round(ab[s] / 1e6, 2),
                              "GBps": round(gbs, 1), "frac_of_hbm_peak": round(gbs / peak_gbs, 4),
                              "frac_of_nominal_8TBps": round(gbs / NOMINAL_HBM_GBS, 4)}
+        if s in res.get("stages_sustained_ms", {}):
+            ms_s = res["stages_sustained_ms"][s]
+            out["kernels"][s]["ms_sustained"] = round(ms_s, 5)
+            out["kernels"][s]["frac_of_hbm_peak_sustained"] = round(ab[s] / ms_s / 1e6 / peak_gbs, 4)
+    if res.get("clocks") is not None:
+        out["clocks"] = res["clocks"]
     other = 32 if w.rng_bits == 16 else 16
     ms = res["encode_other_ms"]
     out["kernels"][f"encode_rng{other}"] = {
@@ -520,11 +550,15 @@ def summarize(res, peak_gbs):
         "frac_of_hbm_peak": round(ab["encode"] / ms / 1e6 / peak_gbs, 4), "note": "timed alone, not part of the step"}
     if "fused_select_ms" in res:
         ms = res["fused_select_ms"]
+        two = res["stages_ms"].get("select_scale", 0.0) + res["stages_ms"].get("encode", 0.0)
         out["kernels"]["select_encode"] = {
             "ms": round(ms, 5), "algorithmic_MB": round(ab["select_encode"] / 1e6, 2),
             "GBps": round(ab["select_encode"] / ms / 1e6, 1),
             "frac_of_hbm_peak": round(ab["select_encode"] / ms / 1e6 / peak_gbs, 4),
-            "note": "selection + encoding as one kernel, timed alone, not part of the step"}
+            "ms_of_the_two_kernels_it_replaces": round(two, 5),
+            "gradient_GBps_of_a_step_with_it": round(w.in_bytes / (res["ms"] - two + ms) / 1e6, 1),
+            "note": "selection + encoding as one call (one kernel for M <= 8: the gradients are read once; bound by "
+                    "instruction issue, not by memory), timed alone, not part of the step"}
     lev = {"i8": 1.0, "i4x2": 0.5, "i2x4": 0.25, "i6p": 0.75}[w.fmt]
     upd_bytes = lev * w.M * w.d + w.idx_bits / 8.0 * w.d + 16 * w.d      # levels, index, theta and momentum r/w
     ms = res["update_ms"]
@@ -542,19 +576,26 @@ def summarize(res, peak_gbs):
     return out
 
 
-def cpu_baseline(name, threads, max_coords):
-    """The oracle, as it stands, on the host cores, over the first `max_coords` coordinates of
-    the workload (all M workers, the segments that fall in that window)."""
-    from oracle import uq_oracle as o
+def cpu_sample(name, max_coords, threads):
+    """(workload, n, segment table, gradients) of the oracle's sample: the first n coordinates of the
+    workload, n = max_coords rounded down to whole segments where the workload has equal buckets."""
     w = wl.WORKLOADS[name]
     n = min(w.d, max_coords)
+    if w.bucket_elems and n < w.d:
+        n = max(1, n // w.bucket_elems) * w.bucket_elems           # whole buckets
     seg_full = wl.segment_offsets(w)
     seg = np.unique(np.concatenate([seg_full[seg_full < n], [n]])).astype(np.int64)
-    sub = wl.scaled(name, n) if n < w.d else w
+    sub = w
     if n < w.d:                                 # same recipe at the window's size
         import dataclasses
         sub = dataclasses.replace(w, d=n, segments="one")
     g = wl.generate(sub, threads=threads)[:, :n]
+    return w, n, seg, g
+
+
+def cpu_pass(w, seg, g, threads):
+    """One pass of the whole path through the oracle, as it stands; seconds."""
+    from oracle import uq_oracle as o
     o.set_threads(threads)
     norm = o.NORM_L2 if w.norm == wl.NORM_L2 else o.NORM_LINF
     t0 = time.perf_counter()
@@ -568,11 +609,24 @@ def cpu_baseline(name, threads, max_coords):
         lev = o.encode_single(g, W, w.s, w.seed, w.rng_bits, seg_off=seg)
         S = o.aggregate(lev)
         o.decode(S, w.M, W, s=w.s, seg_off=seg)
-    dt = time.perf_counter() - t0
+    return time.perf_counter() - t0
+
+
+def sample_text(w, n, seg):
+    if n == w.d:
+        return "full workload"
+    what = f"{len(seg) - 1} whole buckets" if w.bucket_elems else f"{len(seg) - 1} segments"
+    return f"first {n} of {w.d} coordinates ({what}) of all {w.M} workers"
+
+
+def cpu_baseline(name, threads, max_coords):
+    """The oracle on the host cores over a bounded sample of the workload."""
+    from oracle import uq_oracle as o
+    w, n, seg, g = cpu_sample(name, max_coords, threads)
+    dt = cpu_pass(w, seg, g, threads)
     in_bytes = w.M * n * (4 if w.dtype == wl.F32 else 2)
-    sample = "full workload" if n == w.d else f"first {n} of {w.d} coordinates of all {w.M} workers"
     return {"value": in_bytes / dt / 1e9, "unit": UNIT, "cores": o.get_threads(), "kind": "oracle",
-            "sample": sample, "seconds": round(dt, 3)}
+            "sample": sample_text(w, n, seg), "seconds": round(dt, 3)}
 
 
 def max_over_ranks(values, device):
@@ -590,6 +644,26 @@ def max_over_ranks(values, device):
 def whole_job_value(world, in_bytes, ms):
     """Gradient GB/s of the whole job: every one of `world` replicas processed in_bytes in ms."""
     return world * in_bytes / ms / 1e6
+
+
+def other_workloads(rng_bits):
+    """The workloads reported beside the headline one: the other four configurations, c2 on the
+    2-bit and 6-bit wires, and c3 with its shared index sent in 2, 4 and 8 bits."""
+    import dataclasses
+    base = {n: resolve_workload(n, None, rng_bits) for n in ("c1", "c2", "c3", "c4", "c5")}
+    return [
+        ("c1", base["c1"]), ("c2", base["c2"]), ("c3", base["c3"]), ("c4", base["c4"]), ("c5", base["c5"]),
+        ("c2_levels_2bit", resolve_workload("c2", None, rng_bits, "i2x4")),      # levels -1, 0, 1
+        ("c2_levels_6bit", resolve_workload("c2", None, rng_bits, "i6p")),
+        ("c3_idx2", base["c3"]),
+        ("c3_idx4", dataclasses.replace(base["c3"], idx_bits=4)),
+        ("c3_idx8", dataclasses.replace(base["c3"], idx_bits=8)),
+    ]
+
+
+def wire_bytes_per_coordinate(w):
+    """Bytes per coordinate and worker that the method puts on the wire: levels + shared index."""
+    return {"i8": 1.0, "i4x2": 0.5, "i2x4": 0.25, "i6p": 0.75}[w.fmt] + w.idx_bits / 8.0
 
 
 def gpu_main(args):
@@ -612,21 +686,19 @@ def gpu_main(args):
     threads = max(1, min(16, (os.cpu_count() or 8) // max(1, world)))
     peak, peak_kind = hbm_peak()
     name = args.workload
-    w = resolve_workload(name, args.d, args.rng_bits)
+    w = resolve_workload(name, args.d, args.rng_bits, args.levels)
 
-    sampler = ClockSampler(local)
-    sampler.start()
-    res = bench_workload(w, args.steps, args.warmup, barrier, threads, want_e2e=not args.no_e2e,
-                         randk_K=0 if args.no_extra else 10_000)
-    clocks = sampler.stop()
-    sustained = time_sustained(res["q"], res["g_dev"], w, res["ms"])     # after the clock record of the timed runs
-
+    res = bench_workload(w, args.steps, args.warmup, barrier, threads, want_e2e=not args.no_e2e, sustained=True,
+                         flush_between=w.in_bytes < (126 << 20), device_index=local)
+    clocks = res["clocks"]
     ms, e2e_ms = max_over_ranks([res["ms"], res["e2e_ms"] or float("nan")], "cuda")
     summ = summarize(res, peak)
     q = res["q"]
     dom = max(res["stages_ms"], key=lambda s: res["stages_ms"][s])
     ab = algorithmic_bytes(w)
     dom_gbs = ab[dom] / res["stages_ms"][dom] / 1e6
+    dom_sust = res.get("stages_sustained_ms", {}).get(dom)
+    per_coord = NCU_TRAFFIC_BYTES_PER_COORD.get((name, dom))
     line = {
         "metric": METRIC, "value": round(whole_job_value(world, w.in_bytes, ms), 2), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms, 5),
@@ -649,47 +721,54 @@ def gpu_main(args):
         "roofline": {
             "bound": "hbm", "kernel": dom, "achieved": round(dom_gbs, 1), "peak": peak, "unit": "GB/s",
             "frac": round(dom_gbs / peak, 4), "peak_kind": f"of {peak_kind}",
+            "frac_sustained": None if dom_sust is None else round(ab[dom] / dom_sust / 1e6 / peak, 4),
             "frac_of_nominal_8TBps": round(dom_gbs / NOMINAL_HBM_GBS, 4),
             "algorithmic_bytes_per_launch": int(ab[dom]),
             "avg_launch_ms": round(res["stages_ms"][dom], 5),
-            "traffic": NCU_TRAFFIC_BYTES.get(name) if args.d is None and dom == "encode" else None,
+            "avg_launch_ms_sustained": None if dom_sust is None else round(dom_sust, 5),
+            "traffic": None if per_coord is None else int(per_coord * w.d),
+            "traffic_note": None if per_coord is None else
+                            f"{per_coord} B per coordinate under ncu at a smaller d of the same recipe, times d",
         },
         "step_roofline": step_roofline(w, ms, peak),
         "kernels": summ["kernels"],
-        "sustained": sustained_summary(w, sustained),
+        "sustained": sustained_summary(w, res["sustained"]),
     }
-    if "randk" in res:
-        line["global_randk"] = res["randk"]
-    if "randk_two_scale" in res:
-        line["global_randk_two_scale"] = res["randk_two_scale"]
-    if "graph_stats" in res:
-        mean, med, lo = res["graph_stats"]
-        line["cuda_graph_replay"] = {"ms_per_step_mean": round(mean, 5), "ms_per_step_median": round(med, 5),
-                                     "ms_per_step_min": round(lo, 5), "replays": max(args.steps, 20),
-                                     "gradient_GBps_median": round(w.in_bytes / med / 1e6, 1),
-                                     "note": "the whole step captured once and replayed, each replay timed by itself"}
+    if "cold_l2" in summ:
+        line["cold_l2"], line["cuda_graph_warm_l2"] = summ["cold_l2"], summ["cuda_graph_warm_l2"]
     if rank == 0 and world == 1:
-        # the other four workloads (parity-test cases; reported for context, a few steps each)
+        # the other workloads (parity-test cases; reported for context, a few steps each)
         if not args.no_extra and args.d is None:
             extra = {}
-            import dataclasses
-            others = [(o_, resolve_workload(o_, None, args.rng_bits)) for o_ in ("c1", "c3", "c4", "c5")]
-            # c2 on the 2-bit wire (s = 1: levels -1, 0, 1, four per byte)
-            others.append(("c2_levels_2bit", dataclasses.replace(resolve_workload("c2", None, args.rng_bits),
-                                                                 fmt="i2x4", s=1, scales=(1,))))
-            for other, wo in others:
+            for other, wo in other_workloads(args.rng_bits):
+                if other == name:
+                    continue
                 del res, q
                 torch.cuda.empty_cache()
                 small = wo.in_bytes < (126 << 20)
                 res = bench_workload(wo, max(3, min(args.steps, 10)), 3, lambda: None, threads,
-                                     want_e2e=False, flush_between=small, sustained=True)
+                                     want_e2e=False, flush_between=small, sustained=True,
+                                     randk_K=10_000 if other == "c2" else 0, device_index=local)
                 q = res["q"]
                 extra[other] = summarize(res, peak)
                 extra[other]["status_word"] = res["status"]
+                extra[other]["rng_bits"] = wo.rng_bits
+                extra[other]["wire_bytes_per_coordinate_and_worker"] = wire_bytes_per_coordinate(wo)
+                if "randk" in res:
+                    extra[other]["global_randk"] = res["randk"]
+                if "randk_two_scale" in res:
+                    extra[other]["global_randk_two_scale"] = res["randk_two_scale"]
+                if "graph_stats" in res:
+                    mean, med, lo = res["graph_stats"]
+                    extra[other]["cuda_graph_replay"] = {
+                        "ms_per_step_mean": round(mean, 5), "ms_per_step_median": round(med, 5), "ms_per_step_min": round(lo, 5),
+                        "gradient_GBps_median": round(wo.in_bytes / med / 1e6, 1),
+                        "note": "the whole step captured once and replayed, each replay timed by itself"}
             line["other_workloads"] = extra
         if not args.no_cpu:
-            line["cpu_baseline"] = cpu_baseline(name, max(1, os.cpu_count() or 1), args.cpu_coords)
-            one = cpu_baseline(name, 1, max(1, min(w.d, args.cpu_coords) // 8))      # one thread, an eighth of the sample
+            cores = max(1, os.cpu_count() or 1)
+            line["cpu_baseline"] = cpu_baseline(name, cores, args.cpu_coords)
+            one = cpu_baseline(name, 1, max(1, args.cpu_coords // 16))      # one thread, a sixteenth of the sample
             line["cpu_baseline"]["single_thread"] = {"value": one["value"], "unit": UNIT, "sample": one["sample"],
                                                      "seconds": one["seconds"]}
     if rank == 0:
@@ -705,25 +784,25 @@ def gpu_main(args):
 def reference_main(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
-    w = wl.WORKLOADS[args.workload]
+    from oracle import uq_oracle as o
     threads = max(1, os.cpu_count() or 1)
-    n = min(w.d, args.ref_coords)
-    vals = []
+    w, n, seg, g = cpu_sample(args.workload, args.ref_coords, threads)      # the inputs are made once, outside the steps
+    secs = []
     for k in range(args.warmup + args.steps):
-        r = cpu_baseline(args.workload, threads, n)
+        dt = cpu_pass(w, seg, g, threads)
         if k >= args.warmup:
-            vals.append(r)
-    secs = statistics.fmean(v["seconds"] for v in vals)
+            secs.append(dt)
+    sec = statistics.fmean(secs)
     in_bytes = w.M * n * (4 if w.dtype == wl.F32 else 2)
-    value = in_bytes / secs / 1e9
+    value = in_bytes / sec / 1e9
+    sample = sample_text(w, n, seg)
     line = {
         "impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(secs * 1e3, 3),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(sec * 1e3, 3),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32" if w.dtype == wl.F32 else "bf16", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: CPU oracle on {vals[-1]['sample']}"},
-        "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "cores": vals[-1]["cores"], "kind": "oracle",
-                         "sample": vals[-1]["sample"]},
+        "config": {"workload": f"{args.workload}: CPU oracle on the {sample}; a step = one pass of the whole path over that sample"},
+        "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "cores": o.get_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": round(value, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
@@ -735,16 +814,17 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=sorted(wl.WORKLOADS))
-    ap.add_argument("--no-extra", action="store_true", help="skip the four context workloads")
+    ap.add_argument("--workload", default="c5", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--no-extra", action="store_true", help="skip the context workloads")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end timing")
     ap.add_argument("--d", type=int, default=None, help="run the workload's recipe at this smaller d (profiling)")
     ap.add_argument("--rng-bits", type=int, default=None, choices=[16, 32], help="override the draw width")
-    ap.add_argument("--cpu-coords", type=int, default=25_557_032,
-                    help="coordinates of the workload the CPU baseline covers")
-    ap.add_argument("--ref-coords", type=int, default=1 << 20,
-                    help="coordinates per step of the reference (oracle) arm")
+    ap.add_argument("--levels", default=None, choices=sorted(LEVEL_WIRES), help="override the level wire format")
+    ap.add_argument("--cpu-coords", type=int, default=2 * 13_107_200,
+                    help="coordinates of the workload the CPU baseline covers (c5: two whole 25 MiB buckets)")
+    ap.add_argument("--ref-coords", type=int, default=13_107_200,
+                    help="coordinates per step of the reference (oracle) arm (c5: one whole bucket)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":

@@ -111,9 +111,6 @@ const char *uq_error_string(int code);
 /* Bytes of device scratch uq_agree_scale needs for this layout (0 on a bad layout). */
 size_t uq_workspace_bytes(const uq_layout *layout);
 
-/* Bytes of device scratch uq_agree_scale_amax needs (its partials are finer; 0 on a bad layout). */
-size_t uq_workspace_bytes_amax(const uq_layout *layout);
-
 /* Bytes of a packed scale-index stream for this layout: worker_stride * idx_bits / 8. */
 size_t uq_index_bytes(const uq_layout *layout, int idx_bits);
 
@@ -165,23 +162,6 @@ int uq_agree_scale(const uq_layout *layout, const void *g, int norm, float *W, u
  */
 int uq_agree_scale_static(const uq_layout *layout, const void *g, int norm, float *W, uint32_t *status,
                           void *stream);
-
-/*
- * uq_agree_scale with a by-product for the multi-scale quantizer: amax[i] = max over the workers of
- * |g^m_i|, written while the gradients are read for the norms (Algorithm 2, line "MaxAllReduce
- * Norm").  The shared scale index of a coordinate depends on the gradients only through amax[i]
- * (binary32 multiplication by a positive constant is monotone, so the smallest own index over the
- * workers is the index of the largest magnitude), hence
- *     uq_select_scale_multi(layout with M = 1, g = amax, ...)
- * writes the indices that the call on all M rows writes, reading 1/M of the bytes.
- *   amax  out  [worker_stride] elements of layout->dtype, device, 16-byte aligned: the magnitude
- *              (sign bit clear) of the largest entry of coordinate i; elements d.. are padding
- * W may differ from uq_agree_scale's in the last bit (another fixed order of additions); the
- * workspace holds uq_workspace_bytes_amax(layout) bytes; every other argument and error is
- * uq_agree_scale's.
- */
-int uq_agree_scale_amax(const uq_layout *layout, const void *g, int norm, float *W, void *amax,
-                        uint32_t *status, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * Single-scale quantizer Q_s — Section "QSGDMaxNorm Quantization" (Eq. Q_s, definition of
@@ -239,12 +219,16 @@ int uq_encode_multi(const uq_layout *layout, const void *g, const float *W, cons
                     void *lev, uint32_t *status, void *stream);
 
 /*
- * uq_select_scale_multi followed by uq_encode_multi in one kernel — Algorithm 2 lines "Compute
- * coordinate scales", "Scale sharing" and "Quantize with s*".  For callers whose M workers are all
- * in this buffer: a thread reads the 8 coordinates of every worker once to form max_m |g^m_i|,
- * finds the shared indices, and quantizes every worker's coordinates with them, so the gradients
- * cross the memory interface once instead of twice.  idx and lev receive, bit for bit, what the two
- * separate calls write; arguments and errors are theirs.
+ * uq_select_scale_multi followed by uq_encode_multi as one call — Algorithm 2 lines "Compute
+ * coordinate scales", "Scale sharing" and "Quantize with s*" — for callers whose M workers are all
+ * in this buffer.  With M <= 8 it is one kernel: a CTA copies a tile of every worker's row into
+ * shared memory once, takes the maximum over the workers of every magnitude there, finds and stores
+ * the shared indices, and quantizes the workers' rows from the same copy, so the gradients cross
+ * the memory interface once instead of twice.  With more workers the two kernels run one after
+ * the other.  idx and lev receive, bit for bit, what the two separate calls write; arguments and
+ * errors are theirs.  On a B200 it takes about 15 % less time than the two calls (the gradients
+ * are read from memory once), but it is bound by instruction issue rather than by memory, so
+ * uq_step keeps the two streaming kernels and this call is the caller's choice.
  */
 int uq_select_encode_multi(const uq_layout *layout, const void *g, const float *W, const int32_t *scales,
                            int N, int idx_bits, uint64_t seed, int rng_bits, int fmt, uint8_t *idx,
@@ -280,7 +264,8 @@ int uq_decode(const uq_layout *layout, const void *src, int src_kind, int fmt, c
  * array of layout->M device pointers, lev_rows[m] = start of worker m's level row (16-byte
  * aligned, layout as the encoders write it).  The rows need not lie in one buffer, nor on this
  * GPU: a row in a peer GPU's memory that is mapped into this process (peer access, an IPC or
- * symmetric-memory mapping) is read with ordinary loads over NVLink while it is being summed, so
+ * symmetric-memory mapping) is read with ordinary loads over NVLink (on the coherent path, not the
+ * read-only one that the one-buffer call uses for its own memory) while it is being summed, so
  * "AllReduce gradients" + "Reconstruct gradient" of Algorithm 1 / 2 run as one kernel that pulls
  * the other workers' levels itself.  The caller orders the call after the peers' encoders (a
  * barrier between the processes); nothing in the kernel waits on another GPU.
@@ -357,7 +342,7 @@ int uq_step(const uq_layout *layout, const void *g, int norm, int s, const int32
  * Results: idx, lev, S_opt and out are bit for bit those of uq_step given the same W; W is added
  * up in another fixed order (L-inf: identical; L2: within one unit in the last place).
  * The wait at the barrier is bounded: a CTA that gives up sets UQ_STATUS_TIMEOUT and returns
- * (outputs then incomplete).
+ * (outputs then incomplete).  For that reason status must not be NULL here (UQ_ERR_BAD_ARG).
  * Errors: UQ_ERR_BAD_ARG, UQ_ERR_UNSUPPORTED, UQ_ERR_WORKSPACE, UQ_ERR_CUDA.
  */
 size_t uq_workspace_bytes_small(void);

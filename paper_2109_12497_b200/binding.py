@@ -25,10 +25,10 @@ UQ_STATUS_NONFINITE, UQ_STATUS_BAD_SEGMENTS, UQ_STATUS_SCALE_OVERFLOW, UQ_STATUS
 UQ_STATUS_TIMEOUT = 16
 
 EXPORTS = (
-    "uq_version", "uq_last_cuda_error", "uq_error_string", "uq_workspace_bytes", "uq_index_bytes", "uq_workspace_bytes_amax",
+    "uq_version", "uq_last_cuda_error", "uq_error_string", "uq_workspace_bytes", "uq_index_bytes",
     "uq_workspace_bytes_small",
     "uq_agree_scale", "uq_agree_scale_static", "uq_encode_single", "uq_select_scale_multi", "uq_encode_multi",
-    "uq_aggregate", "uq_decode", "uq_decode_update", "uq_randk_gather", "uq_randk_scatter", "uq_randk_update", "uq_index_min", "uq_decode_rows", "uq_select_encode_multi", "uq_agree_scale_amax", "uq_step",
+    "uq_aggregate", "uq_decode", "uq_decode_update", "uq_randk_gather", "uq_randk_scatter", "uq_randk_update", "uq_index_min", "uq_decode_rows", "uq_select_encode_multi", "uq_step",
     "uq_step_small",
 )
 
@@ -75,13 +75,10 @@ def lib() -> C.CDLL:
         L.uq_error_string.argtypes = [I]
         L.uq_workspace_bytes.restype = SZ
         L.uq_workspace_bytes.argtypes = [LP]
-        L.uq_workspace_bytes_amax.restype = SZ
-        L.uq_workspace_bytes_amax.argtypes = [LP]
         L.uq_index_bytes.restype = SZ
         L.uq_index_bytes.argtypes = [LP, I]
         L.uq_agree_scale.argtypes = [LP, P, I, P, P, P, SZ, P]
         L.uq_step.argtypes = [LP, P, I, I, P, I, I, U64, I, I, P, P, P, P, P, P, P, SZ, P]
-        L.uq_agree_scale_amax.argtypes = [LP, P, I, P, P, P, P, SZ, P]
         L.uq_step_small.argtypes = [LP, P, I, I, P, I, I, U64, I, I, P, P, P, P, P, P, P, SZ, P]
         L.uq_workspace_bytes_small.restype = SZ
         L.uq_workspace_bytes_small.argtypes = []
@@ -106,11 +103,20 @@ def lib() -> C.CDLL:
     return _lib
 
 
+def require_current_device(index: Optional[int], current: int, what: str = "tensor") -> None:
+    """Every call launches on the CURRENT device's current stream, so a tensor on another device
+    would hand that device a pointer it cannot use (a fault, or silent peer traffic): refuse."""
+    if index is None or index != current:
+        raise ValueError(f"uq: {what} lives on CUDA device {index}, but the current device is {current}; "
+                         f"make its device current first (torch.cuda.device / set_device)")
+
+
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
     if t is None:
         return None
     if not t.is_cuda:
         raise ValueError("uq: tensors must live on a CUDA device")
+    require_current_device(t.device.index, torch.cuda.current_device())
     return t.data_ptr()
 
 
@@ -153,8 +159,6 @@ class Layout:
     def workspace_bytes(self) -> int:
         return int(lib().uq_workspace_bytes(self.ref()))
 
-    def workspace_bytes_amax(self) -> int:
-        return int(lib().uq_workspace_bytes_amax(self.ref()))
 
     def index_bytes(self, idx_bits: int) -> int:
         return int(lib().uq_index_bytes(self.ref(), idx_bits))
@@ -367,17 +371,6 @@ def uq_select_encode_multi(layout: Layout, g: torch.Tensor, W: torch.Tensor, sca
         layout.ref(), _ptr(g), _ptr(W), arr, N, idx_bits, seed, rng_bits, fmt, _ptr(idx), _ptr(lev), _ptr(status),
         _stream()))
 
-
-def uq_agree_scale_amax(layout: Layout, g: torch.Tensor, norm: int, W: torch.Tensor, amax: torch.Tensor,
-                        status: Optional[torch.Tensor], workspace: torch.Tensor) -> None:
-    """uq_agree_scale that also writes amax[i] = max over the workers of |g[m, i]| (one row of
-    layout.worker_stride elements of g's dtype) for the selector to run on."""
-    layout.check_g(g)
-    layout.check_vec(W, torch.float32, layout.nseg, "W")
-    layout.check_vec(amax, layout.dtype, layout.worker_stride, "amax")
-    _check("uq_agree_scale_amax", lib().uq_agree_scale_amax(
-        layout.ref(), _ptr(g), norm, _ptr(W), _ptr(amax), _ptr(status), _ptr(workspace),
-        workspace.numel() * workspace.element_size(), _stream()))
 
 
 def uq_step(layout: Layout, g: torch.Tensor, norm: int, s: int, scales: Optional[Sequence[int]], idx_bits: int,

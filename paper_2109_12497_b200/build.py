@@ -13,7 +13,7 @@ CSRC = PKG / "csrc"
 INCLUDE = PKG.parent / "include"
 LIB = PKG / "libuq_b200.so"
 
-SOURCES = ["uq_api.cu", "uq_agree.cu", "uq_select.cu", "uq_encode.cu", "uq_encode_f32_r16.cu", "uq_encode_f32_r32.cu", "uq_encode_bf16_r16.cu", "uq_encode_bf16_r32.cu", "uq_decode.cu", "uq_randk.cu", "uq_select_encode.cu", "uq_agree_amax.cu", "uq_small.cu", "uq_small_multi.cu"]
+SOURCES = ["uq_api.cu", "uq_agree.cu", "uq_select.cu", "uq_encode.cu", "uq_encode_f32_r16.cu", "uq_encode_f32_r32.cu", "uq_encode_bf16_r16.cu", "uq_encode_bf16_r32.cu", "uq_decode.cu", "uq_randk.cu", "uq_small.cu", "uq_small_multi.cu"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",

@@ -169,19 +169,6 @@ static cudaError_t launch(const uq_layout &L, const void *g, float *W, uint32_t 
 
 int64_t norm_tiles(int64_t d) { return (d + kNormTile - 1) / kNormTile; }
 
-// The second launch alone, for the kernel that fills the same scratch slots together with amax.
-cudaError_t launch_norm_finalize(const uq_layout &L, int norm, const double *part, int64_t ntiles, int tile_coords,
-                                 float *W, uint32_t *status, cudaStream_t st)
-{
-    if (norm == UQ_NORM_L2)
-        launch_k(norm_finalize_kernel<UQ_NORM_L2>, L.nseg, kThreads, st, part, L.M, L.d, L.nseg, L.seg_off, ntiles, W, status,
-                 tile_coords);
-    else
-        launch_k(norm_finalize_kernel<UQ_NORM_LINF>, L.nseg, kThreads, st, part, L.M, L.d, L.nseg, L.seg_off, ntiles, W, status,
-                 tile_coords);
-    return cudaGetLastError();
-}
-
 cudaError_t launch_agree_scale(const uq_layout &L, const void *g, int norm, float *W, uint32_t *status,
                                void *workspace, cudaStream_t st)
 {

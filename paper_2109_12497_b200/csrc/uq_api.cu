@@ -4,11 +4,8 @@
 
 namespace uq {
 int64_t norm_tiles(int64_t d);
-int64_t norm_tiles_amax(int64_t d);
 cudaError_t launch_agree_scale(const uq_layout &L, const void *g, int norm, float *W, uint32_t *status,
                                void *workspace, cudaStream_t st);
-cudaError_t launch_agree_scale_amax(const uq_layout &L, const void *g, int norm, float *W, void *amax, uint32_t *status,
-                                    void *workspace, cudaStream_t st);
 cudaError_t launch_encode(const uq_layout &L, const void *g, const float *W, const ScaleSet &scales,
                           const uint8_t *idx, int idx_bits, uint64_t seed, int rng_bits, int fmt, void *lev,
                           uint32_t *status, cudaStream_t st);
@@ -131,12 +128,6 @@ size_t uq_workspace_bytes(const uq_layout *L)
     return (size_t)L->M * (size_t)(uq::norm_tiles(L->d) + L->nseg) * sizeof(double);
 }
 
-size_t uq_workspace_bytes_amax(const uq_layout *L)
-{
-    if (!layout_ok(L)) return 0;
-    return (size_t)L->M * (size_t)(uq::norm_tiles_amax(L->d) + L->nseg) * sizeof(double);
-}
-
 size_t uq_index_bytes(const uq_layout *L, int idx_bits)
 {
     if (!layout_ok(L) || !idx_bits_ok(idx_bits)) return 0;
@@ -152,17 +143,6 @@ int uq_agree_scale(const uq_layout *L, const void *g, int norm, float *W, uint32
     if (workspace == nullptr || !aligned(workspace, 8) || workspace_bytes < uq_workspace_bytes(L))
         return UQ_ERR_WORKSPACE;
     return finish(uq::launch_agree_scale(*L, g, norm, W, status, workspace, (cudaStream_t)stream));
-}
-
-int uq_agree_scale_amax(const uq_layout *L, const void *g, int norm, float *W, void *amax, uint32_t *status,
-                        void *workspace, size_t workspace_bytes, void *stream)
-{
-    if (!layout_ok(L) || W == nullptr || !aligned(W, 4) || !aligned(status, 4)) return UQ_ERR_BAD_ARG;
-    if (norm != UQ_NORM_L2 && norm != UQ_NORM_LINF) return UQ_ERR_BAD_ARG;
-    if (L->d > 0 && (g == nullptr || amax == nullptr || !aligned(g, 16) || !aligned(amax, 16))) return UQ_ERR_BAD_ARG;
-    if (workspace == nullptr || !aligned(workspace, 8) || workspace_bytes < uq_workspace_bytes_amax(L))
-        return UQ_ERR_WORKSPACE;
-    return finish(uq::launch_agree_scale_amax(*L, g, norm, W, amax, status, workspace, (cudaStream_t)stream));
 }
 
 int uq_encode_single(const uq_layout *L, const void *g, const float *W, int s, uint64_t seed, int rng_bits,
@@ -325,6 +305,7 @@ int uq_step_small(const uq_layout *L, const void *g, int norm, int s, const int3
 {
     uq::ScaleSet set;
     if (!layout_ok(L) || W == nullptr || !aligned(W, 4) || !aligned(status, 4)) return UQ_ERR_BAD_ARG;
+    if (status == nullptr) return UQ_ERR_BAD_ARG;      // a wait that runs out must be able to say so
     if (norm != UQ_NORM_L2 && norm != UQ_NORM_LINF) return UQ_ERR_BAD_ARG;
     if (scales != nullptr && !scales_ok(scales, N, idx_bits, &set)) return UQ_ERR_BAD_ARG;
     if (!fmt_ok(fmt, scales != nullptr ? set.s[0] : s) || (rng_bits != 32 && rng_bits != 16)) return UQ_ERR_BAD_ARG;

@@ -6,6 +6,8 @@
 // the fp32 average (and, on request, the int32 sums).  A thread owns 16 coordinates of int8 levels
 // (16 B of every worker's stream) or 32 coordinates of the packed formats (16 B of 4-bit, 8 B of
 // 2-bit, 16 + 8 B of the two planes of 6-bit levels).
+#include <type_traits>
+
 #include "uq_device.cuh"
 
 namespace uq {
@@ -25,7 +27,7 @@ struct DecodeParams {
     float *mom;               // momentum buffer, updated in place; NULL for plain SGD
     float lr, mu, wd;         // step size, momentum factor, weight decay
     // ROWS variant: where each worker's level row starts (rows need not be one buffer, nor all on
-    // this GPU: a peer's row is read with ordinary loads over NVLink); lev is unused then
+    // this GPU: a peer's row is read with ordinary coherent loads over NVLink); lev is unused then
     const void *rows[UQ_MAX_WORKERS];
 };
 
@@ -60,8 +62,12 @@ template <int FMT> struct Unit;
 template <> struct Unit<UQ_FMT_I8> {
     static constexpr int C = 16;
     using Q = uint4;                                             // one worker's levels of the unit
-    // row = start of the worker's level row, i = first coordinate of the unit
-    static __device__ __forceinline__ Q load(const char *row, int64_t i, int64_t) { return ld_stream(row + i); }
+    // row = start of the worker's level row, i = first coordinate of the unit; PEER: the row may be
+    // another GPU's memory (coherent loads instead of the read-only path)
+    template <bool PEER> static __device__ __forceinline__ Q load(const char *row, int64_t i, int64_t)
+    {
+        return PEER ? ld_coherent(row + i) : ld_stream(row + i);
+    }
     // Bytes are biased to unsigned (x ^ 0x80) and added in 16-bit lanes: two lanes per word,
     // M <= 64 workers * 255 < 2^16.  lane layout of word w: even = bytes 0,2; odd = bytes 1,3.
     uint32_t even[4] = {0, 0, 0, 0}, odd[4] = {0, 0, 0, 0};
@@ -75,15 +81,17 @@ template <> struct Unit<UQ_FMT_I8> {
             odd[k] += (b >> 8) & 0x00FF00FFu;
         }
     }
-    __device__ __forceinline__ void finish(int M, int (&s)[16]) const
+    __device__ __forceinline__ void prepare() {}
+    // the sums of coordinates E0 .. E0 + 7 of the unit (E0 a multiple of 8)
+    template <int E0> __device__ __forceinline__ void sums8(int M, int (&s)[8]) const
     {
         const int bias = 128 * M;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            s[4 * k + 0] = (int)(even[k] & 0xFFFFu) - bias;
-            s[4 * k + 1] = (int)(odd[k] & 0xFFFFu) - bias;
-            s[4 * k + 2] = (int)(even[k] >> 16) - bias;
-            s[4 * k + 3] = (int)(odd[k] >> 16) - bias;
+        for (int k = 0; k < 2; ++k) {
+            s[4 * k + 0] = (int)(even[E0 / 4 + k] & 0xFFFFu) - bias;
+            s[4 * k + 1] = (int)(odd[E0 / 4 + k] & 0xFFFFu) - bias;
+            s[4 * k + 2] = (int)(even[E0 / 4 + k] >> 16) - bias;
+            s[4 * k + 3] = (int)(odd[E0 / 4 + k] >> 16) - bias;
         }
     }
 };
@@ -91,7 +99,10 @@ template <> struct Unit<UQ_FMT_I8> {
 template <> struct Unit<UQ_FMT_I4X2> {
     static constexpr int C = 32;
     using Q = uint4;
-    static __device__ __forceinline__ Q load(const char *row, int64_t i, int64_t) { return ld_stream(row + (i >> 1)); }
+    template <bool PEER> static __device__ __forceinline__ Q load(const char *row, int64_t i, int64_t)
+    {
+        return PEER ? ld_coherent(row + (i >> 1)) : ld_stream(row + (i >> 1));
+    }
     // Nibbles are biased to unsigned (x ^ 8) and added in byte lanes for up to 16 workers
     // (16 * 15 < 256), then widened into 16-bit lanes.
     uint32_t lo8[4] = {0, 0, 0, 0}, hi8[4] = {0, 0, 0, 0};       // byte lanes: even / odd nibbles
@@ -120,50 +131,68 @@ template <> struct Unit<UQ_FMT_I4X2> {
         }
         if (++pending == 16) flush();
     }
-    __device__ __forceinline__ void finish(int M, int (&s)[32])
+    __device__ __forceinline__ void prepare() { flush(); }
+    template <int E0> __device__ __forceinline__ void sums8(int M, int (&s)[8]) const
     {
-        flush();
         const int bias = 8 * M;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            s[8 * k + 0] = (int)(acc[k][0] & 0xFFFFu) - bias;
-            s[8 * k + 4] = (int)(acc[k][0] >> 16) - bias;
-            s[8 * k + 2] = (int)(acc[k][1] & 0xFFFFu) - bias;
-            s[8 * k + 6] = (int)(acc[k][1] >> 16) - bias;
-            s[8 * k + 1] = (int)(acc[k][2] & 0xFFFFu) - bias;
-            s[8 * k + 5] = (int)(acc[k][2] >> 16) - bias;
-            s[8 * k + 3] = (int)(acc[k][3] & 0xFFFFu) - bias;
-            s[8 * k + 7] = (int)(acc[k][3] >> 16) - bias;
-        }
+        constexpr int k = E0 / 8;
+        s[0] = (int)(acc[k][0] & 0xFFFFu) - bias;
+        s[4] = (int)(acc[k][0] >> 16) - bias;
+        s[2] = (int)(acc[k][1] & 0xFFFFu) - bias;
+        s[6] = (int)(acc[k][1] >> 16) - bias;
+        s[1] = (int)(acc[k][2] & 0xFFFFu) - bias;
+        s[5] = (int)(acc[k][2] >> 16) - bias;
+        s[3] = (int)(acc[k][3] & 0xFFFFu) - bias;
+        s[7] = (int)(acc[k][3] >> 16) - bias;
     }
 };
 
 template <> struct Unit<UQ_FMT_I2X4> {
     static constexpr int C = 32;
     using Q = uint2;
-    static __device__ __forceinline__ Q load(const char *row, int64_t i, int64_t) { return ld_stream64(row + (i >> 2)); }
-    // 2-bit fields are biased to unsigned (x ^ 2, so 1..3) and added in byte lanes: field t of
-    // every byte of word w goes to acc[w][t]; 64 workers * 3 < 256, so a byte lane never carries.
+    template <bool PEER> static __device__ __forceinline__ Q load(const char *row, int64_t i, int64_t)
+    {
+        return PEER ? ld_coherent64(row + (i >> 2)) : ld_stream64(row + (i >> 2));
+    }
+    // 2-bit fields are biased to unsigned (x ^ 2, so 1..3).  The even and the odd fields of a word
+    // are first added in 4-bit lanes (two masks, one shift and two additions per word and worker)
+    // for up to 4 workers (4 * 3 < 16), then widened into byte lanes: field t of every byte of
+    // word w goes to acc[w][t]; 64 workers * 3 < 256, so a byte lane never carries.
     uint32_t acc[2][4] = {};
+    uint32_t ev4[2] = {0, 0}, od4[2] = {0, 0};                 // 4-bit lanes: fields 0, 2, .. / 1, 3, .. of each word
+    int pending = 0;
+    __device__ __forceinline__ void flush()
+    {
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            acc[k][0] += ev4[k] & 0x0F0F0F0Fu;                   // nibble 2y of the even lanes = field 4y
+            acc[k][2] += (ev4[k] >> 4) & 0x0F0F0F0Fu;            // nibble 2y + 1 = field 4y + 2
+            acc[k][1] += od4[k] & 0x0F0F0F0Fu;                   // field 4y + 1
+            acc[k][3] += (od4[k] >> 4) & 0x0F0F0F0Fu;            // field 4y + 3
+            ev4[k] = 0; od4[k] = 0;
+        }
+        pending = 0;
+    }
     __device__ __forceinline__ void add(const uint2 &q)
     {
         const uint32_t w[2] = { q.x, q.y };
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
             const uint32_t b = w[k] ^ 0xAAAAAAAAu;
-#pragma unroll
-            for (int t = 0; t < 4; ++t) acc[k][t] += (b >> (2 * t)) & 0x03030303u;
+            ev4[k] += b & 0x33333333u;
+            od4[k] += (b >> 2) & 0x33333333u;
         }
+        if (++pending == 4) flush();
     }
-    __device__ __forceinline__ void finish(int M, int (&s)[32]) const
+    __device__ __forceinline__ void prepare() { flush(); }
+    template <int E0> __device__ __forceinline__ void sums8(int M, int (&s)[8]) const
     {
         const int bias = 2 * M;
+        constexpr int k = E0 / 16, y0 = (E0 % 16) / 4;
 #pragma unroll
-        for (int k = 0; k < 2; ++k)
+        for (int y = 0; y < 2; ++y)
 #pragma unroll
-            for (int y = 0; y < 4; ++y)
-#pragma unroll
-                for (int t = 0; t < 4; ++t) s[16 * k + 4 * y + t] = (int)((acc[k][t] >> (8 * y)) & 0xFFu) - bias;
+            for (int t = 0; t < 4; ++t) s[4 * y + t] = (int)((acc[k][t] >> (8 * (y0 + y))) & 0xFFu) - bias;
     }
 };
 
@@ -172,11 +201,11 @@ template <> struct Unit<UQ_FMT_I2X4> {
 template <> struct Unit<UQ_FMT_I6P> {
     static constexpr int C = 32;
     struct Q { uint4 n; uint2 c; };
-    static __device__ __forceinline__ Q load(const char *row, int64_t i, int64_t stride)
+    template <bool PEER> static __device__ __forceinline__ Q load(const char *row, int64_t i, int64_t stride)
     {
         Q q;
-        q.n = ld_stream(row + (i >> 1));
-        q.c = ld_stream64(row + (stride >> 1) + (i >> 2));
+        q.n = PEER ? ld_coherent(row + (i >> 1)) : ld_stream(row + (i >> 1));
+        q.c = PEER ? ld_coherent64(row + (stride >> 1) + (i >> 2)) : ld_stream64(row + (stride >> 1) + (i >> 2));
         return q;
     }
     uint32_t lo8[4] = {0, 0, 0, 0}, hi8[4] = {0, 0, 0, 0};       // nibble plane, byte lanes: even / odd nibbles
@@ -212,27 +241,22 @@ template <> struct Unit<UQ_FMT_I6P> {
             for (int t = 0; t < 4; ++t) cr[k][t] += (b >> (2 * t)) & 0x03030303u;
         }
     }
-    __device__ __forceinline__ void finish(int M, int (&s)[32])
+    __device__ __forceinline__ void prepare() { flush(); }
+    template <int E0> __device__ __forceinline__ void sums8(int M, int (&s)[8]) const
     {
-        flush();
-        int lo[32];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            lo[8 * k + 0] = (int)(acc[k][0] & 0xFFFFu); lo[8 * k + 4] = (int)(acc[k][0] >> 16);
-            lo[8 * k + 2] = (int)(acc[k][1] & 0xFFFFu); lo[8 * k + 6] = (int)(acc[k][1] >> 16);
-            lo[8 * k + 1] = (int)(acc[k][2] & 0xFFFFu); lo[8 * k + 5] = (int)(acc[k][2] >> 16);
-            lo[8 * k + 3] = (int)(acc[k][3] & 0xFFFFu); lo[8 * k + 7] = (int)(acc[k][3] >> 16);
-        }
+        constexpr int kn = E0 / 8;                                   // word of the nibble plane
+        int lo[8];
+        lo[0] = (int)(acc[kn][0] & 0xFFFFu); lo[4] = (int)(acc[kn][0] >> 16);
+        lo[2] = (int)(acc[kn][1] & 0xFFFFu); lo[6] = (int)(acc[kn][1] >> 16);
+        lo[1] = (int)(acc[kn][2] & 0xFFFFu); lo[5] = (int)(acc[kn][2] >> 16);
+        lo[3] = (int)(acc[kn][3] & 0xFFFFu); lo[7] = (int)(acc[kn][3] >> 16);
         const int bias = 2 * M;
+        constexpr int k = E0 / 16, y0 = (E0 % 16) / 4;                // word and bytes of the 2-bit plane
 #pragma unroll
-        for (int k = 0; k < 2; ++k)
+        for (int y = 0; y < 2; ++y)
 #pragma unroll
-            for (int y = 0; y < 4; ++y)
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    const int e = 16 * k + 4 * y + t;
-                    s[e] = 16 * ((int)((cr[k][t] >> (8 * y)) & 0xFFu) - bias) + lo[e];
-                }
+            for (int t = 0; t < 4; ++t)
+                s[4 * y + t] = 16 * ((int)((cr[k][t] >> (8 * (y0 + y))) & 0xFFu) - bias) + lo[4 * y + t];
     }
 };
 
@@ -263,13 +287,13 @@ __global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const __grid
             Q q[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k)
-                q[k] = U::load(ROWS ? (const char *)p.rows[m + k] : (const char *)p.lev + (size_t)(m + k) * row_bytes, i,
-                               p.stride);
+                q[k] = U::template load<ROWS>(ROWS ? (const char *)p.rows[m + k] : (const char *)p.lev + (size_t)(m + k) * row_bytes,
+                                              i, p.stride);
 #pragma unroll
             for (int k = 0; k < 8; ++k) unit.add(q[k]);
         }
         for (; m < p.M; ++m)
-            unit.add(U::load(ROWS ? (const char *)p.rows[m] : (const char *)p.lev + (size_t)m * row_bytes, i, p.stride));
+            unit.add(U::template load<ROWS>(ROWS ? (const char *)p.rows[m] : (const char *)p.lev + (size_t)m * row_bytes, i, p.stride));
         if (MULTI && p.out != nullptr) {
             // idx bits of coordinates i..i+C-1 start at byte i*IB/8 (a multiple of 4 bytes, of 2 for 16 bits)
             if (C * IB == 16) {
@@ -282,85 +306,90 @@ __global__ void __launch_bounds__(kThreads) aggregate_decode_kernel(const __grid
         }
     }
 
-    int s[C];
-    unit.finish(p.M, s);
+    // The sums leave the accumulators eight coordinates at a time: each group is reconstructed,
+    // stored (256 bits per array) and forgotten, which keeps the registers of a thread low enough for
+    // more CTAs per SM than 32 sums and 32 values held at once would allow.
+    unit.prepare();
     const bool full = i + C <= p.d;
-    if (p.S != nullptr && active) {
-        if (full) {
-#pragma unroll
-            for (int e = 0; e < C; e += 8) st_stream256(p.S + i + e, *(const uint32_t(*)[8])(s + e));
-        } else {
-            for (int e = 0; e < C; ++e)
-                if (i + e < p.d) p.S[i + e] = s[e];
-        }
-    }
-    if (p.out == nullptr && !UPDATE) return;
-
+    const bool want_values = p.out != nullptr || UPDATE;
     // every warp looks up the segment of its own row of 32*C coordinates; lane k holds the
     // reconstruction factor of scale k (single-scale: every lane holds the same factor)
     const int64_t row1 = min(row0 + 32 * C, p.d);
-    const int j0 = warp_find_segment(p.seg_off, p.nseg, row0);
-    float r[C];
-    if (segment_end(p.seg_off, p.nseg, j0, p.d) >= row1) {
-        const float c_lane = decode_factor(__ldg(p.W + j0), p.scales.s[lane & (UQ_MAX_SCALES - 1)], p.M);
-#pragma unroll
-        for (int e = 0; e < C; ++e) {
-            const int k = MULTI ? (kw[(e * IB) >> 5] >> ((e * IB) & 31)) & ((1 << IB) - 1) : 0;
-            const float c = MULTI ? __shfl_sync(0xFFFFFFFFu, c_lane, active ? k : 0) : c_lane;
-            r[e] = __fmul_rn((float)s[e], c);
-        }
-    } else if (active) {
-        int j = j0;                              // the row's first segment; walk on from there
-        for (int e = 0; e < C; ++e) {
-            r[e] = 0.0f;
-            if (i + e >= p.d) continue;
-            j = advance_segment(p.seg_off, p.nseg, j, i + e);
-            const int k = MULTI ? index_at<IB>(p.idx, i + e) : 0;
-            r[e] = __fmul_rn((float)s[e], decode_factor(__ldg(p.W + j), p.scales.s[k & (UQ_MAX_SCALES - 1)], p.M));
-        }
+    int j = 0;
+    bool uniform = true;
+    float c_lane = 0.0f;
+    if (want_values) {
+        j = warp_find_segment(p.seg_off, p.nseg, row0);
+        uniform = segment_end(p.seg_off, p.nseg, j, p.d) >= row1;
+        if (uniform) c_lane = decode_factor(__ldg(p.W + j), p.scales.s[lane & (UQ_MAX_SCALES - 1)], p.M);
     }
-    if (!active) return;
-    if (UPDATE) {
-        // Algorithm 1 / 2, line "Update parameters", fused: the reconstructed gradient goes straight
-        // from registers into the parameters (and the momentum buffer)
-        const bool has_mom = p.mom != nullptr;
+    const bool has_mom = UPDATE && p.mom != nullptr;
+    auto group = [&](auto e0_tag) {
+        constexpr int E0 = decltype(e0_tag)::value;
+        int s[8];
+        unit.template sums8<E0>(p.M, s);
+        if (p.S != nullptr && active) {
+            if (full) {
+                st_stream256(p.S + i + E0, *(const uint32_t(*)[8])s);
+            } else {
+                for (int e = 0; e < 8; ++e)
+                    if (i + E0 + e < p.d) p.S[i + E0 + e] = s[e];
+            }
+        }
+        if (!want_values) return;
+        float r[8];
+        if (uniform) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int k = MULTI ? (kw[((E0 + e) * IB) >> 5] >> (((E0 + e) * IB) & 31)) & ((1 << IB) - 1) : 0;
+                const float c = MULTI ? __shfl_sync(0xFFFFFFFFu, c_lane, active ? k : 0) : c_lane;
+                r[e] = __fmul_rn((float)s[e], c);
+            }
+        } else if (active) {                       // a boundary inside the row: walk on from segment j
+            for (int e = 0; e < 8; ++e) {
+                r[e] = 0.0f;
+                if (i + E0 + e >= p.d) continue;
+                j = advance_segment(p.seg_off, p.nseg, j, i + E0 + e);
+                const int k = MULTI ? index_at<IB>(p.idx, i + E0 + e) : 0;
+                r[e] = __fmul_rn((float)s[e], decode_factor(__ldg(p.W + j), p.scales.s[k & (UQ_MAX_SCALES - 1)], p.M));
+            }
+        }
+        if (!active) return;
+        if (UPDATE) {
+            // Algorithm 1 / 2, line "Update parameters", fused: the reconstructed gradient goes straight
+            // from registers into the parameters (and the momentum buffer), 8 coordinates as one
+            // 256-bit access per array: a lane's 32 bytes are one whole sector
+            if (full) {
+                float th[8], bf[8] = {};
+                ld256(p.theta + i + E0, th);
+                if (has_mom) ld256(p.mom + i + E0, bf);
+#pragma unroll
+                for (int t = 0; t < 8; ++t) sgd_coordinate(r[t], th[t], bf[t], has_mom, p.lr, p.mu, p.wd);
+                st256(p.theta + i + E0, th);
+                if (has_mom) st256(p.mom + i + E0, bf);
+            } else {
+                for (int e = 0; e < 8; ++e) {
+                    if (i + E0 + e >= p.d) break;
+                    float th = p.theta[i + E0 + e], bf = has_mom ? p.mom[i + E0 + e] : 0.0f;
+                    sgd_coordinate(r[e], th, bf, has_mom, p.lr, p.mu, p.wd);
+                    p.theta[i + E0 + e] = th;
+                    if (has_mom) p.mom[i + E0 + e] = bf;
+                }
+            }
+        }
+        if (p.out == nullptr) return;
         if (full) {
-            // 16 coordinates at a time as 256-bit accesses: a lane's 32 bytes are one whole sector,
-            // so nothing depends on L1 keeping the other half of a sector until the next access
-#pragma unroll
-            for (int e0 = 0; e0 < C; e0 += 16) {
-                float th[2][8], bf[2][8] = {};
-#pragma unroll
-                for (int k = 0; k < 2; ++k) {
-                    ld256(p.theta + i + e0 + 8 * k, th[k]);
-                    if (has_mom) ld256(p.mom + i + e0 + 8 * k, bf[k]);
-                }
-#pragma unroll
-                for (int k = 0; k < 2; ++k) {
-#pragma unroll
-                    for (int t = 0; t < 8; ++t)
-                        sgd_coordinate(r[e0 + 8 * k + t], th[k][t], bf[k][t], has_mom, p.lr, p.mu, p.wd);
-                    st256(p.theta + i + e0 + 8 * k, th[k]);
-                    if (has_mom) st256(p.mom + i + e0 + 8 * k, bf[k]);
-                }
-            }
+            st_stream256(p.out + i + E0, *(const uint32_t(*)[8])r);
         } else {
-            for (int e = 0; e < C; ++e) {
-                if (i + e >= p.d) break;
-                float th = p.theta[i + e], bf = has_mom ? p.mom[i + e] : 0.0f;
-                sgd_coordinate(r[e], th, bf, has_mom, p.lr, p.mu, p.wd);
-                p.theta[i + e] = th;
-                if (has_mom) p.mom[i + e] = bf;
-            }
+            for (int e = 0; e < 8; ++e)
+                if (i + E0 + e < p.d) p.out[i + E0 + e] = r[e];
         }
-    }
-    if (p.out == nullptr) return;
-    if (full) {
-#pragma unroll
-        for (int e = 0; e < C; e += 8) st_stream256(p.out + i + e, *(const uint32_t(*)[8])(r + e));
-    } else {
-        for (int e = 0; e < C; ++e)
-            if (i + e < p.d) p.out[i + e] = r[e];
+    };
+    group(std::integral_constant<int, 0>());
+    group(std::integral_constant<int, 8>());
+    if (C > 16) {
+        group(std::integral_constant<int, (C > 16 ? 16 : 0)>());
+        group(std::integral_constant<int, (C > 16 ? 24 : 0)>());
     }
 }
 

@@ -26,14 +26,15 @@ __device__ __forceinline__ void grid_dependency_prologue()
 }
 
 template <typename... P, typename... A>
-inline void launch_k(void (*kernel)(P...), dim3 grid, dim3 block, cudaStream_t st, A &&...args)
+inline void launch_k_smem(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem_bytes, cudaStream_t st, A &&...args)
 {
 #ifdef UQ_NO_PDL
-    kernel<<<grid, block, 0, st>>>(static_cast<A &&>(args)...);
+    kernel<<<grid, block, smem_bytes, st>>>(static_cast<A &&>(args)...);
 #else
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -42,6 +43,12 @@ inline void launch_k(void (*kernel)(P...), dim3 grid, dim3 block, cudaStream_t s
     cfg.numAttrs = 1;
     cudaLaunchKernelEx(&cfg, kernel, static_cast<A &&>(args)...);    // an error stays for cudaGetLastError()
 #endif
+}
+
+template <typename... P, typename... A>
+inline void launch_k(void (*kernel)(P...), dim3 grid, dim3 block, cudaStream_t st, A &&...args)
+{
+    launch_k_smem(kernel, grid, block, 0, st, static_cast<A &&>(args)...);
 }
 
 constexpr int kThreads = 256;            // threads per CTA in every streaming kernel
@@ -84,7 +91,32 @@ __device__ __forceinline__ uint2 ld_stream64(const void *p)
     return v;
 }
 
+// The same loads on the coherent path (no .nc): for memory that another GPU wrote (a peer's rows
+// read over NVLink), which must not be assumed read-only or served from a stale non-coherent line.
+__device__ __forceinline__ uint4 ld_coherent(const void *p)
+{
+    uint4 v;
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint2 ld_coherent64(const void *p)
+{
+    uint2 v;
+    asm volatile("ld.global.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p) : "memory");
+    return v;
+}
+
 template <typename T> __device__ __forceinline__ void st_stream(T *p, T v) { __stcs(p, v); }
+
+// 16 bytes from global memory straight into shared memory (no register in between); the copies of
+// a thread are complete for that thread after copy_async_wait().
+__device__ __forceinline__ void copy_async16(void *smem_dst, const void *gmem_src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
+                 : "memory");
+}
+__device__ __forceinline__ void copy_async_wait() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
 // 256-bit streaming load / store (sm_100 and later): 32 bytes per lane in one instruction.
 // The address must be 32-byte aligned.

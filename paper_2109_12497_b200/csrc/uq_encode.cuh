@@ -13,26 +13,23 @@
 // reads only g^m plus the agreed values W and idx.
 #pragma once
 #include "uq_device.cuh"
+#include "uq_select.cuh"
 #include "uq_unit.cuh"
 
 namespace uq {
 
 struct EncodeParams {
-    const void *g;
+    SelectView v;             // g, W, seg_off, d, stride, nseg, M, scales (single-scale: every entry is s) and
+                              // s_hat = (float) of the smallest scale: the largest level
     void *lev;
-    const float *W;
-    const int64_t *seg_off;
-    const uint8_t *idx;
+    uint8_t *idx;             // shared scale indices: read, or (select) written by this launch
     uint32_t *status;
-    int64_t d, stride;
-    int32_t nseg, M;
+    int32_t select;           // multi-scale: 1 = find the shared indices here instead of reading them
     int32_t worker0;          // number, in the whole job, of the worker in row 0 (keys the draws)
     int64_t coord0;           // index, in the whole gradient, of coordinate 0 (keys the draws)
     int64_t ntiles;
     uint32_t main_blocks;     // CTAs that own tiles; the CTAs after them own rows crossed by boundaries
     uint32_t groups;          // CTAs per tile: ceil(M / kWorkerGroup)
-    float cap;                // (float) of the smallest scale: the largest level
-    ScaleSet scales;          // single-scale: every entry is s
     PhiloxKey key;            // the ten round keys of the seed
     uint32_t blk_hi;          // high word of the Philox block numbers the table below was made for
     PhiloxWorkerPart wpart[UQ_MAX_WORKERS];   // per-worker words of the first two Philox rounds (row m)
@@ -55,20 +52,24 @@ template <int DT, int RNG> struct EncodeShape {
 // then holds the end and the scale of segment (first + L), and a coordinate's segment is the
 // number of ends at or before it, counted with shuffles: no dependent loads per coordinate.
 // Rare (a few rows per segment), so kept out of line.
+// own_idx (select mode, rows owned by a CTA that did not select for them): the warp finds the
+// shared indices of its row itself (thr: the warp's 2 * UQ_MAX_SCALES words of shared memory) instead
+// of reading them.
 template <int DT, int FMT, int RNG, int IDXB>
-__device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, int64_t a, int64_t b, int who, int many)
+__device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, int64_t a, int64_t b, int who, int many,
+                                                 bool own_idx = false, int32_t *thr = nullptr)
 {
     using E = Elem<DT>;
     constexpr bool MULTI = IDXB != 0;
     constexpr int IB = MULTI ? IDXB : 8;
-    const char *row = (const char *)p.g + (size_t)m * (size_t)p.stride * E::BYTES;
+    const char *row = (const char *)p.v.g + (size_t)m * (size_t)p.v.stride * E::BYTES;
     const int lane = who & 31;
     for (int64_t row0 = a + (int64_t)(who - lane) * 8; row0 < b; row0 += (int64_t)many * 8) {
         const int64_t row1 = min(row0 + 256, b);
-        const int j_row = warp_find_segment(p.seg_off, p.nseg, row0);
+        const int j_row = warp_find_segment(p.v.seg_off, p.v.nseg, row0);
         const int jl = j_row + lane;
-        const int64_t my_end = jl < p.nseg ? segment_end(p.seg_off, p.nseg, jl, p.d) : INT64_MAX;
-        const float my_W = __ldg(p.W + min(jl, p.nseg - 1));
+        const int64_t my_end = jl < p.v.nseg ? segment_end(p.v.seg_off, p.v.nseg, jl, p.v.d) : INT64_MAX;
+        const float my_W = __ldg(p.v.W + min(jl, p.v.nseg - 1));
         const int64_t i = min(row0 + lane * 8, b - 1);            // lanes beyond b idle but take part in the shuffles
         int seg[8] = {0, 0, 0, 0, 0, 0, 0, 0};                    // segment of each coordinate, relative to j_row
         int nb = 0;
@@ -85,10 +86,13 @@ __device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, i
             int j = j_row;
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-                j = advance_segment(p.seg_off, p.nseg, j, i + e);
-                Wc[e] = __ldg(p.W + j);
+                j = advance_segment(p.v.seg_off, p.v.nseg, j, i + e);
+                Wc[e] = __ldg(p.v.W + j);
             }
         }
+        typename IdxBits<IB>::T kbits = 0;
+        if (MULTI && own_idx)                                     // the whole warp takes part
+            kbits = (typename IdxBits<IB>::T)select_unit<DT, IB, 4>(p.v, row0 + lane * 8, row0, thr);
         if (row0 + lane * 8 >= b) continue;
         float v[8];
         uint4 q[8 / E::G];
@@ -99,22 +103,22 @@ __device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, i
         }
         uint32_t neg_lo, neg_hi;
         unit_signs<DT>(q, neg_lo, neg_hi);          // the sign of a padding coordinate is harmless: its level is 0
-        typename IdxBits<IB>::T kbits = 0;
-        if (MULTI) kbits = IdxBits<IB>::load(p.idx + i * IB / 8);
+        if (MULTI && !own_idx)
+            kbits = p.select ? IdxBits<IB>::load_written(p.idx + i * IB / 8) : IdxBits<IB>::load(p.idx + i * IB / 8);
         float inv[8];
         bool overflow = false;
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-            if (i + e >= p.d) v[e] = 0.0f;                        // padding quantizes to level 0
+            if (i + e >= p.v.d) v[e] = 0.0f;                        // padding quantizes to level 0
             const int k = MULTI ? (int)((kbits >> (e * IB)) & ((1u << IB) - 1u)) : 0;
-            inv[e] = inv_scale(p.scales.s[k & (UQ_MAX_SCALES - 1)], Wc[e]);
+            inv[e] = inv_scale(p.v.scales.s[k & (UQ_MAX_SCALES - 1)], Wc[e]);
             overflow |= not_finite(inv[e]);
         }
         if (overflow && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
         const uint64_t blk = RNG == 32 ? (uint64_t)((p.coord0 + i) >> 2) : (uint64_t)((p.coord0 + i) >> 3);
-        char *lrow = (char *)p.lev + (size_t)m * LevelFmt<FMT>::row_bytes(p.stride);
-        quantize_unit<FMT, RNG>(v, inv, p.cap, neg_lo, neg_hi, p.key, (uint32_t)blk, (uint32_t)(blk >> 32), (uint32_t)(m + p.worker0),
-                                lrow + LevelFmt<FMT>::off(i), lrow + LevelFmt<FMT>::off2(i, p.stride));
+        char *lrow = (char *)p.lev + (size_t)m * LevelFmt<FMT>::row_bytes(p.v.stride);
+        quantize_unit<FMT, RNG>(v, inv, p.v.s_hat, neg_lo, neg_hi, p.key, (uint32_t)blk, (uint32_t)(blk >> 32), (uint32_t)(m + p.worker0),
+                                lrow + LevelFmt<FMT>::off(i), lrow + LevelFmt<FMT>::off2(i, p.v.stride));
     }
 }
 
@@ -133,10 +137,10 @@ __device__ __noinline__ void encode_tile_mixed(const EncodeParams &p, int m, int
     constexpr int H = 8 / E::G;
     constexpr int KMASK = IB < 4 ? (1 << IB) - 1 : UQ_MAX_SCALES - 1;
     const int tid = threadIdx.x, lane = tid & 31;
-    const int32_t my_scale = p.scales.s[lane & KMASK];
-    const int64_t my_end = j + lane < p.nseg ? segment_end(p.seg_off, p.nseg, j + lane, p.d) : INT64_MAX;
-    const char *grow = (const char *)p.g + (size_t)m * (size_t)p.stride * E::BYTES;
-    char *lrow = (char *)p.lev + (size_t)m * LF::row_bytes(p.stride);
+    const int32_t my_scale = p.v.scales.s[lane & KMASK];
+    const int64_t my_end = j + lane < p.v.nseg ? segment_end(p.v.seg_off, p.v.nseg, j + lane, p.v.d) : INT64_MAX;
+    const char *grow = (const char *)p.v.g + (size_t)m * (size_t)p.v.stride * E::BYTES;
+    char *lrow = (char *)p.lev + (size_t)m * LF::row_bytes(p.v.stride);
     bool overflow = false;
 #pragma unroll 1
     for (int u = 0; u < S::UNITS; ++u) {
@@ -148,11 +152,11 @@ __device__ __noinline__ void encode_tile_mixed(const EncodeParams &p, int m, int
             jr = j + cnt;
             end = __shfl_sync(0xFFFFFFFFu, my_end, cnt);
         } else {                                                 // more than 32 segments inside one tile
-            jr = warp_find_segment(p.seg_off, p.nseg, r0);
-            end = segment_end(p.seg_off, p.nseg, jr, p.d);
+            jr = warp_find_segment(p.v.seg_off, p.v.nseg, r0);
+            end = segment_end(p.v.seg_off, p.v.nseg, jr, p.v.d);
         }
         if (end < r0 + 256) continue;                            // warp-uniform
-        const float inv_lane = inv_scale(my_scale, __ldg(p.W + jr));
+        const float inv_lane = inv_scale(my_scale, __ldg(p.v.W + jr));
         overflow |= not_finite(inv_lane);
         const int64_t i = r0 + lane * 8;
         uint4 q[H];
@@ -163,26 +167,41 @@ __device__ __noinline__ void encode_tile_mixed(const EncodeParams &p, int m, int
             E::unpack(q[h], *(float(*)[E::G])(v + h * E::G));
         }
         typename IdxBits<IB>::T kbits = 0;
-        if (MULTI) kbits = IdxBits<IB>::load(p.idx + i * IB / 8);
+        if (MULTI) kbits = p.select ? IdxBits<IB>::load_written(p.idx + i * IB / 8) : IdxBits<IB>::load(p.idx + i * IB / 8);
 #pragma unroll
         for (int e = 0; e < 8; ++e)
             inv[e] = MULTI ? __shfl_sync(0xFFFFFFFFu, inv_lane, (int)(uint32_t)(kbits >> (e * IB))) : inv_lane;
         uint32_t neg_lo, neg_hi;
         unit_signs<DT>(q, neg_lo, neg_hi);
         const uint64_t blk = RNG == 32 ? (uint64_t)((p.coord0 + i) >> 2) : (uint64_t)((p.coord0 + i) >> 3);
-        quantize_unit<FMT, RNG>(v, inv, p.cap, neg_lo, neg_hi, p.key, (uint32_t)blk, (uint32_t)(blk >> 32),
-                                (uint32_t)(m + p.worker0), lrow + LF::off(i), lrow + LF::off2(i, p.stride));
+        quantize_unit<FMT, RNG>(v, inv, p.v.s_hat, neg_lo, neg_hi, p.key, (uint32_t)blk, (uint32_t)(blk >> 32),
+                                (uint32_t)(m + p.worker0), lrow + LF::off(i), lrow + LF::off2(i, p.v.stride));
     }
-    if (overflow && lane < p.scales.N && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
+    if (overflow && lane < p.v.scales.N && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
 }
 
 // The slow forms of a whole tile, workers m0 .. m1 - 1: the ragged last tile, a tile whose Philox block
 // numbers leave the launch's high word, or 16-bit draws with a factor too small for the saturating
 // form (j < 0: per-coordinate lookup), and a full tile crossed by segment boundaries (j = its first
 // segment).  One out-of-line call keeps their registers out of the straight-line path.
+// In select mode the CTA first finds and stores the shared indices of the whole tile (thr: the
+// CTA's kWarps * 2 * UQ_MAX_SCALES words of shared memory); the encoding then reads them back.
 template <int DT, int FMT, int RNG, int IDXB>
-__device__ __noinline__ void encode_tile_slow(const EncodeParams &p, int64_t t0, int64_t t1, int j, int m0, int m1)
+__device__ __noinline__ void encode_tile_slow(const EncodeParams &p, int64_t t0, int64_t t1, int j, int m0, int m1,
+                                              int32_t *thr)
 {
+    if (IDXB != 0 && p.select) {
+        constexpr int IB = IDXB != 0 ? IDXB : 8;
+        const int lane = threadIdx.x & 31;
+        for (int u = 0; u < EncodeShape<DT, RNG>::UNITS; ++u) {
+            const int64_t i = t0 + (int64_t)(u * kThreads + threadIdx.x) * 8;
+            const int64_t row0 = i - lane * 8;
+            if (row0 >= t1) break;                                   // warp-uniform
+            const uint64_t packed = select_unit<DT, IB, 4>(p.v, i, row0, thr + (threadIdx.x >> 5) * 2 * UQ_MAX_SCALES);
+            if (i < p.v.d) store_unit_indices<IB>(p.idx, i, packed);
+        }
+        __syncthreads();                                             // the tile's indices are in memory for all warps
+    }
     for (int m = m0; m < m1; ++m) {
         if (j < 0) encode_span_general<DT, FMT, RNG, IDXB>(p, m, t0, t1, threadIdx.x, kThreads);
         else encode_tile_mixed<DT, FMT, RNG, IDXB>(p, m, t0, j);
@@ -200,11 +219,12 @@ template <int DT, int FMT, int RNG, int IDXB> struct TileState {
     PhiloxBlockPart blk[U * BPU];     // worker-independent rounds of the units' Philox blocks
     SatConstants sc;
     const char *gp;                   // my first coordinate in the gradient row that is loaded next
+    const uint4 *sp;                  // select mode: my slot of that row's copy in shared memory
     char *lp, *lp2;                   // and in the level row that is stored next (second plane for 6-bit)
     size_t grow, lrow;                // bytes between rows
 };
 
-template <int DT, int FMT, int RNG, int IDXB>
+template <bool SEL, int DT, int FMT, int RNG, int IDXB>
 __device__ __forceinline__ void load_units(TileState<DT, FMT, RNG, IDXB> &t,
                                            uint4 (&q)[EncodeShape<DT, RNG>::UNITS][8 / Elem<DT>::G])
 {
@@ -213,14 +233,15 @@ __device__ __forceinline__ void load_units(TileState<DT, FMT, RNG, IDXB> &t,
     for (int u = 0; u < T::U; ++u)
 #pragma unroll
         for (int h = 0; h < T::H; ++h)
-            q[u][h] = ld_stream(t.gp + (u * kThreads * 8 + h * T::E::G) * T::E::BYTES);
-    t.gp += t.grow;
+            q[u][h] = SEL ? t.sp[(u * T::H + h) * kThreads] : ld_stream(t.gp + (u * kThreads * 8 + h * T::E::G) * T::E::BYTES);
+    if (SEL) t.sp += T::U * T::H * kThreads;
+    else t.gp += t.grow;
 }
 
 // Workers m0 .. m0 + G - 1 of the tile, straight-line.  On entry q holds worker m0's units (loaded
 // or in flight); while worker m is quantized the units of worker m + 1 are on their way (MORE: also
 // those of the worker after the last one of this call).
-template <int G, bool MORE, int DT, int FMT, int RNG, int IDXB>
+template <int G, bool MORE, bool SEL, int DT, int FMT, int RNG, int IDXB>
 __device__ __forceinline__ void encode_workers(const EncodeParams &p, TileState<DT, FMT, RNG, IDXB> &t, int m0,
                                                uint4 (&q)[EncodeShape<DT, RNG>::UNITS][8 / Elem<DT>::G])
 {
@@ -232,7 +253,7 @@ __device__ __forceinline__ void encode_workers(const EncodeParams &p, TileState<
     for (int k = 0; k < G; ++k) {
         const int m = m0 + k;
         uint4 qn[T::U][T::H];
-        if (k + 1 < G || MORE) load_units<DT, FMT, RNG, IDXB>(t, qn);
+        if (k + 1 < G || MORE) load_units<SEL, DT, FMT, RNG, IDXB>(t, qn);
         uint4 r[T::U * T::BPU];
         philox_join<T::U * T::BPU>(p.key, t.blk, p.wpart[m], r);
 #pragma unroll
@@ -247,7 +268,7 @@ __device__ __forceinline__ void encode_workers(const EncodeParams &p, TileState<
             } else {
                 UnitWords<RNG> rw;
                 rw.r[0] = r[u * T::BPU]; rw.r[RNG == 32 ? 1 : 0] = r[u * T::BPU + T::BPU - 1];
-                quantize_unit_bytes<RNG>(v, t.inv[u], p.cap, neg_lo, neg_hi, rw, lo, hi);
+                quantize_unit_bytes<RNG>(v, t.inv[u], p.v.s_hat, neg_lo, neg_hi, rw, lo, hi);
             }
             store_unit<FMT>(lo, hi, t.lp + u * kThreads * UB, t.lp2 + u * kThreads * UB2);
         }
@@ -262,8 +283,81 @@ __device__ __forceinline__ void encode_workers(const EncodeParams &p, TileState<
     }
 }
 
-template <int DT, int FMT, int RNG, int IDXB>
-__global__ void __launch_bounds__(kThreads, (EncodeShape<DT, RNG>::MIN_CTAS)) encode_kernel(const __grid_constant__ EncodeParams p)
+// Select mode: copies of the tile's rows of workers m0 .. m0 + cnt - 1 into shared memory, laid out
+// [worker][unit][16 bytes][thread] so that every thread reads back only what it copied (no barrier).
+// CNT > 0: cnt is that compile-time value (no predicates); CNT == 0: cnt at run time.
+template <int CNT, int DT, int RNG>
+__device__ __forceinline__ void stage_rows(uint4 *stage, const char *gp, size_t grow, int cnt)
+{
+    using E = Elem<DT>;
+    constexpr int U = EncodeShape<DT, RNG>::UNITS, H = 8 / E::G;
+    const int tid = threadIdx.x;
+#pragma unroll
+    for (int m = 0; m < kWorkerGroup; ++m) {
+        if (CNT > 0 ? m < CNT : m < cnt) {
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int h = 0; h < H; ++h)
+                    copy_async16(stage + ((m * U + u) * H + h) * kThreads + tid, gp + (u * kThreads * 8 + h * E::G) * E::BYTES);
+            gp += grow;
+        }
+    }
+}
+
+// Select mode: the largest magnitude over the staged workers of the 8 coordinates of unit u, as
+// binary32 bit patterns.  bf16: two coordinates per word.  Its sign-magnitude halves read as
+// signed 16-bit integers order the positive values, read as unsigned ones the negative values
+// (sign bit set) above all others, so max |x| = max(smax & 0x7FFF, umax & 0x7FFF): two packed
+// three-input maxima per two workers and word, no mask per element.  binary32: three-input
+// maxima of absolute values, as the selector's kernel takes them (a NaN is skipped).
+template <int CNT, int DT, int RNG>
+__device__ __forceinline__ void staged_max_magnitude(const uint4 *stage, int u, int cnt, uint32_t (&amag)[8])
+{
+    using E = Elem<DT>;
+    constexpr int U = EncodeShape<DT, RNG>::UNITS, H = 8 / E::G;
+    const int tid = threadIdx.x;
+    if (DT == UQ_F32) {
+        float a[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+        for (int m = 0; m < kWorkerGroup; ++m) {
+            if (CNT > 0 ? m < CNT : m < cnt) {
+#pragma unroll
+                for (int h = 0; h < H; ++h) {
+                    const uint4 x = stage[((m * U + u) * H + h) * kThreads + tid];
+                    a[4 * h + 0] = fmaxf(a[4 * h + 0], fabsf(__uint_as_float(x.x)));
+                    a[4 * h + 1] = fmaxf(a[4 * h + 1], fabsf(__uint_as_float(x.y)));
+                    a[4 * h + 2] = fmaxf(a[4 * h + 2], fabsf(__uint_as_float(x.z)));
+                    a[4 * h + 3] = fmaxf(a[4 * h + 3], fabsf(__uint_as_float(x.w)));
+                }
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) amag[e] = __float_as_uint(a[e]);
+    } else {
+        uint32_t smax[4] = {0x80008000u, 0x80008000u, 0x80008000u, 0x80008000u}, umax[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int m = 0; m < kWorkerGroup; ++m) {
+            if (CNT > 0 ? m < CNT : m < cnt) {
+                const uint4 x = stage[(m * U + u) * kThreads + tid];
+                const uint32_t w4[4] = { x.x, x.y, x.z, x.w };
+#pragma unroll
+                for (int c = 0; c < 4; ++c) { smax[c] = __vmaxs2(smax[c], w4[c]); umax[c] = __vmaxu2(umax[c], w4[c]); }
+            }
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const uint32_t am = __vmaxu2(smax[c] & 0x7FFF7FFFu, umax[c] & 0x7FFF7FFFu);
+            amag[2 * c] = am << 16; amag[2 * c + 1] = am & 0xFFFF0000u;
+        }
+    }
+}
+
+// SEL: the kernel also finds and stores the shared scale indices (multi-scale, all M <= kWorkerGroup
+// workers in one CTA): the tile's rows are copied to shared memory once (every thread its own
+// units, so no barrier), read there for the maximum over the workers and again for quantization.
+template <int DT, int FMT, int RNG, int IDXB, bool SEL>
+__global__ void __launch_bounds__(kThreads, (SEL ? 3 : EncodeShape<DT, RNG>::MIN_CTAS)) encode_kernel(const __grid_constant__ EncodeParams p)
 {
     grid_dependency_prologue();
     using T = TileState<DT, FMT, RNG, IDXB>;
@@ -274,30 +368,32 @@ __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, RNG>::MIN_CTAS)) en
     constexpr int IB = MULTI ? IDXB : 8;
     constexpr int U = T::U, H = T::H, BPU = T::BPU;
     const int tid = threadIdx.x, lane = tid & 31;
+    __shared__ int32_t sh_thr[MULTI ? kWarps * 2 * UQ_MAX_SCALES : 1];   // select mode, slow paths: threshold tables
     if (blockIdx.x >= p.main_blocks) {
         // A CTA of the second kind: each warp takes one segment boundary of one worker and, if the
         // boundary lies strictly inside a 256-coordinate row of a full tile, quantizes that row with
         // per-coordinate scales (the tile's own CTA skips it).  Keeping these rows out of the tile
         // CTAs keeps their lifetime short: the slow path no longer holds a whole CTA slot.
         const uint32_t x = blockIdx.x - p.main_blocks;
-        const int m = (int)(x % (uint32_t)p.M);
-        const int64_t k = 1 + (int64_t)(x / (uint32_t)p.M) * kWarps + (tid >> 5);
-        if (k >= p.nseg) return;
-        const int64_t b = __ldg(p.seg_off + k), prev = __ldg(p.seg_off + k - 1);
+        const int m = (int)(x % (uint32_t)p.v.M);
+        const int64_t k = 1 + (int64_t)(x / (uint32_t)p.v.M) * kWarps + (tid >> 5);
+        if (k >= p.v.nseg) return;
+        const int64_t b = __ldg(p.v.seg_off + k), prev = __ldg(p.v.seg_off + k - 1);
         const int64_t r0 = b & ~(int64_t)255;
-        const int64_t full_end = p.d / S::TILE * S::TILE;          // rows beyond belong to the ragged tile's CTA
+        const int64_t full_end = p.v.d / S::TILE * S::TILE;          // rows beyond belong to the ragged tile's CTA
         if (b <= 0 || b == r0 || r0 >= full_end) return;           // not strictly inside a row of a full tile
         if (prev > r0 && prev <= b) return;                        // an earlier boundary in the same row takes it
-        encode_span_general<DT, FMT, RNG, IDXB>(p, m, r0, r0 + 256, lane, 32);
+        encode_span_general<DT, FMT, RNG, IDXB>(p, m, r0, r0 + 256, lane, 32, MULTI && p.select,
+                                                sh_thr + (MULTI ? (tid >> 5) * 2 * UQ_MAX_SCALES : 0));
         return;
     }
     // CTAs walk the tiles back to front (see launch_encode); a tile's CTAs take 8 workers each
     const uint32_t rev = p.main_blocks - 1u - blockIdx.x;
     const int64_t tile = (int64_t)(rev / p.groups);
     const int m0 = (int)(rev % p.groups) * kWorkerGroup;
-    const int cnt = min(kWorkerGroup, p.M - m0);
+    const int cnt = min(kWorkerGroup, p.v.M - m0);
     const int64_t t0 = tile * S::TILE;
-    const int64_t t1 = min(t0 + (int64_t)S::TILE, p.d);
+    const int64_t t1 = min(t0 + (int64_t)S::TILE, p.v.d);
 
     // Philox block of the tile's first unit.  The units of a tile add less than 2^12 to it; the
     // straight-line path keeps the high word fixed (the per-worker table of the launch was made for
@@ -307,42 +403,81 @@ __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, RNG>::MIN_CTAS)) en
     const uint64_t blk0 = (uint64_t)(p.coord0 >> BSH) + (uint64_t)tile * (uint32_t)(S::TILE >> BSH);
     const bool other_hi = (uint32_t)blk0 > 0xFFFFFFFFu - (uint32_t)(S::TILE >> BSH) || (uint32_t)(blk0 >> 32) != p.blk_hi;
     if (t1 - t0 != S::TILE || other_hi) {
-        encode_tile_slow<DT, FMT, RNG, IDXB>(p, t0, t1, -1, m0, m0 + cnt);
+        encode_tile_slow<DT, FMT, RNG, IDXB>(p, t0, t1, -1, m0, m0 + cnt, sh_thr);
         return;
     }
     // every warp looks the segment up for itself (no shared memory, no barrier)
-    const int j = warp_find_segment(p.seg_off, p.nseg, t0);
-    if (segment_end(p.seg_off, p.nseg, j, p.d) < t1) {
+    const int j = warp_find_segment(p.v.seg_off, p.v.nseg, t0);
+    if (segment_end(p.v.seg_off, p.v.nseg, j, p.v.d) < t1) {
         // A segment boundary crosses the tile (at most nseg - 1 tiles): a compact loop over the
         // rows of every worker, kept out of line so that its registers do not weigh on the path below.
-        encode_tile_slow<DT, FMT, RNG, IDXB>(p, t0, t1, j, m0, m0 + cnt);
+        encode_tile_slow<DT, FMT, RNG, IDXB>(p, t0, t1, j, m0, m0 + cnt, sh_thr);
         return;
     }
-    // the first worker's row and the shared indices
     T t;
-    t.grow = (size_t)p.stride * E::BYTES;
-    t.lrow = LF::row_bytes(p.stride);
-    t.gp = (const char *)p.g + (size_t)m0 * t.grow + ((size_t)t0 + (size_t)tid * 8) * E::BYTES;
+    t.grow = (size_t)p.v.stride * E::BYTES;
+    t.lrow = LF::row_bytes(p.v.stride);
+    t.gp = (const char *)p.v.g + (size_t)m0 * t.grow + ((size_t)t0 + (size_t)tid * 8) * E::BYTES;
     uint4 q[U][H];
-    load_units<DT, FMT, RNG, IDXB>(t, q);
     typename IdxBits<IB>::T kbits[U];
-    if (MULTI) {
-        const uint8_t *ip = p.idx + ((size_t)t0 + (size_t)tid * 8) * IB / 8;
+    extern __shared__ uint4 stage[];                             // SEL: [worker][unit][16 bytes][thread]
+    if (SEL) {
+        t.sp = stage + tid;
+        if (cnt == kWorkerGroup) stage_rows<kWorkerGroup, DT, RNG>(stage, t.gp, t.grow, cnt);
+        else stage_rows<0, DT, RNG>(stage, t.gp, t.grow, cnt);
+    } else {
+        // the first worker's row and the shared indices are on their way during the set-up below
+        load_units<false, DT, FMT, RNG, IDXB>(t, q);
+        if (MULTI) {
+            const uint8_t *ip = p.idx + ((size_t)t0 + (size_t)tid * 8) * IB / 8;
 #pragma unroll
-        for (int u = 0; u < U; ++u) kbits[u] = IdxBits<IB>::load(ip + u * kThreads * IB);
+            for (int u = 0; u < U; ++u) kbits[u] = IdxBits<IB>::load(ip + u * kThreads * IB);
+        }
     }
     // lane k holds s_k / W_j (single-scale: every lane holds s / W_j)
     constexpr int KMASK = IB < 4 ? (1 << IB) - 1 : UQ_MAX_SCALES - 1;    // lane L holds scale L & KMASK
-    const float W = __ldg(p.W + j);
-    float inv_lane = inv_scale(p.scales.s[lane & KMASK], W);
-    if (lane < p.scales.N && not_finite(inv_lane) && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
-    if (RNG == 16) {
-        if (!sat_form_exact(inv_scale(p.scales.s[0], W))) {        // W beyond 2^100: the plain arithmetic
-            encode_tile_slow<DT, FMT, RNG, IDXB>(p, t0, t1, -1, m0, m0 + cnt);
-            return;
+    const float W = __ldg(p.v.W + j);
+    float inv_lane = inv_scale(p.v.scales.s[lane & KMASK], W);
+    if (lane < p.v.scales.N && not_finite(inv_lane) && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
+    if (RNG == 16 && !sat_form_exact(inv_scale(p.v.scales.s[0], W))) {   // W beyond 2^100: the plain arithmetic
+        if (SEL) copy_async_wait();
+        encode_tile_slow<DT, FMT, RNG, IDXB>(p, t0, t1, -1, m0, m0 + cnt, sh_thr);
+        return;
+    }
+    if (SEL) {
+        // Scale selection and sharing for the tile (Algorithm 2 lines "Compute coordinate scales" and
+        // "Scale sharing"): the largest magnitude over the workers decides the shared index (see
+        // uq_select.cuh), found by bisection over the pass thresholds that lanes 0 .. N-1 hold.
+        const int N = p.v.scales.N;
+        const int32_t thr = lane < N ? pass_threshold(inv_lane, p.v.s_hat) : -1;
+        const int top = N > 1 ? 1 << (31 - __clz(N - 1)) : 0;               // first step of the bisection
+        const int32_t thr_top = __shfl_sync(0xFFFFFFFFu, thr, top);
+        copy_async_wait();
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            uint32_t amag[8];
+            if (cnt == kWorkerGroup) staged_max_magnitude<kWorkerGroup, DT, RNG>(stage, u, cnt, amag);
+            else staged_max_magnitude<0, DT, RNG>(stage, u, cnt, amag);
+            int k[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) k[e] = (top != 0 && (int32_t)amag[e] <= thr_top) ? top : 0;   // the first step
+#pragma unroll 1
+            for (int step = top >> 1; step >= 1; step >>= 1) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                    if ((int32_t)amag[e] <= __shfl_sync(0xFFFFFFFFu, thr, k[e] + step)) k[e] += step;
+            }
+            typename IdxBits<IB>::T packed = 0;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) packed |= (typename IdxBits<IB>::T)k[e] << (e * IB);
+            kbits[u] = packed;
+            store_unit_indices<IB>(p.idx, t0 + (int64_t)(u * kThreads + tid) * 8, packed);
         }
+        load_units<true, DT, FMT, RNG, IDXB>(t, q);
+    }
+    if (RNG == 16) {
         inv_lane = __fmul_rn(inv_lane, 0.00390625f);
-        t.sc = sat_constants(p.cap);
+        t.sc = sat_constants(p.v.s_hat);
     }
     // the shuffle reads its source lane modulo 32 and the table repeats every 2^IB lanes (an 8-bit
     // index is below 16), so the index bits need a shift but no mask
@@ -358,51 +493,77 @@ __global__ void __launch_bounds__(kThreads, (EncodeShape<DT, RNG>::MIN_CTAS)) en
         for (int b = 0; b < BPU; ++b) t.blk[u * BPU + b] = philox_block_part(p.key, blk_lo + (uint32_t)(u * kThreads * BPU + b));
     char *lrow0 = (char *)p.lev + (size_t)m0 * t.lrow;
     t.lp = lrow0 + LF::off(t0) + tid * LF::UB;
-    t.lp2 = lrow0 + LF::off2(t0, p.stride) + tid * (FMT == UQ_FMT_I6P ? 2 : 0);
+    t.lp2 = lrow0 + LF::off2(t0, p.v.stride) + tid * (FMT == UQ_FMT_I6P ? 2 : 0);
 
     // The workers of the group straight-line, with no loop around them: all 8, or (the last group
     // of a job whose M is not a multiple of 8) 4, 2 and 1 of them as the count's bits say.
     if (cnt == kWorkerGroup) {
-        encode_workers<kWorkerGroup, false, DT, FMT, RNG, IDXB>(p, t, m0, q);
+        encode_workers<kWorkerGroup, false, SEL, DT, FMT, RNG, IDXB>(p, t, m0, q);
         return;
     }
     int m = m0;
     if (cnt & 4) {
-        if (cnt & 3) encode_workers<4, true, DT, FMT, RNG, IDXB>(p, t, m, q);
-        else encode_workers<4, false, DT, FMT, RNG, IDXB>(p, t, m, q);
+        if (cnt & 3) encode_workers<4, true, SEL, DT, FMT, RNG, IDXB>(p, t, m, q);
+        else encode_workers<4, false, SEL, DT, FMT, RNG, IDXB>(p, t, m, q);
         m += 4;
     }
     if (cnt & 2) {
-        if (cnt & 1) encode_workers<2, true, DT, FMT, RNG, IDXB>(p, t, m, q);
-        else encode_workers<2, false, DT, FMT, RNG, IDXB>(p, t, m, q);
+        if (cnt & 1) encode_workers<2, true, SEL, DT, FMT, RNG, IDXB>(p, t, m, q);
+        else encode_workers<2, false, SEL, DT, FMT, RNG, IDXB>(p, t, m, q);
         m += 2;
     }
-    if (cnt & 1) encode_workers<1, false, DT, FMT, RNG, IDXB>(p, t, m, q);
+    if (cnt & 1) encode_workers<1, false, SEL, DT, FMT, RNG, IDXB>(p, t, m, q);
 }
 
-template <int DT, int FMT, int RNG, int IDXB>
+template <int DT, int FMT, int RNG, int IDXB, bool SEL = false>
 static cudaError_t launch(EncodeParams p, cudaStream_t st)
 {
     using S = EncodeShape<DT, RNG>;
-    p.ntiles = (p.d + S::TILE - 1) / S::TILE;
-    p.groups = (uint32_t)((p.M + kWorkerGroup - 1) / kWorkerGroup);
+    p.ntiles = (p.v.d + S::TILE - 1) / S::TILE;
+    p.groups = (uint32_t)((p.v.M + kWorkerGroup - 1) / kWorkerGroup);
     int64_t blocks = p.ntiles * p.groups;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     p.main_blocks = (uint32_t)blocks;
-    if (p.seg_off != nullptr && p.nseg > 1) blocks += (int64_t)((p.nseg - 1 + kWarps - 1) / kWarps) * p.M;
+    if (p.v.seg_off != nullptr && p.v.nseg > 1) blocks += (int64_t)((p.v.nseg - 1 + kWarps - 1) / kWarps) * p.v.M;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     constexpr int BSH = RNG == 32 ? 2 : 3;
     p.blk_hi = (uint32_t)((uint64_t)(p.coord0 >> BSH) >> 32);
     for (int m = 0; m < UQ_MAX_WORKERS; ++m)
-        p.wpart[m] = philox_worker_part(p.key, p.blk_hi, (uint32_t)(p.worker0 + (m < p.M ? m : 0)));
-    launch_k(encode_kernel<DT, FMT, RNG, IDXB>, (unsigned)blocks, kThreads, st, p);
+        p.wpart[m] = philox_worker_part(p.key, p.blk_hi, (uint32_t)(p.worker0 + (m < p.v.M ? m : 0)));
+    if (SEL) {
+        // the copies of the tile's rows: up to kWorkerGroup workers * TILE coordinates (64 KiB)
+        const size_t smem = (size_t)(p.v.M < kWorkerGroup ? p.v.M : kWorkerGroup) * S::TILE * Elem<DT>::BYTES;
+        // more than 48 KiB of dynamic shared memory needs an opt-in per kernel and device (the call
+        // is idempotent, so a race between host threads on the flag is harmless)
+        static bool opted_in[64] = {};
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= 64 || !opted_in[dev]) {
+            e = cudaFuncSetAttribute(encode_kernel<DT, FMT, RNG, IDXB, SEL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kWorkerGroup * S::TILE * Elem<DT>::BYTES);
+            if (e != cudaSuccess) return e;
+            if (dev >= 0 && dev < 64) opted_in[dev] = true;
+        }
+        launch_k_smem(encode_kernel<DT, FMT, RNG, IDXB, SEL>, (unsigned)blocks, kThreads, smem, st, p);
+    } else {
+        launch_k(encode_kernel<DT, FMT, RNG, IDXB, SEL>, (unsigned)blocks, kThreads, st, p);
+    }
     return cudaGetLastError();
 }
 
 template <int DT, int FMT, int RNG>
 static cudaError_t dispatch_idx(const EncodeParams &p, int idx_bits, cudaStream_t st)
 {
+    if (p.select) {
+        switch (idx_bits) {
+        case 1: return launch<DT, FMT, RNG, 1, true>(p, st);
+        case 2: return launch<DT, FMT, RNG, 2, true>(p, st);
+        case 4: return launch<DT, FMT, RNG, 4, true>(p, st);
+        default: return launch<DT, FMT, RNG, 8, true>(p, st);
+        }
+    }
     switch (idx_bits) {
     case 0: return launch<DT, FMT, RNG, 0>(p, st);
     case 1: return launch<DT, FMT, RNG, 1>(p, st);

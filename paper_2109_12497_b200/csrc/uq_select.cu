@@ -9,159 +9,30 @@
 // non-increasing in |g^m_i|, and min_m k^m_i = k(max_m |g^m_i|) exactly.  The kernel therefore
 // folds the min-all-reduce into a max over the M resident buffers followed by one threshold
 // search per coordinate; the result is bit-identical to selecting per worker and taking the min.
-#include "uq_device.cuh"
+#include "uq_select.cuh"
 
 namespace uq {
 
 struct SelectParams {
-    const void *g;
+    SelectView v;
     uint8_t *idx;
-    const float *W;
-    const int64_t *seg_off;
     uint32_t *status;
-    int64_t d, stride;
-    int32_t nseg, M;
-    float s_hat;
-    ScaleSet scales;
 };
 
 constexpr int kSelectTile = kThreads * 8;
-
-__device__ __forceinline__ float inv_scale_sel(int32_t s, float W)
-{
-    return W > 0.0f ? __fdiv_rn((float)s, W) : 0.0f;
-}
-
-// The general path for one thread's 8 coordinates (row crossed by a segment boundary): the test
-// is evaluated as written, with one division per scale and coordinate.  Rare, kept out of line.
-__device__ __noinline__ uint64_t select_general(const SelectParams &p, int64_t i, const uint32_t (&amag)[8], int idxb,
-                                                 int j)      // j: a segment at or before coordinate i's
-{
-    uint64_t packed = 0;
-    for (int e = 0; e < 8; ++e) {
-        int k = 0;
-        if (i + e < p.d) {                                          // padding keeps index 0
-            j = advance_segment(p.seg_off, p.nseg, j, i + e);
-            const float Wj = __ldg(p.W + j), a = __uint_as_float(amag[e]);
-            for (int kk = 1; kk < p.scales.N; ++kk)
-                if (__fmul_rn(a, inv_scale_sel(p.scales.s[kk], Wj)) <= p.s_hat) k = kk;
-        }
-        packed |= (uint64_t)k << (e * idxb);
-    }
-    return packed;
-}
 
 // LEVELS = ceil(log2 N): the per-coordinate search is a bisection over the N thresholds.
 template <int DT, int IDXB, int LEVELS>
 __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant__ SelectParams p)
 {
     grid_dependency_prologue();
-    using E = Elem<DT>;
-    constexpr int H = 8 / E::G;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int64_t i = ((int64_t)blockIdx.x * kThreads + tid) * 8;   // my first coordinate
     const int64_t row0 = i - (int64_t)lane * 8;                     // my warp's first coordinate
-    if (row0 >= p.d) return;                                        // warp-uniform
-    const bool active = i < p.d;
-
-    // max over the workers of the magnitude bits (bf16: two coordinates per word)
-    uint32_t amag[8];
-    if (DT == UQ_F32) {
-        float amax[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) amax[e] = 0.0f;
-        if (active) {
-            const char *col = (const char *)p.g + (size_t)i * E::BYTES;
-            int m = 0;
-            for (; m + 4 <= p.M; m += 4) {                          // four workers' loads in flight
-                uint4 q[4][H];
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-#pragma unroll
-                    for (int h = 0; h < H; ++h)
-                        q[k][h] = ld_stream(col + ((size_t)(m + k) * (size_t)p.stride + h * E::G) * E::BYTES);
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    float v[8];
-#pragma unroll
-                    for (int h = 0; h < H; ++h) E::unpack(q[k][h], *(float(*)[E::G])(v + h * E::G));
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) amax[e] = fmaxf(amax[e], fabsf(v[e]));
-                }
-            }
-            for (; m < p.M; ++m) {
-                float v[8];
-#pragma unroll
-                for (int h = 0; h < H; ++h)
-                    E::unpack(ld_stream(col + ((size_t)m * (size_t)p.stride + h * E::G) * E::BYTES),
-                              *(float(*)[E::G])(v + h * E::G));
-#pragma unroll
-                for (int e = 0; e < 8; ++e) amax[e] = fmaxf(amax[e], fabsf(v[e]));
-            }
-        }
-#pragma unroll
-        for (int e = 0; e < 8; ++e) amag[e] = __float_as_uint(amax[e]);
-    } else {
-        // bf16 magnitudes order like unsigned 15-bit integers: packed 16-bit max, no unpacking
-        uint32_t am[4] = {0u, 0u, 0u, 0u};
-        if (active) {
-            const char *col = (const char *)p.g + (size_t)i * E::BYTES;
-            int m = 0;
-            for (; m + 8 <= p.M; m += 8) {                          // eight workers' loads in flight
-                uint4 q[8];
-#pragma unroll
-                for (int k = 0; k < 8; ++k) q[k] = ld_stream(col + (size_t)(m + k) * (size_t)p.stride * E::BYTES);
-#pragma unroll
-                for (int k = 0; k < 8; k += 2) {
-                    am[0] = __vimax3_u16x2(am[0], q[k].x & 0x7FFF7FFFu, q[k + 1].x & 0x7FFF7FFFu);
-                    am[1] = __vimax3_u16x2(am[1], q[k].y & 0x7FFF7FFFu, q[k + 1].y & 0x7FFF7FFFu);
-                    am[2] = __vimax3_u16x2(am[2], q[k].z & 0x7FFF7FFFu, q[k + 1].z & 0x7FFF7FFFu);
-                    am[3] = __vimax3_u16x2(am[3], q[k].w & 0x7FFF7FFFu, q[k + 1].w & 0x7FFF7FFFu);
-                }
-            }
-            for (; m < p.M; ++m) {
-                const uint4 q = ld_stream(col + (size_t)m * (size_t)p.stride * E::BYTES);
-                am[0] = __vmaxu2(am[0], q.x & 0x7FFF7FFFu);
-                am[1] = __vmaxu2(am[1], q.y & 0x7FFF7FFFu);
-                am[2] = __vmaxu2(am[2], q.z & 0x7FFF7FFFu);
-                am[3] = __vmaxu2(am[3], q.w & 0x7FFF7FFFu);
-            }
-        }
-#pragma unroll
-        for (int w = 0; w < 4; ++w) { amag[2 * w] = am[w] << 16; amag[2 * w + 1] = am[w] & 0xFFFF0000u; }
-    }
-
-    // every warp looks up the segment of its own row of 256 coordinates and builds the threshold
-    // table of that segment in its own slice of shared memory: entry k is the largest magnitude
-    // that passes scale k, -1 beyond the last scale
+    if (row0 >= p.v.d) return;                                      // warp-uniform
     __shared__ int32_t sh_thr[kWarps][2 * UQ_MAX_SCALES];
-    const int64_t row1 = min(row0 + 256, p.d);
-    const int j0 = warp_find_segment(p.seg_off, p.nseg, row0);
-    uint64_t packed = 0;
-    if (segment_end(p.seg_off, p.nseg, j0, p.d) >= row1) {
-        int32_t thr = -1;
-        if (lane < p.scales.N) thr = pass_threshold(inv_scale_sel(p.scales.s[lane], __ldg(p.W + j0)), p.s_hat);
-        sh_thr[warp][lane] = thr;
-        __syncwarp();
-        const int32_t *T = sh_thr[warp];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int32_t a = (int32_t)amag[e];
-            int k = 0;
-#pragma unroll
-            for (int step = 1 << (LEVELS - 1); step >= 1; step >>= 1)
-                if (a <= T[k + step]) k += step;                    // k + step < 2^LEVELS <= 16
-            if (i + e >= p.d) k = 0;                                // padding keeps index 0
-            packed |= (uint64_t)k << (e * IDXB);
-        }
-    } else if (active) {
-        packed = select_general(p, i, amag, IDXB, j0);
-    }
-    if (!active) return;
-    if (IDXB == 1) p.idx[i >> 3] = (uint8_t)packed;
-    else if (IDXB == 2) *(uint16_t *)(p.idx + (i >> 2)) = (uint16_t)packed;
-    else if (IDXB == 4) *(uint32_t *)(p.idx + (i >> 1)) = (uint32_t)packed;
-    else *(uint64_t *)(p.idx + i) = packed;
+    const uint64_t packed = select_unit<DT, IDXB, LEVELS>(p.v, i, row0, sh_thr[warp]);
+    if (i < p.v.d) store_unit_indices<IDXB>(p.idx, i, packed);
 }
 
 // One row only (M = 1: a single worker, or the row of maxima that uq_agree_scale_amax leaves).
@@ -181,22 +52,22 @@ __global__ void __launch_bounds__(kThreads, 4) select_row_kernel(const __grid_co
     constexpr int H = 8 / E::G;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int64_t t0 = (int64_t)blockIdx.x * (kSelectTile * kRowUnits);
-    const int64_t t1 = min(t0 + (int64_t)kSelectTile * kRowUnits, p.d);
+    const int64_t t1 = min(t0 + (int64_t)kSelectTile * kRowUnits, p.v.d);
     uint4 q[kRowUnits][H];
 #pragma unroll
     for (int u = 0; u < kRowUnits; ++u) {
         const int64_t i = t0 + (int64_t)u * kSelectTile + tid * 8;
 #pragma unroll
         for (int h = 0; h < H; ++h)
-            q[u][h] = i < p.d ? ld_stream((const char *)p.g + (size_t)(i + h * E::G) * E::BYTES) : make_uint4(0, 0, 0, 0);
+            q[u][h] = i < p.v.d ? ld_stream((const char *)p.v.g + (size_t)(i + h * E::G) * E::BYTES) : make_uint4(0, 0, 0, 0);
     }
     __shared__ int32_t sh_thr[kWarps][2 * UQ_MAX_SCALES];
-    const int jt = warp_find_segment(p.seg_off, p.nseg, t0);
-    const bool tile_uniform = segment_end(p.seg_off, p.nseg, jt, p.d) >= t1;
+    const int jt = warp_find_segment(p.v.seg_off, p.v.nseg, t0);
+    const bool tile_uniform = segment_end(p.v.seg_off, p.v.nseg, jt, p.v.d) >= t1;
     int j_table = -1;                                               // segment whose thresholds the table holds
     if (tile_uniform) {
         int32_t thr = -1;
-        if (lane < p.scales.N) thr = pass_threshold(inv_scale_sel(p.scales.s[lane], __ldg(p.W + jt)), p.s_hat);
+        if (lane < p.v.scales.N) thr = pass_threshold(inv_scale_sel(p.v.scales.s[lane], __ldg(p.v.W + jt)), p.v.s_hat);
         sh_thr[warp][lane] = thr;
         __syncwarp();
         j_table = jt;
@@ -205,7 +76,7 @@ __global__ void __launch_bounds__(kThreads, 4) select_row_kernel(const __grid_co
     for (int u = 0; u < kRowUnits; ++u) {
         const int64_t i = t0 + (int64_t)u * kSelectTile + tid * 8;
         const int64_t row0 = i - (int64_t)lane * 8;
-        if (row0 >= p.d) break;                                     // warp-uniform
+        if (row0 >= p.v.d) break;                                     // warp-uniform
         uint32_t amag[8];
         if (DT == UQ_F32) {
             amag[0] = q[u][0].x & 0x7FFFFFFFu; amag[1] = q[u][0].y & 0x7FFFFFFFu;
@@ -221,13 +92,13 @@ __global__ void __launch_bounds__(kThreads, 4) select_row_kernel(const __grid_co
         int j0 = jt;
         bool row_uniform = true;
         if (!tile_uniform) {                                        // per-row setup, as in the general kernel
-            const int64_t row1 = min(row0 + 256, p.d);
-            j0 = warp_find_segment(p.seg_off, p.nseg, row0);
-            row_uniform = segment_end(p.seg_off, p.nseg, j0, p.d) >= row1;
+            const int64_t row1 = min(row0 + 256, p.v.d);
+            j0 = warp_find_segment(p.v.seg_off, p.v.nseg, row0);
+            row_uniform = segment_end(p.v.seg_off, p.v.nseg, j0, p.v.d) >= row1;
             if (row_uniform && j0 != j_table) {
                 __syncwarp();
                 int32_t thr = -1;
-                if (lane < p.scales.N) thr = pass_threshold(inv_scale_sel(p.scales.s[lane], __ldg(p.W + j0)), p.s_hat);
+                if (lane < p.v.scales.N) thr = pass_threshold(inv_scale_sel(p.v.scales.s[lane], __ldg(p.v.W + j0)), p.v.s_hat);
                 sh_thr[warp][lane] = thr;
                 __syncwarp();
                 j_table = j0;
@@ -243,13 +114,13 @@ __global__ void __launch_bounds__(kThreads, 4) select_row_kernel(const __grid_co
 #pragma unroll
                 for (int step = 1 << (LEVELS - 1); step >= 1; step >>= 1)
                     if (a <= T[k + step]) k += step;                // k + step < 2^LEVELS <= 16
-                if (i + e >= p.d) k = 0;                            // padding keeps index 0
+                if (i + e >= p.v.d) k = 0;                            // padding keeps index 0
                 packed |= (decltype(packed))k << (e * IDXB);
             }
-        } else if (i < p.d) {
-            packed = (decltype(packed))select_general(p, i, amag, IDXB, j0);
+        } else if (i < p.v.d) {
+            packed = (decltype(packed))select_general(p.v, i, amag, IDXB, j0);
         }
-        if (i >= p.d) continue;
+        if (i >= p.v.d) continue;
         if (IDXB == 1) p.idx[i >> 3] = (uint8_t)packed;
         else if (IDXB == 2) *(uint16_t *)(p.idx + (i >> 2)) = (uint16_t)packed;
         else if (IDXB == 4) *(uint32_t *)(p.idx + (i >> 1)) = (uint32_t)packed;
@@ -260,7 +131,7 @@ __global__ void __launch_bounds__(kThreads, 4) select_row_kernel(const __grid_co
 template <int DT, int IDXB>
 static cudaError_t dispatch_levels(const SelectParams &p, unsigned blocks, cudaStream_t st)
 {
-    const int N = p.scales.N;
+    const int N = p.v.scales.N;
     if (N <= 2) launch_k(select_kernel<DT, IDXB, 1>, blocks, kThreads, st, p);
     else if (N <= 4) launch_k(select_kernel<DT, IDXB, 2>, blocks, kThreads, st, p);
     else if (N <= 8) launch_k(select_kernel<DT, IDXB, 3>, blocks, kThreads, st, p);
@@ -271,10 +142,10 @@ static cudaError_t dispatch_levels(const SelectParams &p, unsigned blocks, cudaS
 template <int DT>
 static cudaError_t dispatch(const SelectParams &p, int idx_bits, cudaStream_t st)
 {
-    if (p.M == 1 && p.d > 0) {                                      // one row: the kernel without per-row setup
-        const int64_t nb = (p.d + kSelectTile * kRowUnits - 1) / (kSelectTile * kRowUnits);
+    if (p.v.M == 1 && p.v.d > 0) {                                      // one row: the kernel without per-row setup
+        const int64_t nb = (p.v.d + kSelectTile * kRowUnits - 1) / (kSelectTile * kRowUnits);
         if (nb > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
-        const int N = p.scales.N;
+        const int N = p.v.scales.N;
         const int lv = N <= 2 ? 1 : N <= 4 ? 2 : N <= 8 ? 3 : 4;
 #define UQ_ROW(IB, LV) launch_k(select_row_kernel<DT, IB, LV>, (unsigned)nb, kThreads, st, p)
         switch (idx_bits * 8 + lv) {
@@ -293,7 +164,7 @@ static cudaError_t dispatch(const SelectParams &p, int idx_bits, cudaStream_t st
 #undef UQ_ROW
         return cudaGetLastError();
     }
-    const int64_t blocks = (p.d + kSelectTile - 1) / kSelectTile;
+    const int64_t blocks = (p.v.d + kSelectTile - 1) / kSelectTile;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     if (idx_bits == 1) { launch_k(select_kernel<DT, 1, 1>, (unsigned)blocks, kThreads, st, p); return cudaGetLastError(); }
@@ -306,10 +177,10 @@ cudaError_t launch_select(const uq_layout &L, const void *g, const float *W, con
                           int idx_bits, uint8_t *idx, uint32_t *status, cudaStream_t st)
 {
     SelectParams p;
-    p.g = g; p.idx = idx; p.W = W; p.seg_off = L.seg_off; p.status = status;
-    p.d = L.d; p.stride = L.worker_stride; p.nseg = L.nseg; p.M = L.M;
-    p.s_hat = (float)scales.s[0];
-    p.scales = scales;
+    p.v.g = g; p.idx = idx; p.v.W = W; p.v.seg_off = L.seg_off; p.status = status;
+    p.v.d = L.d; p.v.stride = L.worker_stride; p.v.nseg = L.nseg; p.v.M = L.M;
+    p.v.s_hat = (float)scales.s[0];
+    p.v.scales = scales;
     return L.dtype == UQ_F32 ? dispatch<UQ_F32>(p, idx_bits, st) : dispatch<UQ_BF16>(p, idx_bits, st);
 }
 

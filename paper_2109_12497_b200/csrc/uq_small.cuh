@@ -87,6 +87,7 @@ __device__ __forceinline__ bool small_agree(const SmallParams &p, float &W_out)
     __threadfence();
     __syncthreads();
     if (tid == 0) {
+        __threadfence();                  // release: this CTA's partials (ordered before the barrier above) before its arrival
         atomicAdd(p.counter, 1u);
         uint32_t polls = 0;
         int fail = 0;
@@ -94,7 +95,8 @@ __device__ __forceinline__ bool small_agree(const SmallParams &p, float &W_out)
             if (++polls > kSmallSpinLimit) { fail = 1; break; }
             __nanosleep(32);
         }
-        if (fail && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_TIMEOUT);
+        __threadfence();                  // acquire: the other CTAs' partials after their arrivals
+        if (fail) atomicOr(p.status, (uint32_t)UQ_STATUS_TIMEOUT);
         sh_fail = fail;
         // the last CTA to leave the barrier puts both counters back to zero for the next call
         // (every CTA has read its last value of the arrival counter by then)

@@ -16,10 +16,28 @@ __device__ __forceinline__ bool not_finite(float x) { return (__float_as_uint(x)
 
 // The idx_bits * 8 bits that belong to 8 consecutive coordinates starting at a multiple of 8.
 template <int IDXB> struct IdxBits;
-template <> struct IdxBits<1> { using T = uint32_t; static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg(p); } };
-template <> struct IdxBits<2> { using T = uint32_t; static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg((const uint16_t *)p); } };
-template <> struct IdxBits<4> { using T = uint32_t; static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg((const uint32_t *)p); } };
-template <> struct IdxBits<8> { using T = uint64_t; static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg((const unsigned long long *)p); } };
+// load: indices written by an earlier kernel; load_written: indices that this kernel wrote itself
+// (the read-only path must not be used for them).
+template <> struct IdxBits<1> {
+    using T = uint32_t;
+    static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg(p); }
+    static __device__ __forceinline__ T load_written(const uint8_t *p) { return __ldcg(p); }
+};
+template <> struct IdxBits<2> {
+    using T = uint32_t;
+    static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg((const uint16_t *)p); }
+    static __device__ __forceinline__ T load_written(const uint8_t *p) { return __ldcg((const uint16_t *)p); }
+};
+template <> struct IdxBits<4> {
+    using T = uint32_t;
+    static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg((const uint32_t *)p); }
+    static __device__ __forceinline__ T load_written(const uint8_t *p) { return __ldcg((const uint32_t *)p); }
+};
+template <> struct IdxBits<8> {
+    using T = uint64_t;
+    static __device__ __forceinline__ T load(const uint8_t *p) { return __ldg((const unsigned long long *)p); }
+    static __device__ __forceinline__ T load_written(const uint8_t *p) { return __ldcg((const unsigned long long *)p); }
+};
 
 // Eight coordinates: magnitudes scaled by inv[e], random words from the block(s) starting at
 // (blk_lo, blk_hi), levels gathered four to a word, signs applied bytewise (`neg` holds 0xFF in

@@ -23,20 +23,20 @@ class Quantizer:
                  seg_off: Optional[Sequence[int]] = None, s: int = 127,
                  scales: Optional[Sequence[int]] = None, fmt: int = B.UQ_FMT_I8, idx_bits: int = 0,
                  norm: int = B.UQ_NORM_L2, rng_bits: int = 32, keep_sums: bool = False,
-                 device: str | torch.device = "cuda", fused_select: bool = False, amax_select: bool = False,
+                 device: str | torch.device = "cuda", fused_select: bool = False,
                  one_kernel: Optional[bool] = None):
         B.lib()                                     # fail now if the CUDA library is not built
         dev = torch.device(device)
+        if dev.type == "cuda" and dev.index is None:
+            dev = torch.device("cuda", torch.cuda.current_device())
+        self.device = dev
         self.M, self.d, self.dtype = M, d, dtype
         self.stride = -(-d // 32) * 32
         self.multi = scales is not None and idx_bits != 0
-        # multi-scale: selection and encoding in one kernel instead of two (one launch less, the
-        # gradients read once; measured no faster than the two kernels on B200, so off by default)
-        self.fused_select = fused_select
-        # multi-scale: agree-scale also writes max_m |g^m_i| and the selector runs on that one row
-        # instead of on all M rows (a quarter less DRAM traffic per step; measured no faster on B200:
-        # the selector's time is its per-coordinate threshold search, not its reads; off by default)
-        self.amax_select = amax_select and self.multi and not fused_select
+        # multi-scale: selection + sharing + encoding as one call (uq_select_encode_multi: one kernel
+        # for M <= 8, the gradients read once: about 15 % less time for the pair on B200, same bits)
+        # instead of the selector and the encoder as two streaming kernels (uq_step, the default)
+        self.fused_select = fused_select and self.multi
         self.s = int(scales[0]) if self.multi else int(s)
         self.scales = [int(x) for x in scales] if self.multi else None
         self.fmt, self.idx_bits, self.norm, self.rng_bits = fmt, idx_bits if self.multi else 0, norm, rng_bits
@@ -48,21 +48,20 @@ class Quantizer:
         self.W = torch.zeros(nseg, dtype=torch.float32, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         # one segment, few workers, and so small that the step is bound by its launches: the whole step as one cooperative kernel (uq_step_small).  None = decide by size.
-        fits = B.small_step_supported(self.layout, fmt) and not (fused_select or amax_select)
+        fits = B.small_step_supported(self.layout, fmt)
         if one_kernel and not fits:
             raise ValueError("uq: the one-kernel step takes one segment, M <= 8 and one-plane level formats")
         self.one_kernel = fits and (one_kernel if one_kernel is not None
                                     else M * d * (4 if dtype == torch.float32 else 2) <= ONE_KERNEL_MAX_BYTES)
-        # zeroed: the one-kernel step wants its counters zero before the first call and leaves them so
-        self.workspace = torch.zeros(max(8, self.layout.workspace_bytes(), self.layout.workspace_bytes_amax(),
-                                         B.uq_workspace_bytes_small() if self.one_kernel else 0),
-                                     dtype=torch.uint8, device=dev)
+        self.workspace = torch.empty(max(8, self.layout.workspace_bytes()), dtype=torch.uint8, device=dev)
+        # The one-kernel step keeps its barrier counters in the first bytes of its scratch, wants them
+        # zero before the first call and leaves them zero: a buffer of its own, never handed to
+        # uq_agree_scale (whose partial sums would overwrite the counters).
+        self.small_workspace = (torch.zeros(max(8, B.uq_workspace_bytes_small()), dtype=torch.uint8, device=dev)
+                                if self.one_kernel else None)
         self.lev = torch.empty((M, self.layout.level_row_bytes(fmt)), dtype=torch.int8, device=dev)
         self.idx = (torch.empty(max(16, self.layout.index_bytes(self.idx_bits)), dtype=torch.uint8, device=dev)
                     if self.multi else None)
-        if self.amax_select:
-            self.amax = torch.empty((1, self.stride), dtype=dtype, device=dev)
-            self.layout_amax = B.Layout(1, d, self.stride, dtype, seg_dev)
         self.out = torch.empty(max(d, 1), dtype=torch.float32, device=dev)
         self.S = torch.empty(max(d, 1), dtype=torch.int32, device=dev) if keep_sums else None
         self._small_call = None
@@ -71,17 +70,10 @@ class Quantizer:
 
     # the four stages, each one C-ABI call -------------------------------------------------------
     def agree_scale(self, g: torch.Tensor) -> None:
-        if self.amax_select:
-            B.uq_agree_scale_amax(self.layout, g, self.norm, self.W, self.amax.view(-1), self.status, self.workspace)
-        else:
-            B.uq_agree_scale(self.layout, g, self.norm, self.W, self.status, self.workspace)
+        B.uq_agree_scale(self.layout, g, self.norm, self.W, self.status, self.workspace)
 
     def select_scale(self, g: torch.Tensor) -> None:
-        if self.amax_select:      # the index depends on the gradients only through max_m |g^m_i|
-            B.uq_select_scale_multi(self.layout_amax, self.amax, self.W, self.scales, self.idx_bits, self.idx,
-                                    self.status)
-        else:
-            B.uq_select_scale_multi(self.layout, g, self.W, self.scales, self.idx_bits, self.idx, self.status)
+        B.uq_select_scale_multi(self.layout, g, self.W, self.scales, self.idx_bits, self.idx, self.status)
 
     def encode(self, g: torch.Tensor, seed: int) -> None:
         if self.multi:
@@ -92,7 +84,7 @@ class Quantizer:
                                self.status)
 
     def select_encode(self, g: torch.Tensor, seed: int) -> None:
-        """Multi-scale: scale selection, scale sharing and quantization in one kernel."""
+        """Multi-scale: scale selection, scale sharing and quantization in one call."""
         B.uq_select_encode_multi(self.layout, g, self.W, self.scales, self.idx_bits, seed, self.rng_bits, self.fmt,
                                  self.idx, self.lev, self.status)
 
@@ -111,25 +103,21 @@ class Quantizer:
         if self.one_kernel:
             # every buffer but g is this object's own: their addresses are marshalled once, not per
             # step (the checked wrapper B.uq_step_small costs about as much host time as the kernel runs)
-            self.layout.check_g(g)
-            if not g.is_cuda:
-                raise ValueError("uq: tensors must live on a CUDA device")
+            self._check_devices(g)
             if self._small_call is None:
                 ptr = lambda t: None if t is None else t.data_ptr()
                 arr, N = B._scales(self.scales) if self.multi else (None, 0)
                 self._small_call = (B.lib().uq_step_small, self.layout.ref(), arr, N,
                                     (ptr(self.W), ptr(self.idx), ptr(self.lev), ptr(self.out), ptr(self.S),
-                                     ptr(self.status), ptr(self.workspace), self.workspace.numel()))
+                                     ptr(self.status), ptr(self.small_workspace), self.small_workspace.numel()))
             fn, ref, arr, N, tail = self._small_call
             rc = fn(ref, g.data_ptr(), self.norm, self.s, arr, N, self.idx_bits, seed, self.rng_bits, self.fmt, *tail,
                     B._stream())
             if rc != B.UQ_OK:
                 raise B.UqError("uq_step_small", rc)
             return self._out_view
-        if not (self.fused_select or self.amax_select):      # the plain sequence: one trip through the binding
-            self.layout.check_g(g)
-            if not g.is_cuda:
-                raise ValueError("uq: tensors must live on a CUDA device")
+        if not self.fused_select:                             # the default sequence: one trip through the binding (uq_step)
+            self._check_devices(g)
             if self._step_call is None:                      # addresses of my own buffers, marshalled once
                 ptr = lambda t: None if t is None else t.data_ptr()
                 arr, N = B._scales(self.scales) if self.multi else (None, 0)
@@ -142,28 +130,34 @@ class Quantizer:
             if rc != B.UQ_OK:
                 raise B.UqError("uq_step", rc)
             return self._out_view
-        self.agree_scale(g)
-        if self.multi and self.fused_select:
-            self.select_encode(g, seed)
-        else:
-            if self.multi:
-                self.select_scale(g)
-            self.encode(g, seed)
+        self.agree_scale(g)                                   # multi-scale, selection inside the encoder's kernel
+        self.select_encode(g, seed)
         self.aggregate_decode()
         return self.out[: self.d]
+
+    def _check_devices(self, g: torch.Tensor) -> None:
+        """The checks of the marshalling wrappers for the paths that call the library directly: the
+        gradients have the layout's shape, and they, this object's buffers and the current device
+        (on whose current stream the kernels are launched) are one and the same device."""
+        self.layout.check_g(g)
+        if not g.is_cuda:
+            raise ValueError("uq: tensors must live on a CUDA device")
+        current = torch.cuda.current_device()
+        B.require_current_device(g.device.index, current, "g")
+        B.require_current_device(self.device.index, current, "the quantizer")
 
     def kernels_per_step(self) -> int:
         """Kernel launches one step enqueues (norm partials + finalize, [select], encode, decode)."""
         if self.one_kernel:
             return 1
-        separate_select = self.multi and not self.fused_select and self.d > 0
+        separate_select = self.multi and (not self.fused_select or self.M > 8) and self.d > 0
         return (2 if self.d > 0 else 1) + (1 if separate_select else 0) + (2 if self.d > 0 else 0)
 
     def status_bits(self) -> int:
         """Synchronizes and returns the device status word (0 = clean)."""
         bits = int(self.status.item())
-        if bits & B.UQ_STATUS_TIMEOUT:            # a barrier wait ran out: its counters are not back at zero
-            self.workspace.zero_()
+        if bits & B.UQ_STATUS_TIMEOUT and self.small_workspace is not None:   # a barrier wait ran out: its counters are not back at zero
+            self.small_workspace.zero_()
         return bits
 
 
@@ -216,7 +210,7 @@ class RandKQuantizer:
 
 
 def from_workload(w, keep_sums: bool = False, device="cuda", fused_select: bool = False,
-                  amax_select: bool = False, one_kernel: Optional[bool] = None) -> Quantizer:
+                  one_kernel: Optional[bool] = None) -> Quantizer:
     """A Quantizer configured like a ``workloads.Workload``."""
     from . import workloads as wl
     seg = wl.segment_offsets(w)
@@ -225,7 +219,7 @@ def from_workload(w, keep_sums: bool = False, device="cuda", fused_select: bool 
         scales=list(w.scales) if w.quantizer == "multi" else None,
         fmt={"i8": B.UQ_FMT_I8, "i4x2": B.UQ_FMT_I4X2, "i2x4": B.UQ_FMT_I2X4, "i6p": B.UQ_FMT_I6P}[w.fmt], idx_bits=w.idx_bits,
         norm=B.UQ_NORM_L2 if w.norm == wl.NORM_L2 else B.UQ_NORM_LINF, rng_bits=w.rng_bits,
-        keep_sums=keep_sums, device=device, fused_select=fused_select, amax_select=amax_select, one_kernel=one_kernel)
+        keep_sums=keep_sums, device=device, fused_select=fused_select, one_kernel=one_kernel)
 
 
 def randk_from_workload(w, K: int, device="cuda") -> RandKQuantizer:

@@ -35,3 +35,19 @@ def own_scale_index(v: Fraction, W: Fraction, scales) -> int:
 def reconstruct(S: int, W: Fraction, s: int, M: int) -> Fraction:
     """R applied to the averaged levels: W * (S / M) / s."""
     return W * Fraction(S, M) / s
+
+
+def rint_half_even(x: Fraction) -> int:
+    """The integer nearest to x, a tie going to the even one (IEEE round-to-nearest-even)."""
+    f = floor(x)
+    r = x - f
+    if r > Fraction(1, 2) or (r == Fraction(1, 2) and f % 2 == 1):
+        return f + 1
+    return f
+
+
+def q_single_draw(v: Fraction, W: Fraction, s: int, h: int, b: int) -> int:
+    """The reading of "with probability p" for a b-bit draw h, uniform on [0, 2^b): round up iff
+    h < rint(p * 2^b), i.e. with the multiple of 2^-b nearest to p (ties to even)."""
+    l, p = level_and_p(v, W, s)
+    return sign(v) * (l + (1 if h < rint_half_even(p * 2 ** b) else 0))

@@ -29,9 +29,6 @@ class Layout:
     def workspace_bytes(self):
         return 8
 
-    def workspace_bytes_amax(self):
-        return 8
-
     def index_bytes(self, idx_bits):
         return self.worker_stride * idx_bits // 8
 

@@ -21,13 +21,12 @@ def to_device(w, g_np):
 
 
 def run_gpu(w, g_np, seed=None, mode="default"):
-    """All stage outputs of the CUDA path as numpy arrays.  mode picks the form of the multi-scale
-    path: "default" = "rows" (the selector reads all M rows), "amax" (agree-scale writes max_m |g|
-    and the selector runs on that row), "fused" (selection and encoding in one kernel); of the
-    single-scale path: "one" (the whole step as one cooperative kernel), "separate" (the calls one by
-    one), "default" (the library picks by size)."""
-    one_kernel = {"one": True, "separate": False}.get(mode)       # else: the library decides by size
-    q = from_workload(w, keep_sums=True, fused_select=mode == "fused", amax_select=mode == "amax", one_kernel=one_kernel)
+    """All stage outputs of the CUDA path as numpy arrays.  mode picks the form of the path:
+    "default" (what the library picks: the one-kernel step for small gradients, else uq_step),
+    "fused" (multi-scale: selection and encoding as one call, uq_select_encode_multi), "one" (the
+    whole step as one cooperative kernel), "separate" (never the one-kernel step)."""
+    one_kernel = {"one": True, "separate": False, "fused": False}.get(mode)       # else: the library decides by size
+    q = from_workload(w, keep_sums=True, fused_select=mode == "fused", one_kernel=one_kernel)
     g = to_device(w, g_np)
     q.step(g, w.seed if seed is None else seed)
     torch.cuda.synchronize()
@@ -82,11 +81,10 @@ def ulp_distance(a, b):
 
 def check_parity(w, g_np, seed=None):
     """Full comparison; returns the GPU result for further checks.  A multi-scale workload runs in
-    all three forms of its path (see run_gpu), a single-scale one that the one-kernel step takes in
-    both of its forms: each must match the oracle."""
+    both forms of its path (see run_gpu), a workload that the one-kernel step takes in both of
+    its forms: each must match the oracle."""
     if w.quantizer == "multi":
         _check_parity(w, g_np, seed, "fused")
-        _check_parity(w, g_np, seed, "amax")
     if one_kernel_takes(w):
         _check_parity(w, g_np, seed, "one")
         _check_parity(w, g_np, seed, "separate")

@@ -105,9 +105,10 @@ def test_later_entry_points_reject_bad_arguments_on_the_host(lib):
                        None) == B.UQ_ERR_WORKSPACE
     small_bytes = lib.uq_workspace_bytes_small()
     assert small_bytes >= 64 + 148 * 8 * 8 * 8
-    def small(L, s=127, scales=None, N=0, bits=0, fmt=B.UQ_FMT_I8, out=p, idx=None, ws=small_bytes):
-        return lib.uq_step_small(L, p, B.UQ_NORM_L2, s, scales, N, bits, 0, 16, fmt, p, idx, p, out, None, None, p, ws, None)
+    def small(L, s=127, scales=None, N=0, bits=0, fmt=B.UQ_FMT_I8, out=p, idx=None, ws=small_bytes, status=p):
+        return lib.uq_step_small(L, p, B.UQ_NORM_L2, s, scales, N, bits, 0, 16, fmt, p, idx, p, out, None, status, p, ws, None)
     assert small(bad) == B.UQ_ERR_BAD_ARG
+    assert small(ok, status=None) == B.UQ_ERR_BAD_ARG                                      # a timeout must be reportable
     assert small(ok, s=128) == B.UQ_ERR_BAD_ARG
     assert small(ok, out=p + 16) == B.UQ_ERR_BAD_ARG                                      # out: 32-byte aligned
     assert small(ok, scales=sc, N=2, bits=3, idx=p) == B.UQ_ERR_BAD_ARG                     # idx_bits
@@ -116,9 +117,6 @@ def test_later_entry_points_reject_bad_arguments_on_the_host(lib):
     assert small(ok, s=31, fmt=B.UQ_FMT_I6P) == B.UQ_ERR_UNSUPPORTED
     assert small(ok, ws=64) == B.UQ_ERR_WORKSPACE
     assert small(ok, scales=sc, N=2, bits=2, idx=p, ws=64) == B.UQ_ERR_WORKSPACE
-    assert lib.uq_agree_scale_amax(bad, p, B.UQ_NORM_L2, p, p, None, p, 1 << 20, None) == B.UQ_ERR_BAD_ARG
-    assert lib.uq_agree_scale_amax(ok, p, B.UQ_NORM_L2, p, p + 8, None, p, 1 << 20, None) == B.UQ_ERR_BAD_ARG   # alignment
-    assert lib.uq_agree_scale_amax(ok, p, B.UQ_NORM_L2, p, None, None, p, 1 << 20, None) == B.UQ_ERR_BAD_ARG
     assert lib.uq_select_encode_multi(ok, p, p, sc, 2, 3, 0, 16, B.UQ_FMT_I8, p, p, None, None) == B.UQ_ERR_BAD_ARG   # idx_bits
     assert lib.uq_select_encode_multi(ok, p, p, sc, 2, 2, 0, 16, B.UQ_FMT_I4X2, p, p, None, None) == B.UQ_ERR_BAD_ARG  # s_hat > 7
     assert lib.uq_select_encode_multi(ok, p, p, sc, 2, 2, 0, 16, B.UQ_FMT_I8, None, p, None, None) == B.UQ_ERR_BAD_ARG
@@ -147,3 +145,13 @@ def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "LIB_PATH", tmp_path / "missing.so")
     with pytest.raises(RuntimeError, match="no CPU fallback"):
         B.lib()
+
+
+def test_a_tensor_on_another_device_is_refused_before_any_launch():
+    """The calls launch on the current device's current stream; the binding refuses, on the host,
+    a tensor that lives elsewhere (checked here on the rule itself: no GPU, no launch)."""
+    B.require_current_device(0, 0)
+    B.require_current_device(3, 3, "g")
+    for index, current in ((1, 0), (0, 1), (None, 0)):
+        with pytest.raises(ValueError, match="current device"):
+            B.require_current_device(index, current, "g")

@@ -13,7 +13,7 @@ from oracle import uq_oracle as o
 from paper_2109_12497_b200 import binding as B
 from paper_2109_12497_b200 import workloads as wl
 from paper_2109_12497_b200.pipeline import from_workload
-from parity import run_gpu, run_oracle, to_device, ulp_distance
+from parity import check_parity, run_gpu, run_oracle, to_device, ulp_distance
 
 pytestmark = pytest.mark.gpu
 
@@ -112,7 +112,7 @@ def test_decode_over_separate_rows(name, d, M):
     """uq_decode_rows: every worker's level row in an allocation of its own (as a peer's row would
     be), handed over as addresses; same sums and values as the one-buffer call."""
     w = wl.scaled(name, d, M=M)
-    r = run_gpu(w, wl.generate(w))
+    r = check_parity(w, wl.generate(w))            # the one-buffer result, itself compared with the oracle
     q = r["q"]
     rows = [q.lev[m].clone() for m in reversed(range(M))][::-1]          # allocated in reverse order
     out = torch.full((d + 16,), 7.0, device="cuda")
@@ -144,7 +144,7 @@ def test_slice_exchange_replayed_rank_by_rank(name, d, M, R, kw):
     kw = {k: v for k, v in kw.items() if v is not None}
     w = wl.scaled(name, d, M=M, **kw)
     g_np = wl.generate(w)
-    one = run_gpu(w, g_np)
+    one = check_parity(w, g_np)                    # the single-process result, itself compared with the oracle
     q = one["q"]
     P = max(1, -(-d // (R * SLICE_ALIGN))) * SLICE_ALIGN
     stride, shift, M_local = R * P, FMT[w.fmt], M // R
@@ -196,12 +196,13 @@ def test_distributed_quantizer_on_one_rank_equals_the_pipeline():
         for name in ("c2", "c3"):
             w = wl.scaled(name, 200_003, M=4)
             g_np = wl.generate(w)
+            want = check_parity(w, g_np)["out"]    # the pipeline's result, itself compared with the oracle
             q = DistributedQuantizer(
                 w.M, w.d, torch.float32, seg_off=wl.segment_offsets(w), s=w.s,
                 scales=list(w.scales) if w.quantizer == "multi" else None, fmt=FMT[w.fmt], idx_bits=w.idx_bits,
                 norm=B.UQ_NORM_L2, rng_bits=w.rng_bits)
             got = q.step(to_device(w, g_np), w.seed).cpu().numpy()
-            assert np.array_equal(got, run_gpu(w, g_np)["out"]) and int(q.status.item()) == 0
+            assert np.array_equal(got, want) and int(q.status.item()) == 0
             # the same with the level rows in symmetric memory, read where they are
             qp = DistributedQuantizer(
                 w.M, w.d, torch.float32, seg_off=wl.segment_offsets(w), s=w.s,
@@ -209,7 +210,7 @@ def test_distributed_quantizer_on_one_rank_equals_the_pipeline():
                 norm=B.UQ_NORM_L2, rng_bits=w.rng_bits, pull_levels=True)
             for _ in range(2):
                 got = qp.step(to_device(w, g_np), w.seed).cpu().numpy()
-                assert np.array_equal(got, run_gpu(w, g_np)["out"]) and int(qp.status.item()) == 0
+                assert np.array_equal(got, want) and int(qp.status.item()) == 0
             # and the reduce-scatter / all-gather form (rows padded to its stride)
             qs = DistributedQuantizer(
                 w.M, w.d, torch.float32, seg_off=wl.segment_offsets(w), s=w.s,
@@ -218,6 +219,6 @@ def test_distributed_quantizer_on_one_rank_equals_the_pipeline():
             g_pad = torch.zeros((w.M, qs.stride), device="cuda")
             g_pad[:, : g_np.shape[1]] = to_device(w, g_np)
             got = qs.step(g_pad, w.seed).cpu().numpy()
-            assert np.array_equal(got, run_gpu(w, g_np)["out"]) and int(qs.status.item()) == 0
+            assert np.array_equal(got, want) and int(qs.status.item()) == 0
     finally:
         dist.destroy_process_group()

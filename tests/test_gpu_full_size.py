@@ -88,6 +88,52 @@ def test_sampled_windows_of_large_workload(name):
         assert np.abs(lev.astype(int)).max() <= w.s
 
 
+@pytest.mark.parametrize("name", ["c4", "c5"])
+def test_large_workload_in_full(name):
+    """The two largest workloads compared with the oracle in full, not on windows: every scale,
+    shared index, level, integer sum and reconstructed value (the oracle is fed the GPU's scale
+    bits, which may differ from its own by one unit in the last place; see the chain rule in
+    parity.py).  One pass of each side; rows are compared one at a time to bound host memory."""
+    w = wl.WORKLOADS[name]
+    threads = max(1, os.cpu_count() or 1)
+    g_np = wl.generate(w, threads=threads)
+    seg = wl.segment_offsets(w)
+    q = from_workload(w, keep_sums=True)
+    g = torch.empty((w.M, w.stride), dtype=torch.float32 if w.dtype == wl.F32 else torch.bfloat16, device="cuda")
+    for m in range(w.M):
+        g[m].copy_(to_device(w, g_np[m: m + 1])[0])
+    q.step(g, w.seed)
+    torch.cuda.synchronize()
+    assert q.status_bits() == 0
+    del g
+    W = q.W.cpu().numpy()
+    gv = g_np[:, : w.d]
+    assert ulp_distance(W, o.agree_scale(gv, seg, o.NORM_L2)).max() <= 1
+    if w.quantizer == "multi":
+        idx = o.select_scale_multi(gv, W, w.scales, seg_off=seg)
+        nb = w.d * w.idx_bits // 8
+        assert np.array_equal(q.idx[:nb].cpu().numpy(), o.pack_index(idx, w.idx_bits)[:nb]), "scale indices differ"
+        lev = o.encode_multi(gv, W, w.scales, idx, w.seed, w.rng_bits, seg_off=seg)
+    else:
+        lev = o.encode_single(gv, W, w.s, w.seed, w.rng_bits, seg_off=seg)
+    assert np.abs(lev).max() <= w.s
+    for m in range(w.M):
+        row = q.lev[m].cpu().numpy().view(np.uint8)
+        if w.fmt == "i4x2":
+            want = o.pack_levels_i4(lev[m: m + 1])[0]
+        else:
+            want = lev[m].view(np.uint8)
+        assert np.array_equal(row[: want.size], want), f"levels of worker {m} differ"
+    S = o.aggregate(lev)
+    del lev
+    assert np.array_equal(q.S[: w.d].cpu().numpy(), S), "integer sums differ"
+    if w.quantizer == "multi":
+        out = o.decode(S, w.M, W, scales=w.scales, idx=idx, seg_off=seg)
+    else:
+        out = o.decode(S, w.M, W, s=w.s, seg_off=seg)
+    assert np.allclose(q.out[: w.d].cpu().numpy(), out, rtol=FP32_RTOL, atol=0), "reconstruction differs"
+
+
 def _even_stride(lev):
     """Copy with an even row stride, as the 4-bit packer needs."""
     M, n = lev.shape

@@ -62,19 +62,24 @@ def test_unsupported_configurations_are_refused():
     ws = torch.zeros(B.uq_workspace_bytes_small(), dtype=torch.uint8, device="cuda")
     W, out = torch.zeros(1, device="cuda"), torch.zeros(128, device="cuda")
     lev = torch.empty((9, 128), dtype=torch.int8, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
     with pytest.raises(B.UqError) as e:
         B.uq_step_small(B.Layout(9, 100, 128, torch.float32), g, B.UQ_NORM_L2, 127, None, 0, 0, 16, B.UQ_FMT_I8, W, None, lev, out,
-                        None, None, ws)
+                        None, st, ws)
     assert e.value.code == B.UQ_ERR_UNSUPPORTED
     lay = B.Layout(2, 100, 128, torch.float32)
     lev6 = torch.empty((2, lay.level_row_bytes(B.UQ_FMT_I6P)), dtype=torch.int8, device="cuda")
     with pytest.raises(B.UqError) as e:
-        B.uq_step_small(lay, g[:2].contiguous(), B.UQ_NORM_L2, 31, None, 0, 0, 16, B.UQ_FMT_I6P, W, None, lev6, out, None, None, ws)
+        B.uq_step_small(lay, g[:2].contiguous(), B.UQ_NORM_L2, 31, None, 0, 0, 16, B.UQ_FMT_I6P, W, None, lev6, out, None, st, ws)
     assert e.value.code == B.UQ_ERR_UNSUPPORTED
     with pytest.raises(B.UqError) as e:
         B.uq_step_small(lay, g[:2].contiguous(), B.UQ_NORM_L2, 127, None, 0, 0, 16, B.UQ_FMT_I8, W, None, lev[:2].contiguous(), out,
-                        None, None, ws[:64])
+                        None, st, ws[:64])
     assert e.value.code == B.UQ_ERR_WORKSPACE
+    with pytest.raises(B.UqError) as e:                       # a wait that runs out must be able to say so
+        B.uq_step_small(lay, g[:2].contiguous(), B.UQ_NORM_L2, 127, None, 0, 0, 16, B.UQ_FMT_I8, W, None, lev[:2].contiguous(), out,
+                        None, None, ws)
+    assert e.value.code == B.UQ_ERR_BAD_ARG
 
 
 def test_draws_are_keyed_by_worker_and_coordinate_of_the_job():
@@ -131,11 +136,11 @@ def test_the_wait_at_the_barrier_is_bounded():
     g_np = wl.generate(w)
     q = from_workload(w, keep_sums=True, one_kernel=True)
     g = to_device(w, g_np)
-    q.workspace[:4] = torch.tensor([0xC0, 0xFF, 0xFF, 0xFF], dtype=torch.uint8)     # 2^32 - 64, little endian
+    q.small_workspace[:4] = torch.tensor([0xC0, 0xFF, 0xFF, 0xFF], dtype=torch.uint8)     # 2^32 - 64, little endian
     q.step(g, 0)
     bits = q.status_bits()                       # synchronizes; zeroes the scratch after a timeout
     assert bits & B.UQ_STATUS_TIMEOUT
-    assert int(q.workspace[:64].sum().item()) == 0
+    assert int(q.small_workspace[:64].sum().item()) == 0
     q.status.zero_()
     _ = q.step(g, w.seed)
     torch.cuda.synchronize()

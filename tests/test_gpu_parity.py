@@ -34,7 +34,7 @@ def test_segmented_workloads_small(name, d, rng_bits):
 
 
 @pytest.mark.parametrize("name,d,M,kw", [
-    ("c2", 2_100_003, 8, {}), ("c2", 2_100_003, 8, dict(rng_bits=32)), ("c3", 2_100_003, 8, {}),
+    ("c2", 2_100_003, 8, {}), ("c2", 2_100_003, 8, dict(rng_bits=16)), ("c3", 2_100_003, 8, {}),
     ("c4", 1_060_013, 16, {}), ("c5", 1_060_013, 16, {}), ("c5", 2_100_003, 8, dict(rng_bits=32, idx_bits=8)),
     ("c3", 2_100_003, 8, dict(dtype=wl.BF16, fmt="i4x2", s=7, scales=(7, 112, 1792))),
     ("c2", 2_100_003, 8, dict(fmt="i2x4", s=1, scales=(1,))),
@@ -245,7 +245,7 @@ def test_reproducible_bit_for_bit():
     assert np.array_equal(a["idx"][:nb], b["idx"][:nb])
 
 
-@pytest.mark.parametrize("name,kw", [("c2", {}), ("c2", dict(rng_bits=32)), ("c3", {}), ("c5", {}),
+@pytest.mark.parametrize("name,kw", [("c2", {}), ("c2", dict(rng_bits=16)), ("c3", {}), ("c5", {}),
                                       ("c4", {}), ("c3", dict(fmt="i2x4", s=1, scales=(1, 16, 256)))])
 def test_gradient_handed_over_in_pieces(name, kw):
     """The encoders on pieces of the gradient (layout.coord0 = start of the piece, seg_off counted

@@ -7,7 +7,7 @@ import torch
 from oracle import uq_oracle as o
 from paper_2109_12497_b200 import binding as B
 from paper_2109_12497_b200 import workloads as wl
-from parity import FP32_RTOL, run_gpu
+from parity import FP32_RTOL, check_parity, run_gpu
 
 pytestmark = pytest.mark.gpu
 
@@ -26,7 +26,7 @@ def test_fused_update_two_bit_levels():
 
 def _fused_update_case(w, lr, mu, wd, use_mom):
     d = w.d
-    r = run_gpu(w, wl.generate(w))
+    r = check_parity(w, wl.generate(w))            # levels, sums and g_hat of the step, compared with the oracle
     q = r["q"]
     rng = np.random.default_rng(d)
     theta0 = rng.standard_normal(w.d).astype(np.float32)
@@ -41,8 +41,9 @@ def _fused_update_case(w, lr, mu, wd, use_mom):
         B.uq_decode_update(q.layout, q.lev, q.fmt, q.W, q.s, q.scales, q.idx, q.idx_bits,
                            theta[pad: pad + w.d], None if mom is None else mom[pad: pad + w.d], lr, mu, wd, ghat)
         torch.cuda.synchronize()
-        assert np.array_equal(ghat.cpu().numpy(), r["out"])          # same g_hat as the plain decode
-        theta0, mom0 = o.sgd_update(r["out"], theta0, mom0, lr=lr, mu=mu, wd=wd)
+        assert np.array_equal(ghat.cpu().numpy(), r["out"])          # same g_hat as the plain decode ...
+        assert np.allclose(ghat.cpu().numpy(), r["ref"]["out"], rtol=FP32_RTOL, atol=0)    # ... and as the oracle's
+        theta0, mom0 = o.sgd_update(r["ref"]["out"], theta0, mom0, lr=lr, mu=mu, wd=wd)   # the oracle's g_hat, not the GPU's
         got = theta.cpu().numpy()
         assert np.allclose(got[pad: pad + w.d], theta0, rtol=FP32_RTOL, atol=0)
         assert np.array_equal(got[pad: pad + w.d], theta0)           # same operation order: bit-equal

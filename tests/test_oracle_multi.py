@@ -157,6 +157,9 @@ def test_index_packing_layout():
     assert o.pack_index(idx, 2).tolist() == [0b11100100, 0b00011011]
     assert o.pack_index(idx, 4).tolist() == [0x10, 0x32, 0x23, 0x01]
     assert o.pack_index(idx, 8).tolist() == idx.tolist()
+    # 1-bit indices (two scales): coordinate i is bit i % 8 of byte i / 8
+    bits = np.array([1, 0, 0, 1, 1, 1, 0, 1, 1, 0, 1], dtype=np.uint8)
+    assert o.pack_index(bits, 1).tolist() == [0b10111001, 0b00000101]
 
 
 def test_workers_split_over_processes_give_the_same_result():

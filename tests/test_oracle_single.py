@@ -2,12 +2,14 @@
 (Section "QSGDMaxNorm Quantization", Algorithm 1, Lemma 1 and its proof)."""
 import json
 from fractions import Fraction
+from math import floor
 
 import numpy as np
 import pytest
 
 from oracle import uq_oracle as o
 from paper_2109_12497_b200 import workloads as wl
+import exact_model as em
 from exact_model import level_and_p, q_single, reconstruct
 
 
@@ -239,3 +241,45 @@ def test_int6_planar_packing_layout():
     nib = np.repeat(packed[0, :16], 2) >> np.tile([0, 4], 16) & 15
     cr = np.repeat(packed[0, 16:24], 4) >> np.tile([0, 2, 4, 6], 8) & 3
     assert ((16 * ((cr ^ 2) - 2) + nib)[:6] == lev[0]).all()
+
+
+@pytest.mark.parametrize("b,rng_bits", [(16, 16), (23, 32)])
+def test_draw_threshold_is_the_nearest_multiple_ties_to_even(b, rng_bits):
+    """Reading of "with probability p" for a b-bit draw: round up iff h < rint(p * 2^b), ties to
+    even.  Draws are injected on both sides of the threshold; the expected levels come from the
+    exact-rational model, which a ceiling, a floor or round-half-up each fail on one of the cases:
+      two values of p for which p * 2^b has a fraction above and below one half, so the nearest
+        multiple is the ceiling for one and the floor for the other;
+      p * 2^b = k + 1/2 exactly with k even and with k odd: the tie goes to the even neighbour.
+    W = 1 and s a power of two keep x = |v| * (s / W) exact, so the model sees the oracle's p."""
+    s, W = 4, np.float32(1.0)
+    f32 = lambda x: Fraction(float(np.float32(x)))
+    ulp = Fraction(1, 2 ** (b + 1))                                     # half a step of the draw
+    half = Fraction(1, 2)
+    # x = 1.3, 1.7 (nearest binary32): p * 2^16 has fraction 0.8.. / 0.2..; for 23 bits the fraction
+    # bits must lie below 2^-23, so x < 1/2: x = 1/4 + 5 * 2^-25 and 1/4 + 7 * 2^-25 (fractions 1/4, 3/4)
+    vs = [np.float32(0.325), np.float32(-0.425)] if b == 16 else \
+         [np.float32(float((Fraction(1, 4) + Fraction(5, 2 ** 25)) / s)), np.float32(float(-(Fraction(1, 4) + Fraction(7, 2 ** 25)) / s))]
+    vs += [
+          np.float32(float((half + 5 * ulp) / s)), np.float32(float(-(half + 7 * ulp) / s)),   # ties: p * 2^b = k + 1/2, k even / odd
+          np.float32(float(-(half + 9 * ulp) / s)), np.float32(float((half + 3 * ulp) / s))]   # k even / odd
+    assert len(vs) == 6
+    for v in vs:
+        assert Fraction(float(v)) * s == f32(float(v) * s)                # x is exact in binary32
+        l, p = em.level_and_p(Fraction(float(v)), Fraction(1), s)
+        P = em.rint_half_even(p * 2 ** b)
+        assert 0 < P < 2 ** b
+        for h in (P - 1, P, 0, 2 ** b - 1):
+            g = np.array([[v]], dtype=np.float32)
+            got = int(o.encode_single(g, np.array([W]), s, 0, rng_bits, h_inject=np.array([[h]], dtype=np.uint32))[0, 0])
+            want = em.q_single_draw(Fraction(float(v)), Fraction(1), s, h, b)
+            assert got == want, (float(v), h, got, want)
+        # the two draws around the threshold really straddle it
+        assert em.q_single_draw(Fraction(float(v)), Fraction(1), s, P - 1, b) != em.q_single_draw(Fraction(float(v)), Fraction(1), s, P, b)
+    for v, k_par in zip(vs[2:], (0, 1, 0, 1)):                         # the ties really are ties, of both parities
+        pb = em.level_and_p(Fraction(float(v)), Fraction(1), s)[1] * 2 ** b
+        assert pb % 1 == half and floor(pb) % 2 == k_par
+        assert em.rint_half_even(pb) == floor(pb) + k_par
+    # and the rounding direction differs between the cases, so neither ceiling nor floor fits all
+    fr = [(em.level_and_p(Fraction(float(v)), Fraction(1), s)[1] * 2 ** b) % 1 for v in vs[:2]]
+    assert fr[0] > Fraction(1, 2) > fr[1] or fr[1] > Fraction(1, 2) > fr[0]

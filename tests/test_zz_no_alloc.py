@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import uq_oracle as o
 from paper_2109_12497_b200 import binding as B
 from paper_2109_12497_b200 import workloads as wl
 from paper_2109_12497_b200.pipeline import from_workload
@@ -33,6 +34,8 @@ def test_static_scratch_matches_the_workspace_entry_point_on_consecutive_calls()
         g = _device_gradients(w)
         q.agree_scale(g)                                   # existing entry point, caller's workspace
         want = q.W.clone()
+        oracle_W = o.agree_scale(wl.generate(w)[:, : w.d], wl.segment_offsets(w),
+                                 o.NORM_LINF if w.norm == wl.NORM_LINF else o.NORM_L2)
         status = torch.zeros(1, dtype=torch.int32, device="cuda")
         for _ in range(2):
             got = torch.full_like(want, -1.0)
@@ -40,6 +43,8 @@ def test_static_scratch_matches_the_workspace_entry_point_on_consecutive_calls()
             torch.cuda.synchronize()
             ulp = np.abs(got.cpu().numpy().view(np.int32).astype(np.int64) - want.cpu().numpy().view(np.int32))
             assert ulp.max() <= 1 and ulp.max() == 0
+            ulp_oracle = np.abs(got.cpu().numpy().view(np.int32).astype(np.int64) - oracle_W.view(np.int32))
+            assert ulp_oracle.max() <= (0 if w.norm == wl.NORM_LINF else 1)      # the parity tests' bar for the scale
         assert int(status.item()) == 0 and float(want.max()) > 0
 
 
