@@ -646,6 +646,72 @@ def whole_job_value(world, in_bytes, ms):
     return world * in_bytes / ms / 1e6
 
 
+def bench_distributed(w, steps, warmup, device, threads, kernels=None, return_out=False):
+    """The paper's own setting beside the replicas figure: the M workers spread over the processes of
+    the job (M / world_size each), the three all-reduces of Algorithm 1 / 2 as real exchanges between
+    them (distributed.DistributedQuantizer: NCCL collectives on GPUs; no peer loads, no multicast).
+    Times the whole step for the gather and the slice form of the last exchange, max over ranks.
+    device "cpu" with a stand-in for the C ABI (kernels) runs the same code under gloo in the tests."""
+    import torch
+    import torch.distributed as dist
+    from paper_2109_12497_b200.distributed import DistributedQuantizer
+    world, rank = dist.get_world_size(), dist.get_rank()
+    if w.M % world:
+        return {"skipped": f"{w.M} workers do not divide over {world} processes"}
+    on_gpu = str(device).startswith("cuda")
+    K = kernels
+    if K is None:
+        from paper_2109_12497_b200 import binding as K
+    M_local = w.M // world
+    fmt = {"i8": 0, "i4x2": 1, "i2x4": 2, "i6p": 3}[w.fmt]           # UQ_FMT_* of include/uq.h
+    g_np = wl.generate(w, threads=threads, workers=range(rank * M_local, (rank + 1) * M_local))
+    t = torch.from_numpy(g_np.view(np.float32 if w.dtype == wl.F32 else np.int16))
+    if w.dtype == wl.BF16:
+        t = t.view(torch.bfloat16)
+    rec = {"processes": world, "workers_per_process": M_local,
+           "note": "whole step with the workers spread over the processes: max all-reduce of the scales, [exchange + "
+                   "minimum of the packed scale indices,] exchange of the level rows in their wire format, fused sum + "
+                   "reconstruction; gradient GB/s counts the gradients of all processes"}
+    out_last = None
+    for exchange in ("gather", "slices"):
+        if exchange == "slices" and w.fmt == "i6p":
+            continue                                   # two-plane rows are not cut into slices
+        q = DistributedQuantizer(
+            M_local, w.d, torch.float32 if w.dtype == wl.F32 else torch.bfloat16, seg_off=wl.segment_offsets(w),
+            s=w.s, scales=list(w.scales) if w.quantizer == "multi" else None, fmt=fmt, idx_bits=w.idx_bits,
+            norm=K.UQ_NORM_L2 if w.norm == wl.NORM_L2 else K.UQ_NORM_LINF, rng_bits=w.rng_bits, device=device,
+            kernels=kernels, exchange=exchange)
+        g = torch.zeros((M_local, q.stride), dtype=t.dtype, device=device)
+        g[:, : t.shape[1]] = t.to(device)
+        for k in range(warmup):
+            q.step(g, w.seed + k)
+        if on_gpu:
+            st = torch.cuda.current_stream()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+        dist.barrier()
+        t0 = time.perf_counter()
+        if on_gpu:
+            e0.record(st)
+        for k in range(steps):
+            out = q.step(g, w.seed + k)
+        if on_gpu:
+            e1.record(st)
+            torch.cuda.synchronize()
+            ms_mine = e0.elapsed_time(e1) / steps
+        else:
+            ms_mine = (time.perf_counter() - t0) * 1e3 / steps
+        dist.barrier()
+        (ms,) = max_over_ranks([ms_mine], device)
+        rec[exchange] = {"ms_per_step": round(ms, 5), "gradient_GBps": round(w.in_bytes / ms / 1e6, 6),
+                         "wire_bytes_received_per_process_and_step": int(q.wire_bytes_per_step()),
+                         "status_word": int(q.status.item())}
+        if exchange == "gather":
+            out_last = out.detach().cpu().numpy().copy()
+        del q, g
+    return (rec, out_last) if return_out else rec
+
+
 def other_workloads(rng_bits):
     """The workloads reported beside the headline one: the other four configurations, c2 on the
     2-bit and 6-bit wires, and c3 with its shared index sent in 2, 4 and 8 bits."""
@@ -771,6 +837,11 @@ def gpu_main(args):
             one = cpu_baseline(name, 1, max(1, args.cpu_coords // 16))      # one thread, a sixteenth of the sample
             line["cpu_baseline"]["single_thread"] = {"value": one["value"], "unit": UNIT, "sample": one["sample"],
                                                      "seconds": one["seconds"]}
+    if world > 1:
+        # the workers of the same workload spread over the processes, with real exchanges (every rank takes part)
+        del res, q
+        torch.cuda.empty_cache()
+        line["distributed"] = bench_distributed(w, args.steps, args.warmup, "cuda", threads)
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:

@@ -46,7 +46,6 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     objdir = PKG / "build"
     objdir.mkdir(exist_ok=True)
     extra = ["-Xptxas", "-v"] if verbose else []
-    extra += os.environ.get("UQ_NVCC_FLAGS", "").split()        # e.g. -DUQ_ENCODE_MIN_CTAS=3 for tuning runs
 
     def compile_one(src: str) -> Path:
         obj = objdir / (src + ".o")

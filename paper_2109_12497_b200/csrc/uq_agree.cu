@@ -188,6 +188,8 @@ cudaError_t launch_agree_scale(const uq_layout &L, const void *g, int norm, floa
 // ---------------------------------------------------------------------------------------------
 #include <mutex>
 
+namespace uq { int record_cuda_error(cudaError_t e); }
+
 namespace {
 
 // Scratch for the norm partials, part of the library image: every GPU that loads the library
@@ -228,7 +230,8 @@ extern "C" int uq_agree_scale_static(const uq_layout *layout, const void *g, int
     if (need == 0) return UQ_ERR_BAD_ARG;                       // the layout itself is invalid
     if (need > (size_t)UQ_STATIC_SCRATCH_BYTES) return UQ_ERR_WORKSPACE;
     void *scratch = nullptr;
-    if (static_scratch(&scratch) != cudaSuccess) return UQ_ERR_CUDA;
+    const cudaError_t e = static_scratch(&scratch);
+    if (e != cudaSuccess) return uq::record_cuda_error(e);      // the code is kept for uq_last_cuda_error()
     // the partials are all written before they are read, so nothing in the array needs clearing
     return uq_agree_scale(layout, g, norm, W, status, scratch, (size_t)UQ_STATIC_SCRATCH_BYTES, stream);
 }

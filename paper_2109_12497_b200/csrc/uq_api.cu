@@ -40,15 +40,23 @@ cudaError_t launch_small_step_multi(const uq_layout &L, const void *g, int norm,
 }  // namespace uq
 
 namespace {
-
 thread_local int g_last_cuda_error = 0;
+}
 
-int finish(cudaError_t e)
+namespace uq {
+// UQ_OK, or UQ_ERR_CUDA with the code kept for uq_last_cuda_error() (every entry point of the
+// library reports its CUDA failures through here, whichever file it lives in).
+int record_cuda_error(cudaError_t e)
 {
     if (e == cudaSuccess) return UQ_OK;
     g_last_cuda_error = (int)e;
     return UQ_ERR_CUDA;
 }
+}  // namespace uq
+
+namespace {
+
+int finish(cudaError_t e) { return uq::record_cuda_error(e); }
 
 bool aligned(const void *p, size_t a) { return ((uintptr_t)p & (a - 1)) == 0; }
 

@@ -122,12 +122,15 @@ __device__ __noinline__ void encode_span_general(const EncodeParams &p, int m, i
     }
 }
 
-// A full tile that a segment boundary crosses, all 256 threads: the warps walk their 256-coordinate
-// rows one by one.  Lane L takes the end of segment j + L (j = the tile's first segment), so the
-// segment of a row is j + (number of ends at or before the row's start): one ballot per row instead
-// of a search.  A row that itself contains a boundary is skipped: a CTA of the second kind owns it.
+// A full tile that a segment boundary crosses, all 256 threads, workers m0 .. m1 - 1: the warps
+// walk their 256-coordinate rows one by one.  Lane L takes the end of segment j + L (j = the
+// tile's first segment), so the segment of a row is j + (number of ends at or before the row's
+// start): one ballot per row instead of a search.  What a row's workers share (its segment, the
+// factors s_k / W, the shared indices) is found once per row; the rows of four workers are in
+// flight together.  A row that itself contains a boundary is skipped: a CTA of the second kind
+// owns it.
 template <int DT, int FMT, int RNG, int IDXB>
-__device__ __noinline__ void encode_tile_mixed(const EncodeParams &p, int m, int64_t t0, int j)
+__device__ __noinline__ void encode_tile_mixed(const EncodeParams &p, int m0, int m1, int64_t t0, int j)
 {
     using E = Elem<DT>;
     using S = EncodeShape<DT, RNG>;
@@ -136,11 +139,11 @@ __device__ __noinline__ void encode_tile_mixed(const EncodeParams &p, int m, int
     constexpr int IB = MULTI ? IDXB : 8;
     constexpr int H = 8 / E::G;
     constexpr int KMASK = IB < 4 ? (1 << IB) - 1 : UQ_MAX_SCALES - 1;
+    constexpr int G = 4;                                         // workers whose rows are loaded together
     const int tid = threadIdx.x, lane = tid & 31;
     const int32_t my_scale = p.v.scales.s[lane & KMASK];
     const int64_t my_end = j + lane < p.v.nseg ? segment_end(p.v.seg_off, p.v.nseg, j + lane, p.v.d) : INT64_MAX;
-    const char *grow = (const char *)p.v.g + (size_t)m * (size_t)p.v.stride * E::BYTES;
-    char *lrow = (char *)p.lev + (size_t)m * LF::row_bytes(p.v.stride);
+    const size_t grow = (size_t)p.v.stride * E::BYTES, lrow = LF::row_bytes(p.v.stride);
     bool overflow = false;
 #pragma unroll 1
     for (int u = 0; u < S::UNITS; ++u) {
@@ -159,23 +162,39 @@ __device__ __noinline__ void encode_tile_mixed(const EncodeParams &p, int m, int
         const float inv_lane = inv_scale(my_scale, __ldg(p.v.W + jr));
         overflow |= not_finite(inv_lane);
         const int64_t i = r0 + lane * 8;
-        uint4 q[H];
-        float v[8], inv[8];
-#pragma unroll
-        for (int h = 0; h < H; ++h) {
-            q[h] = ld_stream(grow + (i + h * E::G) * E::BYTES);
-            E::unpack(q[h], *(float(*)[E::G])(v + h * E::G));
-        }
         typename IdxBits<IB>::T kbits = 0;
         if (MULTI) kbits = p.select ? IdxBits<IB>::load_written(p.idx + i * IB / 8) : IdxBits<IB>::load(p.idx + i * IB / 8);
+        float inv[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e)
             inv[e] = MULTI ? __shfl_sync(0xFFFFFFFFu, inv_lane, (int)(uint32_t)(kbits >> (e * IB))) : inv_lane;
-        uint32_t neg_lo, neg_hi;
-        unit_signs<DT>(q, neg_lo, neg_hi);
         const uint64_t blk = RNG == 32 ? (uint64_t)((p.coord0 + i) >> 2) : (uint64_t)((p.coord0 + i) >> 3);
-        quantize_unit<FMT, RNG>(v, inv, p.v.s_hat, neg_lo, neg_hi, p.key, (uint32_t)blk, (uint32_t)(blk >> 32),
-                                (uint32_t)(m + p.worker0), lrow + LF::off(i), lrow + LF::off2(i, p.v.stride));
+        const char *gp = (const char *)p.v.g + (size_t)m0 * grow + (size_t)i * E::BYTES;
+        char *lp = (char *)p.lev + (size_t)m0 * lrow;
+#pragma unroll 1
+        for (int m = m0; m < m1; m += G) {
+            uint4 q[G][H];
+#pragma unroll
+            for (int k = 0; k < G; ++k)
+                if (m + k < m1) {
+#pragma unroll
+                    for (int h = 0; h < H; ++h) q[k][h] = ld_stream(gp + (size_t)k * grow + h * E::G * E::BYTES);
+                }
+#pragma unroll
+            for (int k = 0; k < G; ++k)
+                if (m + k < m1) {
+                    float v[8];
+#pragma unroll
+                    for (int h = 0; h < H; ++h) E::unpack(q[k][h], *(float(*)[E::G])(v + h * E::G));
+                    uint32_t neg_lo, neg_hi;
+                    unit_signs<DT>(q[k], neg_lo, neg_hi);
+                    quantize_unit<FMT, RNG>(v, inv, p.v.s_hat, neg_lo, neg_hi, p.key, (uint32_t)blk, (uint32_t)(blk >> 32),
+                                            (uint32_t)(m + k + p.worker0), lp + (size_t)k * lrow + LF::off(i),
+                                            lp + (size_t)k * lrow + LF::off2(i, p.v.stride));
+                }
+            gp += G * grow;
+            lp += G * lrow;
+        }
     }
     if (overflow && lane < p.v.scales.N && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
 }
@@ -202,10 +221,11 @@ __device__ __noinline__ void encode_tile_slow(const EncodeParams &p, int64_t t0,
         }
         __syncthreads();                                             // the tile's indices are in memory for all warps
     }
-    for (int m = m0; m < m1; ++m) {
-        if (j < 0) encode_span_general<DT, FMT, RNG, IDXB>(p, m, t0, t1, threadIdx.x, kThreads);
-        else encode_tile_mixed<DT, FMT, RNG, IDXB>(p, m, t0, j);
+    if (j >= 0) {
+        encode_tile_mixed<DT, FMT, RNG, IDXB>(p, m0, m1, t0, j);
+        return;
     }
+    for (int m = m0; m < m1; ++m) encode_span_general<DT, FMT, RNG, IDXB>(p, m, t0, t1, threadIdx.x, kThreads);
 }
 
 // State of a tile that does not depend on the worker.

@@ -17,9 +17,10 @@ and layer structure are stated recipes:
   c5  multi-scale, M=8, d=335,141,888 bf16, N(0, 0.02^2) with 1% of the coordinates x100
       (same coordinates on every worker), 25 MiB buckets, scale set {127 * 8^k, k<8}, 4-bit index
 
-c1 to c4 draw 32 random bits per coordinate (``rng_bits``, 23 of them used), the library's default;
-c5 draws 16: its bf16 encoder moves 3.5 bytes per coordinate and is bound by arithmetic, not by
-memory, with 32-bit draws.  Both widths are tested and timed on every workload.
+c1 to c3 draw 32 random bits per coordinate (``rng_bits``, 23 of them used), the library's default;
+c4 and c5 draw 16: their encoders move only 4.5 and 3.5 bytes per coordinate and are bound by
+arithmetic, not by memory, with 32-bit draws (measured: 0.70 and 0.58 of the copy peak, ALU and
+multiply pipes the busiest units).  Both widths are tested and timed on every workload.
 
 ``scaled(name, d)`` gives the same recipe at a smaller d for tests.
 """
@@ -77,7 +78,7 @@ WORKLOADS = {
     "c3": Workload("c3", "multi", 8, 25_557_032, F32, "layers", "layers161", 127,
                    _geom(127, 8, 4), "i8", 2, NORM_L2, 0, 1002, nseg_hint=161),
     "c4": Workload("c4", "single", 16, 1 << 26, F32, "student_t3", "one", 7, (7,), "i4x2", 0,
-                   NORM_L2, 0, 1004),
+                   NORM_L2, 0, 1004, rng_bits=16),
     "c5": Workload("c5", "multi", 8, 335_141_888, BF16, "normal_outliers", "buckets25MiB", 127,
                    _geom(127, 8, 8), "i8", 4, NORM_L2, 0, 1005, rng_bits=16,
                    bucket_elems=25 * (1 << 20) // 2),
@@ -188,16 +189,19 @@ def _fill_worker(w: Workload, m: int, row: np.ndarray, seg_off: np.ndarray, std:
             row[c0:c0 + n] = f32_to_bf16_bits(x)
 
 
-def generate(w: Workload, out: Optional[np.ndarray] = None, threads: int = 8) -> np.ndarray:
+def generate(w: Workload, out: Optional[np.ndarray] = None, threads: int = 8, workers=None) -> np.ndarray:
     """Gradients of all workers as an [M, stride] array (float32, or uint16 holding bf16 bits);
-    columns d..stride-1 are zero padding.  ``out`` may be a preallocated (e.g. pinned) buffer."""
+    columns d..stride-1 are zero padding.  ``out`` may be a preallocated (e.g. pinned) buffer.
+    ``workers`` (a sequence of worker numbers) makes only those workers' rows, in that order: a
+    process that holds part of the job's workers gets exactly the rows the whole array has."""
     np_dtype = np.float32 if w.dtype == F32 else np.uint16
+    rows = list(range(w.M)) if workers is None else [int(m) for m in workers]
     if out is None:
-        out = np.zeros((w.M, w.stride), dtype=np_dtype)
-    assert out.shape == (w.M, w.stride) and out.dtype == np_dtype
+        out = np.zeros((len(rows), w.stride), dtype=np_dtype)
+    assert out.shape == (len(rows), w.stride) and out.dtype == np_dtype
     out[:, w.d:] = 0
     seg_off = segment_offsets(w)
     std = _layer_std(w, seg_off) if w.values == "layers" else None
     with ThreadPoolExecutor(max_workers=max(1, threads)) as pool:
-        list(pool.map(lambda m: _fill_worker(w, m, out[m], seg_off, std), range(w.M)))
+        list(pool.map(lambda k: _fill_worker(w, rows[k], out[k], seg_off, std), range(len(rows))))
     return out
