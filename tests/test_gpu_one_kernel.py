@@ -1,6 +1,7 @@
 """uq_step_small: the whole step of either quantizer as one cooperative kernel, against the oracle
 and against the separate calls."""
 import ctypes as C
+import dataclasses
 
 import numpy as np
 import pytest
@@ -189,3 +190,28 @@ def test_multi_scale_steps_back_to_back():
     assert np.array_equal(q.lev.cpu().numpy()[:, : w.d], lev)
     assert np.array_equal(q.S.cpu().numpy()[: w.d], o.aggregate(lev))
     assert np.array_equal(q.out.cpu().numpy()[: w.d], o.decode(o.aggregate(lev), w.M, W, scales=w.scales, idx=idx))
+
+
+def test_agree_scale_between_steps_does_not_disturb_the_barrier():
+    """A one-kernel quantizer whose separate stages are called between its steps (as the benchmark
+    does): the norm kernels' scratch and the step's barrier counters are different buffers, so every
+    step still waits at its barrier and computes its own W.  Different gradients every step, L2
+    norm (a stale or half-written partial would change W), each step compared with the oracle."""
+    w = wl.scaled("c1", 300_001, M=5, norm=wl.NORM_L2)
+    q = from_workload(w, keep_sums=True, one_kernel=True)
+    assert q.one_kernel and q.small_workspace.data_ptr() != q.workspace.data_ptr()
+    for step in range(6):
+        g_np = wl.generate(dataclasses.replace(w, data_seed=w.data_seed + step)) * np.float32(1 + step)
+        g = to_device(w, g_np)
+        other = to_device(w, wl.generate(dataclasses.replace(w, data_seed=77 + step)))
+        q.agree_scale(other)                                  # the separate call, on other data, right before the step
+        q.step(g, 1000 + step)
+        torch.cuda.synchronize()
+        assert q.status_bits() == 0
+        W = q.W.cpu().numpy()
+        W_ref = o.agree_scale(g_np[:, : w.d], None, o.NORM_L2)
+        assert np.abs(W.view(np.int32).astype(np.int64) - W_ref.view(np.int32)).max() <= 1
+        lev = o.encode_single(g_np[:, : w.d], W, w.s, 1000 + step, w.rng_bits)
+        assert np.array_equal(q.lev.cpu().numpy()[:, : w.d], lev)
+        assert np.array_equal(q.S.cpu().numpy()[: w.d], o.aggregate(lev))
+        assert int(q.small_workspace[:64].sum().item()) == 0  # the counters are back at zero after every step

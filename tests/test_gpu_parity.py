@@ -398,3 +398,28 @@ def test_back_to_back_steps_do_not_interfere(name):
         bad += (q.S != S0).sum() + (q.out != out0).sum() + (q.lev[:, : w.d] != lev0[:, : w.d]).sum()
     torch.cuda.synchronize()
     assert int(bad.item()) == 0
+
+
+@pytest.mark.parametrize("name,kw", [("c2", dict(rng_bits=16)), ("c2", dict(rng_bits=32)), ("c3", dict(rng_bits=16)),
+                                      ("c5", {}), ("c4", {})])
+@pytest.mark.parametrize("power", [100, 112, -100])
+def test_gradients_of_extreme_magnitude(name, kw, power):
+    """Gradients scaled by 2^power.  Beyond W = s * 2^100 the factor s / W is too small for the
+    encoder's saturating form of the clamp (its division by 256 would no longer be exact), and the
+    kernel must take its plain path for such tiles; tiny gradients exercise large factors.  A
+    power-of-two scaling changes no level (the oracle says so too), so the levels are also compared
+    with those of the unscaled gradients."""
+    w = wl.scaled(name, 150_001, M=4 if name != "c4" else 16, **kw)
+    g = wl.generate(w)
+    if w.dtype == wl.BF16:
+        f = wl.bf16_bits_to_f32(g) * np.float32(2.0 ** power)
+        big = wl.f32_to_bf16_bits(f)
+    else:
+        big = g * np.float32(2.0 ** power)
+    assert np.isfinite(big.astype(np.float32) if w.dtype == wl.F32 else wl.bf16_bits_to_f32(big)).all()
+    r = check_parity(w, big)
+    if abs(power) <= 100 or w.dtype == wl.F32:
+        base = check_parity(w, g)
+        if power > 0:                                       # nothing underflows on the way up
+            nb = base["ref"]["lev"].shape[1]
+            assert np.array_equal(r["lev"][:, :nb], base["lev"][:, :nb])
