@@ -256,34 +256,47 @@ def time_alone(fn, reps, sustained=False, ms_hint=1.0, lead_s=0.6, span_s=0.4):
 
 def time_end_to_end(q, g_host, out_host, g_dev, w, steps, warmup, barrier):
     """ms per step with the gradients starting in pinned host memory and the result read back.
-    Every step copies its own inputs in and its own result out; the read-back of step k runs on
-    a second stream while the inputs of step k+1 arrive (the two directions of the link are
-    independent), ordered by events: kernels(k) after copy-in(k); copy-in(k+1) and read-back(k)
-    after kernels(k); kernels(k+1) after read-back(k)."""
+    Every step copies its own inputs in and its own result out.  Three streams, ordered by events:
+    the inputs of step k+1 arrive (copy stream, into the other of two device buffers) while the
+    kernels of step k run (main stream) and the result of step k-1 is read back (a third stream;
+    the two directions of the link are independent).  Kernels(k) wait for copy-in(k) and for the
+    read-back of result k-1 (the output buffer is reused); copy-in(k+2) waits for kernels(k) (its
+    buffer is free again)."""
     import torch
     main = torch.cuda.current_stream()
-    back = torch.cuda.Stream()
-    done = [torch.cuda.Event() for _ in range(2)]             # kernels of a step finished / result read back
+    copy, back = torch.cuda.Stream(), torch.cuda.Stream()
+    bufs = [g_dev, torch.empty_like(g_dev)]
+    copied = [torch.cuda.Event() for _ in range(2)]           # inputs of the step using buffer b have arrived
+    computed = [torch.cuda.Event() for _ in range(2)]         # kernels of the step using buffer b have finished
+    read_back = torch.cuda.Event()                            # the latest result has left the output buffer
 
     def one(k):
-        g_dev.copy_(g_host, non_blocking=True)                # main: inputs of this step
-        main.wait_event(done[1])                              # the previous result has left the output buffer
-        out = q.step(g_dev, w.seed + k)
-        done[0].record(main)
-        back.wait_event(done[0])
+        b = k & 1
+        with torch.cuda.stream(copy):
+            copy.wait_event(computed[b])                      # the step that used this buffer before is done
+            bufs[b].copy_(g_host, non_blocking=True)
+            copied[b].record(copy)
+        main.wait_event(copied[b])
+        main.wait_event(read_back)
+        out = q.step(bufs[b], w.seed + k)
+        computed[b].record(main)
         with torch.cuda.stream(back):
+            back.wait_event(computed[b])
             out_host.copy_(out, non_blocking=True)
-            done[1].record(back)
+            read_back.record(back)
 
-    done[1].record(main)
+    for ev in computed:
+        ev.record(main)
+    read_back.record(main)
     for k in range(min(warmup, 3)):
         one(k)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize(); barrier()
     e0.record(main)
+    copy.wait_event(e0)                                       # no copy of a timed step starts before the clock
     for k in range(steps):
         one(k)
-    main.wait_event(done[1])                                  # the last read-back is inside the timed region
+    main.wait_event(read_back)                                # the last read-back is inside the timed region
     e1.record(main)
     torch.cuda.synchronize(); barrier()
     return e0.elapsed_time(e1) / steps
