@@ -379,6 +379,22 @@ __device__ __forceinline__ uint32_t level_draw23(float x, uint32_t word)
 }
 constexpr uint32_t kLevelByte23 = 0;      // which byte of the returned word holds the level
 
+// The same level from the fixed-point form of x (the fast path of the encoder).  inv23 = inv * 2^23
+// and cap23 = cap * 2^23, both exact, so |v| * inv23 = x * 2^23 with the rounding of x (the caller
+// checks that inv23 is finite; a product below the normal range gives threshold 0 either way), and
+//   T = rint(min(x, cap) * 2^23) = floor(x) * 2^23 + rint(p * 2^23)
+// by one conversion (ties to even; x >= 1 is a multiple of 2^-23, so only p < 1 is rounded, and a
+// p that rounds up to 1 carries into the level, as it must: then every draw rounds up).  With
+// r = word >> 9 the level is (T + 2^23 - 1 - r) >> 23.  Doubled, so that it lands on a byte:
+// 2T + (~word >> 8) = 2T + 2 (2^23 - 1 - r) + (0 or 1) has the level in byte 3 (at most
+// 127 * 2^24 + 2^25 - 1: no overflow), and the stray low bit cannot carry.
+__device__ __forceinline__ uint32_t level_draw23_fixed(float v, float inv23, float cap23, uint32_t word)
+{
+    const uint32_t T = (uint32_t)__float2int_rn(fminf(__fmul_rn(fabsf(v), inv23), cap23));
+    return T + T + (~word >> 8);
+}
+constexpr uint32_t kLevelByte23Fixed = 3;
+
 // 16-bit draw.  Returns a word whose byte 2 is the unsigned level.
 // x + 128 rounds x to 16 fractional bits (ties to even): the mantissa of the sum is
 // floor(x) * 2^16 + rint(p * 2^16); adding 0xFFFF - h carries into bit 16 iff

@@ -235,9 +235,10 @@ template <int DT, int FMT, int RNG, int IDXB> struct TileState {
     static constexpr int U = S::UNITS;
     static constexpr int H = 8 / E::G;                           // 16-byte loads per unit
     static constexpr int BPU = RNG == 32 ? 2 : 1;                // Philox blocks per unit
-    float inv[U][8];                  // factor of every coordinate (divided by 256 for 16-bit draws)
+    float inv[U][8];                  // factor of every coordinate: / 256 for 16-bit draws, * 2^23 for 32-bit draws
     PhiloxBlockPart blk[U * BPU];     // worker-independent rounds of the units' Philox blocks
-    SatConstants sc;
+    SatConstants sc;                  // 16-bit draws
+    float cap23;                      // 32-bit draws: the largest level * 2^23
     const char *gp;                   // my first coordinate in the gradient row that is loaded next
     const uint4 *sp;                  // select mode: my slot of that row's copy in shared memory
     char *lp, *lp2;                   // and in the level row that is stored next (second plane for 6-bit)
@@ -286,9 +287,9 @@ __device__ __forceinline__ void encode_workers(const EncodeParams &p, TileState<
             if (RNG == 16) {
                 quantize_unit_bytes_sat16(v, t.inv[u], t.sc, neg_lo, neg_hi, r[u], lo, hi);
             } else {
-                UnitWords<RNG> rw;
-                rw.r[0] = r[u * T::BPU]; rw.r[RNG == 32 ? 1 : 0] = r[u * T::BPU + T::BPU - 1];
-                quantize_unit_bytes<RNG>(v, t.inv[u], p.v.s_hat, neg_lo, neg_hi, rw, lo, hi);
+                UnitWords<32> rw;
+                rw.r[0] = r[u * T::BPU]; rw.r[1] = r[u * T::BPU + T::BPU - 1];
+                quantize_unit_bytes_fixed23(v, t.inv[u], t.cap23, neg_lo, neg_hi, rw, lo, hi);
             }
             store_unit<FMT>(lo, hi, t.lp + u * kThreads * UB, t.lp2 + u * kThreads * UB2);
         }
@@ -459,7 +460,10 @@ __global__ void __launch_bounds__(kThreads, (SEL ? 3 : EncodeShape<DT, RNG>::MIN
     const float W = __ldg(p.v.W + j);
     float inv_lane = inv_scale(p.v.scales.s[lane & KMASK], W);
     if (lane < p.v.scales.N && not_finite(inv_lane) && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
-    if (RNG == 16 && !sat_form_exact(inv_scale(p.v.scales.s[0], W))) {   // W beyond 2^100: the plain arithmetic
+    // a W so large (16-bit draws) or so small (32-bit) that the rescaled factors of the fast forms
+    // would leave the normal range: the plain arithmetic
+    if (RNG == 16 ? !sat_form_exact(inv_scale(p.v.scales.s[0], W))
+                  : !fixed_form_exact(inv_scale(p.v.scales.s[p.v.scales.N - 1], W))) {
         if (SEL) copy_async_wait();
         encode_tile_slow<DT, FMT, RNG, IDXB>(p, t0, t1, -1, m0, m0 + cnt, sh_thr);
         return;
@@ -498,6 +502,9 @@ __global__ void __launch_bounds__(kThreads, (SEL ? 3 : EncodeShape<DT, RNG>::MIN
     if (RNG == 16) {
         inv_lane = __fmul_rn(inv_lane, 0.00390625f);
         t.sc = sat_constants(p.v.s_hat);
+    } else {
+        inv_lane = __fmul_rn(inv_lane, 8388608.0f);
+        t.cap23 = __fmul_rn(p.v.s_hat, 8388608.0f);
     }
     // the shuffle reads its source lane modulo 32 and the table repeats every 2^IB lanes (an 8-bit
     // index is below 16), so the index bits need a shift but no mask

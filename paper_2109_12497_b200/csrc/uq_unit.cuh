@@ -89,6 +89,25 @@ __device__ __forceinline__ void quantize_unit_bytes(const float (&v)[8], const f
     hi = negate_bytes(gather_bytes<LB>(z[4], z[5], z[6], z[7]), neg_hi);
 }
 
+// The same for 23-bit draws in the fixed-point form (level_draw23_fixed): inv23[e] = inv[e] * 2^23,
+// cap23 = cap * 2^23.  fixed_form_exact says whether a tile may take it, given the largest of its
+// factors: beyond 2^100 (W below 2^-93 or so; also Inf and NaN) the scaled factor could overflow,
+// and the tile takes the plain arithmetic.
+__device__ __forceinline__ bool fixed_form_exact(float inv_max) { return inv_max <= 1.2676506e30f; }
+
+__device__ __forceinline__ void quantize_unit_bytes_fixed23(const float (&v)[8], const float (&inv23)[8], float cap23,
+                                                            uint32_t neg_lo, uint32_t neg_hi, const UnitWords<32> &rw,
+                                                            uint32_t &lo, uint32_t &hi)
+{
+    const uint4 r0 = rw.r[0], r1 = rw.r[1];
+    const uint32_t w[8] = { r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w };
+    uint32_t z[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) z[e] = level_draw23_fixed(v[e], inv23[e], cap23, w[e]);
+    lo = negate_bytes(gather_bytes<kLevelByte23Fixed>(z[0], z[1], z[2], z[3]), neg_lo);
+    hi = negate_bytes(gather_bytes<kLevelByte23Fixed>(z[4], z[5], z[6], z[7]), neg_hi);
+}
+
 // The same for 16-bit draws with the clamp in saturating arithmetic (level_draw16_sat): inv256[e]
 // is the coordinate's factor divided by 256, (c0, adj) come from sat_constants(cap).
 struct SatConstants { float c0; uint32_t adj; };

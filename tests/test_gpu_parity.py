@@ -401,12 +401,14 @@ def test_back_to_back_steps_do_not_interfere(name):
 
 
 @pytest.mark.parametrize("name,kw", [("c2", dict(rng_bits=16)), ("c2", dict(rng_bits=32)), ("c3", dict(rng_bits=16)),
-                                      ("c5", {}), ("c4", {})])
-@pytest.mark.parametrize("power", [100, 112, -100])
+                                      ("c3", dict(rng_bits=32)), ("c5", {}), ("c5", dict(rng_bits=32)), ("c4", {}),
+                                      ("c4", dict(rng_bits=32))])
+@pytest.mark.parametrize("power", [100, 112, -80, -100])
 def test_gradients_of_extreme_magnitude(name, kw, power):
     """Gradients scaled by 2^power.  Beyond W = s * 2^100 the factor s / W is too small for the
-    encoder's saturating form of the clamp (its division by 256 would no longer be exact), and the
-    kernel must take its plain path for such tiles; tiny gradients exercise large factors.  A
+    encoder's saturating form of the clamp with 16-bit draws (its division by 256 would no longer be
+    exact), and below W = s * 2^-100 it is too large for the fixed-point form with 32-bit draws
+    (times 2^23 it could overflow): the kernel must take its plain path for such tiles.  A
     power-of-two scaling changes no level (the oracle says so too), so the levels are also compared
     with those of the unscaled gradients."""
     w = wl.scaled(name, 150_001, M=4 if name != "c4" else 16, **kw)
@@ -423,3 +425,39 @@ def test_gradients_of_extreme_magnitude(name, kw, power):
         if power > 0:                                       # nothing underflows on the way up
             nb = base["ref"]["lev"].shape[1]
             assert np.array_equal(r["lev"][:, :nb], base["lev"][:, :nb])
+
+
+@pytest.mark.parametrize("multi", [False, True])
+@pytest.mark.parametrize("rng_bits", [16, 32])
+def test_draws_at_the_edges_of_the_threshold(multi, rng_bits):
+    """Scaled magnitudes x that sit on and next to the points where the draw threshold rint(p * 2^b)
+    changes or carries: just below an integer (p rounds up to 1: every draw rounds up), just above
+    one, exact ties between two thresholds, the clamp at the largest level.  W = 127 under the
+    L-infinity norm with s = 127 makes the factor s / W exactly 1, so x = |v|."""
+    ulp = lambda x: np.spacing(np.float32(x))
+    xs = []
+    for k in [0, 1, 2, 3, 63, 64, 126]:
+        base = np.float32(k)
+        for t in [1.0, 0.5, 0.25, 2.0 ** -15, 2.0 ** -16, 2.0 ** -17, 2.0 ** -22, 2.0 ** -23, 2.0 ** -24, 2.0 ** -25, 2.0 ** -30]:
+            for sgn in (1.0, -1.0):
+                x = np.float32(base + np.float32(0.5) + np.float32(sgn * t * 0.5))
+                xs += [x, np.float32(x - ulp(x)), np.float32(x + ulp(x))]
+                x = np.float32(base + np.float32(1.0 if sgn < 0 else 0.0) + np.float32(sgn * t))
+                xs += [x, np.float32(x - ulp(x)) if x > 0 else x, np.float32(x + ulp(x))]
+    xs = np.array([x for x in xs if 0.0 <= x <= 127.0], dtype=np.float32)
+    xs = np.concatenate([xs, -xs, np.float32([127.0, -127.0, 126.99999, 0.0, -0.0, 1e-38, 1e-44, 0.99999994, 0.49999997])])
+    reps = 40                                                # the same value under many different draws
+    d = xs.size * reps
+    if multi:
+        w = wl.scaled("c3", d, M=3, rng_bits=rng_bits, norm=wl.NORM_LINF)
+        w = dataclasses.replace(w, segments="one")
+    else:
+        w = wl.scaled("c1", d, M=3, rng_bits=rng_bits, norm=wl.NORM_LINF)
+    g = np.zeros((w.M, w.stride), dtype=np.float32)
+    rng = np.random.default_rng(5)
+    for m in range(w.M):
+        g[m, :d] = np.tile(xs, reps)[rng.permutation(d)] if m else np.tile(xs, reps)
+    assert np.abs(g).max() == np.float32(127.0)
+    for seed in (0, 1, 0xFFFF_FFFF_FFFF):
+        r = check_parity(w, g, seed=seed)
+        assert r["W"][0] == np.float32(127.0)
