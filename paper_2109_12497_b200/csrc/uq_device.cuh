@@ -62,12 +62,14 @@ struct ScaleSet {                        // the scale set s_ of the multi-scale 
 
 // The low two bits of the eight bytes of (lo, hi), coordinate order kept: byte t of lo lands in
 // bits 2t..2t+1, byte t of hi in bits 8+2t..9+2t (levels -1, 0, 1 as two's-complement 2-bit fields).
+// One multiply gathers a word's four fields: with x = c0 + c1 2^8 + c2 2^16 + c3 2^24 (c < 4) and
+// K = 2^24 + 2^18 + 2^12 + 2^6 the product has c0, c1, c2, c3 at bits 24, 26, 28, 30; every other
+// partial product that stays below 2^32 lies at bit 22 or lower and their sum is below 2^24, so
+// byte 3 of x * K is the packed byte.  Bits 16..31 of the result are unspecified.
 __device__ __forceinline__ uint32_t bytes_to_crumbs(uint32_t lo, uint32_t hi)
 {
-    lo &= 0x03030303u; hi &= 0x03030303u;
-    lo = (lo | (lo >> 6)) & 0x000F000Fu; hi = (hi | (hi >> 6)) & 0x000F000Fu;
-    lo = (lo | (lo >> 12)) & 0x000000FFu; hi = (hi | (hi >> 12)) & 0x000000FFu;
-    return lo | (hi << 8);
+    constexpr uint32_t K = (1u << 24) | (1u << 18) | (1u << 12) | (1u << 6);
+    return __byte_perm((lo & 0x03030303u) * K, (hi & 0x03030303u) * K, 0x4473);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -469,13 +471,12 @@ __device__ __forceinline__ uint32_t negate_bytes(uint32_t mag, uint32_t neg)
     return (mag & ~neg) | (minus & neg);
 }
 
-// The low nibbles of the eight bytes of (lo, hi), packed into 32 bits (byte k -> nibble k).
+// The low nibbles of the eight bytes of (lo, hi), packed into 32 bits (byte k -> nibble k): the
+// even bytes and the odd bytes are gathered into a word each, and the odd ones move up a nibble.
 __device__ __forceinline__ uint32_t bytes_to_nibbles(uint32_t lo, uint32_t hi)
 {
-    lo &= 0x0F0F0F0Fu; hi &= 0x0F0F0F0Fu;
-    lo = (lo | (lo >> 4)) & 0x00FF00FFu; hi = (hi | (hi >> 4)) & 0x00FF00FFu;
-    lo = (lo | (lo >> 8)) & 0x0000FFFFu; hi = (hi | (hi >> 8)) & 0x0000FFFFu;
-    return lo | (hi << 16);
+    const uint32_t even = __byte_perm(lo, hi, 0x6420), odd = __byte_perm(lo, hi, 0x7531);
+    return (even & 0x0F0F0F0Fu) | ((odd << 4) & 0xF0F0F0F0u);
 }
 
 // ---------------------------------------------------------------------------------------------
