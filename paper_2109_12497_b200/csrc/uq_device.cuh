@@ -387,13 +387,14 @@ constexpr uint32_t kLevelByte23 = 0;      // which byte of the returned word hol
 //   T = rint(min(x, cap) * 2^23) = floor(x) * 2^23 + rint(p * 2^23)
 // by one conversion (ties to even; x >= 1 is a multiple of 2^-23, so only p < 1 is rounded, and a
 // p that rounds up to 1 carries into the level, as it must: then every draw rounds up).  With
-// r = word >> 9 the level is (T + 2^23 - 1 - r) >> 23.  Doubled, so that it lands on a byte:
-// 2T + (~word >> 8) = 2T + 2 (2^23 - 1 - r) + (0 or 1) has the level in byte 3 (at most
-// 127 * 2^24 + 2^25 - 1: no overflow), and the stray low bit cannot carry.
+// r = word >> 9 the level is L = (T + 2^23 - 1 - r) >> 23 = ceil((T - r) / 2^23), so
+// -L = floor((r - T) / 2^23).  The function converts the negated product (-T, exactly) and returns
+// y = 2 (-T) + (word >> 8) = 2 (r - T) + (0 or 1): byte 3 of y is -L as a two's-complement byte
+// (-127 .. 0), the stray low bit changes no floor.  negated_bytes_to_signed puts the signs on.
 __device__ __forceinline__ uint32_t level_draw23_fixed(float v, float inv23, float cap23, uint32_t word)
 {
-    const uint32_t T = (uint32_t)__float2int_rn(fminf(__fmul_rn(fabsf(v), inv23), cap23));
-    return T + T + (~word >> 8);
+    const uint32_t Tn = (uint32_t)__float2int_rn(fmaxf(__fmul_rn(-fabsf(v), inv23), -cap23));
+    return Tn + Tn + (word >> 8);
 }
 constexpr uint32_t kLevelByte23Fixed = 3;
 
@@ -469,6 +470,15 @@ __device__ __forceinline__ uint32_t negate_bytes(uint32_t mag, uint32_t neg)
 {
     const uint32_t minus = (0x80808080u - mag) ^ 0x80808080u;
     return (mag & ~neg) | (minus & neg);
+}
+
+// The same for four bytes that hold -L (0, or 0x81 .. 0xFF): where `neg` is 0xFF the byte stays,
+// elsewhere it becomes L.  b ^ 0x80 = 128 - L lies in 1 .. 128, so 0x80 - (b ^ 0x80) = L borrows
+// nothing from the next byte.
+__device__ __forceinline__ uint32_t negated_bytes_to_signed(uint32_t minus, uint32_t neg)
+{
+    const uint32_t mag = 0x80808080u - (minus ^ 0x80808080u);
+    return (minus & neg) | (mag & ~neg);
 }
 
 // The low nibbles of the eight bytes of (lo, hi), packed into 32 bits (byte k -> nibble k): the

@@ -282,16 +282,19 @@ __device__ __forceinline__ void encode_workers(const EncodeParams &p, TileState<
             float v[8];
 #pragma unroll
             for (int h = 0; h < T::H; ++h) T::E::unpack(q[u][h], *(float(*)[T::E::G])(v + h * T::E::G));
+            // binary32 to 4 bits: the unit's bytes in even / odd order, which the store merges directly
+            constexpr bool EO = FMT == UQ_FMT_I4X2 && DT == UQ_F32;
             uint32_t neg_lo, neg_hi, lo, hi;
-            unit_signs<DT>(q[u], neg_lo, neg_hi);
+            unit_signs<DT, EO>(q[u], neg_lo, neg_hi);
             if (RNG == 16) {
-                quantize_unit_bytes_sat16(v, t.inv[u], t.sc, neg_lo, neg_hi, r[u], lo, hi);
+                quantize_unit_bytes_sat16<EO>(v, t.inv[u], t.sc, neg_lo, neg_hi, r[u], lo, hi);
             } else {
                 UnitWords<32> rw;
                 rw.r[0] = r[u * T::BPU]; rw.r[1] = r[u * T::BPU + T::BPU - 1];
-                quantize_unit_bytes_fixed23(v, t.inv[u], t.cap23, neg_lo, neg_hi, rw, lo, hi);
+                quantize_unit_bytes_fixed23<EO>(v, t.inv[u], t.cap23, neg_lo, neg_hi, rw, lo, hi);
             }
-            store_unit<FMT>(lo, hi, t.lp + u * kThreads * UB, t.lp2 + u * kThreads * UB2);
+            if (EO) store_unit_even_odd(lo, hi, t.lp + u * kThreads * UB);
+            else store_unit<FMT>(lo, hi, t.lp + u * kThreads * UB, t.lp2 + u * kThreads * UB2);
         }
         t.lp += t.lrow;
         if (FMT == UQ_FMT_I6P) t.lp2 += t.lrow;

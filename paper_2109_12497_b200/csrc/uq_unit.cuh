@@ -95,6 +95,10 @@ __device__ __forceinline__ void quantize_unit_bytes(const float (&v)[8], const f
 // and the tile takes the plain arithmetic.
 __device__ __forceinline__ bool fixed_form_exact(float inv_max) { return inv_max <= 1.2676506e30f; }
 
+// EO (here and below): `lo` takes the even coordinates 0, 2, 4, 6 and `hi` the odd ones, with the
+// sign masks in the same order (unit_signs<DT, true>); the 4-bit store merges such a pair without
+// a permute (store_unit_even_odd).
+template <bool EO = false>
 __device__ __forceinline__ void quantize_unit_bytes_fixed23(const float (&v)[8], const float (&inv23)[8], float cap23,
                                                             uint32_t neg_lo, uint32_t neg_hi, const UnitWords<32> &rw,
                                                             uint32_t &lo, uint32_t &hi)
@@ -104,8 +108,9 @@ __device__ __forceinline__ void quantize_unit_bytes_fixed23(const float (&v)[8],
     uint32_t z[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) z[e] = level_draw23_fixed(v[e], inv23[e], cap23, w[e]);
-    lo = negate_bytes(gather_bytes<kLevelByte23Fixed>(z[0], z[1], z[2], z[3]), neg_lo);
-    hi = negate_bytes(gather_bytes<kLevelByte23Fixed>(z[4], z[5], z[6], z[7]), neg_hi);
+    constexpr int S = EO ? 2 : 1, B = EO ? 1 : 4;               // coordinate step within a word, first of `hi`
+    lo = negated_bytes_to_signed(gather_bytes<kLevelByte23Fixed>(z[0], z[S], z[2 * S], z[3 * S]), neg_lo);
+    hi = negated_bytes_to_signed(gather_bytes<kLevelByte23Fixed>(z[B], z[B + S], z[B + 2 * S], z[B + 3 * S]), neg_hi);
 }
 
 // The same for 16-bit draws with the clamp in saturating arithmetic (level_draw16_sat): inv256[e]
@@ -122,6 +127,7 @@ __device__ __forceinline__ SatConstants sat_constants(float cap)
 // factor below 2^-100 by 256 could round.  (0, Inf and NaN divide exactly.)
 __device__ __forceinline__ bool sat_form_exact(float inv0) { return !(inv0 > 0.0f && inv0 < 7.888609052e-31f); }
 
+template <bool EO = false>
 __device__ __forceinline__ void quantize_unit_bytes_sat16(const float (&v)[8], const float (&inv256)[8], const SatConstants &sc,
                                                           uint32_t neg_lo, uint32_t neg_hi, const uint4 &r, uint32_t &lo,
                                                           uint32_t &hi)
@@ -133,8 +139,9 @@ __device__ __forceinline__ void quantize_unit_bytes_sat16(const float (&v)[8], c
         const uint32_t h = (e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu);
         z[e] = level_draw16_sat(v[e], inv256[e], sc.c0, sc.adj, h);
     }
-    lo = negate_bytes(gather_bytes<2>(z[0], z[1], z[2], z[3]), neg_lo);
-    hi = negate_bytes(gather_bytes<2>(z[4], z[5], z[6], z[7]), neg_hi);
+    constexpr int S = EO ? 2 : 1, B = EO ? 1 : 4;
+    lo = negate_bytes(gather_bytes<2>(z[0], z[S], z[2 * S], z[3 * S]), neg_lo);
+    hi = negate_bytes(gather_bytes<2>(z[B], z[B + S], z[B + 2 * S], z[B + 3 * S]), neg_hi);
 }
 
 // The level bytes of a unit packed into the wire format and stored.
@@ -149,6 +156,13 @@ template <int FMT> __device__ __forceinline__ void store_unit(uint32_t lo, uint3
         *(uint32_t *)dst = bytes_to_nibbles(lo, hi);
         *(unsigned short *)dst2 = (unsigned short)bytes_to_crumbs(lo >> 4, hi >> 4);
     }
+}
+
+// 4-bit levels from a unit in even / odd order: byte k of `even` is coordinate 2k and becomes the
+// low nibble of byte k, byte k of `odd` the high one.
+__device__ __forceinline__ void store_unit_even_odd(uint32_t even, uint32_t odd, void *dst)
+{
+    *(uint32_t *)dst = (even & 0x0F0F0F0Fu) | ((odd << 4) & 0xF0F0F0F0u);
 }
 
 template <int FMT, int RNG>
@@ -171,9 +185,15 @@ __device__ __forceinline__ void quantize_unit(const float (&v)[8], const float (
 }
 
 // The sign masks of a unit, from the raw loaded words (before any padding is zeroed).
-template <int DT> __device__ __forceinline__ void unit_signs(const uint4 *q, uint32_t &neg_lo, uint32_t &neg_hi)
+template <int DT, bool EO = false> __device__ __forceinline__ void unit_signs(const uint4 *q, uint32_t &neg_lo, uint32_t &neg_hi)
 {
-    if (DT == UQ_F32) {
+    static_assert(!EO || DT == UQ_F32, "even / odd order: binary32 only (for bf16 the masks would cost two more permutes)");
+    if (EO) {
+        neg_lo = sign_bytes_f32(__uint_as_float(q[0].x), __uint_as_float(q[0].z), __uint_as_float(q[1].x),
+                                __uint_as_float(q[1].z));
+        neg_hi = sign_bytes_f32(__uint_as_float(q[0].y), __uint_as_float(q[0].w), __uint_as_float(q[1].y),
+                                __uint_as_float(q[1].w));
+    } else if (DT == UQ_F32) {
         neg_lo = sign_bytes_f32(__uint_as_float(q[0].x), __uint_as_float(q[0].y), __uint_as_float(q[0].z),
                                 __uint_as_float(q[0].w));
         neg_hi = sign_bytes_f32(__uint_as_float(q[1].x), __uint_as_float(q[1].y), __uint_as_float(q[1].z),

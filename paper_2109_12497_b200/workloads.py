@@ -17,10 +17,11 @@ and layer structure are stated recipes:
   c5  multi-scale, M=8, d=335,141,888 bf16, N(0, 0.02^2) with 1% of the coordinates x100
       (same coordinates on every worker), 25 MiB buckets, scale set {127 * 8^k, k<8}, 4-bit index
 
-c1 to c3 draw 32 random bits per coordinate (``rng_bits``, 23 of them used), the library's default;
-c4 and c5 draw 16: their encoders move only 4.5 and 3.5 bytes per coordinate and are bound by
-arithmetic, not by memory, with 32-bit draws (measured: 0.70 and 0.58 of the copy peak, ALU and
-multiply pipes the busiest units).  Both widths are tested and timed on every workload.
+c1 to c4 draw 32 random bits per coordinate (``rng_bits``, 23 of them used), the library's default;
+c5 draws 16: its encoder moves only 3.5 bytes per coordinate and worker and is bound by arithmetic,
+not by memory, with 32-bit draws (measured: 0.65 of the copy peak, ALU and multiply pipes the
+busiest units; the fp32 encoders reach 0.77 to 0.82).  Both widths are tested and timed on every
+workload.
 
 ``scaled(name, d)`` gives the same recipe at a smaller d for tests.
 """
@@ -78,7 +79,7 @@ WORKLOADS = {
     "c3": Workload("c3", "multi", 8, 25_557_032, F32, "layers", "layers161", 127,
                    _geom(127, 8, 4), "i8", 2, NORM_L2, 0, 1002, nseg_hint=161),
     "c4": Workload("c4", "single", 16, 1 << 26, F32, "student_t3", "one", 7, (7,), "i4x2", 0,
-                   NORM_L2, 0, 1004, rng_bits=16),
+                   NORM_L2, 0, 1004),
     "c5": Workload("c5", "multi", 8, 335_141_888, BF16, "normal_outliers", "buckets25MiB", 127,
                    _geom(127, 8, 8), "i8", 4, NORM_L2, 0, 1005, rng_bits=16,
                    bucket_elems=25 * (1 << 20) // 2),
