@@ -43,7 +43,7 @@ FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only
 # Keyed by (workload, kernel); absent = not captured.
 NCU_TRAFFIC_BYTES_PER_COORD = {
     ("c5", "encode"): 23.40,      # profiles/kernel_encode_c5_small_ncu.md: 1170.1 MB for d = 50,000,000
-    ("c2", "encode"): 38.18,      # profiles/kernel_encode_c2_rng32_ncu.md: 975.7 MB at full size (d = 25,557,032)
+    ("c2", "encode"): 38.15,      # profiles/kernel_encode_c2_rng32_ncu.md: 975.7 MB at full size (d = 25,557,032)
 }
 
 
