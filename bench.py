@@ -665,7 +665,7 @@ def whole_job_value(world, in_bytes, ms):
 def bench_distributed(w, steps, warmup, device, threads, kernels=None, return_out=False):
     """The paper's own setting beside the replicas figure: the M workers spread over the processes of
     the job (M / world_size each), the three all-reduces of Algorithm 1 / 2 as real exchanges between
-    them (distributed.DistributedQuantizer: NCCL collectives on GPUs; no peer loads, no multicast).
+    them (distributed.DistributedQuantizer: NCCL collectives on GPUs, nothing else crosses between them).
     Times the whole step for the gather and the slice form of the last exchange, max over ranks.
     device "cpu" with a stand-in for the C ABI (kernels) runs the same code under gloo in the tests."""
     import torch
