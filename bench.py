@@ -254,6 +254,33 @@ def time_alone(fn, reps, sustained=False, ms_hint=1.0, lead_s=0.6, span_s=0.4):
     return e0.elapsed_time(e1) / reps
 
 
+COPY_CONTEXT_MAX_BYTES = 700e6
+
+
+def time_plain_copy(nbytes, reps=15):
+    """Median ms of a plain device copy that moves nbytes in all (nbytes / 2 read, nbytes / 2
+    written; torch's copy_), timed like a stage (events around single calls, warm L2).  Context for
+    the short stages: the copy that defines the HBM peak moves gigabytes, and a copy of a few hundred
+    megabytes does not get near that rate."""
+    import torch
+    n = max(16, int(nbytes) // 2)
+    a = torch.empty(n, dtype=torch.uint8, device="cuda").fill_(1)
+    b = torch.empty_like(a)
+    for _ in range(3):
+        b.copy_(a)
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        b.copy_(a)
+        e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    del a, b
+    return statistics.median(ts)
+
+
 def time_end_to_end(q, g_host, out_host, g_dev, w, steps, warmup, barrier):
     """ms per step with the gradients starting in pinned host memory and the result read back.
     Every step copies its own inputs in and its own result out.  Three streams, ordered by events:
@@ -500,6 +527,11 @@ def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=F
         res["ms_graph"] = time_graph_replay(q, g_dev, w, max(steps, 20))
     res["ms"], res["stages_ms"] = time_device_resident(q, g_dev, w, steps, warmup, barrier)
     time.sleep(BURST_IDLE_S)
+    if not q.one_kernel:
+        # a plain copy of the same number of bytes beside every stage short enough for its size to matter
+        ab = algorithmic_bytes(w)
+        res["copy_same_bytes_ms"] = {s: time_plain_copy(ab[s]) for s in res["stages_ms"] if ab[s] <= COPY_CONTEXT_MAX_BYTES}
+        time.sleep(BURST_IDLE_S)
     res["encode_other_ms"] = time_encode_other_mode(q, g_dev, w, min(steps, 10))
     res["update_ms"] = time_fused_update(q, w, min(steps, 10))
     if q.multi:
@@ -553,6 +585,11 @@ def summarize(res, peak_gbs):
         out["kernels"][s] = {"ms": round(ms, 5), "algorithmic_MB": round(ab[s] / 1e6, 2),
                              "GBps": round(gbs, 1), "frac_of_hbm_peak": round(gbs / peak_gbs, 4),
                              "frac_of_nominal_8TBps": round(gbs / NOMINAL_HBM_GBS, 4)}
+        if s in res.get("copy_same_bytes_ms", {}):
+            cms = res["copy_same_bytes_ms"][s]
+            out["kernels"][s]["plain_copy_of_the_same_bytes"] = {
+                "ms": round(cms, 5), "frac_of_hbm_peak": round(ab[s] / cms / 1e6 / peak_gbs, 4),
+                "note": "torch copy_ moving as many bytes as this stage (half read, half written), timed the same way"}
         if s in res.get("stages_sustained_ms", {}):
             ms_s = res["stages_sustained_ms"][s]
             out["kernels"][s]["ms_sustained"] = round(ms_s, 5)
