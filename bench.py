@@ -894,7 +894,10 @@ def gpu_main(args):
         # the workers of the same workload spread over the processes, with real exchanges (every rank takes part)
         del res, q
         torch.cuda.empty_cache()
-        line["distributed"] = bench_distributed(w, args.steps, args.warmup, "cuda", threads)
+        try:
+            line["distributed"] = bench_distributed(w, args.steps, args.warmup, "cuda", threads)
+        except Exception as e:           # the replicas figure above stands by itself
+            line["distributed"] = {"error": f"{type(e).__name__}: {e}"[:300]}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
