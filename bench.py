@@ -257,28 +257,26 @@ def time_alone(fn, reps, sustained=False, ms_hint=1.0, lead_s=0.6, span_s=0.4):
 COPY_CONTEXT_MAX_BYTES = 700e6
 
 
-def time_plain_copy(nbytes, reps=15):
-    """Median ms of a plain device copy that moves nbytes in all (nbytes / 2 read, nbytes / 2
-    written; torch's copy_), timed like a stage (events around single calls, warm L2).  Context for
-    the short stages: the copy that defines the HBM peak moves gigabytes, and a copy of a few hundred
-    megabytes does not get near that rate."""
+def time_plain_copy(nbytes, reps=20):
+    """Mean ms of a plain device copy that moves nbytes in all (nbytes / 2 read, nbytes / 2
+    written; torch's copy_), reps copies back to back between two events (so that no launch latency
+    is counted), warm L2.  Context for the short stages: the copy that defines the HBM peak moves
+    gigabytes, and a copy of a few hundred megabytes does not get near that rate."""
     import torch
     n = max(16, int(nbytes) // 2)
     a = torch.empty(n, dtype=torch.uint8, device="cuda").fill_(1)
     b = torch.empty_like(a)
     for _ in range(3):
         b.copy_(a)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
-    ts = []
+    e0.record()
     for _ in range(reps):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
         b.copy_(a)
-        e1.record()
-        torch.cuda.synchronize()
-        ts.append(e0.elapsed_time(e1))
+    e1.record()
+    torch.cuda.synchronize()
     del a, b
-    return statistics.median(ts)
+    return e0.elapsed_time(e1) / reps
 
 
 def time_end_to_end(q, g_host, out_host, g_dev, w, steps, warmup, barrier):
@@ -589,7 +587,7 @@ def summarize(res, peak_gbs):
             cms = res["copy_same_bytes_ms"][s]
             out["kernels"][s]["plain_copy_of_the_same_bytes"] = {
                 "ms": round(cms, 5), "frac_of_hbm_peak": round(ab[s] / cms / 1e6 / peak_gbs, 4),
-                "note": "torch copy_ moving as many bytes as this stage (half read, half written), timed the same way"}
+                "note": "torch copy_ moving as many bytes as this stage (half read, half written), copies back to back"}
         if s in res.get("stages_sustained_ms", {}):
             ms_s = res["stages_sustained_ms"][s]
             out["kernels"][s]["ms_sustained"] = round(ms_s, 5)
