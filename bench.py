@@ -254,7 +254,7 @@ def time_alone(fn, reps, sustained=False, ms_hint=1.0, lead_s=0.6, span_s=0.4):
     return e0.elapsed_time(e1) / reps
 
 
-COPY_CONTEXT_MAX_BYTES = 700e6
+COPY_CONTEXT_MAX_BYTES = 1300e6
 
 
 def time_plain_copy(nbytes, reps=20):
