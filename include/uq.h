@@ -226,9 +226,11 @@ int uq_encode_multi(const uq_layout *layout, const void *g, const float *W, cons
  * the shared indices, and quantizes the workers' rows from the same copy, so the gradients cross
  * the memory interface once instead of twice.  With more workers the two kernels run one after
  * the other.  idx and lev receive, bit for bit, what the two separate calls write; arguments and
- * errors are theirs.  On a B200 it takes about 15 % less time than the two calls (the gradients
- * are read from memory once), but it is bound by instruction issue rather than by memory, so
- * uq_step keeps the two streaming kernels and this call is the caller's choice.
+ * errors are theirs.  On a B200, with bf16 gradients and 16-bit draws, it takes about 15 % less
+ * time than the two calls (the gradients are read from memory once); with 32-bit draws, whose
+ * encoder is bound by its arithmetic either way, it takes the same time.  It is bound by
+ * instruction issue rather than by memory, so uq_step keeps the two streaming kernels and this
+ * call is the caller's choice.
  */
 int uq_select_encode_multi(const uq_layout *layout, const void *g, const float *W, const int32_t *scales,
                            int N, int idx_bits, uint64_t seed, int rng_bits, int fmt, uint8_t *idx,
