@@ -219,6 +219,22 @@ int uq_encode_multi(const uq_layout *layout, const void *g, const float *W, cons
                     void *lev, uint32_t *status, void *stream);
 
 /*
+ * uq_encode_single (scales = NULL) or uq_encode_multi (scales given) followed by
+ * uq_decode(src = UQ_SRC_LEVELS) as one call — Algorithm 1 lines "Quantize gradient", "AllReduce
+ * gradients", "Reconstruct gradient" (Algorithm 2: "Quantize with s*" onwards) — for callers whose
+ * M workers are all in this buffer.  With int8 levels and M <= 8 it is one kernel: the CTA that
+ * takes a tile of coordinates through the workers adds their levels up in registers and writes the
+ * reconstructed average beside the level rows, so the levels are written (they are what would cross
+ * the wire) but never read back.  With other formats or more workers the two kernels run one after
+ * the other.  lev and out receive, bit for bit, what the two separate calls write; arguments and
+ * errors are theirs (the integer sums are not available here: use uq_decode or uq_aggregate).
+ * uq_step makes this call when it is given no S_opt.
+ */
+int uq_encode_decode(const uq_layout *layout, const void *g, const float *W, int s, const int32_t *scales,
+                     int N, const uint8_t *idx, int idx_bits, uint64_t seed, int rng_bits, int fmt,
+                     void *lev, float *out, uint32_t *status, void *stream);
+
+/*
  * uq_select_scale_multi followed by uq_encode_multi as one call — Algorithm 2 lines "Compute
  * coordinate scales", "Scale sharing" and "Quantize with s*" — for callers whose M workers are all
  * in this buffer.  With M <= 8 it is one kernel: a CTA copies a tile of every worker's row into
@@ -317,9 +333,10 @@ int uq_index_min(const uint8_t *rows, int R, int64_t row_bytes, int64_t nbytes, 
  * One whole step in one call — Algorithm 1 lines "MaxAllReduce Norm" to "Reconstruct gradient"
  * (scales = NULL: uq_agree_scale, uq_encode_single, uq_decode) or Algorithm 2 (scales given:
  * uq_agree_scale, uq_select_scale_multi, uq_encode_multi, uq_decode), enqueued in that order on
- * `stream`.  Nothing is computed differently: this saves the caller three trips through the
- * binding when a step is so small that launch overhead counts.  Arguments are those of the calls
- * it makes (idx is not used when scales = NULL); the first error stops the sequence and is returned.
+ * `stream`; without S_opt the last two are made as one call, uq_encode_decode.  Nothing is
+ * computed differently: every output is bit for bit that of the separate calls.  Arguments are
+ * those of the calls it makes (idx is not used when scales = NULL); the first error stops the
+ * sequence and is returned.
  */
 int uq_step(const uq_layout *layout, const void *g, int norm, int s, const int32_t *scales, int N,
             int idx_bits, uint64_t seed, int rng_bits, int fmt, float *W, uint8_t *idx, void *lev,

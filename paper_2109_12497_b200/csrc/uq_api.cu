@@ -20,6 +20,10 @@ cudaError_t launch_aggregate_decode_rows(const uq_layout &L, const void *const *
                                          int32_t *S, cudaStream_t st);
 cudaError_t launch_decode_sums(const uq_layout &L, const int32_t *S, const float *W, const ScaleSet &scales,
                                const uint8_t *idx, int idx_bits, float *out, cudaStream_t st);
+bool encode_decode_fused(const uq_layout &L, int fmt);
+cudaError_t launch_encode_decode(const uq_layout &L, const void *g, const float *W, const ScaleSet &scales,
+                                 const uint8_t *idx, int idx_bits, uint64_t seed, int rng_bits, void *lev, float *out,
+                                 uint32_t *status, cudaStream_t st);
 cudaError_t launch_select_encode(const uq_layout &L, const void *g, const float *W, const ScaleSet &scales, int idx_bits,
                                  uint64_t seed, int rng_bits, int fmt, uint8_t *idx, void *lev, uint32_t *status,
                                  cudaStream_t st);
@@ -241,6 +245,34 @@ int uq_decode(const uq_layout *L, const void *src, int src_kind, int fmt, const 
                                               (cudaStream_t)stream));
 }
 
+int uq_encode_decode(const uq_layout *L, const void *g, const float *W, int s, const int32_t *scales, int N,
+                     const uint8_t *idx, int idx_bits, uint64_t seed, int rng_bits, int fmt, void *lev, float *out,
+                     uint32_t *status, void *stream)
+{
+    uq::ScaleSet set;
+    if (!layout_ok(L) || W == nullptr || !aligned(status, 4)) return UQ_ERR_BAD_ARG;
+    if (scales != nullptr) {
+        if (!scales_ok(scales, N, idx_bits, &set)) return UQ_ERR_BAD_ARG;
+        if (L->d > 0 && (idx == nullptr || !aligned(idx, 16))) return UQ_ERR_BAD_ARG;
+    } else {
+        if (s < 1) return UQ_ERR_BAD_ARG;
+        set = single_scale(s);
+        idx_bits = 0;
+        idx = nullptr;
+    }
+    if (!fmt_ok(fmt, set.s[0]) || (rng_bits != 32 && rng_bits != 16)) return UQ_ERR_BAD_ARG;
+    if (L->d > 0 && (g == nullptr || lev == nullptr || out == nullptr || !aligned(g, 16) || !aligned(lev, 16) ||
+                     !aligned(out, 32)))
+        return UQ_ERR_BAD_ARG;
+    if (uq::encode_decode_fused(*L, fmt))
+        return finish(uq::launch_encode_decode(*L, g, W, set, idx, idx_bits, seed, rng_bits, lev, out, status,
+                                               (cudaStream_t)stream));
+    const cudaError_t e = uq::launch_encode(*L, g, W, set, idx, idx_bits, seed, rng_bits, fmt, lev, status,
+                                            (cudaStream_t)stream);
+    if (e != cudaSuccess) return finish(e);
+    return finish(uq::launch_aggregate_decode(*L, lev, fmt, W, set, idx, idx_bits, out, nullptr, (cudaStream_t)stream));
+}
+
 int uq_decode_rows(const uq_layout *L, const void *const *lev_rows, int fmt, const float *W, int s,
                    const int32_t *scales, int N, const uint8_t *idx, int idx_bits, float *out, int32_t *S_opt,
                    void *stream)
@@ -297,10 +329,13 @@ int uq_step(const uq_layout *L, const void *g, int norm, int s, const int32_t *s
     if (scales != nullptr) {
         rc = uq_select_scale_multi(L, g, W, scales, N, idx_bits, idx, status, stream);
         if (rc != UQ_OK) return rc;
-        rc = uq_encode_multi(L, g, W, scales, N, idx, idx_bits, seed, rng_bits, fmt, lev, status, stream);
-    } else {
-        rc = uq_encode_single(L, g, W, s, seed, rng_bits, fmt, lev, status, stream);
     }
+    if (S_opt == nullptr)       // nobody wants the integer sums: the encoder may add up and reconstruct itself
+        return uq_encode_decode(L, g, W, s, scales, N, idx, idx_bits, seed, rng_bits, fmt, lev, out, status, stream);
+    if (scales != nullptr)
+        rc = uq_encode_multi(L, g, W, scales, N, idx, idx_bits, seed, rng_bits, fmt, lev, status, stream);
+    else
+        rc = uq_encode_single(L, g, W, s, seed, rng_bits, fmt, lev, status, stream);
     if (rc != UQ_OK) return rc;
     return uq_decode(L, lev, UQ_SRC_LEVELS, fmt, W, s, scales, N, idx, idx_bits, out, S_opt, stream);
 }

@@ -43,12 +43,6 @@ __device__ __forceinline__ void sgd_coordinate(float g_hat, float &theta, float 
     theta = __fsub_rn(theta, __fmul_rn(lr, u));
 }
 
-// W / ((float)s * (float)M): product, then one IEEE division.
-__device__ __forceinline__ float decode_factor(float W, int32_t s, int M)
-{
-    return __fdiv_rn(W, __fmul_rn((float)s, (float)M));
-}
-
 template <int IDXB> __device__ __forceinline__ int index_at(const uint8_t *idx, int64_t i)
 {
     if (IDXB == 8) return idx[i];

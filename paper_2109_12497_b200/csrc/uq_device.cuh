@@ -535,6 +535,12 @@ __device__ __forceinline__ int warp_find_segment(const int64_t *__restrict__ seg
     return lo;
 }
 
+// Reconstruction factor W / ((float)s * (float)M): product, then one IEEE division (W = 0 gives 0).
+__device__ __forceinline__ float decode_factor(float W, int32_t s, int M)
+{
+    return __fdiv_rn(W, __fmul_rn((float)s, (float)M));
+}
+
 // ---------------------------------------------------------------------------------------------
 // scale selection: the test |v| * inv <= s_hat as an integer compare
 // ---------------------------------------------------------------------------------------------

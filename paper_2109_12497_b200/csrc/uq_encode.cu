@@ -9,9 +9,10 @@ cudaError_t launch_select(const uq_layout &L, const void *g, const float *W, con
 
 static cudaError_t launch_encode_any(const uq_layout &L, const void *g, const float *W, const ScaleSet &scales,
                                      uint8_t *idx, int idx_bits, bool select, uint64_t seed, int rng_bits, int fmt,
-                                     void *lev, uint32_t *status, cudaStream_t st)
+                                     void *lev, uint32_t *status, cudaStream_t st, float *out = nullptr)
 {
     EncodeParams p;
+    p.out = out;
     p.v.g = g; p.v.W = W; p.v.seg_off = L.seg_off; p.v.d = L.d; p.v.stride = L.worker_stride; p.v.nseg = L.nseg; p.v.M = L.M;
     p.v.s_hat = (float)scales.s[0];
     p.v.scales = scales;
@@ -32,6 +33,18 @@ cudaError_t launch_encode(const uq_layout &L, const void *g, const float *W, con
                           uint32_t *status, cudaStream_t st)
 {
     return launch_encode_any(L, g, W, scales, const_cast<uint8_t *>(idx), idx_bits, false, seed, rng_bits, fmt, lev, status, st);
+}
+
+// Quantization, sum over the workers and reconstruction in one kernel (decode mode of the encoder):
+// int8 levels and at most kWorkerGroup workers, so that the CTA of a tile sees every worker's levels.
+bool encode_decode_fused(const uq_layout &L, int fmt) { return fmt == UQ_FMT_I8 && L.M <= kWorkerGroup; }
+
+cudaError_t launch_encode_decode(const uq_layout &L, const void *g, const float *W, const ScaleSet &scales,
+                                 const uint8_t *idx, int idx_bits, uint64_t seed, int rng_bits, void *lev, float *out,
+                                 uint32_t *status, cudaStream_t st)
+{
+    return launch_encode_any(L, g, W, scales, const_cast<uint8_t *>(idx), idx_bits, false, seed, rng_bits, UQ_FMT_I8, lev, status,
+                             st, out);
 }
 
 // Scale selection, scale sharing and quantization in one kernel: a CTA that takes a tile through

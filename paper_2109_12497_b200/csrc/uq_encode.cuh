@@ -11,6 +11,11 @@
 // indices (one index load and eight shuffles per unit), and the first two rounds of the Philox
 // block, whose counter differs between workers only in one word.  The work done for worker m
 // reads only g^m plus the agreed values W and idx.
+//
+// Decode mode (int8 levels, M <= 8, so that one CTA sees every worker of its tile): the CTA also adds
+// the workers' levels up as it goes and writes the reconstructed average (Algorithm 1 / 2, lines
+// "AllReduce gradients" and "Reconstruct gradient") beside the level rows, which then need not be
+// read back by the aggregation kernel.  Bit for bit what uq_decode makes of the same levels.
 #pragma once
 #include "uq_device.cuh"
 #include "uq_select.cuh"
@@ -22,6 +27,7 @@ struct EncodeParams {
     SelectView v;             // g, W, seg_off, d, stride, nseg, M, scales (single-scale: every entry is s) and
                               // s_hat = (float) of the smallest scale: the largest level
     void *lev;
+    float *out;               // decode mode: the reconstructed average [d]; else unused
     uint8_t *idx;             // shared scale indices: read, or (select) written by this launch
     uint32_t *status;
     int32_t select;           // multi-scale: 1 = find the shared indices here instead of reading them
@@ -42,6 +48,9 @@ constexpr int kWorkerGroup = 8;   // workers that one CTA takes through a tile
 template <int DT, int RNG> struct EncodeShape {
     static constexpr int UNITS = DT == UQ_BF16 ? 2 : 1;                       // 32 B per thread and worker in flight
     static constexpr int MIN_CTAS = (DT == UQ_BF16 && RNG == 32) ? 3 : 4;
+    // decode mode holds the level sums too: at 64 registers the bf16 kernel spills and the fp32 one with
+    // 32-bit draws is slower than at 80
+    static constexpr int MIN_CTAS_DEC = (DT == UQ_F32 && RNG == 16) ? 4 : 3;
     static constexpr int TILE = kThreads * UNITS * 8;
 };
 
@@ -199,6 +208,53 @@ __device__ __noinline__ void encode_tile_mixed(const EncodeParams &p, int m0, in
     if (overflow && lane < p.v.scales.N && p.status) atomicOr(p.status, (uint32_t)UQ_STATUS_SCALE_OVERFLOW);
 }
 
+// Decode mode, slow forms: sum and reconstruction of the unit of 8 coordinates at i from the int8
+// levels that THIS thread stored for every worker just before (own stores are visible to own loads;
+// read around L1), with the segment and the shared index looked up per coordinate.
+template <int IDXB>
+__device__ __noinline__ void decode_unit_general(const EncodeParams &p, int64_t i, uint64_t kbits_own, bool own_idx)
+{
+    constexpr bool MULTI = IDXB != 0;
+    constexpr int IB = MULTI ? IDXB : 8;
+    if (i >= p.v.d) return;
+    int S[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    const char *lp = (const char *)p.lev + i;
+    for (int m = 0; m < p.v.M; ++m) {
+        const uint2 b = __ldcg((const uint2 *)(lp + (size_t)m * (size_t)p.v.stride));
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            S[e] += (int)(int8_t)(b.x >> (8 * e));
+            S[4 + e] += (int)(int8_t)(b.y >> (8 * e));
+        }
+    }
+    uint64_t kbits = kbits_own;
+    if (MULTI && !own_idx) kbits = (uint64_t)IdxBits<IB>::load(p.idx + i * IB / 8);
+    int j = find_segment(p.v.seg_off, p.v.nseg, i);
+    for (int e = 0; e < 8 && i + e < p.v.d; ++e) {
+        j = advance_segment(p.v.seg_off, p.v.nseg, j, i + e);
+        const int k = MULTI ? (int)((kbits >> (e * IB)) & ((1u << IB) - 1u)) : 0;
+        p.out[i + e] = __fmul_rn((float)S[e], decode_factor(__ldg(p.v.W + j), p.v.scales.s[k & (UQ_MAX_SCALES - 1)], p.v.M));
+    }
+}
+
+// The units of tile [t0, t1) that this thread encoded in a slow form (the same assignment of units to
+// threads as encode_span_general and encode_tile_mixed).  mixed: a row that itself contains a
+// boundary was skipped there and is skipped here (a CTA of the second kind owns it).
+template <int DT, int RNG, int IDXB>
+__device__ __noinline__ void decode_tile_slow(const EncodeParams &p, int64_t t0, int64_t t1, bool mixed)
+{
+    for (int u = 0; u < EncodeShape<DT, RNG>::UNITS; ++u) {
+        const int64_t r0 = t0 + (int64_t)(u * kThreads + (threadIdx.x & ~31)) * 8;
+        if (r0 >= t1) break;                                         // warp-uniform
+        if (mixed) {
+            const int jr = warp_find_segment(p.v.seg_off, p.v.nseg, r0);
+            if (segment_end(p.v.seg_off, p.v.nseg, jr, p.v.d) < r0 + 256) continue;
+        }
+        const int64_t i = r0 + (threadIdx.x & 31) * 8;
+        if (i < t1) decode_unit_general<IDXB>(p, i, 0, false);
+    }
+}
+
 // The slow forms of a whole tile, workers m0 .. m1 - 1: the ragged last tile, a tile whose Philox block
 // numbers leave the launch's high word, or 16-bit draws with a factor too small for the saturating
 // form (j < 0: per-coordinate lookup), and a full tile crossed by segment boundaries (j = its first
@@ -229,7 +285,7 @@ __device__ __noinline__ void encode_tile_slow(const EncodeParams &p, int64_t t0,
 }
 
 // State of a tile that does not depend on the worker.
-template <int DT, int FMT, int RNG, int IDXB> struct TileState {
+template <int DT, int FMT, int RNG, int IDXB, bool DEC = false> struct TileState {
     using E = Elem<DT>;
     using S = EncodeShape<DT, RNG>;
     static constexpr int U = S::UNITS;
@@ -239,17 +295,19 @@ template <int DT, int FMT, int RNG, int IDXB> struct TileState {
     PhiloxBlockPart blk[U * BPU];     // worker-independent rounds of the units' Philox blocks
     SatConstants sc;                  // 16-bit draws
     float cap23;                      // 32-bit draws: the largest level * 2^23
+    uint32_t sum[DEC ? U : 1][4];     // decode mode: the unit's level sums, every level biased by 128, in 16-bit
+                                      // lanes: bytes 0, 2 and bytes 1, 3 of the low word, then of the high word
     const char *gp;                   // my first coordinate in the gradient row that is loaded next
     const uint4 *sp;                  // select mode: my slot of that row's copy in shared memory
     char *lp, *lp2;                   // and in the level row that is stored next (second plane for 6-bit)
     size_t grow, lrow;                // bytes between rows
 };
 
-template <bool SEL, int DT, int FMT, int RNG, int IDXB>
-__device__ __forceinline__ void load_units(TileState<DT, FMT, RNG, IDXB> &t,
+template <bool SEL, int DT, int FMT, int RNG, int IDXB, bool DEC>
+__device__ __forceinline__ void load_units(TileState<DT, FMT, RNG, IDXB, DEC> &t,
                                            uint4 (&q)[EncodeShape<DT, RNG>::UNITS][8 / Elem<DT>::G])
 {
-    using T = TileState<DT, FMT, RNG, IDXB>;
+    using T = TileState<DT, FMT, RNG, IDXB, DEC>;
 #pragma unroll
     for (int u = 0; u < T::U; ++u)
 #pragma unroll
@@ -262,11 +320,11 @@ __device__ __forceinline__ void load_units(TileState<DT, FMT, RNG, IDXB> &t,
 // Workers m0 .. m0 + G - 1 of the tile, straight-line.  On entry q holds worker m0's units (loaded
 // or in flight); while worker m is quantized the units of worker m + 1 are on their way (MORE: also
 // those of the worker after the last one of this call).
-template <int G, bool MORE, bool SEL, int DT, int FMT, int RNG, int IDXB>
-__device__ __forceinline__ void encode_workers(const EncodeParams &p, TileState<DT, FMT, RNG, IDXB> &t, int m0,
+template <int G, bool MORE, bool SEL, int DT, int FMT, int RNG, int IDXB, bool DEC>
+__device__ __forceinline__ void encode_workers(const EncodeParams &p, TileState<DT, FMT, RNG, IDXB, DEC> &t, int m0,
                                                uint4 (&q)[EncodeShape<DT, RNG>::UNITS][8 / Elem<DT>::G])
 {
-    using T = TileState<DT, FMT, RNG, IDXB>;
+    using T = TileState<DT, FMT, RNG, IDXB, DEC>;
     using LF = LevelFmt<FMT>;
     constexpr int UB = LF::UB;                                   // bytes of levels per unit: 8, 4 or 2
     constexpr int UB2 = FMT == UQ_FMT_I6P ? 2 : 0;               // and in the second plane of the 6-bit format
@@ -274,7 +332,7 @@ __device__ __forceinline__ void encode_workers(const EncodeParams &p, TileState<
     for (int k = 0; k < G; ++k) {
         const int m = m0 + k;
         uint4 qn[T::U][T::H];
-        if (k + 1 < G || MORE) load_units<SEL, DT, FMT, RNG, IDXB>(t, qn);
+        if (k + 1 < G || MORE) load_units<SEL>(t, qn);
         uint4 r[T::U * T::BPU];
         philox_join<T::U * T::BPU>(p.key, t.blk, p.wpart[m], r);
 #pragma unroll
@@ -295,6 +353,13 @@ __device__ __forceinline__ void encode_workers(const EncodeParams &p, TileState<
             }
             if (EO) store_unit_even_odd(lo, hi, t.lp + u * kThreads * UB);
             else store_unit<FMT>(lo, hi, t.lp + u * kThreads * UB, t.lp2 + u * kThreads * UB2);
+            if (DEC) {
+                // the sum over the workers: the bytes biased to 1 .. 255, bytes 0, 2 and bytes 1, 3 of a
+                // word spread over the 16-bit lanes of a word each (8 * 255 fits a lane)
+                const uint32_t bl = lo ^ 0x80808080u, bh = hi ^ 0x80808080u;
+                t.sum[u][0] += __byte_perm(bl, 0u, 0x4240); t.sum[u][1] += __byte_perm(bl, 0u, 0x4341);
+                t.sum[u][2] += __byte_perm(bh, 0u, 0x4240); t.sum[u][3] += __byte_perm(bh, 0u, 0x4341);
+            }
         }
         t.lp += t.lrow;
         if (FMT == UQ_FMT_I6P) t.lp2 += t.lrow;
@@ -380,11 +445,14 @@ __device__ __forceinline__ void staged_max_magnitude(const uint4 *stage, int u, 
 // SEL: the kernel also finds and stores the shared scale indices (multi-scale, all M <= kWorkerGroup
 // workers in one CTA): the tile's rows are copied to shared memory once (every thread its own
 // units, so no barrier), read there for the maximum over the workers and again for quantization.
-template <int DT, int FMT, int RNG, int IDXB, bool SEL>
-__global__ void __launch_bounds__(kThreads, (SEL ? 3 : EncodeShape<DT, RNG>::MIN_CTAS)) encode_kernel(const __grid_constant__ EncodeParams p)
+// DEC: decode mode (see the head of this file; int8 levels, one CTA per tile, not together with SEL).
+template <int DT, int FMT, int RNG, int IDXB, bool SEL, bool DEC>
+__global__ void __launch_bounds__(kThreads, (SEL ? 3 : DEC ? EncodeShape<DT, RNG>::MIN_CTAS_DEC : EncodeShape<DT, RNG>::MIN_CTAS))
+encode_kernel(const __grid_constant__ EncodeParams p)
 {
+    static_assert(!DEC || (FMT == UQ_FMT_I8 && !SEL), "decode mode: int8 levels, indices given");
     grid_dependency_prologue();
-    using T = TileState<DT, FMT, RNG, IDXB>;
+    using T = TileState<DT, FMT, RNG, IDXB, DEC>;
     using E = Elem<DT>;
     using S = EncodeShape<DT, RNG>;
     using LF = LevelFmt<FMT>;
@@ -398,15 +466,21 @@ __global__ void __launch_bounds__(kThreads, (SEL ? 3 : EncodeShape<DT, RNG>::MIN
         // boundary lies strictly inside a 256-coordinate row of a full tile, quantizes that row with
         // per-coordinate scales (the tile's own CTA skips it).  Keeping these rows out of the tile
         // CTAs keeps their lifetime short: the slow path no longer holds a whole CTA slot.
+        // (decode mode: one warp takes the row of every worker, one after the other, and then decodes it)
         const uint32_t x = blockIdx.x - p.main_blocks;
-        const int m = (int)(x % (uint32_t)p.v.M);
-        const int64_t k = 1 + (int64_t)(x / (uint32_t)p.v.M) * kWarps + (tid >> 5);
+        const int m = DEC ? 0 : (int)(x % (uint32_t)p.v.M);
+        const int64_t k = 1 + (int64_t)(DEC ? x : x / (uint32_t)p.v.M) * kWarps + (tid >> 5);
         if (k >= p.v.nseg) return;
         const int64_t b = __ldg(p.v.seg_off + k), prev = __ldg(p.v.seg_off + k - 1);
         const int64_t r0 = b & ~(int64_t)255;
         const int64_t full_end = p.v.d / S::TILE * S::TILE;          // rows beyond belong to the ragged tile's CTA
         if (b <= 0 || b == r0 || r0 >= full_end) return;           // not strictly inside a row of a full tile
         if (prev > r0 && prev <= b) return;                        // an earlier boundary in the same row takes it
+        if (DEC) {
+            for (int mm = 0; mm < p.v.M; ++mm) encode_span_general<DT, FMT, RNG, IDXB>(p, mm, r0, r0 + 256, lane, 32);
+            decode_unit_general<IDXB>(p, r0 + lane * 8, 0, false);
+            return;
+        }
         encode_span_general<DT, FMT, RNG, IDXB>(p, m, r0, r0 + 256, lane, 32, MULTI && p.select,
                                                 sh_thr + (MULTI ? (tid >> 5) * 2 * UQ_MAX_SCALES : 0));
         return;
@@ -428,6 +502,7 @@ __global__ void __launch_bounds__(kThreads, (SEL ? 3 : EncodeShape<DT, RNG>::MIN
     const bool other_hi = (uint32_t)blk0 > 0xFFFFFFFFu - (uint32_t)(S::TILE >> BSH) || (uint32_t)(blk0 >> 32) != p.blk_hi;
     if (t1 - t0 != S::TILE || other_hi) {
         encode_tile_slow<DT, FMT, RNG, IDXB>(p, t0, t1, -1, m0, m0 + cnt, sh_thr);
+        if (DEC) decode_tile_slow<DT, RNG, IDXB>(p, t0, t1, false);
         return;
     }
     // every warp looks the segment up for itself (no shared memory, no barrier)
@@ -436,6 +511,7 @@ __global__ void __launch_bounds__(kThreads, (SEL ? 3 : EncodeShape<DT, RNG>::MIN
         // A segment boundary crosses the tile (at most nseg - 1 tiles): a compact loop over the
         // rows of every worker, kept out of line so that its registers do not weigh on the path below.
         encode_tile_slow<DT, FMT, RNG, IDXB>(p, t0, t1, j, m0, m0 + cnt, sh_thr);
+        if (DEC) decode_tile_slow<DT, RNG, IDXB>(p, t0, t1, true);
         return;
     }
     T t;
@@ -451,7 +527,7 @@ __global__ void __launch_bounds__(kThreads, (SEL ? 3 : EncodeShape<DT, RNG>::MIN
         else stage_rows<0, DT, RNG>(stage, t.gp, t.grow, cnt);
     } else {
         // the first worker's row and the shared indices are on their way during the set-up below
-        load_units<false, DT, FMT, RNG, IDXB>(t, q);
+        load_units<false>(t, q);
         if (MULTI) {
             const uint8_t *ip = p.idx + ((size_t)t0 + (size_t)tid * 8) * IB / 8;
 #pragma unroll
@@ -469,6 +545,7 @@ __global__ void __launch_bounds__(kThreads, (SEL ? 3 : EncodeShape<DT, RNG>::MIN
                   : !fixed_form_exact(inv_scale(p.v.scales.s[p.v.scales.N - 1], W))) {
         if (SEL) copy_async_wait();
         encode_tile_slow<DT, FMT, RNG, IDXB>(p, t0, t1, -1, m0, m0 + cnt, sh_thr);
+        if (DEC) decode_tile_slow<DT, RNG, IDXB>(p, t0, t1, false);
         return;
     }
     if (SEL) {
@@ -500,7 +577,7 @@ __global__ void __launch_bounds__(kThreads, (SEL ? 3 : EncodeShape<DT, RNG>::MIN
             kbits[u] = packed;
             store_unit_indices<IB>(p.idx, t0 + (int64_t)(u * kThreads + tid) * 8, packed);
         }
-        load_units<true, DT, FMT, RNG, IDXB>(t, q);
+        load_units<true>(t, q);
     }
     if (RNG == 16) {
         inv_lane = __fmul_rn(inv_lane, 0.00390625f);
@@ -525,27 +602,55 @@ __global__ void __launch_bounds__(kThreads, (SEL ? 3 : EncodeShape<DT, RNG>::MIN
     t.lp = lrow0 + LF::off(t0) + tid * LF::UB;
     t.lp2 = lrow0 + LF::off2(t0, p.v.stride) + tid * (FMT == UQ_FMT_I6P ? 2 : 0);
 
+    // decode mode: lane k holds the reconstruction factor of scale k, the sums start at zero
+    float c_lane = 0.0f;
+    if (DEC) {
+        c_lane = decode_factor(W, p.v.scales.s[lane & KMASK], p.v.M);
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) t.sum[u][k] = 0u;
+    }
+
     // The workers of the group straight-line, with no loop around them: all 8, or (the last group
     // of a job whose M is not a multiple of 8) 4, 2 and 1 of them as the count's bits say.
     if (cnt == kWorkerGroup) {
-        encode_workers<kWorkerGroup, false, SEL, DT, FMT, RNG, IDXB>(p, t, m0, q);
-        return;
+        encode_workers<kWorkerGroup, false, SEL>(p, t, m0, q);
+    } else {
+        int m = m0;
+        if (cnt & 4) {
+            if (cnt & 3) encode_workers<4, true, SEL>(p, t, m, q);
+            else encode_workers<4, false, SEL>(p, t, m, q);
+            m += 4;
+        }
+        if (cnt & 2) {
+            if (cnt & 1) encode_workers<2, true, SEL>(p, t, m, q);
+            else encode_workers<2, false, SEL>(p, t, m, q);
+            m += 2;
+        }
+        if (cnt & 1) encode_workers<1, false, SEL>(p, t, m, q);
     }
-    int m = m0;
-    if (cnt & 4) {
-        if (cnt & 3) encode_workers<4, true, SEL, DT, FMT, RNG, IDXB>(p, t, m, q);
-        else encode_workers<4, false, SEL, DT, FMT, RNG, IDXB>(p, t, m, q);
-        m += 4;
+    if (DEC) {
+        // Algorithm 1 / 2, lines "AllReduce gradients" and "Reconstruct gradient" for the tile: the sum
+        // of a coordinate leaves its lane, loses the bias, and is multiplied by the factor of the
+        // coordinate's scale (the same three operations as the aggregation kernel's)
+        const int bias = 128 * p.v.M;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            uint32_t r[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const uint32_t lanes = t.sum[DEC ? u : 0][(e >> 2) * 2 + (e & 1)];
+                const int sum = (int)((lanes >> (16 * ((e & 3) >> 1))) & 0xFFFFu) - bias;
+                const float c = MULTI ? __shfl_sync(0xFFFFFFFFu, c_lane, (int)(uint32_t)(kbits[u] >> (e * IB))) : c_lane;
+                r[e] = __float_as_uint(__fmul_rn((float)sum, c));
+            }
+            st_stream256(p.out + t0 + (int64_t)(u * kThreads + tid) * 8, r);
+        }
     }
-    if (cnt & 2) {
-        if (cnt & 1) encode_workers<2, true, SEL, DT, FMT, RNG, IDXB>(p, t, m, q);
-        else encode_workers<2, false, SEL, DT, FMT, RNG, IDXB>(p, t, m, q);
-        m += 2;
-    }
-    if (cnt & 1) encode_workers<1, false, SEL, DT, FMT, RNG, IDXB>(p, t, m, q);
 }
 
-template <int DT, int FMT, int RNG, int IDXB, bool SEL = false>
+template <int DT, int FMT, int RNG, int IDXB, bool SEL = false, bool DEC = false>
 static cudaError_t launch(EncodeParams p, cudaStream_t st)
 {
     using S = EncodeShape<DT, RNG>;
@@ -555,7 +660,7 @@ static cudaError_t launch(EncodeParams p, cudaStream_t st)
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     p.main_blocks = (uint32_t)blocks;
-    if (p.v.seg_off != nullptr && p.v.nseg > 1) blocks += (int64_t)((p.v.nseg - 1 + kWarps - 1) / kWarps) * p.v.M;
+    if (p.v.seg_off != nullptr && p.v.nseg > 1) blocks += (int64_t)((p.v.nseg - 1 + kWarps - 1) / kWarps) * (DEC ? 1 : p.v.M);
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     constexpr int BSH = RNG == 32 ? 2 : 3;
     p.blk_hi = (uint32_t)((uint64_t)(p.coord0 >> BSH) >> 32);
@@ -571,14 +676,14 @@ static cudaError_t launch(EncodeParams p, cudaStream_t st)
         cudaError_t e = cudaGetDevice(&dev);
         if (e != cudaSuccess) return e;
         if (dev < 0 || dev >= 64 || !opted_in[dev]) {
-            e = cudaFuncSetAttribute(encode_kernel<DT, FMT, RNG, IDXB, SEL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            e = cudaFuncSetAttribute(encode_kernel<DT, FMT, RNG, IDXB, SEL, DEC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      kWorkerGroup * S::TILE * Elem<DT>::BYTES);
             if (e != cudaSuccess) return e;
             if (dev >= 0 && dev < 64) opted_in[dev] = true;
         }
-        launch_k_smem(encode_kernel<DT, FMT, RNG, IDXB, SEL>, (unsigned)blocks, kThreads, smem, st, p);
+        launch_k_smem(encode_kernel<DT, FMT, RNG, IDXB, SEL, DEC>, (unsigned)blocks, kThreads, smem, st, p);
     } else {
-        launch_k(encode_kernel<DT, FMT, RNG, IDXB, SEL>, (unsigned)blocks, kThreads, st, p);
+        launch_k(encode_kernel<DT, FMT, RNG, IDXB, SEL, DEC>, (unsigned)blocks, kThreads, st, p);
     }
     return cudaGetLastError();
 }
@@ -586,6 +691,17 @@ static cudaError_t launch(EncodeParams p, cudaStream_t st)
 template <int DT, int FMT, int RNG>
 static cudaError_t dispatch_idx(const EncodeParams &p, int idx_bits, cudaStream_t st)
 {
+    if constexpr (FMT == UQ_FMT_I8) {
+        if (p.out != nullptr) {                       // decode mode (the caller has checked M <= kWorkerGroup, no select)
+            switch (idx_bits) {
+            case 0: return launch<DT, FMT, RNG, 0, false, true>(p, st);
+            case 1: return launch<DT, FMT, RNG, 1, false, true>(p, st);
+            case 2: return launch<DT, FMT, RNG, 2, false, true>(p, st);
+            case 4: return launch<DT, FMT, RNG, 4, false, true>(p, st);
+            default: return launch<DT, FMT, RNG, 8, false, true>(p, st);
+            }
+        }
+    }
     if (p.select) {
         switch (idx_bits) {
         case 1: return launch<DT, FMT, RNG, 1, true>(p, st);

@@ -92,6 +92,17 @@ class Quantizer:
         B.uq_decode(self.layout, self.lev, B.UQ_SRC_LEVELS, self.fmt, self.W, self.s, self.scales, self.idx,
                     self.idx_bits, self.out, self.S)
 
+    def encode_decode(self, g: torch.Tensor, seed: int) -> None:
+        """Quantization, integer aggregation and reconstruction as one call (what the step makes when
+        the integer sums are not kept; one kernel for int8 levels and M <= 8)."""
+        B.uq_encode_decode(self.layout, g, self.W, self.s, self.scales, self.idx, self.idx_bits, seed, self.rng_bits,
+                           self.fmt, self.lev, self.out, self.status)
+
+    @property
+    def fused_decode(self) -> bool:
+        """Whether the step's encoder also aggregates and reconstructs (uq_encode_decode as one kernel)."""
+        return self.S is None and self.fmt == B.UQ_FMT_I8 and self.layout.M <= B.SMALL_STEP_MAX_WORKERS
+
     def aggregate_decode_update(self, theta: torch.Tensor, momentum: Optional[torch.Tensor], lr: float,
                                 mu: float = 0.0, wd: float = 0.0) -> None:
         """Fused aggregation, reconstruction and SGD step on theta (Algorithm 1/2, last three lines)."""

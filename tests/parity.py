@@ -24,11 +24,16 @@ def run_gpu(w, g_np, seed=None, mode="default"):
     """All stage outputs of the CUDA path as numpy arrays.  mode picks the form of the path:
     "default" (what the library picks: the one-kernel step for small gradients, else uq_step),
     "fused" (multi-scale: selection and encoding as one call, uq_select_encode_multi), "one" (the
-    whole step as one cooperative kernel), "separate" (never the one-kernel step)."""
-    one_kernel = {"one": True, "separate": False, "fused": False}.get(mode)       # else: the library decides by size
-    q = from_workload(w, keep_sums=True, fused_select=mode == "fused", one_kernel=one_kernel)
+    whole step as one cooperative kernel), "separate" (never the one-kernel step), "nosums" (the step
+    without the integer sums among its outputs: quantization, aggregation and reconstruction as one
+    call, uq_encode_decode; the sums compared below then come from uq_aggregate over its levels)."""
+    one_kernel = {"one": True, "separate": False, "fused": False, "nosums": False}.get(mode)   # else: the library decides by size
+    q = from_workload(w, keep_sums=mode != "nosums", fused_select=mode == "fused", one_kernel=one_kernel)
     g = to_device(w, g_np)
     q.step(g, w.seed if seed is None else seed)
+    if mode == "nosums":
+        q.S = torch.empty(max(w.d, 1), dtype=torch.int32, device="cuda")
+        B.uq_aggregate(q.layout, q.lev, q.fmt, q.S)
     torch.cuda.synchronize()
     res = dict(
         W=q.W.cpu().numpy(), lev=q.lev.cpu().numpy().view(np.uint8), S=q.S.cpu().numpy()[: w.d],
@@ -82,9 +87,11 @@ def ulp_distance(a, b):
 def check_parity(w, g_np, seed=None):
     """Full comparison; returns the GPU result for further checks.  A multi-scale workload runs in
     both forms of its path (see run_gpu), a workload that the one-kernel step takes in both of
-    its forms: each must match the oracle."""
+    its forms, and every workload also without the integer sums among the outputs (the form in which
+    the encoder aggregates and reconstructs itself where it can): each must match the oracle."""
     if w.quantizer == "multi":
         _check_parity(w, g_np, seed, "fused")
+    _check_parity(w, g_np, seed, "nosums")
     if one_kernel_takes(w):
         _check_parity(w, g_np, seed, "one")
         _check_parity(w, g_np, seed, "separate")

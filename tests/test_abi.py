@@ -120,6 +120,12 @@ def test_later_entry_points_reject_bad_arguments_on_the_host(lib):
     assert lib.uq_select_encode_multi(ok, p, p, sc, 2, 3, 0, 16, B.UQ_FMT_I8, p, p, None, None) == B.UQ_ERR_BAD_ARG   # idx_bits
     assert lib.uq_select_encode_multi(ok, p, p, sc, 2, 2, 0, 16, B.UQ_FMT_I4X2, p, p, None, None) == B.UQ_ERR_BAD_ARG  # s_hat > 7
     assert lib.uq_select_encode_multi(ok, p, p, sc, 2, 2, 0, 16, B.UQ_FMT_I8, None, p, None, None) == B.UQ_ERR_BAD_ARG
+    # uq_encode_decode: the checks of the encoders and of uq_decode
+    assert lib.uq_encode_decode(ok, p, p, 127, None, 0, None, 0, 0, 24, B.UQ_FMT_I8, p, p, None, None) == B.UQ_ERR_BAD_ARG   # rng_bits
+    assert lib.uq_encode_decode(ok, p, p, 128, None, 0, None, 0, 0, 16, B.UQ_FMT_I8, p, p, None, None) == B.UQ_ERR_BAD_ARG   # s > 127
+    assert lib.uq_encode_decode(ok, p, p, 127, None, 0, None, 0, 0, 16, B.UQ_FMT_I8, p, None, None, None) == B.UQ_ERR_BAD_ARG  # out
+    assert lib.uq_encode_decode(ok, p, p, 127, sc, 2, None, 2, 0, 16, B.UQ_FMT_I8, p, p, None, None) == B.UQ_ERR_BAD_ARG     # idx
+    assert lib.uq_encode_decode(ok, p, p, 127, sc, 2, p, 3, 0, 16, B.UQ_FMT_I8, p, p, None, None) == B.UQ_ERR_BAD_ARG        # idx_bits
     assert lib.uq_index_min(p, 0, 64, 64, 2, p, None) == B.UQ_ERR_BAD_ARG                    # R
     assert lib.uq_index_min(p, 2, 64, 62, 2, p, None) == B.UQ_ERR_BAD_ARG                    # whole words
     assert lib.uq_index_min(p, 2, 32, 64, 2, p, None) == B.UQ_ERR_BAD_ARG                    # rows overlap
