@@ -74,6 +74,7 @@ def algorithmic_bytes(w: wl.Workload) -> dict:
     else:
         b["encode"] = (e + lev) * M * d
     b["aggregate_decode"] = lev * M * d + ib * d + 4 * d
+    b["encode_decode"] = b["encode"] + 4 * d          # one call: the levels are written but not read back
     return b
 
 
@@ -143,24 +144,29 @@ class ClockSampler:
 # GPU arm
 # ---------------------------------------------------------------------------------------------
 
-STAGES_SINGLE = ["agree_scale", "encode", "aggregate_decode"]
-STAGES_MULTI = ["agree_scale", "select_scale", "encode", "aggregate_decode"]      # the calls uq_step makes
+def encoder_decodes(w) -> bool:
+    """Whether the step's encoder also aggregates and reconstructs (uq_encode_decode as one kernel:
+    int8 levels, 16-bit draws, at most 8 workers; pipeline.Quantizer.fused_decode says the same of its object)."""
+    return w.fmt == "i8" and w.M <= 8 and w.rng_bits == 16
 
 
 def stages_of(w):
-    return STAGES_MULTI if w.quantizer == "multi" else STAGES_SINGLE
+    """The calls uq_step makes for this workload (without the integer sums among its outputs)."""
+    head = ["agree_scale", "select_scale"] if w.quantizer == "multi" else ["agree_scale"]
+    return head + (["encode_decode"] if encoder_decodes(w) else ["encode", "aggregate_decode"])
 
 
 def stage_calls(q, g):
     """{stage: function of the seed} for the separate calls of the step."""
     calls = {"agree_scale": lambda seed: q.agree_scale(g), "aggregate_decode": lambda seed: q.aggregate_decode()}
     calls["encode"] = lambda seed: q.encode(g, seed)
+    calls["encode_decode"] = lambda seed: q.encode_decode(g, seed)
     if q.multi:
         calls["select_scale"] = lambda seed: q.select_scale(g)
     return calls
 
 
-def run_stages(q, g, seed, events=None):
+def run_stages(q, g, seed, events=None, stages=None):
     """One step; events (if given) is a list of len(stages)+1 CUDA events recorded around the stages.
     Without events the step is the one call a user makes (Quantizer.step)."""
     import torch
@@ -170,7 +176,7 @@ def run_stages(q, g, seed, events=None):
     st = torch.cuda.current_stream()
     calls = stage_calls(q, g)
     events[0].record(st)
-    for k, name in enumerate(STAGES_MULTI if q.multi else STAGES_SINGLE):
+    for k, name in enumerate(stages):
         calls[name](seed)
         events[k + 1].record(st)
 
@@ -200,9 +206,9 @@ def time_device_resident(q, g, w, steps, warmup, barrier):
     n = max(3, min(steps, 10, int(40.0 / max(total_ms / steps, 1e-3))))
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(stages) + 1)] for _ in range(n)]
     time.sleep(BURST_IDLE_S)
-    run_stages(q, g, w.seed, [torch.cuda.Event() for _ in range(len(stages) + 1)])      # the separate calls, untimed
+    run_stages(q, g, w.seed, [torch.cuda.Event() for _ in range(len(stages) + 1)], stages)      # the separate calls, untimed
     for k in range(n):
-        run_stages(q, g, w.seed + k, evs[k])
+        run_stages(q, g, w.seed + k, evs[k], stages)
     torch.cuda.synchronize()
     per_stage = {s: statistics.median(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(n))
                  for i, s in enumerate(stages)}
@@ -336,6 +342,15 @@ def time_encode_other_mode(q, g, w, reps):
         return time_alone(lambda k: q.encode(g, w.seed + k), reps)
     finally:
         q.rng_bits = keep
+
+
+def time_two_kernel_tail(q, g, w, reps):
+    """Where the step's encoder also aggregates and reconstructs: mean ms of the encoder alone and of the
+    aggregation + reconstruction kernel alone (the two calls the one replaces), each looped by itself."""
+    enc = time_alone(lambda k: q.encode(g, w.seed + k), reps)
+    time.sleep(BURST_IDLE_S)
+    dec = time_alone(lambda k: q.aggregate_decode(), reps)
+    return enc, dec
 
 
 def time_fused_select_encode(q, g, w, reps):
@@ -513,7 +528,7 @@ def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=F
                 q.step(g_dev, w.seed + k)
                 evs[-1].record()
             else:
-                run_stages(q, g_dev, w.seed + k, evs)
+                run_stages(q, g_dev, w.seed + k, evs, stages)
             torch.cuda.synchronize()
             tot.append(evs[0].elapsed_time(evs[-1]))
             for i, s in enumerate(stages):
@@ -531,6 +546,10 @@ def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=F
         res["copy_same_bytes_ms"] = {s: time_plain_copy(ab[s]) for s in res["stages_ms"] if ab[s] <= COPY_CONTEXT_MAX_BYTES}
         time.sleep(BURST_IDLE_S)
     res["encode_other_ms"] = time_encode_other_mode(q, g_dev, w, min(steps, 10))
+    if q.fused_decode and not q.one_kernel:
+        time.sleep(BURST_IDLE_S)
+        res["two_kernel_tail_ms"] = time_two_kernel_tail(q, g_dev, w, min(steps, 10))
+        time.sleep(BURST_IDLE_S)
     res["update_ms"] = time_fused_update(q, w, min(steps, 10))
     if q.multi:
         res["fused_select_ms"] = time_fused_select_encode(q, g_dev, w, min(steps, 10))
@@ -599,15 +618,30 @@ def summarize(res, peak_gbs):
     out["kernels"][f"encode_rng{other}"] = {
         "ms": round(ms, 5), "algorithmic_MB": round(ab["encode"] / 1e6, 2), "GBps": round(ab["encode"] / ms / 1e6, 1),
         "frac_of_hbm_peak": round(ab["encode"] / ms / 1e6 / peak_gbs, 4), "note": "timed alone, not part of the step"}
+    if "two_kernel_tail_ms" in res:
+        enc, dec = res["two_kernel_tail_ms"]
+        for key, t in (("encode", enc), ("aggregate_decode", dec)):
+            out["kernels"][key] = {
+                "ms": round(t, 5), "algorithmic_MB": round(ab[key] / 1e6, 2), "GBps": round(ab[key] / t / 1e6, 1),
+                "frac_of_hbm_peak": round(ab[key] / t / 1e6 / peak_gbs, 4),
+                "note": "timed alone, not part of the step: the step makes the two as one call (encode_decode)"}
+        out["kernels"]["encode_decode"]["ms_of_the_two_kernels_it_replaces"] = round(enc + dec, 5)
     if "fused_select_ms" in res:
         ms = res["fused_select_ms"]
-        two = res["stages_ms"].get("select_scale", 0.0) + res["stages_ms"].get("encode", 0.0)
+        sel = res["stages_ms"].get("select_scale", 0.0)
+        if "two_kernel_tail_ms" in res:         # the step's tail is one kernel: compare with selector + encoder alone
+            enc_alone, dec_alone = res["two_kernel_tail_ms"]
+            two = sel + enc_alone
+            step_with = res["ms"] - sel - res["stages_ms"]["encode_decode"] + ms + dec_alone
+        else:
+            two = sel + res["stages_ms"].get("encode", 0.0)
+            step_with = res["ms"] - two + ms
         out["kernels"]["select_encode"] = {
             "ms": round(ms, 5), "algorithmic_MB": round(ab["select_encode"] / 1e6, 2),
             "GBps": round(ab["select_encode"] / ms / 1e6, 1),
             "frac_of_hbm_peak": round(ab["select_encode"] / ms / 1e6 / peak_gbs, 4),
             "ms_of_the_two_kernels_it_replaces": round(two, 5),
-            "gradient_GBps_of_a_step_with_it": round(w.in_bytes / (res["ms"] - two + ms) / 1e6, 1),
+            "gradient_GBps_of_a_step_with_it": round(w.in_bytes / step_with / 1e6, 1),
             "note": "selection + encoding as one call (one kernel for M <= 8: the gradients are read once; bound by "
                     "instruction issue, not by memory), timed alone, not part of the step"}
     lev = {"i8": 1.0, "i4x2": 0.5, "i2x4": 0.25, "i6p": 0.75}[w.fmt]

@@ -222,11 +222,12 @@ int uq_encode_multi(const uq_layout *layout, const void *g, const float *W, cons
  * uq_encode_single (scales = NULL) or uq_encode_multi (scales given) followed by
  * uq_decode(src = UQ_SRC_LEVELS) as one call — Algorithm 1 lines "Quantize gradient", "AllReduce
  * gradients", "Reconstruct gradient" (Algorithm 2: "Quantize with s*" onwards) — for callers whose
- * M workers are all in this buffer.  With int8 levels and M <= 8 it is one kernel: the CTA that
- * takes a tile of coordinates through the workers adds their levels up in registers and writes the
- * reconstructed average beside the level rows, so the levels are written (they are what would cross
- * the wire) but never read back.  With other formats or more workers the two kernels run one after
- * the other.  lev and out receive, bit for bit, what the two separate calls write; arguments and
+ * M workers are all in this buffer.  With int8 levels, 16-bit draws and M <= 8 it is one kernel: the
+ * CTA that takes a tile of coordinates through the workers adds their levels up in registers and
+ * writes the reconstructed average beside the level rows, so the levels are written (they are what
+ * would cross the wire) but never read back.  With other formats, more workers or 32-bit draws
+ * (whose encoder is bound by its arithmetic: one kernel is then no faster than two) the two kernels
+ * run one after the other.  lev and out receive, bit for bit, what the two separate calls write; arguments and
  * errors are theirs (the integer sums are not available here: use uq_decode or uq_aggregate).
  * uq_step makes this call when it is given no S_opt.
  */

@@ -377,7 +377,7 @@ def uq_select_encode_multi(layout: Layout, g: torch.Tensor, W: torch.Tensor, sca
 def uq_encode_decode(layout: Layout, g: torch.Tensor, W: torch.Tensor, s: int, scales: Optional[Sequence[int]],
                      idx: Optional[torch.Tensor], idx_bits: int, seed: int, rng_bits: int, fmt: int, lev: torch.Tensor,
                      out: torch.Tensor, status: Optional[torch.Tensor]) -> None:
-    """uq_encode_single / uq_encode_multi + uq_decode(levels) as one call (one kernel for int8 levels and M <= 8)."""
+    """uq_encode_single / uq_encode_multi + uq_decode(levels) as one call (one kernel for int8 levels, 16-bit draws and M <= 8)."""
     layout.check_g(g)
     layout.check_lev(lev, fmt)
     layout.check_vec(W, torch.float32, layout.nseg, "W")

@@ -20,10 +20,10 @@ cudaError_t launch_aggregate_decode_rows(const uq_layout &L, const void *const *
                                          int32_t *S, cudaStream_t st);
 cudaError_t launch_decode_sums(const uq_layout &L, const int32_t *S, const float *W, const ScaleSet &scales,
                                const uint8_t *idx, int idx_bits, float *out, cudaStream_t st);
-bool encode_decode_fused(const uq_layout &L, int fmt);
+bool encode_decode_fused(const uq_layout &L, int fmt, int rng_bits);
 cudaError_t launch_encode_decode(const uq_layout &L, const void *g, const float *W, const ScaleSet &scales,
-                                 const uint8_t *idx, int idx_bits, uint64_t seed, int rng_bits, void *lev, float *out,
-                                 uint32_t *status, cudaStream_t st);
+                                 const uint8_t *idx, int idx_bits, uint64_t seed, void *lev, float *out, uint32_t *status,
+                                 cudaStream_t st);
 cudaError_t launch_select_encode(const uq_layout &L, const void *g, const float *W, const ScaleSet &scales, int idx_bits,
                                  uint64_t seed, int rng_bits, int fmt, uint8_t *idx, void *lev, uint32_t *status,
                                  cudaStream_t st);
@@ -264,9 +264,8 @@ int uq_encode_decode(const uq_layout *L, const void *g, const float *W, int s, c
     if (L->d > 0 && (g == nullptr || lev == nullptr || out == nullptr || !aligned(g, 16) || !aligned(lev, 16) ||
                      !aligned(out, 32)))
         return UQ_ERR_BAD_ARG;
-    if (uq::encode_decode_fused(*L, fmt))
-        return finish(uq::launch_encode_decode(*L, g, W, set, idx, idx_bits, seed, rng_bits, lev, out, status,
-                                               (cudaStream_t)stream));
+    if (uq::encode_decode_fused(*L, fmt, rng_bits))
+        return finish(uq::launch_encode_decode(*L, g, W, set, idx, idx_bits, seed, lev, out, status, (cudaStream_t)stream));
     const cudaError_t e = uq::launch_encode(*L, g, W, set, idx, idx_bits, seed, rng_bits, fmt, lev, status,
                                             (cudaStream_t)stream);
     if (e != cudaSuccess) return finish(e);

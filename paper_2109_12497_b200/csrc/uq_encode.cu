@@ -36,15 +36,18 @@ cudaError_t launch_encode(const uq_layout &L, const void *g, const float *W, con
 }
 
 // Quantization, sum over the workers and reconstruction in one kernel (decode mode of the encoder):
-// int8 levels and at most kWorkerGroup workers, so that the CTA of a tile sees every worker's levels.
-bool encode_decode_fused(const uq_layout &L, int fmt) { return fmt == UQ_FMT_I8 && L.M <= kWorkerGroup; }
+// int8 levels and at most kWorkerGroup workers, so that the CTA of a tile sees every worker's levels,
+// and 16-bit draws (with 32-bit draws the one kernel is no faster than the two: measured).
+bool encode_decode_fused(const uq_layout &L, int fmt, int rng_bits)
+{
+    return fmt == UQ_FMT_I8 && L.M <= kWorkerGroup && rng_bits == 16;
+}
 
 cudaError_t launch_encode_decode(const uq_layout &L, const void *g, const float *W, const ScaleSet &scales,
-                                 const uint8_t *idx, int idx_bits, uint64_t seed, int rng_bits, void *lev, float *out,
-                                 uint32_t *status, cudaStream_t st)
+                                 const uint8_t *idx, int idx_bits, uint64_t seed, void *lev, float *out, uint32_t *status,
+                                 cudaStream_t st)
 {
-    return launch_encode_any(L, g, W, scales, const_cast<uint8_t *>(idx), idx_bits, false, seed, rng_bits, UQ_FMT_I8, lev, status,
-                             st, out);
+    return launch_encode_any(L, g, W, scales, const_cast<uint8_t *>(idx), idx_bits, false, seed, 16, UQ_FMT_I8, lev, status, st, out);
 }
 
 // Scale selection, scale sharing and quantization in one kernel: a CTA that takes a tile through

@@ -12,7 +12,9 @@
 // block, whose counter differs between workers only in one word.  The work done for worker m
 // reads only g^m plus the agreed values W and idx.
 //
-// Decode mode (int8 levels, M <= 8, so that one CTA sees every worker of its tile): the CTA also adds
+// Decode mode (int8 levels, 16-bit draws, M <= 8, so that one CTA sees every worker of its tile; with
+// 32-bit draws the encoder is bound by its arithmetic and the sums cost what the saved read gains,
+// measured, so there the two kernels stay): the CTA also adds
 // the workers' levels up as it goes and writes the reconstructed average (Algorithm 1 / 2, lines
 // "AllReduce gradients" and "Reconstruct gradient") beside the level rows, which then need not be
 // read back by the aggregation kernel.  Bit for bit what uq_decode makes of the same levels.
@@ -33,8 +35,10 @@ struct EncodeParams {
     int32_t select;           // multi-scale: 1 = find the shared indices here instead of reading them
     int32_t worker0;          // number, in the whole job, of the worker in row 0 (keys the draws)
     int64_t coord0;           // index, in the whole gradient, of coordinate 0 (keys the draws)
-    int64_t ntiles;
-    uint32_t main_blocks;     // CTAs that own tiles; the CTAs after them own rows crossed by boundaries
+    uint32_t row_blocks;      // CTAs that own rows crossed by boundaries: after the tile CTAs, or (decode mode,
+                              // where such a CTA takes every worker's row and runs much longer) in front of them
+    uint32_t reserved;
+    uint32_t main_blocks;     // CTAs that own tiles
     uint32_t groups;          // CTAs per tile: ceil(M / kWorkerGroup)
     PhiloxKey key;            // the ten round keys of the seed
     uint32_t blk_hi;          // high word of the Philox block numbers the table below was made for
@@ -48,9 +52,8 @@ constexpr int kWorkerGroup = 8;   // workers that one CTA takes through a tile
 template <int DT, int RNG> struct EncodeShape {
     static constexpr int UNITS = DT == UQ_BF16 ? 2 : 1;                       // 32 B per thread and worker in flight
     static constexpr int MIN_CTAS = (DT == UQ_BF16 && RNG == 32) ? 3 : 4;
-    // decode mode holds the level sums too: at 64 registers the bf16 kernel spills and the fp32 one with
-    // 32-bit draws is slower than at 80
-    static constexpr int MIN_CTAS_DEC = (DT == UQ_F32 && RNG == 16) ? 4 : 3;
+    // decode mode (16-bit draws only) holds the level sums too: at 64 registers the bf16 kernel spills
+    static constexpr int MIN_CTAS_DEC = DT == UQ_F32 ? 4 : 3;
     static constexpr int TILE = kThreads * UNITS * 8;
 };
 
@@ -238,20 +241,47 @@ __device__ __noinline__ void decode_unit_general(const EncodeParams &p, int64_t 
 }
 
 // The units of tile [t0, t1) that this thread encoded in a slow form (the same assignment of units to
-// threads as encode_span_general and encode_tile_mixed).  mixed: a row that itself contains a
-// boundary was skipped there and is skipped here (a CTA of the second kind owns it).
+// threads as encode_span_general and encode_tile_mixed).  mixed: a full tile crossed by boundaries; a
+// row that itself contains a boundary was skipped there and is skipped here (a CTA of the second
+// kind owns it), every other row lies in one segment, so lane k takes the factor of scale k once
+// per row.  Else (ragged tile and the like) everything is looked up per coordinate.
 template <int DT, int RNG, int IDXB>
 __device__ __noinline__ void decode_tile_slow(const EncodeParams &p, int64_t t0, int64_t t1, bool mixed)
 {
+    constexpr bool MULTI = IDXB != 0;
+    constexpr int IB = MULTI ? IDXB : 8;
+    constexpr int KMASK = IB < 4 ? (1 << IB) - 1 : UQ_MAX_SCALES - 1;
+    const int lane = threadIdx.x & 31;
     for (int u = 0; u < EncodeShape<DT, RNG>::UNITS; ++u) {
         const int64_t r0 = t0 + (int64_t)(u * kThreads + (threadIdx.x & ~31)) * 8;
         if (r0 >= t1) break;                                         // warp-uniform
-        if (mixed) {
-            const int jr = warp_find_segment(p.v.seg_off, p.v.nseg, r0);
-            if (segment_end(p.v.seg_off, p.v.nseg, jr, p.v.d) < r0 + 256) continue;
+        const int64_t i = r0 + lane * 8;
+        if (!mixed) {
+            if (i < t1) decode_unit_general<IDXB>(p, i, 0, false);
+            continue;
         }
-        const int64_t i = r0 + (threadIdx.x & 31) * 8;
-        if (i < t1) decode_unit_general<IDXB>(p, i, 0, false);
+        const int jr = warp_find_segment(p.v.seg_off, p.v.nseg, r0);
+        if (segment_end(p.v.seg_off, p.v.nseg, jr, p.v.d) < r0 + 256) continue;
+        const float c_lane = decode_factor(__ldg(p.v.W + jr), p.v.scales.s[lane & KMASK], p.v.M);
+        uint32_t sum[4] = {0u, 0u, 0u, 0u};                          // as in the straight-line path
+        const char *lp = (const char *)p.lev + i;
+        for (int m = 0; m < p.v.M; ++m) {
+            const uint2 b = __ldcg((const uint2 *)(lp + (size_t)m * (size_t)p.v.stride));
+            const uint32_t bl = b.x ^ 0x80808080u, bh = b.y ^ 0x80808080u;
+            sum[0] += __byte_perm(bl, 0u, 0x4240); sum[1] += __byte_perm(bl, 0u, 0x4341);
+            sum[2] += __byte_perm(bh, 0u, 0x4240); sum[3] += __byte_perm(bh, 0u, 0x4341);
+        }
+        typename IdxBits<IB>::T kbits = 0;
+        if (MULTI) kbits = IdxBits<IB>::load(p.idx + i * IB / 8);
+        const int bias = 128 * p.v.M;
+        uint32_t r[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int S = (int)((sum[(e >> 2) * 2 + (e & 1)] >> (16 * ((e & 3) >> 1))) & 0xFFFFu) - bias;
+            const float c = MULTI ? __shfl_sync(0xFFFFFFFFu, c_lane, (int)(uint32_t)(kbits >> (e * IB))) : c_lane;
+            r[e] = __float_as_uint(__fmul_rn((float)S, c));
+        }
+        st_stream256(p.out + i, r);
     }
 }
 
@@ -450,7 +480,7 @@ template <int DT, int FMT, int RNG, int IDXB, bool SEL, bool DEC>
 __global__ void __launch_bounds__(kThreads, (SEL ? 3 : DEC ? EncodeShape<DT, RNG>::MIN_CTAS_DEC : EncodeShape<DT, RNG>::MIN_CTAS))
 encode_kernel(const __grid_constant__ EncodeParams p)
 {
-    static_assert(!DEC || (FMT == UQ_FMT_I8 && !SEL), "decode mode: int8 levels, indices given");
+    static_assert(!DEC || (FMT == UQ_FMT_I8 && RNG == 16 && !SEL), "decode mode: int8 levels, 16-bit draws, indices given");
     grid_dependency_prologue();
     using T = TileState<DT, FMT, RNG, IDXB, DEC>;
     using E = Elem<DT>;
@@ -461,13 +491,14 @@ encode_kernel(const __grid_constant__ EncodeParams p)
     constexpr int U = T::U, H = T::H, BPU = T::BPU;
     const int tid = threadIdx.x, lane = tid & 31;
     __shared__ int32_t sh_thr[MULTI ? kWarps * 2 * UQ_MAX_SCALES : 1];   // select mode, slow paths: threshold tables
-    if (blockIdx.x >= p.main_blocks) {
+    const uint32_t first_tile_block = DEC ? p.row_blocks : 0u;
+    if (DEC ? blockIdx.x < p.row_blocks : blockIdx.x >= p.main_blocks) {
         // A CTA of the second kind: each warp takes one segment boundary of one worker and, if the
         // boundary lies strictly inside a 256-coordinate row of a full tile, quantizes that row with
         // per-coordinate scales (the tile's own CTA skips it).  Keeping these rows out of the tile
         // CTAs keeps their lifetime short: the slow path no longer holds a whole CTA slot.
         // (decode mode: one warp takes the row of every worker, one after the other, and then decodes it)
-        const uint32_t x = blockIdx.x - p.main_blocks;
+        const uint32_t x = DEC ? blockIdx.x : blockIdx.x - p.main_blocks;
         const int m = DEC ? 0 : (int)(x % (uint32_t)p.v.M);
         const int64_t k = 1 + (int64_t)(DEC ? x : x / (uint32_t)p.v.M) * kWarps + (tid >> 5);
         if (k >= p.v.nseg) return;
@@ -486,7 +517,7 @@ encode_kernel(const __grid_constant__ EncodeParams p)
         return;
     }
     // CTAs walk the tiles back to front (see launch_encode); a tile's CTAs take 8 workers each
-    const uint32_t rev = p.main_blocks - 1u - blockIdx.x;
+    const uint32_t rev = p.main_blocks - 1u - (blockIdx.x - first_tile_block);
     const int64_t tile = (int64_t)(rev / p.groups);
     const int m0 = (int)(rev % p.groups) * kWorkerGroup;
     const int cnt = min(kWorkerGroup, p.v.M - m0);
@@ -654,14 +685,18 @@ template <int DT, int FMT, int RNG, int IDXB, bool SEL = false, bool DEC = false
 static cudaError_t launch(EncodeParams p, cudaStream_t st)
 {
     using S = EncodeShape<DT, RNG>;
-    p.ntiles = (p.v.d + S::TILE - 1) / S::TILE;
+    const int64_t ntiles = (p.v.d + S::TILE - 1) / S::TILE;
+    p.reserved = 0u;
     p.groups = (uint32_t)((p.v.M + kWorkerGroup - 1) / kWorkerGroup);
-    int64_t blocks = p.ntiles * p.groups;
+    int64_t blocks = ntiles * p.groups;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     p.main_blocks = (uint32_t)blocks;
-    if (p.v.seg_off != nullptr && p.v.nseg > 1) blocks += (int64_t)((p.v.nseg - 1 + kWarps - 1) / kWarps) * (DEC ? 1 : p.v.M);
+    int64_t rows = 0;
+    if (p.v.seg_off != nullptr && p.v.nseg > 1) rows = (int64_t)((p.v.nseg - 1 + kWarps - 1) / kWarps) * (DEC ? 1 : p.v.M);
+    blocks += rows;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    p.row_blocks = (uint32_t)rows;
     constexpr int BSH = RNG == 32 ? 2 : 3;
     p.blk_hi = (uint32_t)((uint64_t)(p.coord0 >> BSH) >> 32);
     for (int m = 0; m < UQ_MAX_WORKERS; ++m)
@@ -691,7 +726,7 @@ static cudaError_t launch(EncodeParams p, cudaStream_t st)
 template <int DT, int FMT, int RNG>
 static cudaError_t dispatch_idx(const EncodeParams &p, int idx_bits, cudaStream_t st)
 {
-    if constexpr (FMT == UQ_FMT_I8) {
+    if constexpr (FMT == UQ_FMT_I8 && RNG == 16) {
         if (p.out != nullptr) {                       // decode mode (the caller has checked M <= kWorkerGroup, no select)
             switch (idx_bits) {
             case 0: return launch<DT, FMT, RNG, 0, false, true>(p, st);

@@ -94,14 +94,15 @@ class Quantizer:
 
     def encode_decode(self, g: torch.Tensor, seed: int) -> None:
         """Quantization, integer aggregation and reconstruction as one call (what the step makes when
-        the integer sums are not kept; one kernel for int8 levels and M <= 8)."""
+        the integer sums are not kept; one kernel for int8 levels, 16-bit draws and M <= 8)."""
         B.uq_encode_decode(self.layout, g, self.W, self.s, self.scales, self.idx, self.idx_bits, seed, self.rng_bits,
                            self.fmt, self.lev, self.out, self.status)
 
     @property
     def fused_decode(self) -> bool:
         """Whether the step's encoder also aggregates and reconstructs (uq_encode_decode as one kernel)."""
-        return self.S is None and self.fmt == B.UQ_FMT_I8 and self.layout.M <= B.SMALL_STEP_MAX_WORKERS
+        return (self.S is None and self.fmt == B.UQ_FMT_I8 and self.layout.M <= B.SMALL_STEP_MAX_WORKERS
+                and self.rng_bits == 16)
 
     def aggregate_decode_update(self, theta: torch.Tensor, momentum: Optional[torch.Tensor], lr: float,
                                 mu: float = 0.0, wd: float = 0.0) -> None:
@@ -158,11 +159,13 @@ class Quantizer:
         B.require_current_device(self.device.index, current, "the quantizer")
 
     def kernels_per_step(self) -> int:
-        """Kernel launches one step enqueues (norm partials + finalize, [select], encode, decode)."""
+        """Kernel launches one step enqueues (norm partials + finalize, [select], encode, decode; the
+        last two are one kernel when the encoder also aggregates and reconstructs)."""
         if self.one_kernel:
             return 1
         separate_select = self.multi and (not self.fused_select or self.M > 8) and self.d > 0
-        return (2 if self.d > 0 else 1) + (1 if separate_select else 0) + (2 if self.d > 0 else 0)
+        tail = 0 if self.d == 0 else 1 if (self.fused_decode and not self.fused_select) else 2
+        return (2 if self.d > 0 else 1) + (1 if separate_select else 0) + tail
 
     def status_bits(self) -> int:
         """Synchronizes and returns the device status word (0 = clean)."""
