@@ -76,6 +76,8 @@ def algorithmic_bytes(w: wl.Workload) -> dict:
         b["encode"] = (e + lev) * M * d
     b["aggregate_decode"] = lev * M * d + ib * d + 4 * d
     b["encode_decode"] = b["encode"] + 4 * d          # one call: the levels are written but not read back
+    if w.quantizer == "multi":
+        b["select_encode_decode"] = b["select_encode"] + 4 * d      # gradients read once, index, levels, average written
     return b
 
 
@@ -153,6 +155,8 @@ def encoder_decodes(w) -> bool:
 
 def stages_of(w):
     """The calls uq_step makes for this workload (without the integer sums among its outputs)."""
+    if w.quantizer == "multi" and encoder_decodes(w):
+        return ["agree_scale", "select_encode_decode"]      # the encoder also selects: two calls do the step
     head = ["agree_scale", "select_scale"] if w.quantizer == "multi" else ["agree_scale"]
     return head + (["encode_decode"] if encoder_decodes(w) else ["encode", "aggregate_decode"])
 
@@ -162,6 +166,8 @@ def stage_calls(q, g):
     calls = {"agree_scale": lambda seed: q.agree_scale(g), "aggregate_decode": lambda seed: q.aggregate_decode()}
     calls["encode"] = lambda seed: q.encode(g, seed)
     calls["encode_decode"] = lambda seed: q.encode_decode(g, seed)
+    if q.multi:
+        calls["select_encode_decode"] = lambda seed: q.select_encode_decode(g, seed)
     if q.multi:
         calls["select_scale"] = lambda seed: q.select_scale(g)
     return calls
@@ -360,6 +366,12 @@ def time_fused_select_encode(q, g, w, reps):
     return time_alone(lambda k: q.select_encode(g, w.seed + k), reps)
 
 
+def time_fused_select_encode_decode(q, g, w, reps):
+    """Multi-scale: mean ms of everything behind the scale agreement as one call
+    (uq_select_encode_decode_multi), timed alone."""
+    return time_alone(lambda k: q.select_encode_decode(g, w.seed + k), reps)
+
+
 def time_graph_replay(q, g, w, reps, stats=False):
     """ms per step when the step's launches are captured once in a CUDA graph and replayed: the
     figure for a working set so small that launch latency, not memory, sets the time.  stats:
@@ -551,9 +563,18 @@ def bench_workload(w, steps, warmup, barrier, threads, want_e2e, flush_between=F
         time.sleep(BURST_IDLE_S)
         res["two_kernel_tail_ms"] = time_two_kernel_tail(q, g_dev, w, min(steps, 10))
         time.sleep(BURST_IDLE_S)
+        if q.multi:       # the step's second call also selects: the calls it stands for, each looped alone
+            res["alone_ms"] = {}
+            for name, fn in (("select_scale", lambda k: q.select_scale(g_dev)),
+                             ("encode_decode", lambda k: q.encode_decode(g_dev, w.seed + k))):
+                res["alone_ms"][name] = time_alone(fn, min(steps, 10))
+                time.sleep(BURST_IDLE_S)
     res["update_ms"] = time_fused_update(q, w, min(steps, 10))
     if q.multi:
         res["fused_select_ms"] = time_fused_select_encode(q, g_dev, w, min(steps, 10))
+        if q.fused_decode and not q.one_kernel and "select_encode_decode" not in res["stages_ms"]:
+            time.sleep(BURST_IDLE_S)
+            res["fused_all_ms"] = time_fused_select_encode_decode(q, g_dev, w, min(steps, 10))
     if randk_K:
         res["randk"] = time_randk(w, g_dev, min(randk_K, w.d), 50)
         if w.quantizer == "single":               # the same choice quantized with a two-scale set (GlobalRandK-MN-TS)
@@ -626,11 +647,30 @@ def summarize(res, peak_gbs):
                 "ms": round(t, 5), "algorithmic_MB": round(ab[key] / 1e6, 2), "GBps": round(ab[key] / t / 1e6, 1),
                 "frac_of_hbm_peak": round(ab[key] / t / 1e6 / peak_gbs, 4),
                 "note": "timed alone, not part of the step: the step makes the two as one call (encode_decode)"}
+        for key, t in res.get("alone_ms", {}).items():
+            out["kernels"][key] = {
+                "ms": round(t, 5), "algorithmic_MB": round(ab[key] / 1e6, 2), "GBps": round(ab[key] / t / 1e6, 1),
+                "frac_of_hbm_peak": round(ab[key] / t / 1e6 / peak_gbs, 4),
+                "note": "timed alone, not part of the step: the step makes selection, encoding, aggregation and "
+                        "reconstruction as one call (select_encode_decode)"}
         out["kernels"]["encode_decode"]["ms_of_the_two_kernels_it_replaces"] = round(enc + dec, 5)
+        if "select_encode_decode" in out["kernels"] and "alone_ms" in res:
+            three = res["alone_ms"]["select_scale"] + res["alone_ms"]["encode_decode"]
+            out["kernels"]["select_encode_decode"]["ms_of_the_two_kernels_it_replaces"] = round(three, 5)
+            out["kernels"]["select_encode_decode"]["gradient_GBps_of_a_step_without_it"] = round(
+                w.in_bytes / (res["ms"] - res["stages_ms"]["select_encode_decode"] + three) / 1e6, 1)
+            out["kernels"]["select_encode_decode"]["note"] = (
+                "selection + encoding + aggregation + reconstruction as one kernel: the gradients are read once and "
+                "nothing is read back; bound by instruction issue (ALU pipe), not by memory, so its fraction of the HBM "
+                "peak is lower than that of the streaming kernels it replaces (timed alone beside it), and its time shorter")
     if "fused_select_ms" in res:
         ms = res["fused_select_ms"]
-        sel = res["stages_ms"].get("select_scale", 0.0)
-        if "two_kernel_tail_ms" in res:         # the step's tail is one kernel: compare with selector + encoder alone
+        sel = res["stages_ms"].get("select_scale", res.get("alone_ms", {}).get("select_scale", 0.0))
+        if "select_encode_decode" in res["stages_ms"]:      # the step already selects inside its second call
+            enc_alone, dec_alone = res["two_kernel_tail_ms"]
+            two = sel + enc_alone
+            step_with = res["ms"] - res["stages_ms"]["select_encode_decode"] + ms + dec_alone
+        elif "two_kernel_tail_ms" in res:       # the step's tail is one kernel: compare with selector + encoder alone
             enc_alone, dec_alone = res["two_kernel_tail_ms"]
             two = sel + enc_alone
             step_with = res["ms"] - sel - res["stages_ms"]["encode_decode"] + ms + dec_alone
@@ -645,6 +685,18 @@ def summarize(res, peak_gbs):
             "gradient_GBps_of_a_step_with_it": round(w.in_bytes / step_with / 1e6, 1),
             "note": "selection + encoding as one call (one kernel for M <= 8: the gradients are read once; bound by "
                     "instruction issue, not by memory), timed alone, not part of the step"}
+    if "fused_all_ms" in res:
+        ms = res["fused_all_ms"]
+        nbytes = ab["select_encode"] + 4 * w.d
+        two = res["stages_ms"]["select_scale"] + res["stages_ms"]["encode_decode"]
+        out["kernels"]["select_encode_decode"] = {
+            "ms": round(ms, 5), "algorithmic_MB": round(nbytes / 1e6, 2), "GBps": round(nbytes / ms / 1e6, 1),
+            "frac_of_hbm_peak": round(nbytes / ms / 1e6 / peak_gbs, 4),
+            "ms_of_the_two_kernels_it_replaces": round(two, 5),
+            "gradient_GBps_of_a_step_with_it": round(w.in_bytes / (res["ms"] - two + ms) / 1e6, 1),
+            "note": "selection + encoding + aggregation + reconstruction as one call (uq_select_encode_decode_multi: one "
+                    "kernel, the gradients are read once and nothing is read back; bound by instruction issue, not by "
+                    "memory), timed alone, not part of the step"}
     lev = {"i8": 1.0, "i4x2": 0.5, "i2x4": 0.25, "i6p": 0.75}[w.fmt]
     upd_bytes = lev * w.M * w.d + w.idx_bits / 8.0 * w.d + 16 * w.d      # levels, index, theta and momentum r/w
     ms = res["update_ms"]

@@ -28,7 +28,7 @@ EXPORTS = (
     "uq_version", "uq_last_cuda_error", "uq_error_string", "uq_workspace_bytes", "uq_index_bytes",
     "uq_workspace_bytes_small",
     "uq_agree_scale", "uq_agree_scale_static", "uq_encode_single", "uq_select_scale_multi", "uq_encode_multi",
-    "uq_aggregate", "uq_decode", "uq_decode_update", "uq_randk_gather", "uq_randk_scatter", "uq_randk_update", "uq_index_min", "uq_decode_rows", "uq_select_encode_multi", "uq_encode_decode", "uq_step",
+    "uq_aggregate", "uq_decode", "uq_decode_update", "uq_randk_gather", "uq_randk_scatter", "uq_randk_update", "uq_index_min", "uq_decode_rows", "uq_select_encode_multi", "uq_encode_decode", "uq_select_encode_decode_multi", "uq_step",
     "uq_step_small",
 )
 
@@ -94,6 +94,7 @@ def lib() -> C.CDLL:
         L.uq_select_encode_multi.argtypes = [LP, P, P, P, I, I, U64, I, I, P, P, P, P]
         L.uq_decode_rows.argtypes = [LP, P, I, P, I, P, I, P, I, P, P, P]
         L.uq_encode_decode.argtypes = [LP, P, P, I, P, I, P, I, U64, I, I, P, P, P, P]
+        L.uq_select_encode_decode_multi.argtypes = [LP, P, P, P, I, I, U64, I, I, P, P, P, P, P]
         L.uq_index_min.argtypes = [P, I, I64, I64, I, P, P]
         L.uq_randk_gather.argtypes = [LP, P, I64, U64, P, P, I64, P, P]
         L.uq_randk_scatter.argtypes = [I64, I64, P, P, P, P, P]
@@ -372,6 +373,21 @@ def uq_select_encode_multi(layout: Layout, g: torch.Tensor, W: torch.Tensor, sca
         layout.ref(), _ptr(g), _ptr(W), arr, N, idx_bits, seed, rng_bits, fmt, _ptr(idx), _ptr(lev), _ptr(status),
         _stream()))
 
+
+
+def uq_select_encode_decode_multi(layout: Layout, g: torch.Tensor, W: torch.Tensor, scales: Sequence[int], idx_bits: int,
+                                  seed: int, rng_bits: int, fmt: int, idx: torch.Tensor, lev: torch.Tensor,
+                                  out: torch.Tensor, status: Optional[torch.Tensor]) -> None:
+    """uq_select_encode_multi + uq_decode(levels) as one call (one kernel where uq_encode_decode is one)."""
+    layout.check_g(g)
+    layout.check_lev(lev, fmt)
+    layout.check_vec(W, torch.float32, layout.nseg, "W")
+    layout.check_vec(out, torch.float32, layout.d, "out")
+    layout.check_vec(idx, torch.uint8, layout.index_bytes(idx_bits), "idx")
+    arr, N = _scales(scales)
+    _check("uq_select_encode_decode_multi", lib().uq_select_encode_decode_multi(
+        layout.ref(), _ptr(g), _ptr(W), arr, N, idx_bits, seed, rng_bits, fmt, _ptr(idx), _ptr(lev), _ptr(out),
+        _ptr(status), _stream()))
 
 
 def uq_encode_decode(layout: Layout, g: torch.Tensor, W: torch.Tensor, s: int, scales: Optional[Sequence[int]],

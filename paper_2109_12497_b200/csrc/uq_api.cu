@@ -20,6 +20,9 @@ cudaError_t launch_aggregate_decode_rows(const uq_layout &L, const void *const *
                                          int32_t *S, cudaStream_t st);
 cudaError_t launch_decode_sums(const uq_layout &L, const int32_t *S, const float *W, const ScaleSet &scales,
                                const uint8_t *idx, int idx_bits, float *out, cudaStream_t st);
+cudaError_t launch_select_encode_decode(const uq_layout &L, const void *g, const float *W, const ScaleSet &scales,
+                                        int idx_bits, uint64_t seed, uint8_t *idx, void *lev, float *out, uint32_t *status,
+                                        cudaStream_t st);
 bool encode_decode_fused(const uq_layout &L, int fmt, int rng_bits);
 cudaError_t launch_encode_decode(const uq_layout &L, const void *g, const float *W, const ScaleSet &scales,
                                  const uint8_t *idx, int idx_bits, uint64_t seed, void *lev, float *out, uint32_t *status,
@@ -272,6 +275,26 @@ int uq_encode_decode(const uq_layout *L, const void *g, const float *W, int s, c
     return finish(uq::launch_aggregate_decode(*L, lev, fmt, W, set, idx, idx_bits, out, nullptr, (cudaStream_t)stream));
 }
 
+int uq_select_encode_decode_multi(const uq_layout *L, const void *g, const float *W, const int32_t *scales, int N,
+                                  int idx_bits, uint64_t seed, int rng_bits, int fmt, uint8_t *idx, void *lev, float *out,
+                                  uint32_t *status, void *stream)
+{
+    uq::ScaleSet set;
+    if (!layout_ok(L) || W == nullptr || !aligned(status, 4)) return UQ_ERR_BAD_ARG;
+    if (!scales_ok(scales, N, idx_bits, &set)) return UQ_ERR_BAD_ARG;
+    if (!fmt_ok(fmt, set.s[0]) || (rng_bits != 32 && rng_bits != 16)) return UQ_ERR_BAD_ARG;
+    if (L->d > 0 && (g == nullptr || lev == nullptr || idx == nullptr || out == nullptr || !aligned(g, 16) ||
+                     !aligned(lev, 16) || !aligned(idx, 16) || !aligned(out, 32)))
+        return UQ_ERR_BAD_ARG;
+    if (uq::encode_decode_fused(*L, fmt, rng_bits))
+        return finish(uq::launch_select_encode_decode(*L, g, W, set, idx_bits, seed, idx, lev, out, status,
+                                                      (cudaStream_t)stream));
+    const cudaError_t e = uq::launch_select_encode(*L, g, W, set, idx_bits, seed, rng_bits, fmt, idx, lev, status,
+                                                   (cudaStream_t)stream);
+    if (e != cudaSuccess) return finish(e);
+    return finish(uq::launch_aggregate_decode(*L, lev, fmt, W, set, idx, idx_bits, out, nullptr, (cudaStream_t)stream));
+}
+
 int uq_decode_rows(const uq_layout *L, const void *const *lev_rows, int fmt, const float *W, int s,
                    const int32_t *scales, int N, const uint8_t *idx, int idx_bits, float *out, int32_t *S_opt,
                    void *stream)
@@ -326,6 +349,11 @@ int uq_step(const uq_layout *L, const void *g, int norm, int s, const int32_t *s
     int rc = uq_agree_scale(L, g, norm, W, status, workspace, workspace_bytes, stream);
     if (rc != UQ_OK) return rc;
     if (scales != nullptr) {
+        // nobody wants the integer sums, and the encoder can select, add up and reconstruct itself: the
+        // rest of the step is one kernel
+        if (S_opt == nullptr && layout_ok(L) && uq::encode_decode_fused(*L, fmt, rng_bits))
+            return uq_select_encode_decode_multi(L, g, W, scales, N, idx_bits, seed, rng_bits, fmt, idx, lev, out, status,
+                                                 stream);
         rc = uq_select_scale_multi(L, g, W, scales, N, idx_bits, idx, status, stream);
         if (rc != UQ_OK) return rc;
     }

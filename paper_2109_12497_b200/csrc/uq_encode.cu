@@ -67,4 +67,13 @@ cudaError_t launch_select_encode(const uq_layout &L, const void *g, const float 
     return launch_encode_any(L, g, W, scales, idx, idx_bits, true, seed, rng_bits, fmt, lev, status, st);
 }
 
+// Select mode and decode mode of the encoder together: everything of a multi-scale step behind the
+// scale agreement in one kernel.  The caller has checked encode_decode_fused().
+cudaError_t launch_select_encode_decode(const uq_layout &L, const void *g, const float *W, const ScaleSet &scales,
+                                        int idx_bits, uint64_t seed, uint8_t *idx, void *lev, float *out, uint32_t *status,
+                                        cudaStream_t st)
+{
+    return launch_encode_any(L, g, W, scales, idx, idx_bits, true, seed, 16, UQ_FMT_I8, lev, status, st, out);
+}
+
 }  // namespace uq

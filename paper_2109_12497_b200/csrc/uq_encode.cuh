@@ -231,7 +231,8 @@ __device__ __noinline__ void decode_unit_general(const EncodeParams &p, int64_t 
         }
     }
     uint64_t kbits = kbits_own;
-    if (MULTI && !own_idx) kbits = (uint64_t)IdxBits<IB>::load(p.idx + i * IB / 8);
+    if (MULTI && !own_idx)        // select mode: the CTA stored the tile's indices itself (behind a barrier)
+        kbits = (uint64_t)(p.select ? IdxBits<IB>::load_written(p.idx + i * IB / 8) : IdxBits<IB>::load(p.idx + i * IB / 8));
     int j = find_segment(p.v.seg_off, p.v.nseg, i);
     for (int e = 0; e < 8 && i + e < p.v.d; ++e) {
         j = advance_segment(p.v.seg_off, p.v.nseg, j, i + e);
@@ -272,7 +273,7 @@ __device__ __noinline__ void decode_tile_slow(const EncodeParams &p, int64_t t0,
             sum[2] += __byte_perm(bh, 0u, 0x4240); sum[3] += __byte_perm(bh, 0u, 0x4341);
         }
         typename IdxBits<IB>::T kbits = 0;
-        if (MULTI) kbits = IdxBits<IB>::load(p.idx + i * IB / 8);
+        if (MULTI) kbits = p.select ? IdxBits<IB>::load_written(p.idx + i * IB / 8) : IdxBits<IB>::load(p.idx + i * IB / 8);
         const int bias = 128 * p.v.M;
         uint32_t r[8];
 #pragma unroll
@@ -475,12 +476,12 @@ __device__ __forceinline__ void staged_max_magnitude(const uint4 *stage, int u, 
 // SEL: the kernel also finds and stores the shared scale indices (multi-scale, all M <= kWorkerGroup
 // workers in one CTA): the tile's rows are copied to shared memory once (every thread its own
 // units, so no barrier), read there for the maximum over the workers and again for quantization.
-// DEC: decode mode (see the head of this file; int8 levels, one CTA per tile, not together with SEL).
+// DEC: decode mode (see the head of this file; int8 levels, 16-bit draws, one CTA per tile; with or without SEL).
 template <int DT, int FMT, int RNG, int IDXB, bool SEL, bool DEC>
 __global__ void __launch_bounds__(kThreads, (SEL ? 3 : DEC ? EncodeShape<DT, RNG>::MIN_CTAS_DEC : EncodeShape<DT, RNG>::MIN_CTAS))
 encode_kernel(const __grid_constant__ EncodeParams p)
 {
-    static_assert(!DEC || (FMT == UQ_FMT_I8 && RNG == 16 && !SEL), "decode mode: int8 levels, 16-bit draws, indices given");
+    static_assert(!DEC || (FMT == UQ_FMT_I8 && RNG == 16), "decode mode: int8 levels, 16-bit draws");
     grid_dependency_prologue();
     using T = TileState<DT, FMT, RNG, IDXB, DEC>;
     using E = Elem<DT>;
@@ -508,8 +509,13 @@ encode_kernel(const __grid_constant__ EncodeParams p)
         if (b <= 0 || b == r0 || r0 >= full_end) return;           // not strictly inside a row of a full tile
         if (prev > r0 && prev <= b) return;                        // an earlier boundary in the same row takes it
         if (DEC) {
-            for (int mm = 0; mm < p.v.M; ++mm) encode_span_general<DT, FMT, RNG, IDXB>(p, mm, r0, r0 + 256, lane, 32);
-            decode_unit_general<IDXB>(p, r0 + lane * 8, 0, false);
+            // (select mode: the tile's own CTA stores the row's shared indices; this warp finds them for itself)
+            const bool own = MULTI && p.select;
+            int32_t *thr = sh_thr + (MULTI ? (tid >> 5) * 2 * UQ_MAX_SCALES : 0);
+            for (int mm = 0; mm < p.v.M; ++mm) encode_span_general<DT, FMT, RNG, IDXB>(p, mm, r0, r0 + 256, lane, 32, own, thr);
+            uint64_t kbits = 0;
+            if (own) kbits = (uint64_t)select_unit<DT, IB, 4>(p.v, r0 + lane * 8, r0, thr);
+            decode_unit_general<IDXB>(p, r0 + lane * 8, kbits, own);
             return;
         }
         encode_span_general<DT, FMT, RNG, IDXB>(p, m, r0, r0 + 256, lane, 32, MULTI && p.select,
@@ -727,13 +733,23 @@ template <int DT, int FMT, int RNG>
 static cudaError_t dispatch_idx(const EncodeParams &p, int idx_bits, cudaStream_t st)
 {
     if constexpr (FMT == UQ_FMT_I8 && RNG == 16) {
-        if (p.out != nullptr) {                       // decode mode (the caller has checked M <= kWorkerGroup, no select)
+        if (p.out != nullptr && !p.select) {          // decode mode (the caller has checked M <= kWorkerGroup)
             switch (idx_bits) {
             case 0: return launch<DT, FMT, RNG, 0, false, true>(p, st);
             case 1: return launch<DT, FMT, RNG, 1, false, true>(p, st);
             case 2: return launch<DT, FMT, RNG, 2, false, true>(p, st);
             case 4: return launch<DT, FMT, RNG, 4, false, true>(p, st);
             default: return launch<DT, FMT, RNG, 8, false, true>(p, st);
+            }
+        }
+    }
+    if constexpr (FMT == UQ_FMT_I8 && RNG == 16) {
+        if (p.out != nullptr && p.select) {           // select mode and decode mode together
+            switch (idx_bits) {
+            case 1: return launch<DT, FMT, RNG, 1, true, true>(p, st);
+            case 2: return launch<DT, FMT, RNG, 2, true, true>(p, st);
+            case 4: return launch<DT, FMT, RNG, 4, true, true>(p, st);
+            default: return launch<DT, FMT, RNG, 8, true, true>(p, st);
             }
         }
     }

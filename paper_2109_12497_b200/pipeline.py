@@ -23,7 +23,7 @@ class Quantizer:
                  seg_off: Optional[Sequence[int]] = None, s: int = 127,
                  scales: Optional[Sequence[int]] = None, fmt: int = B.UQ_FMT_I8, idx_bits: int = 0,
                  norm: int = B.UQ_NORM_L2, rng_bits: int = 32, keep_sums: bool = False,
-                 device: str | torch.device = "cuda", fused_select: bool = False,
+                 device: str | torch.device = "cuda", fused_select: Optional[bool] = None,
                  one_kernel: Optional[bool] = None):
         B.lib()                                     # fail now if the CUDA library is not built
         dev = torch.device(device)
@@ -33,10 +33,11 @@ class Quantizer:
         self.M, self.d, self.dtype = M, d, dtype
         self.stride = -(-d // 32) * 32
         self.multi = scales is not None and idx_bits != 0
-        # multi-scale: selection + sharing + encoding as one call (uq_select_encode_multi: one kernel
-        # for M <= 8, the gradients read once: about 15 % less time for the pair on B200, same bits)
-        # instead of the selector and the encoder as two streaming kernels (uq_step, the default)
-        self.fused_select = fused_select and self.multi
+        # multi-scale: whether selection + sharing run inside the encoder's kernel (one kernel for M <= 8,
+        # the gradients read once, same bits) instead of as a streaming kernel of their own.  None = the
+        # library's own choice (uq_step: inside where the encoder also aggregates and reconstructs, i.e.
+        # int8 levels, 16-bit draws, M <= 8 and no integer sums kept; a kernel of its own otherwise).
+        self.fused_select = None if fused_select is None else bool(fused_select) and self.multi
         self.s = int(scales[0]) if self.multi else int(s)
         self.scales = [int(x) for x in scales] if self.multi else None
         self.fmt, self.idx_bits, self.norm, self.rng_bits = fmt, idx_bits if self.multi else 0, norm, rng_bits
@@ -88,6 +89,11 @@ class Quantizer:
         B.uq_select_encode_multi(self.layout, g, self.W, self.scales, self.idx_bits, seed, self.rng_bits, self.fmt,
                                  self.idx, self.lev, self.status)
 
+    def select_encode_decode(self, g: torch.Tensor, seed: int) -> None:
+        """Multi-scale: everything behind the scale agreement in one call."""
+        B.uq_select_encode_decode_multi(self.layout, g, self.W, self.scales, self.idx_bits, seed, self.rng_bits,
+                                        self.fmt, self.idx, self.lev, self.out, self.status)
+
     def aggregate_decode(self) -> None:
         B.uq_decode(self.layout, self.lev, B.UQ_SRC_LEVELS, self.fmt, self.W, self.s, self.scales, self.idx,
                     self.idx_bits, self.out, self.S)
@@ -97,6 +103,13 @@ class Quantizer:
         the integer sums are not kept; one kernel for int8 levels, 16-bit draws and M <= 8)."""
         B.uq_encode_decode(self.layout, g, self.W, self.s, self.scales, self.idx, self.idx_bits, seed, self.rng_bits,
                            self.fmt, self.lev, self.out, self.status)
+
+    @property
+    def selects_inside(self) -> bool:
+        """Multi-scale: whether the step's selection runs inside the encoder's kernel."""
+        if not self.multi:
+            return False
+        return self.fused_decode if self.fused_select is None else self.fused_select
 
     @property
     def fused_decode(self) -> bool:
@@ -128,7 +141,7 @@ class Quantizer:
             if rc != B.UQ_OK:
                 raise B.UqError("uq_step_small", rc)
             return self._out_view
-        if not self.fused_select:                             # the default sequence: one trip through the binding (uq_step)
+        if self.fused_select is None:                         # the library's sequence: one trip through the binding (uq_step)
             self._check_devices(g)
             if self._step_call is None:                      # addresses of my own buffers, marshalled once
                 ptr = lambda t: None if t is None else t.data_ptr()
@@ -142,9 +155,22 @@ class Quantizer:
             if rc != B.UQ_OK:
                 raise B.UqError("uq_step", rc)
             return self._out_view
-        self.agree_scale(g)                                   # multi-scale, selection inside the encoder's kernel
-        self.select_encode(g, seed)
-        self.aggregate_decode()
+        # the caller's choice of where selection runs, call by call
+        self.agree_scale(g)
+        if self.fused_select:                                 # inside the encoder's kernel
+            if self.S is None:                                # ... and aggregation + reconstruction too, where it can
+                self.select_encode_decode(g, seed)
+            else:
+                self.select_encode(g, seed)
+                self.aggregate_decode()
+            return self.out[: self.d]
+        if self.multi:
+            self.select_scale(g)
+        if self.S is None:
+            self.encode_decode(g, seed)
+        else:
+            self.encode(g, seed)
+            self.aggregate_decode()
         return self.out[: self.d]
 
     def _check_devices(self, g: torch.Tensor) -> None:
@@ -163,8 +189,9 @@ class Quantizer:
         last two are one kernel when the encoder also aggregates and reconstructs)."""
         if self.one_kernel:
             return 1
-        separate_select = self.multi and (not self.fused_select or self.M > 8) and self.d > 0
-        tail = 0 if self.d == 0 else 1 if (self.fused_decode and not self.fused_select) else 2
+        inside = self.selects_inside
+        separate_select = self.multi and (not inside or self.M > 8) and self.d > 0
+        tail = 0 if self.d == 0 else 1 if self.fused_decode else 2
         return (2 if self.d > 0 else 1) + (1 if separate_select else 0) + tail
 
     def status_bits(self) -> int:
@@ -223,7 +250,7 @@ class RandKQuantizer:
         return int(self.status.item())
 
 
-def from_workload(w, keep_sums: bool = False, device="cuda", fused_select: bool = False,
+def from_workload(w, keep_sums: bool = False, device="cuda", fused_select: Optional[bool] = None,
                   one_kernel: Optional[bool] = None) -> Quantizer:
     """A Quantizer configured like a ``workloads.Workload``."""
     from . import workloads as wl

@@ -26,12 +26,19 @@ def run_gpu(w, g_np, seed=None, mode="default"):
     "fused" (multi-scale: selection and encoding as one call, uq_select_encode_multi), "one" (the
     whole step as one cooperative kernel), "separate" (never the one-kernel step), "nosums" (the step
     without the integer sums among its outputs: quantization, aggregation and reconstruction as one
-    call, uq_encode_decode; the sums compared below then come from uq_aggregate over its levels)."""
-    one_kernel = {"one": True, "separate": False, "fused": False, "nosums": False}.get(mode)   # else: the library decides by size
-    q = from_workload(w, keep_sums=mode != "nosums", fused_select=mode == "fused", one_kernel=one_kernel)
+    call, uq_encode_decode; the sums compared below then come from uq_aggregate over its levels),
+    "fused_nosums" (multi-scale: everything behind the scale agreement as one call,
+    uq_select_encode_decode_multi), "auto_nosums" (uq_step without the integer sums: the form a user
+    gets, in which the library picks the fewest kernels itself)."""
+    one_kernel = {"one": True, "separate": False, "fused": False, "nosums": False, "fused_nosums": False,
+                  "auto_nosums": False}.get(mode)               # else: the library decides by size
+    nosums = mode in ("nosums", "fused_nosums", "auto_nosums")
+    # where selection runs: the library's choice (uq_step), or the caller's, call by call
+    fused_select = None if mode in ("default", "auto_nosums") else mode in ("fused", "fused_nosums")
+    q = from_workload(w, keep_sums=not nosums, fused_select=fused_select, one_kernel=one_kernel)
     g = to_device(w, g_np)
     q.step(g, w.seed if seed is None else seed)
-    if mode == "nosums":
+    if nosums:
         q.S = torch.empty(max(w.d, 1), dtype=torch.int32, device="cuda")
         B.uq_aggregate(q.layout, q.lev, q.fmt, q.S)
     torch.cuda.synchronize()
@@ -91,7 +98,9 @@ def check_parity(w, g_np, seed=None):
     the encoder aggregates and reconstructs itself where it can): each must match the oracle."""
     if w.quantizer == "multi":
         _check_parity(w, g_np, seed, "fused")
+        _check_parity(w, g_np, seed, "fused_nosums")
     _check_parity(w, g_np, seed, "nosums")
+    _check_parity(w, g_np, seed, "auto_nosums")
     if one_kernel_takes(w):
         _check_parity(w, g_np, seed, "one")
         _check_parity(w, g_np, seed, "separate")

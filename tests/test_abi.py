@@ -120,6 +120,9 @@ def test_later_entry_points_reject_bad_arguments_on_the_host(lib):
     assert lib.uq_select_encode_multi(ok, p, p, sc, 2, 3, 0, 16, B.UQ_FMT_I8, p, p, None, None) == B.UQ_ERR_BAD_ARG   # idx_bits
     assert lib.uq_select_encode_multi(ok, p, p, sc, 2, 2, 0, 16, B.UQ_FMT_I4X2, p, p, None, None) == B.UQ_ERR_BAD_ARG  # s_hat > 7
     assert lib.uq_select_encode_multi(ok, p, p, sc, 2, 2, 0, 16, B.UQ_FMT_I8, None, p, None, None) == B.UQ_ERR_BAD_ARG
+    assert lib.uq_select_encode_decode_multi(ok, p, p, sc, 2, 3, 0, 16, B.UQ_FMT_I8, p, p, p, None, None) == B.UQ_ERR_BAD_ARG   # idx_bits
+    assert lib.uq_select_encode_decode_multi(ok, p, p, sc, 2, 2, 0, 16, B.UQ_FMT_I8, p, p, None, None, None) == B.UQ_ERR_BAD_ARG  # out
+    assert lib.uq_select_encode_decode_multi(ok, p, p, sc, 2, 2, 0, 16, B.UQ_FMT_I8, p, p, p + 16, None, None) == B.UQ_ERR_BAD_ARG  # out alignment
     # uq_encode_decode: the checks of the encoders and of uq_decode
     assert lib.uq_encode_decode(ok, p, p, 127, None, 0, None, 0, 0, 24, B.UQ_FMT_I8, p, p, None, None) == B.UQ_ERR_BAD_ARG   # rng_bits
     assert lib.uq_encode_decode(ok, p, p, 128, None, 0, None, 0, 0, 16, B.UQ_FMT_I8, p, p, None, None) == B.UQ_ERR_BAD_ARG   # s > 127
