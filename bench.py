@@ -42,6 +42,7 @@ FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only
 # bytes per coordinate * d, since every byte of these kernels belongs to a coordinate.
 # Keyed by (workload, kernel); absent = not captured.
 NCU_TRAFFIC_BYTES_PER_COORD = {
+    ("c5", "select_encode_decode"): 27.64,   # profiles/kernel_select_encode_decode_c5_small_ncu.md: 1381.8 MB for d = 50,000,000
     ("c5", "encode_decode"): 27.39,   # profiles/kernel_encode_decode_c5_small_ncu.md: 1369.4 MB for d = 50,000,000
     ("c5", "encode"): 23.39,      # profiles/kernel_encode_c5_small_ncu.md: 1169.7 MB for d = 50,000,000
     ("c2", "encode"): 38.15,      # profiles/kernel_encode_c2_rng32_ncu.md: 975.7 MB at full size (d = 25,557,032)
