@@ -49,6 +49,17 @@ NCU_TRAFFIC_BYTES_PER_COORD = {
 }
 
 
+# ALU-pipe instructions per coordinate and worker of kernels that the ALU pipe, not memory, bounds
+# (ncu's per-opcode counts in the same summaries: LOP3, IADD3, PRMT, SHF, ISETP, VIMNMX3, SEL), and the
+# pipe's peak: 16 lanes per scheduler (measured: such an instruction occupies its scheduler's pipe for
+# 2 cycles), 4 schedulers per SM, 148 SMs, at the SM clock sampled during the run.
+NCU_ALU_OPS_PER_COORD_WORKER = {
+    ("c5", "select_encode_decode"): 9.99,    # profiles/kernel_select_encode_decode_c5_small_ncu.md
+}
+ALU_LANES_PER_SM = 64
+SM_COUNT = 148
+
+
 def hbm_peak():
     p = ROOT / "MEASURED_PEAKS.json"
     if p.exists():
@@ -904,6 +915,7 @@ def gpu_main(args):
     dom_gbs = ab[dom] / res["stages_ms"][dom] / 1e6
     dom_sust = res.get("stages_sustained_ms", {}).get(dom)
     per_coord = NCU_TRAFFIC_BYTES_PER_COORD.get((name, dom))
+    alu_ops = NCU_ALU_OPS_PER_COORD_WORKER.get((name, dom))
     line = {
         "metric": METRIC, "value": round(whole_job_value(world, w.in_bytes, ms), 2), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms, 5),
@@ -939,6 +951,18 @@ def gpu_main(args):
         "kernels": summ["kernels"],
         "sustained": sustained_summary(w, res["sustained"]),
     }
+    if alu_ops is not None:
+        # this kernel is bound by the ALU pipe and instruction issue, not by memory: the same launch
+        # against that pipe, beside the fraction of the HBM peak that the metric asks for
+        mhz = (clocks or {}).get("sm_mhz") or 1965.0
+        alu_peak = SM_COUNT * ALU_LANES_PER_SM * mhz * 1e6
+        alu_rate = alu_ops * w.M * w.d / (res["stages_ms"][dom] * 1e-3)
+        line["roofline"]["limiter"] = ("ALU pipe and instruction issue, not memory (ncu on a smaller case: ALU pipe 70 %, "
+                                       "DRAM 49 % busy); the streaming kernels whose work it does are timed alone under "
+                                       "kernels: select_scale, encode, aggregate_decode")
+        line["roofline"]["alu"] = {"achieved": round(alu_rate / 1e12, 2), "peak": round(alu_peak / 1e12, 2),
+                                   "unit": "T ALU-pipe thread instructions/s", "frac": round(alu_rate / alu_peak, 4),
+                                   "ops_per_coordinate_and_worker": alu_ops}
     if "cold_l2" in summ:
         line["cold_l2"], line["cuda_graph_warm_l2"] = summ["cold_l2"], summ["cuda_graph_warm_l2"]
     if rank == 0 and world == 1:
