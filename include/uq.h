@@ -225,7 +225,10 @@ int uq_encode_multi(const uq_layout *layout, const void *g, const float *W, cons
  * this is one kernel too: the gradients are read once, the indices, the level rows and the
  * average are written, nothing is read back.  Otherwise the calls it stands for run one after
  * the other.  idx, lev and out receive, bit for bit, what the separate calls write; arguments and
- * errors are theirs.  Like uq_select_encode_multi it is bound by instruction issue, not by memory;
+ * errors are theirs.  The first call of this kind on a device (this call, uq_select_encode_multi,
+ * or a uq_step that uses them) raises the kernel's limit of dynamic shared memory with
+ * cudaFuncSetAttribute before it launches; make that first call during set-up, before any stream
+ * capture.  Like uq_select_encode_multi it is bound by instruction issue, not by memory;
  * on a B200 it takes about 19 % less time than uq_select_scale_multi + uq_encode_decode, burst
  * and sustained, which is why uq_step uses it where it is one kernel.
  */
