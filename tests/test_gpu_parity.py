@@ -461,3 +461,37 @@ def test_draws_at_the_edges_of_the_threshold(multi, rng_bits):
     for seed in (0, 1, 0xFFFF_FFFF_FFFF):
         r = check_parity(w, g, seed=seed)
         assert r["W"][0] == np.float32(127.0)
+
+
+@pytest.mark.parametrize("name,kw", [("c5", {}), ("c2", dict(rng_bits=16)), ("c3", {})])
+def test_step_replayed_from_a_cuda_graph(name, kw):
+    """The step a user gets (uq_step without the integer sums; for c5's recipe two kernels, the second
+    one with its shared-memory limit raised on first use) captured once in a CUDA graph, after a call
+    outside the capture, and replayed on new gradients: every replay must match the oracle."""
+    from paper_2109_12497_b200.pipeline import from_workload
+    w = wl.scaled(name, 300_007, M=8, **kw)
+    g_np = wl.generate(w)
+    q = from_workload(w, one_kernel=False)
+    g = to_device(w, g_np)
+    q.step(g, w.seed)                                   # set-up call, outside any capture
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            q.step(g, w.seed)
+    torch.cuda.current_stream().wait_stream(side)
+    for trial in range(2):
+        g_new = np.roll(g_np, 17 * (trial + 1), axis=1).copy()
+        g_new[:, w.d:] = 0
+        g.copy_(to_device(w, g_new))
+        q.out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert q.status_bits() == 0
+        ref = run_oracle(w, g_new, q.W.cpu().numpy())        # downstream of the GPU's scale bits
+        assert np.abs(q.W.cpu().numpy().view(np.int32).astype(np.int64) - ref["W"].view(np.int32)).max() <= 1
+        nb = ref["lev"].shape[1]
+        assert np.array_equal(q.lev.cpu().numpy().view(np.uint8)[:, :nb], ref["lev"])
+        assert np.allclose(q.out.cpu().numpy()[: w.d], ref["out"], rtol=1e-6, atol=0)
